@@ -1,0 +1,211 @@
+"""CPU oracle for the cached causal Conv3D (TEST INFRASTRUCTURE ONLY).
+
+Only the tests, the smoke check and the benchmark's CPU-baseline leg may import
+this package; the product never does.  It wraps ``ccv3d_oracle.c`` (the plain
+fp64 definition, Section 4.1-4.2, Eq. (1)-(2)) through ctypes, and adds two
+structurally different restatements used to pin it:
+
+  * ``brute_force``       - materialises the zero-padded Z volume and loops
+                            output-outermost in pure Python/numpy (tiny shapes);
+  * ``algorithm1_route``  - the paper's Algorithm 1 taken step by step: per
+                            temporal tap the valid output interval of Eq. (3),
+                            one 2-D correlation per tap folded over the
+                            interval, accumulation, bias once.
+
+Host tensors: fp32 arrays, or uint16 arrays of bf16 bit patterns.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "ccv3d_oracle.c")
+_LIB = os.path.join(_HERE, "libccv3d_oracle.so")
+
+F32, BF16 = 0, 1
+
+
+def build(force: bool = False) -> str:
+    """Compile the C oracle with gcc (no fast-math); returns the library path."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        cmd = ["gcc", "-O3", "-march=native", "-fopenmp", "-fPIC", "-shared", "-std=c11",
+               "-o", _LIB + ".tmp", _SRC]
+        subprocess.run(cmd, check=True)
+        os.replace(_LIB + ".tmp", _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        i, p = ctypes.c_int, ctypes.c_void_p
+        lib.ccv3d_oracle_forward.argtypes = [i, p, p, p, p] + [i] * 9 + [p, p]
+        lib.ccv3d_oracle_forward.restype = i
+        lib.ccv3d_oracle_points.argtypes = [i, p, p, p, p] + [i] * 9 + [p, ctypes.c_int64, p]
+        lib.ccv3d_oracle_points.restype = i
+        lib.ccv3d_oracle_num_threads.restype = i
+        _lib = lib
+    return _lib
+
+
+def num_threads() -> int:
+    return int(_load().ccv3d_oracle_num_threads())
+
+
+def _dtype_of(a: np.ndarray) -> int:
+    if a.dtype == np.uint16:
+        return BF16
+    if a.dtype == np.float32:
+        return F32
+    raise TypeError("oracle tensors are float32 arrays or uint16 bf16 bit patterns")
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _prep(x, cache, w, b):
+    dt = _dtype_of(x)
+    x = np.ascontiguousarray(x)
+    w = np.ascontiguousarray(w)
+    assert _dtype_of(w) == dt
+    N, Cin, T, H, W = x.shape
+    Cout, Cin2, kt, kh, kw = w.shape
+    assert Cin2 == Cin
+    if cache is not None:
+        cache = np.ascontiguousarray(cache)
+        assert _dtype_of(cache) == dt and cache.shape == (N, Cin, kt - 1, H, W)
+    if b is not None:
+        b = np.ascontiguousarray(b)
+        assert _dtype_of(b) == dt and b.shape == (Cout,)
+    return dt, x, cache, w, b, (N, Cin, Cout, T, H, W, kt, kh, kw)
+
+
+def forward(x, cache, w, b, want_cache: bool = True):
+    """Returns (out float64 [N,Cout,T,H,W], new_cache in the storage dtype or None)."""
+    dt, x, cache, w, b, dims = _prep(x, cache, w, b)
+    N, Cin, Cout, T, H, W, kt, kh, kw = dims
+    out = np.empty((N, Cout, T, H, W), dtype=np.float64)
+    nc = np.empty((N, Cin, kt - 1, H, W), dtype=x.dtype) if (want_cache and kt > 1) else None
+    rc = _load().ccv3d_oracle_forward(dt, _ptr(x), _ptr(cache), _ptr(w), _ptr(b), *dims, _ptr(out), _ptr(nc))
+    if rc != 0:
+        raise ValueError("ccv3d_oracle_forward rejected its arguments")
+    return out, nc
+
+
+def points(x, cache, w, b, flat_idx):
+    """Oracle value of the sampled output elements flat_idx (into [N,Cout,T,H,W])."""
+    dt, x, cache, w, b, dims = _prep(x, cache, w, b)
+    idx = np.ascontiguousarray(flat_idx, dtype=np.int64)
+    vals = np.empty(idx.shape, dtype=np.float64)
+    rc = _load().ccv3d_oracle_points(dt, _ptr(x), _ptr(cache), _ptr(w), _ptr(b), *dims, _ptr(idx), idx.size,
+                                     _ptr(vals))
+    if rc != 0:
+        raise ValueError("ccv3d_oracle_points rejected its arguments")
+    return vals
+
+
+# --------------------------------------------------------------------------------------
+# Second opinions (pure numpy / Python, float64, tiny shapes only)
+# --------------------------------------------------------------------------------------
+def _widen(a):
+    if a is None:
+        return None
+    if a.dtype == np.uint16:
+        return (a.astype(np.uint32) << np.uint32(16)).view(np.float32).astype(np.float64)
+    return a.astype(np.float64)
+
+
+def brute_force(x, cache, w, b):
+    """Definition evaluated on a materialised zero-padded Z volume, output-outermost."""
+    xd, cd, wd, bd = _widen(x), _widen(cache), _widen(w), _widen(b)
+    N, Cin, T, H, W = xd.shape
+    Cout, _, kt, kh, kw = wd.shape
+    ph, pw = (kh - 1) // 2, (kw - 1) // 2
+    Zp = np.zeros((N, Cin, kt - 1 + T, H + 2 * ph, W + 2 * pw))
+    if cd is not None and kt > 1:
+        Zp[:, :, :kt - 1, ph:ph + H, pw:pw + W] = cd
+    Zp[:, :, kt - 1:, ph:ph + H, pw:pw + W] = xd
+    out = np.zeros((N, Cout, T, H, W))
+    for n in range(N):
+        for co in range(Cout):
+            for t in range(T):
+                for h in range(H):
+                    for ww in range(W):
+                        patch = Zp[n, :, t:t + kt, h:h + kh, ww:ww + kw]
+                        out[n, co, t, h, ww] = (bd[co] if bd is not None else 0.0) + float(np.sum(patch * wd[co]))
+    Zt = Zp[:, :, :, ph:ph + H, pw:pw + W]
+    return out, Zt[:, :, T:T + kt - 1]
+
+
+def tap_intervals(kt: int, cache_frames: int, T: int, dil_t: int = 1):
+    """Eq. (3): per temporal tap k the valid output interval [o_l, o_h) and its
+    source interval [z_l, z_h) in Z = [C ; X], with p_l^base = d_t (kt-1),
+    p_l = p_l^base - |C|, p_r = 0 and unit temporal stride.  Returns (T_o, list)."""
+    p_base = dil_t * (kt - 1)
+    p_l = p_base - cache_frames
+    zlen = cache_frames + T
+    T_o = (zlen + p_l + 0 - dil_t * (kt - 1) - 1) // 1 + 1
+    taps = []
+    for k in range(kt):
+        delta = k * dil_t - p_l
+        o_l = max(0, -delta)
+        o_h = min(T_o, zlen - delta)
+        taps.append((k, o_l, o_h, o_l + delta, o_h + delta))
+    return T_o, taps
+
+
+def _corr2d_same(img, ker):
+    """Zero-padded 'same' 2-D cross-correlation of one plane with one odd-sized kernel."""
+    H, W = img.shape
+    kh, kw = ker.shape
+    ph, pw = (kh - 1) // 2, (kw - 1) // 2
+    pad = np.zeros((H + 2 * ph, W + 2 * pw))
+    pad[ph:ph + H, pw:pw + W] = img
+    res = np.zeros((H, W))
+    for dh in range(kh):
+        for dw in range(kw):
+            res += ker[dh, dw] * pad[dh:dh + H, dw:dw + W]
+    return res
+
+
+def algorithm1_route(x, cache, w, b):
+    """Algorithm 1, literally: Z = [C;X] if cached else X; for each temporal tap the
+    interval of Eq. (3); skip empty taps; fold the source interval into the batch; one
+    2-D correlation with W_k; accumulate into A[:, o_l:o_h]; add the bias once."""
+    xd, cd, wd, bd = _widen(x), _widen(cache), _widen(w), _widen(b)
+    N, Cin, T, H, W = xd.shape
+    Cout, _, kt, kh, kw = wd.shape
+    if cd is not None and kt > 1:
+        Z, nC = np.concatenate([cd, xd], axis=2), kt - 1
+    else:
+        Z, nC = xd, 0
+    T_o, taps = tap_intervals(kt, nC, T)
+    assert T_o == T
+    A = None
+    for (k, o_l, o_h, z_l, z_h) in taps:
+        if o_l >= o_h:
+            continue
+        Wk = wd[:, :, k]                                   # [Cout, Cin, kh, kw]
+        U2 = Z[:, :, z_l:z_h].transpose(0, 2, 1, 3, 4).reshape(N * (z_h - z_l), Cin, H, W)   # fold time into batch
+        R2 = np.zeros((U2.shape[0], Cout, H, W))
+        for bi in range(U2.shape[0]):
+            for co in range(Cout):
+                for ci in range(Cin):
+                    R2[bi, co] += _corr2d_same(U2[bi, ci], Wk[co, ci])
+        R = R2.reshape(N, z_h - z_l, Cout, H, W)           # unfold
+        if A is None:
+            A = np.zeros((N, T_o, Cout, H, W))
+        A[:, o_l:o_h] += R
+    assert A is not None
+    if bd is not None:
+        A = A + bd[None, None, :, None, None]
+    return np.ascontiguousarray(A.transpose(0, 2, 1, 3, 4))  # restore [N,Cout,T,H,W]
