@@ -1,0 +1,164 @@
+/*
+ * ccv3d - cached causal Conv3D forward pass for NVIDIA B200 (sm_100a).
+ *
+ * C ABI.  Plain pointers and sizes only; every tensor pointer says whether it
+ * is a DEVICE or a HOST address.  All tensors are dense and contiguous in the
+ * stated index order (last index fastest).  Functions return a ccv3d_status;
+ * nothing throws, aborts or traps.  A handle is not thread-safe; distinct
+ * handles are independent.
+ *
+ * The operation (paper Section 4.1-4.2, Eq. (1) source time, Eq. (2) conv3d):
+ * with Z = [cache ; x] concatenated along time (cache = the previous chunk's
+ * last kt-1 input frames, oldest first; all zeros on the first chunk),
+ *
+ *   out[n,co,t,h,w] = b[co] + sum_{ci,dt,dh,dw} w[co,ci,dt,dh,dw]
+ *                                * Z[n,ci,t+dt,h+dh-pad_h,w+dw-pad_w]      0 <= t < T
+ *
+ * (cross-correlation, unit stride and dilation, one group, zero spatial
+ * padding pad_h=(kh-1)/2, pad_w=(kw-1)/2 so that H and W are preserved, causal
+ * temporal padding of kt-1 frames supplied by the cache; the bias is added
+ * exactly once), and
+ *
+ *   new_cache[n,ci,j,h,w] = Z[n,ci,T+j,h,w]                               0 <= j < kt-1
+ *
+ * i.e. the last kt-1 frames of the running input stream (for T < kt-1 this
+ * keeps the newest frames of the old cache in front of x).
+ */
+#ifndef CCV3D_H_
+#define CCV3D_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct ccv3d_handle ccv3d_handle; /* opaque; one per convolution layer */
+
+typedef enum { CCV3D_F32 = 0, CCV3D_BF16 = 1 } ccv3d_dtype;
+
+typedef enum {
+    CCV3D_OK = 0,
+    CCV3D_ERR_INVALID_ARG = 1,    /* NULL pointer, non-positive size, bad enum */
+    CCV3D_ERR_UNSUPPORTED = 2,    /* stride/dilation/groups != 1, even kernel, pad != (k-1)/2, ... (Algorithm 1's reject list) */
+    CCV3D_ERR_ALIGNMENT = 3,      /* a tensor pointer is not 16-byte aligned */
+    CCV3D_ERR_ALIAS = 4,          /* out or new_cache overlaps an input (or each other) */
+    CCV3D_ERR_ARCH = 5,           /* current device is not compute capability 10.x */
+    CCV3D_ERR_NOMEM = 6,          /* device or host allocation failed */
+    CCV3D_ERR_CUDA = 7,           /* a CUDA runtime/driver call or a launch failed */
+    CCV3D_ERR_DEVICE_TIMEOUT = 8  /* a bounded wait inside a kernel gave up (see ccv3d_device_status) */
+} ccv3d_status;
+
+/* ccv3d_desc.flags */
+#define CCV3D_FLAG_FORCE_SIMT 0x1u      /* BF16 layers: use the plain FP32-FMA kernel instead of the tensor-core kernel */
+#define CCV3D_FLAG_TC_PER_TAP_A 0x2u    /* tensor-core kernel: fetch the activation tile once per tap (no halo reuse in shared memory) */
+
+/* Layer description, fixed at create time (Algorithm 1's Require line: W, b, p, s, d, g). */
+typedef struct {
+    int32_t cin, cout;            /* channels */
+    int32_t kt, kh, kw;           /* kernel extent; kh and kw must be odd, 1 <= kt <= 8, kh,kw <= 7 */
+    int32_t pad_t, pad_h, pad_w;  /* framework-style padding: must equal (kt-1)/2 if kt is odd else is ignored; (kh-1)/2; (kw-1)/2.
+                                     The causal left pad kt-1 comes from the cache, never from zeros on the right. */
+    int32_t stride[3];            /* must be {1,1,1} */
+    int32_t dilation[3];          /* must be {1,1,1} */
+    int32_t groups;               /* must be 1 */
+    int32_t dtype;                /* ccv3d_dtype of x, cache, w, b and new_cache */
+    int32_t out_dtype;            /* ccv3d_dtype of out: F32 layers -> F32; BF16 layers -> BF16 or F32 */
+    uint32_t flags;               /* CCV3D_FLAG_* */
+} ccv3d_desc;
+
+/* Route counters (the paper's rho: calls, fast-path hits, rejected calls), per handle. */
+typedef struct {
+    uint64_t calls;           /* ccv3d_forward* calls */
+    uint64_t ok;              /* calls that enqueued all their work */
+    uint64_t tcgen05_bf16;    /* calls served by the tensor-core kernel */
+    uint64_t simt;            /* calls served by the FP32-FMA kernel */
+    uint64_t unsupported;     /* rejected: unsupported */
+    uint64_t invalid;         /* rejected: invalid argument / alignment / alias */
+    uint64_t cuda_error;      /* failed in a CUDA call */
+    uint64_t device_timeout;  /* ccv3d_device_status reports that counted a kernel-side timeout */
+    uint64_t kernel_launches; /* kernels launched by this handle since create */
+} ccv3d_counters;
+
+/*
+ * Create a layer (Algorithm 1's derived-weight caching, done once: the
+ * weights are repacked per tap into the tensor-core operand order and the
+ * bias is widened to FP32 here, never per call).
+ *   out_h   HOST   receives the handle.
+ *   d       HOST   layer description; validated (CCV3D_ERR_UNSUPPORTED / INVALID_ARG).
+ *   w_dev   DEVICE [cout,cin,kt,kh,kw] in d->dtype.  Read during the call (stream-ordered);
+ *                  may be released after the stream has passed this point.
+ *   b_dev   DEVICE [cout] in d->dtype, or NULL for a zero bias.
+ *   stream  a cudaStream_t (NULL = default stream).
+ * The handle owns: packed weights, FP32 bias, a status word, an optional
+ * workspace (see ccv3d_forward).  The caller owns everything else.
+ */
+ccv3d_status ccv3d_create(ccv3d_handle** out_h, const ccv3d_desc* d, const void* w_dev, const void* b_dev,
+                          void* stream);
+
+/*
+ * One forward call on DEVICE buffers: Eq. (2) plus the cache update, all
+ * enqueued on `stream` (asynchronous; no host synchronisation).
+ *   x          DEVICE [N,cin,T,H,W]
+ *   cache      DEVICE [N,cin,kt-1,H,W], or NULL = first chunk (all-zero history;
+ *              the taps that would read it are skipped).  Ignored when kt == 1.
+ *   out        DEVICE [N,cout,T,H,W] in out_dtype; fully overwritten.
+ *   new_cache  DEVICE [N,cin,kt-1,H,W], or NULL to skip the update; fully overwritten,
+ *              bit-exact copy of the last kt-1 frames of [cache ; x].  Ignored when kt == 1.
+ * out must not overlap x or cache; new_cache must not overlap x, cache or out
+ * (CCV3D_ERR_ALIAS): ping-pong two cache buffers.  All pointers must be 16-byte aligned.
+ * The tensor-core path keeps a channels-last staging copy of [cache ; x] in a
+ * workspace owned by the handle; it is (re)allocated when a call needs more than
+ * the handle holds (that call synchronises the device), so steady-state calls of
+ * one shape allocate nothing.  ccv3d_workspace_bytes tells the size in advance.
+ */
+ccv3d_status ccv3d_forward(ccv3d_handle* h, const void* x, const void* cache, void* out, void* new_cache,
+                           int32_t N, int32_t T, int32_t H, int32_t W, void* stream);
+
+/*
+ * The same call on HOST buffers (same shapes and meaning as above): copies x
+ * and cache to device staging owned by the handle, runs ccv3d_forward, copies
+ * out and new_cache back, and returns after the stream has completed.  Pinned
+ * host memory makes the copies asynchronous with respect to each other.
+ */
+ccv3d_status ccv3d_forward_host(ccv3d_handle* h, const void* x_host, const void* cache_host, void* out_host,
+                                void* new_cache_host, int32_t N, int32_t T, int32_t H, int32_t W, void* stream);
+
+/* Bytes of handle-owned workspace a forward call of this shape needs (0 for the FP32-FMA path). */
+ccv3d_status ccv3d_workspace_bytes(const ccv3d_handle* h, int32_t N, int32_t T, int32_t H, int32_t W,
+                                   uint64_t* bytes_host);
+
+/* Destroy a handle and free what it owns.  NULL is accepted. */
+ccv3d_status ccv3d_destroy(ccv3d_handle* h);
+
+/* Copy the counters (HOST struct). */
+ccv3d_status ccv3d_get_counters(const ccv3d_handle* h, ccv3d_counters* out_host);
+
+/*
+ * After the caller has synchronised the stream: CCV3D_OK, or
+ * CCV3D_ERR_DEVICE_TIMEOUT if a kernel gave up on a bounded wait since the
+ * last query (the outputs of that call are then undefined).  Reading clears
+ * the word.  detail_host (may be NULL) receives the raw word:
+ * bits 0-7 wait site, bits 8-31 block index.
+ */
+ccv3d_status ccv3d_device_status(ccv3d_handle* h, uint32_t* detail_host);
+
+/* Static, human-readable name of a status code. */
+const char* ccv3d_status_string(ccv3d_status s);
+
+/*
+ * Element-wise glue of a streamed decoder chain (not part of the paper's
+ * operator; provided so that a chain of layers runs entirely in this library).
+ * All tensors DEVICE, BF16, contiguous.
+ *   ccv3d_add_bf16:        y[i] = bf16(float(a[i]) + float(b[i])),  n elements (round to nearest even).
+ *   ccv3d_upsample_bf16:   y[N,C,T*rt,H*2,W*2] = nearest-neighbour repeat of x[N,C,T,H,W]
+ *                          (each pixel 2x2, each frame rt times, rt >= 1).
+ */
+ccv3d_status ccv3d_add_bf16(const void* a, const void* b, void* y, int64_t n, void* stream);
+ccv3d_status ccv3d_upsample_bf16(const void* x, void* y, int32_t N, int32_t C, int32_t T, int32_t H, int32_t W,
+                                 int32_t rt, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CCV3D_H_ */

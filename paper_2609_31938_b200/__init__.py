@@ -1,0 +1,202 @@
+"""Python binding of the ccv3d C-ABI library (cached causal Conv3D for B200).
+
+Argument marshalling only: every step of the operator runs inside
+``libccv3d.so`` (hand-written CUDA for sm_100a).  The functions below carry the
+names of the C entry points declared in ``include/ccv3d.h`` and take raw
+addresses; ``CausalConv3d`` is a thin convenience wrapper that takes torch
+tensors (torch is used for device memory and streams, nothing else).
+
+There is no CPU or library fallback: importing this package without the built
+library raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+from . import _build
+
+F32, BF16 = 0, 1
+FLAG_FORCE_SIMT = 0x1
+FLAG_TC_PER_TAP_A = 0x2
+
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_ALIAS, ERR_ARCH, ERR_NOMEM, ERR_CUDA, \
+    ERR_DEVICE_TIMEOUT = range(9)
+
+
+class Desc(ctypes.Structure):
+    _fields_ = [("cin", ctypes.c_int32), ("cout", ctypes.c_int32),
+                ("kt", ctypes.c_int32), ("kh", ctypes.c_int32), ("kw", ctypes.c_int32),
+                ("pad_t", ctypes.c_int32), ("pad_h", ctypes.c_int32), ("pad_w", ctypes.c_int32),
+                ("stride", ctypes.c_int32 * 3), ("dilation", ctypes.c_int32 * 3), ("groups", ctypes.c_int32),
+                ("dtype", ctypes.c_int32), ("out_dtype", ctypes.c_int32), ("flags", ctypes.c_uint32)]
+
+
+class Counters(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_uint64) for n in ("calls", "ok", "tcgen05_bf16", "simt", "unsupported", "invalid",
+                                               "cuda_error", "device_timeout", "kernel_launches")]
+
+
+EXPORTS = ("ccv3d_create", "ccv3d_forward", "ccv3d_forward_host", "ccv3d_workspace_bytes", "ccv3d_destroy",
+           "ccv3d_get_counters", "ccv3d_device_status", "ccv3d_status_string", "ccv3d_add_bf16",
+           "ccv3d_upsample_bf16")
+
+
+def _load() -> ctypes.CDLL:
+    path = _build.LIB
+    if not os.path.exists(path):
+        raise ImportError(f"{path} is missing: run `python -c 'import __graft_entry__ as g; g.build()'` "
+                          "(nvcc, sm_100a). There is no fallback path.")
+    lib = ctypes.CDLL(path)
+    vp, i32, u64p = ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(ctypes.c_uint64)
+    lib.ccv3d_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(Desc), vp, vp, vp]
+    lib.ccv3d_forward.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, vp]
+    lib.ccv3d_forward_host.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, vp]
+    lib.ccv3d_workspace_bytes.argtypes = [vp, i32, i32, i32, i32, u64p]
+    lib.ccv3d_destroy.argtypes = [vp]
+    lib.ccv3d_get_counters.argtypes = [vp, ctypes.POINTER(Counters)]
+    lib.ccv3d_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
+    lib.ccv3d_status_string.argtypes = [ctypes.c_int]
+    lib.ccv3d_status_string.restype = ctypes.c_char_p
+    lib.ccv3d_add_bf16.argtypes = [vp, vp, vp, ctypes.c_int64, vp]
+    lib.ccv3d_upsample_bf16.argtypes = [vp, vp, i32, i32, i32, i32, i32, i32, vp]
+    for name in EXPORTS:
+        if name != "ccv3d_status_string":
+            getattr(lib, name).restype = ctypes.c_int
+    return lib
+
+
+lib = _load()
+
+
+class Ccv3dError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {status_string(status)}")
+
+
+def status_string(s: int) -> str:
+    return lib.ccv3d_status_string(int(s)).decode()
+
+
+def make_desc(cin, cout, k=(3, 3, 3), dtype=BF16, out_dtype=None, flags=0, stride=(1, 1, 1), dilation=(1, 1, 1),
+              groups=1, pad=None) -> Desc:
+    kt, kh, kw = k
+    pad = pad if pad is not None else ((kt - 1) // 2, (kh - 1) // 2, (kw - 1) // 2)
+    d = Desc()
+    d.cin, d.cout, d.kt, d.kh, d.kw = cin, cout, kt, kh, kw
+    d.pad_t, d.pad_h, d.pad_w = pad
+    d.stride[:] = stride
+    d.dilation[:] = dilation
+    d.groups = groups
+    d.dtype = dtype
+    d.out_dtype = dtype if out_dtype is None else out_dtype
+    d.flags = flags
+    return d
+
+
+# ---- the C entry points, same names, raw addresses (ints) ----
+def ccv3d_create(desc: Desc, w_dev: int, b_dev: int | None, stream: int = 0):
+    h = ctypes.c_void_p()
+    s = lib.ccv3d_create(ctypes.byref(h), ctypes.byref(desc), w_dev, b_dev, stream)
+    return s, (h.value if s == OK else None)
+
+
+def ccv3d_forward(h, x, cache, out, new_cache, N, T, H, W, stream=0) -> int:
+    return lib.ccv3d_forward(h, x, cache, out, new_cache, N, T, H, W, stream)
+
+
+def ccv3d_forward_host(h, x, cache, out, new_cache, N, T, H, W, stream=0) -> int:
+    return lib.ccv3d_forward_host(h, x, cache, out, new_cache, N, T, H, W, stream)
+
+
+def ccv3d_workspace_bytes(h, N, T, H, W):
+    b = ctypes.c_uint64()
+    s = lib.ccv3d_workspace_bytes(h, N, T, H, W, ctypes.byref(b))
+    return s, b.value
+
+
+def ccv3d_destroy(h) -> int:
+    return lib.ccv3d_destroy(h)
+
+
+def ccv3d_get_counters(h) -> dict:
+    c = Counters()
+    s = lib.ccv3d_get_counters(h, ctypes.byref(c))
+    if s != OK:
+        raise Ccv3dError(s, "ccv3d_get_counters")
+    return {n: int(getattr(c, n)) for n, _ in Counters._fields_}
+
+
+def ccv3d_device_status(h):
+    d = ctypes.c_uint32()
+    s = lib.ccv3d_device_status(h, ctypes.byref(d))
+    return s, d.value
+
+
+def ccv3d_add_bf16(a, b, y, n, stream=0) -> int:
+    return lib.ccv3d_add_bf16(a, b, y, n, stream)
+
+
+def ccv3d_upsample_bf16(x, y, N, C, T, H, W, rt, stream=0) -> int:
+    return lib.ccv3d_upsample_bf16(x, y, N, C, T, H, W, rt, stream)
+
+
+class CausalConv3d:
+    """One cached causal Conv3D layer on the current CUDA device (torch tensors in, torch tensors out)."""
+
+    def __init__(self, w, b=None, out_dtype=None, flags=0):
+        import torch
+        assert w.is_cuda and w.is_contiguous() and w.dim() == 5
+        self.torch = torch
+        self.dtype = BF16 if w.dtype == torch.bfloat16 else F32
+        assert w.dtype in (torch.bfloat16, torch.float32)
+        cout, cin, kt, kh, kw = w.shape
+        self.k, self.cin, self.cout = (kt, kh, kw), cin, cout
+        self.out_dtype = self.dtype if out_dtype is None else out_dtype
+        self.desc = make_desc(cin, cout, self.k, self.dtype, self.out_dtype, flags)
+        if b is not None:
+            assert b.is_cuda and b.is_contiguous() and b.dtype == w.dtype and b.shape == (cout,)
+        s, h = ccv3d_create(self.desc, w.data_ptr(), None if b is None else b.data_ptr(),
+                            torch.cuda.current_stream().cuda_stream)
+        if s != OK:
+            raise Ccv3dError(s, "ccv3d_create")
+        self.h = h
+
+    def forward(self, x, cache=None, out=None, new_cache=None, want_cache=True):
+        torch = self.torch
+        N, C, T, H, W = x.shape
+        assert C == self.cin and x.is_contiguous() and x.is_cuda
+        tc = self.k[0] - 1
+        odt = torch.bfloat16 if self.out_dtype == BF16 else torch.float32
+        if out is None:
+            out = torch.empty((N, self.cout, T, H, W), dtype=odt, device=x.device)
+        if new_cache is None and want_cache and tc:
+            new_cache = torch.empty((N, C, tc, H, W), dtype=x.dtype, device=x.device)
+        if cache is not None:
+            assert cache.is_contiguous() and cache.shape == (N, C, tc, H, W) and cache.dtype == x.dtype
+        s = ccv3d_forward(self.h, x.data_ptr(), None if cache is None else cache.data_ptr(), out.data_ptr(),
+                          None if new_cache is None else new_cache.data_ptr(), N, T, H, W,
+                          torch.cuda.current_stream().cuda_stream)
+        if s != OK:
+            raise Ccv3dError(s, "ccv3d_forward")
+        return out, new_cache
+
+    __call__ = forward
+
+    def counters(self):
+        return ccv3d_get_counters(self.h)
+
+    def device_status(self):
+        return ccv3d_device_status(self.h)
+
+    def close(self):
+        if getattr(self, "h", None):
+            ccv3d_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,523 @@
+// C-ABI of the cached causal Conv3D library: validation (Algorithm 1's
+// "validate and prepare" step turned into error codes - there is no fallback
+// route), handle life cycle, route selection, launches, counters.
+#include "../../include/ccv3d.h"
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "ccv3d_simt.cuh"
+#include "ccv3d_tc.cuh"
+
+using namespace ccv3d;
+
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+constexpr size_t SMEM_LIMIT = 232448;  // 227 KB of dynamic shared memory per CTA on sm_100
+
+struct TcPlan {      // per-layer choices of the tensor-core route
+    int KB, CB, cin_pad;
+    int NT, NPAD, cout_pad;
+    int NB, ACC;
+};
+
+struct ShapeKey {
+    const void* zs;
+    int N, T, H, W;
+    bool operator==(const ShapeKey& o) const { return zs == o.zs && N == o.N && T == o.T && H == o.H && W == o.W; }
+};
+
+}  // namespace
+
+struct ccv3d_handle {
+    ccv3d_desc d;
+    int device;
+    int sm_count;
+    bool use_tc;
+    TcPlan plan;
+    void* w_copy;        // SIMT route: weights in their original order (device)
+    void* wp;            // TC route: packed weights (device)
+    float* bias32;       // FP32 bias, padded (device)
+    unsigned int* status;  // device status word
+    void* workspace;
+    uint64_t workspace_bytes;
+    // host-entry staging (device buffers)
+    void* hx; void* hc; void* ho; void* hn;
+    uint64_t hx_b, hc_b, ho_b, hn_b;
+    EncodeTiledFn encode;
+    CUtensorMap tm_w;
+    CUtensorMap tm_a;
+    ShapeKey tm_a_key;
+    uint64_t wait_limit_ns;
+    ccv3d_counters ctr;
+};
+
+namespace {
+
+inline size_t esize(int dt) { return dt == CCV3D_BF16 ? 2 : 4; }
+inline uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
+
+bool overlap(const void* a, uint64_t an, const void* b, uint64_t bn) {
+    if (!a || !b || an == 0 || bn == 0) return false;
+    const uintptr_t a0 = (uintptr_t)a, b0 = (uintptr_t)b;
+    return a0 < b0 + bn && b0 < a0 + an;
+}
+
+ccv3d_status validate_desc(const ccv3d_desc* d) {
+    if (!d) return CCV3D_ERR_INVALID_ARG;
+    if (d->cin < 1 || d->cout < 1 || d->kt < 1 || d->kh < 1 || d->kw < 1) return CCV3D_ERR_INVALID_ARG;
+    if (d->dtype != CCV3D_F32 && d->dtype != CCV3D_BF16) return CCV3D_ERR_INVALID_ARG;
+    if (d->out_dtype != CCV3D_F32 && d->out_dtype != CCV3D_BF16) return CCV3D_ERR_INVALID_ARG;
+    // Algorithm 1 rejects temporal stride != 1 and groups != 1; this build fixes all strides and dilations at 1.
+    for (int i = 0; i < 3; ++i)
+        if (d->stride[i] != 1 || d->dilation[i] != 1) return CCV3D_ERR_UNSUPPORTED;
+    if (d->groups != 1) return CCV3D_ERR_UNSUPPORTED;
+    if (!(d->kh & 1) || !(d->kw & 1) || d->kh > 7 || d->kw > 7 || d->kt > 8) return CCV3D_ERR_UNSUPPORTED;
+    if (d->pad_h != (d->kh - 1) / 2 || d->pad_w != (d->kw - 1) / 2) return CCV3D_ERR_UNSUPPORTED;
+    if ((d->kt & 1) && d->pad_t != (d->kt - 1) / 2) return CCV3D_ERR_UNSUPPORTED;
+    if (d->dtype == CCV3D_F32 && d->out_dtype != CCV3D_F32) return CCV3D_ERR_UNSUPPORTED;
+    if (d->cin > 65536 || d->cout > 65536) return CCV3D_ERR_UNSUPPORTED;
+    return CCV3D_OK;
+}
+
+void make_plan(const ccv3d_desc& d, TcPlan* pl) {
+    pl->KB = (d.cin % 64 == 0) ? 64 : 32;
+    pl->CB = (d.cin + pl->KB - 1) / pl->KB;
+    pl->cin_pad = pl->CB * pl->KB;
+    pl->NT = (d.cout + 255) / 256;
+    const int per = (d.cout + pl->NT - 1) / pl->NT;
+    pl->NPAD = (per + 15) / 16 * 16;
+    pl->cout_pad = pl->NT * pl->NPAD;
+    pl->NB = 2;
+    pl->ACC = (2 * pl->NB * pl->NPAD <= 512) ? 2 : 1;
+}
+
+uint32_t pow2_cols(uint32_t c) {
+    uint32_t v = 32;
+    while (v < c) v <<= 1;
+    return v;
+}
+
+ccv3d_status count(ccv3d_handle* h, ccv3d_status s) {
+    switch (s) {
+        case CCV3D_OK: h->ctr.ok++; break;
+        case CCV3D_ERR_UNSUPPORTED: h->ctr.unsupported++; break;
+        case CCV3D_ERR_INVALID_ARG:
+        case CCV3D_ERR_ALIGNMENT:
+        case CCV3D_ERR_ALIAS: h->ctr.invalid++; break;
+        default: h->ctr.cuda_error++; break;
+    }
+    return s;
+}
+
+ccv3d_status cuda_fail() {
+    cudaGetLastError();  // clear the sticky-less error so that later calls start clean
+    return CCV3D_ERR_CUDA;
+}
+
+ccv3d_status grow(void** buf, uint64_t* have, uint64_t need) {
+    if (need <= *have) return CCV3D_OK;
+    if (*buf) {
+        if (cudaDeviceSynchronize() != cudaSuccess) return cuda_fail();
+        cudaFree(*buf);
+        *buf = nullptr;
+        *have = 0;
+    }
+    if (cudaMalloc(buf, need) != cudaSuccess) {
+        cudaGetLastError();
+        *buf = nullptr;
+        return CCV3D_ERR_NOMEM;
+    }
+    *have = need;
+    return CCV3D_OK;
+}
+
+ccv3d_status encode_weight_map(ccv3d_handle* h) {
+    const TcPlan& pl = h->plan;
+    const int taps = h->d.kt * h->d.kh * h->d.kw;
+    cuuint64_t dims[3] = {(cuuint64_t)pl.cin_pad, (cuuint64_t)pl.cout_pad, (cuuint64_t)taps};
+    cuuint64_t strides[2] = {(cuuint64_t)pl.cin_pad * 2, (cuuint64_t)pl.cin_pad * pl.cout_pad * 2};
+    cuuint32_t box[3] = {(cuuint32_t)pl.KB, (cuuint32_t)pl.NPAD, 1};
+    cuuint32_t es[3] = {1, 1, 1};
+    CUresult r = h->encode(&h->tm_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, h->wp, dims, strides, box, es,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           pl.KB == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? CCV3D_OK : CCV3D_ERR_CUDA;
+}
+
+ccv3d_status encode_act_map(ccv3d_handle* h, int N, int T, int H, int W, int BW, int BH) {
+    const TcPlan& pl = h->plan;
+    const int F = h->d.kt - 1 + T;
+    const uint64_t rowb = (uint64_t)pl.KB * 2;
+    cuuint64_t dims[5] = {(cuuint64_t)pl.KB, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)pl.CB, (cuuint64_t)N * F};
+    cuuint64_t strides[4] = {rowb, rowb * W, rowb * W * H, rowb * W * H * pl.CB};
+    cuuint32_t box[5] = {(cuuint32_t)pl.KB, (cuuint32_t)BW, (cuuint32_t)BH, 1, 1};
+    cuuint32_t es[5] = {1, 1, 1, 1, 1};
+    CUresult r = h->encode(&h->tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, h->workspace, dims, strides, box, es,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE,
+                           pl.KB == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? CCV3D_OK : CCV3D_ERR_CUDA;
+}
+
+uint64_t tc_workspace_bytes(const ccv3d_handle* h, int N, int T, int H, int W) {
+    const int F = h->d.kt - 1 + T;
+    return (uint64_t)N * F * h->plan.cin_pad * H * W * 2;
+}
+
+template <int KB, int NB>
+ccv3d_status launch_tc(ccv3d_handle* h, const TcParams& p, size_t smem, int grid, cudaStream_t st) {
+    auto kern = conv3d_tcgen05_kernel<KB, NB>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return cuda_fail();
+    kern<<<grid, TC_THREADS, smem, st>>>(h->tm_a, h->tm_w, p);
+    if (cudaGetLastError() != cudaSuccess) return cuda_fail();
+    h->ctr.kernel_launches++;
+    return CCV3D_OK;
+}
+
+ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void* out, void* new_cache, int N, int T,
+                        int H, int W, cudaStream_t st) {
+    const ccv3d_desc& d = h->d;
+    const TcPlan& pl = h->plan;
+    const int tc = d.kt - 1;
+    const int F = tc + T;
+
+    ccv3d_status s = grow(&h->workspace, &h->workspace_bytes, tc_workspace_bytes(h, N, T, H, W));
+    if (s != CCV3D_OK) return s;
+
+    // ---- stage [cache ; x] channels-last, cache update in the same pass ----
+    StageParams sp;
+    sp.x = (const __nv_bfloat16*)x;
+    sp.cache = tc ? (const __nv_bfloat16*)cache : nullptr;
+    sp.zs = (__nv_bfloat16*)h->workspace;
+    sp.new_cache = tc ? (__nv_bfloat16*)new_cache : nullptr;
+    sp.N = N; sp.Cin = d.cin; sp.T = T; sp.H = H; sp.W = W; sp.tc = tc; sp.CB = pl.CB;
+    sp.f_begin = sp.cache ? 0 : (tc < T ? tc : T);
+    const bool vec = (W % 8 == 0);
+    dim3 sgrid((W + STG_PX - 1) / STG_PX, H, (unsigned)(N * (F - sp.f_begin) * pl.CB));
+    if (sgrid.y > 65535 || sgrid.z > 65535) return CCV3D_ERR_UNSUPPORTED;
+    if (pl.KB == 64) {
+        if (vec) stage_frames_kernel<64, true><<<sgrid, 256, 0, st>>>(sp);
+        else stage_frames_kernel<64, false><<<sgrid, 256, 0, st>>>(sp);
+    } else {
+        if (vec) stage_frames_kernel<32, true><<<sgrid, 128, 0, st>>>(sp);
+        else stage_frames_kernel<32, false><<<sgrid, 128, 0, st>>>(sp);
+    }
+    if (cudaGetLastError() != cudaSuccess) return cuda_fail();
+    h->ctr.kernel_launches++;
+
+    // ---- implicit GEMM ----
+    const int per_tap = (d.flags & CCV3D_FLAG_TC_PER_TAP_A) ? 1 : 0;
+    const int NB = pl.NB;
+    const int TW = 8 * NB;
+    const int BW = per_tap ? TW : TW + d.kw - 1;
+    const int BH = per_tap ? 16 : 16 + d.kh - 1;
+    ShapeKey key{h->workspace, N, T, H, W};
+    if (!(key == h->tm_a_key)) {
+        s = encode_act_map(h, N, T, H, W, BW, BH);
+        if (s != CCV3D_OK) return s;
+        h->tm_a_key = key;
+    }
+    TcParams p;
+    memset(&p, 0, sizeof(p));
+    p.N = N; p.T = T; p.H = H; p.W = W; p.Cout = d.cout; p.F = F;
+    p.kt = d.kt; p.kh = d.kh; p.kw = d.kw;
+    p.CB = pl.CB; p.NT = pl.NT; p.NPAD = pl.NPAD;
+    p.tiles_h = (H + 15) / 16;
+    p.tiles_w = (W + TW - 1) / TW;
+    const int64_t total = (int64_t)N * p.tiles_h * p.tiles_w * T * pl.NT;
+    if (total > 0x7FFFFFFF) return CCV3D_ERR_UNSUPPORTED;
+    p.total_tiles = (int)total;
+    p.first_frame = (tc && !cache) ? tc : 0;
+    p.out_f32 = d.out_dtype == CCV3D_F32;
+    p.per_tap_a = per_tap;
+    p.ACC = pl.ACC;
+    p.a_slot = (uint32_t)align_up((uint64_t)BW * BH * pl.KB * 2, 1024);
+    p.b_slot = (uint32_t)align_up((uint64_t)pl.NPAD * pl.KB * 2, 1024);
+    const size_t fixed = 1024 /*alignment slack*/ + align_up(sizeof(TcShared), 128);
+    const size_t budget = SMEM_LIMIT - fixed;
+    int SA = per_tap ? 3 : 2;
+    if ((size_t)SA * p.a_slot + 2 * (size_t)p.b_slot > budget) return CCV3D_ERR_UNSUPPORTED;
+    int SB = (int)((budget - (size_t)SA * p.a_slot) / p.b_slot);
+    if (SB > 8) SB = 8;
+    while (SA < 4 && (size_t)(SA + 1) * p.a_slot + (size_t)SB * p.b_slot <= budget) ++SA;
+    p.SA = SA; p.SB = SB;
+    p.tmem_cols = pow2_cols((uint32_t)(NB * pl.NPAD * pl.ACC));
+    if (p.tmem_cols > 512) return CCV3D_ERR_UNSUPPORTED;
+    p.wait_limit_ns = h->wait_limit_ns;
+    p.bias = h->bias32;
+    p.out = out;
+    p.status = h->status;
+    const size_t smem = fixed + (size_t)SA * p.a_slot + (size_t)SB * p.b_slot;
+    const int grid = p.total_tiles < h->sm_count ? p.total_tiles : h->sm_count;
+    if (pl.KB == 64) s = launch_tc<64, 2>(h, p, smem, grid, st);
+    else s = launch_tc<32, 2>(h, p, smem, grid, st);
+    if (s == CCV3D_OK) h->ctr.tcgen05_bf16++;
+    return s;
+}
+
+ccv3d_status forward_simt(ccv3d_handle* h, const void* x, const void* cache, void* out, void* new_cache, int N, int T,
+                          int H, int W, cudaStream_t st) {
+    const ccv3d_desc& d = h->d;
+    const int tc = d.kt - 1;
+    SimtParams p;
+    p.x = x; p.cache = tc ? cache : nullptr; p.w = h->w_copy; p.bias = h->bias32; p.out = out;
+    p.N = N; p.Cin = d.cin; p.Cout = d.cout; p.T = T; p.H = H; p.W = W; p.kt = d.kt; p.kh = d.kh; p.kw = d.kw;
+    const int64_t npix = (int64_t)N * T * H * W;
+    const int64_t gx = (npix + SIMT_THREADS - 1) / SIMT_THREADS;
+    if (gx > 0x7FFFFFFF) return CCV3D_ERR_UNSUPPORTED;
+    dim3 grid((unsigned)gx, (d.cout + SIMT_CO - 1) / SIMT_CO);
+    if (d.dtype == CCV3D_F32) conv3d_direct_kernel<float, float><<<grid, SIMT_THREADS, 0, st>>>(p);
+    else if (d.out_dtype == CCV3D_BF16) conv3d_direct_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, SIMT_THREADS, 0, st>>>(p);
+    else conv3d_direct_kernel<__nv_bfloat16, float><<<grid, SIMT_THREADS, 0, st>>>(p);
+    if (cudaGetLastError() != cudaSuccess) return cuda_fail();
+    h->ctr.kernel_launches++;
+    h->ctr.simt++;
+
+    if (tc && new_cache) {
+        const uint64_t fbytes = (uint64_t)H * W * esize(d.dtype);
+        const int64_t planes = (int64_t)N * d.cin * tc;
+        const unsigned gy = (unsigned)(planes < 65535 ? planes : 65535);  // the kernel strides over the rest
+        if (fbytes % 16 == 0) {
+            const int64_t units = fbytes / 16;
+            dim3 g((unsigned)((units + 255) / 256 > 1024 ? 1024 : (units + 255) / 256), gy);
+            cache_update_kernel<uint4><<<g, 256, 0, st>>>((const uint4*)x, (const uint4*)cache, (uint4*)new_cache, d.cin, T,
+                                                          tc, units, planes);
+        } else if (d.dtype == CCV3D_F32) {
+            const int64_t units = (int64_t)H * W;
+            dim3 g((unsigned)((units + 255) / 256 > 1024 ? 1024 : (units + 255) / 256), gy);
+            cache_update_kernel<uint32_t><<<g, 256, 0, st>>>((const uint32_t*)x, (const uint32_t*)cache,
+                                                             (uint32_t*)new_cache, d.cin, T, tc, units, planes);
+        } else {
+            const int64_t units = (int64_t)H * W;
+            dim3 g((unsigned)((units + 255) / 256 > 1024 ? 1024 : (units + 255) / 256), gy);
+            cache_update_kernel<uint16_t><<<g, 256, 0, st>>>((const uint16_t*)x, (const uint16_t*)cache,
+                                                             (uint16_t*)new_cache, d.cin, T, tc, units, planes);
+        }
+        if (cudaGetLastError() != cudaSuccess) return cuda_fail();
+        h->ctr.kernel_launches++;
+    }
+    return CCV3D_OK;
+}
+
+ccv3d_status check_forward_args(const ccv3d_handle* h, const void* x, const void* cache, void* out, void* new_cache,
+                                int N, int T, int H, int W, bool device_ptrs) {
+    if (!h || !x || !out) return CCV3D_ERR_INVALID_ARG;
+    if (N < 1 || T < 1 || H < 1 || W < 1) return CCV3D_ERR_INVALID_ARG;
+    const ccv3d_desc& d = h->d;
+    const uint64_t px = (uint64_t)N * H * W;
+    if ((double)px * T * (d.cin > d.cout ? d.cin : d.cout) > 9.0e15) return CCV3D_ERR_UNSUPPORTED;
+    if ((uint64_t)H * W > 0x7FFFFFFFull) return CCV3D_ERR_UNSUPPORTED;
+    const int tc = d.kt - 1;
+    const uint64_t xb = px * d.cin * T * esize(d.dtype), cb = px * d.cin * tc * esize(d.dtype);
+    const uint64_t ob = px * d.cout * T * esize(d.out_dtype);
+    if (!tc) { cache = nullptr; new_cache = nullptr; }
+    if (device_ptrs) {
+        const uintptr_t m = (uintptr_t)x | (uintptr_t)cache | (uintptr_t)out | (uintptr_t)new_cache;
+        if (m & 15u) return CCV3D_ERR_ALIGNMENT;
+    }
+    if (overlap(out, ob, x, xb) || overlap(out, ob, cache, cb)) return CCV3D_ERR_ALIAS;
+    if (overlap(new_cache, cb, x, xb) || overlap(new_cache, cb, cache, cb) || overlap(new_cache, cb, out, ob))
+        return CCV3D_ERR_ALIAS;
+    return CCV3D_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* ccv3d_status_string(ccv3d_status s) {
+    switch (s) {
+        case CCV3D_OK: return "CCV3D_OK";
+        case CCV3D_ERR_INVALID_ARG: return "CCV3D_ERR_INVALID_ARG";
+        case CCV3D_ERR_UNSUPPORTED: return "CCV3D_ERR_UNSUPPORTED";
+        case CCV3D_ERR_ALIGNMENT: return "CCV3D_ERR_ALIGNMENT";
+        case CCV3D_ERR_ALIAS: return "CCV3D_ERR_ALIAS";
+        case CCV3D_ERR_ARCH: return "CCV3D_ERR_ARCH";
+        case CCV3D_ERR_NOMEM: return "CCV3D_ERR_NOMEM";
+        case CCV3D_ERR_CUDA: return "CCV3D_ERR_CUDA";
+        case CCV3D_ERR_DEVICE_TIMEOUT: return "CCV3D_ERR_DEVICE_TIMEOUT";
+    }
+    return "CCV3D_ERR_UNKNOWN";
+}
+
+ccv3d_status ccv3d_create(ccv3d_handle** out_h, const ccv3d_desc* d, const void* w_dev, const void* b_dev,
+                          void* stream) {
+    if (!out_h) return CCV3D_ERR_INVALID_ARG;
+    *out_h = nullptr;
+    ccv3d_status s = validate_desc(d);   // host-only checks come first: they need no device
+    if (s != CCV3D_OK) return s;
+    if (!w_dev) return CCV3D_ERR_INVALID_ARG;
+    if (((uintptr_t)w_dev | (uintptr_t)b_dev) & 15u) return CCV3D_ERR_ALIGNMENT;
+
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return cuda_fail();
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return cuda_fail();
+    if (prop.major != 10) return CCV3D_ERR_ARCH;
+
+    ccv3d_handle* h = new (std::nothrow) ccv3d_handle();
+    if (!h) return CCV3D_ERR_NOMEM;
+    memset(h, 0, sizeof(*h));
+    h->d = *d;
+    h->device = dev;
+    h->sm_count = prop.multiProcessorCount;
+    h->use_tc = (d->dtype == CCV3D_BF16) && !(d->flags & CCV3D_FLAG_FORCE_SIMT);
+    h->wait_limit_ns = 1000000000ull;
+    if (const char* e = getenv("CCV3D_WAIT_LIMIT_MS")) {
+        const long v = atol(e);
+        if (v > 0 && v <= 10000) h->wait_limit_ns = (uint64_t)v * 1000000ull;
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    const int taps = d->kt * d->kh * d->kw;
+
+    auto fail = [&](ccv3d_status e) {
+        ccv3d_destroy(h);
+        return e;
+    };
+
+    if (cudaMalloc((void**)&h->status, sizeof(unsigned int)) != cudaSuccess) return fail(CCV3D_ERR_NOMEM);
+    if (cudaMemsetAsync(h->status, 0, sizeof(unsigned int), st) != cudaSuccess) return fail(cuda_fail());
+
+    int bias_n = d->cout;
+    if (h->use_tc) {
+        make_plan(*d, &h->plan);
+        bias_n = h->plan.cout_pad;
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+            qres != cudaDriverEntryPointSuccess)
+            return fail(cuda_fail());
+        h->encode = (EncodeTiledFn)fn;
+        const uint64_t wpb = (uint64_t)taps * h->plan.cout_pad * h->plan.cin_pad * 2;
+        if (cudaMalloc(&h->wp, wpb) != cudaSuccess) return fail(CCV3D_ERR_NOMEM);
+        pack_weights_kernel<<<1024, 256, 0, st>>>((const __nv_bfloat16*)w_dev, (__nv_bfloat16*)h->wp, d->cout, d->cin,
+                                                  taps, h->plan.cout_pad, h->plan.cin_pad);
+        if (cudaGetLastError() != cudaSuccess) return fail(cuda_fail());
+        h->ctr.kernel_launches++;
+        if (encode_weight_map(h) != CCV3D_OK) return fail(CCV3D_ERR_CUDA);
+    } else {
+        const uint64_t wb = (uint64_t)d->cout * d->cin * taps * esize(d->dtype);
+        if (cudaMalloc(&h->w_copy, wb) != cudaSuccess) return fail(CCV3D_ERR_NOMEM);
+        if (cudaMemcpyAsync(h->w_copy, w_dev, wb, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return fail(cuda_fail());
+    }
+    if (cudaMalloc((void**)&h->bias32, (size_t)bias_n * sizeof(float)) != cudaSuccess) return fail(CCV3D_ERR_NOMEM);
+    if (d->dtype == CCV3D_BF16)
+        bias_to_f32_kernel<__nv_bfloat16><<<(bias_n + 255) / 256, 256, 0, st>>>((const __nv_bfloat16*)b_dev, h->bias32,
+                                                                                d->cout, bias_n);
+    else
+        bias_to_f32_kernel<float><<<(bias_n + 255) / 256, 256, 0, st>>>((const float*)b_dev, h->bias32, d->cout, bias_n);
+    if (cudaGetLastError() != cudaSuccess) return fail(cuda_fail());
+    h->ctr.kernel_launches++;
+    *out_h = h;
+    return CCV3D_OK;
+}
+
+ccv3d_status ccv3d_destroy(ccv3d_handle* h) {
+    if (!h) return CCV3D_OK;
+    cudaDeviceSynchronize();
+    void* bufs[] = {h->w_copy, h->wp, h->bias32, h->status, h->workspace, h->hx, h->hc, h->ho, h->hn};
+    for (void* b : bufs)
+        if (b) cudaFree(b);
+    cudaGetLastError();
+    delete h;
+    return CCV3D_OK;
+}
+
+ccv3d_status ccv3d_workspace_bytes(const ccv3d_handle* h, int32_t N, int32_t T, int32_t H, int32_t W,
+                                   uint64_t* bytes_host) {
+    if (!h || !bytes_host || N < 1 || T < 1 || H < 1 || W < 1) return CCV3D_ERR_INVALID_ARG;
+    *bytes_host = h->use_tc ? tc_workspace_bytes(h, N, T, H, W) : 0;
+    return CCV3D_OK;
+}
+
+ccv3d_status ccv3d_forward(ccv3d_handle* h, const void* x, const void* cache, void* out, void* new_cache, int32_t N,
+                           int32_t T, int32_t H, int32_t W, void* stream) {
+    if (!h) return CCV3D_ERR_INVALID_ARG;
+    h->ctr.calls++;
+    ccv3d_status s = check_forward_args(h, x, cache, out, new_cache, N, T, H, W, true);
+    if (s != CCV3D_OK) return count(h, s);
+    cudaStream_t st = (cudaStream_t)stream;
+    if (h->use_tc) s = forward_tc(h, x, cache, out, new_cache, N, T, H, W, st);
+    else s = forward_simt(h, x, cache, out, new_cache, N, T, H, W, st);
+    return count(h, s);
+}
+
+ccv3d_status ccv3d_forward_host(ccv3d_handle* h, const void* x_host, const void* cache_host, void* out_host,
+                                void* new_cache_host, int32_t N, int32_t T, int32_t H, int32_t W, void* stream) {
+    if (!h) return CCV3D_ERR_INVALID_ARG;
+    ccv3d_status s = check_forward_args(h, x_host, cache_host, out_host, new_cache_host, N, T, H, W, false);
+    if (s != CCV3D_OK) {
+        h->ctr.calls++;
+        return count(h, s);
+    }
+    const ccv3d_desc& d = h->d;
+    const int tc = d.kt - 1;
+    const uint64_t px = (uint64_t)N * H * W;
+    const uint64_t xb = px * d.cin * T * esize(d.dtype), cb = px * d.cin * tc * esize(d.dtype);
+    const uint64_t ob = px * d.cout * T * esize(d.out_dtype);
+    cudaStream_t st = (cudaStream_t)stream;
+    const bool has_c = tc && cache_host, has_n = tc && new_cache_host;
+    if ((s = grow(&h->hx, &h->hx_b, xb)) != CCV3D_OK) return s;
+    if ((s = grow(&h->ho, &h->ho_b, ob)) != CCV3D_OK) return s;
+    if (has_c && (s = grow(&h->hc, &h->hc_b, cb)) != CCV3D_OK) return s;
+    if (has_n && (s = grow(&h->hn, &h->hn_b, cb)) != CCV3D_OK) return s;
+    if (cudaMemcpyAsync(h->hx, x_host, xb, cudaMemcpyHostToDevice, st) != cudaSuccess) return cuda_fail();
+    if (has_c && cudaMemcpyAsync(h->hc, cache_host, cb, cudaMemcpyHostToDevice, st) != cudaSuccess) return cuda_fail();
+    s = ccv3d_forward(h, h->hx, has_c ? h->hc : nullptr, h->ho, has_n ? h->hn : nullptr, N, T, H, W, stream);
+    if (s != CCV3D_OK) return s;
+    if (cudaMemcpyAsync(out_host, h->ho, ob, cudaMemcpyDeviceToHost, st) != cudaSuccess) return cuda_fail();
+    if (has_n && cudaMemcpyAsync(new_cache_host, h->hn, cb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return cuda_fail();
+    if (cudaStreamSynchronize(st) != cudaSuccess) return cuda_fail();
+    return ccv3d_device_status(h, nullptr);
+}
+
+ccv3d_status ccv3d_get_counters(const ccv3d_handle* h, ccv3d_counters* out_host) {
+    if (!h || !out_host) return CCV3D_ERR_INVALID_ARG;
+    *out_host = h->ctr;
+    return CCV3D_OK;
+}
+
+ccv3d_status ccv3d_device_status(ccv3d_handle* h, uint32_t* detail_host) {
+    if (!h) return CCV3D_ERR_INVALID_ARG;
+    unsigned int word = 0;
+    if (cudaMemcpy(&word, h->status, sizeof(word), cudaMemcpyDeviceToHost) != cudaSuccess) return cuda_fail();
+    if (detail_host) *detail_host = word;
+    if (word == 0) return CCV3D_OK;
+    cudaMemset(h->status, 0, sizeof(word));
+    h->ctr.device_timeout++;
+    return CCV3D_ERR_DEVICE_TIMEOUT;
+}
+
+ccv3d_status ccv3d_add_bf16(const void* a, const void* b, void* y, int64_t n, void* stream) {
+    if (!a || !b || !y || n < 0) return CCV3D_ERR_INVALID_ARG;
+    if (n == 0) return CCV3D_OK;
+    const int64_t blocks = (n + 255) / 256;
+    add_bf16_kernel<<<(unsigned)(blocks > 148 * 16 ? 148 * 16 : blocks), 256, 0, (cudaStream_t)stream>>>(
+        (const __nv_bfloat16*)a, (const __nv_bfloat16*)b, (__nv_bfloat16*)y, n);
+    return cudaGetLastError() == cudaSuccess ? CCV3D_OK : cuda_fail();
+}
+
+ccv3d_status ccv3d_upsample_bf16(const void* x, void* y, int32_t N, int32_t C, int32_t T, int32_t H, int32_t W,
+                                 int32_t rt, void* stream) {
+    if (!x || !y || N < 1 || C < 1 || T < 1 || H < 1 || W < 1 || rt < 1) return CCV3D_ERR_INVALID_ARG;
+    const int64_t total = (int64_t)N * C * T * rt * 4 * H * W;
+    const int64_t blocks = (total + 255) / 256;
+    upsample_bf16_kernel<<<(unsigned)(blocks > 148 * 16 ? 148 * 16 : blocks), 256, 0, (cudaStream_t)stream>>>(
+        (const __nv_bfloat16*)x, (__nv_bfloat16*)y, (int64_t)N * C, T, H, W, rt);
+    return cudaGetLastError() == cudaSuccess ? CCV3D_OK : cuda_fail();
+}
+
+}  // extern "C"

@@ -1,0 +1,148 @@
+// Plain FP32-FMA kernels: the direct causal Conv3D (FP32 layers, and the
+// BF16 reference route), the cache-update copy, and the chain glue.
+//
+// The direct kernel evaluates Eq. (2) as written: for an output element it
+// walks (ci, dt, dh, dw), picks the source frame of tap dt from the cache or
+// from x (Eq. (1) with p_l = 0: Z frame t+dt), treats out-of-image taps as
+// zero and adds the bias once.  FP32 accumulation in registers; one rounding
+// at the store.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace ccv3d {
+
+__device__ __forceinline__ float ld_as_float(const float* p) { return __ldg(p); }
+__device__ __forceinline__ float ld_as_float(const __nv_bfloat16* p) {
+    return __bfloat162float(__ldg(p));
+}
+__device__ __forceinline__ void st_from_float(float* p, float v) { *p = v; }
+__device__ __forceinline__ void st_from_float(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+
+struct SimtParams {
+    const void* x;
+    const void* cache;  // may be null: first chunk, absent frames are skipped
+    const void* w;      // original [Cout,Cin,kt,kh,kw] order, storage dtype
+    const float* bias;  // FP32, [Cout]
+    void* out;
+    int N, Cin, Cout, T, H, W, kt, kh, kw;
+};
+
+constexpr int SIMT_CO = 8;       // output channels per thread
+constexpr int SIMT_THREADS = 128;
+
+// grid.x: ceil(N*T*H*W / SIMT_THREADS), grid.y: ceil(Cout / SIMT_CO)
+template <typename TIn, typename TOut>
+__global__ void __launch_bounds__(SIMT_THREADS) conv3d_direct_kernel(const SimtParams p) {
+    const int64_t HW = (int64_t)p.H * p.W;
+    const int64_t npix = (int64_t)p.N * p.T * HW;
+    const int64_t pix = (int64_t)blockIdx.x * SIMT_THREADS + threadIdx.x;
+    if (pix >= npix) return;
+    const int w0 = (int)(pix % p.W);
+    const int h0 = (int)((pix / p.W) % p.H);
+    const int t = (int)((pix / HW) % p.T);
+    const int n = (int)(pix / (HW * p.T));
+    const int co0 = blockIdx.y * SIMT_CO;
+    const int ph = (p.kh - 1) / 2, pw = (p.kw - 1) / 2, tc = p.kt - 1;
+    const int taps = p.kt * p.kh * p.kw;
+
+    float acc[SIMT_CO];
+#pragma unroll
+    for (int j = 0; j < SIMT_CO; ++j) acc[j] = (co0 + j < p.Cout) ? p.bias[co0 + j] : 0.f;
+
+    const TIn* x = (const TIn*)p.x;
+    const TIn* cache = (const TIn*)p.cache;
+    const TIn* wt = (const TIn*)p.w;
+    for (int ci = 0; ci < p.Cin; ++ci) {
+        for (int dt = 0; dt < p.kt; ++dt) {
+            const int tau = t + dt;  // frame of Z = [cache ; x]
+            const TIn* frame;
+            if (tau < tc) {
+                if (!cache) continue;
+                frame = cache + (((int64_t)n * p.Cin + ci) * tc + tau) * HW;
+            } else {
+                frame = x + (((int64_t)n * p.Cin + ci) * p.T + (tau - tc)) * HW;
+            }
+            for (int dh = 0; dh < p.kh; ++dh) {
+                const int hs = h0 + dh - ph;
+                if (hs < 0 || hs >= p.H) continue;
+                for (int dw = 0; dw < p.kw; ++dw) {
+                    const int ws = w0 + dw - pw;
+                    if (ws < 0 || ws >= p.W) continue;
+                    const float v = ld_as_float(frame + (int64_t)hs * p.W + ws);
+                    const int64_t wofs = ((int64_t)ci * p.kt + dt) * p.kh * p.kw + dh * p.kw + dw;
+#pragma unroll
+                    for (int j = 0; j < SIMT_CO; ++j) {
+                        if (co0 + j < p.Cout)
+                            acc[j] = fmaf(v, ld_as_float(wt + (int64_t)(co0 + j) * p.Cin * taps + wofs), acc[j]);
+                    }
+                }
+            }
+        }
+    }
+    TOut* out = (TOut*)p.out;
+#pragma unroll
+    for (int j = 0; j < SIMT_CO; ++j)
+        if (co0 + j < p.Cout)
+            st_from_float(out + (((int64_t)n * p.Cout + co0 + j) * p.T + t) * HW + (int64_t)h0 * p.W + w0, acc[j]);
+}
+
+// new_cache[n,ci,j,:,:] = Z[n,ci,T+j,:,:], Z = [cache ; x]; pure bit copy in units of `unit` bytes
+// (16 when the frame size allows it, else the element size).
+// grid.x covers one frame in units, grid.y strides over the N*Cin*(kt-1) planes.
+template <typename U>
+__global__ void cache_update_kernel(const U* __restrict__ x, const U* __restrict__ cache, U* __restrict__ new_cache,
+                                    int Cin, int T, int tc, int64_t frame_units, int64_t planes) {
+    for (int64_t plane = blockIdx.y; plane < planes; plane += gridDim.y) {  // plane = (n*Cin + ci)*tc + j
+        const int j = (int)(plane % tc);
+        const int64_t nc = plane / tc;
+        const int tau = T + j;
+        const U* src = nullptr;
+        if (tau < tc) {
+            if (cache) src = cache + (nc * tc + tau) * frame_units;
+        } else {
+            src = x + (nc * T + (tau - tc)) * frame_units;
+        }
+        U* dst = new_cache + plane * frame_units;
+        for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < frame_units;
+             i += (int64_t)gridDim.x * blockDim.x) {
+            if (src) {
+                dst[i] = src[i];
+            } else {
+                U z;
+                memset(&z, 0, sizeof(U));
+                dst[i] = z;
+            }
+        }
+    }
+}
+
+// FP32 bias from the stored bias (or zeros), padded with zeros up to n_pad.
+template <typename TIn>
+__global__ void bias_to_f32_kernel(const TIn* __restrict__ b, float* __restrict__ out, int n, int n_pad) {
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n_pad) out[i] = (b && i < n) ? ld_as_float(b + i) : 0.f;
+}
+
+// ---- chain glue ----
+__global__ void add_bf16_kernel(const __nv_bfloat16* __restrict__ a, const __nv_bfloat16* __restrict__ b,
+                                __nv_bfloat16* __restrict__ y, int64_t n) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        y[i] = __float2bfloat16_rn(__bfloat162float(a[i]) + __bfloat162float(b[i]));
+}
+
+// y[nc, t*rt + r, 2h + a, 2w + b] = x[nc, t, h, w]
+__global__ void upsample_bf16_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ y,
+                                     int64_t NC, int T, int H, int W, int rt) {
+    const int64_t total = NC * T * rt * (int64_t)(2 * H) * (2 * W);
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int wo = (int)(i % (2 * W));
+        const int ho = (int)((i / (2 * W)) % (2 * H));
+        const int to = (int)((i / ((int64_t)4 * W * H)) % (T * rt));
+        const int64_t nc = i / ((int64_t)4 * W * H * T * rt);
+        y[i] = x[((nc * T + to / rt) * H + ho / 2) * W + wo / 2];
+    }
+}
+
+}  // namespace ccv3d

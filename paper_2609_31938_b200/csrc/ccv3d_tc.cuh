@@ -1,0 +1,532 @@
+// Tensor-core route for BF16 layers on sm_100a.
+//
+//   pack_weights_kernel   once per layer: w[Cout,Cin,kt,kh,kw] -> Wp[tap][Cout_pad][Cin_pad]
+//                         (per-tap, Cin-contiguous: the K-major B operand).
+//   stage_frames_kernel   per call: Z = [cache ; x] (NCTHW) -> channels-last blocks
+//                         Zs[n][frame][cb][h][w][KB], and in the same pass the
+//                         bit-exact cache update new_cache = last kt-1 frames of Z.
+//   conv3d_tcgen05_kernel per call: persistent implicit GEMM.  For an output tile of
+//                         16 rows x 8*NB pixels of one frame t, D[pixel, co] =
+//                         sum over (dt, ci-block, dh, dw) of A_tap[pixel, ci] * Wp[tap][co, ci]
+//                         (Eq. (2) with all taps folded into one K loop).  One TMA load
+//                         brings the (16+kh-1) x (8*NB+kw-1) pixel halo of a (frame, ci-block)
+//                         into shared memory (out-of-image pixels arrive as zeros = the
+//                         spatial padding); the kh*kw spatial taps are shared-memory
+//                         descriptor offsets into that one halo tile.  Accumulation is FP32
+//                         in tensor memory; the epilogue adds the bias once, rounds once
+//                         and stores NCTHW.
+//
+// Every wait on an mbarrier is bounded: when a limit expires the CTA records the
+// wait site in a global status word, raises a shared abort flag so that its other
+// roles stop too, releases its tensor memory and returns.
+#pragma once
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace ccv3d {
+
+// ------------------------------------------------------------------------------------------------
+// weight packing (create time)
+// ------------------------------------------------------------------------------------------------
+// Wp[tap][co][ci] for co < cout_pad, ci < cin_pad; zero outside the real extents.
+__global__ void pack_weights_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wp, int Cout,
+                                    int Cin, int taps, int cout_pad, int cin_pad) {
+    const int64_t total = (int64_t)taps * cout_pad * cin_pad;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int ci = (int)(i % cin_pad);
+        const int co = (int)((i / cin_pad) % cout_pad);
+        const int tap = (int)(i / ((int64_t)cin_pad * cout_pad));
+        __nv_bfloat16 v = __float2bfloat16_rn(0.f);
+        if (ci < Cin && co < Cout) v = w[((int64_t)co * Cin + ci) * taps + tap];
+        wp[i] = v;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// staging: NCTHW -> channels-last blocks, fused with the cache update
+// ------------------------------------------------------------------------------------------------
+struct StageParams {
+    const __nv_bfloat16* x;      // [N,Cin,T,H,W]
+    const __nv_bfloat16* cache;  // [N,Cin,tc,H,W] or null
+    __nv_bfloat16* zs;           // [N][F][CB][H][W][KB], F = tc + T
+    __nv_bfloat16* new_cache;    // [N,Cin,tc,H,W] or null
+    int N, Cin, T, H, W, tc, CB;
+    int f_begin;                 // first Z frame to stage (tc when there is no cache and nothing older is needed)
+};
+
+constexpr int STG_PX = 64;  // pixels of one image row handled per block
+
+// grid: (ceil(W/64), H, N*(F - f_begin)*CB); block: 32 * (KB/8) threads.
+// VEC: W % 8 == 0 and all bases 16-byte aligned -> 16-byte loads along w.
+template <int KB, bool VEC>
+__global__ void __launch_bounds__(32 * (KB / 8)) stage_frames_kernel(const StageParams p) {
+    constexpr int NTHR = 32 * (KB / 8);
+    constexpr int PITCH = STG_PX / 2 + 1;  // 32-bit words per channel row (+1: bank spread)
+    __shared__ uint32_t tile[KB * PITCH];
+
+    const int F = p.tc + p.T;
+    const int nf = F - p.f_begin;
+    int z = blockIdx.z;
+    const int cb = z % p.CB;
+    z /= p.CB;
+    const int f = p.f_begin + z % nf;
+    const int n = z / nf;
+    const int h = blockIdx.y;
+    const int w0 = blockIdx.x * STG_PX;
+    const int64_t HW = (int64_t)p.H * p.W;
+
+    // source frame of Z: cache frames first (oldest first), then x
+    const __nv_bfloat16* src = nullptr;  // base of channel 0 of this (n, frame); channel stride cstride
+    int64_t cstride = 0;
+    if (f < p.tc) {
+        if (p.cache) {
+            src = p.cache + ((int64_t)n * p.Cin * p.tc + f) * HW;
+            cstride = (int64_t)p.tc * HW;
+        }
+    } else {
+        src = p.x + ((int64_t)n * p.Cin * p.T + (f - p.tc)) * HW;
+        cstride = (int64_t)p.T * HW;
+    }
+    // does this frame belong to the updated cache?  new_cache[j] = Z[T + j]
+    const int jc = f - p.T;
+    __nv_bfloat16* ncdst = nullptr;
+    if (p.new_cache && jc >= 0 && jc < p.tc) ncdst = p.new_cache + ((int64_t)n * p.Cin * p.tc + jc) * HW;
+    const int64_t ncstride = (int64_t)p.tc * HW;
+
+    // ---- load phase: KB channel rows of up to 64 pixels ----
+    if (VEC) {
+        // 8 vectors of 8 pixels per row
+        for (int i = threadIdx.x; i < KB * 8; i += NTHR) {
+            const int c = i >> 3, v = i & 7;
+            const int ci = cb * KB + c;
+            const int w = w0 + v * 8;
+            uint4 val = make_uint4(0u, 0u, 0u, 0u);
+            if (w < p.W && ci < p.Cin) {
+                if (src) val = __ldg(reinterpret_cast<const uint4*>(src + ci * cstride + (int64_t)h * p.W + w));
+                if (ncdst) *reinterpret_cast<uint4*>(ncdst + ci * ncstride + (int64_t)h * p.W + w) = val;
+            }
+            uint32_t* row = tile + c * PITCH + v * 4;
+            row[0] = val.x; row[1] = val.y; row[2] = val.z; row[3] = val.w;
+        }
+    } else {
+        unsigned short* t16 = reinterpret_cast<unsigned short*>(tile);
+        for (int i = threadIdx.x; i < KB * STG_PX; i += NTHR) {
+            const int c = i / STG_PX, px = i % STG_PX;
+            const int ci = cb * KB + c;
+            const int w = w0 + px;
+            unsigned short val = 0;
+            if (w < p.W && ci < p.Cin) {
+                if (src) val = __ldg(reinterpret_cast<const unsigned short*>(src + ci * cstride + (int64_t)h * p.W + w));
+                if (ncdst) *reinterpret_cast<unsigned short*>(ncdst + ci * ncstride + (int64_t)h * p.W + w) = val;
+            }
+            t16[c * (2 * PITCH) + px] = val;
+        }
+    }
+    __syncthreads();
+
+    // ---- store phase: each thread builds the 16-byte channel octet of two neighbouring pixels ----
+    constexpr int OCT = KB / 8;
+    const int oct = threadIdx.x % OCT;
+    const int pp = threadIdx.x / OCT;  // pixel pair 0..31
+    uint32_t lo[4], hi[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        const uint32_t a = tile[(oct * 8 + 2 * k) * PITCH + pp];      // channel 2k:   pixels (2pp, 2pp+1)
+        const uint32_t b = tile[(oct * 8 + 2 * k + 1) * PITCH + pp];  // channel 2k+1
+        lo[k] = __byte_perm(a, b, 0x5410);                            // pixel 2pp:   (ch 2k, ch 2k+1)
+        hi[k] = __byte_perm(a, b, 0x7632);                            // pixel 2pp+1
+    }
+    __nv_bfloat16* dst = p.zs + ((((int64_t)n * F + f) * p.CB + cb) * HW + (int64_t)h * p.W) * KB;
+    const int wa = w0 + 2 * pp;
+    if (wa < p.W) *reinterpret_cast<uint4*>(dst + (int64_t)wa * KB + oct * 8) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+    if (wa + 1 < p.W)
+        *reinterpret_cast<uint4*>(dst + (int64_t)(wa + 1) * KB + oct * 8) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+}
+
+// ------------------------------------------------------------------------------------------------
+// PTX wrappers (sm_100a)
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+__device__ __forceinline__ uint64_t globaltimer_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2,
+                                            int c3, int c4) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, "
+        "%6}], [%7];" ::"r"(dst),
+        "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::
+            "r"(dst),
+        "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, "
+        "[%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// ------------------------------------------------------------------------------------------------
+// the implicit-GEMM kernel
+// ------------------------------------------------------------------------------------------------
+struct TcParams {
+    int N, T, H, W, Cout;
+    int F;            // frames of Z held in the staging buffer (kt-1 + T)
+    int kt, kh, kw;
+    int CB;           // input-channel blocks of KB
+    int NT, NPAD;     // output-channel tiles and their (padded) width, NPAD % 16 == 0, <= 256
+    int tiles_h, tiles_w, total_tiles;
+    int first_frame;  // Z frames below this are absent (first chunk): their taps are skipped
+    int out_f32;      // 1: out is FP32, 0: BF16
+    int per_tap_a;    // 1: one A load per tap (box without halo), 0: one halo load per (dt, ci-block)
+    int SA, SB, ACC;  // ring depths and accumulator buffers
+    uint32_t a_slot, b_slot;  // bytes per ring slot (multiples of 1024)
+    uint32_t tmem_cols;       // power of two >= NB*NPAD*ACC
+    uint64_t wait_limit_ns;
+    const float* bias;        // [NT*NPAD]
+    void* out;
+    unsigned int* status;     // 0 = fine; else (block << 8) | site
+};
+
+enum : uint32_t {
+    SITE_A_EMPTY = 1, SITE_B_EMPTY = 2, SITE_A_FULL = 3, SITE_B_FULL = 4, SITE_ACC_EMPTY = 5, SITE_ACC_FULL = 6,
+    SITE_DRAIN = 7
+};
+
+constexpr int TC_THREADS = 256;
+constexpr int TC_MAX_STAGES = 12;
+
+struct TcShared {  // placed after the rings
+    uint64_t full_a[TC_MAX_STAGES], empty_a[TC_MAX_STAGES];
+    uint64_t full_b[TC_MAX_STAGES], empty_b[TC_MAX_STAGES];
+    uint64_t acc_full[2], acc_empty[2];
+    uint32_t tmem_base;
+    volatile int abort_flag;
+};
+
+// Bounded wait.  Returns false when the limit expired or another role aborted.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, TcShared* sh, const TcParams& p, uint32_t site) {
+    const uint32_t b = smem_u32(bar);
+    if (mbar_try_wait(b, parity)) return true;
+    const uint64_t t0 = globaltimer_ns();
+    for (uint32_t it = 1;; ++it) {
+        if (mbar_try_wait(b, parity)) return true;
+        if ((it & 255u) == 0u) {
+            if (sh->abort_flag) return false;
+            if (globaltimer_ns() - t0 > p.wait_limit_ns) {
+                sh->abort_flag = 1;
+                atomicCAS(p.status, 0u, (blockIdx.x << 8) | site);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ uint64_t make_desc_hi(uint32_t sbo_bytes, uint32_t layout_type) {
+    // bits 32-45: stride-dimension byte offset >> 4; bits 46-47: descriptor version 1; bits 61-63: swizzle mode
+    return ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | ((uint64_t)layout_type << 61);
+}
+
+template <int KB, int NB>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged activations (c, w, h, cb, n*F+f)
+                      const __grid_constant__ CUtensorMap tm_w,   // packed weights (ci, co, tap)
+                      const TcParams p) {
+    constexpr uint32_t ROWB = KB * 2;                       // bytes per pixel row (one swizzle span)
+    constexpr uint32_t LAYOUT = (KB == 64) ? 2u : 4u;       // 128-byte / 64-byte swizzle
+    constexpr uint32_t B_SBO = 8 * ROWB;                    // 8-row group pitch of the weight tile
+    constexpr int KSTEPS = KB / 16;
+    constexpr int TW = 8 * NB;                              // tile width in pixels; tile height is 16
+
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t* ring_a = smem;
+    uint8_t* ring_b = smem + (size_t)p.SA * p.a_slot;
+    TcShared* sh = reinterpret_cast<TcShared*>(ring_b + (size_t)p.SB * p.b_slot);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int ph = (p.kh - 1) / 2, pw = (p.kw - 1) / 2;
+    const int BW = p.per_tap_a ? TW : TW + p.kw - 1;        // pixels per smem image row
+    const int BH = p.per_tap_a ? 16 : 16 + p.kh - 1;
+    const uint32_t a_bytes = (uint32_t)BW * BH * ROWB;
+    const uint32_t b_bytes = (uint32_t)p.NPAD * ROWB;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < p.SA; ++i) { mbar_init(smem_u32(&sh->full_a[i]), 1); mbar_init(smem_u32(&sh->empty_a[i]), 1); }
+        for (int i = 0; i < p.SB; ++i) { mbar_init(smem_u32(&sh->full_b[i]), 1); mbar_init(smem_u32(&sh->empty_b[i]), 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&sh->acc_full[i]), 1); mbar_init(smem_u32(&sh->acc_empty[i]), 4); }
+        sh->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 3) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)),
+                     "r"(p.tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = sh->tmem_base;
+
+    // ---------------------------------------------------------------- A producer
+    if (warp == 0) {
+        if (lane == 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_a) : "memory");
+            int s = 0;
+            uint32_t phase = 1;
+            int issued = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+                int r = tile / p.NT;
+                const int t = r % p.T; r /= p.T;
+                const int tx = r % p.tiles_w; r /= p.tiles_w;
+                const int ty = r % p.tiles_h;
+                const int n = r / p.tiles_h;
+                const int h0 = ty * 16, w0 = tx * TW;
+                const int dt0 = (p.first_frame - t > 0) ? p.first_frame - t : 0;
+                for (int dt = dt0; ok && dt < p.kt; ++dt)
+                    for (int cb = 0; ok && cb < p.CB; ++cb) {
+                        const int fz = n * p.F + t + dt;
+                        const int ntap = p.per_tap_a ? p.kh * p.kw : 1;
+                        for (int tp = 0; tp < ntap; ++tp) {
+                            if (!(ok = mbar_wait(&sh->empty_a[s], phase, sh, p, SITE_A_EMPTY))) break;
+                            const uint32_t bar = smem_u32(&sh->full_a[s]);
+                            mbar_expect_tx(bar, a_bytes);
+                            const int dh = p.per_tap_a ? tp / p.kw : 0, dw = p.per_tap_a ? tp % p.kw : 0;
+                            tma_load_5d(smem_u32(ring_a + (size_t)s * p.a_slot), &tm_a, bar, 0, w0 - pw + dw, h0 - ph + dh, cb,
+                                        fz);
+                            ++issued;
+                            if (++s == p.SA) { s = 0; phase ^= 1; }
+                        }
+                    }
+            }
+            if (!ok && issued) {  // give copies in flight a bounded chance to land before the CTA goes away
+                const uint64_t t0 = globaltimer_ns();
+                while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+            }
+        }
+    }
+    // ---------------------------------------------------------------- B producer
+    else if (warp == 1) {
+        if (lane == 0) {
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_w) : "memory");
+            int s = 0;
+            uint32_t phase = 1;
+            int issued = 0;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+                const int nt = tile % p.NT;
+                const int t = (tile / p.NT) % p.T;
+                const int dt0 = (p.first_frame - t > 0) ? p.first_frame - t : 0;
+                for (int dt = dt0; ok && dt < p.kt; ++dt)
+                    for (int cb = 0; ok && cb < p.CB; ++cb)
+                        for (int tp = 0; tp < p.kh * p.kw; ++tp) {
+                            if (!(ok = mbar_wait(&sh->empty_b[s], phase, sh, p, SITE_B_EMPTY))) break;
+                            const uint32_t bar = smem_u32(&sh->full_b[s]);
+                            mbar_expect_tx(bar, b_bytes);
+                            tma_load_3d(smem_u32(ring_b + (size_t)s * p.b_slot), &tm_w, bar, cb * KB, nt * p.NPAD,
+                                        dt * p.kh * p.kw + tp);
+                            ++issued;
+                            if (++s == p.SB) { s = 0; phase ^= 1; }
+                        }
+            }
+            if (!ok && issued) {
+                const uint64_t t0 = globaltimer_ns();
+                while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
+            }
+        }
+    }
+    // ---------------------------------------------------------------- MMA issuer
+    else if (warp == 2) {
+        if (lane == 0) {
+            // instruction descriptor: D=F32, A=B=BF16, both K-major, N = NPAD, M = 128
+            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.NPAD >> 3) << 17) | ((128u >> 4) << 24);
+            const uint64_t a_hi = make_desc_hi((uint32_t)BW * ROWB, LAYOUT);  // 8-pixel groups are one image row apart
+            const uint64_t b_hi = make_desc_hi(B_SBO, LAYOUT);
+            const uint32_t lbo = 1u << 16;                                    // unused for swizzled K-major; canonical value
+            int sa = 0, sb = 0, acc = 0;
+            uint32_t pa = 0, pb = 0, pacc = 1;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+                const int t = (tile / p.NT) % p.T;
+                const int dt0 = (p.first_frame - t > 0) ? p.first_frame - t : 0;
+                if (!(ok = mbar_wait(&sh->acc_empty[acc], pacc, sh, p, SITE_ACC_EMPTY))) break;
+                tc_fence_after();
+                const uint32_t d0 = tmem_base + (uint32_t)acc * NB * p.NPAD;
+                uint32_t accumulate = 0;
+                for (int dt = dt0; ok && dt < p.kt; ++dt)
+                    for (int cb = 0; ok && cb < p.CB; ++cb) {
+                        uint32_t a_addr = 0;
+                        if (!p.per_tap_a) {
+                            if (!(ok = mbar_wait(&sh->full_a[sa], pa, sh, p, SITE_A_FULL))) break;
+                            a_addr = smem_u32(ring_a + (size_t)sa * p.a_slot);
+                        }
+                        for (int tp = 0; tp < p.kh * p.kw; ++tp) {
+                            uint32_t a_tap;
+                            if (p.per_tap_a) {
+                                if (!(ok = mbar_wait(&sh->full_a[sa], pa, sh, p, SITE_A_FULL))) break;
+                                a_tap = smem_u32(ring_a + (size_t)sa * p.a_slot);
+                            } else {
+                                a_tap = a_addr + (uint32_t)((tp / p.kw) * BW + (tp % p.kw)) * ROWB;
+                            }
+                            if (!(ok = mbar_wait(&sh->full_b[sb], pb, sh, p, SITE_B_FULL))) break;
+                            tc_fence_after();
+                            const uint32_t b_addr = smem_u32(ring_b + (size_t)sb * p.b_slot);
+#pragma unroll
+                            for (int blk = 0; blk < NB; ++blk) {
+#pragma unroll
+                                for (int k = 0; k < KSTEPS; ++k) {
+                                    // The start address is only 16-byte granular and need not sit on the 1024-byte
+                                    // swizzle period: the swizzle is a function of the absolute shared-memory
+                                    // address (as the TMA unit applied it), so the base-offset field stays 0.
+                                    const uint64_t ad = a_hi | lbo | (((a_tap + blk * 8 * ROWB + k * 32) & 0x3FFFFu) >> 4);
+                                    const uint64_t bd = b_hi | lbo | (((b_addr + k * 32) & 0x3FFFFu) >> 4);
+                                    tc_mma_bf16(d0 + blk * p.NPAD, ad, bd, idesc, (k == 0) ? accumulate : 1u);
+                                }
+                            }
+                            accumulate = 1;
+                            tc_commit(smem_u32(&sh->empty_b[sb]));
+                            if (++sb == p.SB) { sb = 0; pb ^= 1; }
+                            if (p.per_tap_a) {
+                                tc_commit(smem_u32(&sh->empty_a[sa]));
+                                if (++sa == p.SA) { sa = 0; pa ^= 1; }
+                            }
+                        }
+                        if (ok && !p.per_tap_a) {
+                            tc_commit(smem_u32(&sh->empty_a[sa]));
+                            if (++sa == p.SA) { sa = 0; pa ^= 1; }
+                        }
+                    }
+                if (!ok) break;
+                tc_commit(smem_u32(&sh->acc_full[acc]));
+                if (++acc == p.ACC) { acc = 0; pacc ^= 1; }
+            }
+        }
+    }
+    // ---------------------------------------------------------------- epilogue (warps 4..7)
+    else if (warp >= 4) {
+        const int q = warp & 3;  // TMEM lane quarter this warp may read
+        int acc = 0;
+        uint32_t pacc = 0;
+        bool ok = true;
+        const int64_t HW = (int64_t)p.H * p.W;
+        for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+            const int nt = tile % p.NT;
+            int r = tile / p.NT;
+            const int t = r % p.T; r /= p.T;
+            const int tx = r % p.tiles_w; r /= p.tiles_w;
+            const int ty = r % p.tiles_h;
+            const int n = r / p.tiles_h;
+            ok = mbar_wait(&sh->acc_full[acc], pacc, sh, p, SITE_ACC_FULL);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const int m = q * 32 + lane;          // accumulator row = pixel m of the 128-pixel block
+            const int h = ty * 16 + (m >> 3);
+            const bool hval = h < p.H;
+#pragma unroll 1
+            for (int blk = 0; blk < NB; ++blk) {
+                const int w = tx * TW + blk * 8 + (m & 7);
+                const bool valid = hval && w < p.W;
+                const int64_t pix = (int64_t)t * HW + (int64_t)h * p.W + w;
+#pragma unroll 1
+                for (int c0 = 0; c0 < p.NPAD; c0 += 32) {
+                    uint32_t v[32];
+                    const uint32_t taddr = tmem_base + (uint32_t)(acc * NB + blk) * p.NPAD + c0 + ((uint32_t)(q * 32) << 16);
+                    const int nc = (p.NPAD - c0 >= 32) ? 32 : 16;
+                    if (nc == 32) tc_ld32(taddr, v); else tc_ld16(taddr, v);
+                    tc_wait_ld();
+                    const int co0 = nt * p.NPAD + c0;
+                    if (valid) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            const int co = co0 + j;
+                            if (j < nc && co < p.Cout) {
+                                const float val = __uint_as_float(v[j]) + __ldg(p.bias + co);
+                                const int64_t o = ((int64_t)n * p.Cout + co) * p.T * HW + pix;
+                                if (p.out_f32) reinterpret_cast<float*>(p.out)[o] = val;
+                                else reinterpret_cast<__nv_bfloat16*>(p.out)[o] = __float2bfloat16_rn(val);
+                            }
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&sh->acc_empty[acc]));
+            if (++acc == p.ACC) { acc = 0; pacc ^= 1; }
+        }
+    }
+
+    // ---------------------------------------------------------------- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 3) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
+    }
+}
+
+}  // namespace ccv3d
