@@ -55,10 +55,12 @@ struct ccv3d_handle {
     void* hx; void* hc; void* ho; void* hn;
     uint64_t hx_b, hc_b, ho_b, hn_b;
     EncodeTiledFn encode;
-    CUtensorMap tm_w;
+    CUtensorMap tm_w;      // weight tiles of one tap
+    CUtensorMap tm_w_row;  // weight tiles of one kernel row (kw taps)
     CUtensorMap tm_a;
     ShapeKey tm_a_key;
-    uint64_t wait_limit_ns;
+    CUtensorMap tm_o;
+    long long wait_limit_clk;
     ccv3d_counters ctr;
 };
 
@@ -142,14 +144,14 @@ ccv3d_status grow(void** buf, uint64_t* have, uint64_t need) {
     return CCV3D_OK;
 }
 
-ccv3d_status encode_weight_map(ccv3d_handle* h) {
+ccv3d_status encode_weight_map(ccv3d_handle* h, CUtensorMap* tm, int taps_per_box) {
     const TcPlan& pl = h->plan;
     const int taps = h->d.kt * h->d.kh * h->d.kw;
     cuuint64_t dims[3] = {(cuuint64_t)pl.cin_pad, (cuuint64_t)pl.cout_pad, (cuuint64_t)taps};
     cuuint64_t strides[2] = {(cuuint64_t)pl.cin_pad * 2, (cuuint64_t)pl.cin_pad * pl.cout_pad * 2};
-    cuuint32_t box[3] = {(cuuint32_t)pl.KB, (cuuint32_t)pl.NPAD, 1};
+    cuuint32_t box[3] = {(cuuint32_t)pl.KB, (cuuint32_t)pl.NPAD, (cuuint32_t)taps_per_box};
     cuuint32_t es[3] = {1, 1, 1};
-    CUresult r = h->encode(&h->tm_w, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, h->wp, dims, strides, box, es,
+    CUresult r = h->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, h->wp, dims, strides, box, es,
                            CU_TENSOR_MAP_INTERLEAVE_NONE,
                            pl.KB == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -171,6 +173,18 @@ ccv3d_status encode_act_map(ccv3d_handle* h, int N, int T, int H, int W, int BW,
     return r == CUDA_SUCCESS ? CCV3D_OK : CCV3D_ERR_CUDA;
 }
 
+ccv3d_status encode_out_map(ccv3d_handle* h, void* out, int N, int T, int H, int W, int TW, int ECH) {
+    const uint64_t es2 = 2;  // BF16 output only
+    cuuint64_t dims[5] = {(cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)T, (cuuint64_t)h->d.cout, (cuuint64_t)N};
+    cuuint64_t strides[4] = {es2 * W, es2 * W * H, es2 * W * H * T, es2 * W * H * T * h->d.cout};
+    cuuint32_t box[5] = {(cuuint32_t)TW, 16, 1, (cuuint32_t)ECH, 1};
+    cuuint32_t es[5] = {1, 1, 1, 1, 1};
+    CUresult r = h->encode(&h->tm_o, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, out, dims, strides, box, es,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? CCV3D_OK : CCV3D_ERR_CUDA;
+}
+
 uint64_t tc_workspace_bytes(const ccv3d_handle* h, int N, int T, int H, int W) {
     const int F = h->d.kt - 1 + T;
     return (uint64_t)N * F * h->plan.cin_pad * H * W * 2;
@@ -181,7 +195,7 @@ ccv3d_status launch_tc(ccv3d_handle* h, const TcParams& p, size_t smem, int grid
     auto kern = conv3d_tcgen05_kernel<KB, NB>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return cuda_fail();
-    kern<<<grid, TC_THREADS, smem, st>>>(h->tm_a, h->tm_w, p);
+    kern<<<grid, TC_THREADS, smem, st>>>(h->tm_a, p.TPB > 1 ? h->tm_w_row : h->tm_w, h->tm_o, p);
     if (cudaGetLastError() != cudaSuccess) return cuda_fail();
     h->ctr.kernel_launches++;
     return CCV3D_OK;
@@ -245,21 +259,39 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     p.per_tap_a = per_tap;
     p.ACC = pl.ACC;
     p.a_slot = (uint32_t)align_up((uint64_t)BW * BH * pl.KB * 2, 1024);
-    p.b_slot = (uint32_t)align_up((uint64_t)pl.NPAD * pl.KB * 2, 1024);
-    const size_t fixed = 1024 /*alignment slack*/ + align_up(sizeof(TcShared), 128);
+    p.b_tap = (uint32_t)pl.NPAD * pl.KB * 2;
+    // epilogue: BF16 output rows that TMA can address (W*2 bytes a multiple of 16) go through shared memory
+    p.epi_tma = (!p.out_f32 && W % 8 == 0) ? 1 : 0;
+    p.ECH = (pl.NPAD % 32 == 0) ? 32 : 16;
+    p.e_slot = p.epi_tma ? (uint32_t)(p.ECH * 16 * TW * 2) : 0;
+    const size_t fixed = 1024 /*alignment slack*/ + align_up(sizeof(TcShared), 128) + 2 * (size_t)p.e_slot;
     const size_t budget = SMEM_LIMIT - fixed;
+    // weight stage: a whole kernel row of taps when that stays small, so that a stage carries enough MMAs
+    p.TPB = (!per_tap && (size_t)p.b_tap * d.kw <= 40960) ? d.kw : 1;
     int SA = per_tap ? 3 : 2;
-    if ((size_t)SA * p.a_slot + 2 * (size_t)p.b_slot > budget) return CCV3D_ERR_UNSUPPORTED;
+    for (;;) {
+        p.b_slot = (uint32_t)align_up((uint64_t)p.b_tap * p.TPB, 1024);
+        if ((size_t)SA * p.a_slot + 3 * (size_t)p.b_slot <= budget) break;
+        if (p.TPB > 1) { p.TPB = 1; continue; }
+        if ((size_t)SA * p.a_slot + 2 * (size_t)p.b_slot <= budget) break;
+        return CCV3D_ERR_UNSUPPORTED;
+    }
     int SB = (int)((budget - (size_t)SA * p.a_slot) / p.b_slot);
     if (SB > 8) SB = 8;
     while (SA < 4 && (size_t)(SA + 1) * p.a_slot + (size_t)SB * p.b_slot <= budget) ++SA;
     p.SA = SA; p.SB = SB;
     p.tmem_cols = pow2_cols((uint32_t)(NB * pl.NPAD * pl.ACC));
     if (p.tmem_cols > 512) return CCV3D_ERR_UNSUPPORTED;
-    p.wait_limit_ns = h->wait_limit_ns;
+    p.wait_limit_clk = h->wait_limit_clk;
     p.bias = h->bias32;
     p.out = out;
     p.status = h->status;
+    if (p.epi_tma) {
+        s = encode_out_map(h, out, N, T, H, W, TW, p.ECH);
+        if (s != CCV3D_OK) return s;
+    } else {
+        h->tm_o = h->tm_w;  // never dereferenced on this path; any valid descriptor will do
+    }
     const size_t smem = fixed + (size_t)SA * p.a_slot + (size_t)SB * p.b_slot;
     const int grid = p.total_tiles < h->sm_count ? p.total_tiles : h->sm_count;
     if (pl.KB == 64) s = launch_tc<64, 2>(h, p, smem, grid, st);
@@ -375,10 +407,11 @@ ccv3d_status ccv3d_create(ccv3d_handle** out_h, const ccv3d_desc* d, const void*
     h->device = dev;
     h->sm_count = prop.multiProcessorCount;
     h->use_tc = (d->dtype == CCV3D_BF16) && !(d->flags & CCV3D_FLAG_FORCE_SIMT);
-    h->wait_limit_ns = 1000000000ull;
+    // bound of every in-kernel wait: about one second of SM clocks (clock rate is reported in kHz)
+    h->wait_limit_clk = (long long)prop.clockRate * 1000ll;
     if (const char* e = getenv("CCV3D_WAIT_LIMIT_MS")) {
         const long v = atol(e);
-        if (v > 0 && v <= 10000) h->wait_limit_ns = (uint64_t)v * 1000000ull;
+        if (v > 0 && v <= 10000) h->wait_limit_clk = (long long)prop.clockRate * v;
     }
     cudaStream_t st = (cudaStream_t)stream;
     const int taps = d->kt * d->kh * d->kw;
@@ -407,7 +440,8 @@ ccv3d_status ccv3d_create(ccv3d_handle** out_h, const ccv3d_desc* d, const void*
                                                   taps, h->plan.cout_pad, h->plan.cin_pad);
         if (cudaGetLastError() != cudaSuccess) return fail(cuda_fail());
         h->ctr.kernel_launches++;
-        if (encode_weight_map(h) != CCV3D_OK) return fail(CCV3D_ERR_CUDA);
+        if (encode_weight_map(h, &h->tm_w, 1) != CCV3D_OK) return fail(CCV3D_ERR_CUDA);
+        if (encode_weight_map(h, &h->tm_w_row, d->kw) != CCV3D_OK) return fail(CCV3D_ERR_CUDA);
     } else {
         const uint64_t wb = (uint64_t)d->cout * d->cin * taps * esize(d->dtype);
         if (cudaMalloc(&h->w_copy, wb) != cudaSuccess) return fail(CCV3D_ERR_NOMEM);

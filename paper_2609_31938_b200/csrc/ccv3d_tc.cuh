@@ -170,11 +170,6 @@ __device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity)
         : "memory");
     return ok;
 }
-__device__ __forceinline__ uint64_t globaltimer_ns() {
-    uint64_t t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
 __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2,
                                             int c3, int c4) {
     asm volatile(
@@ -226,6 +221,19 @@ __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[32]) {
 }
 __device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+__device__ __forceinline__ void tma_store_5d(const CUtensorMap* tm, uint32_t src, int c0, int c1, int c2, int c3, int c4) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5, %6}], [%1];" ::"l"(tm),
+        "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
+        : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
+
 // ------------------------------------------------------------------------------------------------
 // the implicit-GEMM kernel
 // ------------------------------------------------------------------------------------------------
@@ -239,18 +247,21 @@ struct TcParams {
     int first_frame;  // Z frames below this are absent (first chunk): their taps are skipped
     int out_f32;      // 1: out is FP32, 0: BF16
     int per_tap_a;    // 1: one A load per tap (box without halo), 0: one halo load per (dt, ci-block)
+    int TPB;          // spatial taps per weight stage (1 or kw); kh*kw % TPB == 0
+    int epi_tma;      // 1: epilogue stages BF16 tiles in shared memory and stores them with TMA; 0: direct stores
+    int ECH;          // output channels per epilogue chunk (32 or 16) when epi_tma
     int SA, SB, ACC;  // ring depths and accumulator buffers
-    uint32_t a_slot, b_slot;  // bytes per ring slot (multiples of 1024)
+    uint32_t a_slot, b_slot, b_tap;  // bytes per ring slot (multiples of 1024) and per tap inside a weight slot
+    uint32_t e_slot;          // bytes of one epilogue staging buffer (two are allocated when epi_tma)
     uint32_t tmem_cols;       // power of two >= NB*NPAD*ACC
-    uint64_t wait_limit_ns;
+    long long wait_limit_clk; // bound of every mbarrier wait, in SM clocks
     const float* bias;        // [NT*NPAD]
     void* out;
     unsigned int* status;     // 0 = fine; else (block << 8) | site
 };
 
 enum : uint32_t {
-    SITE_A_EMPTY = 1, SITE_B_EMPTY = 2, SITE_A_FULL = 3, SITE_B_FULL = 4, SITE_ACC_EMPTY = 5, SITE_ACC_FULL = 6,
-    SITE_DRAIN = 7
+    SITE_A_EMPTY = 1, SITE_B_EMPTY = 2, SITE_A_FULL = 3, SITE_B_FULL = 4, SITE_ACC_EMPTY = 5, SITE_ACC_FULL = 6
 };
 
 constexpr int TC_THREADS = 256;
@@ -264,16 +275,18 @@ struct TcShared {  // placed after the rings
     volatile int abort_flag;
 };
 
-// Bounded wait.  Returns false when the limit expired or another role aborted.
+// Bounded wait.  Returns false when the limit expired or another role of this CTA aborted.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, TcShared* sh, const TcParams& p, uint32_t site) {
     const uint32_t b = smem_u32(bar);
     if (mbar_try_wait(b, parity)) return true;
-    const uint64_t t0 = globaltimer_ns();
+    long long t0 = 0;
     for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(b, parity)) return true;
-        if ((it & 255u) == 0u) {
+        if ((it & 63u) == 0u) {
             if (sh->abort_flag) return false;
-            if (globaltimer_ns() - t0 > p.wait_limit_ns) {
+            const long long now = clock64();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > p.wait_limit_clk) {
                 sh->abort_flag = 1;
                 atomicCAS(p.status, 0u, (blockIdx.x << 8) | site);
                 return false;
@@ -282,15 +295,28 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, TcShar
     }
 }
 
-__device__ __forceinline__ uint64_t make_desc_hi(uint32_t sbo_bytes, uint32_t layout_type) {
-    // bits 32-45: stride-dimension byte offset >> 4; bits 46-47: descriptor version 1; bits 61-63: swizzle mode
-    return ((uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32) | (1ull << 46) | ((uint64_t)layout_type << 61);
+// After an abort: give copies in flight a bounded time to land before the CTA goes away.
+__device__ __forceinline__ void drain_delay() {
+    const long long t0 = clock64();
+    while (clock64() - t0 < 400000) __nanosleep(1000);
+}
+
+__device__ __forceinline__ uint32_t make_desc_hi(uint32_t sbo_bytes, uint32_t layout_type) {
+    // upper word of a shared-memory matrix descriptor: bits 32-45 stride-dimension byte offset >> 4,
+    // bits 46-47 descriptor version 1, bits 61-63 swizzle mode
+    return ((sbo_bytes >> 4) & 0x3FFFu) | (1u << 14) | (layout_type << 29);
+}
+__device__ __forceinline__ uint64_t make_desc(uint32_t hi, uint32_t addr) {
+    // lower word: bits 0-13 start address >> 4, bits 16-29 leading-dimension byte offset >> 4 (unused for
+    // swizzled K-major operands; canonical value 1)
+    return ((uint64_t)hi << 32) | (uint64_t)(((addr & 0x3FFFFu) >> 4) | (1u << 16));
 }
 
 template <int KB, int NB>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged activations (c, w, h, cb, n*F+f)
                       const __grid_constant__ CUtensorMap tm_w,   // packed weights (ci, co, tap)
+                      const __grid_constant__ CUtensorMap tm_o,   // out (w, h, t, co, n); used when p.epi_tma
                       const TcParams p) {
     constexpr uint32_t ROWB = KB * 2;                       // bytes per pixel row (one swizzle span)
     constexpr uint32_t LAYOUT = (KB == 64) ? 2u : 4u;       // 128-byte / 64-byte swizzle
@@ -301,16 +327,16 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* ring_a = smem;
-    uint8_t* ring_b = smem + (size_t)p.SA * p.a_slot;
-    TcShared* sh = reinterpret_cast<TcShared*>(ring_b + (size_t)p.SB * p.b_slot);
+    uint8_t* ring_b = ring_a + (size_t)p.SA * p.a_slot;
+    uint8_t* epi_buf = ring_b + (size_t)p.SB * p.b_slot;
+    TcShared* sh = reinterpret_cast<TcShared*>(epi_buf + (p.epi_tma ? 2 * (size_t)p.e_slot : 0));
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
     const int ph = (p.kh - 1) / 2, pw = (p.kw - 1) / 2;
     const int BW = p.per_tap_a ? TW : TW + p.kw - 1;        // pixels per smem image row
     const int BH = p.per_tap_a ? 16 : 16 + p.kh - 1;
-    const uint32_t a_bytes = (uint32_t)BW * BH * ROWB;
-    const uint32_t b_bytes = (uint32_t)p.NPAD * ROWB;
+    const int spatial = p.kh * p.kw;
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < p.SA; ++i) { mbar_init(smem_u32(&sh->full_a[i]), 1); mbar_init(smem_u32(&sh->empty_a[i]), 1); }
@@ -334,9 +360,9 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     if (warp == 0) {
         if (lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_a) : "memory");
+            const uint32_t a_bytes = (uint32_t)BW * BH * ROWB;
             int s = 0;
             uint32_t phase = 1;
-            int issued = 0;
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
                 int r = tile / p.NT;
@@ -349,7 +375,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                 for (int dt = dt0; ok && dt < p.kt; ++dt)
                     for (int cb = 0; ok && cb < p.CB; ++cb) {
                         const int fz = n * p.F + t + dt;
-                        const int ntap = p.per_tap_a ? p.kh * p.kw : 1;
+                        const int ntap = p.per_tap_a ? spatial : 1;
                         for (int tp = 0; tp < ntap; ++tp) {
                             if (!(ok = mbar_wait(&sh->empty_a[s], phase, sh, p, SITE_A_EMPTY))) break;
                             const uint32_t bar = smem_u32(&sh->full_a[s]);
@@ -357,24 +383,20 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                             const int dh = p.per_tap_a ? tp / p.kw : 0, dw = p.per_tap_a ? tp % p.kw : 0;
                             tma_load_5d(smem_u32(ring_a + (size_t)s * p.a_slot), &tm_a, bar, 0, w0 - pw + dw, h0 - ph + dh, cb,
                                         fz);
-                            ++issued;
                             if (++s == p.SA) { s = 0; phase ^= 1; }
                         }
                     }
             }
-            if (!ok && issued) {  // give copies in flight a bounded chance to land before the CTA goes away
-                const uint64_t t0 = globaltimer_ns();
-                while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
-            }
+            if (!ok) drain_delay();
         }
     }
     // ---------------------------------------------------------------- B producer
     else if (warp == 1) {
         if (lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_w) : "memory");
+            const uint32_t b_bytes = (uint32_t)p.NPAD * ROWB * p.TPB;
             int s = 0;
             uint32_t phase = 1;
-            int issued = 0;
             bool ok = true;
             for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
                 const int nt = tile % p.NT;
@@ -382,20 +404,16 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                 const int dt0 = (p.first_frame - t > 0) ? p.first_frame - t : 0;
                 for (int dt = dt0; ok && dt < p.kt; ++dt)
                     for (int cb = 0; ok && cb < p.CB; ++cb)
-                        for (int tp = 0; tp < p.kh * p.kw; ++tp) {
+                        for (int tp = 0; tp < spatial; tp += p.TPB) {
                             if (!(ok = mbar_wait(&sh->empty_b[s], phase, sh, p, SITE_B_EMPTY))) break;
                             const uint32_t bar = smem_u32(&sh->full_b[s]);
                             mbar_expect_tx(bar, b_bytes);
                             tma_load_3d(smem_u32(ring_b + (size_t)s * p.b_slot), &tm_w, bar, cb * KB, nt * p.NPAD,
-                                        dt * p.kh * p.kw + tp);
-                            ++issued;
+                                        dt * spatial + tp);
                             if (++s == p.SB) { s = 0; phase ^= 1; }
                         }
             }
-            if (!ok && issued) {
-                const uint64_t t0 = globaltimer_ns();
-                while (globaltimer_ns() - t0 < 200000ull) __nanosleep(1000);
-            }
+            if (!ok) drain_delay();
         }
     }
     // ---------------------------------------------------------------- MMA issuer
@@ -403,9 +421,8 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
         if (lane == 0) {
             // instruction descriptor: D=F32, A=B=BF16, both K-major, N = NPAD, M = 128
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.NPAD >> 3) << 17) | ((128u >> 4) << 24);
-            const uint64_t a_hi = make_desc_hi((uint32_t)BW * ROWB, LAYOUT);  // 8-pixel groups are one image row apart
-            const uint64_t b_hi = make_desc_hi(B_SBO, LAYOUT);
-            const uint32_t lbo = 1u << 16;                                    // unused for swizzled K-major; canonical value
+            const uint32_t a_hi = make_desc_hi((uint32_t)BW * ROWB, LAYOUT);  // 8-pixel groups are one image row apart
+            const uint32_t b_hi = make_desc_hi(B_SBO, LAYOUT);
             int sa = 0, sb = 0, acc = 0;
             uint32_t pa = 0, pb = 0, pacc = 1;
             bool ok = true;
@@ -423,36 +440,43 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                             if (!(ok = mbar_wait(&sh->full_a[sa], pa, sh, p, SITE_A_FULL))) break;
                             a_addr = smem_u32(ring_a + (size_t)sa * p.a_slot);
                         }
-                        for (int tp = 0; tp < p.kh * p.kw; ++tp) {
-                            uint32_t a_tap;
-                            if (p.per_tap_a) {
-                                if (!(ok = mbar_wait(&sh->full_a[sa], pa, sh, p, SITE_A_FULL))) break;
-                                a_tap = smem_u32(ring_a + (size_t)sa * p.a_slot);
-                            } else {
-                                a_tap = a_addr + (uint32_t)((tp / p.kw) * BW + (tp % p.kw)) * ROWB;
-                            }
+                        uint32_t a_row = a_addr;  // start of the halo row of tap row dh
+                        for (int tp = 0, dw = 0; tp < spatial; tp += p.TPB) {
                             if (!(ok = mbar_wait(&sh->full_b[sb], pb, sh, p, SITE_B_FULL))) break;
-                            tc_fence_after();
-                            const uint32_t b_addr = smem_u32(ring_b + (size_t)sb * p.b_slot);
-#pragma unroll
-                            for (int blk = 0; blk < NB; ++blk) {
-#pragma unroll
-                                for (int k = 0; k < KSTEPS; ++k) {
-                                    // The start address is only 16-byte granular and need not sit on the 1024-byte
-                                    // swizzle period: the swizzle is a function of the absolute shared-memory
-                                    // address (as the TMA unit applied it), so the base-offset field stays 0.
-                                    const uint64_t ad = a_hi | lbo | (((a_tap + blk * 8 * ROWB + k * 32) & 0x3FFFFu) >> 4);
-                                    const uint64_t bd = b_hi | lbo | (((b_addr + k * 32) & 0x3FFFFu) >> 4);
-                                    tc_mma_bf16(d0 + blk * p.NPAD, ad, bd, idesc, (k == 0) ? accumulate : 1u);
+                            uint32_t b_addr = smem_u32(ring_b + (size_t)sb * p.b_slot);
+                            for (int u = 0; u < p.TPB; ++u) {
+                                uint32_t a_tap;
+                                if (p.per_tap_a) {
+                                    if (!(ok = mbar_wait(&sh->full_a[sa], pa, sh, p, SITE_A_FULL))) break;
+                                    a_tap = smem_u32(ring_a + (size_t)sa * p.a_slot);
+                                } else {
+                                    a_tap = a_row + (uint32_t)dw * ROWB;
                                 }
+                                tc_fence_after();
+                                // The A start address is only 16-byte granular and need not sit on the swizzle
+                                // period: the swizzle is a function of the absolute shared-memory address (as the
+                                // TMA unit applied it), so the descriptor's base-offset field stays 0.
+                                const uint64_t ad = make_desc(a_hi, a_tap);
+                                const uint64_t bd = make_desc(b_hi, b_addr);
+#pragma unroll
+                                for (int blk = 0; blk < NB; ++blk) {
+#pragma unroll
+                                    for (int k = 0; k < KSTEPS; ++k) {
+                                        tc_mma_bf16(d0 + blk * p.NPAD, ad + (uint64_t)((blk * 8 * ROWB + k * 32) >> 4),
+                                                    bd + (uint64_t)((k * 32) >> 4), idesc, (k == 0) ? accumulate : 1u);
+                                    }
+                                }
+                                accumulate = 1;
+                                b_addr += p.b_tap;
+                                if (p.per_tap_a) {
+                                    tc_commit(smem_u32(&sh->empty_a[sa]));
+                                    if (++sa == p.SA) { sa = 0; pa ^= 1; }
+                                }
+                                if (++dw == p.kw) { dw = 0; a_row += (uint32_t)BW * ROWB; }
                             }
-                            accumulate = 1;
+                            if (!ok) break;
                             tc_commit(smem_u32(&sh->empty_b[sb]));
                             if (++sb == p.SB) { sb = 0; pb ^= 1; }
-                            if (p.per_tap_a) {
-                                tc_commit(smem_u32(&sh->empty_a[sa]));
-                                if (++sa == p.SA) { sa = 0; pa ^= 1; }
-                            }
                         }
                         if (ok && !p.per_tap_a) {
                             tc_commit(smem_u32(&sh->empty_a[sa]));
@@ -472,6 +496,9 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
         uint32_t pacc = 0;
         bool ok = true;
         const int64_t HW = (int64_t)p.H * p.W;
+        const int m = q * 32 + lane;  // accumulator row = pixel m of a 128-pixel block: image row m/8, pixel m%8
+        const bool elected = (threadIdx.x == 4 * 32);
+        int ebuf = 0;
         for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
             const int nt = tile % p.NT;
             int r = tile / p.NT;
@@ -483,31 +510,57 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            const int m = q * 32 + lane;          // accumulator row = pixel m of the 128-pixel block
-            const int h = ty * 16 + (m >> 3);
-            const bool hval = h < p.H;
-#pragma unroll 1
-            for (int blk = 0; blk < NB; ++blk) {
-                const int w = tx * TW + blk * 8 + (m & 7);
-                const bool valid = hval && w < p.W;
-                const int64_t pix = (int64_t)t * HW + (int64_t)h * p.W + w;
-#pragma unroll 1
-                for (int c0 = 0; c0 < p.NPAD; c0 += 32) {
-                    uint32_t v[32];
-                    const uint32_t taddr = tmem_base + (uint32_t)(acc * NB + blk) * p.NPAD + c0 + ((uint32_t)(q * 32) << 16);
-                    const int nc = (p.NPAD - c0 >= 32) ? 32 : 16;
-                    if (nc == 32) tc_ld32(taddr, v); else tc_ld16(taddr, v);
-                    tc_wait_ld();
+            const uint32_t t_acc = tmem_base + (uint32_t)(acc * NB) * p.NPAD + ((uint32_t)(q * 32) << 16);
+            if (p.epi_tma) {
+                // BF16 tile chunks [ECH channels][16 rows][TW pixels] -> shared memory -> one TMA store per chunk
+                for (int c0 = 0; c0 < p.NPAD; c0 += p.ECH) {
+                    if (elected) bulk_wait_read<1>();   // the store that last read this buffer has finished reading
+                    epi_bar_sync();
+                    __nv_bfloat16* stg = reinterpret_cast<__nv_bfloat16*>(epi_buf + (size_t)ebuf * p.e_slot);
                     const int co0 = nt * p.NPAD + c0;
-                    if (valid) {
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            const int co = co0 + j;
-                            if (j < nc && co < p.Cout) {
-                                const float val = __uint_as_float(v[j]) + __ldg(p.bias + co);
-                                const int64_t o = ((int64_t)n * p.Cout + co) * p.T * HW + pix;
-                                if (p.out_f32) reinterpret_cast<float*>(p.out)[o] = val;
-                                else reinterpret_cast<__nv_bfloat16*>(p.out)[o] = __float2bfloat16_rn(val);
+                    for (int blk = 0; blk < NB; ++blk) {
+                        uint32_t v[32];
+                        if (p.ECH == 32) tc_ld32(t_acc + blk * p.NPAD + c0, v); else tc_ld16(t_acc + blk * p.NPAD + c0, v);
+                        tc_wait_ld();
+                        __nv_bfloat16* dst = stg + (m >> 3) * TW + blk * 8 + (m & 7);
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (j < p.ECH)
+                                dst[j * 16 * TW] = __float2bfloat16_rn(__uint_as_float(v[j]) + __ldg(p.bias + co0 + j));
+                    }
+                    fence_async_smem();
+                    epi_bar_sync();
+                    if (elected) {
+                        tma_store_5d(&tm_o, smem_u32(stg), tx * TW, ty * 16, t, co0, n);
+                        bulk_commit();
+                    }
+                    ebuf ^= 1;
+                }
+            } else {
+                const int h = ty * 16 + (m >> 3);
+#pragma unroll 1
+                for (int blk = 0; blk < NB; ++blk) {
+                    const int w = tx * TW + blk * 8 + (m & 7);
+                    const bool valid = h < p.H && w < p.W;
+                    const int64_t pix = (int64_t)t * HW + (int64_t)h * p.W + w;
+#pragma unroll 1
+                    for (int c0 = 0; c0 < p.NPAD; c0 += 32) {
+                        uint32_t v[32];
+                        const int nc = (p.NPAD - c0 >= 32) ? 32 : 16;
+                        if (nc == 32) tc_ld32(t_acc + blk * p.NPAD + c0, v); else tc_ld16(t_acc + blk * p.NPAD + c0, v);
+                        tc_wait_ld();
+                        const int co0 = nt * p.NPAD + c0;
+                        if (valid) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) {
+                                const int co = co0 + j;
+                                if (j < nc && co < p.Cout) {
+                                    const float val = __uint_as_float(v[j]) + __ldg(p.bias + co);
+                                    const int64_t o = ((int64_t)n * p.Cout + co) * p.T * HW + pix;
+                                    if (p.out_f32) reinterpret_cast<float*>(p.out)[o] = val;
+                                    else reinterpret_cast<__nv_bfloat16*>(p.out)[o] = __float2bfloat16_rn(val);
+                                }
                             }
                         }
                     }
@@ -518,6 +571,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
             if (lane == 0) mbar_arrive(smem_u32(&sh->acc_empty[acc]));
             if (++acc == p.ACC) { acc = 0; pacc ^= 1; }
         }
+        if (p.epi_tma && elected) bulk_wait_all();   // all stores of this CTA are complete before it exits
     }
 
     // ---------------------------------------------------------------- teardown
