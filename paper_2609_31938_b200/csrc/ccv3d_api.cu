@@ -55,8 +55,6 @@ struct ccv3d_handle {
     void* hx; void* hc; void* ho; void* hn;
     uint64_t hx_b, hc_b, ho_b, hn_b;
     EncodeTiledFn encode;
-    CUtensorMap tm_w;      // weight tiles of one tap
-    CUtensorMap tm_w_row;  // weight tiles of one kernel row (kw taps)
     CUtensorMap tm_a;
     ShapeKey tm_a_key;
     CUtensorMap tm_o;
@@ -144,20 +142,6 @@ ccv3d_status grow(void** buf, uint64_t* have, uint64_t need) {
     return CCV3D_OK;
 }
 
-ccv3d_status encode_weight_map(ccv3d_handle* h, CUtensorMap* tm, int taps_per_box) {
-    const TcPlan& pl = h->plan;
-    const int taps = h->d.kt * h->d.kh * h->d.kw;
-    cuuint64_t dims[3] = {(cuuint64_t)pl.cin_pad, (cuuint64_t)pl.cout_pad, (cuuint64_t)taps};
-    cuuint64_t strides[2] = {(cuuint64_t)pl.cin_pad * 2, (cuuint64_t)pl.cin_pad * pl.cout_pad * 2};
-    cuuint32_t box[3] = {(cuuint32_t)pl.KB, (cuuint32_t)pl.NPAD, (cuuint32_t)taps_per_box};
-    cuuint32_t es[3] = {1, 1, 1};
-    CUresult r = h->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, h->wp, dims, strides, box, es,
-                           CU_TENSOR_MAP_INTERLEAVE_NONE,
-                           pl.KB == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
-                           CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
-    return r == CUDA_SUCCESS ? CCV3D_OK : CCV3D_ERR_CUDA;
-}
-
 ccv3d_status encode_act_map(ccv3d_handle* h, int N, int T, int H, int W, int BW, int BH) {
     const TcPlan& pl = h->plan;
     const int F = h->d.kt - 1 + T;
@@ -195,7 +179,7 @@ ccv3d_status launch_tc(ccv3d_handle* h, const TcParams& p, size_t smem, int grid
     auto kern = conv3d_tcgen05_kernel<KB, NB>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return cuda_fail();
-    kern<<<grid, TC_THREADS, smem, st>>>(h->tm_a, p.TPB > 1 ? h->tm_w_row : h->tm_w, h->tm_o, p);
+    kern<<<grid, TC_THREADS, smem, st>>>(h->tm_a, h->tm_o, p);
     if (cudaGetLastError() != cudaSuccess) return cuda_fail();
     h->ctr.kernel_launches++;
     return CCV3D_OK;
@@ -284,13 +268,14 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     if (p.tmem_cols > 512) return CCV3D_ERR_UNSUPPORTED;
     p.wait_limit_clk = h->wait_limit_clk;
     p.bias = h->bias32;
+    p.wq = (const uint8_t*)h->wp;
     p.out = out;
     p.status = h->status;
     if (p.epi_tma) {
         s = encode_out_map(h, out, N, T, H, W, TW, p.ECH);
         if (s != CCV3D_OK) return s;
     } else {
-        h->tm_o = h->tm_w;  // never dereferenced on this path; any valid descriptor will do
+        h->tm_o = h->tm_a;  // never dereferenced on this path; any valid descriptor will do
     }
     const size_t smem = fixed + (size_t)SA * p.a_slot + (size_t)SB * p.b_slot;
     const int grid = p.total_tiles < h->sm_count ? p.total_tiles : h->sm_count;
@@ -437,11 +422,10 @@ ccv3d_status ccv3d_create(ccv3d_handle** out_h, const ccv3d_desc* d, const void*
         const uint64_t wpb = (uint64_t)taps * h->plan.cout_pad * h->plan.cin_pad * 2;
         if (cudaMalloc(&h->wp, wpb) != cudaSuccess) return fail(CCV3D_ERR_NOMEM);
         pack_weights_kernel<<<1024, 256, 0, st>>>((const __nv_bfloat16*)w_dev, (__nv_bfloat16*)h->wp, d->cout, d->cin,
-                                                  taps, h->plan.cout_pad, h->plan.cin_pad);
+                                                  d->kt, d->kh * d->kw, h->plan.CB, h->plan.KB, h->plan.NT,
+                                                  h->plan.NPAD);
         if (cudaGetLastError() != cudaSuccess) return fail(cuda_fail());
         h->ctr.kernel_launches++;
-        if (encode_weight_map(h, &h->tm_w, 1) != CCV3D_OK) return fail(CCV3D_ERR_CUDA);
-        if (encode_weight_map(h, &h->tm_w_row, d->kw) != CCV3D_OK) return fail(CCV3D_ERR_CUDA);
     } else {
         const uint64_t wb = (uint64_t)d->cout * d->cin * taps * esize(d->dtype);
         if (cudaMalloc(&h->w_copy, wb) != cudaSuccess) return fail(CCV3D_ERR_NOMEM);

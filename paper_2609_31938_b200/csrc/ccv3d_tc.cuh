@@ -1,7 +1,7 @@
 // Tensor-core route for BF16 layers on sm_100a.
 //
-//   pack_weights_kernel   once per layer: w[Cout,Cin,kt,kh,kw] -> Wp[tap][Cout_pad][Cin_pad]
-//                         (per-tap, Cin-contiguous: the K-major B operand).
+//   pack_weights_kernel   once per layer: w[Cout,Cin,kt,kh,kw] -> per (tap, ci-block, co-tile) tiles stored
+//                         as the swizzled shared-memory image of the K-major B operand.
 //   stage_frames_kernel   per call: Z = [cache ; x] (NCTHW) -> channels-last blocks
 //                         Zs[n][frame][cb][h][w][KB], and in the same pass the
 //                         bit-exact cache update new_cache = last kt-1 frames of Z.
@@ -30,17 +30,30 @@ namespace ccv3d {
 // ------------------------------------------------------------------------------------------------
 // weight packing (create time)
 // ------------------------------------------------------------------------------------------------
-// Wp[tap][co][ci] for co < cout_pad, ci < cin_pad; zero outside the real extents.
-__global__ void pack_weights_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wp, int Cout,
-                                    int Cin, int taps, int cout_pad, int cin_pad) {
-    const int64_t total = (int64_t)taps * cout_pad * cin_pad;
+// Wq[dt][cb][nt][sp][r][e]: for temporal tap dt, input-channel block cb, output-channel tile nt and spatial
+// tap sp = dh*kw + dw, a tile of NPAD rows (output channels) x KB input channels, stored as the exact
+// shared-memory image the tensor core expects for a K-major operand with 128-byte (KB = 64) or 64-byte
+// (KB = 32) swizzle: the 16-byte chunk c of row r sits at chunk position c ^ (r & 7), respectively
+// c ^ ((r >> 1) & 3).  A tile, or a run of consecutive spatial taps, is then one contiguous bulk copy.
+// Zero outside the real channel extents.
+__global__ void pack_weights_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wq, int Cout,
+                                    int Cin, int kt, int spatial, int CB, int KB, int NT, int NPAD) {
+    const int64_t total = (int64_t)kt * CB * NT * spatial * NPAD * KB;
     for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-        const int ci = (int)(i % cin_pad);
-        const int co = (int)((i / cin_pad) % cout_pad);
-        const int tap = (int)(i / ((int64_t)cin_pad * cout_pad));
+        int64_t q = i;
+        const int e = (int)(q % KB); q /= KB;
+        const int r = (int)(q % NPAD); q /= NPAD;
+        const int sp = (int)(q % spatial); q /= spatial;
+        const int nt = (int)(q % NT); q /= NT;
+        const int cb = (int)(q % CB);
+        const int dt = (int)(q / CB);
+        const int chunk_stored = e >> 3;
+        const int chunk = chunk_stored ^ (KB == 64 ? (r & 7) : ((r >> 1) & 3));
+        const int ci = cb * KB + chunk * 8 + (e & 7);
+        const int co = nt * NPAD + r;
         __nv_bfloat16 v = __float2bfloat16_rn(0.f);
-        if (ci < Cin && co < Cout) v = w[((int64_t)co * Cin + ci) * taps + tap];
-        wp[i] = v;
+        if (ci < Cin && co < Cout) v = w[(((int64_t)co * Cin + ci) * kt + dt) * spatial + sp];
+        wq[i] = v;
     }
 }
 
@@ -178,25 +191,27 @@ __device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* tm,
         "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar)
         : "memory");
 }
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::
-            "r"(dst),
-        "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
-        : "memory");
+__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
-__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                            uint32_t accumulate) {
+// D[tmem] (+)= A[smem] * B[smem]^T, M = 128, K = 16, BF16 inputs, FP32 accumulate.  The 64-bit shared-memory
+// descriptors are passed as halves so that stepping along K or to another pixel block is one 32-bit add.
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                            uint32_t idesc, uint32_t accumulate) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
-        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "mov.b64 da, {%1, %2};\n\t"
+        "mov.b64 db, {%3, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
         : "memory");
 }
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
@@ -256,6 +271,7 @@ struct TcParams {
     uint32_t tmem_cols;       // power of two >= NB*NPAD*ACC
     long long wait_limit_clk; // bound of every mbarrier wait, in SM clocks
     const float* bias;        // [NT*NPAD]
+    const uint8_t* wq;        // packed weight tiles [dt][cb][nt][sp] of b_tap bytes each
     void* out;
     unsigned int* status;     // 0 = fine; else (block << 8) | site
 };
@@ -306,16 +322,15 @@ __device__ __forceinline__ uint32_t make_desc_hi(uint32_t sbo_bytes, uint32_t la
     // bits 46-47 descriptor version 1, bits 61-63 swizzle mode
     return ((sbo_bytes >> 4) & 0x3FFFu) | (1u << 14) | (layout_type << 29);
 }
-__device__ __forceinline__ uint64_t make_desc(uint32_t hi, uint32_t addr) {
+__device__ __forceinline__ uint32_t make_desc_lo(uint32_t addr) {
     // lower word: bits 0-13 start address >> 4, bits 16-29 leading-dimension byte offset >> 4 (unused for
     // swizzled K-major operands; canonical value 1)
-    return ((uint64_t)hi << 32) | (uint64_t)(((addr & 0x3FFFFu) >> 4) | (1u << 16));
+    return ((addr & 0x3FFFFu) >> 4) | (1u << 16);
 }
 
 template <int KB, int NB>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged activations (c, w, h, cb, n*F+f)
-                      const __grid_constant__ CUtensorMap tm_w,   // packed weights (ci, co, tap)
                       const __grid_constant__ CUtensorMap tm_o,   // out (w, h, t, co, n); used when p.epi_tma
                       const TcParams p) {
     constexpr uint32_t ROWB = KB * 2;                       // bytes per pixel row (one swizzle span)
@@ -323,6 +338,8 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     constexpr uint32_t B_SBO = 8 * ROWB;                    // 8-row group pitch of the weight tile
     constexpr int KSTEPS = KB / 16;
     constexpr int TW = 8 * NB;                              // tile width in pixels; tile height is 16
+    constexpr int NI = (NB >= 2) ? 2 : 1;                   // MMA-issuing warps (2 and 3), each owning NB/NI pixel blocks
+    constexpr int NBW = NB / NI;
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -339,9 +356,9 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     const int spatial = p.kh * p.kw;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < p.SA; ++i) { mbar_init(smem_u32(&sh->full_a[i]), 1); mbar_init(smem_u32(&sh->empty_a[i]), 1); }
-        for (int i = 0; i < p.SB; ++i) { mbar_init(smem_u32(&sh->full_b[i]), 1); mbar_init(smem_u32(&sh->empty_b[i]), 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&sh->acc_full[i]), 1); mbar_init(smem_u32(&sh->acc_empty[i]), 4); }
+        for (int i = 0; i < p.SA; ++i) { mbar_init(smem_u32(&sh->full_a[i]), 1); mbar_init(smem_u32(&sh->empty_a[i]), NI); }
+        for (int i = 0; i < p.SB; ++i) { mbar_init(smem_u32(&sh->full_b[i]), 1); mbar_init(smem_u32(&sh->empty_b[i]), NI); }
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&sh->acc_full[i]), NI); mbar_init(smem_u32(&sh->acc_empty[i]), 4); }
         sh->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -393,8 +410,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     // ---------------------------------------------------------------- B producer
     else if (warp == 1) {
         if (lane == 0) {
-            asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_w) : "memory");
-            const uint32_t b_bytes = (uint32_t)p.NPAD * ROWB * p.TPB;
+            const uint32_t b_bytes = p.b_tap * p.TPB;
             int s = 0;
             uint32_t phase = 1;
             bool ok = true;
@@ -403,26 +419,34 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                 const int t = (tile / p.NT) % p.T;
                 const int dt0 = (p.first_frame - t > 0) ? p.first_frame - t : 0;
                 for (int dt = dt0; ok && dt < p.kt; ++dt)
-                    for (int cb = 0; ok && cb < p.CB; ++cb)
+                    for (int cb = 0; ok && cb < p.CB; ++cb) {
+                        const uint8_t* src = p.wq + (size_t)((dt * p.CB + cb) * p.NT + nt) * spatial * p.b_tap;
                         for (int tp = 0; tp < spatial; tp += p.TPB) {
                             if (!(ok = mbar_wait(&sh->empty_b[s], phase, sh, p, SITE_B_EMPTY))) break;
                             const uint32_t bar = smem_u32(&sh->full_b[s]);
                             mbar_expect_tx(bar, b_bytes);
-                            tma_load_3d(smem_u32(ring_b + (size_t)s * p.b_slot), &tm_w, bar, cb * KB, nt * p.NPAD,
-                                        dt * spatial + tp);
+                            bulk_load(smem_u32(ring_b + (size_t)s * p.b_slot), src + (size_t)tp * p.b_tap, b_bytes, bar);
                             if (++s == p.SB) { s = 0; phase ^= 1; }
                         }
+                    }
             }
             if (!ok) drain_delay();
         }
     }
-    // ---------------------------------------------------------------- MMA issuer
-    else if (warp == 2) {
+    // ---------------------------------------------------------------- MMA issuers
+    // One thread of warp 2 (and of warp 3 when NB >= 2) issues the MMAs of its own pixel blocks.  A commit
+    // only tracks the MMAs of the committing thread, so the "slot free" and "accumulator full" barriers
+    // count one arrival per issuer.
+    else if (warp == 2 || (warp == 3 && NI == 2)) {
         if (lane == 0) {
+            const int iss = warp - 2;
             // instruction descriptor: D=F32, A=B=BF16, both K-major, N = NPAD, M = 128
             const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.NPAD >> 3) << 17) | ((128u >> 4) << 24);
             const uint32_t a_hi = make_desc_hi((uint32_t)BW * ROWB, LAYOUT);  // 8-pixel groups are one image row apart
             const uint32_t b_hi = make_desc_hi(B_SBO, LAYOUT);
+            const uint32_t a_blk = (uint32_t)(iss * NBW) * ((8 * ROWB) >> 4);  // descriptor offset of this issuer's first block
+            const uint32_t a_rowstep = ((uint32_t)BW * ROWB) >> 4;
+            const uint32_t b_tapstep = p.b_tap >> 4;
             int sa = 0, sb = 0, acc = 0;
             uint32_t pa = 0, pb = 0, pacc = 1;
             bool ok = true;
@@ -431,48 +455,45 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                 const int dt0 = (p.first_frame - t > 0) ? p.first_frame - t : 0;
                 if (!(ok = mbar_wait(&sh->acc_empty[acc], pacc, sh, p, SITE_ACC_EMPTY))) break;
                 tc_fence_after();
-                const uint32_t d0 = tmem_base + (uint32_t)acc * NB * p.NPAD;
+                const uint32_t d0 = tmem_base + (uint32_t)(acc * NB + iss * NBW) * p.NPAD;
                 uint32_t accumulate = 0;
                 for (int dt = dt0; ok && dt < p.kt; ++dt)
                     for (int cb = 0; ok && cb < p.CB; ++cb) {
-                        uint32_t a_addr = 0;
+                        uint32_t a_row = 0;  // descriptor low word of the halo row of the current tap row
                         if (!p.per_tap_a) {
                             if (!(ok = mbar_wait(&sh->full_a[sa], pa, sh, p, SITE_A_FULL))) break;
-                            a_addr = smem_u32(ring_a + (size_t)sa * p.a_slot);
+                            a_row = make_desc_lo(smem_u32(ring_a + (size_t)sa * p.a_slot)) + a_blk;
                         }
-                        uint32_t a_row = a_addr;  // start of the halo row of tap row dh
                         for (int tp = 0, dw = 0; tp < spatial; tp += p.TPB) {
                             if (!(ok = mbar_wait(&sh->full_b[sb], pb, sh, p, SITE_B_FULL))) break;
-                            uint32_t b_addr = smem_u32(ring_b + (size_t)sb * p.b_slot);
+                            tc_fence_after();
+                            uint32_t b_lo = make_desc_lo(smem_u32(ring_b + (size_t)sb * p.b_slot));
                             for (int u = 0; u < p.TPB; ++u) {
-                                uint32_t a_tap;
+                                uint32_t a_lo;
                                 if (p.per_tap_a) {
                                     if (!(ok = mbar_wait(&sh->full_a[sa], pa, sh, p, SITE_A_FULL))) break;
-                                    a_tap = smem_u32(ring_a + (size_t)sa * p.a_slot);
+                                    tc_fence_after();
+                                    a_lo = make_desc_lo(smem_u32(ring_a + (size_t)sa * p.a_slot)) + a_blk;
                                 } else {
-                                    a_tap = a_row + (uint32_t)dw * ROWB;
+                                    // The start address is only 16-byte granular and need not sit on the swizzle
+                                    // period: the swizzle is a function of the absolute shared-memory address (as
+                                    // the TMA unit applied it), so the descriptor's base-offset field stays 0.
+                                    a_lo = a_row + (uint32_t)dw * (ROWB >> 4);
                                 }
-                                tc_fence_after();
-                                // The A start address is only 16-byte granular and need not sit on the swizzle
-                                // period: the swizzle is a function of the absolute shared-memory address (as the
-                                // TMA unit applied it), so the descriptor's base-offset field stays 0.
-                                const uint64_t ad = make_desc(a_hi, a_tap);
-                                const uint64_t bd = make_desc(b_hi, b_addr);
 #pragma unroll
-                                for (int blk = 0; blk < NB; ++blk) {
+                                for (int j = 0; j < NBW; ++j) {
 #pragma unroll
-                                    for (int k = 0; k < KSTEPS; ++k) {
-                                        tc_mma_bf16(d0 + blk * p.NPAD, ad + (uint64_t)((blk * 8 * ROWB + k * 32) >> 4),
-                                                    bd + (uint64_t)((k * 32) >> 4), idesc, (k == 0) ? accumulate : 1u);
-                                    }
+                                    for (int k = 0; k < KSTEPS; ++k)
+                                        tc_mma_bf16(d0 + j * p.NPAD, a_lo + j * ((8 * ROWB) >> 4) + 2 * k, a_hi, b_lo + 2 * k, b_hi,
+                                                    idesc, (k == 0) ? accumulate : 1u);
                                 }
                                 accumulate = 1;
-                                b_addr += p.b_tap;
+                                b_lo += b_tapstep;
                                 if (p.per_tap_a) {
                                     tc_commit(smem_u32(&sh->empty_a[sa]));
                                     if (++sa == p.SA) { sa = 0; pa ^= 1; }
                                 }
-                                if (++dw == p.kw) { dw = 0; a_row += (uint32_t)BW * ROWB; }
+                                if (++dw == p.kw) { dw = 0; a_row += a_rowstep; }
                             }
                             if (!ok) break;
                             tc_commit(smem_u32(&sh->empty_b[sb]));
