@@ -174,9 +174,9 @@ uint64_t tc_workspace_bytes(const ccv3d_handle* h, int N, int T, int H, int W) {
     return (uint64_t)N * F * h->plan.cin_pad * H * W * 2;
 }
 
-template <int KB, int NB>
+template <int KB, int NB, int KS, int TPBC>
 ccv3d_status launch_tc(ccv3d_handle* h, const TcParams& p, size_t smem, int grid, cudaStream_t st) {
-    auto kern = conv3d_tcgen05_kernel<KB, NB>;
+    auto kern = conv3d_tcgen05_kernel<KB, NB, KS, TPBC>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return cuda_fail();
     kern<<<grid, TC_THREADS, smem, st>>>(h->tm_a, h->tm_o, p);
@@ -279,8 +279,18 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     }
     const size_t smem = fixed + (size_t)SA * p.a_slot + (size_t)SB * p.b_slot;
     const int grid = p.total_tiles < h->sm_count ? p.total_tiles : h->sm_count;
-    if (pl.KB == 64) s = launch_tc<64, 2>(h, p, smem, grid, st);
-    else s = launch_tc<32, 2>(h, p, smem, grid, st);
+    // straight-line tap loops for the common kernels; the run-time variant takes everything else
+    const int ks = (!per_tap && d.kh == d.kw && (d.kh == 1 || d.kh == 3)) ? d.kh : 0;
+#define CCV3D_LAUNCH(KBv)                                                                      \
+    do {                                                                                       \
+        if (ks == 3 && p.TPB == 3) s = launch_tc<KBv, 2, 3, 3>(h, p, smem, grid, st);          \
+        else if (ks == 3 && p.TPB == 1) s = launch_tc<KBv, 2, 3, 1>(h, p, smem, grid, st);     \
+        else if (ks == 1) s = launch_tc<KBv, 2, 1, 1>(h, p, smem, grid, st);                   \
+        else s = launch_tc<KBv, 2, 0, 0>(h, p, smem, grid, st);                                \
+    } while (0)
+    if (pl.KB == 64) CCV3D_LAUNCH(64);
+    else CCV3D_LAUNCH(32);
+#undef CCV3D_LAUNCH
     if (s == CCV3D_OK) h->ctr.tcgen05_bf16++;
     return s;
 }

@@ -196,6 +196,17 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
                  "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
 }
+// One lane of a fully converged warp; the others get 0.  Keeps the surrounding code warp-uniform so that
+// descriptors and addresses can live in uniform registers.
+__device__ __forceinline__ uint32_t elect_one() {
+    uint32_t pred;
+    asm volatile(
+        "{\n\t.reg .pred P;\n\t"
+        "elect.sync _|P, 0xffffffff;\n\t"
+        "selp.b32 %0, 1, 0, P;\n\t}"
+        : "=r"(pred));
+    return pred;
+}
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -328,7 +339,11 @@ __device__ __forceinline__ uint32_t make_desc_lo(uint32_t addr) {
     return ((addr & 0x3FFFFu) >> 4) | (1u << 16);
 }
 
-template <int KB, int NB>
+// KB: input channels per K block (64 -> 128-byte swizzle, 32 -> 64-byte swizzle).  NB: 128-pixel blocks per tile.
+// KS/TPBC: compile-time spatial kernel size (kh = kw = KS) and taps per weight stage, which turn the tap loop
+// into straight-line code with immediate descriptor offsets; KS = 0 keeps everything run-time (any odd kh, kw,
+// and the per-tap A mode).
+template <int KB, int NB, int KS, int TPBC>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged activations (c, w, h, cb, n*F+f)
                       const __grid_constant__ CUtensorMap tm_o,   // out (w, h, t, co, n); used when p.epi_tma
@@ -348,7 +363,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     uint8_t* epi_buf = ring_b + (size_t)p.SB * p.b_slot;
     TcShared* sh = reinterpret_cast<TcShared*>(epi_buf + (p.epi_tma ? 2 * (size_t)p.e_slot : 0));
 
-    const int warp = threadIdx.x >> 5;
+    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);  // provably warp-uniform
     const int lane = threadIdx.x & 31;
     const int ph = (p.kh - 1) / 2, pw = (p.kw - 1) / 2;
     const int BW = p.per_tap_a ? TW : TW + p.kw - 1;        // pixels per smem image row
@@ -434,22 +449,28 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
         }
     }
     // ---------------------------------------------------------------- MMA issuers
-    // One thread of warp 2 (and of warp 3 when NB >= 2) issues the MMAs of its own pixel blocks.  A commit
+    // Warp 2 (and warp 3 when NB >= 2) issues the MMAs of its own pixel blocks.  A commit
     // only tracks the MMAs of the committing thread, so the "slot free" and "accumulator full" barriers
     // count one arrival per issuer.
     else if (warp == 2 || (warp == 3 && NI == 2)) {
-        if (lane == 0) {
-            const int iss = warp - 2;
-            // instruction descriptor: D=F32, A=B=BF16, both K-major, N = NPAD, M = 128
-            const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.NPAD >> 3) << 17) | ((128u >> 4) << 24);
-            const uint32_t a_hi = make_desc_hi((uint32_t)BW * ROWB, LAYOUT);  // 8-pixel groups are one image row apart
-            const uint32_t b_hi = make_desc_hi(B_SBO, LAYOUT);
-            const uint32_t a_blk = (uint32_t)(iss * NBW) * ((8 * ROWB) >> 4);  // descriptor offset of this issuer's first block
-            const uint32_t a_rowstep = ((uint32_t)BW * ROWB) >> 4;
-            const uint32_t b_tapstep = p.b_tap >> 4;
-            int sa = 0, sb = 0, acc = 0;
-            uint32_t pa = 0, pb = 0, pacc = 1;
-            bool ok = true;
+        // The whole warp runs the loop (warp-uniform control flow); one elected lane issues.
+        const int iss = warp - 2;
+        // instruction descriptor: D=F32, A=B=BF16, both K-major, N = NPAD, M = 128
+        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.NPAD >> 3) << 17) | ((128u >> 4) << 24);
+        const uint32_t a_hi = make_desc_hi((uint32_t)BW * ROWB, LAYOUT);  // 8-pixel groups are one image row apart
+        const uint32_t b_hi = make_desc_hi(B_SBO, LAYOUT);
+        const uint32_t a_blk = (uint32_t)(iss * NBW) * ((8 * ROWB) >> 4);  // descriptor offset of this issuer's first block
+        const uint32_t a_rowstep = ((uint32_t)BW * ROWB) >> 4;
+        const uint32_t b_tapstep = p.b_tap >> 4;
+        int sa = 0, sb = 0, acc = 0;
+        uint32_t pa = 0, pb = 0, pacc = 1;
+        bool ok = true;
+        if constexpr (KS > 0) {
+            constexpr uint32_t A_ROWSTEP = ((uint32_t)(TW + KS - 1) * ROWB) >> 4;
+            constexpr int STAGES = KS * KS / TPBC;
+            uint32_t a_ring = make_desc_lo(smem_u32(ring_a)) + a_blk, b_ring = make_desc_lo(smem_u32(ring_b));
+            const uint32_t a_slotstep = p.a_slot >> 4, b_slotstep = p.b_slot >> 4;
+            const uint32_t a_ring0 = a_ring, b_ring0 = b_ring;
             for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
                 const int t = (tile / p.NT) % p.T;
                 const int dt0 = (p.first_frame - t > 0) ? p.first_frame - t : 0;
@@ -457,29 +478,80 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                 tc_fence_after();
                 const uint32_t d0 = tmem_base + (uint32_t)(acc * NB + iss * NBW) * p.NPAD;
                 uint32_t accumulate = 0;
-                for (int dt = dt0; ok && dt < p.kt; ++dt)
-                    for (int cb = 0; ok && cb < p.CB; ++cb) {
-                        uint32_t a_row = 0;  // descriptor low word of the halo row of the current tap row
-                        if (!p.per_tap_a) {
-                            if (!(ok = mbar_wait(&sh->full_a[sa], pa, sh, p, SITE_A_FULL))) break;
-                            a_row = make_desc_lo(smem_u32(ring_a + (size_t)sa * p.a_slot)) + a_blk;
-                        }
-                        for (int tp = 0, dw = 0; tp < spatial; tp += p.TPB) {
-                            if (!(ok = mbar_wait(&sh->full_b[sb], pb, sh, p, SITE_B_FULL))) break;
-                            tc_fence_after();
-                            uint32_t b_lo = make_desc_lo(smem_u32(ring_b + (size_t)sb * p.b_slot));
-                            for (int u = 0; u < p.TPB; ++u) {
-                                uint32_t a_lo;
-                                if (p.per_tap_a) {
-                                    if (!(ok = mbar_wait(&sh->full_a[sa], pa, sh, p, SITE_A_FULL))) break;
-                                    tc_fence_after();
-                                    a_lo = make_desc_lo(smem_u32(ring_a + (size_t)sa * p.a_slot)) + a_blk;
-                                } else {
-                                    // The start address is only 16-byte granular and need not sit on the swizzle
-                                    // period: the swizzle is a function of the absolute shared-memory address (as
-                                    // the TMA unit applied it), so the descriptor's base-offset field stays 0.
-                                    a_lo = a_row + (uint32_t)dw * (ROWB >> 4);
+                for (int kb = (p.kt - dt0) * p.CB; ok && kb > 0; --kb) {     // (dt, ci-block) stages
+                    if (!(ok = mbar_wait(&sh->full_a[sa], pa, sh, p, SITE_A_FULL))) break;
+#pragma unroll
+                    for (int g = 0; g < STAGES; ++g) {
+                        if (!(ok = mbar_wait(&sh->full_b[sb], pb, sh, p, SITE_B_FULL))) break;
+                        tc_fence_after();
+                        if (elect_one()) {
+#pragma unroll
+                            for (int u = 0; u < TPBC; ++u) {
+                                const int tap = g * TPBC + u;
+                                // tap (dh, dw) = a descriptor offset into the one halo tile.  The start address is only
+                                // 16-byte granular and need not sit on the swizzle period: the swizzle is a function of
+                                // the absolute shared-memory address (as the TMA unit applied it), so the descriptor's
+                                // base-offset field stays 0.
+                                const uint32_t a_lo = a_ring + (uint32_t)(tap / KS) * A_ROWSTEP + (uint32_t)(tap % KS) * (ROWB >> 4);
+                                const uint32_t b_lo = b_ring + (uint32_t)u * b_tapstep;
+#pragma unroll
+                                for (int j = 0; j < NBW; ++j) {
+#pragma unroll
+                                    for (int k = 0; k < KSTEPS; ++k)
+                                        tc_mma_bf16(d0 + j * p.NPAD, a_lo + j * ((8 * ROWB) >> 4) + 2 * k, a_hi, b_lo + 2 * k, b_hi,
+                                                    idesc, (tap == 0 && k == 0) ? accumulate : 1u);
                                 }
+                            }
+                            tc_commit(smem_u32(&sh->empty_b[sb]));
+                        }
+                        __syncwarp();
+                        b_ring += b_slotstep;
+                        if (++sb == p.SB) { sb = 0; pb ^= 1; b_ring = b_ring0; }
+                    }
+                    if (!ok) break;
+                    accumulate = 1;
+                    if (elect_one()) tc_commit(smem_u32(&sh->empty_a[sa]));
+                    __syncwarp();
+                    a_ring += a_slotstep;
+                    if (++sa == p.SA) { sa = 0; pa ^= 1; a_ring = a_ring0; }
+                }
+                if (!ok) break;
+                if (elect_one()) tc_commit(smem_u32(&sh->acc_full[acc]));
+                __syncwarp();
+                if (++acc == p.ACC) { acc = 0; pacc ^= 1; }
+            }
+        } else
+        for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+            const int t = (tile / p.NT) % p.T;
+            const int dt0 = (p.first_frame - t > 0) ? p.first_frame - t : 0;
+            if (!(ok = mbar_wait(&sh->acc_empty[acc], pacc, sh, p, SITE_ACC_EMPTY))) break;
+            tc_fence_after();
+            const uint32_t d0 = tmem_base + (uint32_t)(acc * NB + iss * NBW) * p.NPAD;
+            uint32_t accumulate = 0;
+            for (int dt = dt0; ok && dt < p.kt; ++dt)
+                for (int cb = 0; ok && cb < p.CB; ++cb) {
+                    uint32_t a_row = 0;  // descriptor low word of the halo row of the current tap row
+                    if (!p.per_tap_a) {
+                        if (!(ok = mbar_wait(&sh->full_a[sa], pa, sh, p, SITE_A_FULL))) break;
+                        a_row = make_desc_lo(smem_u32(ring_a + (size_t)sa * p.a_slot)) + a_blk;
+                    }
+                    for (int tp = 0, dw = 0; tp < spatial; tp += p.TPB) {
+                        if (!(ok = mbar_wait(&sh->full_b[sb], pb, sh, p, SITE_B_FULL))) break;
+                        tc_fence_after();
+                        uint32_t b_lo = make_desc_lo(smem_u32(ring_b + (size_t)sb * p.b_slot));
+                        for (int u = 0; u < p.TPB; ++u) {
+                            uint32_t a_lo;
+                            if (p.per_tap_a) {
+                                if (!(ok = mbar_wait(&sh->full_a[sa], pa, sh, p, SITE_A_FULL))) break;
+                                tc_fence_after();
+                                a_lo = make_desc_lo(smem_u32(ring_a + (size_t)sa * p.a_slot)) + a_blk;
+                            } else {
+                                // The start address is only 16-byte granular and need not sit on the swizzle
+                                // period: the swizzle is a function of the absolute shared-memory address (as
+                                // the TMA unit applied it), so the descriptor's base-offset field stays 0.
+                                a_lo = a_row + (uint32_t)dw * (ROWB >> 4);
+                            }
+                            if (elect_one()) {
 #pragma unroll
                                 for (int j = 0; j < NBW; ++j) {
 #pragma unroll
@@ -487,27 +559,31 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                                         tc_mma_bf16(d0 + j * p.NPAD, a_lo + j * ((8 * ROWB) >> 4) + 2 * k, a_hi, b_lo + 2 * k, b_hi,
                                                     idesc, (k == 0) ? accumulate : 1u);
                                 }
-                                accumulate = 1;
-                                b_lo += b_tapstep;
-                                if (p.per_tap_a) {
-                                    tc_commit(smem_u32(&sh->empty_a[sa]));
-                                    if (++sa == p.SA) { sa = 0; pa ^= 1; }
-                                }
-                                if (++dw == p.kw) { dw = 0; a_row += a_rowstep; }
+                                if (p.per_tap_a) tc_commit(smem_u32(&sh->empty_a[sa]));
                             }
-                            if (!ok) break;
-                            tc_commit(smem_u32(&sh->empty_b[sb]));
-                            if (++sb == p.SB) { sb = 0; pb ^= 1; }
+                            __syncwarp();
+                            accumulate = 1;
+                            b_lo += b_tapstep;
+                            if (p.per_tap_a) {
+                                if (++sa == p.SA) { sa = 0; pa ^= 1; }
+                            }
+                            if (++dw == p.kw) { dw = 0; a_row += a_rowstep; }
                         }
-                        if (ok && !p.per_tap_a) {
-                            tc_commit(smem_u32(&sh->empty_a[sa]));
-                            if (++sa == p.SA) { sa = 0; pa ^= 1; }
-                        }
+                        if (!ok) break;
+                        if (elect_one()) tc_commit(smem_u32(&sh->empty_b[sb]));
+                        __syncwarp();
+                        if (++sb == p.SB) { sb = 0; pb ^= 1; }
                     }
-                if (!ok) break;
-                tc_commit(smem_u32(&sh->acc_full[acc]));
-                if (++acc == p.ACC) { acc = 0; pacc ^= 1; }
-            }
+                    if (ok && !p.per_tap_a) {
+                        if (elect_one()) tc_commit(smem_u32(&sh->empty_a[sa]));
+                        __syncwarp();
+                        if (++sa == p.SA) { sa = 0; pa ^= 1; }
+                    }
+                }
+            if (!ok) break;
+            if (elect_one()) tc_commit(smem_u32(&sh->acc_full[acc]));
+            __syncwarp();
+            if (++acc == p.ACC) { acc = 0; pacc ^= 1; }
         }
     }
     // ---------------------------------------------------------------- epilogue (warps 4..7)
