@@ -52,6 +52,8 @@ def _load():
         lib.ccv3d_oracle_points.argtypes = [i, p, p, p, p] + [i] * 9 + [p, ctypes.c_int64, p]
         lib.ccv3d_oracle_points.restype = i
         lib.ccv3d_oracle_num_threads.restype = i
+        lib.ccv3d_oracle_cache_update.argtypes = [i, p, p] + [i] * 6 + [p]
+        lib.ccv3d_oracle_cache_update.restype = i
         _lib = lib
     return _lib
 
@@ -111,6 +113,21 @@ def points(x, cache, w, b, flat_idx):
     if rc != 0:
         raise ValueError("ccv3d_oracle_points rejected its arguments")
     return vals
+
+
+def cache_update(x, cache, kt: int):
+    """new_cache = last kt-1 frames of [cache ; x] (zeros where there is no history); storage dtype, bit copy."""
+    dt = _dtype_of(x)
+    x = np.ascontiguousarray(x)
+    N, Cin, T, H, W = x.shape
+    if cache is not None:
+        cache = np.ascontiguousarray(cache)
+        assert cache.shape == (N, Cin, kt - 1, H, W) and cache.dtype == x.dtype
+    nc = np.empty((N, Cin, kt - 1, H, W), dtype=x.dtype)
+    rc = _load().ccv3d_oracle_cache_update(dt, _ptr(x), _ptr(cache), N, Cin, T, H, W, kt, _ptr(nc))
+    if rc != 0:
+        raise ValueError("ccv3d_oracle_cache_update rejected its arguments")
+    return nc
 
 
 # --------------------------------------------------------------------------------------

@@ -165,6 +165,25 @@ int ccv3d_oracle_points(int dtype, const void* x, const void* cache, const void*
     return 0;
 }
 
+/* The cache update alone (the last kt-1 frames of Z = [cache ; x], bit copy), for problems whose full
+ * forward pass is too large to run on the CPU. */
+int ccv3d_oracle_cache_update(int dtype, const void* x, const void* cache, int N, int Cin, int T, int H, int W, int kt,
+                              void* new_cache) {
+    if (!x || !new_cache || kt < 2) return -1;
+    const int tc = kt - 1;
+    const int64_t HW = (int64_t)H * W;
+    const size_t fb = (size_t)HW * esize(dtype);
+    for (int n = 0; n < N; ++n)
+        for (int ci = 0; ci < Cin; ++ci)
+            for (int j = 0; j < tc; ++j) {
+                char* dst = (char*)new_cache + (size_t)(((int64_t)n * Cin + ci) * tc + j) * fb;
+                const char* zf = z_frame(x, cache, dtype, Cin, T, HW, kt, n, ci, T + j);
+                if (zf) memcpy(dst, zf, fb);
+                else memset(dst, 0, fb);
+            }
+    return 0;
+}
+
 int ccv3d_oracle_num_threads(void) {
 #ifdef _OPENMP
     extern int omp_get_max_threads(void);

@@ -17,7 +17,11 @@ bias: variance 0.1).
 """
 from __future__ import annotations
 
+import ctypes
 import math
+import os
+import subprocess
+
 import numpy as np
 
 F32 = 0
@@ -26,29 +30,31 @@ BF16 = 1
 # tensor ids (sub-streams); layer l of a chain uses id + 16*l
 TID_X, TID_CACHE, TID_W, TID_B = 1, 2, 3, 4
 
-_M1 = np.uint64(0xBF58476D1CE4E5B9)
-_M2 = np.uint64(0x94D049BB133111EB)
-_GOLD = np.uint64(0x9E3779B97F4A7C15)
-_CHUNK = 1 << 22
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "gen.c")
+_LIB = os.path.join(_HERE, "libsynth_inputs.so")
+_lib = None
 
 
-def _mix(z: np.ndarray) -> np.ndarray:
-    z = (z ^ (z >> np.uint64(30))) * _M1
-    z = (z ^ (z >> np.uint64(27))) * _M2
-    return z ^ (z >> np.uint64(31))
+def build(force: bool = False) -> str:
+    """Compile the generator (gcc, OpenMP, no fast-math); returns the library path."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        subprocess.run(["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-o", _LIB + ".tmp", _SRC, "-lm"],
+                       check=True)
+        os.replace(_LIB + ".tmp", _LIB)
+    return _LIB
 
 
-def _key(seed: int, tid: int, lane: int) -> np.uint64:
-    k = (seed * 0x632BE59BD9B4E019 + tid * 0xD1B54A32D192ED03 + lane * 0x8CB92BA72F3D8DD7 + 0x1234567) % (1 << 64)
-    return np.uint64(k)
-
-
-def _uniform01(seed: int, tid: int, lane: int, start: int, count: int) -> np.ndarray:
-    """count doubles in (0,1), element i at flat index start+i."""
-    with np.errstate(over="ignore"):
-        idx = np.arange(start, start + count, dtype=np.uint64)
-        z = _mix(_mix(idx * _GOLD + _key(seed, tid, lane)))
-    return ((z >> np.uint64(11)).astype(np.float64) + 0.5) * (1.0 / 9007199254740992.0)
+def _fill(shape, kind: int, a: float, b: float, dtype: int, seed: int, tid: int) -> np.ndarray:
+    global _lib
+    if _lib is None:
+        _lib = ctypes.CDLL(build())
+        _lib.synth_fill.argtypes = [ctypes.c_void_p, ctypes.c_int64, ctypes.c_int64, ctypes.c_int, ctypes.c_double,
+                                    ctypes.c_double, ctypes.c_int, ctypes.c_uint64, ctypes.c_uint64]
+        _lib.synth_fill.restype = None
+    out = np.empty(shape, dtype=np.uint16 if dtype == BF16 else np.float32)
+    _lib.synth_fill(out.ctypes.data_as(ctypes.c_void_p), 0, out.size, kind, a, b, dtype, seed, tid)
+    return out
 
 
 def to_bf16_bits(a32: np.ndarray) -> np.ndarray:
@@ -69,32 +75,13 @@ def to_f64(a: np.ndarray) -> np.ndarray:
     return a.astype(np.float64)
 
 
-def _store(vals64: np.ndarray, dtype: int) -> np.ndarray:
-    a32 = vals64.astype(np.float32)
-    return to_bf16_bits(a32) if dtype == BF16 else a32
-
-
 def uniform(shape, lo: float, hi: float, dtype: int, seed: int, tid: int) -> np.ndarray:
-    n = int(np.prod(shape))
-    out = np.empty(n, dtype=np.uint16 if dtype == BF16 else np.float32)
-    for s in range(0, n, _CHUNK):
-        c = min(_CHUNK, n - s)
-        u = _uniform01(seed, tid, 0, s, c)
-        out[s:s + c] = _store(lo + (hi - lo) * u, dtype)
-    return out.reshape(shape)
+    return _fill(shape, 0, lo, hi, dtype, seed, tid)
 
 
 def normal(shape, std: float, dtype: int, seed: int, tid: int) -> np.ndarray:
     """N(0, std^2) by Box-Muller on two independent hashed uniforms per element."""
-    n = int(np.prod(shape))
-    out = np.empty(n, dtype=np.uint16 if dtype == BF16 else np.float32)
-    for s in range(0, n, _CHUNK):
-        c = min(_CHUNK, n - s)
-        u1 = _uniform01(seed, tid, 0, s, c)
-        u2 = _uniform01(seed, tid, 1, s, c)
-        z = np.sqrt(-2.0 * np.log(u1)) * np.cos((2.0 * math.pi) * u2)
-        out[s:s + c] = _store(std * z, dtype)
-    return out.reshape(shape)
+    return _fill(shape, 1, std, 0.0, dtype, seed, tid)
 
 
 def zeros(shape, dtype: int) -> np.ndarray:

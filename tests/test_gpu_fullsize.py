@@ -1,0 +1,67 @@
+"""GPU parity at the benchmark's full sizes, in the launch configuration bench.py times: the outputs are too
+many for the CPU oracle to compute whole, so it evaluates sampled output elements one dot product at a time
+(random samples plus the corners and seams of the kernel's 16 x 16-pixel tiles); the cache update is compared
+whole, bit for bit."""
+import numpy as np
+import pytest
+
+import oracle
+import synth_inputs as si
+from _util import bits, to_dev
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+
+def _sample_indices(shape, n_random, seed):
+    N, C, T, H, W = shape
+    rng = np.random.default_rng(seed)
+    idx = [rng.integers(0, int(np.prod(shape)), size=n_random, dtype=np.int64)]
+    hs = sorted({0, 1, 15, 16, 17, H // 2, H - 17, H - 16, H - 1} & set(range(H)))
+    ws = sorted({0, 1, 7, 8, 15, 16, 17, W // 2, W - 9, W - 8, W - 1} & set(range(W)))
+    cs = sorted({0, 1, 31, 32, C // 2, C - 1} & set(range(C)))
+    g = np.stack(np.meshgrid(np.arange(N), cs, np.arange(T), hs, ws, indexing="ij"), axis=-1).reshape(-1, 5)
+    idx.append(np.ravel_multi_index(g.T, shape).astype(np.int64))
+    return np.unique(np.concatenate(idx))
+
+
+@pytest.mark.parametrize("name,cache", [
+    ("cfg3_bf16_192", "random"),
+    ("cfg3_bf16_192", None),              # the first-chunk form of configuration 3
+    ("cfg4a_bf16_96", "random"),
+    ("cfg4b_bf16_192_96", "random"),
+    ("cfg4c_bf16_pw_192_96", None),
+])
+def test_full_size_sampled(name, cache):
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import paper_2609_31938_b200 as ccv
+    torch.cuda.set_device(0)
+    cfg = dict(si.CONFIGS[name])
+    c = si.conv_case(cache=cache, **cfg)
+    kt = c["k"][0]
+    layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]))
+    x, cch = to_dev(c["x"]), to_dev(c["cache"])
+    out, nc = layer(x, cch)
+    torch.cuda.synchronize()
+    assert layer.device_status()[0] == ccv.OK
+    ctr = layer.counters()
+    assert ctr["ok"] == 1 and ctr["tcgen05_bf16"] == 1
+
+    idx = _sample_indices(tuple(out.shape), 3000, seed=1)
+    got = out.view(-1)[torch.from_numpy(idx).cuda()].float().cpu().numpy().astype(np.float64)
+    ref = oracle.points(c["x"], c["cache"], c["w"], c["b"], idx)
+    rms = float(np.sqrt(np.mean(ref ** 2)))
+    err = np.abs(got - ref)
+    assert np.isfinite(got).all()
+    assert err.max() <= 2e-2 * rms, (err.max() / rms, idx[np.argmax(err)])
+    assert err.mean() <= 2e-3 * rms, err.mean() / rms
+    # nothing left unwritten anywhere (the output buffer came from torch.empty): finite everywhere, and its
+    # overall RMS is that of the sampled oracle values
+    assert bool(torch.isfinite(out).all())
+    assert abs(float(out.float().pow(2).mean().sqrt()) / rms - 1.0) < 0.05
+    if kt > 1:
+        assert np.array_equal(bits(nc), oracle.cache_update(c["x"], c["cache"], kt)), "cache update is not bit-exact"
+    layer.close()
+    del out, nc, x, cch
+    torch.cuda.empty_cache()

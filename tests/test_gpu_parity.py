@@ -1,0 +1,258 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle on
+the same seeded inputs, element by element.  Tolerances, relative to
+RMS(oracle out): FP32 max <= 1e-4; BF16 (FP32 accumulate) max <= 2e-2 and
+mean <= 2e-3; the cache update is bit-exact."""
+import numpy as np
+import pytest
+
+import oracle
+import synth_inputs as si
+from _util import as_f64, bits, check, metrics, to_dev
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+GUARD = 64  # elements of guard band on each side of out / new_cache
+
+
+@pytest.fixture(scope="module")
+def ccv():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import paper_2609_31938_b200 as m
+    torch.cuda.set_device(0)
+    return m
+
+
+def _guarded(shape, dtype):
+    """A poison-filled buffer with guard bands; returns (whole buffer, view of the payload)."""
+    n = int(np.prod(shape))
+    buf = torch.full((n + 2 * GUARD,), float("nan"), dtype=dtype, device="cuda:0")
+    return buf, buf[GUARD:GUARD + n].view(shape)
+
+
+def _guards_intact(buf):
+    return bool(torch.isnan(buf[:GUARD]).all() and torch.isnan(buf[-GUARD:]).all())
+
+
+def run_case(ccv, c, flags=0, out_dtype=None, kind=None):
+    """One forward call with poison-filled, guarded outputs; full comparison with the oracle."""
+    ref, ref_nc = oracle.forward(c["x"], c["cache"], c["w"], c["b"])
+    layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), flags=flags, out_dtype=out_dtype)
+    x, cache = to_dev(c["x"]), to_dev(c["cache"])
+    N, Cin, T, H, W = c["x"].shape
+    tc = c["k"][0] - 1
+    odt = torch.float32 if (c["dtype"] == si.F32 or out_dtype == ccv.F32) else torch.bfloat16
+    obuf, out = _guarded(ref.shape, odt)
+    nbuf, nc = (_guarded((N, Cin, tc, H, W), x.dtype) if tc else (None, None))
+    layer(x, cache, out=out, new_cache=nc)
+    torch.cuda.synchronize()
+    st, detail = layer.device_status()
+    assert st == ccv.OK, (ccv.status_string(st), hex(detail))
+    assert _guards_intact(obuf) and (nbuf is None or _guards_intact(nbuf)), "guard band overwritten"
+    if kind is None:
+        kind = "f32" if c["dtype"] == si.F32 else ("bf16_f32out" if out_dtype == ccv.F32 else "bf16")
+    m = check(as_f64(out), ref, kind)                       # NaN poison left behind fails the non-finite check
+    if tc:
+        assert np.array_equal(bits(nc), ref_nc), "cache update is not bit-exact"
+    ctr = layer.counters()
+    assert ctr["calls"] == ctr["ok"] == 1 and ctr["unsupported"] == ctr["invalid"] == ctr["cuda_error"] == 0
+    layer.close()
+    return m, ctr
+
+
+# ---------------------------------------------------------------------------- FP32 (plain FMA kernel)
+def test_cfg1_fp32(ccv):
+    m, ctr = run_case(ccv, si.conv_case(**si.CONFIGS["cfg1_f32_16"]))
+    assert ctr["simt"] == 1 and m["cos"] > 0.9999999
+
+
+@pytest.mark.parametrize("N,Cin,Cout,T,H,W,k,cache", [
+    (2, 3, 5, 3, 7, 9, (3, 3, 3), "random"),
+    (1, 16, 16, 1, 5, 13, (3, 3, 3), None),
+    (1, 7, 9, 2, 4, 6, (1, 1, 1), None),
+    (1, 4, 4, 4, 3, 5, (3, 1, 1), "zeros"),
+    (1, 5, 3, 2, 6, 7, (1, 3, 3), None),
+    (1, 6, 10, 3, 8, 8, (2, 3, 3), "random"),
+])
+def test_fp32_shapes(ccv, N, Cin, Cout, T, H, W, k, cache):
+    run_case(ccv, si.conv_case(N, Cin, Cout, T, H, W, k=k, dtype=si.F32, cache=cache, seed=3))
+
+
+# ---------------------------------------------------------------------------- BF16, plain FMA route
+@pytest.mark.parametrize("N,Cin,Cout,T,H,W,k,cache", [
+    (1, 16, 16, 2, 8, 8, (3, 3, 3), "random"),
+    (2, 24, 40, 1, 5, 11, (3, 3, 3), None),
+    (1, 32, 8, 3, 6, 6, (1, 1, 1), None),
+])
+def test_bf16_fma_route(ccv, N, Cin, Cout, T, H, W, k, cache):
+    m, ctr = run_case(ccv, si.conv_case(N, Cin, Cout, T, H, W, k=k, cache=cache, seed=4), flags=ccv.FLAG_FORCE_SIMT)
+    assert ctr["simt"] == 1 and ctr["tcgen05_bf16"] == 0
+
+
+# ---------------------------------------------------------------------------- BF16, tensor-core route
+TC_CASES = [
+    # N, Cin, Cout, T, H,  W,  k,         cache,    bias
+    (1, 64, 64, 2, 16, 16, (3, 3, 3), "random", True),     # exactly one tile
+    (1, 64, 64, 1, 1, 8, (3, 3, 3), "random", True),       # a single image row, T < kt-1
+    (1, 16, 16, 3, 3, 24, (3, 3, 3), "zeros", True),       # Cin below one K block (zero-padded channels)
+    (1, 48, 96, 2, 8, 72, (3, 3, 3), "random", False),     # Cin = 32 + 16, no bias
+    (1, 96, 96, 4, 44, 80, (3, 3, 3), "random", True),     # 64-byte swizzle route, ragged tile rows
+    (1, 96, 192, 5, 20, 24, (3, 3, 3), None, True),        # first chunk, T > kt-1
+    (2, 192, 192, 2, 17, 40, (3, 3, 3), "random", True),   # batch 2, H = tile + 1
+    (1, 192, 384, 1, 16, 16, (3, 3, 3), "random", True),   # two output-channel tiles
+    (1, 64, 80, 2, 16, 32, (3, 3, 3), "random", True),     # Cout % 32 == 16: 16-channel epilogue chunks
+    (1, 64, 100, 2, 9, 16, (3, 3, 3), "random", True),     # Cout not a multiple of 16
+    (1, 64, 300, 1, 8, 8, (3, 3, 3), None, True),          # two padded output-channel tiles
+    (1, 128, 64, 3, 24, 13, (3, 3, 3), "random", True),    # W % 8 != 0: scalar staging, direct-store epilogue
+    (1, 64, 64, 2, 5, 7, (3, 3, 3), None, False),          # everything smaller than a tile, odd W
+    (1, 192, 96, 2, 32, 48, (1, 1, 1), None, True),        # 1x1x1: per-pixel matmul, no cache
+    (2, 96, 96, 3, 10, 16, (1, 1, 1), None, True),
+    (1, 64, 64, 4, 12, 16, (3, 1, 1), "random", True),     # temporal-only kernel
+    (1, 64, 64, 2, 18, 24, (1, 3, 3), None, True),         # spatial-only kernel
+    (1, 64, 32, 3, 16, 16, (2, 3, 3), "random", True),     # even temporal extent: one cache frame
+    (1, 32, 48, 2, 20, 40, (3, 5, 5), "random", True),     # 5x5 spatial: run-time tap loop
+    (1, 64, 64, 2, 16, 24, (3, 3, 1), "random", True),     # kh != kw
+]
+
+
+@pytest.mark.parametrize("N,Cin,Cout,T,H,W,k,cache,bias", TC_CASES)
+def test_bf16_tensor_core_route(ccv, N, Cin, Cout, T, H, W, k, cache, bias):
+    m, ctr = run_case(ccv, si.conv_case(N, Cin, Cout, T, H, W, k=k, cache=cache, bias=bias, seed=5))
+    assert ctr["tcgen05_bf16"] == 1 and ctr["simt"] == 0
+
+
+@pytest.mark.parametrize("N,Cin,Cout,T,H,W,k,cache,bias", [TC_CASES[0], TC_CASES[4], TC_CASES[6], TC_CASES[11]])
+def test_bf16_tensor_core_fp32_output(ccv, N, Cin, Cout, T, H, W, k, cache, bias):
+    # FP32 output exposes the accumulation itself: FP32 accumulate over K is ~1e-5 x RMS
+    run_case(ccv, si.conv_case(N, Cin, Cout, T, H, W, k=k, cache=cache, bias=bias, seed=6), out_dtype=ccv.F32)
+
+
+@pytest.mark.parametrize("N,Cin,Cout,T,H,W,k,cache,bias", [TC_CASES[0], TC_CASES[4], TC_CASES[7], TC_CASES[18]])
+def test_bf16_tensor_core_per_tap_loads(ccv, N, Cin, Cout, T, H, W, k, cache, bias):
+    run_case(ccv, si.conv_case(N, Cin, Cout, T, H, W, k=k, cache=cache, bias=bias, seed=7), flags=ccv.FLAG_TC_PER_TAP_A)
+
+
+def test_cfg2_bf16_384(ccv):
+    m, ctr = run_case(ccv, si.conv_case(**si.CONFIGS["cfg2_bf16_384"]))
+    assert ctr["tcgen05_bf16"] == 1 and m["cos"] > 0.99998
+
+
+# ---------------------------------------------------------------------------- exact cases
+def test_delta_and_ones_kernels_are_exact_in_bf16(ccv):
+    N, Cin, Cout, T, H, W = 1, 64, 64, 3, 20, 24
+    c = si.conv_case(N, Cin, Cout, T, H, W, seed=8)
+    # small integers: every product and partial sum is exact in FP32 and the result is exact in BF16
+    rng = np.random.default_rng(0)
+    xi = rng.integers(-3, 4, size=c["x"].shape).astype(np.float32)
+    ci = rng.integers(-3, 4, size=c["cache"].shape).astype(np.float32)
+    for kind in ("delta", "ones"):
+        w = np.zeros((Cout, Cin, 3, 3, 3), np.float32)
+        if kind == "delta":
+            for co in range(Cout):
+                w[co, (co * 7) % Cin, co % 3, (co // 3) % 3, (co // 9) % 3] = 1.0
+        else:
+            w[:, :2] = 1.0                                   # 54 ones per output channel: |sum| <= 162
+        b = rng.integers(-2, 3, size=(Cout,)).astype(np.float32)
+        cc = dict(c, x=si.to_bf16_bits(xi), cache=si.to_bf16_bits(ci), w=si.to_bf16_bits(w), b=si.to_bf16_bits(b))
+        ref, _ = oracle.forward(cc["x"], cc["cache"], cc["w"], cc["b"])
+        layer = ccv.CausalConv3d(to_dev(cc["w"]), to_dev(cc["b"]))
+        out, _ = layer(to_dev(cc["x"]), to_dev(cc["cache"]))
+        torch.cuda.synchronize()
+        assert np.array_equal(as_f64(out), ref), kind
+        layer.close()
+
+
+def test_null_cache_equals_zero_cache_bitwise(ccv):
+    c = si.conv_case(1, 96, 96, 3, 24, 32, cache="zeros", seed=9)
+    layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]))
+    x = to_dev(c["x"])
+    o0, n0 = layer(x, to_dev(c["cache"]))
+    o1, n1 = layer(x, None)
+    torch.cuda.synchronize()
+    assert torch.equal(o0, o1) and torch.equal(n0, n1)
+    x1 = x[:, :, :1].contiguous()                           # T < kt-1 with no history: a zero frame stays in front
+    _, n2 = layer(x1, None)
+    torch.cuda.synchronize()
+    assert np.array_equal(bits(n2), oracle.cache_update(np.ascontiguousarray(c["x"][:, :, :1]), None, 3))
+    layer.close()
+
+
+@pytest.mark.parametrize("chunks", [[1] * 6, [4, 2], [2, 1, 3]])
+def test_streaming_equivalence_on_gpu(ccv, chunks):
+    """Chunked calls with the cache carried equal one whole-sequence call from an empty history: bit-identical on
+    the GPU too (the K order of an output element does not depend on the chunking), and within tolerance of the
+    oracle's whole-sequence run."""
+    c = si.conv_case(1, 96, 64, 6, 20, 24, cache=None, seed=10)
+    layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]))
+    x = to_dev(c["x"])
+    whole, whole_nc = layer(x, None)
+    cache, outs, pos = None, [], 0
+    for n in chunks:
+        o, cache = layer(x[:, :, pos:pos + n].contiguous(), cache)
+        outs.append(o)
+        pos += n
+    torch.cuda.synchronize()
+    assert torch.equal(torch.cat(outs, dim=2), whole) and torch.equal(cache, whole_nc)
+    ref, ref_nc = oracle.forward(c["x"], None, c["w"], c["b"])
+    check(as_f64(whole), ref, "bf16")
+    assert np.array_equal(bits(cache), ref_nc)
+    layer.close()
+
+
+# ---------------------------------------------------------------------------- argument checks on a live handle
+def test_forward_argument_errors_and_counters(ccv):
+    c = si.conv_case(1, 64, 64, 2, 16, 16, seed=11)
+    layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]))
+    x, cache = to_dev(c["x"]), to_dev(c["cache"])
+    out = torch.empty((1, 64, 2, 16, 16), dtype=torch.bfloat16, device="cuda:0")
+    nc = torch.empty_like(cache)
+    h = layer.h
+    f = lambda *a: ccv.ccv3d_forward(h, *a)
+    assert f(x.data_ptr(), cache.data_ptr(), x.data_ptr(), nc.data_ptr(), 1, 2, 16, 16) == ccv.ERR_ALIAS       # out is x
+    assert f(x.data_ptr(), cache.data_ptr(), out.data_ptr(), cache.data_ptr(), 1, 2, 16, 16) == ccv.ERR_ALIAS  # in-place cache
+    assert f(x.data_ptr(), cache.data_ptr(), out.data_ptr(), out.data_ptr(), 1, 2, 16, 16) == ccv.ERR_ALIAS
+    assert f(x.data_ptr() + 2, cache.data_ptr(), out.data_ptr(), nc.data_ptr(), 1, 2, 16, 16) == ccv.ERR_ALIGNMENT
+    assert f(None, cache.data_ptr(), out.data_ptr(), nc.data_ptr(), 1, 2, 16, 16) == ccv.ERR_INVALID_ARG
+    assert f(x.data_ptr(), cache.data_ptr(), out.data_ptr(), nc.data_ptr(), 1, 0, 16, 16) == ccv.ERR_INVALID_ARG
+    assert f(x.data_ptr(), cache.data_ptr(), out.data_ptr(), nc.data_ptr(), 1, 2, 16, 16) == ccv.OK
+    torch.cuda.synchronize()
+    ctr = layer.counters()
+    assert ctr["calls"] == 7 and ctr["ok"] == 1 and ctr["invalid"] == 6 and ctr["tcgen05_bf16"] == 1
+    assert layer.device_status()[0] == ccv.OK
+    s, ws = ccv.ccv3d_workspace_bytes(h, 1, 2, 16, 16)
+    assert s == ccv.OK and ws == 4 * 64 * 16 * 16 * 2
+    layer.close()
+
+
+def test_host_entry_point_matches_device_entry_point(ccv):
+    c = si.conv_case(1, 64, 96, 3, 24, 40, seed=12)
+    layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]))
+    out_d, nc_d = layer(to_dev(c["x"]), to_dev(c["cache"]))
+    torch.cuda.synchronize()
+    out_h = np.empty((1, 96, 3, 24, 40), np.uint16)
+    nc_h = np.empty_like(c["cache"])
+    s = ccv.ccv3d_forward_host(layer.h, c["x"].ctypes.data, c["cache"].ctypes.data, out_h.ctypes.data,
+                               nc_h.ctypes.data, 1, 3, 24, 40, torch.cuda.current_stream().cuda_stream)
+    assert s == ccv.OK
+    assert np.array_equal(out_h, bits(out_d)) and np.array_equal(nc_h, bits(nc_d))
+    ref, ref_nc = oracle.forward(c["x"], c["cache"], c["w"], c["b"])
+    check(si.to_f64(out_h), ref, "bf16")
+    assert np.array_equal(nc_h, ref_nc)
+    layer.close()
+
+
+def test_chain_glue_kernels(ccv):
+    rng = np.random.default_rng(1)
+    a = si.to_bf16_bits(rng.standard_normal((2, 3, 2, 5, 6)).astype(np.float32))
+    b = si.to_bf16_bits(rng.standard_normal((2, 3, 2, 5, 6)).astype(np.float32))
+    da, db = to_dev(a), to_dev(b)
+    y = torch.empty_like(da)
+    assert ccv.ccv3d_add_bf16(da.data_ptr(), db.data_ptr(), y.data_ptr(), da.numel()) == ccv.OK
+    exp = si.to_bf16_bits((si.bf16_bits_to_f32(a) + si.bf16_bits_to_f32(b)).astype(np.float32))
+    assert np.array_equal(bits(y), exp)
+    up = torch.empty((2, 3, 6, 10, 12), dtype=torch.bfloat16, device="cuda:0")
+    assert ccv.ccv3d_upsample_bf16(da.data_ptr(), up.data_ptr(), 2, 3, 2, 5, 6, 3) == ccv.OK
+    torch.cuda.synchronize()
+    exp_up = np.repeat(np.repeat(np.repeat(a, 3, axis=2), 2, axis=3), 2, axis=4)
+    assert np.array_equal(bits(up), exp_up)

@@ -138,6 +138,9 @@ def test_streaming_equivalence(chunks, dtype):
     assert np.array_equal(np.concatenate(outs, axis=2), whole)      # bit-identical
     assert np.array_equal(cache, whole_nc)
     assert np.array_equal(cache, x[:, :, -2:])                      # the last kt-1 input frames
+    assert np.array_equal(oracle.cache_update(x, None, 3), x[:, :, -2:])
+    c1 = oracle.cache_update(np.ascontiguousarray(x[:, :, :1]), None, 3)
+    assert np.array_equal(oracle.cache_update(np.ascontiguousarray(x[:, :, 1:2]), c1, 3), x[:, :, :2])
 
 
 def test_linearity_in_x_and_w():
