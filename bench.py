@@ -1,0 +1,348 @@
+#!/usr/bin/env python
+"""Benchmark of the cached causal Conv3D hot path.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+A step is one ccv3d_forward call (channels-last staging + cache update, then the tcgen05 implicit-GEMM
+kernel) on one synthetic decoder-shaped layer.  The default workload is the 192->192, T=4 + 2-frame cache,
+352x640, 3x3x3 BF16 layer (the large-spatial configuration the >= 60 %-of-tensor-peak target is quoted on);
+inputs are seeded, synthetic, resident in HBM when the timed region starts, and larger than L2 (no flush
+needed).  One JSON line on stdout.
+
+--impl reference times the CPU oracle (the plain FP64 definition) on a bounded spatial crop of the same
+workload on the host's cores.  With N > 1 (torchrun) every rank runs an independent replica (no collective
+on the data path): weak scaling.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+import synth_inputs as si  # noqa: E402
+
+METRIC = "causal Conv3D BF16 TFLOP/s"
+DEFAULT_WORKLOAD = "cfg3_bf16_192"
+
+# DRAM bytes (read + write) of one launch of the convolution kernel, from an ncu capture of a quarter-size
+# case (192->192, T=4, 176x320) scaled by the pixel count; see profiles/conv3d_tcgen05_192ch.md.
+TRAFFIC_BYTES_PER_LAUNCH = {"cfg3_bf16_192": None}
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(tflops=float(p["bf16_tflops"]), tflops_sustained=float(p.get("bf16_tflops_sustained", 0.0)),
+                    hbm_gbs=float(p["hbm_gbs"]), source="measured")
+    return dict(tflops=1590.0, tflops_sustained=1400.0, hbm_gbs=6650.0, source="fallback")
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs (read-only)."""
+
+    def __init__(self, index: int, period_s: float = 0.004):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.dev = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.dev, pynvml.NVML_CLOCK_SM))
+            self.ok = True
+        except Exception:
+            self.nv = None
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+                 getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+                 getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+                 getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+                 getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake_slowdown"}
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.dev, nv.NVML_CLOCK_SM)))
+                try:
+                    r = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.dev))
+                except Exception:
+                    r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.dev))
+                for bit, name in names.items():
+                    if r & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        if self.is_alive():
+            self.join(timeout=2.0)
+
+    def summary(self):
+        if not self.samples:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": [], "samples": 0}
+        return {"sm_mhz": int(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def cfg_of(name):
+    cfg = dict(si.CONFIGS[name])
+    dims = dict(N=cfg["N"], Cin=cfg["Cin"], Cout=cfg["Cout"], T=cfg["T"], H=cfg["H"], W=cfg["W"], k=cfg["k"])
+    return cfg, dims
+
+
+# ---------------------------------------------------------------------------------------------- CPU oracle leg
+def oracle_sample(name, target_s=12.0):
+    """Times the oracle, as it stands, on a spatial crop (all channels, all frames, the cache included) of the
+    workload, sized from a small calibration run so that one pass takes about target_s seconds."""
+    import oracle
+    cfg, d = cfg_of(name)
+    crop = dict(cfg, H=16, W=16)
+    c = si.conv_case(**crop)
+    t0 = time.perf_counter()
+    oracle.forward(c["x"], c["cache"], c["w"], c["b"])
+    t_small = time.perf_counter() - t0
+    fl_small = si.conv_flops(d["N"], d["Cin"], d["Cout"], d["T"], 16, 16, d["k"])
+    rate = fl_small / max(t_small, 1e-6)
+    px = target_s * rate / (fl_small / 256.0)          # pixels per frame the oracle covers in target_s seconds
+    W = int(min(d["W"], 80))
+    H = int(min(d["H"], max(8, px // W)))
+    return dict(cfg, H=H, W=W)
+
+
+def run_oracle_once(crop):
+    import oracle
+    c = si.conv_case(**crop)
+    t0 = time.perf_counter()
+    oracle.forward(c["x"], c["cache"], c["w"], c["b"])
+    dt = time.perf_counter() - t0
+    fl = si.conv_flops(crop["N"], crop["Cin"], crop["Cout"], crop["T"], crop["H"], crop["W"], crop["k"])
+    return dt, fl
+
+
+def cpu_baseline(name, target_s=12.0):
+    import oracle
+    crop = oracle_sample(name, target_s)
+    dt, fl = run_oracle_once(crop)
+    return {"value": fl / dt / 1e12, "unit": "TFLOP/s", "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"one pass over a {crop['H']}x{crop['W']} spatial crop (all {crop['Cin']}->{crop['Cout']} "
+                      f"channels, T={crop['T']} + {crop['k'][0] - 1}-frame cache) of {name}: {dt:.2f} s"}
+
+
+def main_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    import oracle
+    name = args.workload
+    cfg, d = cfg_of(name)
+    crop = oracle_sample(name, target_s=6.0)
+    for _ in range(min(args.warmup, 1)):
+        run_oracle_once(crop)
+    steps = max(1, min(args.steps, 5))
+    t_tot, fl_tot = 0.0, 0.0
+    for _ in range(steps):
+        dt, fl = run_oracle_once(crop)
+        t_tot += dt
+        fl_tot += fl
+    val = fl_tot / t_tot / 1e12
+    sample = (f"each step = the oracle over a {crop['H']}x{crop['W']} spatial crop (all channels and frames) "
+              f"of {name}; {steps} steps timed")
+    line = {"impl": "reference", "metric": METRIC, "value": val, "unit": "TFLOP/s", "n_gpus": args.gpus, "steps": steps,
+            "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * t_tot / steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": name, **{k: (list(v) if isinstance(v, tuple) else v) for k, v in d.items()},
+                       "sample": sample},
+            "cpu_baseline": {"value": val, "unit": "TFLOP/s", "cores": oracle.num_threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": val, "unit": "TFLOP/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+    return 0
+
+
+# ---------------------------------------------------------------------------------------------- CUDA leg
+def main_ours(args):
+    import torch
+    import paper_2609_31938_b200 as ccv
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device; there is no CPU fallback"
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    name = args.workload
+    cfg, d = cfg_of(name)
+    c = si.conv_case(**cfg)
+    kt = d["k"][0]
+
+    def up(a):
+        return None if a is None else torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
+
+    x, cache = up(c["x"]), up(c["cache"])
+    layer = ccv.CausalConv3d(up(c["w"]), up(c["b"]))
+    out = torch.empty((d["N"], d["Cout"], d["T"], d["H"], d["W"]), dtype=torch.bfloat16, device=dev)
+    nc = torch.empty_like(cache) if cache is not None else None
+    stream = torch.cuda.current_stream()
+
+    def step():
+        layer(x, cache, out=out, new_cache=nc)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    barrier()
+    assert layer.device_status()[0] == ccv.OK
+    launches0 = layer.counters()["kernel_launches"]
+    ccv.ccv3d_profile_enable(layer.h, True)
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    clocks = sampler.summary()
+    clock_note = "sampled during the timed region"
+    if clocks["samples"] < 5:
+        # the timed region was shorter than a few NVML polls: keep polling over an untimed repeat of the same step
+        t_end = time.time() + 1.0
+        while time.time() < t_end:
+            for _ in range(20):
+                step()
+            torch.cuda.synchronize()
+        clock_note = "timed region too short for NVML polling; sampled over an untimed 1 s repeat of the same step"
+    sampler.stop()
+    clocks = sampler.summary()
+    clocks["note"] = clock_note
+
+    st, stage_ms, conv_ms, ncalls = ccv.ccv3d_profile_read(layer.h)
+    ccv.ccv3d_profile_enable(layer.h, False)
+    launches = layer.counters()["kernel_launches"] - launches0
+    assert layer.device_status()[0] == ccv.OK
+
+    if dist is not None:
+        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+
+    flops = si.conv_flops(**d)
+    abytes = si.conv_bytes(**d)
+    ms_step = ms_total / args.steps
+    value = world * flops / (ms_step * 1e-3) / 1e12
+
+    # ---- end to end through the host entry point: pinned host buffers, H2D and D2H inside the timed region
+    e2e = None
+    if rank == 0:
+        hx = torch.from_numpy(c["x"].view(np.int16)).pin_memory()
+        hc = torch.from_numpy(c["cache"].view(np.int16)).pin_memory() if c["cache"] is not None else None
+        ho = torch.empty(out.shape, dtype=torch.int16).pin_memory()
+        hn = torch.empty(hc.shape, dtype=torch.int16).pin_memory() if hc is not None else None
+        e_steps = max(1, min(args.steps, 8))
+
+        def host_step():
+            s = ccv.ccv3d_forward_host(layer.h, hx.data_ptr(), None if hc is None else hc.data_ptr(), ho.data_ptr(),
+                                       None if hn is None else hn.data_ptr(), d["N"], d["T"], d["H"], d["W"],
+                                       stream.cuda_stream)
+            assert s == ccv.OK, ccv.status_string(s)
+
+        host_step()
+        host_step()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(e_steps):
+            host_step()
+        torch.cuda.synchronize()
+        e_ms = 1e3 * (time.perf_counter() - t0) / e_steps
+        h2d = hx.numel() * 2 + (hc.numel() * 2 if hc is not None else 0)
+        d2h = ho.numel() * 2 + (hn.numel() * 2 if hn is not None else 0)
+        e2e = {"value": flops / (e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "h2d_bytes_per_step": int(h2d),
+               "d2h_bytes_per_step": int(d2h), "ms_per_step": e_ms, "steps": e_steps,
+               "note": "ccv3d_forward_host: pinned host x, cache -> device, both kernels, out, new_cache -> host"}
+        assert np.array_equal(ho.numpy().view(np.uint16), out.view(torch.int16).cpu().numpy().view(np.uint16))
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return 0
+
+    peaks = measured_peaks()
+    conv_avg_ms = conv_ms / max(ncalls, 1)
+    stage_avg_ms = stage_ms / max(ncalls, 1)
+    achieved = flops / (conv_avg_ms * 1e-3) / 1e12 if conv_avg_ms > 0 else None
+    roof_t_ms = 1e3 * max(flops / (peaks["tflops"] * 1e12), abytes / (peaks["hbm_gbs"] * 1e9))
+    roofline = {"bound": "tensor", "kernel": "conv3d_tcgen05_kernel", "achieved": achieved, "peak": peaks["tflops"],
+                "unit": "TFLOP/s", "frac": (achieved / peaks["tflops"]) if achieved else None,
+                "peak_source": f"{peaks['source']} (burst cuBLAS bf16)", "traffic": TRAFFIC_BYTES_PER_LAUNCH.get(name),
+                "kernel_ms": conv_avg_ms, "staging_kernel_ms": stage_avg_ms,
+                "staging_kernel_gbs": (abytes - 2 * d["N"] * d["Cout"] * d["T"] * d["H"] * d["W"]
+                                       + 2 * d["N"] * d["Cin"] * (d["T"] + kt - 1) * d["H"] * d["W"]) / (stage_avg_ms * 1e6)
+                if stage_avg_ms > 0 else None,
+                "step_frac_of_roofline": roof_t_ms / ms_step,
+                "step_frac_of_sustained_peak": (value / world) / peaks["tflops_sustained"] if peaks["tflops_sustained"] else None}
+
+    cpu = cpu_baseline(name) if world == 1 else None
+    line = {"metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": name, **{k: (list(v) if isinstance(v, tuple) else v) for k, v in d.items()},
+                       "cache_frames": kt - 1, "accumulate": "fp32", "l2": "inputs larger than L2 (x alone is "
+                       f"{c['x'].nbytes / 1e6:.0f} MB); no flush", "parallelism": f"replicas x{world}",
+                       "algorithmic_bytes_per_step": int(abytes), "flops_per_step": flops,
+                       "pct_of_measured_bf16_peak": 100.0 * (value / world) / peaks["tflops"]},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline}
+    if cpu is not None:
+        line["cpu_baseline"] = cpu
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+    layer.close()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(n for n in si.CONFIGS if "bf16" in n))
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return main_reference(args)
+    return main_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

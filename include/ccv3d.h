@@ -143,6 +143,17 @@ ccv3d_status ccv3d_get_counters(const ccv3d_handle* h, ccv3d_counters* out_host)
  */
 ccv3d_status ccv3d_device_status(ccv3d_handle* h, uint32_t* detail_host);
 
+/*
+ * Optional per-kernel timing for benchmarks.  While enabled, every ccv3d_forward records CUDA events on the
+ * caller's stream before the staging kernel, between the two kernels and after the convolution kernel (up to
+ * 1024 calls are kept; later calls overwrite the oldest).  ccv3d_profile_read must be called after the stream
+ * has been synchronised; it returns the summed device time of the staging (or FP32-FMA route: zero) and of the
+ * convolution kernel over the calls recorded since the last read, and their number, then clears the record.
+ * All three outputs are HOST pointers.
+ */
+ccv3d_status ccv3d_profile_enable(ccv3d_handle* h, int32_t enable);
+ccv3d_status ccv3d_profile_read(ccv3d_handle* h, double* stage_ms_host, double* conv_ms_host, int64_t* calls_host);
+
 /* Static, human-readable name of a status code. */
 const char* ccv3d_status_string(ccv3d_status s);
 

@@ -39,7 +39,7 @@ class Counters(ctypes.Structure):
 
 EXPORTS = ("ccv3d_create", "ccv3d_forward", "ccv3d_forward_host", "ccv3d_workspace_bytes", "ccv3d_destroy",
            "ccv3d_get_counters", "ccv3d_device_status", "ccv3d_status_string", "ccv3d_add_bf16",
-           "ccv3d_upsample_bf16")
+           "ccv3d_upsample_bf16", "ccv3d_profile_enable", "ccv3d_profile_read")
 
 
 def _load() -> ctypes.CDLL:
@@ -58,6 +58,9 @@ def _load() -> ctypes.CDLL:
     lib.ccv3d_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
     lib.ccv3d_status_string.argtypes = [ctypes.c_int]
     lib.ccv3d_status_string.restype = ctypes.c_char_p
+    lib.ccv3d_profile_enable.argtypes = [vp, i32]
+    lib.ccv3d_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double),
+                                       ctypes.POINTER(ctypes.c_int64)]
     lib.ccv3d_add_bf16.argtypes = [vp, vp, vp, ctypes.c_int64, vp]
     lib.ccv3d_upsample_bf16.argtypes = [vp, vp, i32, i32, i32, i32, i32, i32, vp]
     for name in EXPORTS:
@@ -132,6 +135,17 @@ def ccv3d_device_status(h):
     d = ctypes.c_uint32()
     s = lib.ccv3d_device_status(h, ctypes.byref(d))
     return s, d.value
+
+
+def ccv3d_profile_enable(h, enable: bool) -> int:
+    return lib.ccv3d_profile_enable(h, 1 if enable else 0)
+
+
+def ccv3d_profile_read(h):
+    """(status, staging-kernel ms, convolution-kernel ms, calls) summed since the last read; sync the stream first."""
+    a, b, n = ctypes.c_double(), ctypes.c_double(), ctypes.c_int64()
+    s = lib.ccv3d_profile_read(h, ctypes.byref(a), ctypes.byref(b), ctypes.byref(n))
+    return s, a.value, b.value, n.value
 
 
 def ccv3d_add_bf16(a, b, y, n, stream=0) -> int:

@@ -23,6 +23,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+constexpr int PROF_SLOTS = 1024;
 constexpr size_t SMEM_LIMIT = 232448;  // 227 KB of dynamic shared memory per CTA on sm_100
 
 struct TcPlan {      // per-layer choices of the tensor-core route
@@ -59,6 +60,10 @@ struct ccv3d_handle {
     ShapeKey tm_a_key;
     CUtensorMap tm_o;
     long long wait_limit_clk;
+    // optional per-kernel timing
+    int prof_on;
+    int64_t prof_n;
+    cudaEvent_t* prof_ev;   // PROF_SLOTS x 3 events, created on first enable
     ccv3d_counters ctr;
 };
 
@@ -203,6 +208,8 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     sp.new_cache = tc ? (__nv_bfloat16*)new_cache : nullptr;
     sp.N = N; sp.Cin = d.cin; sp.T = T; sp.H = H; sp.W = W; sp.tc = tc; sp.CB = pl.CB;
     sp.f_begin = sp.cache ? 0 : (tc < T ? tc : T);
+    cudaEvent_t* pev = (h->prof_on && h->prof_ev) ? h->prof_ev + 3 * (h->prof_n % PROF_SLOTS) : nullptr;
+    if (pev) cudaEventRecord(pev[0], st);
     const bool vec = (W % 8 == 0);
     dim3 sgrid((W + STG_PX - 1) / STG_PX, H, (unsigned)(N * (F - sp.f_begin) * pl.CB));
     if (sgrid.y > 65535 || sgrid.z > 65535) return CCV3D_ERR_UNSUPPORTED;
@@ -215,6 +222,8 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     }
     if (cudaGetLastError() != cudaSuccess) return cuda_fail();
     h->ctr.kernel_launches++;
+
+    if (pev) cudaEventRecord(pev[1], st);
 
     // ---- implicit GEMM ----
     const int per_tap = (d.flags & CCV3D_FLAG_TC_PER_TAP_A) ? 1 : 0;
@@ -292,6 +301,10 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     else CCV3D_LAUNCH(32);
 #undef CCV3D_LAUNCH
     if (s == CCV3D_OK) h->ctr.tcgen05_bf16++;
+    if (pev) {
+        cudaEventRecord(pev[2], st);
+        h->prof_n++;
+    }
     return s;
 }
 
@@ -306,12 +319,18 @@ ccv3d_status forward_simt(ccv3d_handle* h, const void* x, const void* cache, voi
     const int64_t gx = (npix + SIMT_THREADS - 1) / SIMT_THREADS;
     if (gx > 0x7FFFFFFF) return CCV3D_ERR_UNSUPPORTED;
     dim3 grid((unsigned)gx, (d.cout + SIMT_CO - 1) / SIMT_CO);
+    cudaEvent_t* pev = (h->prof_on && h->prof_ev) ? h->prof_ev + 3 * (h->prof_n % PROF_SLOTS) : nullptr;
+    if (pev) { cudaEventRecord(pev[0], st); cudaEventRecord(pev[1], st); }
     if (d.dtype == CCV3D_F32) conv3d_direct_kernel<float, float><<<grid, SIMT_THREADS, 0, st>>>(p);
     else if (d.out_dtype == CCV3D_BF16) conv3d_direct_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, SIMT_THREADS, 0, st>>>(p);
     else conv3d_direct_kernel<__nv_bfloat16, float><<<grid, SIMT_THREADS, 0, st>>>(p);
     if (cudaGetLastError() != cudaSuccess) return cuda_fail();
     h->ctr.kernel_launches++;
     h->ctr.simt++;
+    if (pev) {
+        cudaEventRecord(pev[2], st);
+        h->prof_n++;
+    }
 
     if (tc && new_cache) {
         const uint64_t fbytes = (uint64_t)H * W * esize(d.dtype);
@@ -459,6 +478,10 @@ ccv3d_status ccv3d_destroy(ccv3d_handle* h) {
     void* bufs[] = {h->w_copy, h->wp, h->bias32, h->status, h->workspace, h->hx, h->hc, h->ho, h->hn};
     for (void* b : bufs)
         if (b) cudaFree(b);
+    if (h->prof_ev) {
+        for (int i = 0; i < 3 * PROF_SLOTS; ++i) cudaEventDestroy(h->prof_ev[i]);
+        delete[] h->prof_ev;
+    }
     cudaGetLastError();
     delete h;
     return CCV3D_OK;
@@ -510,6 +533,43 @@ ccv3d_status ccv3d_forward_host(ccv3d_handle* h, const void* x_host, const void*
     if (has_n && cudaMemcpyAsync(new_cache_host, h->hn, cb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return cuda_fail();
     if (cudaStreamSynchronize(st) != cudaSuccess) return cuda_fail();
     return ccv3d_device_status(h, nullptr);
+}
+
+ccv3d_status ccv3d_profile_enable(ccv3d_handle* h, int32_t enable) {
+    if (!h) return CCV3D_ERR_INVALID_ARG;
+    if (enable && !h->prof_ev) {
+        h->prof_ev = new (std::nothrow) cudaEvent_t[3 * PROF_SLOTS];
+        if (!h->prof_ev) return CCV3D_ERR_NOMEM;
+        for (int i = 0; i < 3 * PROF_SLOTS; ++i)
+            if (cudaEventCreate(&h->prof_ev[i]) != cudaSuccess) {
+                for (int j = 0; j < i; ++j) cudaEventDestroy(h->prof_ev[j]);
+                delete[] h->prof_ev;
+                h->prof_ev = nullptr;
+                return cuda_fail();
+            }
+    }
+    h->prof_on = enable ? 1 : 0;
+    h->prof_n = 0;
+    return CCV3D_OK;
+}
+
+ccv3d_status ccv3d_profile_read(ccv3d_handle* h, double* stage_ms_host, double* conv_ms_host, int64_t* calls_host) {
+    if (!h || !stage_ms_host || !conv_ms_host || !calls_host) return CCV3D_ERR_INVALID_ARG;
+    double a = 0.0, b = 0.0;
+    const int64_t n = h->prof_n < PROF_SLOTS ? h->prof_n : PROF_SLOTS;
+    for (int64_t i = 0; i < n && h->prof_ev; ++i) {
+        float t0 = 0.f, t1 = 0.f;
+        if (cudaEventElapsedTime(&t0, h->prof_ev[3 * i], h->prof_ev[3 * i + 1]) != cudaSuccess ||
+            cudaEventElapsedTime(&t1, h->prof_ev[3 * i + 1], h->prof_ev[3 * i + 2]) != cudaSuccess)
+            return cuda_fail();
+        a += t0;
+        b += t1;
+    }
+    *stage_ms_host = a;
+    *conv_ms_host = b;
+    *calls_host = n;
+    h->prof_n = 0;
+    return CCV3D_OK;
 }
 
 ccv3d_status ccv3d_get_counters(const ccv3d_handle* h, ccv3d_counters* out_host) {
