@@ -1,0 +1,45 @@
+"""Run a few forward calls of one layer shape on cuda:0 - a small, self-ending program to put under a profiler.
+
+    python -m paper_2609_31938_b200.profile_case --cin 192 --cout 192 --t 4 --h 176 --w 320 [--k 3 3 3] [--calls 3]
+
+Inputs are the seeded synthetic tensors of the benchmark (normal activations, fan-in-scaled weights).
+"""
+import argparse
+import os
+import sys
+
+import numpy as np
+
+sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+
+
+def main():
+    import torch
+    import synth_inputs as si
+    import paper_2609_31938_b200 as ccv
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--cin", type=int, default=192)
+    ap.add_argument("--cout", type=int, default=192)
+    ap.add_argument("--t", type=int, default=4)
+    ap.add_argument("--h", type=int, default=176)
+    ap.add_argument("--w", type=int, default=320)
+    ap.add_argument("--k", type=int, nargs=3, default=[3, 3, 3])
+    ap.add_argument("--calls", type=int, default=3)
+    ap.add_argument("--no-cache", action="store_true")
+    a = ap.parse_args()
+    c = si.conv_case(1, a.cin, a.cout, a.t, a.h, a.w, k=tuple(a.k), cache=None if a.no_cache else "random")
+    up = lambda v: None if v is None else torch.from_numpy(v.view(np.int16)).cuda().view(torch.bfloat16)
+    layer = ccv.CausalConv3d(up(c["w"]), up(c["b"]))
+    x, cache = up(c["x"]), up(c["cache"])
+    out = torch.empty((1, a.cout, a.t, a.h, a.w), dtype=torch.bfloat16, device="cuda")
+    nc = torch.empty_like(cache) if cache is not None else None
+    for _ in range(a.calls):
+        layer(x, cache, out=out, new_cache=nc)
+    torch.cuda.synchronize()
+    st, detail = layer.device_status()
+    assert st == ccv.OK, (ccv.status_string(st), hex(detail))
+    print("ok", layer.counters())
+
+
+if __name__ == "__main__":
+    main()
