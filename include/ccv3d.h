@@ -116,6 +116,33 @@ ccv3d_status ccv3d_forward(ccv3d_handle* h, const void* x, const void* cache, vo
                            int32_t N, int32_t T, int32_t H, int32_t W, void* stream);
 
 /*
+ * ccv3d_forward without any allocation.  (The paper has no counterpart: its route runs inside a framework
+ * that allocates freely.)
+ *
+ * Who needs it: code that must not, or cannot, call the device allocator when it runs the layer - a real-time
+ * loop that may not block on cudaMalloc, a callback running where allocation is forbidden, an embedding
+ * runtime that owns all device memory and hands this library none.  ccv3d_forward keeps its channels-last
+ * staging copy in a workspace it allocates on demand; this entry point keeps it instead in a fixed 32 MiB
+ * array that is part of the library's device image, so it calls neither cudaMalloc nor cudaFree nor any other
+ * allocating routine.  Every GPU whose context loads the library holds those 32 MiB until the process exits.
+ *
+ * Same arguments, meaning, aliasing and alignment rules as ccv3d_forward (x, cache, out, new_cache are DEVICE
+ * pointers owned by the caller).  Differences:
+ *   - BF16 tensor-core layers only (a handle created with CCV3D_FLAG_FORCE_SIMT or with FP32 data, and the
+ *     CCV3D_FLAG_TC_PER_TAP_A mode, return CCV3D_ERR_UNSUPPORTED);
+ *   - the staging copy, ccv3d_workspace_bytes(h, N, T, H, W), must fit the 32 MiB array, otherwise the call
+ *     returns CCV3D_ERR_UNSUPPORTED and launches nothing;
+ *   - the first call on each device looks up the array's device address (a one-time set-up with that device
+ *     current); make that first call outside any stream capture;
+ *   - all handles and all calls on one GPU share the one array.  Calls that may overlap on the GPU (different
+ *     streams, no ordering between them) race on it and corrupt each other's results: order them.  The array
+ *     keeps the previous call's bytes; each call overwrites everything it later reads, so stale contents are
+ *     never consumed and nothing has to be cleared.
+ */
+ccv3d_status ccv3d_forward_static(ccv3d_handle* h, const void* x, const void* cache, void* out, void* new_cache,
+                                  int32_t N, int32_t T, int32_t H, int32_t W, void* stream);
+
+/*
  * The same call on HOST buffers (same shapes and meaning as above): copies x
  * and cache to device staging owned by the handle, runs ccv3d_forward, copies
  * out and new_cache back, and returns after the stream has completed.  Pinned

@@ -308,6 +308,161 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     return s;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Allocation-free variant of the tensor-core route (ccv3d_forward_static).  Its channels-last staging copy
+// lives in a fixed array in device memory that is part of the loaded library image, so the call needs no
+// allocator.  Everything below is separate from forward_tc: it has its own tensor maps and launch helper.
+// ------------------------------------------------------------------------------------------------
+constexpr uint64_t STATIC_SCRATCH_BYTES = 32ull << 20;   // 32 MiB per GPU that loads the library, until exit
+static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_BYTES];
+constexpr int MAX_DEVICES = 64;
+static void* g_static_scratch_addr[MAX_DEVICES];         // device address of the array, per device; set on first use
+
+// In host code the name g_static_scratch is only a stand-in for the symbol: the address a kernel can use has
+// to be asked for, once per device, with that device current.
+ccv3d_status static_scratch_for_current_device(void** out_ptr) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return cuda_fail();
+    if (dev < 0 || dev >= MAX_DEVICES) return CCV3D_ERR_UNSUPPORTED;
+    if (!g_static_scratch_addr[dev]) {
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return cuda_fail();
+        g_static_scratch_addr[dev] = ptr;
+    }
+    *out_ptr = g_static_scratch_addr[dev];
+    return CCV3D_OK;
+}
+
+template <int KB, int NB, int KS, int TPBC>
+ccv3d_status launch_tc_with_maps(ccv3d_handle* h, const CUtensorMap& tm_a, const CUtensorMap& tm_o, const TcParams& p,
+                                 size_t smem, int grid, cudaStream_t st) {
+    auto kern = conv3d_tcgen05_kernel<KB, NB, KS, TPBC>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return cuda_fail();
+    kern<<<grid, TC_THREADS, smem, st>>>(tm_a, tm_o, p);
+    if (cudaGetLastError() != cudaSuccess) return cuda_fail();
+    h->ctr.kernel_launches++;
+    return CCV3D_OK;
+}
+
+ccv3d_status forward_tc_static(ccv3d_handle* h, const void* x, const void* cache, void* out, void* new_cache, int N,
+                               int T, int H, int W, cudaStream_t st) {
+    const ccv3d_desc& d = h->d;
+    const TcPlan& pl = h->plan;
+    const int tc = d.kt - 1;
+    const int F = tc + T;
+    if (d.flags & CCV3D_FLAG_TC_PER_TAP_A) return CCV3D_ERR_UNSUPPORTED;
+    if (tc_workspace_bytes(h, N, T, H, W) > STATIC_SCRATCH_BYTES) return CCV3D_ERR_UNSUPPORTED;
+    void* scratch = nullptr;
+    ccv3d_status s = static_scratch_for_current_device(&scratch);
+    if (s != CCV3D_OK) return s;
+
+    // staging pass: it overwrites every byte of the scratch that the convolution kernel will read (padded
+    // channels included), so nothing of an earlier call's contents is ever consumed and nothing needs clearing
+    StageParams sp;
+    sp.x = (const __nv_bfloat16*)x;
+    sp.cache = tc ? (const __nv_bfloat16*)cache : nullptr;
+    sp.zs = (__nv_bfloat16*)scratch;
+    sp.new_cache = tc ? (__nv_bfloat16*)new_cache : nullptr;
+    sp.N = N; sp.Cin = d.cin; sp.T = T; sp.H = H; sp.W = W; sp.tc = tc; sp.CB = pl.CB;
+    sp.f_begin = sp.cache ? 0 : (tc < T ? tc : T);
+    const bool vec = (W % 8 == 0);
+    dim3 sgrid((W + STG_PX - 1) / STG_PX, H, (unsigned)(N * (F - sp.f_begin) * pl.CB));
+    if (sgrid.y > 65535 || sgrid.z > 65535) return CCV3D_ERR_UNSUPPORTED;
+    if (pl.KB == 64) {
+        if (vec) stage_frames_kernel<64, true><<<sgrid, 256, 0, st>>>(sp);
+        else stage_frames_kernel<64, false><<<sgrid, 256, 0, st>>>(sp);
+    } else {
+        if (vec) stage_frames_kernel<32, true><<<sgrid, 128, 0, st>>>(sp);
+        else stage_frames_kernel<32, false><<<sgrid, 128, 0, st>>>(sp);
+    }
+    if (cudaGetLastError() != cudaSuccess) return cuda_fail();
+    h->ctr.kernel_launches++;
+
+    const int NB = pl.NB, TW = 8 * NB, BW = TW + d.kw - 1, BH = 16 + d.kh - 1;
+    CUtensorMap tm_a, tm_o;
+    {
+        const uint64_t rowb = (uint64_t)pl.KB * 2;
+        cuuint64_t dims[5] = {(cuuint64_t)pl.KB, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)pl.CB, (cuuint64_t)N * F};
+        cuuint64_t strides[4] = {rowb, rowb * W, rowb * W * H, rowb * W * H * pl.CB};
+        cuuint32_t box[5] = {(cuuint32_t)pl.KB, (cuuint32_t)BW, (cuuint32_t)BH, 1, 1};
+        cuuint32_t es[5] = {1, 1, 1, 1, 1};
+        if (h->encode(&tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, scratch, dims, strides, box, es,
+                      CU_TENSOR_MAP_INTERLEAVE_NONE,
+                      pl.KB == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
+                      CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return CCV3D_ERR_CUDA;
+    }
+    TcParams p;
+    memset(&p, 0, sizeof(p));
+    p.N = N; p.T = T; p.H = H; p.W = W; p.Cout = d.cout; p.F = F;
+    p.kt = d.kt; p.kh = d.kh; p.kw = d.kw;
+    p.CB = pl.CB; p.NT = pl.NT; p.NPAD = pl.NPAD;
+    p.tiles_h = (H + 15) / 16;
+    p.tiles_w = (W + TW - 1) / TW;
+    const int64_t total = (int64_t)N * p.tiles_h * p.tiles_w * T * pl.NT;
+    if (total > 0x7FFFFFFF) return CCV3D_ERR_UNSUPPORTED;
+    p.total_tiles = (int)total;
+    p.first_frame = (tc && !cache) ? tc : 0;
+    p.out_f32 = d.out_dtype == CCV3D_F32;
+    p.per_tap_a = 0;
+    p.ACC = pl.ACC;
+    p.a_slot = (uint32_t)align_up((uint64_t)BW * BH * pl.KB * 2, 1024);
+    p.b_tap = (uint32_t)pl.NPAD * pl.KB * 2;
+    p.epi_tma = (!p.out_f32 && W % 8 == 0) ? 1 : 0;
+    p.ECH = (pl.NPAD % 32 == 0) ? 32 : 16;
+    p.e_slot = p.epi_tma ? (uint32_t)(p.ECH * 16 * TW * 2) : 0;
+    const size_t fixed = 1024 + align_up(sizeof(TcShared), 128) + 2 * (size_t)p.e_slot;
+    const size_t budget = SMEM_LIMIT - fixed;
+    p.TPB = ((size_t)p.b_tap * d.kw <= 40960) ? d.kw : 1;
+    int SA = 2;
+    for (;;) {
+        p.b_slot = (uint32_t)align_up((uint64_t)p.b_tap * p.TPB, 1024);
+        if ((size_t)SA * p.a_slot + 3 * (size_t)p.b_slot <= budget) break;
+        if (p.TPB > 1) { p.TPB = 1; continue; }
+        if ((size_t)SA * p.a_slot + 2 * (size_t)p.b_slot <= budget) break;
+        return CCV3D_ERR_UNSUPPORTED;
+    }
+    int SB = (int)((budget - (size_t)SA * p.a_slot) / p.b_slot);
+    if (SB > 8) SB = 8;
+    while (SA < 4 && (size_t)(SA + 1) * p.a_slot + (size_t)SB * p.b_slot <= budget) ++SA;
+    p.SA = SA; p.SB = SB;
+    p.tmem_cols = pow2_cols((uint32_t)(NB * pl.NPAD * pl.ACC));
+    if (p.tmem_cols > 512) return CCV3D_ERR_UNSUPPORTED;
+    p.wait_limit_clk = h->wait_limit_clk;
+    p.bias = h->bias32;
+    p.wq = (const uint8_t*)h->wp;
+    p.out = out;
+    p.status = h->status;
+    if (p.epi_tma) {
+        cuuint64_t dims[5] = {(cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)T, (cuuint64_t)d.cout, (cuuint64_t)N};
+        cuuint64_t strides[4] = {2ull * W, 2ull * W * H, 2ull * W * H * T, 2ull * W * H * T * d.cout};
+        cuuint32_t box[5] = {(cuuint32_t)TW, 16, 1, (cuuint32_t)p.ECH, 1};
+        cuuint32_t es[5] = {1, 1, 1, 1, 1};
+        if (h->encode(&tm_o, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, out, dims, strides, box, es,
+                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return CCV3D_ERR_CUDA;
+    } else {
+        tm_o = tm_a;   // never dereferenced on this path
+    }
+    const size_t smem = fixed + (size_t)SA * p.a_slot + (size_t)SB * p.b_slot;
+    const int grid = p.total_tiles < h->sm_count ? p.total_tiles : h->sm_count;
+    const int ks = (d.kh == d.kw && (d.kh == 1 || d.kh == 3)) ? d.kh : 0;
+#define CCV3D_LAUNCH_STATIC(KBv)                                                                              \
+    do {                                                                                                      \
+        if (ks == 3 && p.TPB == 3) s = launch_tc_with_maps<KBv, 2, 3, 3>(h, tm_a, tm_o, p, smem, grid, st);   \
+        else if (ks == 3 && p.TPB == 1) s = launch_tc_with_maps<KBv, 2, 3, 1>(h, tm_a, tm_o, p, smem, grid, st); \
+        else if (ks == 1) s = launch_tc_with_maps<KBv, 2, 1, 1>(h, tm_a, tm_o, p, smem, grid, st);            \
+        else s = launch_tc_with_maps<KBv, 2, 0, 0>(h, tm_a, tm_o, p, smem, grid, st);                         \
+    } while (0)
+    if (pl.KB == 64) CCV3D_LAUNCH_STATIC(64);
+    else CCV3D_LAUNCH_STATIC(32);
+#undef CCV3D_LAUNCH_STATIC
+    if (s == CCV3D_OK) h->ctr.tcgen05_bf16++;
+    return s;
+}
+
 ccv3d_status forward_simt(ccv3d_handle* h, const void* x, const void* cache, void* out, void* new_cache, int N, int T,
                           int H, int W, cudaStream_t st) {
     const ccv3d_desc& d = h->d;
@@ -504,6 +659,16 @@ ccv3d_status ccv3d_forward(ccv3d_handle* h, const void* x, const void* cache, vo
     if (h->use_tc) s = forward_tc(h, x, cache, out, new_cache, N, T, H, W, st);
     else s = forward_simt(h, x, cache, out, new_cache, N, T, H, W, st);
     return count(h, s);
+}
+
+ccv3d_status ccv3d_forward_static(ccv3d_handle* h, const void* x, const void* cache, void* out, void* new_cache,
+                                  int32_t N, int32_t T, int32_t H, int32_t W, void* stream) {
+    if (!h) return CCV3D_ERR_INVALID_ARG;
+    h->ctr.calls++;
+    ccv3d_status s = check_forward_args(h, x, cache, out, new_cache, N, T, H, W, true);
+    if (s != CCV3D_OK) return count(h, s);
+    if (!h->use_tc) return count(h, CCV3D_ERR_UNSUPPORTED);   // the FP32-FMA route has no scratch to replace
+    return count(h, forward_tc_static(h, x, cache, out, new_cache, N, T, H, W, (cudaStream_t)stream));
 }
 
 ccv3d_status ccv3d_forward_host(ccv3d_handle* h, const void* x_host, const void* cache_host, void* out_host,
