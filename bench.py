@@ -180,6 +180,45 @@ def main_reference(args):
 
 
 # ---------------------------------------------------------------------------------------------- CUDA leg
+def chain_leg(dev):
+    """Streamed synthetic decoder chain (configuration 5): 21 one-latent-frame chunks through six cached 3x3x3
+    convolutions (384 ch @ 44x80 T=1, 192 ch @ 88x160 T=4, 96 ch @ 176x320 T=4), two 1x1x1 transitions, residual
+    adds and upsampling, caches carried per layer.  Returns ms per output frame (84 frames)."""
+    import math
+    import torch
+    from paper_2609_31938_b200.chain import DecoderChain, LAYERS
+    shapes = {"A1": (384, 384, 3), "A2": (384, 384, 3), "PA": (192, 384, 1), "B1": (192, 192, 3), "B2": (192, 192, 3),
+              "PB": (96, 192, 1), "C1": (96, 96, 3), "C2": (96, 96, 3)}
+    up = lambda a: torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
+    w, b = {}, {}
+    for i, n in enumerate(LAYERS):
+        co, ci, k = shapes[n]
+        w[n] = up(si.normal((co, ci, k, k, k), 1.0 / math.sqrt(ci * k ** 3), si.BF16, 0, si.TID_W + 16 * (i + 1)))
+        b[n] = up(si.normal((co,), math.sqrt(0.1), si.BF16, 0, si.TID_B + 16 * (i + 1)))
+    u = up(si.normal((1, 384, 21, 44, 80), 1.0, si.BF16, 0, si.TID_X))
+    chunks = [u[:, :, i:i + 1].contiguous() for i in range(21)]
+    ch = DecoderChain(w, b)
+    for c in chunks[:3]:
+        ch.step(c)
+    ch.reset()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for c in chunks:
+        ch.step(c)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    launches = sum(l.counters()["kernel_launches"] for l in ch.layers.values())
+    flops = 21 * (2 * si.conv_flops(1, 384, 384, 1, 44, 80, (3, 3, 3)) + si.conv_flops(1, 384, 192, 1, 44, 80, (1, 1, 1))
+                  + 2 * si.conv_flops(1, 192, 192, 4, 88, 160, (3, 3, 3)) + si.conv_flops(1, 192, 96, 4, 88, 160, (1, 1, 1))
+                  + 2 * si.conv_flops(1, 96, 96, 4, 176, 320, (3, 3, 3)))
+    ch.close()
+    return {"workload": "cfg5 streamed decoder chain, 21 chunks -> 84 frames of 96x176x320", "ms_total": ms,
+            "ms_per_chunk": ms / 21, "ms_per_output_frame": ms / 84, "tflops": flops / (ms * 1e-3) / 1e12,
+            "conv_kernel_launches": int(launches)}
+
+
 def main_ours(args):
     import torch
     import paper_2609_31938_b200 as ccv
@@ -314,6 +353,7 @@ def main_ours(args):
                 "step_frac_of_sustained_peak": (value / world) / peaks["tflops_sustained"] if peaks["tflops_sustained"] else None}
 
     cpu = cpu_baseline(name) if world == 1 else None
+    chain = chain_leg(dev) if (world == 1 and not args.no_chain) else None
     line = {"metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
@@ -325,6 +365,8 @@ def main_ours(args):
             "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline}
     if cpu is not None:
         line["cpu_baseline"] = cpu
+    if chain is not None:
+        line["decoder_chain"] = chain
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
@@ -338,6 +380,7 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-chain", action="store_true", help="skip the decoder-chain leg")
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(n for n in si.CONFIGS if "bf16" in n))
     args = ap.parse_args()
     if args.impl == "reference":

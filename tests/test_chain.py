@@ -1,0 +1,136 @@
+"""The streamed synthetic decoder chain: 3x3x3 cached causal convolutions at three resolutions with residual
+adds, 1x1x1 transitions and nearest-neighbour upsampling, caches carried per layer across chunks.
+
+CPU: the chain oracle satisfies streaming equivalence exactly (chunked = whole sequence, bit for bit).
+GPU: the library's chain equals its own whole-sequence run bit for bit, and matches the oracle's whole-sequence
+run within the BF16 tolerances (reduced spatial size so that the oracle finishes in seconds); at the full size
+of the benchmark configuration (21 latent frames of 44x80) the bit-for-bit streaming property is checked."""
+import math
+
+import numpy as np
+import pytest
+
+import synth_inputs as si
+from oracle.chain import ChainOracle, LAYERS, _bf16_to_f64, _f64_to_bf16_bits
+
+
+def make_chain_params(ca, cb, cc, seed=0):
+    shapes = {"A1": (ca, ca, 3), "A2": (ca, ca, 3), "PA": (cb, ca, 1), "B1": (cb, cb, 3), "B2": (cb, cb, 3),
+              "PB": (cc, cb, 1), "C1": (cc, cc, 3), "C2": (cc, cc, 3)}
+    w, b = {}, {}
+    for i, n in enumerate(LAYERS):
+        co, ci, k = shapes[n]
+        w[n] = si.normal((co, ci, k, k, k), 1.0 / math.sqrt(ci * k ** 3), si.BF16, seed, si.TID_W + 16 * (i + 1))
+        b[n] = si.normal((co,), math.sqrt(0.1), si.BF16, seed, si.TID_B + 16 * (i + 1))
+    return w, b
+
+
+def test_rounding_helper_is_nearest_even():
+    t = np.array([1.00390625, 1.01171875, -1.00390625, 1 + 2 ** -8 + 2 ** -40, 1 + 2 ** -8 - 2 ** -40, 255.5, 0.0])
+    assert _bf16_to_f64(_f64_to_bf16_bits(t)).tolist() == [1.0, 1.015625, -1.0, 1.0078125, 1.0, 256.0, 0.0]
+    rng = np.random.default_rng(0)
+    a = rng.standard_normal(200000) * 3
+    v = _bf16_to_f64(_f64_to_bf16_bits(a))
+    assert np.all(np.abs(v - a) <= np.abs(a) * 2.0 ** -8)
+
+
+@pytest.mark.parametrize("chunks", [[1, 1, 1, 1], [2, 1, 1], [3, 1]])
+def test_chain_oracle_streaming_equivalence(chunks):
+    w, b = make_chain_params(8, 6, 4, seed=1)
+    u = si.normal((1, 8, sum(chunks), 3, 4), 1.0, si.BF16, 1, si.TID_X)
+    whole = ChainOracle(w, b).step(u)
+    co, outs, pos = ChainOracle(w, b), [], 0
+    for n in chunks:
+        outs.append(co.step(np.ascontiguousarray(u[:, :, pos:pos + n])))
+        pos += n
+    assert whole.shape == (1, 4, 4 * sum(chunks), 12, 16)
+    assert np.array_equal(np.concatenate(outs, axis=2), whole)
+
+
+# ------------------------------------------------------------------------------------------------ GPU
+def _gpu_chain(w, b):
+    import torch
+    from _util import to_dev
+    from paper_2609_31938_b200.chain import DecoderChain
+    return DecoderChain({n: to_dev(w[n]) for n in LAYERS}, {n: to_dev(b[n]) for n in LAYERS})
+
+
+@pytest.mark.gpu
+def test_chain_gpu_vs_oracle_reduced_size():
+    torch = pytest.importorskip("torch")
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from _util import as_f64, bits, metrics, to_dev
+    torch.cuda.set_device(0)
+    w, b = make_chain_params(384, 192, 96, seed=0)
+    frames, H, W = 5, 6, 8
+    u = si.normal((1, 384, frames, H, W), 1.0, si.BF16, 0, si.TID_X)
+    ref = ChainOracle(w, b).step(u)                               # oracle, whole sequence, zero history
+    ch = _gpu_chain(w, b)
+    ud = to_dev(u)
+    outs = [ch.step(ud[:, :, i:i + 1].contiguous()) for i in range(frames)]
+    chunked = torch.cat(outs, dim=2)
+    ch.reset()
+    whole = ch.step(ud)
+    torch.cuda.synchronize()
+    for l in ch.layers.values():
+        assert l.device_status()[0] == 0
+    assert torch.equal(chunked, whole)                            # streaming equivalence on the GPU, bit for bit
+    # End to end, both sides round to BF16 at 11 points (8 convolutions, 3 adds).  A GPU accumulation that differs
+    # from FP64 in its last FP32 bits flips a few roundings per layer (0.4 % of the elements), every flipped
+    # element perturbs ~10^4 outputs of the next layer by ~1 % of a BF16 step and flips some of those, so after a
+    # few layers the two chains carry independent rounding noise: the difference is that of 2 x 11 independent
+    # roundings of unit gain, mean <= sqrt(22) x 1.13e-3 = 5.3e-3 x RMS.  Hence the end-to-end bounds below; the
+    # tight, layer-by-layer comparison follows.
+    m = metrics(as_f64(chunked), _bf16_to_f64(ref))
+    assert m["nonfinite"] == 0 and m["mean"] <= 6e-3 and m["max"] <= 1e-1 and m["cos"] > 0.9999, m
+
+    # Layer by layer on identical inputs: replay every convolution call of the oracle's chunked run (its input,
+    # its incoming cache) through the GPU layer.  Outputs may differ from the oracle's BF16 output only by such
+    # rounding flips: at most one BF16 step, on at most 2 % of the elements; the cache update is bit-exact.
+    trace = []
+    co = ChainOracle(w, b, trace=trace)
+    for i in range(frames):
+        co.step(np.ascontiguousarray(u[:, :, i:i + 1]))
+    assert len(trace) == 8 * frames
+    for (name, x, cache_in, out_ref, nc_ref) in trace:
+        out, nc = ch.layers[name](to_dev(x), to_dev(cache_in))
+        torch.cuda.synchronize()
+        got = bits(out)
+        diff = got != out_ref
+        assert diff.mean() <= 0.02, (name, diff.mean())
+        r64, g64 = _bf16_to_f64(out_ref), _bf16_to_f64(got)
+        rms = float(np.sqrt(np.mean(r64 ** 2)))
+        # one BF16 step of the value (2^-7 relative covers the step on either side of a binade), plus the FP32
+        # accumulation error for values near zero, where a step is smaller than that error
+        assert np.all(np.abs(g64 - r64) <= 2.0 ** -7 * np.abs(r64) + 1e-4 * rms), name
+        if nc_ref is not None:
+            assert np.array_equal(bits(nc), nc_ref), name
+    ch.close()
+
+
+@pytest.mark.gpu
+def test_chain_gpu_streaming_full_size():
+    torch = pytest.importorskip("torch")
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from _util import to_dev
+    torch.cuda.set_device(0)
+    w, b = make_chain_params(384, 192, 96, seed=0)
+    frames, H, W = 21, 44, 80
+    ud = to_dev(si.normal((1, 384, frames, H, W), 1.0, si.BF16, 0, si.TID_X))
+    ch = _gpu_chain(w, b)
+    outs = [ch.step(ud[:, :, i:i + 1].contiguous()) for i in range(frames)]
+    chunked = torch.cat(outs, dim=2)
+    assert chunked.shape == (1, 96, 84, 176, 320)
+    del outs
+    ch.reset()
+    whole = ch.step(ud)
+    torch.cuda.synchronize()
+    for l in ch.layers.values():
+        assert l.device_status()[0] == 0
+        c = l.counters()
+        assert c["calls"] == c["ok"] == frames + 1 and c["tcgen05_bf16"] == frames + 1
+    assert torch.equal(chunked, whole)
+    assert bool(torch.isfinite(whole).all())
+    ch.close()
