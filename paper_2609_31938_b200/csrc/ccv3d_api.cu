@@ -308,6 +308,84 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     return s;
 }
 
+// 1x1x1 layers whose weights fit in shared memory stream straight from NCTHW (no staging copy).
+bool pointwise_eligible(const ccv3d_handle* h, int T, int H, int W) {
+    const ccv3d_desc& d = h->d;
+    const TcPlan& pl = h->plan;
+    if (!(d.kt == 1 && d.kh == 1 && d.kw == 1)) return false;
+    if (d.flags & CCV3D_FLAG_TC_PER_TAP_A) return false;
+    if (pl.KB != 64 || pl.NT != 1 || d.out_dtype != CCV3D_BF16) return false;
+    if (((int64_t)T * H * W) % 8 != 0) return false;                       // TMA strides are multiples of 16 bytes
+    return (uint64_t)pl.CB * pl.NPAD * 128 <= 98304;
+}
+
+ccv3d_status forward_pointwise(ccv3d_handle* h, const void* x, void* out, int N, int T, int H, int W, cudaStream_t st) {
+    const ccv3d_desc& d = h->d;
+    const TcPlan& pl = h->plan;
+    const uint64_t P = (uint64_t)T * H * W;
+    if (P > 0x7FFFFFFFull) return CCV3D_ERR_UNSUPPORTED;
+    PwParams p;
+    memset(&p, 0, sizeof(p));
+    p.N = N; p.Cout = d.cout; p.CB = pl.CB; p.NPAD = pl.NPAD;
+    p.tiles_p = (int)((P + 127) / 128);
+    const int64_t total = (int64_t)N * p.tiles_p;
+    if (total > 0x7FFFFFFF) return CCV3D_ERR_UNSUPPORTED;
+    p.total_tiles = (int)total;
+    p.ECH = (pl.NPAD % 32 == 0) ? 32 : 16;
+    p.a_slot = 2 * 64 * 128;
+    p.e_slot = (uint32_t)(p.ECH * 128 * 2);
+    p.b_tap = (uint32_t)pl.NPAD * 128;
+    p.w_bytes = (uint32_t)pl.CB * p.b_tap;
+    p.tmem_cols = pow2_cols((uint32_t)(2 * pl.NPAD));
+    p.wait_limit_clk = h->wait_limit_clk;
+    p.bias = h->bias32;
+    p.wq = (const uint8_t*)h->wp;
+    p.status = h->status;
+    const size_t w_al = align_up(p.w_bytes, 1024);
+    const size_t fixed = 1024 + align_up(sizeof(TcShared), 128) + 2 * (size_t)p.e_slot + w_al;
+    int SA = (int)((SMEM_LIMIT - fixed) / p.a_slot);
+    if (SA > TC_MAX_STAGES) SA = TC_MAX_STAGES;
+    if (SA < 2) return CCV3D_ERR_UNSUPPORTED;
+    p.SA = SA;
+    p.w_bytes = (uint32_t)w_al;   // ring starts on a 1024-byte boundary; the copy itself is CB*b_tap bytes (a multiple of 1024)
+    CUtensorMap tm_x, tm_o;
+    {
+        cuuint64_t dims[3] = {(cuuint64_t)P, (cuuint64_t)d.cin, (cuuint64_t)N};
+        cuuint64_t strides[2] = {2ull * P, 2ull * P * d.cin};
+        cuuint32_t box[3] = {64, 64, 1};
+        cuuint32_t es[3] = {1, 1, 1};
+        if (h->encode(&tm_x, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(x), dims, strides, box, es,
+                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return CCV3D_ERR_CUDA;
+    }
+    {
+        cuuint64_t dims[3] = {(cuuint64_t)P, (cuuint64_t)d.cout, (cuuint64_t)N};
+        cuuint64_t strides[2] = {2ull * P, 2ull * P * d.cout};
+        cuuint32_t box[3] = {128, (cuuint32_t)p.ECH, 1};
+        cuuint32_t es[3] = {1, 1, 1};
+        if (h->encode(&tm_o, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, out, dims, strides, box, es,
+                      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return CCV3D_ERR_CUDA;
+    }
+    const size_t smem = fixed + (size_t)SA * p.a_slot;
+    if (cudaFuncSetAttribute(conv1x1_tcgen05_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return cuda_fail();
+    cudaEvent_t* pev = (h->prof_on && h->prof_ev) ? h->prof_ev + 3 * (h->prof_n % PROF_SLOTS) : nullptr;
+    if (pev) { cudaEventRecord(pev[0], st); cudaEventRecord(pev[1], st); }
+    const int grid = p.total_tiles < h->sm_count ? p.total_tiles : h->sm_count;
+    conv1x1_tcgen05_kernel<<<grid, TC_THREADS, smem, st>>>(tm_x, tm_o, p);
+    if (cudaGetLastError() != cudaSuccess) return cuda_fail();
+    if (pev) {
+        cudaEventRecord(pev[2], st);
+        h->prof_n++;
+    }
+    h->ctr.kernel_launches++;
+    h->ctr.tcgen05_bf16++;
+    return CCV3D_OK;
+}
+
 // ------------------------------------------------------------------------------------------------
 // Allocation-free variant of the tensor-core route (ccv3d_forward_static).  Its channels-last staging copy
 // lives in a fixed array in device memory that is part of the loaded library image, so the call needs no
@@ -656,7 +734,8 @@ ccv3d_status ccv3d_forward(ccv3d_handle* h, const void* x, const void* cache, vo
     ccv3d_status s = check_forward_args(h, x, cache, out, new_cache, N, T, H, W, true);
     if (s != CCV3D_OK) return count(h, s);
     cudaStream_t st = (cudaStream_t)stream;
-    if (h->use_tc) s = forward_tc(h, x, cache, out, new_cache, N, T, H, W, st);
+    if (h->use_tc && pointwise_eligible(h, T, H, W)) s = forward_pointwise(h, x, out, N, T, H, W, st);
+    else if (h->use_tc) s = forward_tc(h, x, cache, out, new_cache, N, T, H, W, st);
     else s = forward_simt(h, x, cache, out, new_cache, N, T, H, W, st);
     return count(h, s);
 }
