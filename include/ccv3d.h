@@ -51,6 +51,7 @@ typedef enum {
 
 /* ccv3d_desc.flags */
 #define CCV3D_FLAG_FORCE_SIMT 0x1u      /* BF16 layers: use the plain FP32-FMA kernel instead of the tensor-core kernel */
+#define CCV3D_FLAG_OVERLAP 0x4u          /* tensor-core route: process large images in bands, staging band k+1 on a side stream while band k is convolved */
 #define CCV3D_FLAG_TC_PER_TAP_A 0x2u    /* tensor-core kernel: fetch the activation tile once per tap (no halo reuse in shared memory) */
 
 /* Layer description, fixed at create time (Algorithm 1's Require line: W, b, p, s, d, g). */
@@ -107,6 +108,10 @@ ccv3d_status ccv3d_create(ccv3d_handle** out_h, const ccv3d_desc* d, const void*
  *              bit-exact copy of the last kt-1 frames of [cache ; x].  Ignored when kt == 1.
  * out must not overlap x or cache; new_cache must not overlap x, cache or out
  * (CCV3D_ERR_ALIAS): ping-pong two cache buffers.  All pointers must be 16-byte aligned.
+ * With CCV3D_FLAG_OVERLAP large images are processed in bands of rows on three side streams owned by the handle
+ * (staging of the next band overlaps the convolution of the current one); they fork from `stream` after
+ * everything enqueued on it so far and join it before the call returns, so the caller only ever needs to order
+ * against `stream`.
  * The tensor-core path keeps a channels-last staging copy of [cache ; x] in a
  * workspace owned by the handle; it is (re)allocated when a call needs more than
  * the handle holds (that call synchronises the device), so steady-state calls of

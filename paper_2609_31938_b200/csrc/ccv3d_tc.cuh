@@ -67,11 +67,12 @@ struct StageParams {
     __nv_bfloat16* new_cache;    // [N,Cin,tc,H,W] or null
     int N, Cin, T, H, W, tc, CB;
     int f_begin;                 // first Z frame to stage (tc when there is no cache and nothing older is needed)
+    int h_begin;                 // first image row of this launch (grid.y rows are staged)
 };
 
 constexpr int STG_PX = 64;  // pixels of one image row handled per block
 
-// grid: (ceil(W/64), H, N*(F - f_begin)*CB); block: 32 * (KB/8) threads.
+// grid: (ceil(W/64), rows of this launch, N*(F - f_begin)*CB); block: 32 * (KB/8) threads.
 // VEC: W % 8 == 0 and all bases 16-byte aligned -> 16-byte loads along w.
 template <int KB, bool VEC>
 __global__ void __launch_bounds__(32 * (KB / 8)) stage_frames_kernel(const StageParams p) {
@@ -86,7 +87,7 @@ __global__ void __launch_bounds__(32 * (KB / 8)) stage_frames_kernel(const Stage
     z /= p.CB;
     const int f = p.f_begin + z % nf;
     const int n = z / nf;
-    const int h = blockIdx.y;
+    const int h = p.h_begin + blockIdx.y;
     const int w0 = blockIdx.x * STG_PX;
     const int64_t HW = (int64_t)p.H * p.W;
 
@@ -281,7 +282,8 @@ struct TcParams {
     int kt, kh, kw;
     int CB;           // input-channel blocks of KB
     int NT, NPAD;     // output-channel tiles and their (padded) width, NPAD % 16 == 0, <= 256
-    int tiles_h, tiles_w, total_tiles;
+    int tiles_h, tiles_w, total_tiles;   // tile rows handled by this launch, tile columns, tiles of this launch
+    int ty_begin;                        // first tile row of this launch (a launch may cover a band of the image)
     int first_frame;  // Z frames below this are absent (first chunk): their taps are skipped
     int out_f32;      // 1: out is FP32, 0: BF16
     int per_tap_a;    // 1: one A load per tap (box without halo), 0: one halo load per (dt, ci-block)
@@ -412,7 +414,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                 int r = tile / p.NT;
                 const int t = r % p.T; r /= p.T;
                 const int tx = r % p.tiles_w; r /= p.tiles_w;
-                const int ty = r % p.tiles_h;
+                const int ty = p.ty_begin + r % p.tiles_h;
                 const int n = r / p.tiles_h;
                 const int h0 = ty * 16, w0 = tx * TW;
                 const int dt0 = (p.first_frame - t > 0) ? p.first_frame - t : 0;
@@ -613,7 +615,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
             int r = tile / p.NT;
             const int t = r % p.T; r /= p.T;
             const int tx = r % p.tiles_w; r /= p.tiles_w;
-            const int ty = r % p.tiles_h;
+            const int ty = p.ty_begin + r % p.tiles_h;
             const int n = r / p.tiles_h;
             ok = mbar_wait(&sh->acc_full[acc], pacc, sh, p, SITE_ACC_FULL);
             ok = __all_sync(0xffffffffu, ok);

@@ -135,6 +135,27 @@ def test_bf16_tensor_core_per_tap_loads(ccv, N, Cin, Cout, T, H, W, k, cache, bi
     run_case(ccv, si.conv_case(N, Cin, Cout, T, H, W, k=k, cache=cache, bias=bias, seed=7), flags=ccv.FLAG_TC_PER_TAP_A)
 
 
+@pytest.mark.parametrize("N,Cin,Cout,T,H,W,k,cache", [
+    (1, 64, 64, 3, 150, 160, (3, 3, 3), "random"),          # 10 tile rows -> 4 bands, ragged last band
+    (2, 96, 96, 3, 100, 128, (3, 3, 3), None),
+])
+def test_bf16_tensor_core_banded_overlap(ccv, N, Cin, Cout, T, H, W, k, cache):
+    """Banded schedule on side streams (staging of band k+1 overlaps the convolution of band k): same result,
+    bit for bit, as the single-stream schedule."""
+    c = si.conv_case(N, Cin, Cout, T, H, W, k=k, cache=cache, seed=13)
+    m, ctr = run_case(ccv, c, flags=ccv.FLAG_OVERLAP)
+    assert ctr["tcgen05_bf16"] == 1 and ctr["kernel_launches"] > 4          # several staging + convolution launches
+    a = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), flags=ccv.FLAG_OVERLAP)
+    b = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]))
+    x, cache_d = to_dev(c["x"]), to_dev(c["cache"])
+    oa, na = a(x, cache_d)
+    ob, nb = b(x, cache_d)
+    torch.cuda.synchronize()
+    assert torch.equal(oa, ob) and torch.equal(na, nb)
+    a.close()
+    b.close()
+
+
 def test_cfg2_bf16_384(ccv):
     m, ctr = run_case(ccv, si.conv_case(**si.CONFIGS["cfg2_bf16_384"]))
     assert ctr["tcgen05_bf16"] == 1 and m["cos"] > 0.99998
