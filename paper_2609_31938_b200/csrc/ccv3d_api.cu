@@ -36,8 +36,10 @@ struct TcPlan {      // per-layer choices of the tensor-core route
 
 struct ShapeKey {
     const void* zs;
-    int N, T, H, W;
-    bool operator==(const ShapeKey& o) const { return zs == o.zs && N == o.N && T == o.T && H == o.H && W == o.W; }
+    int N, T, H, W, BW;
+    bool operator==(const ShapeKey& o) const {
+        return zs == o.zs && N == o.N && T == o.T && H == o.H && W == o.W && BW == o.BW;
+    }
 };
 
 }  // namespace
@@ -214,7 +216,7 @@ ccv3d_status launch_stage(ccv3d_handle* h, StageParams sp, int h0, int h1, int n
     return CCV3D_OK;
 }
 
-ccv3d_status launch_conv(ccv3d_handle* h, TcParams p, int ty0, int ty1, size_t smem, int ks, cudaStream_t st) {
+ccv3d_status launch_conv(ccv3d_handle* h, TcParams p, int nb, int ty0, int ty1, size_t smem, int ks, cudaStream_t st) {
     const TcPlan& pl = h->plan;
     p.ty_begin = ty0;
     p.tiles_h = ty1 - ty0;
@@ -224,15 +226,17 @@ ccv3d_status launch_conv(ccv3d_handle* h, TcParams p, int ty0, int ty1, size_t s
     const int grid = p.total_tiles < h->sm_count ? p.total_tiles : h->sm_count;
     ccv3d_status s;
     // straight-line tap loops for the common kernels; the run-time variant takes everything else
-#define CCV3D_LAUNCH(KBv)                                                                      \
-    do {                                                                                       \
-        if (ks == 3 && p.TPB == 3) s = launch_tc<KBv, 2, 3, 3>(h, p, smem, grid, st);          \
-        else if (ks == 3 && p.TPB == 1) s = launch_tc<KBv, 2, 3, 1>(h, p, smem, grid, st);     \
-        else if (ks == 1) s = launch_tc<KBv, 2, 1, 1>(h, p, smem, grid, st);                   \
-        else s = launch_tc<KBv, 2, 0, 0>(h, p, smem, grid, st);                                \
+#define CCV3D_LAUNCH(KBv, NBv)                                                                   \
+    do {                                                                                         \
+        if (ks == 3 && p.TPB == 3) s = launch_tc<KBv, NBv, 3, 3>(h, p, smem, grid, st);          \
+        else if (ks == 3 && p.TPB == 1) s = launch_tc<KBv, NBv, 3, 1>(h, p, smem, grid, st);     \
+        else if (ks == 1) s = launch_tc<KBv, NBv, 1, 1>(h, p, smem, grid, st);                   \
+        else s = launch_tc<KBv, NBv, 0, 0>(h, p, smem, grid, st);                                \
     } while (0)
-    if (pl.KB == 64) CCV3D_LAUNCH(64);
-    else CCV3D_LAUNCH(32);
+    if (pl.KB == 64 && nb == 2) CCV3D_LAUNCH(64, 2);
+    else if (pl.KB == 64) CCV3D_LAUNCH(64, 1);
+    else if (nb == 2) CCV3D_LAUNCH(32, 2);
+    else CCV3D_LAUNCH(32, 1);
 #undef CCV3D_LAUNCH
     return s;
 }
@@ -260,11 +264,14 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
 
     // ---- implicit GEMM parameters ----
     const int per_tap = (d.flags & CCV3D_FLAG_TC_PER_TAP_A) ? 1 : 0;
-    const int NB = pl.NB;
+    // 256-pixel tiles (two 128-pixel blocks sharing every weight tile) unless that leaves SMs without a tile
+    int NB = pl.NB;
+    if ((int64_t)N * ((H + 15) / 16) * ((W + 15) / 16) * T * pl.NT < h->sm_count) NB = 1;
+    const int ACC = (2 * NB * pl.NPAD <= 512) ? 2 : 1;
     const int TW = 8 * NB;
     const int BW = per_tap ? TW : TW + d.kw - 1;
     const int BH = per_tap ? 16 : 16 + d.kh - 1;
-    ShapeKey key{h->workspace, N, T, H, W};
+    ShapeKey key{h->workspace, N, T, H, W, BW};
     if (!(key == h->tm_a_key)) {
         s = encode_act_map(h, N, T, H, W, BW, BH);
         if (s != CCV3D_OK) return s;
@@ -280,7 +287,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     p.first_frame = (tc && !cache) ? tc : 0;
     p.out_f32 = d.out_dtype == CCV3D_F32;
     p.per_tap_a = per_tap;
-    p.ACC = pl.ACC;
+    p.ACC = ACC;
     p.a_slot = (uint32_t)align_up((uint64_t)BW * BH * pl.KB * 2, 1024);
     p.b_tap = (uint32_t)pl.NPAD * pl.KB * 2;
     // epilogue: BF16 output rows that TMA can address (W*2 bytes a multiple of 16) go through shared memory
@@ -318,7 +325,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     if (SB > 8) SB = 8;
     while (SA < 4 && (size_t)(SA + 1) * p.a_slot + (size_t)SB * p.b_slot <= budget) ++SA;
     p.SA = SA; p.SB = SB;
-    p.tmem_cols = pow2_cols((uint32_t)(NB * pl.NPAD * pl.ACC));
+    p.tmem_cols = pow2_cols((uint32_t)(NB * pl.NPAD * ACC));
     if (p.tmem_cols > 512) return CCV3D_ERR_UNSUPPORTED;
     p.wait_limit_clk = h->wait_limit_clk;
     p.bias = h->bias32;
@@ -341,7 +348,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
         s = launch_stage(h, sp, 0, H, nframes, st);
         if (s != CCV3D_OK) return s;
         if (pev) cudaEventRecord(pev[1], st);
-        s = launch_conv(h, p, 0, tiles_h, smem, ks, st);
+        s = launch_conv(h, p, NB, 0, tiles_h, smem, ks, st);
         if (s != CCV3D_OK) return s;
     } else {
         cudaStream_t s_stage = h->side[0];
@@ -363,7 +370,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
             cudaStream_t s_conv = h->side[1 + (k & 1)];
             if (cudaStreamWaitEvent(s_conv, h->ev_band[k], 0) != cudaSuccess) return cuda_fail();
             if (k == 0 && pev) cudaEventRecord(pev[1], s_conv);
-            s = launch_conv(h, p, ty0, ty1, smem, ks, s_conv);
+            s = launch_conv(h, p, NB, ty0, ty1, smem, ks, s_conv);
             if (s != CCV3D_OK) return s;
         }
         for (int i = 1; i < 3; ++i) {
@@ -924,19 +931,31 @@ ccv3d_status ccv3d_device_status(ccv3d_handle* h, uint32_t* detail_host) {
 ccv3d_status ccv3d_add_bf16(const void* a, const void* b, void* y, int64_t n, void* stream) {
     if (!a || !b || !y || n < 0) return CCV3D_ERR_INVALID_ARG;
     if (n == 0) return CCV3D_OK;
-    const int64_t blocks = (n + 255) / 256;
-    add_bf16_kernel<<<(unsigned)(blocks > 148 * 16 ? 148 * 16 : blocks), 256, 0, (cudaStream_t)stream>>>(
-        (const __nv_bfloat16*)a, (const __nv_bfloat16*)b, (__nv_bfloat16*)y, n);
+    const bool vec = (n % 8 == 0) && !(((uintptr_t)a | (uintptr_t)b | (uintptr_t)y) & 15u);
+    const int64_t work = vec ? n / 8 : n;
+    const int64_t blocks = (work + 255) / 256;
+    const unsigned grid = (unsigned)(blocks > 148 * 16 ? 148 * 16 : blocks);
+    if (vec)
+        add_bf16_vec_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>((const uint4*)a, (const uint4*)b, (uint4*)y, work);
+    else
+        add_bf16_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)a, (const __nv_bfloat16*)b,
+                                                               (__nv_bfloat16*)y, n);
     return cudaGetLastError() == cudaSuccess ? CCV3D_OK : cuda_fail();
 }
 
 ccv3d_status ccv3d_upsample_bf16(const void* x, void* y, int32_t N, int32_t C, int32_t T, int32_t H, int32_t W,
                                  int32_t rt, void* stream) {
     if (!x || !y || N < 1 || C < 1 || T < 1 || H < 1 || W < 1 || rt < 1) return CCV3D_ERR_INVALID_ARG;
-    const int64_t total = (int64_t)N * C * T * rt * 4 * H * W;
-    const int64_t blocks = (total + 255) / 256;
-    upsample_bf16_kernel<<<(unsigned)(blocks > 148 * 16 ? 148 * 16 : blocks), 256, 0, (cudaStream_t)stream>>>(
-        (const __nv_bfloat16*)x, (__nv_bfloat16*)y, (int64_t)N * C, T, H, W, rt);
+    const bool vec = (W % 4 == 0) && !(((uintptr_t)x | (uintptr_t)y) & 15u);
+    const int64_t work = vec ? (int64_t)N * C * T * H * (W / 4) : (int64_t)N * C * T * rt * 4 * H * W;
+    const int64_t blocks = (work + 255) / 256;
+    const unsigned grid = (unsigned)(blocks > 148 * 16 ? 148 * 16 : blocks);
+    if (vec)
+        upsample_bf16_vec_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>((const uint2*)x, (uint4*)y, (int64_t)N * C, T, H,
+                                                                       W, rt);
+    else
+        upsample_bf16_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)y,
+                                                                   (int64_t)N * C, T, H, W, rt);
     return cudaGetLastError() == cudaSuccess ? CCV3D_OK : cuda_fail();
 }
 

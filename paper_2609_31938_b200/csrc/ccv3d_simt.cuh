@@ -132,6 +132,24 @@ __global__ void add_bf16_kernel(const __nv_bfloat16* __restrict__ a, const __nv_
         y[i] = __float2bfloat16_rn(__bfloat162float(a[i]) + __bfloat162float(b[i]));
 }
 
+// 8 elements (16 bytes) per thread; n8 = n / 8, all pointers 16-byte aligned
+__global__ void add_bf16_vec_kernel(const uint4* __restrict__ a, const uint4* __restrict__ b, uint4* __restrict__ y,
+                                    int64_t n8) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n8; i += (int64_t)gridDim.x * blockDim.x) {
+        const uint4 va = __ldg(a + i), vb = __ldg(b + i);
+        const uint32_t wa[4] = {va.x, va.y, va.z, va.w}, wb[4] = {vb.x, vb.y, vb.z, vb.w};
+        uint32_t wy[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float lo = __uint_as_float(wa[k] << 16) + __uint_as_float(wb[k] << 16);
+            const float hi = __uint_as_float(wa[k] & 0xFFFF0000u) + __uint_as_float(wb[k] & 0xFFFF0000u);
+            const __nv_bfloat162 r = __floats2bfloat162_rn(lo, hi);
+            wy[k] = *reinterpret_cast<const uint32_t*>(&r);
+        }
+        y[i] = make_uint4(wy[0], wy[1], wy[2], wy[3]);
+    }
+}
+
 // y[nc, t*rt + r, 2h + a, 2w + b] = x[nc, t, h, w]
 __global__ void upsample_bf16_kernel(const __nv_bfloat16* __restrict__ x, __nv_bfloat16* __restrict__ y,
                                      int64_t NC, int T, int H, int W, int rt) {
@@ -142,6 +160,32 @@ __global__ void upsample_bf16_kernel(const __nv_bfloat16* __restrict__ x, __nv_b
         const int to = (int)((i / ((int64_t)4 * W * H)) % (T * rt));
         const int64_t nc = i / ((int64_t)4 * W * H * T * rt);
         y[i] = x[((nc * T + to / rt) * H + ho / 2) * W + wo / 2];
+    }
+}
+
+// Same, W % 4 == 0 and 16-byte aligned bases: a thread reads 4 input pixels (8 bytes), doubles them to 8 output
+// pixels (16 bytes) and writes that vector to the 2 output rows of each of the rt output frames.
+__global__ void upsample_bf16_vec_kernel(const uint2* __restrict__ x, uint4* __restrict__ y, int64_t NC, int T, int H,
+                                         int W, int rt) {
+    const int W4 = W / 4;
+    const int64_t total = NC * T * (int64_t)H * W4;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int w4 = (int)(i % W4);
+        const int h = (int)((i / W4) % H);
+        const int t = (int)((i / ((int64_t)W4 * H)) % T);
+        const int64_t nc = i / ((int64_t)W4 * H * T);
+        const uint2 v = __ldg(x + i);
+        uint4 o;
+        o.x = __byte_perm(v.x, v.x, 0x1010);   // pixel 0 twice
+        o.y = __byte_perm(v.x, v.x, 0x3232);   // pixel 1 twice
+        o.z = __byte_perm(v.y, v.y, 0x1010);
+        o.w = __byte_perm(v.y, v.y, 0x3232);
+        const int64_t row_vecs = W4;           // 16-byte vectors per output row (2W pixels)
+        for (int r = 0; r < rt; ++r) {
+            uint4* dst = y + (((nc * T * rt + (int64_t)t * rt + r) * (2 * H) + 2 * h) * row_vecs + w4);
+            dst[0] = o;
+            dst[row_vecs] = o;
+        }
     }
 }
 

@@ -265,17 +265,22 @@ def test_host_entry_point_matches_device_entry_point(ccv):
     layer.close()
 
 
-def test_chain_glue_kernels(ccv):
+@pytest.mark.parametrize("shape,rt", [((2, 3, 2, 5, 6), 3), ((1, 4, 3, 6, 8), 4), ((1, 2, 2, 4, 12), 1)])
+def test_chain_glue_kernels(ccv, shape, rt):
+    """Residual add (exact sum, one RNE rounding) and nearest-neighbour upsampling (exact copies), scalar and
+    vector code paths, against their definitions written out in numpy."""
     rng = np.random.default_rng(1)
-    a = si.to_bf16_bits(rng.standard_normal((2, 3, 2, 5, 6)).astype(np.float32))
-    b = si.to_bf16_bits(rng.standard_normal((2, 3, 2, 5, 6)).astype(np.float32))
+    a = si.to_bf16_bits(rng.standard_normal(shape).astype(np.float32))
+    b = si.to_bf16_bits(rng.standard_normal(shape).astype(np.float32))
     da, db = to_dev(a), to_dev(b)
-    y = torch.empty_like(da)
+    ybuf, y = _guarded(shape, torch.bfloat16)
     assert ccv.ccv3d_add_bf16(da.data_ptr(), db.data_ptr(), y.data_ptr(), da.numel()) == ccv.OK
     exp = si.to_bf16_bits((si.bf16_bits_to_f32(a) + si.bf16_bits_to_f32(b)).astype(np.float32))
     assert np.array_equal(bits(y), exp)
-    up = torch.empty((2, 3, 6, 10, 12), dtype=torch.bfloat16, device="cuda:0")
-    assert ccv.ccv3d_upsample_bf16(da.data_ptr(), up.data_ptr(), 2, 3, 2, 5, 6, 3) == ccv.OK
+    N, C, T, H, W = shape
+    ubuf, up = _guarded((N, C, T * rt, 2 * H, 2 * W), torch.bfloat16)
+    assert ccv.ccv3d_upsample_bf16(da.data_ptr(), up.data_ptr(), N, C, T, H, W, rt) == ccv.OK
     torch.cuda.synchronize()
-    exp_up = np.repeat(np.repeat(np.repeat(a, 3, axis=2), 2, axis=3), 2, axis=4)
+    assert _guards_intact(ybuf) and _guards_intact(ubuf), "glue kernel wrote outside its output"
+    exp_up = np.repeat(np.repeat(np.repeat(a, rt, axis=2), 2, axis=3), 2, axis=4)
     assert np.array_equal(bits(up), exp_up)
