@@ -186,6 +186,15 @@ ccv3d_status ccv3d_device_status(ccv3d_handle* h, uint32_t* detail_host);
 ccv3d_status ccv3d_profile_enable(ccv3d_handle* h, int32_t enable);
 ccv3d_status ccv3d_profile_read(ccv3d_handle* h, double* stage_ms_host, double* conv_ms_host, int64_t* calls_host);
 
+/*
+ * Self-test of the bounded-wait mechanism (no counterpart in the paper).  Enqueues a one-block kernel that waits
+ * on a barrier nothing will ever signal, with the given limit (1..1000 ms).  The wait gives up, the kernel
+ * returns normally and the handle's status word is set, so that after synchronising the stream
+ * ccv3d_device_status returns CCV3D_ERR_DEVICE_TIMEOUT with detail 0x7F in its low byte.  Nothing faults,
+ * traps or hangs; the handle stays usable.
+ */
+ccv3d_status ccv3d_selftest_wait_timeout(ccv3d_handle* h, int32_t limit_ms, void* stream);
+
 /* Static, human-readable name of a status code. */
 const char* ccv3d_status_string(ccv3d_status s);
 

@@ -40,7 +40,7 @@ class Counters(ctypes.Structure):
 
 EXPORTS = ("ccv3d_create", "ccv3d_forward", "ccv3d_forward_host", "ccv3d_workspace_bytes", "ccv3d_destroy",
            "ccv3d_get_counters", "ccv3d_device_status", "ccv3d_status_string", "ccv3d_add_bf16",
-           "ccv3d_upsample_bf16", "ccv3d_profile_enable", "ccv3d_profile_read", "ccv3d_forward_static")
+           "ccv3d_upsample_bf16", "ccv3d_profile_enable", "ccv3d_profile_read", "ccv3d_forward_static", "ccv3d_selftest_wait_timeout")
 
 
 def _load() -> ctypes.CDLL:
@@ -63,6 +63,7 @@ def _load() -> ctypes.CDLL:
     lib.ccv3d_profile_enable.argtypes = [vp, i32]
     lib.ccv3d_profile_read.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double),
                                        ctypes.POINTER(ctypes.c_int64)]
+    lib.ccv3d_selftest_wait_timeout.argtypes = [vp, i32, vp]
     lib.ccv3d_add_bf16.argtypes = [vp, vp, vp, ctypes.c_int64, vp]
     lib.ccv3d_upsample_bf16.argtypes = [vp, vp, i32, i32, i32, i32, i32, i32, vp]
     for name in EXPORTS:
@@ -153,6 +154,10 @@ def ccv3d_profile_read(h):
     a, b, n = ctypes.c_double(), ctypes.c_double(), ctypes.c_int64()
     s = lib.ccv3d_profile_read(h, ctypes.byref(a), ctypes.byref(b), ctypes.byref(n))
     return s, a.value, b.value, n.value
+
+
+def ccv3d_selftest_wait_timeout(h, limit_ms: int, stream=0) -> int:
+    return lib.ccv3d_selftest_wait_timeout(h, limit_ms, stream)
 
 
 def ccv3d_add_bf16(a, b, y, n, stream=0) -> int:

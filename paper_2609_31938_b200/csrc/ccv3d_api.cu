@@ -928,6 +928,16 @@ ccv3d_status ccv3d_device_status(ccv3d_handle* h, uint32_t* detail_host) {
     return CCV3D_ERR_DEVICE_TIMEOUT;
 }
 
+ccv3d_status ccv3d_selftest_wait_timeout(ccv3d_handle* h, int32_t limit_ms, void* stream) {
+    if (!h || limit_ms < 1 || limit_ms > 1000) return CCV3D_ERR_INVALID_ARG;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, h->device) != cudaSuccess) return cuda_fail();
+    wait_timeout_selftest_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(h->status, (long long)prop.clockRate * limit_ms);
+    if (cudaGetLastError() != cudaSuccess) return cuda_fail();
+    h->ctr.kernel_launches++;
+    return CCV3D_OK;
+}
+
 ccv3d_status ccv3d_add_bf16(const void* a, const void* b, void* y, int64_t n, void* stream) {
     if (!a || !b || !y || n < 0) return CCV3D_ERR_INVALID_ARG;
     if (n == 0) return CCV3D_OK;

@@ -877,4 +877,30 @@ conv1x1_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_x,   // x as (pixe
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// Self-test of the bounded-wait path: one CTA waits on an mbarrier phase that nothing ever completes.
+// The wait gives up after limit_clk clocks, records (block << 8) | site in the status word and the kernel
+// returns normally - the same code path a lost TMA completion would take in the convolution kernels.
+// ------------------------------------------------------------------------------------------------
+__global__ void wait_timeout_selftest_kernel(unsigned int* status, long long limit_clk) {
+    __shared__ uint64_t bar;
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const uint32_t b = smem_u32(&bar);
+        const long long t0 = clock64();
+        for (uint32_t it = 1;; ++it) {
+            if (mbar_try_wait(b, 0)) break;                       // phase 0 never completes: nobody arrives
+            if ((it & 63u) == 0u && clock64() - t0 > limit_clk) {
+                atomicCAS(status, 0u, (blockIdx.x << 8) | 0x7Fu);  // site 0x7F: the self-test
+                break;
+            }
+        }
+    }
+    __syncthreads();
+}
+
 }  // namespace ccv3d

@@ -248,6 +248,30 @@ def test_forward_argument_errors_and_counters(ccv):
     layer.close()
 
 
+def test_bounded_wait_reports_a_timeout_and_the_handle_stays_usable(ccv):
+    """A wait that can never be satisfied (a barrier nothing signals) gives up after its limit: the kernel
+    returns, the status word says where, and the next call on the same handle works."""
+    import time
+    c = si.conv_case(1, 64, 64, 2, 16, 16, seed=14)
+    layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]))
+    stream = torch.cuda.current_stream().cuda_stream
+    t0 = time.time()
+    assert ccv.ccv3d_selftest_wait_timeout(layer.h, 20, stream) == ccv.OK
+    torch.cuda.synchronize()
+    assert time.time() - t0 < 5.0
+    st, detail = layer.device_status()
+    assert st == ccv.ERR_DEVICE_TIMEOUT and (detail & 0xFF) == 0x7F
+    assert layer.device_status()[0] == ccv.OK                   # reading cleared the word
+    assert layer.counters()["device_timeout"] == 1
+    ref, ref_nc = oracle.forward(c["x"], c["cache"], c["w"], c["b"])
+    out, nc = layer(to_dev(c["x"]), to_dev(c["cache"]))
+    torch.cuda.synchronize()
+    assert layer.device_status()[0] == ccv.OK
+    check(as_f64(out), ref, "bf16")
+    assert np.array_equal(bits(nc), ref_nc)
+    layer.close()
+
+
 def test_host_entry_point_matches_device_entry_point(ccv):
     c = si.conv_case(1, 64, 96, 3, 24, 40, seed=12)
     layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]))
