@@ -111,20 +111,23 @@ def cfg_of(name):
 
 # ---------------------------------------------------------------------------------------------- CPU oracle leg
 def oracle_sample(name, target_s=12.0):
-    """Times the oracle, as it stands, on a spatial crop (all channels, all frames, the cache included) of the
-    workload, sized from a small calibration run so that one pass takes about target_s seconds."""
+    """Picks a spatial crop (all channels, all frames, the cache included) of the workload on which one pass of
+    the oracle, as it stands, takes about target_s seconds on this host: a small calibration pass (run twice, the
+    second timed, so that thread start-up is not counted) gives the rate."""
     import oracle
     cfg, d = cfg_of(name)
-    crop = dict(cfg, H=16, W=16)
+    crop = dict(cfg, H=min(d["H"], 32), W=min(d["W"], 32))
     c = si.conv_case(**crop)
+    oracle.forward(c["x"], c["cache"], c["w"], c["b"])
     t0 = time.perf_counter()
     oracle.forward(c["x"], c["cache"], c["w"], c["b"])
     t_small = time.perf_counter() - t0
-    fl_small = si.conv_flops(d["N"], d["Cin"], d["Cout"], d["T"], 16, 16, d["k"])
-    rate = fl_small / max(t_small, 1e-6)
-    px = target_s * rate / (fl_small / 256.0)          # pixels per frame the oracle covers in target_s seconds
+    px_small = crop["H"] * crop["W"]
+    px = target_s / max(t_small, 1e-6) * px_small        # pixels per frame the oracle covers in target_s seconds
     W = int(min(d["W"], 80))
     H = int(min(d["H"], max(8, px // W)))
+    if H == d["H"]:
+        W = int(min(d["W"], max(W, px // H)))
     return dict(cfg, H=H, W=W)
 
 
