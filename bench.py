@@ -246,7 +246,7 @@ def main_ours(args):
         return None if a is None else torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
 
     x, cache = up(c["x"]), up(c["cache"])
-    layer = ccv.CausalConv3d(up(c["w"]), up(c["b"]))
+    layer = ccv.CausalConv3d(up(c["w"]), up(c["b"]), flags=args.flags)
     out = torch.empty((d["N"], d["Cout"], d["T"], d["H"], d["W"]), dtype=torch.bfloat16, device=dev)
     nc = torch.empty_like(cache) if cache is not None else None
     stream = torch.cuda.current_stream()
@@ -384,6 +384,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-chain", action="store_true", help="skip the decoder-chain leg")
+    ap.add_argument("--flags", type=int, default=0, help="CCV3D_FLAG_* bits for the layer (e.g. 8 = fused route without staging copy)")
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(n for n in si.CONFIGS if "bf16" in n))
     args = ap.parse_args()
     if args.impl == "reference":

@@ -32,6 +32,7 @@ struct TcPlan {      // per-layer choices of the tensor-core route
     int KB, CB, cin_pad;
     int NT, NPAD, cout_pad;
     int NB, ACC;
+    bool fused;      // CCV3D_FLAG_FUSED: no staging copy when the call's W allows TMA rows (W % 8 == 0)
 };
 
 struct ShapeKey {
@@ -103,7 +104,12 @@ ccv3d_status validate_desc(const ccv3d_desc* d) {
 }
 
 void make_plan(const ccv3d_desc& d, TcPlan* pl) {
-    pl->KB = (d.cin % 64 == 0) ? 64 : 32;
+    // 64-channel K blocks for the staged route and the 1x1x1 streaming kernel when Cin allows; the fused route
+    // (CCV3D_FLAG_FUSED) transposes 32-channel blocks, so its layers are packed for 32
+    const bool pointwise = d.kt == 1 && d.kh == 1 && d.kw == 1;
+    pl->fused = (d.flags & CCV3D_FLAG_FUSED) && !(d.flags & (CCV3D_FLAG_TC_PER_TAP_A | CCV3D_FLAG_OVERLAP)) && !pointwise &&
+                d.out_dtype == CCV3D_BF16;
+    pl->KB = (d.cin % 64 == 0 && !pl->fused) ? 64 : 32;
     pl->CB = (d.cin + pl->KB - 1) / pl->KB;
     pl->cin_pad = pl->CB * pl->KB;
     pl->NT = (d.cout + 255) / 256;
@@ -188,10 +194,10 @@ uint64_t tc_workspace_bytes(const ccv3d_handle* h, int N, int T, int H, int W) {
 
 template <int KB, int NB, int KS, int TPBC>
 ccv3d_status launch_tc(ccv3d_handle* h, const TcParams& p, size_t smem, int grid, cudaStream_t st) {
-    auto kern = conv3d_tcgen05_kernel<KB, NB, KS, TPBC>;
+    auto kern = conv3d_tcgen05_kernel<KB, NB, KS, TPBC, false>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return cuda_fail();
-    kern<<<grid, TC_THREADS, smem, st>>>(h->tm_a, h->tm_o, p);
+    kern<<<grid, TC_THREADS, smem, st>>>(h->tm_a, h->tm_a, h->tm_o, p);
     if (cudaGetLastError() != cudaSuccess) return cuda_fail();
     h->ctr.kernel_launches++;
     return CCV3D_OK;
@@ -386,6 +392,138 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     return CCV3D_OK;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Fused route: no staging copy.  The convolution kernel reads x and the cache through two tensor maps and
+// transposes in shared memory; the cache update is a separate bit-copy kernel.
+// ------------------------------------------------------------------------------------------------
+template <int NB, int KS, int TPBC>
+ccv3d_status launch_fused(ccv3d_handle* h, const CUtensorMap& tm_x, const CUtensorMap& tm_c, const CUtensorMap& tm_o,
+                          const TcParams& p, size_t smem, int grid, cudaStream_t st) {
+    auto kern = conv3d_tcgen05_kernel<32, NB, KS, TPBC, true>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return cuda_fail();
+    kern<<<grid, TC_THREADS_FUSED, smem, st>>>(tm_x, tm_c, tm_o, p);
+    if (cudaGetLastError() != cudaSuccess) return cuda_fail();
+    h->ctr.kernel_launches++;
+    return CCV3D_OK;
+}
+
+ccv3d_status encode_ncthw_map(ccv3d_handle* h, CUtensorMap* tm, const void* base, int N, int C, int T, int H, int W,
+                              int box_w, int box_h, int box_c, CUtensorMapSwizzle swz) {
+    cuuint64_t dims[5] = {(cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)T, (cuuint64_t)C, (cuuint64_t)N};
+    cuuint64_t strides[4] = {2ull * W, 2ull * W * H, 2ull * W * H * T, 2ull * W * H * T * C};
+    cuuint32_t box[5] = {(cuuint32_t)box_w, (cuuint32_t)box_h, 1, (cuuint32_t)box_c, 1};
+    cuuint32_t es[5] = {1, 1, 1, 1, 1};
+    CUresult r = h->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, strides, box, es,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? CCV3D_OK : CCV3D_ERR_CUDA;
+}
+
+bool fused_eligible(const ccv3d_handle* h, int W) { return h->plan.fused && W % 8 == 0; }
+
+ccv3d_status forward_fused(ccv3d_handle* h, const void* x, const void* cache, void* out, void* new_cache, int N, int T,
+                           int H, int W, cudaStream_t st) {
+    const ccv3d_desc& d = h->d;
+    const TcPlan& pl = h->plan;
+    const int tc = d.kt - 1;
+    if (!tc) cache = nullptr;
+    int NB = pl.NB;
+    if ((int64_t)N * ((H + 15) / 16) * ((W + 15) / 16) * T * pl.NT < h->sm_count) NB = 1;
+    const int ACC = (2 * NB * pl.NPAD <= 512) ? 2 : 1;
+    const int TW = 8 * NB, BW = TW + d.kw - 1, BH = 16 + d.kh - 1;
+
+    TcParams p;
+    memset(&p, 0, sizeof(p));
+    p.N = N; p.T = T; p.H = H; p.W = W; p.Cout = d.cout; p.F = tc + T;
+    p.kt = d.kt; p.kh = d.kh; p.kw = d.kw; p.tc = tc;
+    p.CB = pl.CB; p.NT = pl.NT; p.NPAD = pl.NPAD;
+    p.tiles_h = (H + 15) / 16;
+    p.tiles_w = (W + TW - 1) / TW;
+    const int64_t total = (int64_t)N * p.tiles_h * p.tiles_w * T * pl.NT;
+    if (total > 0x7FFFFFFF) return CCV3D_ERR_UNSUPPORTED;
+    p.total_tiles = (int)total;
+    p.first_frame = (tc && !cache) ? tc : 0;
+    p.ACC = ACC;
+    p.a_slot = (uint32_t)align_up((uint64_t)BW * BH * 64, 1024);
+    p.raw_slot = (uint32_t)align_up((uint64_t)32 * BH * RAW_PX * 2, 1024);
+    p.b_tap = (uint32_t)pl.NPAD * 64;
+    p.epi_tma = 1;
+    p.ECH = (pl.NPAD % 32 == 0) ? 32 : 16;
+    p.e_slot = (uint32_t)(p.ECH * 16 * TW * 2);
+    const size_t fixed = 1024 + align_up(sizeof(TcShared), 128) + 2 * (size_t)p.e_slot + 2 * (size_t)p.raw_slot + 2048;
+    if (fixed + 2 * (size_t)p.a_slot + 2 * (size_t)p.b_tap > SMEM_LIMIT) return CCV3D_ERR_UNSUPPORTED;
+    const size_t budget = SMEM_LIMIT - fixed;
+    p.TPB = ((size_t)p.b_tap * d.kw <= 24576) ? d.kw : 1;
+    int SA = 2;
+    for (;;) {
+        p.b_slot = (uint32_t)align_up((uint64_t)p.b_tap * p.TPB, 1024);
+        if ((size_t)SA * p.a_slot + 3 * (size_t)p.b_slot <= budget) break;
+        if (p.TPB > 1) { p.TPB = 1; continue; }
+        if ((size_t)SA * p.a_slot + 2 * (size_t)p.b_slot <= budget) break;
+        return CCV3D_ERR_UNSUPPORTED;
+    }
+    int SB = (int)((budget - (size_t)SA * p.a_slot) / p.b_slot);
+    if (SB > TC_MAX_STAGES) SB = TC_MAX_STAGES;
+    p.SA = SA; p.SB = SB;
+    p.tmem_cols = pow2_cols((uint32_t)(NB * pl.NPAD * ACC));
+    if (p.tmem_cols > 512) return CCV3D_ERR_UNSUPPORTED;
+    p.wait_limit_clk = h->wait_limit_clk;
+    p.bias = h->bias32;
+    p.wq = (const uint8_t*)h->wp;
+    p.out = out;
+    p.status = h->status;
+
+    // The raw boxes have 64-byte rows, so they take the 64-byte swizzle: a swizzle span wider than the box row
+    // (128-byte swizzle here) made the copy land outside its shared-memory slot.
+    CUtensorMap tm_x, tm_c, tm_o;
+    ccv3d_status s = encode_ncthw_map(h, &tm_x, x, N, d.cin, T, H, W, RAW_PX, BH, 32, CU_TENSOR_MAP_SWIZZLE_64B);
+    if (s != CCV3D_OK) return s;
+    if (cache) {
+        s = encode_ncthw_map(h, &tm_c, cache, N, d.cin, tc, H, W, RAW_PX, BH, 32, CU_TENSOR_MAP_SWIZZLE_64B);
+        if (s != CCV3D_OK) return s;
+    } else {
+        tm_c = tm_x;   // never dereferenced: the taps that would read the cache are skipped
+    }
+    s = encode_ncthw_map(h, &tm_o, out, N, d.cout, T, H, W, TW, 16, p.ECH, CU_TENSOR_MAP_SWIZZLE_NONE);
+    if (s != CCV3D_OK) return s;
+
+    const size_t smem = fixed + (size_t)SA * p.a_slot + (size_t)SB * p.b_slot;
+    const int grid = p.total_tiles < h->sm_count ? p.total_tiles : h->sm_count;
+    const int ks = (d.kh == d.kw && (d.kh == 1 || d.kh == 3)) ? d.kh : 0;
+    cudaEvent_t* pev = (h->prof_on && h->prof_ev) ? h->prof_ev + 3 * (h->prof_n % PROF_SLOTS) : nullptr;
+    if (pev) cudaEventRecord(pev[0], st);
+    // cache update: bit copy of the last kt-1 frames of [cache ; x]
+    if (tc && new_cache) {
+        const uint64_t fbytes = (uint64_t)H * W * 2;          // W % 8 == 0: whole frames in 16-byte units
+        const int64_t planes = (int64_t)N * d.cin * tc;
+        const int64_t units = (int64_t)(fbytes / 16);
+        dim3 g((unsigned)((units + 255) / 256 > 64 ? 64 : (units + 255) / 256), (unsigned)(planes < 65535 ? planes : 65535));
+        cache_update_kernel<uint4><<<g, 256, 0, st>>>((const uint4*)x, (const uint4*)cache, (uint4*)new_cache, d.cin, T, tc,
+                                                     units, planes);
+        if (cudaGetLastError() != cudaSuccess) return cuda_fail();
+        h->ctr.kernel_launches++;
+    }
+    if (pev) cudaEventRecord(pev[1], st);
+#define CCV3D_LAUNCH_FUSED(NBv)                                                                              \
+    do {                                                                                                     \
+        if (ks == 3 && p.TPB == 3) s = launch_fused<NBv, 3, 3>(h, tm_x, tm_c, tm_o, p, smem, grid, st);      \
+        else if (ks == 3 && p.TPB == 1) s = launch_fused<NBv, 3, 1>(h, tm_x, tm_c, tm_o, p, smem, grid, st); \
+        else if (ks == 1) s = launch_fused<NBv, 1, 1>(h, tm_x, tm_c, tm_o, p, smem, grid, st);               \
+        else s = launch_fused<NBv, 0, 0>(h, tm_x, tm_c, tm_o, p, smem, grid, st);                            \
+    } while (0)
+    if (NB == 2) CCV3D_LAUNCH_FUSED(2);
+    else CCV3D_LAUNCH_FUSED(1);
+#undef CCV3D_LAUNCH_FUSED
+    if (s != CCV3D_OK) return s;
+    h->ctr.tcgen05_bf16++;
+    if (pev) {
+        cudaEventRecord(pev[2], st);
+        h->prof_n++;
+    }
+    return CCV3D_OK;
+}
+
 // 1x1x1 layers whose weights fit in shared memory stream straight from NCTHW (no staging copy).
 bool pointwise_eligible(const ccv3d_handle* h, int T, int H, int W) {
     const ccv3d_desc& d = h->d;
@@ -492,10 +630,10 @@ ccv3d_status static_scratch_for_current_device(void** out_ptr) {
 template <int KB, int NB, int KS, int TPBC>
 ccv3d_status launch_tc_with_maps(ccv3d_handle* h, const CUtensorMap& tm_a, const CUtensorMap& tm_o, const TcParams& p,
                                  size_t smem, int grid, cudaStream_t st) {
-    auto kern = conv3d_tcgen05_kernel<KB, NB, KS, TPBC>;
+    auto kern = conv3d_tcgen05_kernel<KB, NB, KS, TPBC, false>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return cuda_fail();
-    kern<<<grid, TC_THREADS, smem, st>>>(tm_a, tm_o, p);
+    kern<<<grid, TC_THREADS, smem, st>>>(tm_a, tm_a, tm_o, p);
     if (cudaGetLastError() != cudaSuccess) return cuda_fail();
     h->ctr.kernel_launches++;
     return CCV3D_OK;
@@ -818,7 +956,8 @@ ccv3d_status ccv3d_destroy(ccv3d_handle* h) {
 ccv3d_status ccv3d_workspace_bytes(const ccv3d_handle* h, int32_t N, int32_t T, int32_t H, int32_t W,
                                    uint64_t* bytes_host) {
     if (!h || !bytes_host || N < 1 || T < 1 || H < 1 || W < 1) return CCV3D_ERR_INVALID_ARG;
-    *bytes_host = h->use_tc ? tc_workspace_bytes(h, N, T, H, W) : 0;
+    const bool scratch_free = !h->use_tc || pointwise_eligible(h, T, H, W) || fused_eligible(h, W);
+    *bytes_host = scratch_free ? 0 : tc_workspace_bytes(h, N, T, H, W);
     return CCV3D_OK;
 }
 
@@ -830,6 +969,7 @@ ccv3d_status ccv3d_forward(ccv3d_handle* h, const void* x, const void* cache, vo
     if (s != CCV3D_OK) return count(h, s);
     cudaStream_t st = (cudaStream_t)stream;
     if (h->use_tc && pointwise_eligible(h, T, H, W)) s = forward_pointwise(h, x, out, N, T, H, W, st);
+    else if (h->use_tc && fused_eligible(h, W)) s = forward_fused(h, x, cache, out, new_cache, N, T, H, W, st);
     else if (h->use_tc) s = forward_tc(h, x, cache, out, new_cache, N, T, H, W, st);
     else s = forward_simt(h, x, cache, out, new_cache, N, T, H, W, st);
     return count(h, s);

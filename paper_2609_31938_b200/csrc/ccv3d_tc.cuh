@@ -5,6 +5,10 @@
 //   stage_frames_kernel   per call: Z = [cache ; x] (NCTHW) -> channels-last blocks
 //                         Zs[n][frame][cb][h][w][KB], and in the same pass the
 //                         bit-exact cache update new_cache = last kt-1 frames of Z.
+//   (fused mode)          no staging pass: a producer thread fetches raw [channel][row][32 pixels] boxes by TMA
+//                         straight from x or from the cache (whichever holds the tap's frame), and four
+//                         transposer warps turn each into the channels-last halo tile in shared memory
+//                         (ldmatrix.trans + stmatrix); the cache update is then a separate copy kernel.
 //   conv3d_tcgen05_kernel per call: persistent implicit GEMM.  For an output tile of
 //                         16 rows x 8*NB pixels of one frame t, D[pixel, co] =
 //                         sum over (dt, ci-block, dh, dw) of A_tap[pixel, ci] * Wp[tap][co, ci]
@@ -273,6 +277,20 @@ __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wa
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
 
+// Four 8x8 16-bit matrices, transposed on the way from shared memory to registers; lane l gives the address of
+// row l%8 of matrix l/8.  The registers come out in the fragment layout stmatrix takes.
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+                 : "r"(addr)
+                 : "memory");
+}
+__device__ __forceinline__ void stmatrix_x4(uint32_t addr, const uint32_t (&r)[4]) {
+    asm volatile("stmatrix.sync.aligned.m8n8.x4.shared.b16 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(r[0]), "r"(r[1]),
+                 "r"(r[2]), "r"(r[3])
+                 : "memory");
+}
+
 // ------------------------------------------------------------------------------------------------
 // the implicit-GEMM kernel
 // ------------------------------------------------------------------------------------------------
@@ -293,6 +311,8 @@ struct TcParams {
     int SA, SB, ACC;  // ring depths and accumulator buffers
     uint32_t a_slot, b_slot, b_tap;  // bytes per ring slot (multiples of 1024) and per tap inside a weight slot
     uint32_t e_slot;          // bytes of one epilogue staging buffer (two are allocated when epi_tma)
+    uint32_t raw_slot;        // fused mode: bytes of one raw [32 ch][BH rows][32 px] box (two are allocated)
+    int tc;                   // fused mode: cache frames (kt-1); Z frame f < tc comes from the cache map
     uint32_t tmem_cols;       // power of two >= NB*NPAD*ACC
     long long wait_limit_clk; // bound of every mbarrier wait, in SM clocks
     const float* bias;        // [NT*NPAD]
@@ -302,16 +322,20 @@ struct TcParams {
 };
 
 enum : uint32_t {
-    SITE_A_EMPTY = 1, SITE_B_EMPTY = 2, SITE_A_FULL = 3, SITE_B_FULL = 4, SITE_ACC_EMPTY = 5, SITE_ACC_FULL = 6
+    SITE_A_EMPTY = 1, SITE_B_EMPTY = 2, SITE_A_FULL = 3, SITE_B_FULL = 4, SITE_ACC_EMPTY = 5, SITE_ACC_FULL = 6,
+    SITE_RAW_EMPTY = 7, SITE_RAW_FULL = 8
 };
 
 constexpr int TC_THREADS = 256;
+constexpr int TC_THREADS_FUSED = 384;    // + 4 transposer warps
+constexpr int RAW_PX = 32;               // pixels per row of a raw box (64 bytes), starting 8 pixels left of the tile
 constexpr int TC_MAX_STAGES = 12;
 
 struct TcShared {  // placed after the rings
     uint64_t full_a[TC_MAX_STAGES], empty_a[TC_MAX_STAGES];
     uint64_t full_b[TC_MAX_STAGES], empty_b[TC_MAX_STAGES];
     uint64_t acc_full[2], acc_empty[2];
+    uint64_t raw_full[2], raw_empty[2];
     uint32_t tmem_base;
     volatile int abort_flag;
 };
@@ -357,11 +381,14 @@ __device__ __forceinline__ uint32_t make_desc_lo(uint32_t addr) {
 // KS/TPBC: compile-time spatial kernel size (kh = kw = KS) and taps per weight stage, which turn the tap loop
 // into straight-line code with immediate descriptor offsets; KS = 0 keeps everything run-time (any odd kh, kw,
 // and the per-tap A mode).
-template <int KB, int NB, int KS, int TPBC>
-__global__ void __launch_bounds__(TC_THREADS, 1)
-conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged activations (c, w, h, cb, n*F+f)
+// FUSED: no staging copy; tm_a is x as (w, h, t, c, n), tm_c the cache as (w, h, frame, c, n); needs KB = 32.
+template <int KB, int NB, int KS, int TPBC, bool FUSED>
+__global__ void __launch_bounds__(FUSED ? TC_THREADS_FUSED : TC_THREADS, 1)
+conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged activations (c, w, h, cb, n*F+f), or x
+                      const __grid_constant__ CUtensorMap tm_c,   // fused mode: the cache
                       const __grid_constant__ CUtensorMap tm_o,   // out (w, h, t, co, n); used when p.epi_tma
                       const TcParams p) {
+    static_assert(!FUSED || KB == 32, "the fused mode transposes 32-channel blocks");
     constexpr uint32_t ROWB = KB * 2;                       // bytes per pixel row (one swizzle span)
     constexpr uint32_t LAYOUT = (KB == 64) ? 2u : 4u;       // 128-byte / 64-byte swizzle
     constexpr uint32_t B_SBO = 8 * ROWB;                    // 8-row group pitch of the weight tile
@@ -375,7 +402,9 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     uint8_t* ring_a = smem;
     uint8_t* ring_b = ring_a + (size_t)p.SA * p.a_slot;
     uint8_t* epi_buf = ring_b + (size_t)p.SB * p.b_slot;
-    TcShared* sh = reinterpret_cast<TcShared*>(epi_buf + (p.epi_tma ? 2 * (size_t)p.e_slot : 0));
+    uint8_t* ring_raw = epi_buf + (p.epi_tma ? 2 * (size_t)p.e_slot : 0);
+    uint8_t* dummy = ring_raw + (FUSED ? 2 * (size_t)p.raw_slot : 0);   // 2 KB sink for the unused rows of edge blocks
+    TcShared* sh = reinterpret_cast<TcShared*>(dummy + (FUSED ? 2048 : 0));
 
     const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);  // provably warp-uniform
     const int lane = threadIdx.x & 31;
@@ -385,7 +414,8 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     const int spatial = p.kh * p.kw;
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < p.SA; ++i) { mbar_init(smem_u32(&sh->full_a[i]), 1); mbar_init(smem_u32(&sh->empty_a[i]), NI); }
+        for (int i = 0; i < p.SA; ++i) { mbar_init(smem_u32(&sh->full_a[i]), FUSED ? 4 : 1); mbar_init(smem_u32(&sh->empty_a[i]), NI); }
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&sh->raw_full[i]), 1); mbar_init(smem_u32(&sh->raw_empty[i]), 4); }
         for (int i = 0; i < p.SB; ++i) { mbar_init(smem_u32(&sh->full_b[i]), 1); mbar_init(smem_u32(&sh->empty_b[i]), NI); }
         for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&sh->acc_full[i]), NI); mbar_init(smem_u32(&sh->acc_empty[i]), 4); }
         sh->abort_flag = 0;
@@ -404,7 +434,38 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
 
     // ---------------------------------------------------------------- A producer
     if (warp == 0) {
-        if (lane == 0) {
+        if (lane == 0 && FUSED) {
+            // raw boxes [32 ch][BH rows][32 px] straight from x or the cache: tap dt of output frame t reads frame
+            // t+dt of Z = [cache ; x]; columns start 8 pixels left of the tile so that the start is 16-byte aligned
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_a) : "memory");
+            asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_c) : "memory");
+            const uint32_t raw_bytes = (uint32_t)KB * BH * RAW_PX * 2;
+            int s = 0;
+            uint32_t phase = 1;
+            bool ok = true;
+            for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+                int r = tile / p.NT;
+                const int t = r % p.T; r /= p.T;
+                const int tx = r % p.tiles_w; r /= p.tiles_w;
+                const int ty = p.ty_begin + r % p.tiles_h;
+                const int n = r / p.tiles_h;
+                const int h0 = ty * 16, w0 = tx * TW;
+                const int dt0 = (p.first_frame - t > 0) ? p.first_frame - t : 0;
+                for (int dt = dt0; ok && dt < p.kt; ++dt)
+                    for (int cb = 0; ok && cb < p.CB; ++cb) {
+                        if (!(ok = mbar_wait(&sh->raw_empty[s], phase, sh, p, SITE_RAW_EMPTY))) break;
+                        const uint32_t bar = smem_u32(&sh->raw_full[s]);
+                        mbar_expect_tx(bar, raw_bytes);
+                        const int fz = t + dt;
+                        const uint32_t dst = smem_u32(ring_raw + (size_t)s * p.raw_slot);
+                        if (fz < p.tc) tma_load_5d(dst, &tm_c, bar, w0 - 8, h0 - ph, fz, cb * KB, n);
+                        else tma_load_5d(dst, &tm_a, bar, w0 - 8, h0 - ph, fz - p.tc, cb * KB, n);
+                        s ^= 1;
+                        if (s == 0) phase ^= 1;
+                    }
+            }
+            if (!ok) drain_delay();
+        } else if (lane == 0) {
             asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_a) : "memory");
             const uint32_t a_bytes = (uint32_t)BW * BH * ROWB;
             int s = 0;
@@ -601,7 +662,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
         }
     }
     // ---------------------------------------------------------------- epilogue (warps 4..7)
-    else if (warp >= 4) {
+    else if (warp >= 4 && warp < 8) {
         const int q = warp & 3;  // TMEM lane quarter this warp may read
         int acc = 0;
         uint32_t pacc = 0;
@@ -683,6 +744,52 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
             if (++acc == p.ACC) { acc = 0; pacc ^= 1; }
         }
         if (p.epi_tma && elected) bulk_wait_all();   // all stores of this CTA are complete before it exits
+    }
+
+    // ---------------------------------------------------------------- transposers (fused mode, warps 8..11)
+    if (FUSED && warp >= 8) {
+        // raw [c][row][32 px] (64-byte rows, 64-byte swizzle as TMA wrote it) -> halo tile [pixel][32 ch] (64-byte
+        // rows, 64-byte swizzle: the K-major operand).  Per step a warp moves 8 pixels x 32 channels: ldmatrix.trans
+        // reads four 8x8 blocks (one per channel octet, rows = channels), stmatrix writes them with rows = pixels.
+        const int tw = warp - 8;
+        const int colshift = 8 - pw;                       // raw column of halo column 0
+        const int mi = lane >> 3, mj = lane & 7;           // this lane addresses row mj of matrix (channel octet) mi
+        const uint32_t src_lane = (uint32_t)(mi * 8 + mj) * (uint32_t)(BH * RAW_PX * 2);
+        const uint32_t dummy_addr = smem_u32(dummy) + (uint32_t)(tw * 32 + lane) * 16;
+        int rs = 0, sa = 0;
+        uint32_t pr = 0, pea = 1;
+        bool ok = true;
+        for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+            const int t = (tile / p.NT) % p.T;
+            const int dt0 = (p.first_frame - t > 0) ? p.first_frame - t : 0;
+            for (int kb = (p.kt - dt0) * p.CB; ok && kb > 0; --kb) {
+                ok = mbar_wait(&sh->raw_full[rs], pr, sh, p, SITE_RAW_FULL) && mbar_wait(&sh->empty_a[sa], pea, sh, p, SITE_A_EMPTY);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                const uint32_t raw_base = smem_u32(ring_raw + (size_t)rs * p.raw_slot);
+                const uint32_t a_base = smem_u32(ring_a + (size_t)sa * p.a_slot);
+                for (int q = tw; q < BH * 4; q += 4) {
+                    const int hh = q >> 2, wblk = q & 3;
+                    uint32_t so = src_lane + (uint32_t)hh * (RAW_PX * 2) + (uint32_t)wblk * 16;
+                    so ^= ((so >> 7) & 3u) << 4;             // the 64-byte swizzle TMA applied to the raw box
+                    uint32_t frag[4];
+                    ldmatrix_x4_trans(raw_base + so, frag);
+                    const int col = 8 * wblk + mj - colshift;
+                    const uint32_t r = (uint32_t)(hh * BW + col);
+                    const uint32_t dst = (col >= 0 && col < BW) ? a_base + r * 64 + (((uint32_t)mi ^ ((r >> 1) & 3u)) << 4) : dummy_addr;
+                    stmatrix_x4(dst, frag);
+                }
+                fence_async_smem();                        // generic-proxy writes -> visible to the tensor core's reads
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(smem_u32(&sh->full_a[sa]));
+                    mbar_arrive(smem_u32(&sh->raw_empty[rs]));
+                }
+                rs ^= 1;
+                if (rs == 0) pr ^= 1;
+                if (++sa == p.SA) { sa = 0; pea ^= 1; }
+            }
+        }
     }
 
     // ---------------------------------------------------------------- teardown

@@ -156,6 +156,35 @@ def test_bf16_tensor_core_banded_overlap(ccv, N, Cin, Cout, T, H, W, k, cache):
     b.close()
 
 
+FUSED_CASES = [TC_CASES[i] for i in (0, 1, 2, 3, 4, 5, 6, 7, 9, 11, 17, 19, 20, 21)] + [
+    (1, 192, 192, 4, 48, 80, (3, 3, 3), "random", True),     # 256-pixel tiles, several waves
+    (1, 40, 24, 2, 33, 56, (3, 3, 3), None, True),           # Cin not a multiple of 32: channels beyond Cin arrive as zeros
+]
+
+
+@pytest.mark.parametrize("N,Cin,Cout,T,H,W,k,cache,bias", FUSED_CASES)
+def test_bf16_tensor_core_fused_route(ccv, N, Cin, Cout, T, H, W, k, cache, bias):
+    """CCV3D_FLAG_FUSED: no staging copy - the kernel reads x and the cache through tensor maps and transposes in
+    shared memory; the cache update is a separate copy kernel.  (W % 8 != 0 falls back to the staged route.)"""
+    c = si.conv_case(N, Cin, Cout, T, H, W, k=k, cache=cache, bias=bias, seed=15)
+    m, ctr = run_case(ccv, c, flags=ccv.FLAG_FUSED)
+    assert ctr["tcgen05_bf16"] == 1 and ctr["simt"] == 0
+
+
+def test_fused_route_equals_staged_route_bitwise(ccv):
+    c = si.conv_case(1, 96, 192, 3, 40, 64, seed=16)
+    a = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), flags=ccv.FLAG_FUSED)
+    b = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]))
+    x, cache_d = to_dev(c["x"]), to_dev(c["cache"])
+    oa, na = a(x, cache_d)
+    ob, nb = b(x, cache_d)
+    torch.cuda.synchronize()
+    assert torch.equal(oa, ob) and torch.equal(na, nb)          # same K order per output element in both routes
+    assert ccv.ccv3d_workspace_bytes(a.h, 1, 3, 40, 64) == (ccv.OK, 0)
+    a.close()
+    b.close()
+
+
 def test_cfg2_bf16_384(ccv):
     m, ctr = run_case(ccv, si.conv_case(**si.CONFIGS["cfg2_bf16_384"]))
     assert ctr["tcgen05_bf16"] == 1 and m["cos"] > 0.99998
