@@ -182,6 +182,58 @@ def main_reference(args):
     return 0
 
 
+# ---------------------------------------------------------------------------------------------- multi-rank plumbing
+def init_ranks(backend, device=None):
+    """(world, rank, local_rank, dist or None) from the torchrun environment; one process per GPU, replicas only."""
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        if backend == "nccl":
+            dist.init_process_group("nccl", device_id=device)
+        else:
+            dist.init_process_group(backend)
+    return world, rank, local, dist
+
+
+def max_over_ranks(ms_local, dist, device=None):
+    """The slowest rank's time: the job is done when the last replica is."""
+    if dist is None:
+        return float(ms_local)
+    import torch
+    t = torch.tensor([ms_local], dtype=torch.float64, device=device if device is not None else "cpu")
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def weak_scaling_value(world, flops_per_step, ms_per_step):
+    """Whole-job TFLOP/s of `world` independent replicas that each run the full workload."""
+    return world * flops_per_step / (ms_per_step * 1e-3) / 1e12
+
+
+def main_selftest_dist(args):
+    """Host-side check of the multi-rank path without GPUs (gloo): every rank pretends to have measured a
+    rank-dependent step time; rank 0 prints the aggregated line.  Used by tests/test_bench_ranks.py."""
+    world, rank, local, dist = init_ranks("gloo")
+    if dist is not None:
+        dist.barrier()
+    cfg, d = cfg_of(args.workload)
+    flops = si.conv_flops(**d)
+    ms_local = 1.0 + 0.25 * rank                     # the last rank is the slowest
+    ms = max_over_ranks(ms_local * args.steps, dist) / args.steps
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "value": weak_scaling_value(world, flops, ms), "unit": "TFLOP/s",
+                          "n_gpus": world, "steps": args.steps, "ms_per_step": ms, "scaling": "weak",
+                          "selftest": "gloo ranks with fabricated step times"}))
+    return 0
+
+
 # ---------------------------------------------------------------------------------------------- CUDA leg
 def chain_leg(dev):
     """Streamed synthetic decoder chain (configuration 5): 21 one-latent-frame chunks through six cached 3x3x3
@@ -226,16 +278,11 @@ def main_ours(args):
     import torch
     import paper_2609_31938_b200 as ccv
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
     assert torch.cuda.is_available(), "bench.py needs a CUDA device; there is no CPU fallback"
+    local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
+    world, rank, local, dist = init_ranks("nccl", dev)
 
     name = args.workload
     cfg, d = cfg_of(name)
@@ -295,15 +342,12 @@ def main_ours(args):
     launches = layer.counters()["kernel_launches"] - launches0
     assert layer.device_status()[0] == ccv.OK
 
-    if dist is not None:
-        t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, dist, dev)
 
     flops = si.conv_flops(**d)
     abytes = si.conv_bytes(**d)
     ms_step = ms_total / args.steps
-    value = world * flops / (ms_step * 1e-3) / 1e12
+    value = weak_scaling_value(world, flops, ms_step)
 
     # ---- end to end through the host entry point: pinned host buffers, H2D and D2H inside the timed region
     e2e = None
@@ -384,9 +428,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-chain", action="store_true", help="skip the decoder-chain leg")
+    ap.add_argument("--selftest-dist", action="store_true", help=argparse.SUPPRESS)
     ap.add_argument("--flags", type=int, default=0, help="CCV3D_FLAG_* bits for the layer (e.g. 8 = fused route without staging copy)")
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(n for n in si.CONFIGS if "bf16" in n))
     args = ap.parse_args()
+    if args.selftest_dist:
+        return main_selftest_dist(args)
     if args.impl == "reference":
         return main_reference(args)
     return main_ours(args)

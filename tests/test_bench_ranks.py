@@ -1,0 +1,38 @@
+"""The multi-rank path of bench.py without GPUs: two gloo ranks on 127.0.0.1 run the same rendezvous, barrier,
+max-over-ranks and rank-0 reporting code the NCCL run uses (replicas only: no collective on the data path), and
+the reference arm prints from rank 0 only."""
+import json
+import os
+import subprocess
+import sys
+
+import synth_inputs as si
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _torchrun(extra, nproc=2, port=29641):
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={nproc}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.join(ROOT, "bench.py")] + extra
+    env = dict(os.environ, OMP_NUM_THREADS="2")
+    return subprocess.run(cmd, cwd=ROOT, env=env, capture_output=True, text=True, timeout=600)
+
+
+def test_two_ranks_aggregate_to_one_line():
+    r = _torchrun(["--gpus", "2", "--steps", "4", "--selftest-dist"])
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1, r.stdout                         # rank 0 alone reports
+    d = json.loads(lines[0])
+    flops = si.conv_flops(**{k: v for k, v in si.CONFIGS["cfg3_bf16_192"].items() if k in "N Cin Cout T H W k".split()})
+    assert d["n_gpus"] == 2 and d["scaling"] == "weak"
+    assert abs(d["ms_per_step"] - 1.25) < 1e-9                # the slower rank's time
+    assert abs(d["value"] - 2 * flops / 1.25e-3 / 1e12) < 1e-6 * d["value"]
+
+
+def test_single_process_selftest():
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--selftest-dist", "--steps", "2"], cwd=ROOT,
+                       capture_output=True, text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    d = json.loads(r.stdout.strip().splitlines()[-1])
+    assert d["n_gpus"] == 1 and abs(d["ms_per_step"] - 1.0) < 1e-9
