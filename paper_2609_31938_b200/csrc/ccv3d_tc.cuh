@@ -768,16 +768,30 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                 if (!ok) break;
                 const uint32_t raw_base = smem_u32(ring_raw + (size_t)rs * p.raw_slot);
                 const uint32_t a_base = smem_u32(ring_a + (size_t)sa * p.a_slot);
-                for (int q = tw; q < BH * 4; q += 4) {
-                    const int hh = q >> 2, wblk = q & 3;
-                    uint32_t so = src_lane + (uint32_t)hh * (RAW_PX * 2) + (uint32_t)wblk * 16;
-                    so ^= ((so >> 7) & 3u) << 4;             // the 64-byte swizzle TMA applied to the raw box
-                    uint32_t frag[4];
-                    ldmatrix_x4_trans(raw_base + so, frag);
-                    const int col = 8 * wblk + mj - colshift;
-                    const uint32_t r = (uint32_t)(hh * BW + col);
-                    const uint32_t dst = (col >= 0 && col < BW) ? a_base + r * 64 + (((uint32_t)mi ^ ((r >> 1) & 3u)) << 4) : dummy_addr;
-                    stmatrix_x4(dst, frag);
+                // warp tw owns column block tw of every halo row; rows go in batches of TR so that the loads of a
+                // batch are in flight together before its stores
+                constexpr int TR = 6;
+                const int col = 8 * tw + mj - colshift;
+                const bool col_ok = col >= 0 && col < BW;
+                uint32_t so0 = src_lane + (uint32_t)tw * 16;
+                for (int hb = 0; hb < BH; hb += TR) {
+                    uint32_t frag[TR][4];
+#pragma unroll
+                    for (int u = 0; u < TR; ++u) {
+                        if (hb + u < BH) {
+                            uint32_t so = so0 + (uint32_t)(hb + u) * (RAW_PX * 2);
+                            so ^= ((so >> 7) & 3u) << 4;             // the 64-byte swizzle TMA applied to the raw box
+                            ldmatrix_x4_trans(raw_base + so, frag[u]);
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < TR; ++u) {
+                        if (hb + u < BH) {
+                            const uint32_t r = (uint32_t)((hb + u) * BW + col);
+                            const uint32_t dst = col_ok ? a_base + r * 64 + (((uint32_t)mi ^ ((r >> 1) & 3u)) << 4) : dummy_addr;
+                            stmatrix_x4(dst, frag[u]);
+                        }
+                    }
                 }
                 fence_async_smem();                        // generic-proxy writes -> visible to the tensor core's reads
                 __syncwarp();
