@@ -124,6 +124,17 @@ ccv3d_status ccv3d_forward(ccv3d_handle* h, const void* x, const void* cache, vo
                            int32_t N, int32_t T, int32_t H, int32_t W, void* stream);
 
 /*
+ * ccv3d_forward with a history shorter than kt-1 frames (the paper's Table 1 lists such calls: T_c = 1 with
+ * a temporal kernel of 3).  cache is DEVICE [N,cin,cache_frames,H,W] with 0 <= cache_frames <= kt-1 (NULL allowed
+ * only with cache_frames = 0); the kt-1-cache_frames frames before it do not exist and contribute zero, exactly as
+ * Eq. (1)-(3) prescribe with p_l = kt-1-cache_frames (their taps are skipped).  new_cache still receives kt-1
+ * frames, zero where the stream has no history yet.  Everything else as ccv3d_forward, which is this call with
+ * cache_frames = kt-1 (or 0 for a NULL cache).
+ */
+ccv3d_status ccv3d_forward_ex(ccv3d_handle* h, const void* x, const void* cache, int32_t cache_frames, void* out,
+                              void* new_cache, int32_t N, int32_t T, int32_t H, int32_t W, void* stream);
+
+/*
  * ccv3d_forward without any allocation.  (The paper has no counterpart: its route runs inside a framework
  * that allocates freely.)
  *
@@ -159,7 +170,8 @@ ccv3d_status ccv3d_forward_static(ccv3d_handle* h, const void* x, const void* ca
 ccv3d_status ccv3d_forward_host(ccv3d_handle* h, const void* x_host, const void* cache_host, void* out_host,
                                 void* new_cache_host, int32_t N, int32_t T, int32_t H, int32_t W, void* stream);
 
-/* Bytes of handle-owned workspace a forward call of this shape needs (0 for the FP32-FMA path). */
+/* Bytes of handle-owned workspace a forward call of this shape needs (0 for the FP32-FMA route, the 1x1x1
+ * streaming kernel and the fused route). */
 ccv3d_status ccv3d_workspace_bytes(const ccv3d_handle* h, int32_t N, int32_t T, int32_t H, int32_t W,
                                    uint64_t* bytes_host);
 

@@ -41,7 +41,7 @@ class Counters(ctypes.Structure):
 
 EXPORTS = ("ccv3d_create", "ccv3d_forward", "ccv3d_forward_host", "ccv3d_workspace_bytes", "ccv3d_destroy",
            "ccv3d_get_counters", "ccv3d_device_status", "ccv3d_status_string", "ccv3d_add_bf16",
-           "ccv3d_upsample_bf16", "ccv3d_profile_enable", "ccv3d_profile_read", "ccv3d_forward_static", "ccv3d_selftest_wait_timeout")
+           "ccv3d_upsample_bf16", "ccv3d_profile_enable", "ccv3d_profile_read", "ccv3d_forward_static", "ccv3d_selftest_wait_timeout", "ccv3d_forward_ex")
 
 
 def _load() -> ctypes.CDLL:
@@ -53,6 +53,7 @@ def _load() -> ctypes.CDLL:
     vp, i32, u64p = ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(ctypes.c_uint64)
     lib.ccv3d_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(Desc), vp, vp, vp]
     lib.ccv3d_forward.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, vp]
+    lib.ccv3d_forward_ex.argtypes = [vp, vp, vp, i32, vp, vp, i32, i32, i32, i32, vp]
     lib.ccv3d_forward_static.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, vp]
     lib.ccv3d_forward_host.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, vp]
     lib.ccv3d_workspace_bytes.argtypes = [vp, i32, i32, i32, i32, u64p]
@@ -111,6 +112,11 @@ def ccv3d_create(desc: Desc, w_dev: int, b_dev: int | None, stream: int = 0):
 
 def ccv3d_forward(h, x, cache, out, new_cache, N, T, H, W, stream=0) -> int:
     return lib.ccv3d_forward(h, x, cache, out, new_cache, N, T, H, W, stream)
+
+
+def ccv3d_forward_ex(h, x, cache, cache_frames, out, new_cache, N, T, H, W, stream=0) -> int:
+    """ccv3d_forward with a cache of cache_frames <= kt-1 frames (older history absent = zero)."""
+    return lib.ccv3d_forward_ex(h, x, cache, cache_frames, out, new_cache, N, T, H, W, stream)
 
 
 def ccv3d_forward_static(h, x, cache, out, new_cache, N, T, H, W, stream=0) -> int:

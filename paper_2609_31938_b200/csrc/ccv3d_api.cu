@@ -72,6 +72,7 @@ struct ccv3d_handle {
     int prof_on;
     int64_t prof_n;
     cudaEvent_t* prof_ev;   // PROF_SLOTS x 3 events, created on first enable
+    int call_cf;         // history frames held by the cache of the call being served (set by the entry points)
     ccv3d_counters ctr;
 };
 
@@ -264,11 +265,13 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     StageParams sp;
     memset(&sp, 0, sizeof(sp));
     sp.x = (const __nv_bfloat16*)x;
-    sp.cache = tc ? (const __nv_bfloat16*)cache : nullptr;
+    const int cf = (tc && cache) ? h->call_cf : 0;          // older history frames are absent: their taps are skipped
+    sp.cache = cf ? (const __nv_bfloat16*)cache : nullptr;
+    sp.cf = cf;
     sp.zs = (__nv_bfloat16*)h->workspace;
     sp.new_cache = tc ? (__nv_bfloat16*)new_cache : nullptr;
     sp.N = N; sp.Cin = d.cin; sp.T = T; sp.H = H; sp.W = W; sp.tc = tc; sp.CB = pl.CB;
-    sp.f_begin = sp.cache ? 0 : (tc < T ? tc : T);
+    sp.f_begin = (tc - cf) < T ? (tc - cf) : T;
     const int nframes = F - sp.f_begin;
 
     // ---- implicit GEMM parameters ----
@@ -293,7 +296,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     p.CB = pl.CB; p.NT = pl.NT; p.NPAD = pl.NPAD;
     const int tiles_h = (H + 15) / 16;
     p.tiles_w = (W + TW - 1) / TW;
-    p.first_frame = (tc && !cache) ? tc : 0;
+    p.first_frame = tc - cf;
     p.out_f32 = d.out_dtype == CCV3D_F32;
     p.per_tap_a = per_tap;
     p.ACC = ACC;
@@ -430,7 +433,8 @@ ccv3d_status forward_fused(ccv3d_handle* h, const void* x, const void* cache, vo
     const ccv3d_desc& d = h->d;
     const TcPlan& pl = h->plan;
     const int tc = d.kt - 1;
-    if (!tc) cache = nullptr;
+    const int cf = (tc && cache) ? h->call_cf : 0;
+    if (!cf) cache = nullptr;
     int NB = 2;   // 256-pixel tiles: the raw-box requests per FLOP, this route's bottleneck, halve against 128-pixel tiles
     if ((int64_t)N * ((H + 15) / 16) * ((W + 15) / 16) * T * pl.NT < h->sm_count) NB = 1;
     const int ACC = (2 * NB * pl.NPAD <= 512) ? 2 : 1;
@@ -439,14 +443,14 @@ ccv3d_status forward_fused(ccv3d_handle* h, const void* x, const void* cache, vo
     TcParams p;
     memset(&p, 0, sizeof(p));
     p.N = N; p.T = T; p.H = H; p.W = W; p.Cout = d.cout; p.F = tc + T;
-    p.kt = d.kt; p.kh = d.kh; p.kw = d.kw; p.tc = tc;
+    p.kt = d.kt; p.kh = d.kh; p.kw = d.kw; p.tc = tc; p.cf = cf;
     p.CB = pl.CB; p.NT = pl.NT; p.NPAD = pl.NPAD;
     p.tiles_h = (H + 15) / 16;
     p.tiles_w = (W + TW - 1) / TW;
     const int64_t total = (int64_t)N * p.tiles_h * p.tiles_w * T * pl.NT;
     if (total > 0x7FFFFFFF) return CCV3D_ERR_UNSUPPORTED;
     p.total_tiles = (int)total;
-    p.first_frame = (tc && !cache) ? tc : 0;
+    p.first_frame = tc - cf;
     p.ACC = ACC;
     p.a_slot = (uint32_t)align_up((uint64_t)BW * BH * 64, 1024);
     p.raw_slot = (uint32_t)align_up((uint64_t)32 * BH * RAW_PX * 2, 1024);
@@ -483,7 +487,7 @@ ccv3d_status forward_fused(ccv3d_handle* h, const void* x, const void* cache, vo
     ccv3d_status s = encode_ncthw_map(h, &tm_x, x, N, d.cin, T, H, W, RAW_PX, BH, 32, CU_TENSOR_MAP_SWIZZLE_64B);
     if (s != CCV3D_OK) return s;
     if (cache) {
-        s = encode_ncthw_map(h, &tm_c, cache, N, d.cin, tc, H, W, RAW_PX, BH, 32, CU_TENSOR_MAP_SWIZZLE_64B);
+        s = encode_ncthw_map(h, &tm_c, cache, N, d.cin, cf, H, W, RAW_PX, BH, 32, CU_TENSOR_MAP_SWIZZLE_64B);
         if (s != CCV3D_OK) return s;
     } else {
         tm_c = tm_x;   // never dereferenced: the taps that would read the cache are skipped
@@ -503,7 +507,7 @@ ccv3d_status forward_fused(ccv3d_handle* h, const void* x, const void* cache, vo
         const int64_t units = (int64_t)(fbytes / 16);
         dim3 g((unsigned)((units + 255) / 256 > 64 ? 64 : (units + 255) / 256), (unsigned)(planes < 65535 ? planes : 65535));
         cache_update_kernel<uint4><<<g, 256, 0, st>>>((const uint4*)x, (const uint4*)cache, (uint4*)new_cache, d.cin, T, tc,
-                                                     units, planes);
+                                                     cf, units, planes);
         if (cudaGetLastError() != cudaSuccess) return cuda_fail();
         h->ctr.kernel_launches++;
     }
@@ -659,6 +663,7 @@ ccv3d_status forward_tc_static(ccv3d_handle* h, const void* x, const void* cache
     StageParams sp;
     sp.x = (const __nv_bfloat16*)x;
     sp.cache = tc ? (const __nv_bfloat16*)cache : nullptr;
+    sp.cf = sp.cache ? tc : 0;
     sp.zs = (__nv_bfloat16*)scratch;
     sp.new_cache = tc ? (__nv_bfloat16*)new_cache : nullptr;
     sp.N = N; sp.Cin = d.cin; sp.T = T; sp.H = H; sp.W = W; sp.tc = tc; sp.CB = pl.CB;
@@ -767,7 +772,8 @@ ccv3d_status forward_simt(ccv3d_handle* h, const void* x, const void* cache, voi
     const ccv3d_desc& d = h->d;
     const int tc = d.kt - 1;
     SimtParams p;
-    p.x = x; p.cache = tc ? cache : nullptr; p.w = h->w_copy; p.bias = h->bias32; p.out = out;
+    const int cf = (tc && cache) ? h->call_cf : 0;
+    p.x = x; p.cache = cf ? cache : nullptr; p.cf = cf; p.w = h->w_copy; p.bias = h->bias32; p.out = out;
     p.N = N; p.Cin = d.cin; p.Cout = d.cout; p.T = T; p.H = H; p.W = W; p.kt = d.kt; p.kh = d.kh; p.kw = d.kw;
     const int64_t npix = (int64_t)N * T * H * W;
     const int64_t gx = (npix + SIMT_THREADS - 1) / SIMT_THREADS;
@@ -794,17 +800,17 @@ ccv3d_status forward_simt(ccv3d_handle* h, const void* x, const void* cache, voi
             const int64_t units = fbytes / 16;
             dim3 g((unsigned)((units + 255) / 256 > 1024 ? 1024 : (units + 255) / 256), gy);
             cache_update_kernel<uint4><<<g, 256, 0, st>>>((const uint4*)x, (const uint4*)cache, (uint4*)new_cache, d.cin, T,
-                                                          tc, units, planes);
+                                                          tc, cf, units, planes);
         } else if (d.dtype == CCV3D_F32) {
             const int64_t units = (int64_t)H * W;
             dim3 g((unsigned)((units + 255) / 256 > 1024 ? 1024 : (units + 255) / 256), gy);
             cache_update_kernel<uint32_t><<<g, 256, 0, st>>>((const uint32_t*)x, (const uint32_t*)cache,
-                                                             (uint32_t*)new_cache, d.cin, T, tc, units, planes);
+                                                             (uint32_t*)new_cache, d.cin, T, tc, cf, units, planes);
         } else {
             const int64_t units = (int64_t)H * W;
             dim3 g((unsigned)((units + 255) / 256 > 1024 ? 1024 : (units + 255) / 256), gy);
             cache_update_kernel<uint16_t><<<g, 256, 0, st>>>((const uint16_t*)x, (const uint16_t*)cache,
-                                                             (uint16_t*)new_cache, d.cin, T, tc, units, planes);
+                                                             (uint16_t*)new_cache, d.cin, T, tc, cf, units, planes);
         }
         if (cudaGetLastError() != cudaSuccess) return cuda_fail();
         h->ctr.kernel_launches++;
@@ -822,14 +828,15 @@ ccv3d_status check_forward_args(const ccv3d_handle* h, const void* x, const void
     if ((uint64_t)H * W > 0x7FFFFFFFull) return CCV3D_ERR_UNSUPPORTED;
     const int tc = d.kt - 1;
     const uint64_t xb = px * d.cin * T * esize(d.dtype), cb = px * d.cin * tc * esize(d.dtype);
+    const uint64_t ccb = px * d.cin * (uint64_t)h->call_cf * esize(d.dtype);     // bytes of the cache actually passed
     const uint64_t ob = px * d.cout * T * esize(d.out_dtype);
     if (!tc) { cache = nullptr; new_cache = nullptr; }
     if (device_ptrs) {
         const uintptr_t m = (uintptr_t)x | (uintptr_t)cache | (uintptr_t)out | (uintptr_t)new_cache;
         if (m & 15u) return CCV3D_ERR_ALIGNMENT;
     }
-    if (overlap(out, ob, x, xb) || overlap(out, ob, cache, cb)) return CCV3D_ERR_ALIAS;
-    if (overlap(new_cache, cb, x, xb) || overlap(new_cache, cb, cache, cb) || overlap(new_cache, cb, out, ob))
+    if (overlap(out, ob, x, xb) || overlap(out, ob, cache, ccb)) return CCV3D_ERR_ALIAS;
+    if (overlap(new_cache, cb, x, xb) || overlap(new_cache, cb, cache, ccb) || overlap(new_cache, cb, out, ob))
         return CCV3D_ERR_ALIAS;
     return CCV3D_OK;
 }
@@ -965,10 +972,15 @@ ccv3d_status ccv3d_workspace_bytes(const ccv3d_handle* h, int32_t N, int32_t T, 
     return CCV3D_OK;
 }
 
-ccv3d_status ccv3d_forward(ccv3d_handle* h, const void* x, const void* cache, void* out, void* new_cache, int32_t N,
-                           int32_t T, int32_t H, int32_t W, void* stream) {
+ccv3d_status ccv3d_forward_ex(ccv3d_handle* h, const void* x, const void* cache, int32_t cache_frames, void* out,
+                              void* new_cache, int32_t N, int32_t T, int32_t H, int32_t W, void* stream) {
     if (!h) return CCV3D_ERR_INVALID_ARG;
     h->ctr.calls++;
+    const int tc = h->d.kt - 1;
+    if (cache_frames < 0 || cache_frames > tc) return count(h, CCV3D_ERR_INVALID_ARG);
+    if (cache_frames > 0 && !cache) return count(h, CCV3D_ERR_INVALID_ARG);
+    if (cache_frames == 0) cache = nullptr;
+    h->call_cf = cache_frames;
     ccv3d_status s = check_forward_args(h, x, cache, out, new_cache, N, T, H, W, true);
     if (s != CCV3D_OK) return count(h, s);
     cudaStream_t st = (cudaStream_t)stream;
@@ -979,10 +991,17 @@ ccv3d_status ccv3d_forward(ccv3d_handle* h, const void* x, const void* cache, vo
     return count(h, s);
 }
 
+ccv3d_status ccv3d_forward(ccv3d_handle* h, const void* x, const void* cache, void* out, void* new_cache, int32_t N,
+                           int32_t T, int32_t H, int32_t W, void* stream) {
+    if (!h) return CCV3D_ERR_INVALID_ARG;
+    return ccv3d_forward_ex(h, x, cache, cache ? h->d.kt - 1 : 0, out, new_cache, N, T, H, W, stream);
+}
+
 ccv3d_status ccv3d_forward_static(ccv3d_handle* h, const void* x, const void* cache, void* out, void* new_cache,
                                   int32_t N, int32_t T, int32_t H, int32_t W, void* stream) {
     if (!h) return CCV3D_ERR_INVALID_ARG;
     h->ctr.calls++;
+    h->call_cf = cache ? h->d.kt - 1 : 0;
     ccv3d_status s = check_forward_args(h, x, cache, out, new_cache, N, T, H, W, true);
     if (s != CCV3D_OK) return count(h, s);
     if (!h->use_tc) return count(h, CCV3D_ERR_UNSUPPORTED);   // the FP32-FMA route has no scratch to replace
@@ -992,6 +1011,7 @@ ccv3d_status ccv3d_forward_static(ccv3d_handle* h, const void* x, const void* ca
 ccv3d_status ccv3d_forward_host(ccv3d_handle* h, const void* x_host, const void* cache_host, void* out_host,
                                 void* new_cache_host, int32_t N, int32_t T, int32_t H, int32_t W, void* stream) {
     if (!h) return CCV3D_ERR_INVALID_ARG;
+    h->call_cf = cache_host ? h->d.kt - 1 : 0;
     ccv3d_status s = check_forward_args(h, x_host, cache_host, out_host, new_cache_host, N, T, H, W, false);
     if (s != CCV3D_OK) {
         h->ctr.calls++;

@@ -22,12 +22,14 @@ __device__ __forceinline__ void st_from_float(__nv_bfloat16* p, float v) { *p = 
 
 struct SimtParams {
     const void* x;
-    const void* cache;  // may be null: first chunk, absent frames are skipped
+    const void* cache;  // [N,Cin,cf,H,W]; may be null: first chunk, absent frames are skipped
+    int cf;             // history frames the cache holds (0..kt-1); older ones are absent (zero)
     const void* w;      // original [Cout,Cin,kt,kh,kw] order, storage dtype
     const float* bias;  // FP32, [Cout]
     void* out;
     int N, Cin, Cout, T, H, W, kt, kh, kw;
 };
+// Z = [absent x (kt-1-cf) ; cache ; x]: frame tau < kt-1 of Z is cache frame tau-(kt-1-cf) when that is >= 0.
 
 constexpr int SIMT_CO = 8;       // output channels per thread
 constexpr int SIMT_THREADS = 128;
@@ -59,8 +61,9 @@ __global__ void __launch_bounds__(SIMT_THREADS) conv3d_direct_kernel(const SimtP
             const int tau = t + dt;  // frame of Z = [cache ; x]
             const TIn* frame;
             if (tau < tc) {
-                if (!cache) continue;
-                frame = cache + (((int64_t)n * p.Cin + ci) * tc + tau) * HW;
+                const int cfr = tau - (tc - p.cf);
+                if (!cache || cfr < 0) continue;
+                frame = cache + (((int64_t)n * p.Cin + ci) * p.cf + cfr) * HW;
             } else {
                 frame = x + (((int64_t)n * p.Cin + ci) * p.T + (tau - tc)) * HW;
             }
@@ -93,14 +96,15 @@ __global__ void __launch_bounds__(SIMT_THREADS) conv3d_direct_kernel(const SimtP
 // grid.x covers one frame in units, grid.y strides over the N*Cin*(kt-1) planes.
 template <typename U>
 __global__ void cache_update_kernel(const U* __restrict__ x, const U* __restrict__ cache, U* __restrict__ new_cache,
-                                    int Cin, int T, int tc, int64_t frame_units, int64_t planes) {
+                                    int Cin, int T, int tc, int cf, int64_t frame_units, int64_t planes) {
     for (int64_t plane = blockIdx.y; plane < planes; plane += gridDim.y) {  // plane = (n*Cin + ci)*tc + j
         const int j = (int)(plane % tc);
         const int64_t nc = plane / tc;
         const int tau = T + j;
         const U* src = nullptr;
         if (tau < tc) {
-            if (cache) src = cache + (nc * tc + tau) * frame_units;
+            const int cfr = tau - (tc - cf);
+            if (cache && cfr >= 0) src = cache + (nc * cf + cfr) * frame_units;
         } else {
             src = x + (nc * T + (tau - tc)) * frame_units;
         }

@@ -66,7 +66,8 @@ __global__ void pack_weights_kernel(const __nv_bfloat16* __restrict__ w, __nv_bf
 // ------------------------------------------------------------------------------------------------
 struct StageParams {
     const __nv_bfloat16* x;      // [N,Cin,T,H,W]
-    const __nv_bfloat16* cache;  // [N,Cin,tc,H,W] or null
+    const __nv_bfloat16* cache;  // [N,Cin,cf,H,W] or null
+    int cf;                      // history frames the cache holds (0..tc); Z frame f < tc is cache frame f-(tc-cf) if >= 0
     __nv_bfloat16* zs;           // [N][F][CB][H][W][KB], F = tc + T
     __nv_bfloat16* new_cache;    // [N,Cin,tc,H,W] or null
     int N, Cin, T, H, W, tc, CB;
@@ -99,9 +100,10 @@ __global__ void __launch_bounds__(32 * (KB / 8)) stage_frames_kernel(const Stage
     const __nv_bfloat16* src = nullptr;  // base of channel 0 of this (n, frame); channel stride cstride
     int64_t cstride = 0;
     if (f < p.tc) {
-        if (p.cache) {
-            src = p.cache + ((int64_t)n * p.Cin * p.tc + f) * HW;
-            cstride = (int64_t)p.tc * HW;
+        const int cfr = f - (p.tc - p.cf);
+        if (p.cache && cfr >= 0) {
+            src = p.cache + ((int64_t)n * p.Cin * p.cf + cfr) * HW;
+            cstride = (int64_t)p.cf * HW;
         }
     } else {
         src = p.x + ((int64_t)n * p.Cin * p.T + (f - p.tc)) * HW;
@@ -312,7 +314,7 @@ struct TcParams {
     uint32_t a_slot, b_slot, b_tap;  // bytes per ring slot (multiples of 1024) and per tap inside a weight slot
     uint32_t e_slot;          // bytes of one epilogue staging buffer (two are allocated when epi_tma)
     uint32_t raw_slot;        // fused mode: bytes of one raw [32 ch][BH rows][32 px] box (two are allocated)
-    int tc;                   // fused mode: cache frames (kt-1); Z frame f < tc comes from the cache map
+    int tc, cf;               // fused mode: kt-1 and the history frames the cache holds; Z frame f < tc is cache frame f-(tc-cf)
     uint32_t tmem_cols;       // power of two >= NB*NPAD*ACC
     long long wait_limit_clk; // bound of every mbarrier wait, in SM clocks
     const float* bias;        // [NT*NPAD]
@@ -458,7 +460,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                         mbar_expect_tx(bar, raw_bytes);
                         const int fz = t + dt;
                         const uint32_t dst = smem_u32(ring_raw + (size_t)s * p.raw_slot);
-                        if (fz < p.tc) tma_load_5d(dst, &tm_c, bar, w0 - 8, h0 - ph, fz, cb * KB, n);
+                        if (fz < p.tc) tma_load_5d(dst, &tm_c, bar, w0 - 8, h0 - ph, fz - (p.tc - p.cf), cb * KB, n);
                         else tma_load_5d(dst, &tm_a, bar, w0 - 8, h0 - ph, fz - p.tc, cb * KB, n);
                         s ^= 1;
                         if (s == 0) phase ^= 1;

@@ -185,6 +185,37 @@ def test_fused_route_equals_staged_route_bitwise(ccv):
     b.close()
 
 
+@pytest.mark.parametrize("dtype,flags,T", [(si.F32, 0, 3), (si.BF16, 0, 4), (si.BF16, 0, 1), (si.BF16, 8, 4), (si.BF16, 1, 2)])
+def test_short_cache_is_zero_history_in_front(ccv, dtype, flags, T):
+    """ccv3d_forward_ex with one cache frame and a temporal kernel of 3 (the T_c = 1 calls of the paper's Table 1):
+    the missing older frame does not exist, i.e. Eq. (1)-(3) with p_l = 1 - identical to a two-frame cache whose
+    first frame is zero, which is what the oracle is given."""
+    N, Cin, Cout, H, W = 1, 64, 48, 20, 24
+    c = si.conv_case(N, Cin, Cout, T, H, W, dtype=dtype, seed=17)
+    short = np.ascontiguousarray(c["cache"][:, :, 1:])                 # the newest history frame only
+    padded = c["cache"].copy()
+    padded[:, :, 0] = 0
+    ref, ref_nc = oracle.forward(c["x"], padded, c["w"], c["b"])
+    layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), flags=flags)
+    x, cd = to_dev(c["x"]), to_dev(short)
+    odt = torch.float32 if dtype == si.F32 else torch.bfloat16
+    obuf, out = _guarded(ref.shape, odt)
+    nbuf, nc = _guarded((N, Cin, 2, H, W), x.dtype)
+    s = ccv.ccv3d_forward_ex(layer.h, x.data_ptr(), cd.data_ptr(), 1, out.data_ptr(), nc.data_ptr(), N, T, H, W,
+                             torch.cuda.current_stream().cuda_stream)
+    assert s == ccv.OK, ccv.status_string(s)
+    torch.cuda.synchronize()
+    assert layer.device_status()[0] == ccv.OK and _guards_intact(obuf) and _guards_intact(nbuf)
+    check(as_f64(out), ref, "f32" if dtype == si.F32 else "bf16")
+    assert np.array_equal(bits(nc), ref_nc)
+    # argument checks of the extended call
+    assert ccv.ccv3d_forward_ex(layer.h, x.data_ptr(), cd.data_ptr(), 3, out.data_ptr(), nc.data_ptr(), N, T, H, W) \
+        == ccv.ERR_INVALID_ARG
+    assert ccv.ccv3d_forward_ex(layer.h, x.data_ptr(), None, 1, out.data_ptr(), nc.data_ptr(), N, T, H, W) \
+        == ccv.ERR_INVALID_ARG
+    layer.close()
+
+
 def test_cfg2_bf16_384(ccv):
     m, ctr = run_case(ccv, si.conv_case(**si.CONFIGS["cfg2_bf16_384"]))
     assert ctr["tcgen05_bf16"] == 1 and m["cos"] > 0.99998
