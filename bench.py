@@ -3,8 +3,9 @@
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
 
-A step is one ccv3d_forward call (channels-last staging + cache update, then the tcgen05 implicit-GEMM
-kernel) on one synthetic decoder-shaped layer.  The default workload is the 192->192, T=4 + 2-frame cache,
+A step is one ccv3d_forward call (channels-last staging + cache update and the tcgen05 implicit GEMM; in the
+default schedule one kernel does all three, its stager warps running a band ahead of its MMA tiles) on one
+synthetic decoder-shaped layer.  The default workload is the 192->192, T=4 + 2-frame cache,
 352x640, 3x3x3 BF16 layer (the large-spatial configuration the >= 60 %-of-tensor-peak target is quoted on);
 inputs are seeded, synthetic, resident in HBM when the timed region starts, and larger than L2 (no flush
 needed).  One JSON line on stdout.

@@ -52,6 +52,8 @@ typedef enum {
 /* ccv3d_desc.flags */
 #define CCV3D_FLAG_FORCE_SIMT 0x1u      /* BF16 layers: use the plain FP32-FMA kernel instead of the tensor-core kernel */
 #define CCV3D_FLAG_OVERLAP 0x4u          /* tensor-core route: process large images in bands, staging band k+1 on a side stream while band k is convolved */
+#define CCV3D_FLAG_TWO_KERNELS 0x10u     /* tensor-core route: run the staging pass as its own kernel before the convolution kernel instead of
+                                            inside it (cooperative staging, the default when W % 8 == 0) */
 #define CCV3D_FLAG_FUSED 0x8u            /* tensor-core route without scratch memory: no channels-last staging copy; the kernel reads x and the cache
                                             by TMA and transposes in shared memory (needs W % 8 == 0, else the staged route is taken). About as fast as
                                             the default route in short bursts, ~3 % slower sustained; for callers that cannot afford the workspace. */

@@ -25,6 +25,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 constexpr int PROF_SLOTS = 1024;
 constexpr int MAX_BANDS = 4;
+constexpr int MAX_COOP_BANDS = 4096;     // image rows / 16 that cooperative staging can track
 constexpr size_t STAGE_COEXIST_BYTES = 20480;  // shared memory left free for staging blocks next to a convolution CTA
 constexpr size_t SMEM_LIMIT = 232448;  // 227 KB of dynamic shared memory per CTA on sm_100
 
@@ -55,6 +56,7 @@ struct ccv3d_handle {
     void* wp;            // TC route: packed weights (device)
     float* bias32;       // FP32 bias, padded (device)
     unsigned int* status;  // device status word
+    unsigned int* band_ctr;  // cooperative staging: per-band arrival counters (MAX_COOP_BANDS words, device)
     void* workspace;
     uint64_t workspace_bytes;
     // host-entry staging (device buffers)
@@ -197,11 +199,25 @@ uint64_t tc_workspace_bytes(const ccv3d_handle* h, int N, int T, int H, int W) {
 }
 
 template <int KB, int NB, int KS, int TPBC>
-ccv3d_status launch_tc(ccv3d_handle* h, const TcParams& p, size_t smem, int grid, cudaStream_t st) {
-    auto kern = conv3d_tcgen05_kernel<KB, NB, KS, TPBC, false>;
+ccv3d_status launch_tc_coop(ccv3d_handle* h, const TcParams& p, const StageParams& sp, size_t smem, int grid,
+                            cudaStream_t st) {
+    auto kern = conv3d_tcgen05_kernel<KB, NB, KS, TPBC, false, true>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return cuda_fail();
-    kern<<<grid, TC_THREADS, smem, st>>>(h->tm_a, h->tm_a, h->tm_o, p);
+    kern<<<grid, TC_THREADS_FUSED, smem, st>>>(h->tm_a, h->tm_a, h->tm_o, p, sp);
+    if (cudaGetLastError() != cudaSuccess) return cuda_fail();
+    h->ctr.kernel_launches++;
+    return CCV3D_OK;
+}
+
+template <int KB, int NB, int KS, int TPBC>
+ccv3d_status launch_tc(ccv3d_handle* h, const TcParams& p, size_t smem, int grid, cudaStream_t st) {
+    auto kern = conv3d_tcgen05_kernel<KB, NB, KS, TPBC, false, false>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return cuda_fail();
+    StageParams nosp;
+    memset(&nosp, 0, sizeof(nosp));
+    kern<<<grid, TC_THREADS, smem, st>>>(h->tm_a, h->tm_a, h->tm_o, p, nosp);
     if (cudaGetLastError() != cudaSuccess) return cuda_fail();
     h->ctr.kernel_launches++;
     return CCV3D_OK;
@@ -319,7 +335,12 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
         (int64_t)N * tiles_h * p.tiles_w * T * pl.NT >= 2LL * h->sm_count && tiles_h >= 4)
         nbands = tiles_h / 2 < MAX_BANDS ? tiles_h / 2 : MAX_BANDS;
 
-    size_t fixed = 1024 /*alignment slack*/ + align_up(sizeof(TcShared), 128) + 2 * (size_t)p.e_slot;
+    // Cooperative staging (default when W % 8 == 0): the staging pass runs inside the convolution kernel, on four
+    // extra warps per CTA, one band of 16 rows ahead of the tiles that read it.
+    const bool coop = nbands == 1 && !per_tap && !(d.flags & CCV3D_FLAG_TWO_KERNELS) && W % 8 == 0 &&
+                      tiles_h <= MAX_COOP_BANDS && tiles_h >= 4 && pl.KB == 64 &&   // 32-channel blocks: the stagers cannot keep up
+                      (int64_t)N * tiles_h * p.tiles_w * T * pl.NT >= 4LL * h->sm_count;   // small problems: two kernels
+    size_t fixed = 1024 /*alignment slack*/ + align_up(sizeof(TcShared), 128) + 2 * (size_t)p.e_slot + (coop ? 9216 : 0);
     // leave room for staging blocks to be resident next to a convolution CTA when the two overlap
     const size_t limit = nbands > 1 ? SMEM_LIMIT - STAGE_COEXIST_BYTES : SMEM_LIMIT;
     const size_t budget = limit - fixed;
@@ -355,7 +376,31 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     const int ph = (d.kh - 1) / 2;
     cudaEvent_t* pev = (h->prof_on && h->prof_ev) ? h->prof_ev + 3 * (h->prof_n % PROF_SLOTS) : nullptr;
 
-    if (nbands == 1) {
+    if (coop) {
+        if (pev) { cudaEventRecord(pev[0], st); cudaEventRecord(pev[1], st); }
+        if (cudaMemsetAsync(h->band_ctr, 0, (size_t)tiles_h * sizeof(unsigned int), st) != cudaSuccess) return cuda_fail();
+        p.band_ctr = h->band_ctr;
+        p.nbands = tiles_h;
+        p.ty_begin = 0;
+        p.tiles_h = tiles_h;
+        const int64_t total = (int64_t)N * tiles_h * p.tiles_w * T * pl.NT;
+        if (total > 0x7FFFFFFF) return CCV3D_ERR_UNSUPPORTED;
+        p.total_tiles = (int)total;
+        const int grid = p.total_tiles < h->sm_count ? p.total_tiles : h->sm_count;
+#define CCV3D_LAUNCH_COOP(KBv, NBv)                                                                        \
+    do {                                                                                                   \
+        if (ks == 3 && p.TPB == 3) s = launch_tc_coop<KBv, NBv, 3, 3>(h, p, sp, smem, grid, st);           \
+        else if (ks == 3 && p.TPB == 1) s = launch_tc_coop<KBv, NBv, 3, 1>(h, p, sp, smem, grid, st);      \
+        else if (ks == 1) s = launch_tc_coop<KBv, NBv, 1, 1>(h, p, sp, smem, grid, st);                    \
+        else s = launch_tc_coop<KBv, NBv, 0, 0>(h, p, sp, smem, grid, st);                                 \
+    } while (0)
+        if (pl.KB == 64 && NB == 2) CCV3D_LAUNCH_COOP(64, 2);
+        else if (pl.KB == 64) CCV3D_LAUNCH_COOP(64, 1);
+        else if (NB == 2) CCV3D_LAUNCH_COOP(32, 2);
+        else CCV3D_LAUNCH_COOP(32, 1);
+#undef CCV3D_LAUNCH_COOP
+        if (s != CCV3D_OK) return s;
+    } else if (nbands == 1) {
         if (pev) cudaEventRecord(pev[0], st);
         s = launch_stage(h, sp, 0, H, nframes, st);
         if (s != CCV3D_OK) return s;
@@ -405,10 +450,12 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
 template <int NB, int KS, int TPBC>
 ccv3d_status launch_fused(ccv3d_handle* h, const CUtensorMap& tm_x, const CUtensorMap& tm_c, const CUtensorMap& tm_o,
                           const TcParams& p, size_t smem, int grid, cudaStream_t st) {
-    auto kern = conv3d_tcgen05_kernel<32, NB, KS, TPBC, true>;
+    auto kern = conv3d_tcgen05_kernel<32, NB, KS, TPBC, true, false>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return cuda_fail();
-    kern<<<grid, TC_THREADS_FUSED, smem, st>>>(tm_x, tm_c, tm_o, p);
+    StageParams nosp;
+    memset(&nosp, 0, sizeof(nosp));
+    kern<<<grid, TC_THREADS_FUSED, smem, st>>>(tm_x, tm_c, tm_o, p, nosp);
     if (cudaGetLastError() != cudaSuccess) return cuda_fail();
     h->ctr.kernel_launches++;
     return CCV3D_OK;
@@ -637,10 +684,12 @@ ccv3d_status static_scratch_for_current_device(void** out_ptr) {
 template <int KB, int NB, int KS, int TPBC>
 ccv3d_status launch_tc_with_maps(ccv3d_handle* h, const CUtensorMap& tm_a, const CUtensorMap& tm_o, const TcParams& p,
                                  size_t smem, int grid, cudaStream_t st) {
-    auto kern = conv3d_tcgen05_kernel<KB, NB, KS, TPBC, false>;
+    auto kern = conv3d_tcgen05_kernel<KB, NB, KS, TPBC, false, false>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return cuda_fail();
-    kern<<<grid, TC_THREADS, smem, st>>>(tm_a, tm_a, tm_o, p);
+    StageParams nosp;
+    memset(&nosp, 0, sizeof(nosp));
+    kern<<<grid, TC_THREADS, smem, st>>>(tm_a, tm_a, tm_o, p, nosp);
     if (cudaGetLastError() != cudaSuccess) return cuda_fail();
     h->ctr.kernel_launches++;
     return CCV3D_OK;
@@ -897,6 +946,7 @@ ccv3d_status ccv3d_create(ccv3d_handle** out_h, const ccv3d_desc* d, const void*
     };
 
     if (cudaMalloc((void**)&h->status, sizeof(unsigned int)) != cudaSuccess) return fail(CCV3D_ERR_NOMEM);
+    if (cudaMalloc((void**)&h->band_ctr, MAX_COOP_BANDS * sizeof(unsigned int)) != cudaSuccess) return fail(CCV3D_ERR_NOMEM);
     if (cudaMemsetAsync(h->status, 0, sizeof(unsigned int), st) != cudaSuccess) return fail(cuda_fail());
 
     int bias_n = d->cout;
@@ -945,7 +995,7 @@ ccv3d_status ccv3d_create(ccv3d_handle** out_h, const ccv3d_desc* d, const void*
 ccv3d_status ccv3d_destroy(ccv3d_handle* h) {
     if (!h) return CCV3D_OK;
     cudaDeviceSynchronize();
-    void* bufs[] = {h->w_copy, h->wp, h->bias32, h->status, h->workspace, h->hx, h->hc, h->ho, h->hn};
+    void* bufs[] = {h->w_copy, h->wp, h->bias32, h->status, h->band_ctr, h->workspace, h->hx, h->hc, h->ho, h->hn};
     for (void* b : bufs)
         if (b) cudaFree(b);
     for (int i = 0; i < 3; ++i)

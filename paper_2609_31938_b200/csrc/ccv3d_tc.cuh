@@ -165,6 +165,97 @@ __global__ void __launch_bounds__(32 * (KB / 8)) stage_frames_kernel(const Stage
         *reinterpret_cast<uint4*>(dst + (int64_t)(wa + 1) * KB + oct * 8) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
 }
 
+// Addresses of one staging task: image row h, pixels [w0, w0+64), channel block cb of Z frame f of sample n.
+struct StageTask {
+    const __nv_bfloat16* src;   // channel 0 of the source frame at (h, 0), or null (absent history: zeros)
+    int64_t cstride;            // source channel stride
+    __nv_bfloat16* ncdst;       // channel 0 of the new-cache frame at (h, 0), or null
+    __nv_bfloat16* dst;         // channels-last destination of pixel (h, 0)
+    int cb, w0;
+};
+
+__device__ __forceinline__ StageTask make_stage_task(const StageParams& p, int KB, int n, int f, int cb, int h, int w0) {
+    StageTask t;
+    const int F = p.tc + p.T;
+    const int64_t HW = (int64_t)p.H * p.W;
+    t.src = nullptr;
+    t.cstride = 0;
+    if (f < p.tc) {
+        const int cfr = f - (p.tc - p.cf);
+        if (p.cache && cfr >= 0) {
+            t.src = p.cache + ((int64_t)n * p.Cin * p.cf + cfr) * HW + (int64_t)h * p.W;
+            t.cstride = (int64_t)p.cf * HW;
+        }
+    } else {
+        t.src = p.x + ((int64_t)n * p.Cin * p.T + (f - p.tc)) * HW + (int64_t)h * p.W;
+        t.cstride = (int64_t)p.T * HW;
+    }
+    const int jc = f - p.T;
+    t.ncdst = nullptr;
+    if (p.new_cache && jc >= 0 && jc < p.tc) t.ncdst = p.new_cache + ((int64_t)n * p.Cin * p.tc + jc) * HW + (int64_t)h * p.W;
+    t.dst = p.zs + ((((int64_t)n * F + f) * p.CB + cb) * HW + (int64_t)h * p.W) * KB;
+    t.cb = cb;
+    t.w0 = w0;
+    return t;
+}
+
+// The same tile move as stage_frames_kernel<KB, true>, run by the 128 threads of the stager warps inside the
+// convolution kernel (cooperative staging): [KB channels][64 pixels] of an image row -> [64 pixels][KB channels],
+// plus the cache update when the frame belongs to the new cache.  Split in two so that the loads of several
+// tasks can be in flight before the first is written: stage_task_load fills val[], stage_task_store moves it
+// through `tile` (KB*33 words of shared memory; phases separated by the stagers' named barrier, id 2).
+__device__ __forceinline__ void stager_bar() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
+
+template <int KB>
+__device__ __forceinline__ void stage_task_load(const StageParams& p, const StageTask& t, int tid, uint4 (&val)[KB * 8 / 128]) {
+#pragma unroll
+    for (int k = 0; k < KB * 8 / 128; ++k) {
+        const int i = tid + 128 * k;
+        const int c = i >> 3, v = i & 7;
+        const int ci = t.cb * KB + c;
+        const int w = t.w0 + v * 8;
+        val[k] = make_uint4(0u, 0u, 0u, 0u);
+        if (w < p.W && ci < p.Cin && t.src) val[k] = __ldg(reinterpret_cast<const uint4*>(t.src + ci * t.cstride + w));
+    }
+}
+
+template <int KB>
+__device__ __forceinline__ void stage_task_store(const StageParams& p, const StageTask& t, int tid,
+                                                 const uint4 (&val)[KB * 8 / 128], uint32_t* tile) {
+    constexpr int PITCH = STG_PX / 2 + 1;
+    constexpr int OCT = KB / 8;
+    const int64_t ncstride = (int64_t)p.tc * p.H * p.W;
+#pragma unroll
+    for (int k = 0; k < KB * 8 / 128; ++k) {
+        const int i = tid + 128 * k;
+        const int c = i >> 3, v = i & 7;
+        const int ci = t.cb * KB + c;
+        const int w = t.w0 + v * 8;
+        if (t.ncdst && w < p.W && ci < p.Cin) *reinterpret_cast<uint4*>(t.ncdst + ci * ncstride + w) = val[k];
+        uint32_t* row = tile + c * PITCH + v * 4;
+        row[0] = val[k].x; row[1] = val[k].y; row[2] = val[k].z; row[3] = val[k].w;
+    }
+    stager_bar();
+#pragma unroll
+    for (int k = 0; k < (32 * OCT) / 128; ++k) {
+        const int vt = tid + 128 * k;
+        const int oct = vt % OCT, pp = vt / OCT;
+        uint32_t lo[4], hi[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const uint32_t a = tile[(oct * 8 + 2 * q) * PITCH + pp];
+            const uint32_t b = tile[(oct * 8 + 2 * q + 1) * PITCH + pp];
+            lo[q] = __byte_perm(a, b, 0x5410);
+            hi[q] = __byte_perm(a, b, 0x7632);
+        }
+        const int wa = t.w0 + 2 * pp;
+        if (wa < p.W) *reinterpret_cast<uint4*>(t.dst + (int64_t)wa * KB + oct * 8) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        if (wa + 1 < p.W)
+            *reinterpret_cast<uint4*>(t.dst + (int64_t)(wa + 1) * KB + oct * 8) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+    }
+    stager_bar();                                           // the tile may be overwritten by the next task
+}
+
 // ------------------------------------------------------------------------------------------------
 // PTX wrappers (sm_100a)
 // ------------------------------------------------------------------------------------------------
@@ -317,6 +408,8 @@ struct TcParams {
     int tc, cf;               // fused mode: kt-1 and the history frames the cache holds; Z frame f < tc is cache frame f-(tc-cf)
     uint32_t tmem_cols;       // power of two >= NB*NPAD*ACC
     long long wait_limit_clk; // bound of every mbarrier wait, in SM clocks
+    unsigned int* band_ctr;   // cooperative staging: per 16-row band, the number of CTAs that have staged their share
+    int nbands;               // cooperative staging: bands of the image (= tile rows)
     const float* bias;        // [NT*NPAD]
     const uint8_t* wq;        // packed weight tiles [dt][cb][nt][sp] of b_tap bytes each
     void* out;
@@ -325,7 +418,7 @@ struct TcParams {
 
 enum : uint32_t {
     SITE_A_EMPTY = 1, SITE_B_EMPTY = 2, SITE_A_FULL = 3, SITE_B_FULL = 4, SITE_ACC_EMPTY = 5, SITE_ACC_FULL = 6,
-    SITE_RAW_EMPTY = 7, SITE_RAW_FULL = 8
+    SITE_RAW_EMPTY = 7, SITE_RAW_FULL = 8, SITE_BAND = 9
 };
 
 constexpr int TC_THREADS = 256;
@@ -384,12 +477,19 @@ __device__ __forceinline__ uint32_t make_desc_lo(uint32_t addr) {
 // into straight-line code with immediate descriptor offsets; KS = 0 keeps everything run-time (any odd kh, kw,
 // and the per-tap A mode).
 // FUSED: no staging copy; tm_a is x as (w, h, t, c, n), tm_c the cache as (w, h, frame, c, n); needs KB = 32.
-template <int KB, int NB, int KS, int TPBC, bool FUSED>
-__global__ void __launch_bounds__(FUSED ? TC_THREADS_FUSED : TC_THREADS, 1)
+// COOP: cooperative staging - there is no separate staging kernel; four extra warps of every CTA move the
+// channels-last copy of [cache ; x] (and the cache update) band by band of 16 image rows, ahead of the tiles that
+// read it, so that this HBM-bound work hides under the tensor-core work of the same kernel.  A band is usable
+// when every CTA has signalled it (release: fence + atomic; acquire: polled load + proxy fence before the TMA
+// loads).  All CTAs are co-resident (grid <= SM count, 1 CTA per SM) and stagers never wait on consumers, so the
+// dependency is acyclic; the wait is bounded like every other.
+template <int KB, int NB, int KS, int TPBC, bool FUSED, bool COOP>
+__global__ void __launch_bounds__((FUSED || COOP) ? TC_THREADS_FUSED : TC_THREADS, 1)
 conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged activations (c, w, h, cb, n*F+f), or x
                       const __grid_constant__ CUtensorMap tm_c,   // fused mode: the cache
                       const __grid_constant__ CUtensorMap tm_o,   // out (w, h, t, co, n); used when p.epi_tma
-                      const TcParams p) {
+                      const TcParams p, const StageParams sp) {
+    static_assert(!(FUSED && COOP), "one or the other");
     static_assert(!FUSED || KB == 32, "the fused mode transposes 32-channel blocks");
     constexpr uint32_t ROWB = KB * 2;                       // bytes per pixel row (one swizzle span)
     constexpr uint32_t LAYOUT = (KB == 64) ? 2u : 4u;       // 128-byte / 64-byte swizzle
@@ -406,7 +506,8 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     uint8_t* epi_buf = ring_b + (size_t)p.SB * p.b_slot;
     uint8_t* ring_raw = epi_buf + (p.epi_tma ? 2 * (size_t)p.e_slot : 0);
     uint8_t* dummy = ring_raw + (FUSED ? 2 * (size_t)p.raw_slot : 0);   // 2 KB sink for the unused rows of edge blocks
-    TcShared* sh = reinterpret_cast<TcShared*>(dummy + (FUSED ? 2048 : 0));
+    uint32_t* coop_tile = reinterpret_cast<uint32_t*>(ring_raw);          // COOP: KB*33 words for the stagers
+    TcShared* sh = reinterpret_cast<TcShared*>(dummy + (FUSED ? 2048 : 0) + (COOP ? 9216 : 0));
 
     const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);  // provably warp-uniform
     const int lane = threadIdx.x & 31;
@@ -473,6 +574,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
             int s = 0;
             uint32_t phase = 1;
             bool ok = true;
+            int bands_ready = 0;                       // COOP: bands [0, bands_ready) are known to be staged
             for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
                 int r = tile / p.NT;
                 const int t = r % p.T; r /= p.T;
@@ -480,6 +582,26 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                 const int ty = p.ty_begin + r % p.tiles_h;
                 const int n = r / p.tiles_h;
                 const int h0 = ty * 16, w0 = tx * TW;
+                if (COOP) {
+                    // the halo of tile row ty reaches into bands ty-1 .. ty+1
+                    const int need = (ty + 2 < p.nbands) ? ty + 2 : p.nbands;
+                    if (bands_ready < need) {
+                        const long long t0 = clock64();
+                        while (ok && bands_ready < need) {
+                            unsigned int v;
+                            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p.band_ctr + bands_ready) : "memory");
+                            if (v >= gridDim.x) { ++bands_ready; continue; }
+                            if (sh->abort_flag) ok = false;
+                            else if (clock64() - t0 > p.wait_limit_clk) {
+                                sh->abort_flag = 1;
+                                atomicCAS(p.status, 0u, (blockIdx.x << 8) | SITE_BAND);
+                                ok = false;
+                            } else __nanosleep(200);
+                        }
+                        if (!ok) break;
+                        asm volatile("fence.proxy.async;" ::: "memory");   // other SMs' generic writes -> this SM's TMA reads
+                    }
+                }
                 const int dt0 = (p.first_frame - t > 0) ? p.first_frame - t : 0;
                 for (int dt = dt0; ok && dt < p.kt; ++dt)
                     for (int cb = 0; ok && cb < p.CB; ++cb) {
@@ -746,6 +868,45 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
             if (++acc == p.ACC) { acc = 0; pacc ^= 1; }
         }
         if (p.epi_tma && elected) bulk_wait_all();   // all stores of this CTA are complete before it exits
+    }
+
+    // ---------------------------------------------------------------- stagers (cooperative staging, warps 8..11)
+    if (COOP && warp >= 8) {
+        const int tid = threadIdx.x - 256;
+        const int nchunks = (sp.W + STG_PX - 1) / STG_PX;
+        const int nf = sp.tc + sp.T - sp.f_begin;
+        // Stagers wait on nothing but their own named barrier, so they always run to completion (also when a
+        // consumer role of some CTA has given up on a wait): every thread of the four warps takes every branch.
+        for (int b = 0; b < p.nbands; ++b) {
+            const int h_lo = 16 * b;
+            const int rows = (sp.H - h_lo < 16) ? sp.H - h_lo : 16;
+            const int ntask = sp.N * nf * sp.CB * rows * nchunks;
+            constexpr int G = (KB == 64) ? 2 : 4;            // tasks whose loads are in flight together (16 KB per CTA)
+            for (int task0 = blockIdx.x; task0 < ntask; task0 += G * gridDim.x) {
+                StageTask tk[G];
+                uint4 val[G][KB * 8 / 128];
+#pragma unroll
+                for (int g = 0; g < G; ++g) {
+                    const int task = task0 + g * gridDim.x;
+                    if (task < ntask) {
+                        int r = task;
+                        const int wc = r % nchunks; r /= nchunks;
+                        const int h = h_lo + r % rows; r /= rows;
+                        const int cb = r % sp.CB; r /= sp.CB;
+                        const int f = sp.f_begin + r % nf;
+                        const int n = r / nf;
+                        tk[g] = make_stage_task(sp, KB, n, f, cb, h, wc * STG_PX);
+                        stage_task_load<KB>(sp, tk[g], tid, val[g]);
+                    }
+                }
+#pragma unroll
+                for (int g = 0; g < G; ++g)
+                    if (task0 + g * gridDim.x < ntask) stage_task_store<KB>(sp, tk[g], tid, val[g], coop_tile);
+            }
+            __threadfence();                               // this thread's stores are visible GPU-wide ...
+            stager_bar();                                  // ... for all 128 stager threads, before the band is signalled
+            if (tid == 0) atomicAdd(p.band_ctr + b, 1u);
+        }
     }
 
     // ---------------------------------------------------------------- transposers (fused mode, warps 8..11)

@@ -216,6 +216,27 @@ def test_short_cache_is_zero_history_in_front(ccv, dtype, flags, T):
     layer.close()
 
 
+def test_bf16_tensor_core_cooperative_staging(ccv):
+    """Large enough for the default schedule to stage inside the convolution kernel (four stager warps per CTA, a
+    band of 16 rows ahead of the tiles that read it): one launch per call, and the same bits as the two-kernel
+    schedule."""
+    c = si.conv_case(1, 64, 64, 8, 125, 160, seed=18)                # 8 tile rows (ragged last), 640 tiles
+    m, ctr = run_case(ccv, c)
+    assert ctr["tcgen05_bf16"] == 1 and ctr["kernel_launches"] == 3    # weight pack, bias, one fused staging+convolution launch
+    a = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]))
+    b = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), flags=ccv.FLAG_TWO_KERNELS)
+    x, cache_d = to_dev(c["x"]), to_dev(c["cache"])
+    oa, na = a(x, cache_d)
+    ob, nb = b(x, cache_d)
+    oa2, na2 = a(x[:, :, :3].contiguous(), None)                       # first chunk, T < tile count threshold: two kernels
+    torch.cuda.synchronize()
+    assert torch.equal(oa, ob) and torch.equal(na, nb)
+    assert b.counters()["kernel_launches"] == 4
+    assert a.device_status()[0] == ccv.OK and bool(torch.isfinite(oa2).all())
+    a.close()
+    b.close()
+
+
 def test_cfg2_bf16_384(ccv):
     m, ctr = run_case(ccv, si.conv_case(**si.CONFIGS["cfg2_bf16_384"]))
     assert ctr["tcgen05_bf16"] == 1 and m["cos"] > 0.99998
