@@ -34,10 +34,10 @@ import synth_inputs as si  # noqa: E402
 METRIC = "causal Conv3D BF16 TFLOP/s"
 DEFAULT_WORKLOAD = "cfg3_bf16_192"
 
-# DRAM bytes (read + write) of one launch of the convolution kernel, from an ncu capture of a quarter-size
-# case (192->192, T=4, 176x320: 133.2 MB read + 53.0 MB written) scaled by the pixel count; the summary is
-# profiles/conv3d_tcgen05_192ch_176x320.md.
-TRAFFIC_BYTES_PER_LAUNCH = {"cfg3_bf16_192": 4 * (133.2e6 + 53.0e6)}
+# DRAM bytes (read + write) of one launch of the step's kernel (default schedule: staging, cache update and
+# convolution in one kernel), from an ncu capture of a quarter-size case (192->192, T=4, 176x320: 241.4 MB read +
+# 222.6 MB written) scaled by the pixel count; the summary is profiles/conv3d_tcgen05_coop_192ch_176x320.md.
+TRAFFIC_BYTES_PER_LAUNCH = {"cfg3_bf16_192": 4 * (241.4e6 + 222.6e6)}
 
 
 def measured_peaks():

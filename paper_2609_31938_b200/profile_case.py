@@ -26,10 +26,11 @@ def main():
     ap.add_argument("--k", type=int, nargs=3, default=[3, 3, 3])
     ap.add_argument("--calls", type=int, default=3)
     ap.add_argument("--no-cache", action="store_true")
+    ap.add_argument("--flags", type=int, default=0, help="CCV3D_FLAG_* bits (16 = two-kernel schedule, 8 = fused route)")
     a = ap.parse_args()
     c = si.conv_case(1, a.cin, a.cout, a.t, a.h, a.w, k=tuple(a.k), cache=None if a.no_cache else "random")
     up = lambda v: None if v is None else torch.from_numpy(v.view(np.int16)).cuda().view(torch.bfloat16)
-    layer = ccv.CausalConv3d(up(c["w"]), up(c["b"]))
+    layer = ccv.CausalConv3d(up(c["w"]), up(c["b"]), flags=a.flags)
     x, cache = up(c["x"]), up(c["cache"])
     out = torch.empty((1, a.cout, a.t, a.h, a.w), dtype=torch.bfloat16, device="cuda")
     nc = torch.empty_like(cache) if cache is not None else None
