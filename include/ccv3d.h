@@ -227,6 +227,68 @@ ccv3d_status ccv3d_add_bf16(const void* a, const void* b, void* y, int64_t n, vo
 ccv3d_status ccv3d_upsample_bf16(const void* x, void* y, int32_t N, int32_t C, int32_t T, int32_t H, int32_t W,
                                  int32_t rt, void* stream);
 
+/*
+ * ------------------------------------------------------------------------------------------------
+ * Resident activations: frame rings in the tensor-core operand order
+ * ------------------------------------------------------------------------------------------------
+ * Algorithm 1 ends every call by restoring the framework layout and returning a contiguous tensor, and
+ * Section 7.2 names the temporaries around the call (folded inputs, the cache concatenation, accumulation
+ * buffers) as the overhead that is left.  Between two layers of one decoder nobody needs the framework layout,
+ * so this library can keep the activations in the order its tensor-core kernel consumes, and keep the temporal
+ * history in place instead of copying a cache:
+ *
+ *   a frame ring is a DEVICE BF16 buffer  [N][F][C/KB][H][W][KB]  (KB = 64 or 32 channels innermost),
+ *   F >= T + kt - 1 frame slots used modulo F.
+ *
+ * A layer reads its input x from slots x_slot .. x_slot+T-1 (mod F) of its input ring and its history from the
+ * kt-1 slots before x_slot - the frames a previous call left there, so Eq. (1)'s source frame of tap dt for
+ * output t is simply slot x_slot + t + dt - (kt-1), and there is no cache tensor, no concatenation and no cache
+ * update.  It writes its output either into the next layer's ring (channels-last, by TMA store) or as NCTHW.
+ * An optional residual (a ring holding cout channels) is added in the epilogue with the chain's rounding:
+ *   out = bf16( float(bf16(conv + b)) + float(res) ),
+ * i.e. bit-identical to ccv3d_forward followed by ccv3d_add_bf16.
+ * Results are those of ccv3d_forward on the same values (same accumulation order per output element).
+ * Rings have no width restriction (any W; the NCTHW TMA paths need W % 8 == 0).
+ */
+typedef struct {
+    void*   base;        /* DEVICE, 16-byte aligned, ccv3d_ring_bytes() bytes; owned by the caller */
+    int32_t N, C, F, H, W;
+    int32_t KB;          /* channels per innermost block: 64 or 32; C % KB == 0.  A ring read by a layer must use
+                            KB = 64 if cin % 64 == 0 else 32 (ccv3d_ring_kb(cin)). */
+} ccv3d_ring;
+
+/* 64 if C % 64 == 0, 32 if C % 32 == 0, else 0 (such a tensor cannot live in a ring). */
+int32_t ccv3d_ring_kb(int32_t C);
+/* N*F*C*H*W*2, or 0 for an invalid geometry. */
+uint64_t ccv3d_ring_bytes(const ccv3d_ring* r);
+
+/* x DEVICE [N,C,T,H,W] BF16 -> ring slots (slot0 + t) mod F, t < T <= F.  Stream-ordered. */
+ccv3d_status ccv3d_ring_load(const ccv3d_ring* r, int32_t slot0, const void* x, int32_t T, void* stream);
+/* ring slots (slot0 + t) mod F -> y DEVICE [N,C,T,H,W] BF16 (bit-exact inverse of ccv3d_ring_load). */
+ccv3d_status ccv3d_ring_store(const ccv3d_ring* r, int32_t slot0, void* y, int32_t T, void* stream);
+/* Nearest-neighbour 2x2 spatial upsample with frame repeat rt between rings of equal C and KB:
+ * out slot (out_slot0 + t*rt + j) mod F_out <- in slot (in_slot0 + t) mod F_in, j < rt; out->H = 2*in->H,
+ * out->W = 2*in->W. */
+ccv3d_status ccv3d_upsample_ring(const ccv3d_ring* in, int32_t in_slot0, const ccv3d_ring* out, int32_t out_slot0,
+                                 int32_t T, int32_t rt, void* stream);
+
+/*
+ * One forward call on resident activations (BF16 tensor-core layers only; others: CCV3D_ERR_UNSUPPORTED).
+ *   in          ring with C = cin, KB = ccv3d_ring_kb(cin), F >= T + kt - 1; x frame t is slot (x_slot + t) mod F.
+ *   hist_frames how many of the kt-1 slots before x_slot hold history (0..kt-1); older ones do not exist and
+ *               contribute zero (first chunks).  The caller advances x_slot by T per call, so the history is
+ *               whatever the previous calls wrote; nothing is copied.
+ *   res         optional ring with C = cout (any KB), same N, H, W: residual frame t is slot (res_slot + t) mod F.
+ *               May be the input ring itself.  Requires out_dtype BF16.
+ *   out_ring    ring with C = cout, same N, H, W; output frame t goes to slot (out_slot + t) mod F (only those
+ *               slots are written).  Must not overlap `in` or `res`.  Requires cout/ceil(cout/256) % 32 == 0.
+ *   out_ncthw   DEVICE [N,cout,T,H,W] in out_dtype.  Exactly one of out_ring / out_ncthw is non-NULL.
+ * All ring structs are HOST pointers read during the call.  Stream-ordered, allocates nothing.
+ */
+ccv3d_status ccv3d_forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int32_t x_slot, int32_t hist_frames,
+                                const ccv3d_ring* res, int32_t res_slot, const ccv3d_ring* out_ring,
+                                int32_t out_slot, void* out_ncthw, int32_t T, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

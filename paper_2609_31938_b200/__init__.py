@@ -40,9 +40,17 @@ class Counters(ctypes.Structure):
                                                "cuda_error", "device_timeout", "kernel_launches")]
 
 
+class Ring(ctypes.Structure):
+    """ccv3d_ring: a frame ring [N][F][C/KB][H][W][KB] of BF16 activations on the device."""
+    _fields_ = [("base", ctypes.c_void_p), ("N", ctypes.c_int32), ("C", ctypes.c_int32), ("F", ctypes.c_int32),
+                ("H", ctypes.c_int32), ("W", ctypes.c_int32), ("KB", ctypes.c_int32)]
+
+
 EXPORTS = ("ccv3d_create", "ccv3d_forward", "ccv3d_forward_host", "ccv3d_workspace_bytes", "ccv3d_destroy",
            "ccv3d_get_counters", "ccv3d_device_status", "ccv3d_status_string", "ccv3d_add_bf16",
-           "ccv3d_upsample_bf16", "ccv3d_profile_enable", "ccv3d_profile_read", "ccv3d_forward_static", "ccv3d_selftest_wait_timeout", "ccv3d_forward_ex")
+           "ccv3d_upsample_bf16", "ccv3d_profile_enable", "ccv3d_profile_read", "ccv3d_forward_static", "ccv3d_selftest_wait_timeout", "ccv3d_forward_ex",
+           "ccv3d_ring_kb", "ccv3d_ring_bytes", "ccv3d_ring_load", "ccv3d_ring_store", "ccv3d_upsample_ring",
+           "ccv3d_forward_ring")
 
 
 def _load() -> ctypes.CDLL:
@@ -69,9 +77,17 @@ def _load() -> ctypes.CDLL:
     lib.ccv3d_selftest_wait_timeout.argtypes = [vp, i32, vp]
     lib.ccv3d_add_bf16.argtypes = [vp, vp, vp, ctypes.c_int64, vp]
     lib.ccv3d_upsample_bf16.argtypes = [vp, vp, i32, i32, i32, i32, i32, i32, vp]
+    rp = ctypes.POINTER(Ring)
+    lib.ccv3d_ring_kb.argtypes = [i32]
+    lib.ccv3d_ring_bytes.argtypes = [rp]
+    lib.ccv3d_ring_load.argtypes = [rp, i32, vp, i32, vp]
+    lib.ccv3d_ring_store.argtypes = [rp, i32, vp, i32, vp]
+    lib.ccv3d_upsample_ring.argtypes = [rp, i32, rp, i32, i32, i32, vp]
+    lib.ccv3d_forward_ring.argtypes = [vp, rp, i32, i32, rp, i32, rp, i32, vp, i32, vp]
     for name in EXPORTS:
-        if name != "ccv3d_status_string":
+        if name not in ("ccv3d_status_string", "ccv3d_ring_bytes"):
             getattr(lib, name).restype = ctypes.c_int
+    lib.ccv3d_ring_bytes.restype = ctypes.c_uint64
     return lib
 
 
@@ -176,6 +192,65 @@ def ccv3d_upsample_bf16(x, y, N, C, T, H, W, rt, stream=0) -> int:
     return lib.ccv3d_upsample_bf16(x, y, N, C, T, H, W, rt, stream)
 
 
+def ccv3d_ring_kb(C: int) -> int:
+    return lib.ccv3d_ring_kb(C)
+
+
+def ccv3d_ring_bytes(ring: Ring) -> int:
+    return int(lib.ccv3d_ring_bytes(ctypes.byref(ring)))
+
+
+def ccv3d_ring_load(ring: Ring, slot0: int, x: int, T: int, stream=0) -> int:
+    return lib.ccv3d_ring_load(ctypes.byref(ring), slot0, x, T, stream)
+
+
+def ccv3d_ring_store(ring: Ring, slot0: int, y: int, T: int, stream=0) -> int:
+    return lib.ccv3d_ring_store(ctypes.byref(ring), slot0, y, T, stream)
+
+
+def ccv3d_upsample_ring(rin: Ring, in_slot0: int, rout: Ring, out_slot0: int, T: int, rt: int, stream=0) -> int:
+    return lib.ccv3d_upsample_ring(ctypes.byref(rin), in_slot0, ctypes.byref(rout), out_slot0, T, rt, stream)
+
+
+def ccv3d_forward_ring(h, rin: Ring, x_slot: int, hist_frames: int, res: Ring | None, res_slot: int,
+                       out_ring: Ring | None, out_slot: int, out_ncthw: int | None, T: int, stream=0) -> int:
+    return lib.ccv3d_forward_ring(h, ctypes.byref(rin), x_slot, hist_frames,
+                                  None if res is None else ctypes.byref(res), res_slot,
+                                  None if out_ring is None else ctypes.byref(out_ring), out_slot, out_ncthw, T, stream)
+
+
+class FrameRing:
+    """A frame ring on the current CUDA device: torch owns the memory, `c` is the struct the C calls take."""
+
+    def __init__(self, N, C, F, H, W, zero=False):
+        import torch
+        kb = ccv3d_ring_kb(C)
+        if kb == 0:
+            raise ValueError(f"{C} channels cannot live in a frame ring (need a multiple of 32)")
+        self.N, self.C, self.F, self.H, self.W, self.KB = N, C, F, H, W, kb
+        alloc = torch.zeros if zero else torch.empty
+        self.buf = alloc((N, F, C // kb, H, W, kb), dtype=torch.bfloat16, device="cuda")
+        self.c = Ring(self.buf.data_ptr(), N, C, F, H, W, kb)
+        self._stream = lambda: torch.cuda.current_stream().cuda_stream
+
+    def load(self, slot0, x):
+        """x [N,C,T,H,W] -> slots slot0.. (mod F)."""
+        assert x.is_cuda and x.is_contiguous() and x.shape[:2] == (self.N, self.C) and x.shape[3:] == (self.H, self.W)
+        s = ccv3d_ring_load(self.c, slot0, x.data_ptr(), x.shape[2], self._stream())
+        if s != OK:
+            raise Ccv3dError(s, "ccv3d_ring_load")
+
+    def store(self, slot0, T, y=None):
+        """slots slot0.. (mod F) -> y [N,C,T,H,W]."""
+        import torch
+        if y is None:
+            y = torch.empty((self.N, self.C, T, self.H, self.W), dtype=torch.bfloat16, device="cuda")
+        s = ccv3d_ring_store(self.c, slot0, y.data_ptr(), T, self._stream())
+        if s != OK:
+            raise Ccv3dError(s, "ccv3d_ring_store")
+        return y
+
+
 class CausalConv3d:
     """One cached causal Conv3D layer on the current CUDA device (torch tensors in, torch tensors out)."""
 
@@ -217,6 +292,16 @@ class CausalConv3d:
         return out, new_cache
 
     __call__ = forward
+
+    def forward_ring(self, rin: FrameRing, x_slot, hist_frames, T, out_ring: FrameRing | None = None, out_slot=0,
+                     out=None, res: FrameRing | None = None, res_slot=0):
+        """The layer on resident activations (see ccv3d_forward_ring): reads `rin`, writes `out_ring` or NCTHW `out`."""
+        s = ccv3d_forward_ring(self.h, rin.c, x_slot, hist_frames, None if res is None else res.c, res_slot,
+                               None if out_ring is None else out_ring.c, out_slot,
+                               None if out is None else out.data_ptr(), T, self.torch.cuda.current_stream().cuda_stream)
+        if s != OK:
+            raise Ccv3dError(s, "ccv3d_forward_ring")
+        return out_ring if out_ring is not None else out
 
     def counters(self):
         return ccv3d_get_counters(self.h)

@@ -14,7 +14,7 @@ normalisation or non-linearity: the chain exists to exercise streaming, caches a
 """
 from __future__ import annotations
 
-from . import CausalConv3d, Ccv3dError, OK, ccv3d_add_bf16, ccv3d_upsample_bf16
+from . import CausalConv3d, Ccv3dError, FrameRing, OK, ccv3d_add_bf16, ccv3d_upsample_bf16, ccv3d_upsample_ring
 
 LAYERS = ("A1", "A2", "PA", "B1", "B2", "PB", "C1", "C2")
 
@@ -61,6 +61,80 @@ class DecoderChain:
         c = self._up(self._conv("PB", b), 1)
         c = self._add(c, self._conv("C2", self._conv("C1", c)))
         return c
+
+    def close(self):
+        for l in self.layers.values():
+            l.close()
+
+
+class ResidentDecoderChain:
+    """The same chain with every activation between the chunk input and the chunk output resident in frame rings
+    (channels-last blocks, the order the tensor-core kernel reads): a layer writes straight into the next layer's
+    ring, the temporal history of a layer is whatever earlier chunks left in its ring (no cache tensors, no cache
+    update), and the residual additions run in the convolution epilogues.  Per chunk: one layout move for the
+    input, eight convolution kernels, two upsample kernels.  Results are bit-identical to DecoderChain."""
+
+    def __init__(self, weights: dict, biases: dict):
+        import torch
+        self.torch = torch
+        self.layers = {n: CausalConv3d(weights[n], biases[n]) for n in LAYERS}
+        self.ch = {n: (weights[n].shape[1], weights[n].shape[0]) for n in LAYERS}   # (cin, cout)
+        self.geom = None
+        self.reset()
+
+    def reset(self):
+        """Forget all temporal state (next chunk is a first chunk)."""
+        self.seen = 0            # latent frames consumed since the last reset
+        self.slot = {"A": 0, "B": 0, "C": 0}
+
+    def _alloc(self, N, T, H, W):
+        ca, cb, cc = self.ch["A1"][0], self.ch["B1"][0], self.ch["C1"][0]
+        R = FrameRing
+        self.rings = {
+            "A1": R(N, ca, T + 2, H, W), "A2": R(N, ca, T + 2, H, W), "PA": R(N, ca, T, H, W), "UA": R(N, cb, T, H, W),
+            "B1": R(N, cb, 4 * T + 2, 2 * H, 2 * W), "B2": R(N, cb, 4 * T + 2, 2 * H, 2 * W),
+            "PB": R(N, cb, 4 * T, 2 * H, 2 * W), "UB": R(N, cc, 4 * T, 2 * H, 2 * W),
+            "C1": R(N, cc, 4 * T + 2, 4 * H, 4 * W), "C2": R(N, cc, 4 * T + 2, 4 * H, 4 * W),
+        }
+        self.geom = (N, T, H, W)
+
+    def _up(self, rin, rout, out_slot, T, rt):
+        s = ccv3d_upsample_ring(rin.c, 0, rout.c, out_slot, T, rt, self.torch.cuda.current_stream().cuda_stream)
+        if s != OK:
+            raise Ccv3dError(s, "ccv3d_upsample_ring")
+
+    def _block(self, first, second, nxt, slot, hist, T, out=None):
+        """x <- x + conv2(conv1(x)) with x in ring `first`: the sum goes to ring `nxt` (slot 0) or to NCTHW `out`."""
+        r, L = self.rings, self.layers
+        L[first].forward_ring(r[first], slot, hist, T, out_ring=r[second], out_slot=slot)
+        if out is None:
+            L[second].forward_ring(r[second], slot, hist, T, out_ring=r[nxt], out_slot=0, res=r[first], res_slot=slot)
+        else:
+            L[second].forward_ring(r[second], slot, hist, T, out=out, res=r[first], res_slot=slot)
+
+    def step(self, a, out=None):
+        """One chunk: a [N,C_a,T,H,W] BF16 -> [N,C_c,4T,4H,4W] BF16 (T at most the first chunk's T after a reset
+        or a change of geometry)."""
+        N, C, T, H, W = a.shape
+        if self.geom is None or self.geom[0] != N or self.geom[2:] != (H, W) or T > self.geom[1]:
+            self._alloc(N, T, H, W)
+            self.reset()
+        r, L = self.rings, self.layers
+        if out is None:
+            out = self.torch.empty((N, self.ch["C2"][1], 4 * T, 4 * H, 4 * W), dtype=a.dtype, device=a.device)
+        sa, sb, sc = self.slot["A"], self.slot["B"], self.slot["C"]
+        ha, hb = min(2, self.seen), min(2, 4 * self.seen)
+        r["A1"].load(sa, a)
+        self._block("A1", "A2", "PA", sa, ha, T)
+        L["PA"].forward_ring(r["PA"], 0, 0, T, out_ring=r["UA"], out_slot=0)
+        self._up(r["UA"], r["B1"], sb, T, 4)
+        self._block("B1", "B2", "PB", sb, hb, 4 * T)
+        L["PB"].forward_ring(r["PB"], 0, 0, 4 * T, out_ring=r["UB"], out_slot=0)
+        self._up(r["UB"], r["C1"], sc, 4 * T, 1)
+        self._block("C1", "C2", None, sc, hb, 4 * T, out=out)
+        self.seen += T
+        self.slot = {"A": (sa + T) % r["A1"].F, "B": (sb + 4 * T) % r["B1"].F, "C": (sc + 4 * T) % r["C1"].F}
+        return out
 
     def close(self):
         for l in self.layers.values():

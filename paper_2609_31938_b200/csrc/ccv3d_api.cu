@@ -816,6 +816,181 @@ ccv3d_status forward_tc_static(ccv3d_handle* h, const void* x, const void* cache
     return s;
 }
 
+// ------------------------------------------------------------------------------------------------
+// Resident activations: frame rings [N][F][C/KB][H][W][KB] in the tensor-core operand order.  The convolution
+// kernel reads its halo tiles straight from the input ring (history = the slots before x, left there by earlier
+// calls), and writes the next layer's ring, so a chain of layers needs no staging pass, no cache tensor and no
+// cache update.
+// ------------------------------------------------------------------------------------------------
+bool ring_valid(const ccv3d_ring* r) {
+    if (!r || !r->base) return false;
+    if (r->N < 1 || r->C < 1 || r->F < 1 || r->H < 1 || r->W < 1) return false;
+    if (r->KB != 64 && r->KB != 32) return false;
+    if (r->C % r->KB) return false;
+    if ((uint64_t)r->H * r->W > 0x7FFFFFFFull) return false;
+    return true;
+}
+
+uint64_t ring_bytes_of(const ccv3d_ring* r) { return (uint64_t)r->N * r->F * r->C * r->H * r->W * 2; }
+
+RingGeom ring_geom(const ccv3d_ring* r) {
+    RingGeom g;
+    g.base = (__nv_bfloat16*)r->base;
+    g.N = r->N; g.F = r->F; g.CB = r->C / r->KB; g.H = r->H; g.W = r->W; g.KB = r->KB;
+    return g;
+}
+
+// Tensor map over a ring as (channel in block, w, h, channel block, n*F + slot).
+ccv3d_status encode_ring_map(ccv3d_handle* h, CUtensorMap* tm, const ccv3d_ring* r, int box_c, int box_w, int box_h,
+                             CUtensorMapSwizzle swz) {
+    const uint64_t rowb = (uint64_t)r->KB * 2;
+    cuuint64_t dims[5] = {(cuuint64_t)r->KB, (cuuint64_t)r->W, (cuuint64_t)r->H, (cuuint64_t)(r->C / r->KB),
+                          (cuuint64_t)r->N * r->F};
+    cuuint64_t strides[4] = {rowb, rowb * r->W, rowb * r->W * r->H, rowb * r->W * r->H * (r->C / r->KB)};
+    cuuint32_t box[5] = {(cuuint32_t)box_c, (cuuint32_t)box_w, (cuuint32_t)box_h, 1, 1};
+    cuuint32_t es[5] = {1, 1, 1, 1, 1};
+    CUresult rc = h->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, r->base, dims, strides, box, es,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return rc == CUDA_SUCCESS ? CCV3D_OK : CCV3D_ERR_CUDA;
+}
+
+ccv3d_status forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int x_slot, int hist, const ccv3d_ring* res, int res_slot,
+                          const ccv3d_ring* oring, int out_slot, void* out_ncthw, int T, cudaStream_t st) {
+    const ccv3d_desc& d = h->d;
+    const TcPlan& pl = h->plan;
+    const int tc = d.kt - 1;
+    if (!h->use_tc || (d.flags & CCV3D_FLAG_TC_PER_TAP_A)) return CCV3D_ERR_UNSUPPORTED;
+    if (!ring_valid(in) || T < 1 || (oring != nullptr) == (out_ncthw != nullptr)) return CCV3D_ERR_INVALID_ARG;
+    if (((uintptr_t)in->base | (uintptr_t)out_ncthw) & 15u) return CCV3D_ERR_ALIGNMENT;
+    if (in->C != d.cin || in->F < T + tc || x_slot < 0 || x_slot >= in->F || hist < 0 || hist > tc) return CCV3D_ERR_INVALID_ARG;
+    if (in->KB != pl.KB) return CCV3D_ERR_UNSUPPORTED;
+    const int N = in->N, H = in->H, W = in->W;
+    const bool chunked = (d.cout / pl.NT) % 32 == 0 && pl.NT * pl.NPAD == d.cout;   // whole 32-channel chunks per tile
+    if (res) {
+        if (!ring_valid(res) || res->C != d.cout || res->N != N || res->H != H || res->W != W || res->F < T || res_slot < 0 ||
+            res_slot >= res->F)
+            return CCV3D_ERR_INVALID_ARG;
+        if ((uintptr_t)res->base & 15u) return CCV3D_ERR_ALIGNMENT;
+        if (d.out_dtype != CCV3D_BF16 || !chunked) return CCV3D_ERR_UNSUPPORTED;
+    }
+    const uint64_t in_b = ring_bytes_of(in);
+    if (oring) {
+        if (!ring_valid(oring) || oring->C != d.cout || oring->N != N || oring->H != H || oring->W != W || oring->F < T ||
+            out_slot < 0 || out_slot >= oring->F)
+            return CCV3D_ERR_INVALID_ARG;
+        if ((uintptr_t)oring->base & 15u) return CCV3D_ERR_ALIGNMENT;
+        if (d.out_dtype != CCV3D_BF16 || !chunked) return CCV3D_ERR_UNSUPPORTED;
+        if (overlap(oring->base, ring_bytes_of(oring), in->base, in_b) ||
+            (res && overlap(oring->base, ring_bytes_of(oring), res->base, ring_bytes_of(res))))
+            return CCV3D_ERR_ALIAS;
+    } else {
+        const uint64_t ob = (uint64_t)N * d.cout * T * H * W * esize(d.out_dtype);
+        if (overlap(out_ncthw, ob, in->base, in_b) || (res && overlap(out_ncthw, ob, res->base, ring_bytes_of(res))))
+            return CCV3D_ERR_ALIAS;
+    }
+
+    int NB = pl.NB;
+    if ((int64_t)N * ((H + 15) / 16) * ((W + 15) / 16) * T * pl.NT < h->sm_count) NB = 1;
+    const int ACC = (2 * NB * pl.NPAD <= 512) ? 2 : 1;
+    const int TW = 8 * NB, BW = TW + d.kw - 1, BH = 16 + d.kh - 1;
+    CUtensorMap tm_a, tm_o;
+    ccv3d_status s = encode_ring_map(h, &tm_a, in, pl.KB, BW, BH, pl.KB == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B);
+    if (s != CCV3D_OK) return s;
+
+    TcParams p;
+    memset(&p, 0, sizeof(p));
+    p.N = N; p.T = T; p.H = H; p.W = W; p.Cout = d.cout;
+    p.F = in->F;
+    p.f0 = (x_slot - tc + in->F) % in->F;
+    p.kt = d.kt; p.kh = d.kh; p.kw = d.kw;
+    p.CB = pl.CB; p.NT = pl.NT; p.NPAD = pl.NPAD;
+    p.tiles_h = (H + 15) / 16;
+    p.tiles_w = (W + TW - 1) / TW;
+    const int64_t total = (int64_t)N * p.tiles_h * p.tiles_w * T * pl.NT;
+    if (total > 0x7FFFFFFF) return CCV3D_ERR_UNSUPPORTED;
+    p.total_tiles = (int)total;
+    p.first_frame = tc - hist;
+    p.out_f32 = d.out_dtype == CCV3D_F32;
+    p.ACC = ACC;
+    p.a_slot = (uint32_t)align_up((uint64_t)BW * BH * pl.KB * 2, 1024);
+    p.b_tap = (uint32_t)pl.NPAD * pl.KB * 2;
+    if (oring) {
+        p.epi_tma = 2;
+        p.ECH = 32;
+        p.e_slot = (uint32_t)(16 * TW * 64);
+        p.out_F = oring->F; p.out_f0 = out_slot; p.out_KB = oring->KB;
+        s = encode_ring_map(h, &tm_o, oring, 32, TW, 16, CU_TENSOR_MAP_SWIZZLE_64B);
+        if (s != CCV3D_OK) return s;
+    } else {
+        p.epi_tma = (!p.out_f32 && W % 8 == 0) ? 1 : 0;
+        p.ECH = (pl.NPAD % 32 == 0) ? 32 : 16;
+        p.e_slot = p.epi_tma ? (uint32_t)(p.ECH * 16 * TW * 2) : 0;
+        if (p.epi_tma) {
+            cuuint64_t dims[5] = {(cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)T, (cuuint64_t)d.cout, (cuuint64_t)N};
+            cuuint64_t strides[4] = {2ull * W, 2ull * W * H, 2ull * W * H * T, 2ull * W * H * T * d.cout};
+            cuuint32_t box[5] = {(cuuint32_t)TW, 16, 1, (cuuint32_t)p.ECH, 1};
+            cuuint32_t es[5] = {1, 1, 1, 1, 1};
+            if (h->encode(&tm_o, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, out_ncthw, dims, strides, box, es,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+                return CCV3D_ERR_CUDA;
+        } else {
+            tm_o = tm_a;   // never dereferenced on this path
+        }
+    }
+    if (res) {
+        p.res = (const __nv_bfloat16*)res->base;
+        p.res_F = res->F; p.res_f0 = res_slot; p.res_CB = res->C / res->KB; p.res_KB = res->KB;
+    }
+    const size_t fixed = 1024 + align_up(sizeof(TcShared), 128) + 2 * (size_t)p.e_slot;
+    const size_t budget = SMEM_LIMIT - fixed;
+    p.TPB = ((size_t)p.b_tap * d.kw <= 40960) ? d.kw : 1;
+    int SA = 2;
+    for (;;) {
+        p.b_slot = (uint32_t)align_up((uint64_t)p.b_tap * p.TPB, 1024);
+        if ((size_t)SA * p.a_slot + 3 * (size_t)p.b_slot <= budget) break;
+        if (p.TPB > 1) { p.TPB = 1; continue; }
+        if ((size_t)SA * p.a_slot + 2 * (size_t)p.b_slot <= budget) break;
+        return CCV3D_ERR_UNSUPPORTED;
+    }
+    int SB = (int)((budget - (size_t)SA * p.a_slot) / p.b_slot);
+    if (SB > 8) SB = 8;
+    while (SA < 4 && (size_t)(SA + 1) * p.a_slot + (size_t)SB * p.b_slot <= budget) ++SA;
+    p.SA = SA; p.SB = SB;
+    p.tmem_cols = pow2_cols((uint32_t)(NB * pl.NPAD * ACC));
+    if (p.tmem_cols > 512) return CCV3D_ERR_UNSUPPORTED;
+    p.wait_limit_clk = h->wait_limit_clk;
+    p.bias = h->bias32;
+    p.wq = (const uint8_t*)h->wp;
+    p.out = out_ncthw;
+    p.status = h->status;
+    const size_t smem = fixed + (size_t)SA * p.a_slot + (size_t)SB * p.b_slot;
+    const int grid = p.total_tiles < h->sm_count ? p.total_tiles : h->sm_count;
+    const int ks = (d.kh == d.kw && (d.kh == 1 || d.kh == 3)) ? d.kh : 0;
+    cudaEvent_t* pev = (h->prof_on && h->prof_ev) ? h->prof_ev + 3 * (h->prof_n % PROF_SLOTS) : nullptr;
+    if (pev) { cudaEventRecord(pev[0], st); cudaEventRecord(pev[1], st); }
+#define CCV3D_LAUNCH_RING(KBv, NBv)                                                                              \
+    do {                                                                                                         \
+        if (ks == 3 && p.TPB == 3) s = launch_tc_with_maps<KBv, NBv, 3, 3>(h, tm_a, tm_o, p, smem, grid, st);    \
+        else if (ks == 3 && p.TPB == 1) s = launch_tc_with_maps<KBv, NBv, 3, 1>(h, tm_a, tm_o, p, smem, grid, st); \
+        else if (ks == 1) s = launch_tc_with_maps<KBv, NBv, 1, 1>(h, tm_a, tm_o, p, smem, grid, st);             \
+        else s = launch_tc_with_maps<KBv, NBv, 0, 0>(h, tm_a, tm_o, p, smem, grid, st);                          \
+    } while (0)
+    if (pl.KB == 64 && NB == 2) CCV3D_LAUNCH_RING(64, 2);
+    else if (pl.KB == 64) CCV3D_LAUNCH_RING(64, 1);
+    else if (NB == 2) CCV3D_LAUNCH_RING(32, 2);
+    else CCV3D_LAUNCH_RING(32, 1);
+#undef CCV3D_LAUNCH_RING
+    if (s != CCV3D_OK) return s;
+    h->ctr.tcgen05_bf16++;
+    if (pev) {
+        cudaEventRecord(pev[2], st);
+        h->prof_n++;
+    }
+    return CCV3D_OK;
+}
+
 ccv3d_status forward_simt(ccv3d_handle* h, const void* x, const void* cache, void* out, void* new_cache, int N, int T,
                           int H, int W, cudaStream_t st) {
     const ccv3d_desc& d = h->d;
@@ -1181,6 +1356,75 @@ ccv3d_status ccv3d_upsample_bf16(const void* x, void* y, int32_t N, int32_t C, i
         upsample_bf16_kernel<<<grid, 256, 0, (cudaStream_t)stream>>>((const __nv_bfloat16*)x, (__nv_bfloat16*)y,
                                                                    (int64_t)N * C, T, H, W, rt);
     return cudaGetLastError() == cudaSuccess ? CCV3D_OK : cuda_fail();
+}
+
+int32_t ccv3d_ring_kb(int32_t C) { return C < 1 ? 0 : (C % 64 == 0 ? 64 : (C % 32 == 0 ? 32 : 0)); }
+
+uint64_t ccv3d_ring_bytes(const ccv3d_ring* r) {
+    if (!r || r->N < 1 || r->C < 1 || r->F < 1 || r->H < 1 || r->W < 1) return 0;
+    if ((r->KB != 64 && r->KB != 32) || r->C % r->KB) return 0;
+    return ring_bytes_of(r);
+}
+
+ccv3d_status ccv3d_ring_load(const ccv3d_ring* r, int32_t slot0, const void* x, int32_t T, void* stream) {
+    if (!ring_valid(r) || !x || T < 1 || T > r->F || slot0 < 0 || slot0 >= r->F) return CCV3D_ERR_INVALID_ARG;
+    if (((uintptr_t)r->base | (uintptr_t)x) & 15u) return CCV3D_ERR_ALIGNMENT;
+    if (overlap(r->base, ring_bytes_of(r), x, (uint64_t)r->N * r->C * T * r->H * r->W * 2)) return CCV3D_ERR_ALIAS;
+    StageParams sp;
+    memset(&sp, 0, sizeof(sp));
+    sp.x = (const __nv_bfloat16*)x;
+    sp.zs = (__nv_bfloat16*)r->base;
+    sp.N = r->N; sp.Cin = r->C; sp.T = T; sp.H = r->H; sp.W = r->W; sp.tc = 0; sp.CB = r->C / r->KB;
+    sp.ring_F = r->F; sp.ring_f0 = slot0;
+    const bool vec = (r->W % 8 == 0);
+    dim3 grid((r->W + STG_PX - 1) / STG_PX, r->H, (unsigned)((int64_t)r->N * T * sp.CB));
+    if (r->H > 65535 || (int64_t)r->N * T * sp.CB > 65535) return CCV3D_ERR_UNSUPPORTED;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (r->KB == 64) {
+        if (vec) stage_frames_kernel<64, true><<<grid, 256, 0, st>>>(sp);
+        else stage_frames_kernel<64, false><<<grid, 256, 0, st>>>(sp);
+    } else {
+        if (vec) stage_frames_kernel<32, true><<<grid, 128, 0, st>>>(sp);
+        else stage_frames_kernel<32, false><<<grid, 128, 0, st>>>(sp);
+    }
+    return cudaGetLastError() == cudaSuccess ? CCV3D_OK : cuda_fail();
+}
+
+ccv3d_status ccv3d_ring_store(const ccv3d_ring* r, int32_t slot0, void* y, int32_t T, void* stream) {
+    if (!ring_valid(r) || !y || T < 1 || T > r->F || slot0 < 0 || slot0 >= r->F) return CCV3D_ERR_INVALID_ARG;
+    if (((uintptr_t)r->base | (uintptr_t)y) & 15u) return CCV3D_ERR_ALIGNMENT;
+    if (overlap(r->base, ring_bytes_of(r), y, (uint64_t)r->N * r->C * T * r->H * r->W * 2)) return CCV3D_ERR_ALIAS;
+    const int CB = r->C / r->KB;
+    if (r->H > 65535 || (int64_t)r->N * T * CB > 65535) return CCV3D_ERR_UNSUPPORTED;
+    dim3 grid((r->W + STG_PX - 1) / STG_PX, r->H, (unsigned)((int64_t)r->N * T * CB));
+    cudaStream_t st = (cudaStream_t)stream;
+    if (r->KB == 64) ring_store_kernel<64><<<grid, 256, 0, st>>>(ring_geom(r), slot0, T, r->C, (__nv_bfloat16*)y);
+    else ring_store_kernel<32><<<grid, 256, 0, st>>>(ring_geom(r), slot0, T, r->C, (__nv_bfloat16*)y);
+    return cudaGetLastError() == cudaSuccess ? CCV3D_OK : cuda_fail();
+}
+
+ccv3d_status ccv3d_upsample_ring(const ccv3d_ring* in, int32_t in_slot0, const ccv3d_ring* out, int32_t out_slot0,
+                                 int32_t T, int32_t rt, void* stream) {
+    if (!ring_valid(in) || !ring_valid(out) || T < 1 || rt < 1 || T > in->F || (int64_t)T * rt > out->F) return CCV3D_ERR_INVALID_ARG;
+    if (in_slot0 < 0 || in_slot0 >= in->F || out_slot0 < 0 || out_slot0 >= out->F) return CCV3D_ERR_INVALID_ARG;
+    if (out->N != in->N || out->C != in->C || out->KB != in->KB || out->H != 2 * in->H || out->W != 2 * in->W)
+        return CCV3D_ERR_INVALID_ARG;
+    if (((uintptr_t)in->base | (uintptr_t)out->base) & 15u) return CCV3D_ERR_ALIGNMENT;
+    if (overlap(in->base, ring_bytes_of(in), out->base, ring_bytes_of(out))) return CCV3D_ERR_ALIAS;
+    const int64_t total = (int64_t)in->N * T * (in->C / 8) * in->H * in->W;
+    const int64_t blocks = (total + 255) / 256;
+    ring_upsample_kernel<<<(unsigned)(blocks < 65536 ? blocks : 65536), 256, 0, (cudaStream_t)stream>>>(
+        ring_geom(in), in_slot0, ring_geom(out), out_slot0, T, rt);
+    return cudaGetLastError() == cudaSuccess ? CCV3D_OK : cuda_fail();
+}
+
+ccv3d_status ccv3d_forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int32_t x_slot, int32_t hist_frames,
+                                const ccv3d_ring* res, int32_t res_slot, const ccv3d_ring* out_ring,
+                                int32_t out_slot, void* out_ncthw, int32_t T, void* stream) {
+    if (!h) return CCV3D_ERR_INVALID_ARG;
+    h->ctr.calls++;
+    return count(h, forward_ring(h, in, x_slot, hist_frames, res, res_slot, out_ring, out_slot, out_ncthw, T,
+                                 (cudaStream_t)stream));
 }
 
 }  // extern "C"

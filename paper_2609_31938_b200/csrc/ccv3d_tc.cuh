@@ -73,6 +73,8 @@ struct StageParams {
     int N, Cin, T, H, W, tc, CB;
     int f_begin;                 // first Z frame to stage (tc when there is no cache and nothing older is needed)
     int h_begin;                 // first image row of this launch (grid.y rows are staged)
+    int ring_F = 0, ring_f0 = 0; // ring_F > 0 (separate staging kernel only): zs is a frame ring of ring_F slots and
+                                 // Z frame f goes to slot (ring_f0 + f) mod ring_F
 };
 
 constexpr int STG_PX = 64;  // pixels of one image row handled per block
@@ -158,11 +160,84 @@ __global__ void __launch_bounds__(32 * (KB / 8)) stage_frames_kernel(const Stage
         lo[k] = __byte_perm(a, b, 0x5410);                            // pixel 2pp:   (ch 2k, ch 2k+1)
         hi[k] = __byte_perm(a, b, 0x7632);                            // pixel 2pp+1
     }
-    __nv_bfloat16* dst = p.zs + ((((int64_t)n * F + f) * p.CB + cb) * HW + (int64_t)h * p.W) * KB;
+    const int FS = p.ring_F > 0 ? p.ring_F : F;         // frame slots per sample
+    int fs = p.ring_f0 + f;
+    if (fs >= FS) fs -= FS;
+    __nv_bfloat16* dst = p.zs + ((((int64_t)n * FS + fs) * p.CB + cb) * HW + (int64_t)h * p.W) * KB;
     const int wa = w0 + 2 * pp;
     if (wa < p.W) *reinterpret_cast<uint4*>(dst + (int64_t)wa * KB + oct * 8) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
     if (wa + 1 < p.W)
         *reinterpret_cast<uint4*>(dst + (int64_t)(wa + 1) * KB + oct * 8) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
+}
+
+// ------------------------------------------------------------------------------------------------
+// frame rings: the inverse move (ring -> NCTHW) and the nearest-neighbour upsample between rings
+// ------------------------------------------------------------------------------------------------
+struct RingGeom {
+    __nv_bfloat16* base;         // [N][F][CB][H][W][KB]
+    int N, F, CB, H, W, KB;
+};
+
+// grid: (ceil(W/64), H, N*T*CB); block 256.  [64 pixels][KB channels] of an image row -> KB channel rows of 64 pixels.
+template <int KB>
+__global__ void __launch_bounds__(256) ring_store_kernel(const RingGeom r, int slot0, int T, int C, __nv_bfloat16* __restrict__ y) {
+    constexpr int PITCH = KB + 2;                         // BF16 elements per pixel row (+2: bank spread)
+    __shared__ __align__(16) unsigned short tile[STG_PX * PITCH];
+    int z = blockIdx.z;
+    const int cb = z % r.CB; z /= r.CB;
+    const int t = z % T;
+    const int n = z / T;
+    const int h = blockIdx.y;
+    const int w0 = blockIdx.x * STG_PX;
+    const int64_t HW = (int64_t)r.H * r.W;
+    int fs = slot0 + t;
+    if (fs >= r.F) fs -= r.F;
+    const __nv_bfloat16* src = r.base + ((((int64_t)n * r.F + fs) * r.CB + cb) * HW + (int64_t)h * r.W + w0) * KB;
+    const int npx = (r.W - w0 < STG_PX) ? r.W - w0 : STG_PX;
+    constexpr int OCT = KB / 8;
+    for (int i = threadIdx.x; i < npx * OCT; i += 256) {   // contiguous 16-byte chunks
+        const int px = i / OCT, oct = i % OCT;
+        const uint4 u = __ldg(reinterpret_cast<const uint4*>(src) + i);
+        uint32_t* d = reinterpret_cast<uint32_t*>(tile + px * PITCH + oct * 8);
+        d[0] = u.x; d[1] = u.y; d[2] = u.z; d[3] = u.w;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < KB * STG_PX; i += 256) {
+        const int c = i / STG_PX, px = i % STG_PX;
+        if (px < npx)
+            reinterpret_cast<unsigned short*>(y)[(((int64_t)n * C + cb * KB + c) * T + t) * HW + (int64_t)h * r.W + w0 + px] =
+                tile[px * PITCH + c];
+    }
+}
+
+// One thread per 16-byte chunk of the source frames; each chunk is written to 2x2 pixels of rt output frames.
+__global__ void __launch_bounds__(256) ring_upsample_kernel(const RingGeom in, int in_slot0, const RingGeom out, int out_slot0,
+                                                            int T, int rt) {
+    const int OCT = in.KB / 8;
+    const int64_t per_frame = (int64_t)in.CB * in.H * in.W * OCT;
+    const int64_t total = (int64_t)in.N * T * per_frame;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        int64_t q = i;
+        const int oct = (int)(q % OCT); q /= OCT;
+        const int w = (int)(q % in.W); q /= in.W;
+        const int h = (int)(q % in.H); q /= in.H;
+        const int cb = (int)(q % in.CB); q /= in.CB;
+        const int t = (int)(q % T);
+        const int n = (int)(q / T);
+        int fs = in_slot0 + t;
+        if (fs >= in.F) fs -= in.F;
+        const uint4 u = __ldg(reinterpret_cast<const uint4*>(
+            in.base + ((((int64_t)n * in.F + fs) * in.CB + cb) * in.H * in.W + (int64_t)h * in.W + w) * in.KB + oct * 8));
+        for (int j = 0; j < rt; ++j) {
+            int os = (out_slot0 + t * rt + j) % out.F;
+            __nv_bfloat16* o = out.base + ((((int64_t)n * out.F + os) * out.CB + cb) * out.H * out.W +
+                                           (int64_t)(2 * h) * out.W + 2 * w) * out.KB + oct * 8;
+            *reinterpret_cast<uint4*>(o) = u;
+            *reinterpret_cast<uint4*>(o + out.KB) = u;
+            *reinterpret_cast<uint4*>(o + (int64_t)out.W * out.KB) = u;
+            *reinterpret_cast<uint4*>(o + (int64_t)(out.W + 1) * out.KB) = u;
+        }
+    }
 }
 
 // Addresses of one staging task: image row h, pixels [w0, w0+64), channel block cb of Z frame f of sample n.
@@ -399,7 +474,8 @@ struct TcParams {
     int out_f32;      // 1: out is FP32, 0: BF16
     int per_tap_a;    // 1: one A load per tap (box without halo), 0: one halo load per (dt, ci-block)
     int TPB;          // spatial taps per weight stage (1 or kw); kh*kw % TPB == 0
-    int epi_tma;      // 1: epilogue stages BF16 tiles in shared memory and stores them with TMA; 0: direct stores
+    int epi_tma;      // 1: epilogue stages BF16 tiles in shared memory and stores them with TMA; 0: direct stores;
+                      // 2: the output is a frame ring (channels-last), staged pixel-major and stored with TMA
     int ECH;          // output channels per epilogue chunk (32 or 16) when epi_tma
     int SA, SB, ACC;  // ring depths and accumulator buffers
     uint32_t a_slot, b_slot, b_tap;  // bytes per ring slot (multiples of 1024) and per tap inside a weight slot
@@ -410,6 +486,10 @@ struct TcParams {
     long long wait_limit_clk; // bound of every mbarrier wait, in SM clocks
     unsigned int* band_ctr;   // cooperative staging: per 16-row band, the number of CTAs that have staged their share
     int nbands;               // cooperative staging: bands of the image (= tile rows)
+    int f0;                   // ring input: the slot of Z frame 0; Z frame f lives in slot (f0 + f) mod F (0 for a staged copy)
+    const __nv_bfloat16* res; // optional residual ring [N][res_F][res_CB][H][W][res_KB] holding Cout channels, or null
+    int res_F, res_f0, res_CB, res_KB;   // residual frame t is slot (res_f0 + t) mod res_F
+    int out_F, out_f0, out_KB;           // epi_tma == 2: output frame t goes to slot (out_f0 + t) mod out_F
     const float* bias;        // [NT*NPAD]
     const uint8_t* wq;        // packed weight tiles [dt][cb][nt][sp] of b_tap bytes each
     void* out;
@@ -470,6 +550,37 @@ __device__ __forceinline__ uint32_t make_desc_lo(uint32_t addr) {
     // lower word: bits 0-13 start address >> 4, bits 16-29 leading-dimension byte offset >> 4 (unused for
     // swizzled K-major operands; canonical value 1)
     return ((addr & 0x3FFFFu) >> 4) | (1u << 16);
+}
+
+// Residual of one pixel: 32 consecutive channels (64 bytes) starting at channel co0 of a frame ring, as 16 BF16
+// pairs.  res_row addresses channel block 0 of the pixel's image row; zeros when there is no residual or the
+// pixel lies outside the image.
+__device__ __forceinline__ void load_res32(const __nv_bfloat16* res_row, bool valid, int w, int co0, const TcParams& p,
+                                           int64_t HW, uint32_t (&rr)[16]) {
+    if (res_row && valid) {
+        const uint4* src = reinterpret_cast<const uint4*>(res_row + ((int64_t)(co0 / p.res_KB) * HW + w) * p.res_KB +
+                                                          (co0 % p.res_KB));
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const uint4 u = __ldg(src + c);
+            rr[4 * c] = u.x; rr[4 * c + 1] = u.y; rr[4 * c + 2] = u.z; rr[4 * c + 3] = u.w;
+        }
+    } else {
+#pragma unroll
+        for (int j = 0; j < 16; ++j) rr[j] = 0u;
+    }
+}
+
+// Two neighbouring output channels: round conv + bias to BF16 once; with a residual, add it to that rounded value
+// in FP32 and round again (the result of a BF16 convolution followed by a BF16 addition).
+__device__ __forceinline__ uint32_t epi_pair(float a0, float a1, uint32_t res_pair, bool has_res) {
+    __nv_bfloat162 o = __floats2bfloat162_rn(a0, a1);
+    if (has_res) {
+        const float2 of = __bfloat1622float2(o);
+        const float2 rf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&res_pair));
+        o = __floats2bfloat162_rn(of.x + rf.x, of.y + rf.y);
+    }
+    return *reinterpret_cast<const uint32_t*>(&o);
 }
 
 // KB: input channels per K block (64 -> 128-byte swizzle, 32 -> 64-byte swizzle).  NB: 128-pixel blocks per tile.
@@ -605,7 +716,9 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                 const int dt0 = (p.first_frame - t > 0) ? p.first_frame - t : 0;
                 for (int dt = dt0; ok && dt < p.kt; ++dt)
                     for (int cb = 0; ok && cb < p.CB; ++cb) {
-                        const int fz = n * p.F + t + dt;
+                        int fr = p.f0 + t + dt;                   // ring slot of Z frame t+dt (f0 = 0: the frame itself)
+                        if (fr >= p.F) fr -= p.F;
+                        const int fz = n * p.F + fr;
                         const int ntap = p.per_tap_a ? spatial : 1;
                         for (int tp = 0; tp < ntap; ++tp) {
                             if (!(ok = mbar_wait(&sh->empty_a[s], phase, sh, p, SITE_A_EMPTY))) break;
@@ -794,6 +907,8 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
         const int64_t HW = (int64_t)p.H * p.W;
         const int m = q * 32 + lane;  // accumulator row = pixel m of a 128-pixel block: image row m/8, pixel m%8
         const bool elected = (threadIdx.x == 4 * 32);
+        constexpr bool RING = !FUSED && !COOP;                 // frame-ring output and residual: plain variant only
+        const bool has_res = RING && p.res != nullptr;
         int ebuf = 0;
         for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
             const int nt = tile % p.NT;
@@ -802,39 +917,74 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
             const int tx = r % p.tiles_w; r /= p.tiles_w;
             const int ty = p.ty_begin + r % p.tiles_h;
             const int n = r / p.tiles_h;
+            const int h = ty * 16 + (m >> 3);
+            // residual: pixel (h, w) of frame t holds its Cout channels in blocks of res_KB (64 bytes per 32 channels)
+            const __nv_bfloat16* res_row = nullptr;
+            if (has_res && h < p.H) {
+                int rs = p.res_f0 + t;
+                if (rs >= p.res_F) rs -= p.res_F;
+                res_row = p.res + (((int64_t)n * p.res_F + rs) * p.res_CB * HW + (int64_t)h * p.W) * p.res_KB;
+            }
             ok = mbar_wait(&sh->acc_full[acc], pacc, sh, p, SITE_ACC_FULL);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
             const uint32_t t_acc = tmem_base + (uint32_t)(acc * NB) * p.NPAD + ((uint32_t)(q * 32) << 16);
             if (p.epi_tma) {
-                // BF16 tile chunks [ECH channels][16 rows][TW pixels] -> shared memory -> one TMA store per chunk
+                // BF16 tile chunks -> shared memory -> one TMA store per chunk.  NCTHW output: [ECH channels][16 rows]
+                // [TW pixels]; ring output: [16 rows][TW pixels][32 channels] with the 64-byte swizzle of the tensor map.
                 for (int c0 = 0; c0 < p.NPAD; c0 += p.ECH) {
                     if (elected) bulk_wait_read<1>();   // the store that last read this buffer has finished reading
                     epi_bar_sync();
-                    __nv_bfloat16* stg = reinterpret_cast<__nv_bfloat16*>(epi_buf + (size_t)ebuf * p.e_slot);
+                    uint8_t* stg = epi_buf + (size_t)ebuf * p.e_slot;
                     const int co0 = nt * p.NPAD + c0;
 #pragma unroll
                     for (int blk = 0; blk < NB; ++blk) {
+                        const int w = tx * TW + blk * 8 + (m & 7);
+                        uint32_t rr[16];
+                        load_res32(res_row, w < p.W, w, co0, p, HW, rr);
                         uint32_t v[32];
                         if (p.ECH == 32) tc_ld32(t_acc + blk * p.NPAD + c0, v); else tc_ld16(t_acc + blk * p.NPAD + c0, v);
                         tc_wait_ld();
-                        __nv_bfloat16* dst = stg + (m >> 3) * TW + blk * 8 + (m & 7);
+                        uint32_t pk[16];
 #pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (j < p.ECH)
-                                dst[j * 16 * TW] = __float2bfloat16_rn(__uint_as_float(v[j]) + __ldg(p.bias + co0 + j));
+                        for (int j = 0; j < 16; ++j)
+                            pk[j] = (2 * j < p.ECH) ? epi_pair(__uint_as_float(v[2 * j]) + __ldg(p.bias + co0 + 2 * j),
+                                                               __uint_as_float(v[2 * j + 1]) + __ldg(p.bias + co0 + 2 * j + 1),
+                                                               rr[j], has_res)
+                                                    : 0u;
+                        const uint32_t px = (uint32_t)((m >> 3) * TW + blk * 8 + (m & 7));   // pixel of the tile, row-major
+                        if (RING && p.epi_tma == 2) {
+                            uint4* row = reinterpret_cast<uint4*>(stg + (size_t)px * 64);
+                            const uint32_t sw = (px >> 1) & 3u;
+#pragma unroll
+                            for (int c = 0; c < 4; ++c)
+                                row[c ^ sw] = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+                        } else {
+                            unsigned short* dst = reinterpret_cast<unsigned short*>(stg) + px;
+#pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                if (2 * j < p.ECH) {
+                                    dst[(2 * j) * 16 * TW] = (unsigned short)(pk[j] & 0xFFFFu);
+                                    dst[(2 * j + 1) * 16 * TW] = (unsigned short)(pk[j] >> 16);
+                                }
+                        }
                     }
                     fence_async_smem();
                     epi_bar_sync();
                     if (elected) {
-                        tma_store_5d(&tm_o, smem_u32(stg), tx * TW, ty * 16, t, co0, n);
+                        if (RING && p.epi_tma == 2) {
+                            int os = p.out_f0 + t;
+                            if (os >= p.out_F) os -= p.out_F;
+                            tma_store_5d(&tm_o, smem_u32(stg), co0 % p.out_KB, tx * TW, ty * 16, co0 / p.out_KB, n * p.out_F + os);
+                        } else {
+                            tma_store_5d(&tm_o, smem_u32(stg), tx * TW, ty * 16, t, co0, n);
+                        }
                         bulk_commit();
                     }
                     ebuf ^= 1;
                 }
             } else {
-                const int h = ty * 16 + (m >> 3);
 #pragma unroll 1
                 for (int blk = 0; blk < NB; ++blk) {
                     const int w = tx * TW + blk * 8 + (m & 7);
@@ -842,20 +992,34 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                     const int64_t pix = (int64_t)t * HW + (int64_t)h * p.W + w;
 #pragma unroll 1
                     for (int c0 = 0; c0 < p.NPAD; c0 += 32) {
+                        const int co0 = nt * p.NPAD + c0;
+                        uint32_t rr[16];
+                        load_res32(res_row, valid, w, co0, p, HW, rr);
                         uint32_t v[32];
                         const int nc = (p.NPAD - c0 >= 32) ? 32 : 16;
                         if (nc == 32) tc_ld32(t_acc + blk * p.NPAD + c0, v); else tc_ld16(t_acc + blk * p.NPAD + c0, v);
                         tc_wait_ld();
-                        const int co0 = nt * p.NPAD + c0;
                         if (valid) {
+                            if (p.out_f32) {
 #pragma unroll
-                            for (int j = 0; j < 32; ++j) {
-                                const int co = co0 + j;
-                                if (j < nc && co < p.Cout) {
-                                    const float val = __uint_as_float(v[j]) + __ldg(p.bias + co);
-                                    const int64_t o = ((int64_t)n * p.Cout + co) * p.T * HW + pix;
-                                    if (p.out_f32) reinterpret_cast<float*>(p.out)[o] = val;
-                                    else reinterpret_cast<__nv_bfloat16*>(p.out)[o] = __float2bfloat16_rn(val);
+                                for (int j = 0; j < 32; ++j) {
+                                    const int co = co0 + j;
+                                    if (j < nc && co < p.Cout)
+                                        reinterpret_cast<float*>(p.out)[((int64_t)n * p.Cout + co) * p.T * HW + pix] =
+                                            __uint_as_float(v[j]) + __ldg(p.bias + co);
+                                }
+                            } else {
+#pragma unroll
+                                for (int j = 0; j < 16; ++j) {
+                                    const int co = co0 + 2 * j;
+                                    if (2 * j < nc) {
+                                        const uint32_t pr = epi_pair(__uint_as_float(v[2 * j]) + __ldg(p.bias + co),
+                                                                     __uint_as_float(v[2 * j + 1]) + __ldg(p.bias + co + 1), rr[j], has_res);
+                                        unsigned short* o = reinterpret_cast<unsigned short*>(p.out) +
+                                                            ((int64_t)n * p.Cout + co) * p.T * HW + pix;
+                                        if (co < p.Cout) o[0] = (unsigned short)(pr & 0xFFFFu);
+                                        if (co + 1 < p.Cout) o[(int64_t)p.T * HW] = (unsigned short)(pr >> 16);
+                                    }
                                 }
                             }
                         }

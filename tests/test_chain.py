@@ -134,3 +134,39 @@ def test_chain_gpu_streaming_full_size():
     assert torch.equal(chunked, whole)
     assert bool(torch.isfinite(whole).all())
     ch.close()
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("frames,H,W,chunks", [(5, 6, 8, [1, 1, 1, 1, 1]), (6, 10, 12, [2, 2, 2]), (21, 44, 80, [1] * 21)])
+def test_resident_chain_equals_the_ncthw_chain_bit_for_bit(frames, H, W, chunks):
+    """Activations kept in frame rings between the layers (history in place, residual in the epilogue) against the
+    chain that returns to NCTHW after every layer: the same bits, chunked and whole-sequence, at a reduced size,
+    with multi-frame chunks, and at the full size of the benchmark configuration."""
+    torch = pytest.importorskip("torch")
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from _util import to_dev
+    from paper_2609_31938_b200.chain import ResidentDecoderChain
+    torch.cuda.set_device(0)
+    w, b = make_chain_params(384, 192, 96, seed=0)
+    ud = to_dev(si.normal((1, 384, frames, H, W), 1.0, si.BF16, 0, si.TID_X))
+    ch = _gpu_chain(w, b)
+    whole = ch.step(ud)                                           # NCTHW chain, whole sequence
+    rc = ResidentDecoderChain({n: to_dev(w[n]) for n in LAYERS}, {n: to_dev(b[n]) for n in LAYERS})
+    outs, pos = [], 0
+    for n in chunks:
+        outs.append(rc.step(ud[:, :, pos:pos + n].contiguous()))
+        pos += n
+    chunked = torch.cat(outs, dim=2)
+    del outs
+    rc.reset()
+    rwhole = rc.step(ud)
+    torch.cuda.synchronize()
+    for l in rc.layers.values():
+        assert l.device_status()[0] == 0
+        c = l.counters()
+        assert c["calls"] == c["ok"] == c["tcgen05_bf16"] == len(chunks) + 1
+    assert torch.equal(chunked, whole)
+    assert torch.equal(rwhole, whole)
+    ch.close()
+    rc.close()
