@@ -246,7 +246,7 @@ ccv3d_status launch_conv(ccv3d_handle* h, TcParams p, int nb, int ty0, int ty1, 
     const TcPlan& pl = h->plan;
     p.ty_begin = ty0;
     p.tiles_h = ty1 - ty0;
-    const int64_t total = (int64_t)p.N * p.tiles_h * p.tiles_w * p.T * pl.NT;
+    const int64_t total = (int64_t)p.N * p.tiles_h * p.tiles_w * p.T * p.NT;
     if (total > 0x7FFFFFFF) return CCV3D_ERR_UNSUPPORTED;
     p.total_tiles = (int)total;
     const int grid = p.total_tiles < h->sm_count ? p.total_tiles : h->sm_count;
@@ -295,7 +295,15 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     // 256-pixel tiles (two 128-pixel blocks sharing every weight tile) unless that leaves SMs without a tile
     int NB = pl.NB;
     if ((int64_t)N * ((H + 15) / 16) * ((W + 15) / 16) * T * pl.NT < h->sm_count) NB = 1;
-    const int ACC = (2 * NB * pl.NPAD <= 512) ? 2 : 1;
+    // Still fewer than half as many work items as SMs (the 44x80 layers): run half-width output-channel tiles.
+    // Twice the items, each streaming half of the weights through its SM - the per-SM weight stream is what
+    // bounds a 128-pixel tile - and nothing to reduce afterwards.
+    int NT = pl.NT, NPAD = pl.NPAD, split_n = 0;
+    if (NB == 1 && !per_tap && pl.NPAD % 32 == 0 &&
+        2 * (int64_t)N * ((H + 15) / 16) * ((W + 7) / 8) * T * pl.NT <= h->sm_count) {
+        split_n = 1; NT = 2 * pl.NT; NPAD = pl.NPAD / 2;
+    }
+    const int ACC = (2 * NB * NPAD <= 512) ? 2 : 1;
     const int TW = 8 * NB;
     const int BW = per_tap ? TW : TW + d.kw - 1;
     const int BH = per_tap ? 16 : 16 + d.kh - 1;
@@ -309,7 +317,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     memset(&p, 0, sizeof(p));
     p.N = N; p.T = T; p.H = H; p.W = W; p.Cout = d.cout; p.F = F;
     p.kt = d.kt; p.kh = d.kh; p.kw = d.kw;
-    p.CB = pl.CB; p.NT = pl.NT; p.NPAD = pl.NPAD;
+    p.CB = pl.CB; p.NT = NT; p.NPAD = NPAD;
     const int tiles_h = (H + 15) / 16;
     p.tiles_w = (W + TW - 1) / TW;
     p.first_frame = tc - cf;
@@ -317,10 +325,12 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     p.per_tap_a = per_tap;
     p.ACC = ACC;
     p.a_slot = (uint32_t)align_up((uint64_t)BW * BH * pl.KB * 2, 1024);
-    p.b_tap = (uint32_t)pl.NPAD * pl.KB * 2;
+    p.b_tap = (uint32_t)NPAD * pl.KB * 2;
+    p.split_n = split_n;
+    p.b_src_tap = split_n ? (uint32_t)pl.NPAD * pl.KB * 2 : 0;
     // epilogue: BF16 output rows that TMA can address (W*2 bytes a multiple of 16) go through shared memory
     p.epi_tma = (!p.out_f32 && W % 8 == 0) ? 1 : 0;
-    p.ECH = (pl.NPAD % 32 == 0) ? 32 : 16;
+    p.ECH = (NPAD % 32 == 0) ? 32 : 16;
     p.e_slot = p.epi_tma ? (uint32_t)(p.ECH * 16 * TW * 2) : 0;
 
     // Optional (CCV3D_FLAG_OVERLAP): large images are cut into bands of tile rows; band k is staged on a side
@@ -332,14 +342,14 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     // persistent convolution CTAs), which is why it is not the default.
     int nbands = 1;
     if ((d.flags & CCV3D_FLAG_OVERLAP) && h->side[0] &&
-        (int64_t)N * tiles_h * p.tiles_w * T * pl.NT >= 2LL * h->sm_count && tiles_h >= 4)
+        (int64_t)N * tiles_h * p.tiles_w * T * NT >= 2LL * h->sm_count && tiles_h >= 4)
         nbands = tiles_h / 2 < MAX_BANDS ? tiles_h / 2 : MAX_BANDS;
 
     // Cooperative staging (default when W % 8 == 0): the staging pass runs inside the convolution kernel, on four
     // extra warps per CTA, one band of 16 rows ahead of the tiles that read it.
     const bool coop = nbands == 1 && !per_tap && !(d.flags & CCV3D_FLAG_TWO_KERNELS) && W % 8 == 0 &&
                       tiles_h <= MAX_COOP_BANDS && tiles_h >= 4 && pl.KB == 64 &&   // 32-channel blocks: the stagers cannot keep up
-                      (int64_t)N * tiles_h * p.tiles_w * T * pl.NT >= 4LL * h->sm_count;   // small problems: two kernels
+                      (int64_t)N * tiles_h * p.tiles_w * T * NT >= 4LL * h->sm_count;   // small problems: two kernels
     size_t fixed = 1024 /*alignment slack*/ + align_up(sizeof(TcShared), 128) + 2 * (size_t)p.e_slot + (coop ? 9216 : 0);
     // leave room for staging blocks to be resident next to a convolution CTA when the two overlap
     const size_t limit = nbands > 1 ? SMEM_LIMIT - STAGE_COEXIST_BYTES : SMEM_LIMIT;
@@ -358,7 +368,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     if (SB > 8) SB = 8;
     while (SA < 4 && (size_t)(SA + 1) * p.a_slot + (size_t)SB * p.b_slot <= budget) ++SA;
     p.SA = SA; p.SB = SB;
-    p.tmem_cols = pow2_cols((uint32_t)(NB * pl.NPAD * ACC));
+    p.tmem_cols = pow2_cols((uint32_t)(NB * NPAD * ACC));
     if (p.tmem_cols > 512) return CCV3D_ERR_UNSUPPORTED;
     p.wait_limit_clk = h->wait_limit_clk;
     p.bias = h->bias32;
@@ -383,7 +393,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
         p.nbands = tiles_h;
         p.ty_begin = 0;
         p.tiles_h = tiles_h;
-        const int64_t total = (int64_t)N * tiles_h * p.tiles_w * T * pl.NT;
+        const int64_t total = (int64_t)N * tiles_h * p.tiles_w * T * NT;
         if (total > 0x7FFFFFFF) return CCV3D_ERR_UNSUPPORTED;
         p.total_tiles = (int)total;
         const int grid = p.total_tiles < h->sm_count ? p.total_tiles : h->sm_count;
@@ -892,7 +902,12 @@ ccv3d_status forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int x_slot, int
 
     int NB = pl.NB;
     if ((int64_t)N * ((H + 15) / 16) * ((W + 15) / 16) * T * pl.NT < h->sm_count) NB = 1;
-    const int ACC = (2 * NB * pl.NPAD <= 512) ? 2 : 1;
+    // fewer than half as many work items as SMs: half-width output-channel tiles (see forward_tc)
+    int NT = pl.NT, NPAD = pl.NPAD, split_n = 0;
+    if (NB == 1 && pl.NPAD % 64 == 0 && 2 * (int64_t)N * ((H + 15) / 16) * ((W + 7) / 8) * T * pl.NT <= h->sm_count) {
+        split_n = 1; NT = 2 * pl.NT; NPAD = pl.NPAD / 2;
+    }
+    const int ACC = (2 * NB * NPAD <= 512) ? 2 : 1;
     const int TW = 8 * NB, BW = TW + d.kw - 1, BH = 16 + d.kh - 1;
     CUtensorMap tm_a, tm_o;
     ccv3d_status s = encode_ring_map(h, &tm_a, in, pl.KB, BW, BH, pl.KB == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B);
@@ -904,17 +919,19 @@ ccv3d_status forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int x_slot, int
     p.F = in->F;
     p.f0 = (x_slot - tc + in->F) % in->F;
     p.kt = d.kt; p.kh = d.kh; p.kw = d.kw;
-    p.CB = pl.CB; p.NT = pl.NT; p.NPAD = pl.NPAD;
+    p.CB = pl.CB; p.NT = NT; p.NPAD = NPAD;
     p.tiles_h = (H + 15) / 16;
     p.tiles_w = (W + TW - 1) / TW;
-    const int64_t total = (int64_t)N * p.tiles_h * p.tiles_w * T * pl.NT;
+    const int64_t total = (int64_t)N * p.tiles_h * p.tiles_w * T * NT;
     if (total > 0x7FFFFFFF) return CCV3D_ERR_UNSUPPORTED;
     p.total_tiles = (int)total;
     p.first_frame = tc - hist;
     p.out_f32 = d.out_dtype == CCV3D_F32;
     p.ACC = ACC;
     p.a_slot = (uint32_t)align_up((uint64_t)BW * BH * pl.KB * 2, 1024);
-    p.b_tap = (uint32_t)pl.NPAD * pl.KB * 2;
+    p.b_tap = (uint32_t)NPAD * pl.KB * 2;
+    p.split_n = split_n;
+    p.b_src_tap = split_n ? (uint32_t)pl.NPAD * pl.KB * 2 : 0;
     if (oring) {
         p.epi_tma = 2;
         p.ECH = 32;
@@ -924,7 +941,7 @@ ccv3d_status forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int x_slot, int
         if (s != CCV3D_OK) return s;
     } else {
         p.epi_tma = (!p.out_f32 && W % 8 == 0) ? 1 : 0;
-        p.ECH = (pl.NPAD % 32 == 0) ? 32 : 16;
+        p.ECH = (NPAD % 32 == 0) ? 32 : 16;
         p.e_slot = p.epi_tma ? (uint32_t)(p.ECH * 16 * TW * 2) : 0;
         if (p.epi_tma) {
             cuuint64_t dims[5] = {(cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)T, (cuuint64_t)d.cout, (cuuint64_t)N};
@@ -958,7 +975,7 @@ ccv3d_status forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int x_slot, int
     if (SB > 8) SB = 8;
     while (SA < 4 && (size_t)(SA + 1) * p.a_slot + (size_t)SB * p.b_slot <= budget) ++SA;
     p.SA = SA; p.SB = SB;
-    p.tmem_cols = pow2_cols((uint32_t)(NB * pl.NPAD * ACC));
+    p.tmem_cols = pow2_cols((uint32_t)(NB * NPAD * ACC));
     if (p.tmem_cols > 512) return CCV3D_ERR_UNSUPPORTED;
     p.wait_limit_clk = h->wait_limit_clk;
     p.bias = h->bias32;

@@ -479,6 +479,8 @@ struct TcParams {
     int ECH;          // output channels per epilogue chunk (32 or 16) when epi_tma
     int SA, SB, ACC;  // ring depths and accumulator buffers
     uint32_t a_slot, b_slot, b_tap;  // bytes per ring slot (multiples of 1024) and per tap inside a weight slot
+    uint32_t b_src_tap;       // bytes per tap in the packed weights when that differs from b_tap (split_n), else 0
+    int split_n;              // 1: NT and NPAD describe half-width output-channel tiles of a layer packed at full width
     uint32_t e_slot;          // bytes of one epilogue staging buffer (two are allocated when epi_tma)
     uint32_t raw_slot;        // fused mode: bytes of one raw [32 ch][BH rows][32 px] box (two are allocated)
     int tc, cf;               // fused mode: kt-1 and the history frames the cache holds; Z frame f < tc is cache frame f-(tc-cf)
@@ -738,6 +740,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     else if (warp == 1) {
         if (lane == 0) {
             const uint32_t b_bytes = p.b_tap * p.TPB;
+            const uint32_t src_tap = p.b_src_tap ? p.b_src_tap : p.b_tap;   // bytes between taps in the packed weights
             int s = 0;
             uint32_t phase = 1;
             bool ok = true;
@@ -747,12 +750,19 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                 const int dt0 = (p.first_frame - t > 0) ? p.first_frame - t : 0;
                 for (int dt = dt0; ok && dt < p.kt; ++dt)
                     for (int cb = 0; ok && cb < p.CB; ++cb) {
-                        const uint8_t* src = p.wq + (size_t)((dt * p.CB + cb) * p.NT + nt) * spatial * p.b_tap;
+                        // split_n: this launch runs half-width output-channel tiles; the packed image of a full tile
+                        // holds its two halves back to back (the swizzle repeats every 8 rows), so a half tile of a
+                        // tap is a contiguous piece of it and only the distance between taps differs
+                        const uint8_t* src = p.wq + (size_t)((dt * p.CB + cb) * (p.NT >> p.split_n) + (nt >> p.split_n)) * spatial * src_tap +
+                                             (size_t)(nt & p.split_n) * p.b_tap;
                         for (int tp = 0; tp < spatial; tp += p.TPB) {
                             if (!(ok = mbar_wait(&sh->empty_b[s], phase, sh, p, SITE_B_EMPTY))) break;
                             const uint32_t bar = smem_u32(&sh->full_b[s]);
                             mbar_expect_tx(bar, b_bytes);
-                            bulk_load(smem_u32(ring_b + (size_t)s * p.b_slot), src + (size_t)tp * p.b_tap, b_bytes, bar);
+                            const uint32_t dst = smem_u32(ring_b + (size_t)s * p.b_slot);
+                            if (src_tap == p.b_tap) bulk_load(dst, src + (size_t)tp * src_tap, b_bytes, bar);
+                            else
+                                for (int u = 0; u < p.TPB; ++u) bulk_load(dst + u * p.b_tap, src + (size_t)(tp + u) * src_tap, p.b_tap, bar);
                             if (++s == p.SB) { s = 0; phase ^= 1; }
                         }
                     }
@@ -925,6 +935,10 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                 if (rs >= p.res_F) rs -= p.res_F;
                 res_row = p.res + (((int64_t)n * p.res_F + rs) * p.res_CB * HW + (int64_t)h * p.W) * p.res_KB;
             }
+            // the residual of the first chunk is fetched while the MMAs of this tile still run; every later chunk's
+            // residual is fetched one chunk ahead
+            uint32_t rr_next[16];
+            if (p.epi_tma) load_res32(res_row, tx * TW + (m & 7) < p.W, tx * TW + (m & 7), nt * p.NPAD, p, HW, rr_next);
             ok = mbar_wait(&sh->acc_full[acc], pacc, sh, p, SITE_ACC_FULL);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -940,9 +954,14 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                     const int co0 = nt * p.NPAD + c0;
 #pragma unroll
                     for (int blk = 0; blk < NB; ++blk) {
-                        const int w = tx * TW + blk * 8 + (m & 7);
                         uint32_t rr[16];
-                        load_res32(res_row, w < p.W, w, co0, p, HW, rr);
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) rr[j] = rr_next[j];
+                        if (has_res) {
+                            const int wn = tx * TW + ((blk + 1 < NB) ? blk + 1 : 0) * 8 + (m & 7);
+                            const int con = (blk + 1 < NB) ? co0 : co0 + p.ECH;
+                            load_res32(res_row, wn < p.W && con < (nt + 1) * p.NPAD, wn, con, p, HW, rr_next);
+                        }
                         uint32_t v[32];
                         if (p.ECH == 32) tc_ld32(t_acc + blk * p.NPAD + c0, v); else tc_ld16(t_acc + blk * p.NPAD + c0, v);
                         tc_wait_ld();
