@@ -1,6 +1,6 @@
 """Run a few forward calls of one layer shape on cuda:0 - a small, self-ending program to put under a profiler.
 
-    python -m paper_2609_31938_b200.profile_case --cin 192 --cout 192 --t 4 --h 176 --w 320 [--k 3 3 3] [--calls 3]
+    python -m paper_2609_31938_b200.profile_case --cin 192 --cout 192 --t 4 --h 176 --w 320 [--k 3 3 3] [--calls 3] [--ring]
 
 Inputs are the seeded synthetic tensors of the benchmark (normal activations, fan-in-scaled weights).
 """
@@ -27,6 +27,7 @@ def main():
     ap.add_argument("--calls", type=int, default=3)
     ap.add_argument("--no-cache", action="store_true")
     ap.add_argument("--flags", type=int, default=0, help="CCV3D_FLAG_* bits (16 = two-kernel schedule, 8 = fused route)")
+    ap.add_argument("--ring", action="store_true", help="resident activations: input and output in frame rings")
     a = ap.parse_args()
     c = si.conv_case(1, a.cin, a.cout, a.t, a.h, a.w, k=tuple(a.k), cache=None if a.no_cache else "random")
     up = lambda v: None if v is None else torch.from_numpy(v.view(np.int16)).cuda().view(torch.bfloat16)
@@ -34,8 +35,20 @@ def main():
     x, cache = up(c["x"]), up(c["cache"])
     out = torch.empty((1, a.cout, a.t, a.h, a.w), dtype=torch.bfloat16, device="cuda")
     nc = torch.empty_like(cache) if cache is not None else None
-    for _ in range(a.calls):
-        layer(x, cache, out=out, new_cache=nc)
+    if a.ring:
+        tc = a.k[0] - 1
+        rin = ccv.FrameRing(1, a.cin, a.t + tc, a.h, a.w)
+        rout = ccv.FrameRing(1, a.cout, a.t, a.h, a.w)
+        if cache is not None:
+            rin.load(0, cache)
+        rin.load(tc, x)
+        slot = tc
+        for _ in range(a.calls):
+            layer.forward_ring(rin, slot, tc if cache is not None else 0, a.t, out_ring=rout)
+            slot = (slot + a.t) % rin.F
+    else:
+        for _ in range(a.calls):
+            layer(x, cache, out=out, new_cache=nc)
     torch.cuda.synchronize()
     st, detail = layer.device_status()
     assert st == ccv.OK, (ccv.status_string(st), hex(detail))
