@@ -84,3 +84,26 @@ def test_null_and_misaligned_arguments():
     assert ccv.ccv3d_upsample_bf16(None, None, 1, 1, 1, 1, 1, 1) == ccv.ERR_INVALID_ARG
     with pytest.raises(ccv.Ccv3dError):
         ccv.ccv3d_get_counters(None)
+
+
+def test_ring_geometry_and_argument_checks_need_no_device():
+    """Frame rings: the block-size rule, the byte count, and every rejection that happens before a launch."""
+    assert [ccv.ccv3d_ring_kb(c) for c in (0, 16, 32, 64, 96, 100, 192, 384)] == [0, 0, 32, 64, 32, 0, 64, 64]
+    assert ctypes.sizeof(ccv.Ring) == 8 + 6 * 4
+    r = ccv.Ring(4096, 2, 96, 5, 7, 9, 32)
+    assert ccv.ccv3d_ring_bytes(r) == 2 * 5 * 96 * 7 * 9 * 2
+    assert ccv.ccv3d_ring_bytes(ccv.Ring(4096, 1, 96, 5, 7, 9, 64)) == 0          # 96 channels do not split into 64s
+    assert ccv.ccv3d_ring_bytes(ccv.Ring(4096, 1, 64, 0, 7, 9, 64)) == 0
+    big = ccv.Ring(1 << 20, 1, 64, 4, 8, 8, 64)
+    assert ccv.ccv3d_ring_load(big, 0, None, 1) == ccv.ERR_INVALID_ARG             # no source
+    assert ccv.ccv3d_ring_load(big, 4, 1 << 24, 1) == ccv.ERR_INVALID_ARG          # slot out of range
+    assert ccv.ccv3d_ring_load(big, 0, 1 << 24, 5) == ccv.ERR_INVALID_ARG          # more frames than slots
+    assert ccv.ccv3d_ring_load(big, 0, (1 << 24) + 4, 1) == ccv.ERR_ALIGNMENT
+    assert ccv.ccv3d_ring_load(big, 0, (1 << 20) + 256, 1) == ccv.ERR_ALIAS        # source inside the ring
+    assert ccv.ccv3d_ring_store(ccv.Ring(None, 1, 64, 4, 8, 8, 64), 0, 1 << 24, 1) == ccv.ERR_INVALID_ARG
+    assert ccv.ccv3d_ring_store(big, 0, (1 << 20) + 256, 1) == ccv.ERR_ALIAS
+    twice = ccv.Ring(1 << 26, 1, 64, 4, 16, 16, 64)
+    assert ccv.ccv3d_upsample_ring(big, 0, twice, 0, 2, 3) == ccv.ERR_INVALID_ARG  # 2 x 3 frames > 4 slots
+    assert ccv.ccv3d_upsample_ring(big, 0, big, 0, 1, 1) == ccv.ERR_INVALID_ARG    # not twice the size
+    assert ccv.ccv3d_upsample_ring(big, 0, ccv.Ring(1 << 26, 1, 32, 4, 16, 16, 32), 0, 1, 1) == ccv.ERR_INVALID_ARG
+    assert ccv.ccv3d_forward_ring(None, big, 0, 0, None, 0, twice, 0, None, 1) == ccv.ERR_INVALID_ARG
