@@ -12,6 +12,9 @@ structurally different restatements used to pin it:
                             one 2-D correlation per tap folded over the
                             interval, accumulation, bias once.
 
+``forward_general`` / ``brute_force_general`` are the operator with the layer's own
+spatial stride, padding, dilation and a temporal dilation (Eq. (1)-(2) as printed).
+
 Host tensors: fp32 arrays, or uint16 arrays of bf16 bit patterns.
 """
 from __future__ import annotations
@@ -42,6 +45,11 @@ def build(force: bool = False) -> str:
 _lib = None
 
 
+class _Geom(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in ("N", "Cin", "Cout", "T", "H", "W", "kt", "kh", "kw", "sh", "sw", "ph", "pw",
+                                            "dh", "dw", "dil_t", "cf")]
+
+
 def _load():
     global _lib
     if _lib is None:
@@ -54,6 +62,10 @@ def _load():
         lib.ccv3d_oracle_num_threads.restype = i
         lib.ccv3d_oracle_cache_update.argtypes = [i, p, p] + [i] * 6 + [p]
         lib.ccv3d_oracle_cache_update.restype = i
+        lib.ccv3d_oracle_forward_general.argtypes = [i, p, p, p, p, ctypes.POINTER(_Geom), p, p]
+        lib.ccv3d_oracle_forward_general.restype = i
+        lib.ccv3d_oracle_out_dims.argtypes = [ctypes.POINTER(_Geom), ctypes.POINTER(i), ctypes.POINTER(i)]
+        lib.ccv3d_oracle_out_dims.restype = i
         _lib = lib
     return _lib
 
@@ -113,6 +125,72 @@ def points(x, cache, w, b, flat_idx):
     if rc != 0:
         raise ValueError("ccv3d_oracle_points rejected its arguments")
     return vals
+
+
+def forward_general(x, cache, w, b, stride=(1, 1), pad=None, dil=(1, 1), dil_t=1, want_cache: bool = True):
+    """The operator with the paper's full supported contract (Eq. (1)-(2) with s, p, d and d_t; unit temporal
+    stride): spatial stride/padding/dilation per tap, temporal dilation, a cache of up to d_t (kt-1) frames
+    (fewer = older history absent).  pad None = ((kh-1) d_h / 2, (kw-1) d_w / 2).
+    Returns (out float64 [N,Cout,T,H_o,W_o], new_cache [N,Cin,d_t (kt-1),H,W] or None)."""
+    dt = _dtype_of(x)
+    x, w = np.ascontiguousarray(x), np.ascontiguousarray(w)
+    assert _dtype_of(w) == dt
+    N, Cin, T, H, W = x.shape
+    Cout, Cin2, kt, kh, kw = w.shape
+    assert Cin2 == Cin
+    if pad is None:
+        pad = ((kh - 1) * dil[0] // 2, (kw - 1) * dil[1] // 2)
+    tc = dil_t * (kt - 1)
+    cf = 0
+    if cache is not None and tc > 0:
+        cache = np.ascontiguousarray(cache)
+        cf = cache.shape[2]
+        assert _dtype_of(cache) == dt and cache.shape == (N, Cin, cf, H, W) and 0 < cf <= tc
+    else:
+        cache = None
+    if b is not None:
+        b = np.ascontiguousarray(b)
+        assert _dtype_of(b) == dt and b.shape == (Cout,)
+    g = _Geom(N, Cin, Cout, T, H, W, kt, kh, kw, stride[0], stride[1], pad[0], pad[1], dil[0], dil[1], dil_t, cf)
+    ho, wo = ctypes.c_int(), ctypes.c_int()
+    if _load().ccv3d_oracle_out_dims(ctypes.byref(g), ctypes.byref(ho), ctypes.byref(wo)) != 0:
+        raise ValueError("bad geometry")
+    out = np.empty((N, Cout, T, ho.value, wo.value), dtype=np.float64)
+    nc = np.empty((N, Cin, tc, H, W), dtype=x.dtype) if (want_cache and tc > 0) else None
+    rc = _load().ccv3d_oracle_forward_general(dt, _ptr(x), _ptr(cache), _ptr(w), _ptr(b), ctypes.byref(g), _ptr(out),
+                                              _ptr(nc))
+    if rc != 0:
+        raise ValueError("ccv3d_oracle_forward_general rejected its arguments")
+    return out, nc
+
+
+def brute_force_general(x, cache, w, b, stride=(1, 1), pad=(0, 0), dil=(1, 1), dil_t=1):
+    """The same contract on a materialised, zero-padded Z volume with strided slicing per tap (pure numpy,
+    tap-outermost: structurally different from the C routine).  Tiny shapes only."""
+    xd, cd, wd, bd = _widen(x), _widen(cache), _widen(w), _widen(b)
+    N, Cin, T, H, W = xd.shape
+    Cout, _, kt, kh, kw = wd.shape
+    tc = dil_t * (kt - 1)
+    ph, pw = pad
+    Zp = np.zeros((N, Cin, tc + T, H + 2 * ph, W + 2 * pw))
+    if cd is not None and tc > 0:
+        cf = cd.shape[2]
+        Zp[:, :, tc - cf:tc, ph:ph + H, pw:pw + W] = cd
+    Zp[:, :, tc:, ph:ph + H, pw:pw + W] = xd
+    Ho = (H + 2 * ph - dil[0] * (kh - 1) - 1) // stride[0] + 1
+    Wo = (W + 2 * pw - dil[1] * (kw - 1) - 1) // stride[1] + 1
+    out = np.zeros((N, Cout, T, Ho, Wo))
+    if bd is not None:
+        out += bd[None, :, None, None, None]
+    for k in range(kt):
+        for a in range(kh):
+            for c in range(kw):
+                src = Zp[:, :, k * dil_t:k * dil_t + T,
+                         a * dil[0]:a * dil[0] + (Ho - 1) * stride[0] + 1:stride[0],
+                         c * dil[1]:c * dil[1] + (Wo - 1) * stride[1] + 1:stride[1]]          # [N,Cin,T,Ho,Wo]
+                out += np.einsum("nithw,oi->nothw", src, wd[:, :, k, a, c])
+    Zt = Zp[:, :, :, ph:ph + H, pw:pw + W]
+    return out, Zt[:, :, T:T + tc]
 
 
 def cache_update(x, cache, kt: int):

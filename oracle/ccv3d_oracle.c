@@ -28,6 +28,13 @@
  * concatenated input, and the invariants (causality, streaming equivalence,
  * linearity, 1x1x1 = per-pixel matmul, delta kernel).
  * Parity unpinned: behaviour on NaN/Inf/subnormal inputs.
+ *
+ * ccv3d_oracle_forward_general (end of file) is the same operator with the
+ * layer's own spatial stride, padding and dilation and a temporal dilation
+ * (Eq. (1)-(2) as printed); its pins are in tests/test_oracle_general.py:
+ * hand-worked values, bit-for-bit reduction to ccv3d_oracle_forward, a numpy
+ * routine of different structure, the fp64 library conv3d, Eq. (3)'s interval
+ * route, streaming equivalence and causality under temporal dilation.
  */
 #include <stdint.h>
 #include <stdlib.h>
@@ -191,4 +198,112 @@ int ccv3d_oracle_num_threads(void) {
 #else
     return 1;
 #endif
+}
+
+/* ------------------------------------------------------------------------------------------------
+ * The operator with the paper's full supported contract (Section 4.1, Eq. (1)-(2) as printed): original
+ * spatial stride s = (s_h, s_w), padding p = (p_h, p_w) and dilation d = (d_h, d_w) inside every temporal
+ * tap's 2-D correlation, temporal dilation d_t in the source time q_k(t) = t + k d_t - p_l, unit temporal
+ * stride, one group.  The causal pad is p_l^base = d_t (kt-1) frames; the cache holds the newest cf of them
+ * (0 <= cf <= d_t (kt-1)), older ones do not exist and contribute zero:
+ *
+ *   tc = d_t (kt-1)
+ *   Z[n,ci,tau]      = 0                          0 <= tau < tc-cf
+ *                    = cache[n,ci,tau-(tc-cf)]    tc-cf <= tau < tc
+ *                    = x[n,ci,tau-tc]             tc <= tau < tc+T
+ *   H_o = floor((H + 2 p_h - d_h (kh-1) - 1) / s_h) + 1,   W_o likewise
+ *   out[n,co,t,ho,wo] = b[co] + sum_{ci,k,dh,dw} w[co,ci,k,dh,dw]
+ *                                * Z[n,ci, t + k d_t, ho s_h + dh d_h - p_h, wo s_w + dw d_w - p_w]
+ *   new_cache[n,ci,j] = Z[n,ci,T+j]               0 <= j < tc
+ *
+ * Written separately from ccv3d_oracle_forward (which it must reproduce bit for bit at s = d = d_t = 1,
+ * p = (k-1)/2, cf = kt-1: a test holds it to that), output-element-outermost, same arithmetic rules: exact
+ * widening, double products and sums, bias first, then (ci, k, dh, dw) lexicographic.
+ * ------------------------------------------------------------------------------------------------ */
+typedef struct {
+    int N, Cin, Cout, T, H, W;
+    int kt, kh, kw;
+    int sh, sw, ph, pw, dh, dw, dil_t;
+    int cf; /* frames the cache holds */
+} orc_geom;
+
+static inline int out_extent(int in, int pad, int dil, int k, int stride) {
+    const int span = in + 2 * pad - dil * (k - 1) - 1;
+    return span < 0 ? 0 : span / stride + 1;
+}
+
+static inline const char* zg_frame(const orc_geom* g, int dtype, const void* x, const void* cache, int n, int ci,
+                                   int tau) {
+    const int tc = g->dil_t * (g->kt - 1);
+    const int64_t HW = (int64_t)g->H * g->W;
+    if (tau < tc) {
+        const int cfr = tau - (tc - g->cf);
+        if (!cache || cfr < 0) return NULL;
+        return (const char*)cache + (size_t)((((int64_t)n * g->Cin + ci) * g->cf + cfr) * HW) * esize(dtype);
+    }
+    return (const char*)x + (size_t)((((int64_t)n * g->Cin + ci) * g->T + (tau - tc)) * HW) * esize(dtype);
+}
+
+static int geom_ok(const orc_geom* g) {
+    if (g->N < 1 || g->Cin < 1 || g->Cout < 1 || g->T < 1 || g->H < 1 || g->W < 1) return 0;
+    if (g->kt < 1 || g->kh < 1 || g->kw < 1) return 0;
+    if (g->sh < 1 || g->sw < 1 || g->dh < 1 || g->dw < 1 || g->dil_t < 1 || g->ph < 0 || g->pw < 0) return 0;
+    if (g->cf < 0 || g->cf > g->dil_t * (g->kt - 1)) return 0;
+    return 1;
+}
+
+int ccv3d_oracle_out_dims(const orc_geom* g, int* Ho, int* Wo) {
+    if (!g || !geom_ok(g)) return -1;
+    *Ho = out_extent(g->H, g->ph, g->dh, g->kh, g->sh);
+    *Wo = out_extent(g->W, g->pw, g->dw, g->kw, g->sw);
+    return 0;
+}
+
+/* out: double[N,Cout,T,H_o,W_o]; new_cache (may be NULL): [N,Cin,d_t(kt-1),H,W] in the storage dtype. */
+int ccv3d_oracle_forward_general(int dtype, const void* x, const void* cache, const void* w, const void* b,
+                                 const orc_geom* g, double* out, void* new_cache) {
+    if (!x || !w || !out || !g || !geom_ok(g)) return -1;
+    if (g->cf > 0 && !cache) return -1;
+    const int Ho = out_extent(g->H, g->ph, g->dh, g->kh, g->sh), Wo = out_extent(g->W, g->pw, g->dw, g->kw, g->sw);
+    const int tc = g->dil_t * (g->kt - 1);
+    const int64_t total = (int64_t)g->N * g->Cout * g->T * Ho * Wo;
+#pragma omp parallel for schedule(static)
+    for (int64_t e = 0; e < total; ++e) {
+        int64_t r = e;
+        const int wo = (int)(r % Wo); r /= Wo;
+        const int ho = (int)(r % Ho); r /= Ho;
+        const int t = (int)(r % g->T); r /= g->T;
+        const int co = (int)(r % g->Cout);
+        const int n = (int)(r / g->Cout);
+        double acc = b ? widen(b, dtype, co) : 0.0;
+        for (int ci = 0; ci < g->Cin; ++ci)
+            for (int k = 0; k < g->kt; ++k) {
+                const char* zf = zg_frame(g, dtype, x, cache, n, ci, t + k * g->dil_t);
+                if (!zf) continue;
+                for (int a = 0; a < g->kh; ++a) {
+                    const int hs = ho * g->sh + a * g->dh - g->ph;
+                    if (hs < 0 || hs >= g->H) continue;
+                    for (int c = 0; c < g->kw; ++c) {
+                        const int ws = wo * g->sw + c * g->dw - g->pw;
+                        if (ws < 0 || ws >= g->W) continue;
+                        const double wv =
+                            widen(w, dtype, ((((int64_t)co * g->Cin + ci) * g->kt + k) * g->kh + a) * g->kw + c);
+                        acc += wv * widen(zf, dtype, (int64_t)hs * g->W + ws);
+                    }
+                }
+            }
+        out[e] = acc;
+    }
+    if (new_cache && tc > 0) {
+        const size_t fb = (size_t)g->H * g->W * esize(dtype);
+        for (int n = 0; n < g->N; ++n)
+            for (int ci = 0; ci < g->Cin; ++ci)
+                for (int j = 0; j < tc; ++j) {
+                    char* dst = (char*)new_cache + (size_t)(((int64_t)n * g->Cin + ci) * tc + j) * fb;
+                    const char* zf = zg_frame(g, dtype, x, cache, n, ci, g->T + j);
+                    if (zf) memcpy(dst, zf, fb);
+                    else memset(dst, 0, fb);
+                }
+    }
+    return 0;
 }
