@@ -59,14 +59,26 @@ typedef enum {
                                             the default route in short bursts, ~3 % slower sustained; for callers that cannot afford the workspace. */
 #define CCV3D_FLAG_TC_PER_TAP_A 0x2u    /* tensor-core kernel: fetch the activation tile once per tap (no halo reuse in shared memory) */
 
-/* Layer description, fixed at create time (Algorithm 1's Require line: W, b, p, s, d, g). */
+/* Layer description, fixed at create time (Algorithm 1's Require line: W, b, p, s, d, g).
+ * The supported contract is the paper's (Section 4.1): any spatial stride, padding and dilation of the layer
+ * inside each temporal tap (Eq. (2)), a temporal dilation d_t in the source time (Eq. (1)), unit temporal
+ * stride, one group.  With these the output extents are
+ *   H_o = floor((H + 2 pad_h - dilation[1] (kh-1) - 1) / stride[1]) + 1,   W_o likewise,   T_o = T,
+ * the history a call reads is dilation[0]*(kt-1) frames (the cache length; ccv3d_out_dims reports all three),
+ * and out[n,co,t,ho,wo] = b + sum w[co,ci,k,a,c] * Z[n,ci, t + k d_t, ho s_h + a d_h - pad_h, wo s_w + c d_w - pad_w].
+ * Layers with unit strides and dilations, odd kh and kw and size-preserving padding (pad = (k-1)/2) are the
+ * "standard" geometry of the header comment; only they can use the cooperative-staging, fused, 1x1x1-streaming,
+ * allocation-free and frame-ring paths.  Other geometries run on the tensor-core kernel's run-time tap path
+ * (spatial stride > 1: one strided TMA box per tap) or, for FP32 layers, on the FP32-FMA kernel. */
 typedef struct {
     int32_t cin, cout;            /* channels */
-    int32_t kt, kh, kw;           /* kernel extent; kh and kw must be odd, 1 <= kt <= 8, kh,kw <= 7 */
-    int32_t pad_t, pad_h, pad_w;  /* framework-style padding: must equal (kt-1)/2 if kt is odd else is ignored; (kh-1)/2; (kw-1)/2.
-                                     The causal left pad kt-1 comes from the cache, never from zeros on the right. */
-    int32_t stride[3];            /* must be {1,1,1} */
-    int32_t dilation[3];          /* must be {1,1,1} */
+    int32_t kt, kh, kw;           /* kernel extent; 1 <= kt <= 8, 1 <= kh,kw <= 7 */
+    int32_t pad_t, pad_h, pad_w;  /* pad_h, pad_w: symmetric spatial zero padding, 0..32.  pad_t: the temporal padding is causal - all
+                                     dilation[0]*(kt-1) frames on the left, supplied by the cache, never zeros on the right; the
+                                     framework-style value must describe the same total (2 pad_t = dilation[0]*(kt-1)) when that
+                                     is even and is ignored otherwise. */
+    int32_t stride[3];            /* {1, s_h, s_w}, 1..8; a temporal stride other than 1 is CCV3D_ERR_UNSUPPORTED (as in Algorithm 1) */
+    int32_t dilation[3];          /* {d_t, d_h, d_w}, 1..8 */
     int32_t groups;               /* must be 1 */
     int32_t dtype;                /* ccv3d_dtype of x, cache, w, b and new_cache */
     int32_t out_dtype;            /* ccv3d_dtype of out: F32 layers -> F32; BF16 layers -> BF16 or F32 */
@@ -111,6 +123,8 @@ ccv3d_status ccv3d_create(ccv3d_handle** out_h, const ccv3d_desc* d, const void*
  *   out        DEVICE [N,cout,T,H,W] in out_dtype; fully overwritten.
  *   new_cache  DEVICE [N,cin,kt-1,H,W], or NULL to skip the update; fully overwritten,
  *              bit-exact copy of the last kt-1 frames of [cache ; x].  Ignored when kt == 1.
+ *   (General geometry: out is [N,cout,T,H_o,W_o] and both caches hold dilation[0]*(kt-1) frames; H and W are
+ *   always the INPUT extents.  See ccv3d_out_dims.)
  * out must not overlap x or cache; new_cache must not overlap x, cache or out
  * (CCV3D_ERR_ALIAS): ping-pong two cache buffers.  All pointers must be 16-byte aligned.
  * With CCV3D_FLAG_OVERLAP large images are processed in bands of rows on three side streams owned by the handle
@@ -124,6 +138,10 @@ ccv3d_status ccv3d_create(ccv3d_handle** out_h, const ccv3d_desc* d, const void*
  */
 ccv3d_status ccv3d_forward(ccv3d_handle* h, const void* x, const void* cache, void* out, void* new_cache,
                            int32_t N, int32_t T, int32_t H, int32_t W, void* stream);
+
+/* Output extents and history length of a layer for an input of H x W (HOST outputs, each may be NULL). */
+ccv3d_status ccv3d_out_dims(const ccv3d_handle* h, int32_t H, int32_t W, int32_t* out_h_host, int32_t* out_w_host,
+                            int32_t* cache_frames_host);
 
 /*
  * ccv3d_forward with a history shorter than kt-1 frames (the paper's Table 1 lists such calls: T_c = 1 with

@@ -50,7 +50,7 @@ EXPORTS = ("ccv3d_create", "ccv3d_forward", "ccv3d_forward_host", "ccv3d_workspa
            "ccv3d_get_counters", "ccv3d_device_status", "ccv3d_status_string", "ccv3d_add_bf16",
            "ccv3d_upsample_bf16", "ccv3d_profile_enable", "ccv3d_profile_read", "ccv3d_forward_static", "ccv3d_selftest_wait_timeout", "ccv3d_forward_ex",
            "ccv3d_ring_kb", "ccv3d_ring_bytes", "ccv3d_ring_load", "ccv3d_ring_store", "ccv3d_upsample_ring",
-           "ccv3d_forward_ring")
+           "ccv3d_forward_ring", "ccv3d_out_dims")
 
 
 def _load() -> ctypes.CDLL:
@@ -77,6 +77,8 @@ def _load() -> ctypes.CDLL:
     lib.ccv3d_selftest_wait_timeout.argtypes = [vp, i32, vp]
     lib.ccv3d_add_bf16.argtypes = [vp, vp, vp, ctypes.c_int64, vp]
     lib.ccv3d_upsample_bf16.argtypes = [vp, vp, i32, i32, i32, i32, i32, i32, vp]
+    i32p = ctypes.POINTER(ctypes.c_int32)
+    lib.ccv3d_out_dims.argtypes = [vp, i32, i32, i32p, i32p, i32p]
     rp = ctypes.POINTER(Ring)
     lib.ccv3d_ring_kb.argtypes = [i32]
     lib.ccv3d_ring_bytes.argtypes = [rp]
@@ -143,6 +145,13 @@ def ccv3d_forward_static(h, x, cache, out, new_cache, N, T, H, W, stream=0) -> i
 
 def ccv3d_forward_host(h, x, cache, out, new_cache, N, T, H, W, stream=0) -> int:
     return lib.ccv3d_forward_host(h, x, cache, out, new_cache, N, T, H, W, stream)
+
+
+def ccv3d_out_dims(h, H, W):
+    """(status, H_o, W_o, history frames) of a layer for an H x W input."""
+    a, b, c = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
+    s = lib.ccv3d_out_dims(h, H, W, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c))
+    return s, a.value, b.value, c.value
 
 
 def ccv3d_workspace_bytes(h, N, T, H, W):
@@ -254,7 +263,7 @@ class FrameRing:
 class CausalConv3d:
     """One cached causal Conv3D layer on the current CUDA device (torch tensors in, torch tensors out)."""
 
-    def __init__(self, w, b=None, out_dtype=None, flags=0):
+    def __init__(self, w, b=None, out_dtype=None, flags=0, stride=(1, 1, 1), dilation=(1, 1, 1), pad=None):
         import torch
         assert w.is_cuda and w.is_contiguous() and w.dim() == 5
         self.torch = torch
@@ -263,7 +272,11 @@ class CausalConv3d:
         cout, cin, kt, kh, kw = w.shape
         self.k, self.cin, self.cout = (kt, kh, kw), cin, cout
         self.out_dtype = self.dtype if out_dtype is None else out_dtype
-        self.desc = make_desc(cin, cout, self.k, self.dtype, self.out_dtype, flags)
+        if pad is None:          # size-preserving spatial padding; the temporal entry only has to describe the causal total
+            pad = (dilation[0] * (kt - 1) // 2, dilation[1] * (kh - 1) // 2, dilation[2] * (kw - 1) // 2)
+        self.desc = make_desc(cin, cout, self.k, self.dtype, self.out_dtype, flags, stride=stride, dilation=dilation,
+                              pad=pad)
+        self.tc = dilation[0] * (kt - 1)
         if b is not None:
             assert b.is_cuda and b.is_contiguous() and b.dtype == w.dtype and b.shape == (cout,)
         s, h = ccv3d_create(self.desc, w.data_ptr(), None if b is None else b.data_ptr(),
@@ -276,19 +289,22 @@ class CausalConv3d:
         torch = self.torch
         N, C, T, H, W = x.shape
         assert C == self.cin and x.is_contiguous() and x.is_cuda
-        tc = self.k[0] - 1
+        tc = self.tc
         odt = torch.bfloat16 if self.out_dtype == BF16 else torch.float32
         if out is None:
-            out = torch.empty((N, self.cout, T, H, W), dtype=odt, device=x.device)
+            _, Ho, Wo, _ = ccv3d_out_dims(self.h, H, W)
+            out = torch.empty((N, self.cout, T, Ho, Wo), dtype=odt, device=x.device)
         if new_cache is None and want_cache and tc:
             new_cache = torch.empty((N, C, tc, H, W), dtype=x.dtype, device=x.device)
+        cf = 0
         if cache is not None:
-            assert cache.is_contiguous() and cache.shape == (N, C, tc, H, W) and cache.dtype == x.dtype
-        s = ccv3d_forward(self.h, x.data_ptr(), None if cache is None else cache.data_ptr(), out.data_ptr(),
-                          None if new_cache is None else new_cache.data_ptr(), N, T, H, W,
-                          torch.cuda.current_stream().cuda_stream)
+            cf = cache.shape[2]      # a cache shorter than the full history: the older frames do not exist yet
+            assert cache.is_contiguous() and cache.shape == (N, C, cf, H, W) and cache.dtype == x.dtype and 0 < cf <= tc
+        s = ccv3d_forward_ex(self.h, x.data_ptr(), None if cache is None else cache.data_ptr(), cf, out.data_ptr(),
+                             None if new_cache is None else new_cache.data_ptr(), N, T, H, W,
+                             torch.cuda.current_stream().cuda_stream)
         if s != OK:
-            raise Ccv3dError(s, "ccv3d_forward")
+            raise Ccv3dError(s, "ccv3d_forward_ex")
         return out, new_cache
 
     __call__ = forward
@@ -300,7 +316,7 @@ class CausalConv3d:
                                None if out_ring is None else out_ring.c, out_slot,
                                None if out is None else out.data_ptr(), T, self.torch.cuda.current_stream().cuda_stream)
         if s != OK:
-            raise Ccv3dError(s, "ccv3d_forward_ring")
+            raise Ccv3dError(s, "ccv3d_forward_ring", "ccv3d_out_dims")
         return out_ring if out_ring is not None else out
 
     def counters(self):

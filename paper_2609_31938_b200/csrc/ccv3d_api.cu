@@ -89,18 +89,43 @@ bool overlap(const void* a, uint64_t an, const void* b, uint64_t bn) {
     return a0 < b0 + bn && b0 < a0 + an;
 }
 
+// History frames a layer reads: the causal left pad p_l^base = d_t (kt-1) of Section 4.2.
+inline int hist_len(const ccv3d_desc& d) { return d.dilation[0] * (d.kt - 1); }
+
+// The geometry every route handles: unit strides and dilations, odd kh and kw, padding that preserves H and W.
+// Anything else within the paper's supported contract (spatial stride, padding, dilation; temporal dilation) is
+// "general": served by the FP32-FMA kernel and by the tensor-core kernel's run-time tap path.
+inline bool standard_geom(const ccv3d_desc& d) {
+    for (int i = 0; i < 3; ++i)
+        if (d.stride[i] != 1 || d.dilation[i] != 1) return false;
+    return (d.kh & 1) && (d.kw & 1) && d.pad_h == (d.kh - 1) / 2 && d.pad_w == (d.kw - 1) / 2;
+}
+
+inline int out_extent(int in, int pad, int dil, int k, int stride) {
+    const int span = in + 2 * pad - dil * (k - 1) - 1;
+    return span < 0 ? 0 : span / stride + 1;
+}
+inline int out_h(const ccv3d_desc& d, int H) { return out_extent(H, d.pad_h, d.dilation[1], d.kh, d.stride[1]); }
+inline int out_w(const ccv3d_desc& d, int W) { return out_extent(W, d.pad_w, d.dilation[2], d.kw, d.stride[2]); }
+
 ccv3d_status validate_desc(const ccv3d_desc* d) {
     if (!d) return CCV3D_ERR_INVALID_ARG;
     if (d->cin < 1 || d->cout < 1 || d->kt < 1 || d->kh < 1 || d->kw < 1) return CCV3D_ERR_INVALID_ARG;
     if (d->dtype != CCV3D_F32 && d->dtype != CCV3D_BF16) return CCV3D_ERR_INVALID_ARG;
     if (d->out_dtype != CCV3D_F32 && d->out_dtype != CCV3D_BF16) return CCV3D_ERR_INVALID_ARG;
-    // Algorithm 1 rejects temporal stride != 1 and groups != 1; this build fixes all strides and dilations at 1.
     for (int i = 0; i < 3; ++i)
-        if (d->stride[i] != 1 || d->dilation[i] != 1) return CCV3D_ERR_UNSUPPORTED;
-    if (d->groups != 1) return CCV3D_ERR_UNSUPPORTED;
-    if (!(d->kh & 1) || !(d->kw & 1) || d->kh > 7 || d->kw > 7 || d->kt > 8) return CCV3D_ERR_UNSUPPORTED;
-    if (d->pad_h != (d->kh - 1) / 2 || d->pad_w != (d->kw - 1) / 2) return CCV3D_ERR_UNSUPPORTED;
-    if ((d->kt & 1) && d->pad_t != (d->kt - 1) / 2) return CCV3D_ERR_UNSUPPORTED;
+        if (d->stride[i] < 1 || d->dilation[i] < 1) return CCV3D_ERR_INVALID_ARG;
+    if (d->pad_h < 0 || d->pad_w < 0 || d->pad_t < 0) return CCV3D_ERR_INVALID_ARG;
+    // Algorithm 1 rejects temporal stride != 1 and groups != 1; the spatial stride, padding and dilation of the
+    // layer and its temporal dilation are part of the supported contract (Eq. (1)-(2)).
+    if (d->stride[0] != 1 || d->groups != 1) return CCV3D_ERR_UNSUPPORTED;
+    for (int i = 0; i < 3; ++i)
+        if (d->stride[i] > 8 || d->dilation[i] > 8) return CCV3D_ERR_UNSUPPORTED;
+    if (d->kh > 7 || d->kw > 7 || d->kt > 8 || d->pad_h > 32 || d->pad_w > 32) return CCV3D_ERR_UNSUPPORTED;
+    // the temporal padding is causal: all d_t (kt-1) frames on the left, supplied by the cache.  A framework-style
+    // symmetric value is accepted when it describes the same total (2 pad_t = d_t (kt-1)); nothing else is.
+    const int tc = d->dilation[0] * (d->kt - 1);
+    if (!(tc & 1) && d->pad_t != tc / 2) return CCV3D_ERR_UNSUPPORTED;
     if (d->dtype == CCV3D_F32 && d->out_dtype != CCV3D_F32) return CCV3D_ERR_UNSUPPORTED;
     if (d->cin > 65536 || d->cout > 65536) return CCV3D_ERR_UNSUPPORTED;
     return CCV3D_OK;
@@ -166,14 +191,17 @@ ccv3d_status grow(void** buf, uint64_t* have, uint64_t need) {
     return CCV3D_OK;
 }
 
-ccv3d_status encode_act_map(ccv3d_handle* h, int N, int T, int H, int W, int BW, int BH) {
+// es_w, es_h: traversal strides of the box along w and h (the layer's spatial stride in the per-tap mode, else 1);
+// the box then spans BW*es_w x BH*es_h pixels and delivers BW x BH of them.
+ccv3d_status encode_act_map(ccv3d_handle* h, int N, int T, int H, int W, int BW, int BH, int es_w = 1, int es_h = 1) {
     const TcPlan& pl = h->plan;
-    const int F = h->d.kt - 1 + T;
+    const int F = hist_len(h->d) + T;
     const uint64_t rowb = (uint64_t)pl.KB * 2;
     cuuint64_t dims[5] = {(cuuint64_t)pl.KB, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)pl.CB, (cuuint64_t)N * F};
     cuuint64_t strides[4] = {rowb, rowb * W, rowb * W * H, rowb * W * H * pl.CB};
-    cuuint32_t box[5] = {(cuuint32_t)pl.KB, (cuuint32_t)BW, (cuuint32_t)BH, 1, 1};
-    cuuint32_t es[5] = {1, 1, 1, 1, 1};
+    cuuint32_t box[5] = {(cuuint32_t)pl.KB, (cuuint32_t)(BW * es_w), (cuuint32_t)(BH * es_h), 1, 1};
+    cuuint32_t es[5] = {1, (cuuint32_t)es_w, (cuuint32_t)es_h, 1, 1};
+    if (box[1] > 256 || box[2] > 256) return CCV3D_ERR_UNSUPPORTED;
     CUresult r = h->encode(&h->tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, h->workspace, dims, strides, box, es,
                            CU_TENSOR_MAP_INTERLEAVE_NONE,
                            pl.KB == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
@@ -194,7 +222,7 @@ ccv3d_status encode_out_map(ccv3d_handle* h, void* out, int N, int T, int H, int
 }
 
 uint64_t tc_workspace_bytes(const ccv3d_handle* h, int N, int T, int H, int W) {
-    const int F = h->d.kt - 1 + T;
+    const int F = hist_len(h->d) + T;
     return (uint64_t)N * F * h->plan.cin_pad * H * W * 2;
 }
 
@@ -271,8 +299,11 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
                         int H, int W, cudaStream_t st) {
     const ccv3d_desc& d = h->d;
     const TcPlan& pl = h->plan;
-    const int tc = d.kt - 1;
+    const int tc = hist_len(d);
     const int F = tc + T;
+    const bool general = !standard_geom(d);
+    const int Ho = out_h(d, H), Wo = out_w(d, W);          // output extents; H, W are the input's
+    const bool strided = d.stride[1] > 1 || d.stride[2] > 1;
 
     ccv3d_status s = grow(&h->workspace, &h->workspace_bytes, tc_workspace_bytes(h, N, T, H, W));
     if (s != CCV3D_OK) return s;
@@ -291,35 +322,39 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     const int nframes = F - sp.f_begin;
 
     // ---- implicit GEMM parameters ----
-    const int per_tap = (d.flags & CCV3D_FLAG_TC_PER_TAP_A) ? 1 : 0;
+    // a spatial stride cannot be a shift inside one halo tile: those layers fetch one strided box per tap
+    const int per_tap = ((d.flags & CCV3D_FLAG_TC_PER_TAP_A) || strided) ? 1 : 0;
     // 256-pixel tiles (two 128-pixel blocks sharing every weight tile) unless that leaves SMs without a tile
     int NB = pl.NB;
-    if ((int64_t)N * ((H + 15) / 16) * ((W + 15) / 16) * T * pl.NT < h->sm_count) NB = 1;
+    if ((int64_t)N * ((Ho + 15) / 16) * ((Wo + 15) / 16) * T * pl.NT < h->sm_count) NB = 1;
     // Still fewer than half as many work items as SMs (the 44x80 layers): run half-width output-channel tiles.
     // Twice the items, each streaming half of the weights through its SM - the per-SM weight stream is what
     // bounds a 128-pixel tile - and nothing to reduce afterwards.
     int NT = pl.NT, NPAD = pl.NPAD, split_n = 0;
     if (NB == 1 && !per_tap && pl.NPAD % 32 == 0 &&
-        2 * (int64_t)N * ((H + 15) / 16) * ((W + 7) / 8) * T * pl.NT <= h->sm_count) {
+        2 * (int64_t)N * ((Ho + 15) / 16) * ((Wo + 7) / 8) * T * pl.NT <= h->sm_count) {
         split_n = 1; NT = 2 * pl.NT; NPAD = pl.NPAD / 2;
     }
     const int ACC = (2 * NB * NPAD <= 512) ? 2 : 1;
     const int TW = 8 * NB;
-    const int BW = per_tap ? TW : TW + d.kw - 1;
-    const int BH = per_tap ? 16 : 16 + d.kh - 1;
+    const int BW = per_tap ? TW : TW + (d.kw - 1) * d.dilation[2];
+    const int BH = per_tap ? 16 : 16 + (d.kh - 1) * d.dilation[1];
     ShapeKey key{h->workspace, N, T, H, W, BW};
     if (!(key == h->tm_a_key)) {
-        s = encode_act_map(h, N, T, H, W, BW, BH);
+        s = encode_act_map(h, N, T, H, W, BW, BH, per_tap ? d.stride[2] : 1, per_tap ? d.stride[1] : 1);
         if (s != CCV3D_OK) return s;
         h->tm_a_key = key;
     }
     TcParams p;
     memset(&p, 0, sizeof(p));
-    p.N = N; p.T = T; p.H = H; p.W = W; p.Cout = d.cout; p.F = F;
+    p.N = N; p.T = T; p.H = Ho; p.W = Wo; p.Cout = d.cout; p.F = F;
     p.kt = d.kt; p.kh = d.kh; p.kw = d.kw;
+    p.general = general ? 1 : 0;
+    p.pad_h = d.pad_h; p.pad_w = d.pad_w; p.dil_h = d.dilation[1]; p.dil_w = d.dilation[2]; p.dil_t = d.dilation[0];
+    p.str_h = d.stride[1]; p.str_w = d.stride[2];
     p.CB = pl.CB; p.NT = NT; p.NPAD = NPAD;
-    const int tiles_h = (H + 15) / 16;
-    p.tiles_w = (W + TW - 1) / TW;
+    const int tiles_h = (Ho + 15) / 16;
+    p.tiles_w = (Wo + TW - 1) / TW;
     p.first_frame = tc - cf;
     p.out_f32 = d.out_dtype == CCV3D_F32;
     p.per_tap_a = per_tap;
@@ -329,7 +364,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     p.split_n = split_n;
     p.b_src_tap = split_n ? (uint32_t)pl.NPAD * pl.KB * 2 : 0;
     // epilogue: BF16 output rows that TMA can address (W*2 bytes a multiple of 16) go through shared memory
-    p.epi_tma = (!p.out_f32 && W % 8 == 0) ? 1 : 0;
+    p.epi_tma = (!p.out_f32 && Wo % 8 == 0) ? 1 : 0;
     p.ECH = (NPAD % 32 == 0) ? 32 : 16;
     p.e_slot = p.epi_tma ? (uint32_t)(p.ECH * 16 * TW * 2) : 0;
 
@@ -341,13 +376,13 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     // effect on B200: 0 to -6 % time (the co-resident staging blocks make little headway next to the
     // persistent convolution CTAs), which is why it is not the default.
     int nbands = 1;
-    if ((d.flags & CCV3D_FLAG_OVERLAP) && h->side[0] &&
+    if ((d.flags & CCV3D_FLAG_OVERLAP) && h->side[0] && !general &&
         (int64_t)N * tiles_h * p.tiles_w * T * NT >= 2LL * h->sm_count && tiles_h >= 4)
         nbands = tiles_h / 2 < MAX_BANDS ? tiles_h / 2 : MAX_BANDS;
 
     // Cooperative staging (default when W % 8 == 0): the staging pass runs inside the convolution kernel, on four
     // extra warps per CTA, one band of 16 rows ahead of the tiles that read it.
-    const bool coop = nbands == 1 && !per_tap && !(d.flags & CCV3D_FLAG_TWO_KERNELS) && W % 8 == 0 &&
+    const bool coop = nbands == 1 && !per_tap && !general && !(d.flags & CCV3D_FLAG_TWO_KERNELS) && W % 8 == 0 &&
                       tiles_h <= MAX_COOP_BANDS && tiles_h >= 4 && pl.KB == 64 &&   // 32-channel blocks: the stagers cannot keep up
                       (int64_t)N * tiles_h * p.tiles_w * T * NT >= 4LL * h->sm_count;   // small problems: two kernels
     size_t fixed = 1024 /*alignment slack*/ + align_up(sizeof(TcShared), 128) + 2 * (size_t)p.e_slot + (coop ? 9216 : 0);
@@ -376,13 +411,13 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     p.out = out;
     p.status = h->status;
     if (p.epi_tma) {
-        s = encode_out_map(h, out, N, T, H, W, TW, p.ECH);
+        s = encode_out_map(h, out, N, T, Ho, Wo, TW, p.ECH);
         if (s != CCV3D_OK) return s;
     } else {
         h->tm_o = h->tm_a;  // never dereferenced on this path; any valid descriptor will do
     }
     const size_t smem = fixed + (size_t)SA * p.a_slot + (size_t)SB * p.b_slot;
-    const int ks = (!per_tap && d.kh == d.kw && (d.kh == 1 || d.kh == 3)) ? d.kh : 0;
+    const int ks = (!per_tap && !general && d.kh == d.kw && (d.kh == 1 || d.kh == 3)) ? d.kh : 0;
     const int ph = (d.kh - 1) / 2;
     cudaEvent_t* pev = (h->prof_on && h->prof_ev) ? h->prof_ev + 3 * (h->prof_n % PROF_SLOTS) : nullptr;
 
@@ -483,7 +518,7 @@ ccv3d_status encode_ncthw_map(ccv3d_handle* h, CUtensorMap* tm, const void* base
     return r == CUDA_SUCCESS ? CCV3D_OK : CCV3D_ERR_CUDA;
 }
 
-bool fused_eligible(const ccv3d_handle* h, int W) { return h->plan.fused && W % 8 == 0; }
+bool fused_eligible(const ccv3d_handle* h, int W) { return h->plan.fused && W % 8 == 0 && standard_geom(h->d); }
 
 ccv3d_status forward_fused(ccv3d_handle* h, const void* x, const void* cache, void* out, void* new_cache, int N, int T,
                            int H, int W, cudaStream_t st) {
@@ -592,7 +627,7 @@ ccv3d_status forward_fused(ccv3d_handle* h, const void* x, const void* cache, vo
 bool pointwise_eligible(const ccv3d_handle* h, int T, int H, int W) {
     const ccv3d_desc& d = h->d;
     const TcPlan& pl = h->plan;
-    if (!(d.kt == 1 && d.kh == 1 && d.kw == 1)) return false;
+    if (!(d.kt == 1 && d.kh == 1 && d.kw == 1) || !standard_geom(d)) return false;
     if (d.flags & CCV3D_FLAG_TC_PER_TAP_A) return false;
     if (pl.KB != 64 || pl.NT != 1 || d.out_dtype != CCV3D_BF16) return false;
     if (((int64_t)T * H * W) % 8 != 0) return false;                       // TMA strides are multiples of 16 bytes
@@ -870,7 +905,7 @@ ccv3d_status forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int x_slot, int
     const ccv3d_desc& d = h->d;
     const TcPlan& pl = h->plan;
     const int tc = d.kt - 1;
-    if (!h->use_tc || (d.flags & CCV3D_FLAG_TC_PER_TAP_A)) return CCV3D_ERR_UNSUPPORTED;
+    if (!h->use_tc || (d.flags & CCV3D_FLAG_TC_PER_TAP_A) || !standard_geom(d)) return CCV3D_ERR_UNSUPPORTED;
     if (!ring_valid(in) || T < 1 || (oring != nullptr) == (out_ncthw != nullptr)) return CCV3D_ERR_INVALID_ARG;
     if (((uintptr_t)in->base | (uintptr_t)out_ncthw) & 15u) return CCV3D_ERR_ALIGNMENT;
     if (in->C != d.cin || in->F < T + tc || x_slot < 0 || x_slot >= in->F || hist < 0 || hist > tc) return CCV3D_ERR_INVALID_ARG;
@@ -1011,12 +1046,15 @@ ccv3d_status forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int x_slot, int
 ccv3d_status forward_simt(ccv3d_handle* h, const void* x, const void* cache, void* out, void* new_cache, int N, int T,
                           int H, int W, cudaStream_t st) {
     const ccv3d_desc& d = h->d;
-    const int tc = d.kt - 1;
+    const int tc = hist_len(d);
     SimtParams p;
     const int cf = (tc && cache) ? h->call_cf : 0;
     p.x = x; p.cache = cf ? cache : nullptr; p.cf = cf; p.w = h->w_copy; p.bias = h->bias32; p.out = out;
     p.N = N; p.Cin = d.cin; p.Cout = d.cout; p.T = T; p.H = H; p.W = W; p.kt = d.kt; p.kh = d.kh; p.kw = d.kw;
-    const int64_t npix = (int64_t)N * T * H * W;
+    p.Ho = out_h(d, H); p.Wo = out_w(d, W);
+    p.sh = d.stride[1]; p.sw = d.stride[2]; p.ph = d.pad_h; p.pw = d.pad_w; p.dh = d.dilation[1]; p.dw = d.dilation[2];
+    p.dil_t = d.dilation[0];
+    const int64_t npix = (int64_t)N * T * p.Ho * p.Wo;
     const int64_t gx = (npix + SIMT_THREADS - 1) / SIMT_THREADS;
     if (gx > 0x7FFFFFFF) return CCV3D_ERR_UNSUPPORTED;
     dim3 grid((unsigned)gx, (d.cout + SIMT_CO - 1) / SIMT_CO);
@@ -1067,10 +1105,12 @@ ccv3d_status check_forward_args(const ccv3d_handle* h, const void* x, const void
     const uint64_t px = (uint64_t)N * H * W;
     if ((double)px * T * (d.cin > d.cout ? d.cin : d.cout) > 9.0e15) return CCV3D_ERR_UNSUPPORTED;
     if ((uint64_t)H * W > 0x7FFFFFFFull) return CCV3D_ERR_UNSUPPORTED;
-    const int tc = d.kt - 1;
+    const int tc = hist_len(d);
+    const int Ho = out_h(d, H), Wo = out_w(d, W);
+    if (Ho < 1 || Wo < 1) return CCV3D_ERR_INVALID_ARG;                          // the kernel does not fit the padded input
     const uint64_t xb = px * d.cin * T * esize(d.dtype), cb = px * d.cin * tc * esize(d.dtype);
     const uint64_t ccb = px * d.cin * (uint64_t)h->call_cf * esize(d.dtype);     // bytes of the cache actually passed
-    const uint64_t ob = px * d.cout * T * esize(d.out_dtype);
+    const uint64_t ob = (uint64_t)N * Ho * Wo * d.cout * T * esize(d.out_dtype);
     if (!tc) { cache = nullptr; new_cache = nullptr; }
     if (device_ptrs) {
         const uintptr_t m = (uintptr_t)x | (uintptr_t)cache | (uintptr_t)out | (uintptr_t)new_cache;
@@ -1214,11 +1254,20 @@ ccv3d_status ccv3d_workspace_bytes(const ccv3d_handle* h, int32_t N, int32_t T, 
     return CCV3D_OK;
 }
 
+ccv3d_status ccv3d_out_dims(const ccv3d_handle* h, int32_t H, int32_t W, int32_t* out_h_host, int32_t* out_w_host,
+                            int32_t* cache_frames_host) {
+    if (!h || H < 1 || W < 1) return CCV3D_ERR_INVALID_ARG;
+    if (out_h_host) *out_h_host = out_h(h->d, H);
+    if (out_w_host) *out_w_host = out_w(h->d, W);
+    if (cache_frames_host) *cache_frames_host = hist_len(h->d);
+    return CCV3D_OK;
+}
+
 ccv3d_status ccv3d_forward_ex(ccv3d_handle* h, const void* x, const void* cache, int32_t cache_frames, void* out,
                               void* new_cache, int32_t N, int32_t T, int32_t H, int32_t W, void* stream) {
     if (!h) return CCV3D_ERR_INVALID_ARG;
     h->ctr.calls++;
-    const int tc = h->d.kt - 1;
+    const int tc = hist_len(h->d);
     if (cache_frames < 0 || cache_frames > tc) return count(h, CCV3D_ERR_INVALID_ARG);
     if (cache_frames > 0 && !cache) return count(h, CCV3D_ERR_INVALID_ARG);
     if (cache_frames == 0) cache = nullptr;
@@ -1236,34 +1285,35 @@ ccv3d_status ccv3d_forward_ex(ccv3d_handle* h, const void* x, const void* cache,
 ccv3d_status ccv3d_forward(ccv3d_handle* h, const void* x, const void* cache, void* out, void* new_cache, int32_t N,
                            int32_t T, int32_t H, int32_t W, void* stream) {
     if (!h) return CCV3D_ERR_INVALID_ARG;
-    return ccv3d_forward_ex(h, x, cache, cache ? h->d.kt - 1 : 0, out, new_cache, N, T, H, W, stream);
+    return ccv3d_forward_ex(h, x, cache, cache ? hist_len(h->d) : 0, out, new_cache, N, T, H, W, stream);
 }
 
 ccv3d_status ccv3d_forward_static(ccv3d_handle* h, const void* x, const void* cache, void* out, void* new_cache,
                                   int32_t N, int32_t T, int32_t H, int32_t W, void* stream) {
     if (!h) return CCV3D_ERR_INVALID_ARG;
     h->ctr.calls++;
-    h->call_cf = cache ? h->d.kt - 1 : 0;
+    h->call_cf = cache ? hist_len(h->d) : 0;
     ccv3d_status s = check_forward_args(h, x, cache, out, new_cache, N, T, H, W, true);
     if (s != CCV3D_OK) return count(h, s);
     if (!h->use_tc) return count(h, CCV3D_ERR_UNSUPPORTED);   // the FP32-FMA route has no scratch to replace
+    if (!standard_geom(h->d)) return count(h, CCV3D_ERR_UNSUPPORTED);   // unit stride and dilation, size-preserving padding only
     return count(h, forward_tc_static(h, x, cache, out, new_cache, N, T, H, W, (cudaStream_t)stream));
 }
 
 ccv3d_status ccv3d_forward_host(ccv3d_handle* h, const void* x_host, const void* cache_host, void* out_host,
                                 void* new_cache_host, int32_t N, int32_t T, int32_t H, int32_t W, void* stream) {
     if (!h) return CCV3D_ERR_INVALID_ARG;
-    h->call_cf = cache_host ? h->d.kt - 1 : 0;
+    h->call_cf = cache_host ? hist_len(h->d) : 0;
     ccv3d_status s = check_forward_args(h, x_host, cache_host, out_host, new_cache_host, N, T, H, W, false);
     if (s != CCV3D_OK) {
         h->ctr.calls++;
         return count(h, s);
     }
     const ccv3d_desc& d = h->d;
-    const int tc = d.kt - 1;
+    const int tc = hist_len(d);
     const uint64_t px = (uint64_t)N * H * W;
     const uint64_t xb = px * d.cin * T * esize(d.dtype), cb = px * d.cin * tc * esize(d.dtype);
-    const uint64_t ob = px * d.cout * T * esize(d.out_dtype);
+    const uint64_t ob = (uint64_t)N * out_h(d, H) * out_w(d, W) * d.cout * T * esize(d.out_dtype);
     cudaStream_t st = (cudaStream_t)stream;
     const bool has_c = tc && cache_host, has_n = tc && new_cache_host;
     if ((s = grow(&h->hx, &h->hx_b, xb)) != CCV3D_OK) return s;

@@ -50,13 +50,16 @@ def test_status_strings():
 
 @pytest.mark.parametrize("kwargs,expected", [
     (dict(stride=(2, 1, 1)), ccv.ERR_UNSUPPORTED),       # temporal stride != 1 (Algorithm 1, validation)
-    (dict(stride=(1, 2, 2)), ccv.ERR_UNSUPPORTED),
-    (dict(dilation=(1, 2, 1)), ccv.ERR_UNSUPPORTED),
+    (dict(stride=(1, 9, 1)), ccv.ERR_UNSUPPORTED),       # beyond what a TMA traversal stride can express
+    (dict(stride=(1, 0, 1)), ccv.ERR_INVALID_ARG),
+    (dict(dilation=(1, 0, 1)), ccv.ERR_INVALID_ARG),
+    (dict(dilation=(9, 1, 1)), ccv.ERR_UNSUPPORTED),
     (dict(groups=2), ccv.ERR_UNSUPPORTED),               # groups != 1 (Algorithm 1, validation)
-    (dict(k=(3, 2, 3)), ccv.ERR_UNSUPPORTED),            # even spatial kernel
     (dict(k=(3, 9, 9)), ccv.ERR_UNSUPPORTED),
-    (dict(pad=(1, 0, 1)), ccv.ERR_UNSUPPORTED),          # spatial padding that does not preserve H, W
-    (dict(pad=(0, 1, 1)), ccv.ERR_UNSUPPORTED),
+    (dict(pad=(1, -1, 1)), ccv.ERR_INVALID_ARG),
+    (dict(pad=(1, 40, 1)), ccv.ERR_UNSUPPORTED),
+    (dict(pad=(0, 1, 1)), ccv.ERR_UNSUPPORTED),          # temporal padding that is not the causal total 2 pad_t = d_t (kt-1)
+    (dict(dilation=(2, 1, 1), pad=(1, 1, 1)), ccv.ERR_UNSUPPORTED),
     (dict(dtype=ccv.F32, out_dtype=ccv.BF16), ccv.ERR_UNSUPPORTED),
     (dict(dtype=7), ccv.ERR_INVALID_ARG),
     (dict(cin=0), ccv.ERR_INVALID_ARG),

@@ -1,0 +1,168 @@
+"""GPU parity for the paper's full supported contract (Eq. (1)-(2) as printed): the layer's own spatial stride,
+padding and dilation inside each temporal tap, temporal dilation in the source time, unit temporal stride - on the
+FP32-FMA kernel (FP32 layers, BF16 reference route) and on the tensor-core kernel (halo tiles with dilated tap
+offsets; spatial stride through one strided TMA box per tap).  Same tolerances as the standard geometry; the cache
+update (d_t (kt-1) frames) is bit-exact."""
+import numpy as np
+import pytest
+
+import oracle
+import synth_inputs as si
+from _util import as_f64, bits, check, to_dev
+
+torch = pytest.importorskip("torch")
+pytestmark = pytest.mark.gpu
+
+GUARD = 64
+
+
+@pytest.fixture(scope="module")
+def ccv():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import paper_2609_31938_b200 as m
+    torch.cuda.set_device(0)
+    return m
+
+
+def _guarded(shape, dtype):
+    n = int(np.prod(shape))
+    buf = torch.full((n + 2 * GUARD,), float("nan"), dtype=dtype, device="cuda:0")
+    return buf, buf[GUARD:GUARD + n].view(shape)
+
+
+def _intact(buf):
+    return bool(torch.isnan(buf[:GUARD]).all() and torch.isnan(buf[-GUARD:]).all())
+
+
+def _case(N, Cin, Cout, T, H, W, k, dtype, cf, seed):
+    c = si.conv_case(N, Cin, Cout, T, H, W, k=k, dtype=dtype, cache=None, seed=seed,
+                     x_dist="uniform" if dtype == si.F32 else "normal")
+    draw = (lambda shp: si.uniform(shp, -1.0, 1.0, dtype, seed, si.TID_CACHE)) if dtype == si.F32 else \
+           (lambda shp: si.normal(shp, 1.0, dtype, seed, si.TID_CACHE))
+    c["cache"] = draw((N, Cin, cf, H, W)) if cf else None
+    return c
+
+
+def run_general(ccv, c, stride, pad, dil, dil_t, flags=0, kind=None):
+    kt, kh, kw = c["k"]
+    ref, ref_nc = oracle.forward_general(c["x"], c["cache"], c["w"], c["b"], stride=stride, pad=pad, dil=dil, dil_t=dil_t)
+    tc = dil_t * (kt - 1)
+    layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), flags=flags, stride=(1, *stride), dilation=(dil_t, *dil),
+                             pad=(tc // 2, *pad))
+    x, cache = to_dev(c["x"]), to_dev(c["cache"])
+    N, Cin, T, H, W = c["x"].shape
+    s, Ho, Wo, frames = ccv.ccv3d_out_dims(layer.h, H, W)
+    assert s == ccv.OK and (Ho, Wo) == ref.shape[3:] and frames == tc
+    odt = torch.float32 if c["dtype"] == si.F32 else torch.bfloat16
+    obuf, out = _guarded(ref.shape, odt)
+    nbuf, nc = (_guarded((N, Cin, tc, H, W), x.dtype) if tc else (None, None))
+    layer(x, cache, out=out, new_cache=nc)
+    torch.cuda.synchronize()
+    st, detail = layer.device_status()
+    assert st == ccv.OK, (ccv.status_string(st), hex(detail))
+    assert _intact(obuf) and (nbuf is None or _intact(nbuf)), "guard band overwritten"
+    m = check(as_f64(out), ref, kind or ("f32" if c["dtype"] == si.F32 else "bf16"))
+    if tc:
+        assert np.array_equal(bits(nc), ref_nc), "cache update is not bit-exact"
+    ctr = layer.counters()
+    assert ctr["calls"] == ctr["ok"] == 1 and ctr["unsupported"] == ctr["invalid"] == ctr["cuda_error"] == 0
+    layer.close()
+    return m, ctr
+
+
+GEOMS = [  # k, stride, pad, dil, dil_t
+    ((3, 3, 3), (1, 1), (2, 2), (2, 2), 1),     # dilation 2, size preserved
+    ((3, 3, 3), (1, 1), (0, 0), (1, 1), 1),     # no padding: output shrinks
+    ((3, 3, 3), (1, 1), (1, 1), (1, 1), 2),     # temporal dilation 2: 4 history frames
+    ((3, 3, 3), (2, 2), (1, 1), (1, 1), 1),     # spatial stride 2 (downsampling layer)
+    ((3, 3, 3), (2, 1), (0, 2), (1, 2), 2),     # everything at once
+    ((1, 3, 3), (3, 2), (1, 0), (1, 1), 1),
+    ((2, 2, 2), (1, 1), (1, 0), (1, 1), 3),     # even kernels
+    ((3, 1, 1), (2, 2), (0, 0), (1, 1), 1),     # strided temporal-only kernel
+    ((1, 1, 1), (2, 2), (0, 0), (1, 1), 1),     # strided 1x1x1 (a downsampling shortcut)
+    ((3, 5, 3), (1, 2), (3, 1), (1, 1), 1),
+]
+
+
+@pytest.mark.parametrize("k,stride,pad,dil,dil_t", GEOMS)
+@pytest.mark.parametrize("cache_mode", ["full", "short", "none"])
+def test_fp32_general_geometry(ccv, k, stride, pad, dil, dil_t, cache_mode):
+    tc = dil_t * (k[0] - 1)
+    cf = {"full": tc, "short": tc // 2, "none": 0}[cache_mode]
+    c = _case(2, 5, 7, 3, 13, 18, k, si.F32, cf, seed=31)
+    m, ctr = run_general(ccv, c, stride, pad, dil, dil_t)
+    assert ctr["simt"] == 1
+
+
+@pytest.mark.parametrize("k,stride,pad,dil,dil_t", GEOMS)
+@pytest.mark.parametrize("Cin,Cout,H,W,cache_mode", [(64, 64, 37, 40, "full"), (96, 48, 20, 27, "short"), (32, 200, 18, 33, "none")])
+def test_bf16_tensor_core_general_geometry(ccv, k, stride, pad, dil, dil_t, Cin, Cout, H, W, cache_mode):
+    tc = dil_t * (k[0] - 1)
+    cf = {"full": tc, "short": tc // 2, "none": 0}[cache_mode]
+    c = _case(1, Cin, Cout, 3, H, W, k, si.BF16, cf, seed=32)
+    m, ctr = run_general(ccv, c, stride, pad, dil, dil_t)
+    assert ctr["tcgen05_bf16"] == 1 and ctr["simt"] == 0
+
+
+@pytest.mark.parametrize("k,stride,pad,dil,dil_t", [GEOMS[0], GEOMS[3], GEOMS[4]])
+def test_bf16_fma_route_general_geometry(ccv, k, stride, pad, dil, dil_t):
+    c = _case(1, 24, 20, 2, 11, 14, k, si.BF16, dil_t * (k[0] - 1), seed=33)
+    m, ctr = run_general(ccv, c, stride, pad, dil, dil_t, flags=ccv.FLAG_FORCE_SIMT)
+    assert ctr["simt"] == 1
+
+
+def test_tensor_core_equals_fma_route_closely_on_a_strided_dilated_layer(ccv):
+    """Two independent kernels on the same general layer: both within tolerance of the oracle (above), and within
+    BF16 rounding of each other."""
+    k, stride, pad, dil, dil_t = GEOMS[4]
+    c = _case(1, 64, 64, 3, 33, 40, k, si.BF16, dil_t * (k[0] - 1), seed=34)
+    outs = []
+    for flags in (0, 1):
+        layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), flags=flags, stride=(1, *stride), dilation=(dil_t, *dil),
+                                 pad=(dil_t * (k[0] - 1) // 2, *pad))
+        o, _ = layer(to_dev(c["x"]), to_dev(c["cache"]))
+        outs.append(as_f64(o))
+        layer.close()
+    rms = float(np.sqrt(np.mean(outs[1] ** 2)))
+    assert np.abs(outs[0] - outs[1]).max() <= 2e-2 * rms
+
+
+@pytest.mark.parametrize("chunks", [[1] * 6, [4, 2], [2, 1, 3]])
+def test_streaming_equivalence_with_temporal_dilation_on_gpu(ccv, chunks):
+    k, dil_t = (3, 3, 3), 2
+    c = _case(1, 64, 32, 6, 20, 24, k, si.BF16, 0, seed=35)
+    layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), dilation=(dil_t, 1, 1))
+    x = to_dev(c["x"])
+    whole, whole_nc = layer(x, None)
+    cache, outs, pos = None, [], 0
+    for n in chunks:
+        o, cache = layer(x[:, :, pos:pos + n].contiguous(), cache)
+        outs.append(o)
+        pos += n
+    torch.cuda.synchronize()
+    assert torch.equal(torch.cat(outs, dim=2), whole) and torch.equal(cache, whole_nc)
+    ref, ref_nc = oracle.forward_general(c["x"], None, c["w"], c["b"], dil_t=dil_t)
+    check(as_f64(whole), ref, "bf16")
+    assert np.array_equal(bits(cache), ref_nc)
+    layer.close()
+
+
+def test_general_geometry_is_refused_by_the_standard_only_entry_points(ccv):
+    c = _case(1, 64, 64, 2, 16, 16, (3, 3, 3), si.BF16, 2, seed=36)
+    layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), stride=(1, 2, 2))
+    x, cache = to_dev(c["x"]), to_dev(c["cache"])
+    out = torch.empty((1, 64, 2, 8, 8), dtype=torch.bfloat16, device="cuda")
+    nc = torch.empty_like(cache)
+    st = torch.cuda.current_stream().cuda_stream
+    assert ccv.ccv3d_forward_static(layer.h, x.data_ptr(), cache.data_ptr(), out.data_ptr(), nc.data_ptr(), 1, 2, 16, 16,
+                                    st) == ccv.ERR_UNSUPPORTED
+    rin, rout = ccv.FrameRing(1, 64, 4, 16, 16, zero=True), ccv.FrameRing(1, 64, 2, 16, 16)
+    assert ccv.ccv3d_forward_ring(layer.h, rin.c, 2, 2, None, 0, rout.c, 0, None, 2, st) == ccv.ERR_UNSUPPORTED
+    # an input the kernel does not fit into
+    tiny = torch.empty((1, 64, 2, 1, 1), dtype=torch.bfloat16, device="cuda")
+    valid = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), pad=(1, 0, 0))
+    assert ccv.ccv3d_forward(valid.h, tiny.data_ptr(), None, out.data_ptr(), None, 1, 2, 1, 1, st) == ccv.ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    layer.close()
+    valid.close()
