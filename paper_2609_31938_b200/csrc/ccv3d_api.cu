@@ -417,7 +417,9 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
         h->tm_o = h->tm_a;  // never dereferenced on this path; any valid descriptor will do
     }
     const size_t smem = fixed + (size_t)SA * p.a_slot + (size_t)SB * p.b_slot;
-    const int ks = (!per_tap && !general && d.kh == d.kw && (d.kh == 1 || d.kh == 3)) ? d.kh : 0;
+    // straight-line tap loops need unit spatial dilation (the tap offsets are compile-time); padding and the temporal
+    // dilation only move the producer's TMA coordinates
+    const int ks = (!per_tap && d.dilation[1] == 1 && d.dilation[2] == 1 && d.kh == d.kw && (d.kh == 1 || d.kh == 3)) ? d.kh : 0;
     const int ph = (d.kh - 1) / 2;
     cudaEvent_t* pev = (h->prof_on && h->prof_ev) ? h->prof_ev + 3 * (h->prof_n % PROF_SLOTS) : nullptr;
 
