@@ -74,6 +74,7 @@ struct ccv3d_handle {
     int prof_on;
     int64_t prof_n;
     cudaEvent_t* prof_ev;   // PROF_SLOTS x 3 events, created on first enable
+    int pdl;             // 1: convolution kernels on frame rings are launched with programmatic stream serialization
     int call_cf;         // history frames held by the cache of the call being served (set by the entry points)
     ccv3d_counters ctr;
 };
@@ -736,7 +737,20 @@ ccv3d_status launch_tc_with_maps(ccv3d_handle* h, const CUtensorMap& tm_a, const
         return cuda_fail();
     StageParams nosp;
     memset(&nosp, 0, sizeof(nosp));
-    kern<<<grid, TC_THREADS, smem, st>>>(tm_a, tm_a, tm_o, p, nosp);
+    // programmatic dependent launch: the kernel's set-up may overlap the tail of the previous kernel of the stream
+    // (it waits for that kernel before it touches global data)
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(TC_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = h->pdl ? 1 : 0;
+    if (cudaLaunchKernelEx(&cfg, kern, tm_a, tm_a, tm_o, p, nosp) != cudaSuccess) return cuda_fail();
     if (cudaGetLastError() != cudaSuccess) return cuda_fail();
     h->ctr.kernel_launches++;
     return CCV3D_OK;
@@ -1171,6 +1185,7 @@ ccv3d_status ccv3d_create(ccv3d_handle** out_h, const ccv3d_desc* d, const void*
         const long v = atol(e);
         if (v > 0 && v <= 10000) h->wait_limit_clk = (long long)prop.clockRate * v;
     }
+    h->pdl = getenv("CCV3D_NO_PDL") ? 0 : 1;
     cudaStream_t st = (cudaStream_t)stream;
     const int taps = d->kt * d->kh * d->kw;
 

@@ -653,6 +653,12 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = sh->tmem_base;
+    // Programmatic dependent launch: everything above (barriers, tensor memory) touched no global data, so it may
+    // run while the previous kernel of the stream is still finishing.  From here on the kernel reads what that
+    // kernel wrote: wait for it (returns at once when the launch carried no such dependency), and let the next
+    // kernel of the stream start its own set-up as soon as CTAs of this one retire.
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     // ---------------------------------------------------------------- A producer
     if (warp == 0) {
