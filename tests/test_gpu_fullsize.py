@@ -65,3 +65,44 @@ def test_full_size_sampled(name, cache):
     layer.close()
     del out, nc, x, cch
     torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("name", ["cfg3_bf16_192", "cfg4a_bf16_96"])
+def test_full_size_on_frame_rings_sampled(name):
+    """The resident-activation path at the benchmark's full sizes, in the launch configuration bench.py's
+    `resident` leg times: input and history in a frame ring, output into a frame ring.  Sampled outputs against
+    the oracle, and the whole output bit for bit against the NCTHW entry point."""
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import paper_2609_31938_b200 as ccv
+    torch.cuda.set_device(0)
+    cfg = dict(si.CONFIGS[name])
+    c = si.conv_case(cache="random", **cfg)
+    kt = c["k"][0]
+    N, Cin, T, H, W = c["x"].shape
+    layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]))
+    x, cch = to_dev(c["x"]), to_dev(c["cache"])
+    rin = ccv.FrameRing(N, Cin, T + kt - 1, H, W)
+    rout = ccv.FrameRing(N, cfg["Cout"], T, H, W)
+    rout.buf.fill_(float("nan"))
+    rin.load(T, cch)                       # slots T, T+1 hold the history; x wraps around to slots 0 .. T-1
+    rin.load((T + kt - 1) % rin.F, x)
+    layer.forward_ring(rin, (T + kt - 1) % rin.F, kt - 1, T, out_ring=rout, out_slot=0)
+    out = rout.store(0, T)
+    torch.cuda.synchronize()
+    assert layer.device_status()[0] == ccv.OK
+    idx = _sample_indices(tuple(out.shape), 3000, seed=2)
+    got = out.view(-1)[torch.from_numpy(idx).cuda()].float().cpu().numpy().astype(np.float64)
+    ref = oracle.points(c["x"], c["cache"], c["w"], c["b"], idx)
+    rms = float(np.sqrt(np.mean(ref ** 2)))
+    err = np.abs(got - ref)
+    assert np.isfinite(got).all() and bool(torch.isfinite(out).all())
+    assert err.max() <= 2e-2 * rms and err.mean() <= 2e-3 * rms, (err.max() / rms, err.mean() / rms)
+    del rin, rout
+    torch.cuda.empty_cache()
+    abi, _ = layer(x, cch)
+    torch.cuda.synchronize()
+    assert torch.equal(out, abi)
+    layer.close()
+    del out, abi, x, cch
+    torch.cuda.empty_cache()
