@@ -8,7 +8,7 @@ structurally different restatements used to pin it:
   * ``brute_force``       - materialises the zero-padded Z volume and loops
                             output-outermost in pure Python/numpy (tiny shapes);
   * ``algorithm1_route``  - the paper's Algorithm 1 taken step by step: per
-                            temporal tap the valid output interval of Eq. (3),
+                            temporal tap the valid output interval of Eq. (4),
                             one 2-D correlation per tap folded over the
                             interval, accumulation, bias once.
 
@@ -47,7 +47,7 @@ _lib = None
 
 class _Geom(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in ("N", "Cin", "Cout", "T", "H", "W", "kt", "kh", "kw", "sh", "sw", "ph", "pw",
-                                            "dh", "dw", "dil_t", "cf")]
+                                            "dh", "dw", "dil_t", "cf", "st")]
 
 
 def _load():
@@ -64,7 +64,7 @@ def _load():
         lib.ccv3d_oracle_cache_update.restype = i
         lib.ccv3d_oracle_forward_general.argtypes = [i, p, p, p, p, ctypes.POINTER(_Geom), p, p]
         lib.ccv3d_oracle_forward_general.restype = i
-        lib.ccv3d_oracle_out_dims.argtypes = [ctypes.POINTER(_Geom), ctypes.POINTER(i), ctypes.POINTER(i)]
+        lib.ccv3d_oracle_out_dims.argtypes = [ctypes.POINTER(_Geom), ctypes.POINTER(i), ctypes.POINTER(i), ctypes.POINTER(i)]
         lib.ccv3d_oracle_out_dims.restype = i
         _lib = lib
     return _lib
@@ -127,11 +127,12 @@ def points(x, cache, w, b, flat_idx):
     return vals
 
 
-def forward_general(x, cache, w, b, stride=(1, 1), pad=None, dil=(1, 1), dil_t=1, want_cache: bool = True):
+def forward_general(x, cache, w, b, stride=(1, 1), pad=None, dil=(1, 1), dil_t=1, want_cache: bool = True, stride_t=1):
     """The operator with the paper's full supported contract (Eq. (1)-(2) with s, p, d and d_t; unit temporal
     stride): spatial stride/padding/dilation per tap, temporal dilation, a cache of up to d_t (kt-1) frames
-    (fewer = older history absent).  pad None = ((kh-1) d_h / 2, (kw-1) d_w / 2).
-    Returns (out float64 [N,Cout,T,H_o,W_o], new_cache [N,Cin,d_t (kt-1),H,W] or None)."""
+    (fewer = older history absent).  pad None = ((kh-1) d_h / 2, (kw-1) d_w / 2).  stride_t > 1 (outside the
+    paper's method, which rejects it): output frame o reads Z frames o s_t + k d_t, T_o = floor((T-1)/s_t) + 1.
+    Returns (out float64 [N,Cout,T_o,H_o,W_o], new_cache [N,Cin,d_t (kt-1),H,W] or None)."""
     dt = _dtype_of(x)
     x, w = np.ascontiguousarray(x), np.ascontiguousarray(w)
     assert _dtype_of(w) == dt
@@ -151,11 +152,11 @@ def forward_general(x, cache, w, b, stride=(1, 1), pad=None, dil=(1, 1), dil_t=1
     if b is not None:
         b = np.ascontiguousarray(b)
         assert _dtype_of(b) == dt and b.shape == (Cout,)
-    g = _Geom(N, Cin, Cout, T, H, W, kt, kh, kw, stride[0], stride[1], pad[0], pad[1], dil[0], dil[1], dil_t, cf)
-    ho, wo = ctypes.c_int(), ctypes.c_int()
-    if _load().ccv3d_oracle_out_dims(ctypes.byref(g), ctypes.byref(ho), ctypes.byref(wo)) != 0:
+    g = _Geom(N, Cin, Cout, T, H, W, kt, kh, kw, stride[0], stride[1], pad[0], pad[1], dil[0], dil[1], dil_t, cf, stride_t)
+    to, ho, wo = ctypes.c_int(), ctypes.c_int(), ctypes.c_int()
+    if _load().ccv3d_oracle_out_dims(ctypes.byref(g), ctypes.byref(to), ctypes.byref(ho), ctypes.byref(wo)) != 0:
         raise ValueError("bad geometry")
-    out = np.empty((N, Cout, T, ho.value, wo.value), dtype=np.float64)
+    out = np.empty((N, Cout, to.value, ho.value, wo.value), dtype=np.float64)
     nc = np.empty((N, Cin, tc, H, W), dtype=x.dtype) if (want_cache and tc > 0) else None
     rc = _load().ccv3d_oracle_forward_general(dt, _ptr(x), _ptr(cache), _ptr(w), _ptr(b), ctypes.byref(g), _ptr(out),
                                               _ptr(nc))
@@ -164,7 +165,7 @@ def forward_general(x, cache, w, b, stride=(1, 1), pad=None, dil=(1, 1), dil_t=1
     return out, nc
 
 
-def brute_force_general(x, cache, w, b, stride=(1, 1), pad=(0, 0), dil=(1, 1), dil_t=1):
+def brute_force_general(x, cache, w, b, stride=(1, 1), pad=(0, 0), dil=(1, 1), dil_t=1, stride_t=1):
     """The same contract on a materialised, zero-padded Z volume with strided slicing per tap (pure numpy,
     tap-outermost: structurally different from the C routine).  Tiny shapes only."""
     xd, cd, wd, bd = _widen(x), _widen(cache), _widen(w), _widen(b)
@@ -179,13 +180,14 @@ def brute_force_general(x, cache, w, b, stride=(1, 1), pad=(0, 0), dil=(1, 1), d
     Zp[:, :, tc:, ph:ph + H, pw:pw + W] = xd
     Ho = (H + 2 * ph - dil[0] * (kh - 1) - 1) // stride[0] + 1
     Wo = (W + 2 * pw - dil[1] * (kw - 1) - 1) // stride[1] + 1
-    out = np.zeros((N, Cout, T, Ho, Wo))
+    To = (T - 1) // stride_t + 1
+    out = np.zeros((N, Cout, To, Ho, Wo))
     if bd is not None:
         out += bd[None, :, None, None, None]
     for k in range(kt):
         for a in range(kh):
             for c in range(kw):
-                src = Zp[:, :, k * dil_t:k * dil_t + T,
+                src = Zp[:, :, k * dil_t:k * dil_t + (To - 1) * stride_t + 1:stride_t,
                          a * dil[0]:a * dil[0] + (Ho - 1) * stride[0] + 1:stride[0],
                          c * dil[1]:c * dil[1] + (Wo - 1) * stride[1] + 1:stride[1]]          # [N,Cin,T,Ho,Wo]
                 out += np.einsum("nithw,oi->nothw", src, wd[:, :, k, a, c])
@@ -242,7 +244,7 @@ def brute_force(x, cache, w, b):
 
 
 def tap_intervals(kt: int, cache_frames: int, T: int, dil_t: int = 1):
-    """Eq. (3): per temporal tap k the valid output interval [o_l, o_h) and its
+    """Eq. (4): per temporal tap k the valid output interval [o_l, o_h) and its
     source interval [z_l, z_h) in Z = [C ; X], with p_l^base = d_t (kt-1),
     p_l = p_l^base - |C|, p_r = 0 and unit temporal stride.  Returns (T_o, list)."""
     p_base = dil_t * (kt - 1)
@@ -274,7 +276,7 @@ def _corr2d_same(img, ker):
 
 def algorithm1_route(x, cache, w, b):
     """Algorithm 1, literally: Z = [C;X] if cached else X; for each temporal tap the
-    interval of Eq. (3); skip empty taps; fold the source interval into the batch; one
+    interval of Eq. (4); skip empty taps; fold the source interval into the batch; one
     2-D correlation with W_k; accumulate into A[:, o_l:o_h]; add the bias once."""
     xd, cd, wd, bd = _widen(x), _widen(cache), _widen(w), _widen(b)
     N, Cin, T, H, W = xd.shape

@@ -33,7 +33,7 @@
  * layer's own spatial stride, padding and dilation and a temporal dilation
  * (Eq. (1)-(2) as printed); its pins are in tests/test_oracle_general.py:
  * hand-worked values, bit-for-bit reduction to ccv3d_oracle_forward, a numpy
- * routine of different structure, the fp64 library conv3d, Eq. (3)'s interval
+ * routine of different structure, the fp64 library conv3d, Eq. (4)'s interval
  * route, streaming equivalence and causality under temporal dilation.
  */
 #include <stdint.h>
@@ -225,6 +225,7 @@ typedef struct {
     int kt, kh, kw;
     int sh, sw, ph, pw, dh, dw, dil_t;
     int cf; /* frames the cache holds */
+    int st; /* temporal stride (the paper's method itself handles 1 only; Eq. (3) "output time" is printed for any s_t) */
 } orc_geom;
 
 static inline int out_extent(int in, int pad, int dil, int k, int stride) {
@@ -247,38 +248,44 @@ static inline const char* zg_frame(const orc_geom* g, int dtype, const void* x, 
 static int geom_ok(const orc_geom* g) {
     if (g->N < 1 || g->Cin < 1 || g->Cout < 1 || g->T < 1 || g->H < 1 || g->W < 1) return 0;
     if (g->kt < 1 || g->kh < 1 || g->kw < 1) return 0;
-    if (g->sh < 1 || g->sw < 1 || g->dh < 1 || g->dw < 1 || g->dil_t < 1 || g->ph < 0 || g->pw < 0) return 0;
+    if (g->sh < 1 || g->sw < 1 || g->dh < 1 || g->dw < 1 || g->dil_t < 1 || g->ph < 0 || g->pw < 0 || g->st < 1) return 0;
     if (g->cf < 0 || g->cf > g->dil_t * (g->kt - 1)) return 0;
     return 1;
 }
 
-int ccv3d_oracle_out_dims(const orc_geom* g, int* Ho, int* Wo) {
+/* T_o of the output-time equation with |Z| + p_l = d_t (kt-1) + T and p_r = 0: floor((T - 1) / s_t) + 1. */
+static inline int out_frames(const orc_geom* g) { return (g->T - 1) / g->st + 1; }
+
+int ccv3d_oracle_out_dims(const orc_geom* g, int* To, int* Ho, int* Wo) {
     if (!g || !geom_ok(g)) return -1;
+    *To = out_frames(g);
     *Ho = out_extent(g->H, g->ph, g->dh, g->kh, g->sh);
     *Wo = out_extent(g->W, g->pw, g->dw, g->kw, g->sw);
     return 0;
 }
 
-/* out: double[N,Cout,T,H_o,W_o]; new_cache (may be NULL): [N,Cin,d_t(kt-1),H,W] in the storage dtype. */
+/* With a temporal stride s_t the source time of tap k for output frame o is o s_t + k d_t (in Z), and there are T_o
+ * output frames.  out: double[N,Cout,T_o,H_o,W_o]; new_cache (may be NULL): [N,Cin,d_t(kt-1),H,W] in the storage dtype. */
 int ccv3d_oracle_forward_general(int dtype, const void* x, const void* cache, const void* w, const void* b,
                                  const orc_geom* g, double* out, void* new_cache) {
     if (!x || !w || !out || !g || !geom_ok(g)) return -1;
     if (g->cf > 0 && !cache) return -1;
     const int Ho = out_extent(g->H, g->ph, g->dh, g->kh, g->sh), Wo = out_extent(g->W, g->pw, g->dw, g->kw, g->sw);
     const int tc = g->dil_t * (g->kt - 1);
-    const int64_t total = (int64_t)g->N * g->Cout * g->T * Ho * Wo;
+    const int To = out_frames(g);
+    const int64_t total = (int64_t)g->N * g->Cout * To * Ho * Wo;
 #pragma omp parallel for schedule(static)
     for (int64_t e = 0; e < total; ++e) {
         int64_t r = e;
         const int wo = (int)(r % Wo); r /= Wo;
         const int ho = (int)(r % Ho); r /= Ho;
-        const int t = (int)(r % g->T); r /= g->T;
+        const int t = (int)(r % To); r /= To;
         const int co = (int)(r % g->Cout);
         const int n = (int)(r / g->Cout);
         double acc = b ? widen(b, dtype, co) : 0.0;
         for (int ci = 0; ci < g->Cin; ++ci)
             for (int k = 0; k < g->kt; ++k) {
-                const char* zf = zg_frame(g, dtype, x, cache, n, ci, t + k * g->dil_t);
+                const char* zf = zg_frame(g, dtype, x, cache, n, ci, t * g->st + k * g->dil_t);
                 if (!zf) continue;
                 for (int a = 0; a < g->kh; ++a) {
                     const int hs = ho * g->sh + a * g->dh - g->ph;

@@ -1,7 +1,7 @@
 """Pins for the oracle of the paper's full supported contract (spatial stride, padding, dilation per temporal tap;
 temporal dilation; unit temporal stride - Eq. (1)-(2) as printed): hand-worked values, bit-for-bit reduction to the
 already pinned unit-stride oracle, a structurally different numpy routine, the fp64 library conv3d on the explicitly
-concatenated and padded input, Eq. (3)'s intervals, and the streaming/causality invariants with temporal dilation."""
+concatenated and padded input, Eq. (4)'s intervals, and the streaming/causality invariants with temporal dilation."""
 import json
 import os
 import zlib
@@ -31,13 +31,14 @@ def test_hand_examples_general():
             x = conv(c["x"]).reshape(1, 1, c["T"], 1, c["W"])
             w = conv(c["w"]).reshape(1, 1, *c["k"])
             cache = None if c["cache"] is None else conv(c["cache"]).reshape(1, 1, -1, 1, c["W"])
+            st = c.get("stride_t", 1)
             out, nc = oracle.forward_general(x, cache, w, conv(c["b"]), stride=c["stride"], pad=c["pad"], dil=c["dil"],
-                                             dil_t=c["dil_t"])
+                                             dil_t=c["dil_t"], stride_t=st)
             assert out.ravel().tolist() == c["out"], c["name"]
             if c["new_cache"] is not None:
                 assert si.to_f64(nc).ravel().tolist() == c["new_cache"], c["name"]
             bf, bnc = oracle.brute_force_general(x, cache, w, conv(c["b"]), stride=c["stride"], pad=c["pad"],
-                                                 dil=c["dil"], dil_t=c["dil_t"])
+                                                 dil=c["dil"], dil_t=c["dil_t"], stride_t=st)
             assert bf.ravel().tolist() == c["out"], c["name"]
 
 
@@ -67,14 +68,15 @@ GEOMS = [  # k, stride, pad, dil, dil_t
 
 @pytest.mark.parametrize("k,stride,pad,dil,dil_t", GEOMS)
 @pytest.mark.parametrize("cache_mode", ["full", "short", "none"])
-def test_general_against_numpy_routine_and_library_conv3d(k, stride, pad, dil, dil_t, cache_mode):
+@pytest.mark.parametrize("stride_t", [1, 2, 3])
+def test_general_against_numpy_routine_and_library_conv3d(k, stride, pad, dil, dil_t, cache_mode, stride_t):
     torch = pytest.importorskip("torch")
-    rng = np.random.default_rng(zlib.crc32(repr((k, stride, pad, dil, dil_t, cache_mode)).encode()))
+    rng = np.random.default_rng(zlib.crc32(repr((k, stride, pad, dil, dil_t, cache_mode, stride_t)).encode()))
     tc = dil_t * (k[0] - 1)
     cf = {"full": tc, "short": tc // 2, "none": 0}[cache_mode]
-    x, cache, w, b = _case(rng, 2, 3, 4, 3, 9, 8, k, cf)
-    out, nc = oracle.forward_general(x, cache, w, b, stride=stride, pad=pad, dil=dil, dil_t=dil_t)
-    bf, bnc = oracle.brute_force_general(x, cache, w, b, stride=stride, pad=pad, dil=dil, dil_t=dil_t)
+    x, cache, w, b = _case(rng, 2, 3, 4, 3 + stride_t, 9, 8, k, cf)
+    out, nc = oracle.forward_general(x, cache, w, b, stride=stride, pad=pad, dil=dil, dil_t=dil_t, stride_t=stride_t)
+    bf, bnc = oracle.brute_force_general(x, cache, w, b, stride=stride, pad=pad, dil=dil, dil_t=dil_t, stride_t=stride_t)
     scale = np.abs(out).max() + 1.0
     assert out.shape == bf.shape and np.abs(out - bf).max() <= 1e-12 * scale
     if tc:
@@ -84,12 +86,12 @@ def test_general_against_numpy_routine_and_library_conv3d(k, stride, pad, dil, d
     parts = [np.zeros((2, 3, tc - cf, 9, 8))] + ([cache.astype(np.float64)] if cf else []) + [x.astype(np.float64)]
     Z = torch.from_numpy(np.concatenate(parts, axis=2))
     ref = torch.nn.functional.conv3d(Z, torch.from_numpy(w.astype(np.float64)), torch.from_numpy(b.astype(np.float64)),
-                                     stride=(1, *stride), padding=(0, *pad), dilation=(dil_t, *dil)).numpy()
+                                     stride=(stride_t, *stride), padding=(0, *pad), dilation=(dil_t, *dil)).numpy()
     assert ref.shape == out.shape and np.abs(out - ref).max() <= 1e-12 * scale
 
 
 def test_interval_route_with_temporal_dilation_equals_the_definition():
-    """Algorithm 1's accumulation over Eq. (3) intervals, with d_t in the tap offset: per tap one strided, dilated
+    """Algorithm 1's accumulation over Eq. (4) intervals, with d_t in the tap offset: per tap one strided, dilated
     2-D correlation of the source interval, added into the output interval."""
     rng = np.random.default_rng(5)
     k, stride, pad, dil, dil_t = (3, 3, 3), (2, 1), (1, 2), (1, 2), 2
@@ -122,6 +124,22 @@ def test_streaming_equivalence_with_temporal_dilation(chunks):
     cache, outs, pos = None, [], 0
     for n in chunks:
         o, cache = oracle.forward_general(x[:, :, pos:pos + n], cache, w, b, stride=(2, 1), pad=(1, 1), dil_t=dil_t)
+        outs.append(o)
+        pos += n
+    assert np.array_equal(np.concatenate(outs, axis=2), whole) and np.array_equal(cache, whole_nc)
+
+
+@pytest.mark.parametrize("chunks", [[2, 2, 2, 2], [4, 4], [6, 2]])
+def test_streaming_equivalence_with_temporal_stride(chunks):
+    """Chunks whose lengths are multiples of s_t keep the phase of the strided output frames, so chunked calls
+    with the cache carried equal the whole-sequence run bit for bit."""
+    rng = np.random.default_rng(9)
+    x, _, w, b = _case(rng, 1, 3, 2, sum(chunks), 5, 4, (3, 3, 3), 0)
+    whole, whole_nc = oracle.forward_general(x, None, w, b, stride_t=2)
+    assert whole.shape[2] == sum(chunks) // 2
+    cache, outs, pos = None, [], 0
+    for n in chunks:
+        o, cache = oracle.forward_general(x[:, :, pos:pos + n], cache, w, b, stride_t=2)
         outs.append(o)
         pos += n
     assert np.array_equal(np.concatenate(outs, axis=2), whole) and np.array_equal(cache, whole_nc)

@@ -55,7 +55,7 @@ def test_interval_algebra_matches_worked_cases_and_brute_force():
         T_o, taps = oracle.tap_intervals(3, c["cache_frames"], c["T"])
         assert T_o == c["T"]
         assert [[k, ol, oh] for (k, ol, oh, _, _) in taps] == c["taps"]
-    # Eq. (3) against direct enumeration of Eq. (1) for a range of kernels, dilations, caches
+    # Eq. (4) against direct enumeration of Eq. (1) for a range of kernels, dilations, caches
     for kt in (1, 2, 3):
         for dil in (1, 2):
             for nC in range(0, dil * (kt - 1) + 1):
