@@ -61,11 +61,14 @@ typedef enum {
 
 /* Layer description, fixed at create time (Algorithm 1's Require line: W, b, p, s, d, g).
  * The supported contract is the paper's (Section 4.1): any spatial stride, padding and dilation of the layer
- * inside each temporal tap (Eq. (2)), a temporal dilation d_t in the source time (Eq. (1)), unit temporal
- * stride, one group.  With these the output extents are
- *   H_o = floor((H + 2 pad_h - dilation[1] (kh-1) - 1) / stride[1]) + 1,   W_o likewise,   T_o = T,
- * the history a call reads is dilation[0]*(kt-1) frames (the cache length; ccv3d_out_dims reports all three),
- * and out[n,co,t,ho,wo] = b + sum w[co,ci,k,a,c] * Z[n,ci, t + k d_t, ho s_h + a d_h - pad_h, wo s_w + c d_w - pad_w].
+ * inside each temporal tap (Eq. (2)), a temporal dilation d_t in the source time (Eq. (1)), one group - plus a
+ * temporal stride s_t, which the paper's Algorithm 1 hands back to the framework (the encoder's temporal
+ * downsampling layers) and which is here the same operator with source time t s_t + k d_t.  The output extents are
+ *   H_o = floor((H + 2 pad_h - dilation[1] (kh-1) - 1) / stride[1]) + 1,   W_o likewise,
+ *   T_o = floor((T - 1) / stride[0]) + 1                 (Eq. (3) with the causal pad supplied in full),
+ * the history a call reads is dilation[0]*(kt-1) frames (the cache length; ccv3d_out_dims reports all four),
+ * and out[n,co,t,ho,wo] = b + sum w[co,ci,k,a,c] * Z[n,ci, t s_t + k d_t, ho s_h + a d_h - pad_h, wo s_w + c d_w - pad_w].
+ * Streaming with s_t > 1: chunk lengths that are multiples of s_t keep the phase of the output frames.
  * Layers with unit strides and dilations, odd kh and kw and size-preserving padding (pad = (k-1)/2) are the
  * "standard" geometry of the header comment; only they can use the cooperative-staging, fused, 1x1x1-streaming,
  * allocation-free and frame-ring paths.  Other geometries run on the tensor-core kernel's run-time tap path
@@ -77,7 +80,7 @@ typedef struct {
                                      dilation[0]*(kt-1) frames on the left, supplied by the cache, never zeros on the right; the
                                      framework-style value must describe the same total (2 pad_t = dilation[0]*(kt-1)) when that
                                      is even and is ignored otherwise. */
-    int32_t stride[3];            /* {1, s_h, s_w}, 1..8; a temporal stride other than 1 is CCV3D_ERR_UNSUPPORTED (as in Algorithm 1) */
+    int32_t stride[3];            /* {s_t, s_h, s_w}, 1..8 */
     int32_t dilation[3];          /* {d_t, d_h, d_w}, 1..8 */
     int32_t groups;               /* must be 1 */
     int32_t dtype;                /* ccv3d_dtype of x, cache, w, b and new_cache */
@@ -123,8 +126,8 @@ ccv3d_status ccv3d_create(ccv3d_handle** out_h, const ccv3d_desc* d, const void*
  *   out        DEVICE [N,cout,T,H,W] in out_dtype; fully overwritten.
  *   new_cache  DEVICE [N,cin,kt-1,H,W], or NULL to skip the update; fully overwritten,
  *              bit-exact copy of the last kt-1 frames of [cache ; x].  Ignored when kt == 1.
- *   (General geometry: out is [N,cout,T,H_o,W_o] and both caches hold dilation[0]*(kt-1) frames; H and W are
- *   always the INPUT extents.  See ccv3d_out_dims.)
+ *   (General geometry: out is [N,cout,T_o,H_o,W_o] and both caches hold dilation[0]*(kt-1) frames; T, H and W
+ *   are always the INPUT extents.  See ccv3d_out_dims.)
  * out must not overlap x or cache; new_cache must not overlap x, cache or out
  * (CCV3D_ERR_ALIAS): ping-pong two cache buffers.  All pointers must be 16-byte aligned.
  * With CCV3D_FLAG_OVERLAP large images are processed in bands of rows on three side streams owned by the handle
@@ -139,9 +142,9 @@ ccv3d_status ccv3d_create(ccv3d_handle** out_h, const ccv3d_desc* d, const void*
 ccv3d_status ccv3d_forward(ccv3d_handle* h, const void* x, const void* cache, void* out, void* new_cache,
                            int32_t N, int32_t T, int32_t H, int32_t W, void* stream);
 
-/* Output extents and history length of a layer for an input of H x W (HOST outputs, each may be NULL). */
-ccv3d_status ccv3d_out_dims(const ccv3d_handle* h, int32_t H, int32_t W, int32_t* out_h_host, int32_t* out_w_host,
-                            int32_t* cache_frames_host);
+/* Output extents and history length of a layer for an input of T x H x W (HOST outputs, each may be NULL). */
+ccv3d_status ccv3d_out_dims(const ccv3d_handle* h, int32_t T, int32_t H, int32_t W, int32_t* out_t_host,
+                            int32_t* out_h_host, int32_t* out_w_host, int32_t* cache_frames_host);
 
 /*
  * ccv3d_forward with a history shorter than kt-1 frames (the paper's Table 1 lists such calls: T_c = 1 with

@@ -78,7 +78,7 @@ def _load() -> ctypes.CDLL:
     lib.ccv3d_add_bf16.argtypes = [vp, vp, vp, ctypes.c_int64, vp]
     lib.ccv3d_upsample_bf16.argtypes = [vp, vp, i32, i32, i32, i32, i32, i32, vp]
     i32p = ctypes.POINTER(ctypes.c_int32)
-    lib.ccv3d_out_dims.argtypes = [vp, i32, i32, i32p, i32p, i32p]
+    lib.ccv3d_out_dims.argtypes = [vp, i32, i32, i32, i32p, i32p, i32p, i32p]
     rp = ctypes.POINTER(Ring)
     lib.ccv3d_ring_kb.argtypes = [i32]
     lib.ccv3d_ring_bytes.argtypes = [rp]
@@ -147,11 +147,11 @@ def ccv3d_forward_host(h, x, cache, out, new_cache, N, T, H, W, stream=0) -> int
     return lib.ccv3d_forward_host(h, x, cache, out, new_cache, N, T, H, W, stream)
 
 
-def ccv3d_out_dims(h, H, W):
-    """(status, H_o, W_o, history frames) of a layer for an H x W input."""
-    a, b, c = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
-    s = lib.ccv3d_out_dims(h, H, W, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c))
-    return s, a.value, b.value, c.value
+def ccv3d_out_dims(h, T, H, W):
+    """(status, T_o, H_o, W_o, history frames) of a layer for a T x H x W input."""
+    t, a, b, c = ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32(), ctypes.c_int32()
+    s = lib.ccv3d_out_dims(h, T, H, W, ctypes.byref(t), ctypes.byref(a), ctypes.byref(b), ctypes.byref(c))
+    return s, t.value, a.value, b.value, c.value
 
 
 def ccv3d_workspace_bytes(h, N, T, H, W):
@@ -292,8 +292,8 @@ class CausalConv3d:
         tc = self.tc
         odt = torch.bfloat16 if self.out_dtype == BF16 else torch.float32
         if out is None:
-            _, Ho, Wo, _ = ccv3d_out_dims(self.h, H, W)
-            out = torch.empty((N, self.cout, T, Ho, Wo), dtype=odt, device=x.device)
+            _, To, Ho, Wo, _ = ccv3d_out_dims(self.h, T, H, W)
+            out = torch.empty((N, self.cout, To, Ho, Wo), dtype=odt, device=x.device)
         if new_cache is None and want_cache and tc:
             new_cache = torch.empty((N, C, tc, H, W), dtype=x.dtype, device=x.device)
         cf = 0

@@ -106,6 +106,7 @@ inline int out_extent(int in, int pad, int dil, int k, int stride) {
     const int span = in + 2 * pad - dil * (k - 1) - 1;
     return span < 0 ? 0 : span / stride + 1;
 }
+inline int out_t(const ccv3d_desc& d, int T) { return (T - 1) / d.stride[0] + 1; }   // Eq. (3) with |Z| + p_l = d_t (kt-1) + T
 inline int out_h(const ccv3d_desc& d, int H) { return out_extent(H, d.pad_h, d.dilation[1], d.kh, d.stride[1]); }
 inline int out_w(const ccv3d_desc& d, int W) { return out_extent(W, d.pad_w, d.dilation[2], d.kw, d.stride[2]); }
 
@@ -117,9 +118,10 @@ ccv3d_status validate_desc(const ccv3d_desc* d) {
     for (int i = 0; i < 3; ++i)
         if (d->stride[i] < 1 || d->dilation[i] < 1) return CCV3D_ERR_INVALID_ARG;
     if (d->pad_h < 0 || d->pad_w < 0 || d->pad_t < 0) return CCV3D_ERR_INVALID_ARG;
-    // Algorithm 1 rejects temporal stride != 1 and groups != 1; the spatial stride, padding and dilation of the
-    // layer and its temporal dilation are part of the supported contract (Eq. (1)-(2)).
-    if (d->stride[0] != 1 || d->groups != 1) return CCV3D_ERR_UNSUPPORTED;
+    // Algorithm 1 rejects groups != 1.  The spatial stride, padding and dilation of the layer and its temporal
+    // dilation are part of the paper's supported contract (Eq. (1)-(2)); a temporal stride is not (Algorithm 1
+    // sends it to the framework) but is the same operator with source time o s_t + k d_t and T_o from Eq. (3).
+    if (d->groups != 1) return CCV3D_ERR_UNSUPPORTED;
     for (int i = 0; i < 3; ++i)
         if (d->stride[i] > 8 || d->dilation[i] > 8) return CCV3D_ERR_UNSUPPORTED;
     if (d->kh > 7 || d->kw > 7 || d->kt > 8 || d->pad_h > 32 || d->pad_w > 32) return CCV3D_ERR_UNSUPPORTED;
@@ -303,7 +305,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     const int tc = hist_len(d);
     const int F = tc + T;
     const bool general = !standard_geom(d);
-    const int Ho = out_h(d, H), Wo = out_w(d, W);          // output extents; H, W are the input's
+    const int Ho = out_h(d, H), Wo = out_w(d, W), To = out_t(d, T);   // output extents; T, H, W are the input's
     const bool strided = d.stride[1] > 1 || d.stride[2] > 1;
 
     ccv3d_status s = grow(&h->workspace, &h->workspace_bytes, tc_workspace_bytes(h, N, T, H, W));
@@ -327,13 +329,13 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     const int per_tap = ((d.flags & CCV3D_FLAG_TC_PER_TAP_A) || strided) ? 1 : 0;
     // 256-pixel tiles (two 128-pixel blocks sharing every weight tile) unless that leaves SMs without a tile
     int NB = pl.NB;
-    if ((int64_t)N * ((Ho + 15) / 16) * ((Wo + 15) / 16) * T * pl.NT < h->sm_count) NB = 1;
+    if ((int64_t)N * ((Ho + 15) / 16) * ((Wo + 15) / 16) * To * pl.NT < h->sm_count) NB = 1;
     // Still fewer than half as many work items as SMs (the 44x80 layers): run half-width output-channel tiles.
     // Twice the items, each streaming half of the weights through its SM - the per-SM weight stream is what
     // bounds a 128-pixel tile - and nothing to reduce afterwards.
     int NT = pl.NT, NPAD = pl.NPAD, split_n = 0;
     if (NB == 1 && !per_tap && pl.NPAD % 32 == 0 &&
-        2 * (int64_t)N * ((Ho + 15) / 16) * ((Wo + 7) / 8) * T * pl.NT <= h->sm_count) {
+        2 * (int64_t)N * ((Ho + 15) / 16) * ((Wo + 7) / 8) * To * pl.NT <= h->sm_count) {
         split_n = 1; NT = 2 * pl.NT; NPAD = pl.NPAD / 2;
     }
     const int ACC = (2 * NB * NPAD <= 512) ? 2 : 1;
@@ -348,11 +350,11 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     }
     TcParams p;
     memset(&p, 0, sizeof(p));
-    p.N = N; p.T = T; p.H = Ho; p.W = Wo; p.Cout = d.cout; p.F = F;
+    p.N = N; p.T = To; p.H = Ho; p.W = Wo; p.Cout = d.cout; p.F = F;
     p.kt = d.kt; p.kh = d.kh; p.kw = d.kw;
     p.general = general ? 1 : 0;
     p.pad_h = d.pad_h; p.pad_w = d.pad_w; p.dil_h = d.dilation[1]; p.dil_w = d.dilation[2]; p.dil_t = d.dilation[0];
-    p.str_h = d.stride[1]; p.str_w = d.stride[2];
+    p.str_h = d.stride[1]; p.str_w = d.stride[2]; p.str_t = d.stride[0];
     p.CB = pl.CB; p.NT = NT; p.NPAD = NPAD;
     const int tiles_h = (Ho + 15) / 16;
     p.tiles_w = (Wo + TW - 1) / TW;
@@ -378,14 +380,14 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     // persistent convolution CTAs), which is why it is not the default.
     int nbands = 1;
     if ((d.flags & CCV3D_FLAG_OVERLAP) && h->side[0] && !general &&
-        (int64_t)N * tiles_h * p.tiles_w * T * NT >= 2LL * h->sm_count && tiles_h >= 4)
+        (int64_t)N * tiles_h * p.tiles_w * To * NT >= 2LL * h->sm_count && tiles_h >= 4)
         nbands = tiles_h / 2 < MAX_BANDS ? tiles_h / 2 : MAX_BANDS;
 
     // Cooperative staging (default when W % 8 == 0): the staging pass runs inside the convolution kernel, on four
     // extra warps per CTA, one band of 16 rows ahead of the tiles that read it.
     const bool coop = nbands == 1 && !per_tap && !general && !(d.flags & CCV3D_FLAG_TWO_KERNELS) && W % 8 == 0 &&
                       tiles_h <= MAX_COOP_BANDS && tiles_h >= 4 && pl.KB == 64 &&   // 32-channel blocks: the stagers cannot keep up
-                      (int64_t)N * tiles_h * p.tiles_w * T * NT >= 4LL * h->sm_count;   // small problems: two kernels
+                      (int64_t)N * tiles_h * p.tiles_w * To * NT >= 4LL * h->sm_count;   // small problems: two kernels
     size_t fixed = 1024 /*alignment slack*/ + align_up(sizeof(TcShared), 128) + 2 * (size_t)p.e_slot + (coop ? 9216 : 0);
     // leave room for staging blocks to be resident next to a convolution CTA when the two overlap
     const size_t limit = nbands > 1 ? SMEM_LIMIT - STAGE_COEXIST_BYTES : SMEM_LIMIT;
@@ -412,7 +414,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     p.out = out;
     p.status = h->status;
     if (p.epi_tma) {
-        s = encode_out_map(h, out, N, T, Ho, Wo, TW, p.ECH);
+        s = encode_out_map(h, out, N, To, Ho, Wo, TW, p.ECH);
         if (s != CCV3D_OK) return s;
     } else {
         h->tm_o = h->tm_a;  // never dereferenced on this path; any valid descriptor will do
@@ -431,7 +433,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
         p.nbands = tiles_h;
         p.ty_begin = 0;
         p.tiles_h = tiles_h;
-        const int64_t total = (int64_t)N * tiles_h * p.tiles_w * T * NT;
+        const int64_t total = (int64_t)N * tiles_h * p.tiles_w * To * NT;
         if (total > 0x7FFFFFFF) return CCV3D_ERR_UNSUPPORTED;
         p.total_tiles = (int)total;
         const int grid = p.total_tiles < h->sm_count ? p.total_tiles : h->sm_count;
@@ -1067,10 +1069,10 @@ ccv3d_status forward_simt(ccv3d_handle* h, const void* x, const void* cache, voi
     const int cf = (tc && cache) ? h->call_cf : 0;
     p.x = x; p.cache = cf ? cache : nullptr; p.cf = cf; p.w = h->w_copy; p.bias = h->bias32; p.out = out;
     p.N = N; p.Cin = d.cin; p.Cout = d.cout; p.T = T; p.H = H; p.W = W; p.kt = d.kt; p.kh = d.kh; p.kw = d.kw;
-    p.Ho = out_h(d, H); p.Wo = out_w(d, W);
+    p.To = out_t(d, T); p.Ho = out_h(d, H); p.Wo = out_w(d, W); p.st = d.stride[0];
     p.sh = d.stride[1]; p.sw = d.stride[2]; p.ph = d.pad_h; p.pw = d.pad_w; p.dh = d.dilation[1]; p.dw = d.dilation[2];
     p.dil_t = d.dilation[0];
-    const int64_t npix = (int64_t)N * T * p.Ho * p.Wo;
+    const int64_t npix = (int64_t)N * p.To * p.Ho * p.Wo;
     const int64_t gx = (npix + SIMT_THREADS - 1) / SIMT_THREADS;
     if (gx > 0x7FFFFFFF) return CCV3D_ERR_UNSUPPORTED;
     dim3 grid((unsigned)gx, (d.cout + SIMT_CO - 1) / SIMT_CO);
@@ -1126,7 +1128,7 @@ ccv3d_status check_forward_args(const ccv3d_handle* h, const void* x, const void
     if (Ho < 1 || Wo < 1) return CCV3D_ERR_INVALID_ARG;                          // the kernel does not fit the padded input
     const uint64_t xb = px * d.cin * T * esize(d.dtype), cb = px * d.cin * tc * esize(d.dtype);
     const uint64_t ccb = px * d.cin * (uint64_t)h->call_cf * esize(d.dtype);     // bytes of the cache actually passed
-    const uint64_t ob = (uint64_t)N * Ho * Wo * d.cout * T * esize(d.out_dtype);
+    const uint64_t ob = (uint64_t)N * Ho * Wo * d.cout * out_t(d, T) * esize(d.out_dtype);
     if (!tc) { cache = nullptr; new_cache = nullptr; }
     if (device_ptrs) {
         const uintptr_t m = (uintptr_t)x | (uintptr_t)cache | (uintptr_t)out | (uintptr_t)new_cache;
@@ -1271,9 +1273,10 @@ ccv3d_status ccv3d_workspace_bytes(const ccv3d_handle* h, int32_t N, int32_t T, 
     return CCV3D_OK;
 }
 
-ccv3d_status ccv3d_out_dims(const ccv3d_handle* h, int32_t H, int32_t W, int32_t* out_h_host, int32_t* out_w_host,
-                            int32_t* cache_frames_host) {
-    if (!h || H < 1 || W < 1) return CCV3D_ERR_INVALID_ARG;
+ccv3d_status ccv3d_out_dims(const ccv3d_handle* h, int32_t T, int32_t H, int32_t W, int32_t* out_t_host,
+                            int32_t* out_h_host, int32_t* out_w_host, int32_t* cache_frames_host) {
+    if (!h || T < 1 || H < 1 || W < 1) return CCV3D_ERR_INVALID_ARG;
+    if (out_t_host) *out_t_host = out_t(h->d, T);
     if (out_h_host) *out_h_host = out_h(h->d, H);
     if (out_w_host) *out_w_host = out_w(h->d, W);
     if (cache_frames_host) *cache_frames_host = hist_len(h->d);
@@ -1330,7 +1333,7 @@ ccv3d_status ccv3d_forward_host(ccv3d_handle* h, const void* x_host, const void*
     const int tc = hist_len(d);
     const uint64_t px = (uint64_t)N * H * W;
     const uint64_t xb = px * d.cin * T * esize(d.dtype), cb = px * d.cin * tc * esize(d.dtype);
-    const uint64_t ob = (uint64_t)N * out_h(d, H) * out_w(d, W) * d.cout * T * esize(d.out_dtype);
+    const uint64_t ob = (uint64_t)N * out_h(d, H) * out_w(d, W) * d.cout * out_t(d, T) * esize(d.out_dtype);
     cudaStream_t st = (cudaStream_t)stream;
     const bool has_c = tc && cache_host, has_n = tc && new_cache_host;
     if ((s = grow(&h->hx, &h->hx_b, xb)) != CCV3D_OK) return s;

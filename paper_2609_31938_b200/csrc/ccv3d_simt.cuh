@@ -27,8 +27,9 @@ struct SimtParams {
     const void* w;      // original [Cout,Cin,kt,kh,kw] order, storage dtype
     const float* bias;  // FP32, [Cout]
     void* out;
-    int N, Cin, Cout, T, H, W, kt, kh, kw;   // H, W: input extents
-    int Ho, Wo;                              // output extents
+    int N, Cin, Cout, T, H, W, kt, kh, kw;   // T, H, W: input extents
+    int To, Ho, Wo;                          // output extents
+    int st;                                  // temporal stride: output frame t reads Z frames t*st + dt*dil_t
     int sh, sw, ph, pw, dh, dw, dil_t;       // spatial stride, padding, dilation; temporal dilation (Eq. (1)-(2))
 };
 // With tc = d_t (kt-1): Z = [absent x (tc-cf) ; cache ; x]; frame tau < tc of Z is cache frame tau-(tc-cf) when that is >= 0.
@@ -36,17 +37,17 @@ struct SimtParams {
 constexpr int SIMT_CO = 8;       // output channels per thread
 constexpr int SIMT_THREADS = 128;
 
-// grid.x: ceil(N*T*Ho*Wo / SIMT_THREADS), grid.y: ceil(Cout / SIMT_CO)
+// grid.x: ceil(N*To*Ho*Wo / SIMT_THREADS), grid.y: ceil(Cout / SIMT_CO)
 template <typename TIn, typename TOut>
 __global__ void __launch_bounds__(SIMT_THREADS) conv3d_direct_kernel(const SimtParams p) {
     const int64_t HW = (int64_t)p.H * p.W, HWo = (int64_t)p.Ho * p.Wo;
-    const int64_t npix = (int64_t)p.N * p.T * HWo;
+    const int64_t npix = (int64_t)p.N * p.To * HWo;
     const int64_t pix = (int64_t)blockIdx.x * SIMT_THREADS + threadIdx.x;
     if (pix >= npix) return;
     const int w0 = (int)(pix % p.Wo);
     const int h0 = (int)((pix / p.Wo) % p.Ho);
-    const int t = (int)((pix / HWo) % p.T);
-    const int n = (int)(pix / (HWo * p.T));
+    const int t = (int)((pix / HWo) % p.To);
+    const int n = (int)(pix / (HWo * p.To));
     const int co0 = blockIdx.y * SIMT_CO;
     const int tc = p.dil_t * (p.kt - 1);
     const int taps = p.kt * p.kh * p.kw;
@@ -60,7 +61,7 @@ __global__ void __launch_bounds__(SIMT_THREADS) conv3d_direct_kernel(const SimtP
     const TIn* wt = (const TIn*)p.w;
     for (int ci = 0; ci < p.Cin; ++ci) {
         for (int dt = 0; dt < p.kt; ++dt) {
-            const int tau = t + dt * p.dil_t;  // frame of Z = [cache ; x], Eq. (1)
+            const int tau = t * p.st + dt * p.dil_t;  // frame of Z = [cache ; x], Eq. (1)
             const TIn* frame;
             if (tau < tc) {
                 const int cfr = tau - (tc - p.cf);
@@ -90,7 +91,7 @@ __global__ void __launch_bounds__(SIMT_THREADS) conv3d_direct_kernel(const SimtP
 #pragma unroll
     for (int j = 0; j < SIMT_CO; ++j)
         if (co0 + j < p.Cout)
-            st_from_float(out + (((int64_t)n * p.Cout + co0 + j) * p.T + t) * HWo + (int64_t)h0 * p.Wo + w0, acc[j]);
+            st_from_float(out + (((int64_t)n * p.Cout + co0 + j) * p.To + t) * HWo + (int64_t)h0 * p.Wo + w0, acc[j]);
 }
 
 // new_cache[n,ci,j,:,:] = Z[n,ci,T+j,:,:], Z = [cache ; x]; pure bit copy in units of `unit` bytes

@@ -491,7 +491,7 @@ struct TcParams {
     // general geometry (Eq. (2) with the layer's own padding and dilation, Eq. (1) with d_t); when `general` is 0
     // the kernel uses pad = (k-1)/2 and unit dilation.  H and W above are the OUTPUT extents; the input extents
     // only live in the tensor map.  Spatial stride > 1 is served by the per-tap mode with a strided tensor map.
-    int general, pad_h, pad_w, dil_h, dil_w, dil_t, str_h, str_w;
+    int general, pad_h, pad_w, dil_h, dil_w, dil_t, str_h, str_w, str_t;   // T above counts OUTPUT frames (T_o)
     int f0;                   // ring input: the slot of Z frame 0; Z frame f lives in slot (f0 + f) mod F (0 for a staged copy)
     const __nv_bfloat16* res; // optional residual ring [N][res_F][res_CB][H][W][res_KB] holding Cout channels, or null
     int res_F, res_f0, res_CB, res_KB;   // residual frame t is slot (res_f0 + t) mod res_F
@@ -631,6 +631,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     const int ph = p.general ? p.pad_h : (p.kh - 1) / 2, pw = p.general ? p.pad_w : (p.kw - 1) / 2;
     const int dlh = p.general ? p.dil_h : 1, dlw = p.general ? p.dil_w : 1, dlt = p.general ? p.dil_t : 1;
     const int sth = p.general ? p.str_h : 1, stw = p.general ? p.str_w : 1;      // > 1 only in the per-tap mode
+    const int stt = p.general ? p.str_t : 1;                // temporal stride: output frame t reads Z frames t*stt + dt*dlt
     const int BW = p.per_tap_a ? TW : TW + (p.kw - 1) * dlw;        // pixels per smem image row
     const int BH = p.per_tap_a ? 16 : 16 + (p.kh - 1) * dlh;
     const int spatial = p.kh * p.kw;
@@ -678,7 +679,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                 const int ty = p.ty_begin + r % p.tiles_h;
                 const int n = r / p.tiles_h;
                 const int h0 = ty * 16, w0 = tx * TW;
-                const int dt0 = (p.first_frame - t > 0) ? (p.first_frame - t + dlt - 1) / dlt : 0;   // first tap whose frame exists
+                const int dt0 = (p.first_frame - t * stt > 0) ? (p.first_frame - t * stt + dlt - 1) / dlt : 0;   // first tap whose frame exists
                 for (int dt = dt0; ok && dt < p.kt; ++dt)
                     for (int cb = 0; ok && cb < p.CB; ++cb) {
                         if (!(ok = mbar_wait(&sh->raw_empty[s], phase, sh, p, SITE_RAW_EMPTY))) break;
@@ -727,10 +728,10 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                         asm volatile("fence.proxy.async;" ::: "memory");   // other SMs' generic writes -> this SM's TMA reads
                     }
                 }
-                const int dt0 = (p.first_frame - t > 0) ? (p.first_frame - t + dlt - 1) / dlt : 0;   // first tap whose frame exists
+                const int dt0 = (p.first_frame - t * stt > 0) ? (p.first_frame - t * stt + dlt - 1) / dlt : 0;   // first tap whose frame exists
                 for (int dt = dt0; ok && dt < p.kt; ++dt)
                     for (int cb = 0; ok && cb < p.CB; ++cb) {
-                        int fr = p.f0 + t + dt * dlt;             // ring slot of Z frame t + dt d_t (f0 = 0: the frame itself)
+                        int fr = p.f0 + t * stt + dt * dlt;       // ring slot of Z frame t s_t + dt d_t (f0 = 0: the frame itself)
                         if (fr >= p.F) fr -= p.F;
                         const int fz = n * p.F + fr;
                         const int ntap = p.per_tap_a ? spatial : 1;
@@ -759,7 +760,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
             for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
                 const int nt = tile % p.NT;
                 const int t = (tile / p.NT) % p.T;
-                const int dt0 = (p.first_frame - t > 0) ? (p.first_frame - t + dlt - 1) / dlt : 0;   // first tap whose frame exists
+                const int dt0 = (p.first_frame - t * stt > 0) ? (p.first_frame - t * stt + dlt - 1) / dlt : 0;   // first tap whose frame exists
                 for (int dt = dt0; ok && dt < p.kt; ++dt)
                     for (int cb = 0; ok && cb < p.CB; ++cb) {
                         // split_n: this launch runs half-width output-channel tiles; the packed image of a full tile
@@ -807,7 +808,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
             const uint32_t a_ring0 = a_ring, b_ring0 = b_ring;
             for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
                 const int t = (tile / p.NT) % p.T;
-                const int dt0 = (p.first_frame - t > 0) ? (p.first_frame - t + dlt - 1) / dlt : 0;   // first tap whose frame exists
+                const int dt0 = (p.first_frame - t * stt > 0) ? (p.first_frame - t * stt + dlt - 1) / dlt : 0;   // first tap whose frame exists
                 if (!(ok = mbar_wait(&sh->acc_empty[acc], pacc, sh, p, SITE_ACC_EMPTY))) break;
                 tc_fence_after();
                 const uint32_t d0 = tmem_base + (uint32_t)(acc * NB + iss * NBW) * p.NPAD;
@@ -857,7 +858,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
         } else
         for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
             const int t = (tile / p.NT) % p.T;
-            const int dt0 = (p.first_frame - t > 0) ? (p.first_frame - t + dlt - 1) / dlt : 0;   // first tap whose frame exists
+            const int dt0 = (p.first_frame - t * stt > 0) ? (p.first_frame - t * stt + dlt - 1) / dlt : 0;   // first tap whose frame exists
             if (!(ok = mbar_wait(&sh->acc_empty[acc], pacc, sh, p, SITE_ACC_EMPTY))) break;
             tc_fence_after();
             const uint32_t d0 = tmem_base + (uint32_t)(acc * NB + iss * NBW) * p.NPAD;
@@ -1119,7 +1120,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
         bool ok = true;
         for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
             const int t = (tile / p.NT) % p.T;
-            const int dt0 = (p.first_frame - t > 0) ? (p.first_frame - t + dlt - 1) / dlt : 0;   // first tap whose frame exists
+            const int dt0 = (p.first_frame - t * stt > 0) ? (p.first_frame - t * stt + dlt - 1) / dlt : 0;   // first tap whose frame exists
             for (int kb = (p.kt - dt0) * p.CB; ok && kb > 0; --kb) {
                 ok = mbar_wait(&sh->raw_full[rs], pr, sh, p, SITE_RAW_FULL) && mbar_wait(&sh->empty_a[sa], pea, sh, p, SITE_A_EMPTY);
                 ok = __all_sync(0xffffffffu, ok);

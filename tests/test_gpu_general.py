@@ -44,16 +44,17 @@ def _case(N, Cin, Cout, T, H, W, k, dtype, cf, seed):
     return c
 
 
-def run_general(ccv, c, stride, pad, dil, dil_t, flags=0, kind=None):
+def run_general(ccv, c, stride, pad, dil, dil_t, flags=0, kind=None, stride_t=1):
     kt, kh, kw = c["k"]
-    ref, ref_nc = oracle.forward_general(c["x"], c["cache"], c["w"], c["b"], stride=stride, pad=pad, dil=dil, dil_t=dil_t)
+    ref, ref_nc = oracle.forward_general(c["x"], c["cache"], c["w"], c["b"], stride=stride, pad=pad, dil=dil, dil_t=dil_t,
+                                         stride_t=stride_t)
     tc = dil_t * (kt - 1)
-    layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), flags=flags, stride=(1, *stride), dilation=(dil_t, *dil),
-                             pad=(tc // 2, *pad))
+    layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), flags=flags, stride=(stride_t, *stride),
+                             dilation=(dil_t, *dil), pad=(tc // 2, *pad))
     x, cache = to_dev(c["x"]), to_dev(c["cache"])
     N, Cin, T, H, W = c["x"].shape
-    s, Ho, Wo, frames = ccv.ccv3d_out_dims(layer.h, H, W)
-    assert s == ccv.OK and (Ho, Wo) == ref.shape[3:] and frames == tc
+    s, To, Ho, Wo, frames = ccv.ccv3d_out_dims(layer.h, T, H, W)
+    assert s == ccv.OK and (To, Ho, Wo) == ref.shape[2:] and frames == tc
     odt = torch.float32 if c["dtype"] == si.F32 else torch.bfloat16
     obuf, out = _guarded(ref.shape, odt)
     nbuf, nc = (_guarded((N, Cin, tc, H, W), x.dtype) if tc else (None, None))
@@ -110,6 +111,40 @@ def test_bf16_fma_route_general_geometry(ccv, k, stride, pad, dil, dil_t):
     c = _case(1, 24, 20, 2, 11, 14, k, si.BF16, dil_t * (k[0] - 1), seed=33)
     m, ctr = run_general(ccv, c, stride, pad, dil, dil_t, flags=ccv.FLAG_FORCE_SIMT)
     assert ctr["simt"] == 1
+
+
+@pytest.mark.parametrize("k,stride,pad,dil,dil_t", [GEOMS[2], GEOMS[3], GEOMS[4], GEOMS[7], ((3, 3, 3), (1, 1), (1, 1), (1, 1), 1)])
+@pytest.mark.parametrize("stride_t,T", [(2, 4), (2, 5), (3, 4)])
+@pytest.mark.parametrize("route", ["f32", "bf16_tc", "bf16_fma"])
+def test_temporal_stride(ccv, k, stride, pad, dil, dil_t, stride_t, T, route):
+    """Temporal stride (the encoder's temporal downsampling layers; outside the paper's method, which hands them
+    back to the framework): output frame o reads Z frames o s_t + k d_t, T_o = floor((T-1)/s_t) + 1."""
+    tc = dil_t * (k[0] - 1)
+    if route == "f32":
+        c = _case(1, 5, 6, T, 9, 12, k, si.F32, tc, seed=37)
+    else:
+        c = _case(1, 64, 48, T, 20, 24, k, si.BF16, tc // 2 if T == 5 else tc, seed=38)
+    m, ctr = run_general(ccv, c, stride, pad, dil, dil_t, flags=ccv.FLAG_FORCE_SIMT if route == "bf16_fma" else 0,
+                         stride_t=stride_t)
+    assert ctr["tcgen05_bf16" if route == "bf16_tc" else "simt"] == 1
+
+
+def test_streaming_with_temporal_stride_on_gpu(ccv):
+    c = _case(1, 64, 32, 8, 20, 24, (3, 3, 3), si.BF16, 0, seed=39)
+    layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), stride=(2, 1, 1))
+    x = to_dev(c["x"])
+    whole, whole_nc = layer(x, None)
+    assert whole.shape[2] == 4
+    cache, outs = None, []
+    for pos, n in ((0, 2), (2, 4), (6, 2)):
+        o, cache = layer(x[:, :, pos:pos + n].contiguous(), cache)
+        outs.append(o)
+    torch.cuda.synchronize()
+    assert torch.equal(torch.cat(outs, dim=2), whole) and torch.equal(cache, whole_nc)
+    ref, ref_nc = oracle.forward_general(c["x"], None, c["w"], c["b"], stride_t=2)
+    check(as_f64(whole), ref, "bf16")
+    assert np.array_equal(bits(cache), ref_nc)
+    layer.close()
 
 
 def test_tensor_core_equals_fma_route_closely_on_a_strided_dilated_layer(ccv):
