@@ -386,7 +386,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     // Cooperative staging (default when W % 8 == 0): the staging pass runs inside the convolution kernel, on four
     // extra warps per CTA, one band of 16 rows ahead of the tiles that read it.
     const bool coop = nbands == 1 && !per_tap && !general && !(d.flags & CCV3D_FLAG_TWO_KERNELS) && W % 8 == 0 &&
-                      tiles_h <= MAX_COOP_BANDS && tiles_h >= 4 && pl.KB == 64 &&   // 32-channel blocks: the stagers cannot keep up
+                      tiles_h <= MAX_COOP_BANDS && tiles_h >= 4 &&
                       (int64_t)N * tiles_h * p.tiles_w * To * NT >= 4LL * h->sm_count;   // small problems: two kernels
     size_t fixed = 1024 /*alignment slack*/ + align_up(sizeof(TcShared), 128) + 2 * (size_t)p.e_slot + (coop ? 9216 : 0);
     // leave room for staging blocks to be resident next to a convolution CTA when the two overlap

@@ -278,15 +278,29 @@ __device__ __forceinline__ StageTask make_stage_task(const StageParams& p, int K
 // convolution kernel (cooperative staging): [KB channels][64 pixels] of an image row -> [64 pixels][KB channels],
 // plus the cache update when the frame belongs to the new cache.  Split in two so that the loads of several
 // tasks can be in flight before the first is written: stage_task_load fills val[], stage_task_store moves it
-// through `tile` (KB*33 words of shared memory; phases separated by the stagers' named barrier, id 2).
+// through `tile` (StagerGeom<KB>::TILE_WORDS words of shared memory; phases separated by the stagers' named
+// barrier, id 2).
 __device__ __forceinline__ void stager_bar() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
 
+// PX: pixels of an image row per task.  64 for 64-channel blocks; 128 for 32-channel blocks, so that a task moves
+// the same 8 KB either way (the per-task barriers and address arithmetic are what limits a stager team).
 template <int KB>
-__device__ __forceinline__ void stage_task_load(const StageParams& p, const StageTask& t, int tid, uint4 (&val)[KB * 8 / 128]) {
+struct StagerGeom {
+    static constexpr int PX = (KB == 64) ? 64 : 128;
+    static constexpr int VPR = PX / 8;                    // 16-byte vectors per channel row
+    static constexpr int NLD = KB * VPR / 128;            // vectors per thread
+    static constexpr int PITCH = PX / 2 + 1;              // 32-bit words per channel row in the tile (+1: bank spread)
+    static constexpr int TILE_WORDS = KB * PITCH;
+};
+
+template <int KB>
+__device__ __forceinline__ void stage_task_load(const StageParams& p, const StageTask& t, int tid,
+                                                uint4 (&val)[StagerGeom<KB>::NLD]) {
+    using G = StagerGeom<KB>;
 #pragma unroll
-    for (int k = 0; k < KB * 8 / 128; ++k) {
+    for (int k = 0; k < G::NLD; ++k) {
         const int i = tid + 128 * k;
-        const int c = i >> 3, v = i & 7;
+        const int c = i / G::VPR, v = i % G::VPR;
         const int ci = t.cb * KB + c;
         const int w = t.w0 + v * 8;
         val[k] = make_uint4(0u, 0u, 0u, 0u);
@@ -296,30 +310,30 @@ __device__ __forceinline__ void stage_task_load(const StageParams& p, const Stag
 
 template <int KB>
 __device__ __forceinline__ void stage_task_store(const StageParams& p, const StageTask& t, int tid,
-                                                 const uint4 (&val)[KB * 8 / 128], uint32_t* tile) {
-    constexpr int PITCH = STG_PX / 2 + 1;
+                                                 const uint4 (&val)[StagerGeom<KB>::NLD], uint32_t* tile) {
+    using G = StagerGeom<KB>;
     constexpr int OCT = KB / 8;
     const int64_t ncstride = (int64_t)p.tc * p.H * p.W;
 #pragma unroll
-    for (int k = 0; k < KB * 8 / 128; ++k) {
+    for (int k = 0; k < G::NLD; ++k) {
         const int i = tid + 128 * k;
-        const int c = i >> 3, v = i & 7;
+        const int c = i / G::VPR, v = i % G::VPR;
         const int ci = t.cb * KB + c;
         const int w = t.w0 + v * 8;
         if (t.ncdst && w < p.W && ci < p.Cin) *reinterpret_cast<uint4*>(t.ncdst + ci * ncstride + w) = val[k];
-        uint32_t* row = tile + c * PITCH + v * 4;
+        uint32_t* row = tile + c * G::PITCH + v * 4;
         row[0] = val[k].x; row[1] = val[k].y; row[2] = val[k].z; row[3] = val[k].w;
     }
     stager_bar();
 #pragma unroll
-    for (int k = 0; k < (32 * OCT) / 128; ++k) {
+    for (int k = 0; k < (G::PX / 2 * OCT) / 128; ++k) {
         const int vt = tid + 128 * k;
         const int oct = vt % OCT, pp = vt / OCT;
         uint32_t lo[4], hi[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-            const uint32_t a = tile[(oct * 8 + 2 * q) * PITCH + pp];
-            const uint32_t b = tile[(oct * 8 + 2 * q + 1) * PITCH + pp];
+            const uint32_t a = tile[(oct * 8 + 2 * q) * G::PITCH + pp];
+            const uint32_t b = tile[(oct * 8 + 2 * q + 1) * G::PITCH + pp];
             lo[q] = __byte_perm(a, b, 0x5410);
             hi[q] = __byte_perm(a, b, 0x7632);
         }
@@ -623,7 +637,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     uint8_t* epi_buf = ring_b + (size_t)p.SB * p.b_slot;
     uint8_t* ring_raw = epi_buf + (p.epi_tma ? 2 * (size_t)p.e_slot : 0);
     uint8_t* dummy = ring_raw + (FUSED ? 2 * (size_t)p.raw_slot : 0);   // 2 KB sink for the unused rows of edge blocks
-    uint32_t* coop_tile = reinterpret_cast<uint32_t*>(ring_raw);          // COOP: KB*33 words for the stagers
+    uint32_t* coop_tile = reinterpret_cast<uint32_t*>(ring_raw);          // COOP: the stagers' transposition tile (<= 9216 bytes)
     TcShared* sh = reinterpret_cast<TcShared*>(dummy + (FUSED ? 2048 : 0) + (COOP ? 9216 : 0));
 
     const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);  // provably warp-uniform
@@ -1069,7 +1083,8 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     // ---------------------------------------------------------------- stagers (cooperative staging, warps 8..11)
     if (COOP && warp >= 8) {
         const int tid = threadIdx.x - 256;
-        const int nchunks = (sp.W + STG_PX - 1) / STG_PX;
+        constexpr int SPX = StagerGeom<KB>::PX;
+        const int nchunks = (sp.W + SPX - 1) / SPX;
         const int nf = sp.tc + sp.T - sp.f_begin;
         // Stagers wait on nothing but their own named barrier, so they always run to completion (also when a
         // consumer role of some CTA has given up on a wait): every thread of the four warps takes every branch.
@@ -1077,10 +1092,10 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
             const int h_lo = 16 * b;
             const int rows = (sp.H - h_lo < 16) ? sp.H - h_lo : 16;
             const int ntask = sp.N * nf * sp.CB * rows * nchunks;
-            constexpr int G = (KB == 64) ? 2 : 4;            // tasks whose loads are in flight together (16 KB per CTA)
+            constexpr int G = 2;                             // tasks whose loads are in flight together (16 KB per CTA)
             for (int task0 = blockIdx.x; task0 < ntask; task0 += G * gridDim.x) {
                 StageTask tk[G];
-                uint4 val[G][KB * 8 / 128];
+                uint4 val[G][StagerGeom<KB>::NLD];
 #pragma unroll
                 for (int g = 0; g < G; ++g) {
                     const int task = task0 + g * gridDim.x;
@@ -1091,7 +1106,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                         const int cb = r % sp.CB; r /= sp.CB;
                         const int f = sp.f_begin + r % nf;
                         const int n = r / nf;
-                        tk[g] = make_stage_task(sp, KB, n, f, cb, h, wc * STG_PX);
+                        tk[g] = make_stage_task(sp, KB, n, f, cb, h, wc * SPX);
                         stage_task_load<KB>(sp, tk[g], tid, val[g]);
                     }
                 }
