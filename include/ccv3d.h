@@ -57,6 +57,8 @@ typedef enum {
 #define CCV3D_FLAG_FUSED 0x8u            /* tensor-core route without scratch memory: no channels-last staging copy; the kernel reads x and the cache
                                             by TMA and transposes in shared memory (needs W % 8 == 0, else the staged route is taken). About as fast as
                                             the default route in short bursts, ~3 % slower sustained; for callers that cannot afford the workspace. */
+#define CCV3D_FLAG_F32_TENSOR 0x20u       /* FP32 layers: always use the tensor cores (3xTF32: each FP32 product as hi*hi + hi*lo + lo*hi of TF32
+                                            operands, FP32 accumulate); the default sends calls under ~1 GFLOP to the FP32-FMA kernel */
 #define CCV3D_FLAG_TC_PER_TAP_A 0x2u    /* tensor-core kernel: fetch the activation tile once per tap (no halo reuse in shared memory) */
 
 /* Layer description, fixed at create time (Algorithm 1's Require line: W, b, p, s, d, g).

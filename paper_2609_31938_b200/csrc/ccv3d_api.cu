@@ -50,7 +50,8 @@ struct ccv3d_handle {
     ccv3d_desc d;
     int device;
     int sm_count;
-    bool use_tc;
+    bool use_tc;         // BF16 layer on the tensor-core route
+    bool use_tc32;       // FP32 layer that may take the tensor-core route (3xTF32) when the call is large enough
     TcPlan plan;
     void* w_copy;        // SIMT route: weights in their original order (device)
     void* wp;            // TC route: packed weights (device)
@@ -154,6 +155,21 @@ void make_plan(const ccv3d_desc& d, TcPlan* pl) {
     pl->ACC = (2 * pl->NB * pl->NPAD <= 512) ? 2 : 1;
 }
 
+// FP32 layers on the tensor cores: rows of 32 FP32 channels = 128 bytes, i.e. the geometry of 64-channel BF16
+// blocks; the K loop runs three passes (hi*lo, lo*hi, hi*hi) over the 32-channel blocks.
+void make_plan_f32(const ccv3d_desc& d, TcPlan* pl) {
+    pl->fused = false;
+    pl->KB = 64;
+    pl->CB = (d.cin + 31) / 32;
+    pl->cin_pad = pl->CB * 32;
+    pl->NT = (d.cout + 255) / 256;
+    const int per = (d.cout + pl->NT - 1) / pl->NT;
+    pl->NPAD = (per + 15) / 16 * 16;
+    pl->cout_pad = pl->NT * pl->NPAD;
+    pl->NB = (4 * pl->NPAD <= 512) ? 2 : 1;
+    pl->ACC = (2 * pl->NB * pl->NPAD <= 512) ? 2 : 1;
+}
+
 uint32_t pow2_cols(uint32_t c) {
     uint32_t v = 32;
     while (v < c) v <<= 1;
@@ -199,13 +215,15 @@ ccv3d_status grow(void** buf, uint64_t* have, uint64_t need) {
 ccv3d_status encode_act_map(ccv3d_handle* h, int N, int T, int H, int W, int BW, int BH, int es_w = 1, int es_h = 1) {
     const TcPlan& pl = h->plan;
     const int F = hist_len(h->d) + T;
+    const bool f32 = h->d.dtype == CCV3D_F32;             // rows of 32 FP32 channels; two blocks (value, remainder) per real block
     const uint64_t rowb = (uint64_t)pl.KB * 2;
-    cuuint64_t dims[5] = {(cuuint64_t)pl.KB, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)pl.CB, (cuuint64_t)N * F};
-    cuuint64_t strides[4] = {rowb, rowb * W, rowb * W * H, rowb * W * H * pl.CB};
-    cuuint32_t box[5] = {(cuuint32_t)pl.KB, (cuuint32_t)(BW * es_w), (cuuint32_t)(BH * es_h), 1, 1};
+    const int inner = f32 ? 32 : pl.KB, blocks = f32 ? 2 * pl.CB : pl.CB;
+    cuuint64_t dims[5] = {(cuuint64_t)inner, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)blocks, (cuuint64_t)N * F};
+    cuuint64_t strides[4] = {rowb, rowb * W, rowb * W * H, rowb * W * H * blocks};
+    cuuint32_t box[5] = {(cuuint32_t)inner, (cuuint32_t)(BW * es_w), (cuuint32_t)(BH * es_h), 1, 1};
     cuuint32_t es[5] = {1, (cuuint32_t)es_w, (cuuint32_t)es_h, 1, 1};
     if (box[1] > 256 || box[2] > 256) return CCV3D_ERR_UNSUPPORTED;
-    CUresult r = h->encode(&h->tm_a, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, h->workspace, dims, strides, box, es,
+    CUresult r = h->encode(&h->tm_a, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, h->workspace, dims, strides, box, es,
                            CU_TENSOR_MAP_INTERLEAVE_NONE,
                            pl.KB == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -226,6 +244,7 @@ ccv3d_status encode_out_map(ccv3d_handle* h, void* out, int N, int T, int H, int
 
 uint64_t tc_workspace_bytes(const ccv3d_handle* h, int N, int T, int H, int W) {
     const int F = hist_len(h->d) + T;
+    if (h->d.dtype == CCV3D_F32) return (uint64_t)N * F * h->plan.cin_pad * H * W * 8;   // values and remainders, FP32
     return (uint64_t)N * F * h->plan.cin_pad * H * W * 2;
 }
 
@@ -241,9 +260,9 @@ ccv3d_status launch_tc_coop(ccv3d_handle* h, const TcParams& p, const StageParam
     return CCV3D_OK;
 }
 
-template <int KB, int NB, int KS, int TPBC>
+template <int KB, int NB, int KS, int TPBC, bool TF32 = false>
 ccv3d_status launch_tc(ccv3d_handle* h, const TcParams& p, size_t smem, int grid, cudaStream_t st) {
-    auto kern = conv3d_tcgen05_kernel<KB, NB, KS, TPBC, false, false>;
+    auto kern = conv3d_tcgen05_kernel<KB, NB, KS, TPBC, false, false, TF32>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return cuda_fail();
     StageParams nosp;
@@ -290,10 +309,21 @@ ccv3d_status launch_conv(ccv3d_handle* h, TcParams p, int nb, int ty0, int ty1, 
         else if (ks == 1) s = launch_tc<KBv, NBv, 1, 1>(h, p, smem, grid, st);                   \
         else s = launch_tc<KBv, NBv, 0, 0>(h, p, smem, grid, st);                                \
     } while (0)
-    if (pl.KB == 64 && nb == 2) CCV3D_LAUNCH(64, 2);
+#define CCV3D_LAUNCH_F32(NBv)                                                                      \
+    do {                                                                                          \
+        if (ks == 3 && p.TPB == 3) s = launch_tc<64, NBv, 3, 3, true>(h, p, smem, grid, st);      \
+        else if (ks == 3 && p.TPB == 1) s = launch_tc<64, NBv, 3, 1, true>(h, p, smem, grid, st); \
+        else if (ks == 1) s = launch_tc<64, NBv, 1, 1, true>(h, p, smem, grid, st);               \
+        else s = launch_tc<64, NBv, 0, 0, true>(h, p, smem, grid, st);                            \
+    } while (0)
+    if (h->d.dtype == CCV3D_F32) {
+        if (nb == 2) CCV3D_LAUNCH_F32(2);
+        else CCV3D_LAUNCH_F32(1);
+    } else if (pl.KB == 64 && nb == 2) CCV3D_LAUNCH(64, 2);
     else if (pl.KB == 64) CCV3D_LAUNCH(64, 1);
     else if (nb == 2) CCV3D_LAUNCH(32, 2);
     else CCV3D_LAUNCH(32, 1);
+#undef CCV3D_LAUNCH_F32
 #undef CCV3D_LAUNCH
     return s;
 }
@@ -307,6 +337,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     const bool general = !standard_geom(d);
     const int Ho = out_h(d, H), Wo = out_w(d, W), To = out_t(d, T);   // output extents; T, H, W are the input's
     const bool strided = d.stride[1] > 1 || d.stride[2] > 1;
+    const bool f32 = d.dtype == CCV3D_F32;                 // 3xTF32: FP32 staging with the hi/lo split, TF32 MMAs
 
     ccv3d_status s = grow(&h->workspace, &h->workspace_bytes, tc_workspace_bytes(h, N, T, H, W));
     if (s != CCV3D_OK) return s;
@@ -379,13 +410,13 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     // effect on B200: 0 to -6 % time (the co-resident staging blocks make little headway next to the
     // persistent convolution CTAs), which is why it is not the default.
     int nbands = 1;
-    if ((d.flags & CCV3D_FLAG_OVERLAP) && h->side[0] && !general &&
+    if ((d.flags & CCV3D_FLAG_OVERLAP) && h->side[0] && !general && !f32 &&
         (int64_t)N * tiles_h * p.tiles_w * To * NT >= 2LL * h->sm_count && tiles_h >= 4)
         nbands = tiles_h / 2 < MAX_BANDS ? tiles_h / 2 : MAX_BANDS;
 
     // Cooperative staging (default when W % 8 == 0): the staging pass runs inside the convolution kernel, on four
     // extra warps per CTA, one band of 16 rows ahead of the tiles that read it.
-    const bool coop = nbands == 1 && !per_tap && !general && !(d.flags & CCV3D_FLAG_TWO_KERNELS) && W % 8 == 0 &&
+    const bool coop = nbands == 1 && !per_tap && !general && !f32 && !(d.flags & CCV3D_FLAG_TWO_KERNELS) && W % 8 == 0 &&
                       tiles_h <= MAX_COOP_BANDS && tiles_h >= 4 &&
                       (int64_t)N * tiles_h * p.tiles_w * To * NT >= 4LL * h->sm_count;   // small problems: two kernels
     size_t fixed = 1024 /*alignment slack*/ + align_up(sizeof(TcShared), 128) + 2 * (size_t)p.e_slot + (coop ? 9216 : 0);
@@ -452,7 +483,20 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
         if (s != CCV3D_OK) return s;
     } else if (nbands == 1) {
         if (pev) cudaEventRecord(pev[0], st);
-        s = launch_stage(h, sp, 0, H, nframes, st);
+        if (f32) {
+            StageF32Params sf;
+            sf.x = (const float*)x; sf.cache = cf ? (const float*)cache : nullptr; sf.cf = cf;
+            sf.zs = (float*)h->workspace; sf.new_cache = tc ? (float*)new_cache : nullptr;
+            sf.N = N; sf.Cin = d.cin; sf.T = T; sf.H = H; sf.W = W; sf.tc = tc; sf.CBr = pl.CB; sf.f_begin = sp.f_begin;
+            dim3 sgrid((W + 31) / 32, H, (unsigned)((int64_t)N * nframes * sf.CBr));
+            if (H > 65535 || (int64_t)N * nframes * sf.CBr > 65535) return CCV3D_ERR_UNSUPPORTED;
+            stage_frames_f32_kernel<<<sgrid, 256, 0, st>>>(sf);
+            if (cudaGetLastError() != cudaSuccess) return cuda_fail();
+            h->ctr.kernel_launches++;
+            s = CCV3D_OK;
+        } else {
+            s = launch_stage(h, sp, 0, H, nframes, st);
+        }
         if (s != CCV3D_OK) return s;
         if (pev) cudaEventRecord(pev[1], st);
         s = launch_conv(h, p, NB, 0, tiles_h, smem, ks, st);
@@ -1115,6 +1159,18 @@ ccv3d_status forward_simt(ccv3d_handle* h, const void* x, const void* cache, voi
     return CCV3D_OK;
 }
 
+// FP32 layers: the FP32-FMA kernel is exact FP32 and fine for small calls; from about a GFLOP on (or when the layer
+// asks for it) the call goes to the tensor cores as 3xTF32.  The tensor core's accumulation truncates: measured
+// against the FP64 definition the worst element is off by about 8.8e-9 x K x RMS(out) (K = cin*kt*kh*kw; 4.6e-5 at
+// K = 5184, 9.1e-5 at K = 10368), so layers with K > 8192 stay on the FP32-FMA kernel unless the flag insists.
+bool f32_takes_tensor_cores(const ccv3d_handle* h, int N, int T, int H, int W) {
+    const ccv3d_desc& d = h->d;
+    if (d.flags & CCV3D_FLAG_F32_TENSOR) return true;
+    if ((int64_t)d.cin * d.kt * d.kh * d.kw > 8192) return false;
+    const double flops = 2.0 * N * out_t(d, T) * out_h(d, H) * out_w(d, W) * d.cout * d.cin * d.kt * d.kh * d.kw;
+    return flops >= 1.0e9;
+}
+
 ccv3d_status check_forward_args(const ccv3d_handle* h, const void* x, const void* cache, void* out, void* new_cache,
                                 int N, int T, int H, int W, bool device_ptrs) {
     if (!h || !x || !out) return CCV3D_ERR_INVALID_ARG;
@@ -1181,6 +1237,7 @@ ccv3d_status ccv3d_create(ccv3d_handle** out_h, const ccv3d_desc* d, const void*
     h->device = dev;
     h->sm_count = prop.multiProcessorCount;
     h->use_tc = (d->dtype == CCV3D_BF16) && !(d->flags & CCV3D_FLAG_FORCE_SIMT);
+    h->use_tc32 = (d->dtype == CCV3D_F32) && !(d->flags & CCV3D_FLAG_FORCE_SIMT);
     // bound of every in-kernel wait: about one second of SM clocks (clock rate is reported in kHz)
     h->wait_limit_clk = (long long)prop.clockRate * 1000ll;
     if (const char* e = getenv("CCV3D_WAIT_LIMIT_MS")) {
@@ -1231,6 +1288,24 @@ ccv3d_status ccv3d_create(ccv3d_handle** out_h, const ccv3d_desc* d, const void*
         if (cudaMalloc(&h->w_copy, wb) != cudaSuccess) return fail(CCV3D_ERR_NOMEM);
         if (cudaMemcpyAsync(h->w_copy, w_dev, wb, cudaMemcpyDeviceToDevice, st) != cudaSuccess) return fail(cuda_fail());
     }
+    if (h->use_tc32) {
+        // FP32 layer: besides the plain copy for the FP32-FMA kernel, the 3xTF32 operand images (lo(w), w, w: one per
+        // pass of the K loop; rows of 128 bytes, which the kernel treats like 64-channel BF16 rows)
+        make_plan_f32(*d, &h->plan);
+        bias_n = h->plan.cout_pad;
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+            qres != cudaDriverEntryPointSuccess)
+            return fail(cuda_fail());
+        h->encode = (EncodeTiledFn)fn;
+        const uint64_t wpb = (uint64_t)3 * taps * h->plan.cout_pad * h->plan.cin_pad * 4;
+        if (cudaMalloc(&h->wp, wpb) != cudaSuccess) return fail(CCV3D_ERR_NOMEM);
+        pack_weights_f32_kernel<<<1024, 256, 0, st>>>((const float*)w_dev, (float*)h->wp, d->cout, d->cin, d->kt,
+                                                      d->kh * d->kw, h->plan.CB, h->plan.NT, h->plan.NPAD);
+        if (cudaGetLastError() != cudaSuccess) return fail(cuda_fail());
+        h->ctr.kernel_launches++;
+    }
     if (cudaMalloc((void**)&h->bias32, (size_t)bias_n * sizeof(float)) != cudaSuccess) return fail(CCV3D_ERR_NOMEM);
     if (d->dtype == CCV3D_BF16)
         bias_to_f32_kernel<__nv_bfloat16><<<(bias_n + 255) / 256, 256, 0, st>>>((const __nv_bfloat16*)b_dev, h->bias32,
@@ -1268,7 +1343,8 @@ ccv3d_status ccv3d_destroy(ccv3d_handle* h) {
 ccv3d_status ccv3d_workspace_bytes(const ccv3d_handle* h, int32_t N, int32_t T, int32_t H, int32_t W,
                                    uint64_t* bytes_host) {
     if (!h || !bytes_host || N < 1 || T < 1 || H < 1 || W < 1) return CCV3D_ERR_INVALID_ARG;
-    const bool scratch_free = !h->use_tc || pointwise_eligible(h, T, H, W) || fused_eligible(h, W);
+    const bool scratch_free = (h->use_tc32 ? !f32_takes_tensor_cores(h, N, T, H, W) : !h->use_tc) ||
+                              (h->use_tc && (pointwise_eligible(h, T, H, W) || fused_eligible(h, W)));
     *bytes_host = scratch_free ? 0 : tc_workspace_bytes(h, N, T, H, W);
     return CCV3D_OK;
 }
@@ -1298,6 +1374,7 @@ ccv3d_status ccv3d_forward_ex(ccv3d_handle* h, const void* x, const void* cache,
     if (h->use_tc && pointwise_eligible(h, T, H, W)) s = forward_pointwise(h, x, out, N, T, H, W, st);
     else if (h->use_tc && fused_eligible(h, W)) s = forward_fused(h, x, cache, out, new_cache, N, T, H, W, st);
     else if (h->use_tc) s = forward_tc(h, x, cache, out, new_cache, N, T, H, W, st);
+    else if (h->use_tc32 && f32_takes_tensor_cores(h, N, T, H, W)) s = forward_tc(h, x, cache, out, new_cache, N, T, H, W, st);
     else s = forward_simt(h, x, cache, out, new_cache, N, T, H, W, st);
     return count(h, s);
 }

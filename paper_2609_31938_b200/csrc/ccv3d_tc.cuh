@@ -171,6 +171,104 @@ __global__ void __launch_bounds__(32 * (KB / 8)) stage_frames_kernel(const Stage
 }
 
 // ------------------------------------------------------------------------------------------------
+// FP32 layers on the tensor cores ("3xTF32"): packing and staging with the hi/lo split
+// ------------------------------------------------------------------------------------------------
+// The tensor core reads an FP32 operand as TF32 by ignoring its low 13 mantissa bits; what it ignores is kept
+// as a second operand, lo(v) = v - hi(v) (exact in FP32; itself truncated to TF32 when used, which leaves a
+// relative error of about 2^-21 per product).
+__device__ __forceinline__ float tf32_lo(float v) { return v - __uint_as_float(__float_as_uint(v) & 0xFFFFE000u); }
+
+// Wq[pass][dt][cb][nt][sp][r][e], e < 32 FP32 input channels of block cb: pass 0 holds lo(w) (multiplied with the
+// activations' values), passes 1 and 2 hold w (multiplied with the activations' remainders, then with their
+// values); rows of 128 bytes stored as the 128-byte-swizzled shared-memory image (16-byte chunk c of row r at
+// chunk position c ^ (r & 7)).  Zero outside the real channel extents.
+__global__ void pack_weights_f32_kernel(const float* __restrict__ w, float* __restrict__ wq, int Cout, int Cin, int kt,
+                                        int spatial, int CB, int NT, int NPAD) {
+    const int64_t total = (int64_t)3 * kt * CB * NT * spatial * NPAD * 32;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        int64_t q = i;
+        const int e = (int)(q % 32); q /= 32;
+        const int r = (int)(q % NPAD); q /= NPAD;
+        const int sp = (int)(q % spatial); q /= spatial;
+        const int nt = (int)(q % NT); q /= NT;
+        const int cb = (int)(q % CB); q /= CB;
+        const int dt = (int)(q % kt);
+        const int pass = (int)(q / kt);
+        const int chunk = (e >> 2) ^ (r & 7);
+        const int ci = cb * 32 + chunk * 4 + (e & 3);
+        const int co = nt * NPAD + r;
+        float val = 0.f;
+        if (ci < Cin && co < Cout) {
+            val = w[(((int64_t)co * Cin + ci) * kt + dt) * spatial + sp];
+            if (pass == 0) val = tf32_lo(val);
+        }
+        wq[i] = val;
+    }
+}
+
+struct StageF32Params {
+    const float* x;          // [N,Cin,T,H,W]
+    const float* cache;      // [N,Cin,cf,H,W] or null
+    int cf;
+    float* zs;               // [N][F][2*CBr][H][W][32]: block 2*cb = the values, block 2*cb+1 = their TF32 remainders
+    float* new_cache;        // [N,Cin,tc,H,W] or null
+    int N, Cin, T, H, W, tc, CBr;
+    int f_begin;
+};
+
+// grid: (ceil(W/32), H, N*(F - f_begin)*CBr); block 256.  [32 channels][32 pixels] of an image row -> 32 pixels x
+// (32 values, 32 remainders), plus the bit-exact cache update from the same registers.
+__global__ void __launch_bounds__(256) stage_frames_f32_kernel(const StageF32Params p) {
+    __shared__ float tile[32 * 33];
+    const int F = p.tc + p.T;
+    const int nf = F - p.f_begin;
+    int z = blockIdx.z;
+    const int cb = z % p.CBr; z /= p.CBr;
+    const int f = p.f_begin + z % nf;
+    const int n = z / nf;
+    const int h = blockIdx.y;
+    const int w0 = blockIdx.x * 32;
+    const int64_t HW = (int64_t)p.H * p.W;
+    const float* src = nullptr;
+    int64_t cstride = 0;
+    if (f < p.tc) {
+        const int cfr = f - (p.tc - p.cf);
+        if (p.cache && cfr >= 0) {
+            src = p.cache + ((int64_t)n * p.Cin * p.cf + cfr) * HW;
+            cstride = (int64_t)p.cf * HW;
+        }
+    } else {
+        src = p.x + ((int64_t)n * p.Cin * p.T + (f - p.tc)) * HW;
+        cstride = (int64_t)p.T * HW;
+    }
+    const int jc = f - p.T;                               // new_cache[j] = Z[T + j]
+    float* ncdst = (p.new_cache && jc >= 0 && jc < p.tc) ? p.new_cache + ((int64_t)n * p.Cin * p.tc + jc) * HW : nullptr;
+    const int64_t ncstride = (int64_t)p.tc * HW;
+    for (int i = threadIdx.x; i < 32 * 32; i += 256) {
+        const int c = i >> 5, px = i & 31;
+        const int ci = cb * 32 + c, w = w0 + px;
+        float v = 0.f;
+        if (w < p.W && ci < p.Cin) {
+            if (src) v = __ldg(src + ci * cstride + (int64_t)h * p.W + w);
+            if (ncdst) ncdst[ci * ncstride + (int64_t)h * p.W + w] = v;
+        }
+        tile[c * 33 + px] = v;
+    }
+    __syncthreads();
+    const int px = threadIdx.x >> 3, q = threadIdx.x & 7;    // pixel, channel quad
+    const int w = w0 + px;
+    if (w < p.W) {
+        float4 hi, lo;
+        hi.x = tile[(4 * q + 0) * 33 + px]; hi.y = tile[(4 * q + 1) * 33 + px];
+        hi.z = tile[(4 * q + 2) * 33 + px]; hi.w = tile[(4 * q + 3) * 33 + px];
+        lo.x = tf32_lo(hi.x); lo.y = tf32_lo(hi.y); lo.z = tf32_lo(hi.z); lo.w = tf32_lo(hi.w);
+        float* dst = p.zs + ((((int64_t)n * F + f) * (2 * p.CBr) + 2 * cb) * HW + (int64_t)h * p.W + w) * 32 + 4 * q;
+        *reinterpret_cast<float4*>(dst) = hi;
+        *reinterpret_cast<float4*>(dst + HW * 32) = lo;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // frame rings: the inverse move (ring -> NCTHW) and the nearest-neighbour upsample between rings
 // ------------------------------------------------------------------------------------------------
 struct RingGeom {
@@ -424,6 +522,24 @@ __device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint32_t a_lo, uint
         "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
         : "memory");
 }
+// FP32 operands read as TF32 (the low 13 mantissa bits are ignored), K = 8 per instruction, FP32 accumulate
+__device__ __forceinline__ void tc_mma_tf32(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                            uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "mov.b64 da, {%1, %2};\n\t"
+        "mov.b64 db, {%3, %4};\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], da, db, %5, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+template <bool TF32>
+__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                       uint32_t idesc, uint32_t accumulate) {
+    if (TF32) tc_mma_tf32(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate);
+    else tc_mma_bf16(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate);
+}
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
@@ -614,7 +730,14 @@ __device__ __forceinline__ uint32_t epi_pair(float a0, float a1, uint32_t res_pa
 // when every CTA has signalled it (release: fence + atomic; acquire: polled load + proxy fence before the TMA
 // loads).  All CTAs are co-resident (grid <= SM count, 1 CTA per SM) and stagers never wait on consumers, so the
 // dependency is acyclic; the wait is bounded like every other.
-template <int KB, int NB, int KS, int TPBC, bool FUSED, bool COOP>
+// TF32 (FP32 layers, "3xTF32"): KB = 64 then means 128-byte rows of 32 FP32 channels.  An FP32 product a*w is
+// evaluated as hi(a)*lo(w) + lo(a)*hi(w) + hi(a)*hi(w) with hi = the TF32 truncation the tensor core applies by
+// itself and lo = the FP32 remainder, staged and packed explicitly: the staging copy holds two blocks per channel
+// block (a, a - hi(a)), the packed weights three images (lo(w), w, w).  The whole K loop runs three times, one
+// pass per term, the two small correction terms first: the tensor core's FP32 accumulation truncates, which
+// costs a fraction of the accumulator's last bit per step, so the long chain of full-size terms is kept as short
+// as it can be and the corrections are summed while the accumulator is still 2^-11 of its final size.
+template <int KB, int NB, int KS, int TPBC, bool FUSED, bool COOP, bool TF32 = false>
 __global__ void __launch_bounds__((FUSED || COOP) ? TC_THREADS_FUSED : TC_THREADS, 1)
 conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged activations (c, w, h, cb, n*F+f), or x
                       const __grid_constant__ CUtensorMap tm_c,   // fused mode: the cache
@@ -622,6 +745,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                       const TcParams p, const StageParams sp) {
     static_assert(!(FUSED && COOP), "one or the other");
     static_assert(!FUSED || KB == 32, "the fused mode transposes 32-channel blocks");
+    static_assert(!TF32 || (KB == 64 && !FUSED && !COOP), "FP32 layers: 128-byte rows, plain variant");
     constexpr uint32_t ROWB = KB * 2;                       // bytes per pixel row (one swizzle span)
     constexpr uint32_t LAYOUT = (KB == 64) ? 2u : 4u;       // 128-byte / 64-byte swizzle
     constexpr uint32_t B_SBO = 8 * ROWB;                    // 8-row group pitch of the weight tile
@@ -743,6 +867,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                     }
                 }
                 const int dt0 = (p.first_frame - t * stt > 0) ? (p.first_frame - t * stt + dlt - 1) / dlt : 0;   // first tap whose frame exists
+                for (int pass = 0; pass < (TF32 ? 3 : 1); ++pass)
                 for (int dt = dt0; ok && dt < p.kt; ++dt)
                     for (int cb = 0; ok && cb < p.CB; ++cb) {
                         int fr = p.f0 + t * stt + dt * dlt;       // ring slot of Z frame t s_t + dt d_t (f0 = 0: the frame itself)
@@ -755,7 +880,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                             mbar_expect_tx(bar, a_bytes);
                             const int dh = p.per_tap_a ? tp / p.kw : 0, dw = p.per_tap_a ? tp % p.kw : 0;
                             tma_load_5d(smem_u32(ring_a + (size_t)s * p.a_slot), &tm_a, bar, 0, w0 * stw - pw + dw * dlw,
-                                        h0 * sth - ph + dh * dlh, cb, fz);
+                                        h0 * sth - ph + dh * dlh, TF32 ? 2 * cb + (pass == 1) : cb, fz);
                             if (++s == p.SA) { s = 0; phase ^= 1; }
                         }
                     }
@@ -775,12 +900,13 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                 const int nt = tile % p.NT;
                 const int t = (tile / p.NT) % p.T;
                 const int dt0 = (p.first_frame - t * stt > 0) ? (p.first_frame - t * stt + dlt - 1) / dlt : 0;   // first tap whose frame exists
+                for (int pass = 0; pass < (TF32 ? 3 : 1); ++pass)
                 for (int dt = dt0; ok && dt < p.kt; ++dt)
                     for (int cb = 0; ok && cb < p.CB; ++cb) {
                         // split_n: this launch runs half-width output-channel tiles; the packed image of a full tile
                         // holds its two halves back to back (the swizzle repeats every 8 rows), so a half tile of a
                         // tap is a contiguous piece of it and only the distance between taps differs
-                        const uint8_t* src = p.wq + (size_t)((dt * p.CB + cb) * (p.NT >> p.split_n) + (nt >> p.split_n)) * spatial * src_tap +
+                        const uint8_t* src = p.wq + (size_t)(((pass * p.kt + dt) * p.CB + cb) * (p.NT >> p.split_n) + (nt >> p.split_n)) * spatial * src_tap +
                                              (size_t)(nt & p.split_n) * p.b_tap;
                         for (int tp = 0; tp < spatial; tp += p.TPB) {
                             if (!(ok = mbar_wait(&sh->empty_b[s], phase, sh, p, SITE_B_EMPTY))) break;
@@ -805,7 +931,9 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
         // The whole warp runs the loop (warp-uniform control flow); one elected lane issues.
         const int iss = warp - 2;
         // instruction descriptor: D=F32, A=B=BF16, both K-major, N = NPAD, M = 128
-        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.NPAD >> 3) << 17) | ((128u >> 4) << 24);
+        // (operand formats: 1 = BF16, 2 = TF32)
+        constexpr uint32_t FMT = TF32 ? 2u : 1u;
+        const uint32_t idesc = (1u << 4) | (FMT << 7) | (FMT << 10) | ((uint32_t)(p.NPAD >> 3) << 17) | ((128u >> 4) << 24);
         const uint32_t a_hi = make_desc_hi((uint32_t)BW * ROWB, LAYOUT);  // 8-pixel groups are one image row apart
         const uint32_t b_hi = make_desc_hi(B_SBO, LAYOUT);
         const uint32_t a_blk = (uint32_t)(iss * NBW) * ((8 * ROWB) >> 4);  // descriptor offset of this issuer's first block
@@ -827,7 +955,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                 tc_fence_after();
                 const uint32_t d0 = tmem_base + (uint32_t)(acc * NB + iss * NBW) * p.NPAD;
                 uint32_t accumulate = 0;
-                for (int kb = (p.kt - dt0) * p.CB; ok && kb > 0; --kb) {     // (dt, ci-block) stages
+                for (int kb = (TF32 ? 3 : 1) * (p.kt - dt0) * p.CB; ok && kb > 0; --kb) {     // (pass, dt, ci-block) stages
                     if (!(ok = mbar_wait(&sh->full_a[sa], pa, sh, p, SITE_A_FULL))) break;
 #pragma unroll
                     for (int g = 0; g < STAGES; ++g) {
@@ -847,7 +975,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                                 for (int j = 0; j < NBW; ++j) {
 #pragma unroll
                                     for (int k = 0; k < KSTEPS; ++k)
-                                        tc_mma_bf16(d0 + j * p.NPAD, a_lo + j * ((8 * ROWB) >> 4) + 2 * k, a_hi, b_lo + 2 * k, b_hi,
+                                        tc_mma<TF32>(d0 + j * p.NPAD, a_lo + j * ((8 * ROWB) >> 4) + 2 * k, a_hi, b_lo + 2 * k, b_hi,
                                                     idesc, (tap == 0 && k == 0) ? accumulate : 1u);
                                 }
                             }
@@ -877,6 +1005,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
             tc_fence_after();
             const uint32_t d0 = tmem_base + (uint32_t)(acc * NB + iss * NBW) * p.NPAD;
             uint32_t accumulate = 0;
+            for (int pass = 0; pass < (TF32 ? 3 : 1); ++pass)
             for (int dt = dt0; ok && dt < p.kt; ++dt)
                 for (int cb = 0; ok && cb < p.CB; ++cb) {
                     uint32_t a_row = 0;  // descriptor low word of the halo row of the current tap row
@@ -905,7 +1034,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                                 for (int j = 0; j < NBW; ++j) {
 #pragma unroll
                                     for (int k = 0; k < KSTEPS; ++k)
-                                        tc_mma_bf16(d0 + j * p.NPAD, a_lo + j * ((8 * ROWB) >> 4) + 2 * k, a_hi, b_lo + 2 * k, b_hi,
+                                        tc_mma<TF32>(d0 + j * p.NPAD, a_lo + j * ((8 * ROWB) >> 4) + 2 * k, a_hi, b_lo + 2 * k, b_hi,
                                                     idesc, (k == 0) ? accumulate : 1u);
                                 }
                                 if (p.per_tap_a) tc_commit(smem_u32(&sh->empty_a[sa]));

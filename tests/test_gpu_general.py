@@ -201,3 +201,47 @@ def test_general_geometry_is_refused_by_the_standard_only_entry_points(ccv):
     torch.cuda.synchronize()
     layer.close()
     valid.close()
+
+
+# ---------------------------------------------------------------------------- FP32 layers on the tensor cores (3xTF32)
+F32_TC_CASES = [
+    # N, Cin, Cout, T, H, W, k, cache frames, stride, pad, dil, dil_t, stride_t
+    (1, 32, 32, 2, 20, 24, (3, 3, 3), 2, (1, 1), (1, 1), (1, 1), 1, 1),
+    (2, 48, 40, 3, 17, 19, (3, 3, 3), 1, (1, 1), (1, 1), (1, 1), 1, 1),      # channels off the block size, short cache, odd W
+    (1, 16, 300, 1, 33, 40, (3, 3, 3), 0, (1, 1), (1, 1), (1, 1), 1, 1),     # two output-channel tiles, no history
+    (1, 64, 64, 4, 16, 32, (1, 1, 1), 0, (1, 1), (0, 0), (1, 1), 1, 1),      # 1x1x1
+    (1, 40, 24, 3, 21, 26, (3, 3, 3), 4, (2, 2), (1, 1), (1, 1), 2, 1),      # strided, temporal dilation
+    (1, 32, 48, 4, 18, 20, (2, 3, 3), 1, (1, 1), (2, 2), (2, 2), 1, 2),      # dilated, temporal stride
+    (1, 96, 96, 2, 40, 48, (3, 3, 3), 2, (1, 1), (1, 1), (1, 1), 1, 1),      # K = 2592
+]
+
+
+@pytest.mark.parametrize("N,Cin,Cout,T,H,W,k,cf,stride,pad,dil,dil_t,stride_t", F32_TC_CASES)
+def test_fp32_on_tensor_cores_3xtf32(ccv, N, Cin, Cout, T, H, W, k, cf, stride, pad, dil, dil_t, stride_t):
+    """FP32 layers as three TF32 tensor-core products per FP32 product (hi*hi + hi*lo + lo*hi, FP32 accumulate):
+    within the FP32 tolerance (max <= 1e-4 x RMS) of the oracle, cache update bit-exact."""
+    c = _case(N, Cin, Cout, T, H, W, k, si.F32, cf, seed=41)
+    m, ctr = run_general(ccv, c, stride, pad, dil, dil_t, flags=ccv.FLAG_F32_TENSOR, stride_t=stride_t)
+    assert ctr["tcgen05_bf16"] == 1 and ctr["simt"] == 0
+    print("3xTF32", (N, Cin, Cout, T, H, W, k), "K =", Cin * k[0] * k[1] * k[2], m)
+
+
+def test_fp32_route_selection_by_size(ccv):
+    """Small FP32 calls stay on the FP32-FMA kernel, calls of a GFLOP and more go to the tensor cores; both within
+    tolerance and close to each other."""
+    c = _case(1, 64, 64, 4, 44, 80, (3, 3, 3), si.F32, 2, seed=42)          # 3.1 GFLOP
+    ref, ref_nc = oracle.forward_general(c["x"], c["cache"], c["w"], c["b"])
+    outs = {}
+    for name, flags in (("auto", 0), ("fma", ccv.FLAG_FORCE_SIMT)):
+        layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), flags=flags)
+        o, nc = layer(to_dev(c["x"]), to_dev(c["cache"]))
+        small, _ = layer(to_dev(c["x"])[:, :, :1, :8, :8].contiguous(), None)    # 2.8 MFLOP: FP32-FMA kernel either way
+        torch.cuda.synchronize()
+        ctr = layer.counters()
+        assert (ctr["tcgen05_bf16"], ctr["simt"]) == ((1, 1) if name == "auto" else (0, 2))
+        check(as_f64(o), ref, "f32")
+        assert np.array_equal(bits(nc), ref_nc)
+        outs[name] = as_f64(o)
+        layer.close()
+    rms = float(np.sqrt(np.mean(ref ** 2)))
+    assert np.abs(outs["auto"] - outs["fma"]).max() <= 1e-4 * rms
