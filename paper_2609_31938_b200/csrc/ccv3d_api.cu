@@ -166,8 +166,8 @@ void make_plan_f32(const ccv3d_desc& d, TcPlan* pl) {
     const int per = (d.cout + pl->NT - 1) / pl->NT;
     pl->NPAD = (per + 15) / 16 * 16;
     pl->cout_pad = pl->NT * pl->NPAD;
-    pl->NB = (4 * pl->NPAD <= 512) ? 2 : 1;
-    pl->ACC = (2 * pl->NB * pl->NPAD <= 512) ? 2 : 1;
+    pl->NB = (8 * pl->NPAD <= 512) ? 2 : 1;                 // two accumulators per pixel block (see the kernel)
+    pl->ACC = (4 * pl->NB * pl->NPAD <= 512) ? 2 : 1;
 }
 
 uint32_t pow2_cols(uint32_t c) {
@@ -369,7 +369,8 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
         2 * (int64_t)N * ((Ho + 15) / 16) * ((Wo + 7) / 8) * To * pl.NT <= h->sm_count) {
         split_n = 1; NT = 2 * pl.NT; NPAD = pl.NPAD / 2;
     }
-    const int ACC = (2 * NB * NPAD <= 512) ? 2 : 1;
+    const int asets = (d.dtype == CCV3D_F32) ? 2 : 1;       // FP32 layers keep two accumulators per pixel block
+    const int ACC = (2 * asets * NB * NPAD <= 512) ? 2 : 1;
     const int TW = 8 * NB;
     const int BW = per_tap ? TW : TW + (d.kw - 1) * d.dilation[2];
     const int BH = per_tap ? 16 : 16 + (d.kh - 1) * d.dilation[1];
@@ -437,7 +438,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     if (SB > 8) SB = 8;
     while (SA < 4 && (size_t)(SA + 1) * p.a_slot + (size_t)SB * p.b_slot <= budget) ++SA;
     p.SA = SA; p.SB = SB;
-    p.tmem_cols = pow2_cols((uint32_t)(NB * NPAD * ACC));
+    p.tmem_cols = pow2_cols((uint32_t)(asets * NB * NPAD * ACC));
     if (p.tmem_cols > 512) return CCV3D_ERR_UNSUPPORTED;
     p.wait_limit_clk = h->wait_limit_clk;
     p.bias = h->bias32;
@@ -1161,12 +1162,12 @@ ccv3d_status forward_simt(ccv3d_handle* h, const void* x, const void* cache, voi
 
 // FP32 layers: the FP32-FMA kernel is exact FP32 and fine for small calls; from about a GFLOP on (or when the layer
 // asks for it) the call goes to the tensor cores as 3xTF32.  The tensor core's accumulation truncates: measured
-// against the FP64 definition the worst element is off by about 8.8e-9 x K x RMS(out) (K = cin*kt*kh*kw; 4.6e-5 at
-// K = 5184, 9.1e-5 at K = 10368), so layers with K > 8192 stay on the FP32-FMA kernel unless the flag insists.
+// against the FP64 definition the worst element is off by about 4.5e-9 x K x RMS(out) (K = cin*kt*kh*kw; 2.5e-5 at
+// K = 5184, 4.7e-5 at K = 10368), so layers with K > 16384 stay on the FP32-FMA kernel unless the flag insists.
 bool f32_takes_tensor_cores(const ccv3d_handle* h, int N, int T, int H, int W) {
     const ccv3d_desc& d = h->d;
     if (d.flags & CCV3D_FLAG_F32_TENSOR) return true;
-    if ((int64_t)d.cin * d.kt * d.kh * d.kw > 8192) return false;
+    if ((int64_t)d.cin * d.kt * d.kh * d.kw > 16384) return false;
     const double flops = 2.0 * N * out_t(d, T) * out_h(d, H) * out_w(d, W) * d.cout * d.cin * d.kt * d.kh * d.kw;
     return flops >= 1.0e9;
 }

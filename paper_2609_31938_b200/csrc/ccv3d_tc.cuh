@@ -746,6 +746,8 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     static_assert(!(FUSED && COOP), "one or the other");
     static_assert(!FUSED || KB == 32, "the fused mode transposes 32-channel blocks");
     static_assert(!TF32 || (KB == 64 && !FUSED && !COOP), "FP32 layers: 128-byte rows, plain variant");
+    // (TF32 layers always write FP32 through the direct-store epilogue, which is where the two accumulators of the
+    // last pass are added)
     constexpr uint32_t ROWB = KB * 2;                       // bytes per pixel row (one swizzle span)
     constexpr uint32_t LAYOUT = (KB == 64) ? 2u : 4u;       // 128-byte / 64-byte swizzle
     constexpr uint32_t B_SBO = 8 * ROWB;                    // 8-row group pitch of the weight tile
@@ -753,6 +755,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     constexpr int TW = 8 * NB;                              // tile width in pixels; tile height is 16
     constexpr int NI = (NB >= 2) ? 2 : 1;                   // MMA-issuing warps (2 and 3), each owning NB/NI pixel blocks
     constexpr int NBW = NB / NI;
+    constexpr int ASETS = TF32 ? 2 : 1;                     // accumulators per tile buffer (TF32: the last pass uses two)
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -953,9 +956,15 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                 const int dt0 = (p.first_frame - t * stt > 0) ? (p.first_frame - t * stt + dlt - 1) / dlt : 0;   // first tap whose frame exists
                 if (!(ok = mbar_wait(&sh->acc_empty[acc], pacc, sh, p, SITE_ACC_EMPTY))) break;
                 tc_fence_after();
-                const uint32_t d0 = tmem_base + (uint32_t)(acc * NB + iss * NBW) * p.NPAD;
-                uint32_t accumulate = 0;
-                for (int kb = (TF32 ? 3 : 1) * (p.kt - dt0) * p.CB; ok && kb > 0; --kb) {     // (pass, dt, ci-block) stages
+                const uint32_t d_first = tmem_base + (uint32_t)(acc * ASETS * NB + iss * NBW) * p.NPAD;
+                uint32_t accumulate = 0, accumulate2 = 0;
+                const int nst = (p.kt - dt0) * p.CB;                          // (dt, ci-block) stages per pass
+                for (int st = 0; ok && st < (TF32 ? 3 : 1) * nst; ++st) {     // (pass, dt, ci-block) stages
+                    // TF32: the stages of the last (full-size) pass alternate between two accumulators, which halves
+                    // the length of either truncating chain; the epilogue adds the two
+                    const bool second = TF32 && st >= 2 * nst && ((st - 2 * nst) & 1);
+                    const uint32_t d0 = d_first + (second ? (uint32_t)NB * p.NPAD : 0u);
+                    const uint32_t acc_in = second ? accumulate2 : accumulate;
                     if (!(ok = mbar_wait(&sh->full_a[sa], pa, sh, p, SITE_A_FULL))) break;
 #pragma unroll
                     for (int g = 0; g < STAGES; ++g) {
@@ -976,7 +985,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
 #pragma unroll
                                     for (int k = 0; k < KSTEPS; ++k)
                                         tc_mma<TF32>(d0 + j * p.NPAD, a_lo + j * ((8 * ROWB) >> 4) + 2 * k, a_hi, b_lo + 2 * k, b_hi,
-                                                    idesc, (tap == 0 && k == 0) ? accumulate : 1u);
+                                                    idesc, (tap == 0 && k == 0) ? acc_in : 1u);
                                 }
                             }
                             tc_commit(smem_u32(&sh->empty_b[sb]));
@@ -986,7 +995,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                         if (++sb == p.SB) { sb = 0; pb ^= 1; b_ring = b_ring0; }
                     }
                     if (!ok) break;
-                    accumulate = 1;
+                    if (second) accumulate2 = 1; else accumulate = 1;
                     if (elect_one()) tc_commit(smem_u32(&sh->empty_a[sa]));
                     __syncwarp();
                     a_ring += a_slotstep;
@@ -1003,11 +1012,15 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
             const int dt0 = (p.first_frame - t * stt > 0) ? (p.first_frame - t * stt + dlt - 1) / dlt : 0;   // first tap whose frame exists
             if (!(ok = mbar_wait(&sh->acc_empty[acc], pacc, sh, p, SITE_ACC_EMPTY))) break;
             tc_fence_after();
-            const uint32_t d0 = tmem_base + (uint32_t)(acc * NB + iss * NBW) * p.NPAD;
-            uint32_t accumulate = 0;
+            const uint32_t d_first = tmem_base + (uint32_t)(acc * ASETS * NB + iss * NBW) * p.NPAD;
+            uint32_t accumulate1 = 0, accumulate2 = 0;
+            int st2 = 0;                                       // stage counter of the last pass
             for (int pass = 0; pass < (TF32 ? 3 : 1); ++pass)
             for (int dt = dt0; ok && dt < p.kt; ++dt)
                 for (int cb = 0; ok && cb < p.CB; ++cb) {
+                    const bool second = TF32 && pass == 2 && (st2++ & 1);   // see the straight-line variant
+                    const uint32_t d0 = d_first + (second ? (uint32_t)NB * p.NPAD : 0u);
+                    uint32_t accumulate = second ? accumulate2 : accumulate1;
                     uint32_t a_row = 0;  // descriptor low word of the halo row of the current tap row
                     if (!p.per_tap_a) {
                         if (!(ok = mbar_wait(&sh->full_a[sa], pa, sh, p, SITE_A_FULL))) break;
@@ -1057,6 +1070,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                         __syncwarp();
                         if (++sa == p.SA) { sa = 0; pa ^= 1; }
                     }
+                    if (second) accumulate2 = accumulate; else accumulate1 = accumulate;
                 }
             if (!ok) break;
             if (elect_one()) tc_commit(smem_u32(&sh->acc_full[acc]));
@@ -1099,7 +1113,10 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
             tc_fence_after();
-            const uint32_t t_acc = tmem_base + (uint32_t)(acc * NB) * p.NPAD + ((uint32_t)(q * 32) << 16);
+            const uint32_t t_acc = tmem_base + (uint32_t)(acc * ASETS * NB) * p.NPAD + ((uint32_t)(q * 32) << 16);
+            // TF32: was the second accumulator of the last pass used (at least two stages per pass)?
+            const int dt0e = (p.first_frame - t * stt > 0) ? (p.first_frame - t * stt + dlt - 1) / dlt : 0;
+            const bool two_acc = TF32 && (p.kt - dt0e) * p.CB >= 2;
             if (p.epi_tma) {
                 // BF16 tile chunks -> shared memory -> one TMA store per chunk.  NCTHW output: [ECH channels][16 rows]
                 // [TW pixels]; ring output: [16 rows][TW pixels][32 channels] with the 64-byte swizzle of the tensor map.
@@ -1174,6 +1191,14 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                         const int nc = (p.NPAD - c0 >= 32) ? 32 : 16;
                         if (nc == 32) tc_ld32(t_acc + blk * p.NPAD + c0, v); else tc_ld16(t_acc + blk * p.NPAD + c0, v);
                         tc_wait_ld();
+                        if (two_acc) {
+                            uint32_t v2[32];
+                            if (nc == 32) tc_ld32(t_acc + (NB + blk) * p.NPAD + c0, v2); else tc_ld16(t_acc + (NB + blk) * p.NPAD + c0, v2);
+                            tc_wait_ld();
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (j < nc) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(v2[j]));
+                        }
                         if (valid) {
                             if (p.out_f32) {
 #pragma unroll
