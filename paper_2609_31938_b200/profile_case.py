@@ -28,12 +28,17 @@ def main():
     ap.add_argument("--no-cache", action="store_true")
     ap.add_argument("--flags", type=int, default=0, help="CCV3D_FLAG_* bits (16 = two-kernel schedule, 8 = fused route)")
     ap.add_argument("--ring", action="store_true", help="resident activations: input and output in frame rings")
+    ap.add_argument("--f32", action="store_true", help="FP32 layer (tensor cores by 3xTF32 when the call is large enough)")
     a = ap.parse_args()
-    c = si.conv_case(1, a.cin, a.cout, a.t, a.h, a.w, k=tuple(a.k), cache=None if a.no_cache else "random")
-    up = lambda v: None if v is None else torch.from_numpy(v.view(np.int16)).cuda().view(torch.bfloat16)
+    c = si.conv_case(1, a.cin, a.cout, a.t, a.h, a.w, k=tuple(a.k), cache=None if a.no_cache else "random",
+                     dtype=si.F32 if a.f32 else si.BF16)
+    if a.f32:
+        up = lambda v: None if v is None else torch.from_numpy(v).cuda()
+    else:
+        up = lambda v: None if v is None else torch.from_numpy(v.view(np.int16)).cuda().view(torch.bfloat16)
     layer = ccv.CausalConv3d(up(c["w"]), up(c["b"]), flags=a.flags)
     x, cache = up(c["x"]), up(c["cache"])
-    out = torch.empty((1, a.cout, a.t, a.h, a.w), dtype=torch.bfloat16, device="cuda")
+    out = torch.empty((1, a.cout, a.t, a.h, a.w), dtype=torch.float32 if a.f32 else torch.bfloat16, device="cuda")
     nc = torch.empty_like(cache) if cache is not None else None
     if a.ring:
         tc = a.k[0] - 1
