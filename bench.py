@@ -38,6 +38,9 @@ DEFAULT_WORKLOAD = "cfg3_bf16_192"
 # convolution in one kernel), from an ncu capture of a quarter-size case (192->192, T=4, 176x320: 241.4 MB read +
 # 222.6 MB written) scaled by the pixel count; the summary is profiles/conv3d_tcgen05_coop_192ch_176x320.md.
 TRAFFIC_BYTES_PER_LAUNCH = {"cfg3_bf16_192": 4 * (241.4e6 + 222.6e6)}
+# The same for the kernel on frame rings (profiles/conv3d_tcgen05_ring_192ch_176x320.md: 131.9 MB read + 51.3 MB
+# written during the kernel, the rest of the 86.5 MB output still in L2 when it ends).
+TRAFFIC_BYTES_PER_LAUNCH_RESIDENT = {"cfg3_bf16_192": 4 * (131.9e6 + 51.3e6)}
 
 
 def measured_peaks():
@@ -284,6 +287,70 @@ def chain_leg(dev):
     return res
 
 
+def other_configs_leg(dev):
+    """The remaining benchmark configurations in short bursts (10 calls each after 3 warm-ups), through ccv3d_forward
+    (NCTHW boundary) and, for the cached layers, through ccv3d_forward_ring.  Inputs of these secondary legs are
+    drawn on the device (seeded normal activations, fan-in-scaled weights): same shapes and distributions as the
+    seeded host generator, which the headline workload and the tests use."""
+    import math
+    import torch
+    import paper_2609_31938_b200 as ccv
+    peaks = measured_peaks()
+    out = {}
+    gen = torch.Generator(device=dev).manual_seed(0)
+    # the HBM-bound 1x1x1 layer first, after a pause: right after a long tensor-bound run the part is still in its
+    # power-capped state and the same kernel measures 20 % slower
+    time.sleep(1.0)
+    for name in ("cfg4c_bf16_pw_192_96", "cfg2_bf16_384", "cfg4a_bf16_96", "cfg4b_bf16_192_96"):
+        d = {k: v for k, v in si.CONFIGS[name].items() if k not in ("dtype", "x_dist")}
+        N, Cin, Cout, T, H, W, k = d["N"], d["Cin"], d["Cout"], d["T"], d["H"], d["W"], d["k"]
+        rnd = lambda *shape, std=1.0: (torch.randn(*shape, device=dev, generator=gen) * std).to(torch.bfloat16)
+        x = rnd(N, Cin, T, H, W)
+        cache = rnd(N, Cin, k[0] - 1, H, W) if k[0] > 1 else None
+        layer = ccv.CausalConv3d(rnd(Cout, Cin, *k, std=1.0 / math.sqrt(Cin * k[0] * k[1] * k[2])), rnd(Cout, std=math.sqrt(0.1)))
+        y = torch.empty((N, Cout, T, H, W), dtype=torch.bfloat16, device=dev)
+        nc = torch.empty_like(cache) if cache is not None else None
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+
+        def timed(fn, iters=10):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            e0.record()
+            for _ in range(iters):
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1) / iters
+
+        ms = timed(lambda: layer(x, cache, out=y, new_cache=nc))
+        flops, abytes = si.conv_flops(**d), si.conv_bytes(**d)
+        row = {"ms_per_call": ms, "tflops": flops / (ms * 1e-3) / 1e12, "gbs": abytes / (ms * 1e6),
+               "frac_of_measured_bf16_peak": flops / (ms * 1e-3) / 1e12 / peaks["tflops"],
+               "frac_of_measured_hbm": abytes / (ms * 1e6) / peaks["hbm_gbs"]}
+        if cache is not None:
+            F = T + k[0] - 1
+            rin, rout = ccv.FrameRing(N, Cin, F, H, W), ccv.FrameRing(N, Cout, T, H, W)
+            rin.load(0, cache)
+            rin.load(k[0] - 1, x)
+            slot = [k[0] - 1]
+
+            def ring_step():
+                layer.forward_ring(rin, slot[0], k[0] - 1, T, out_ring=rout)
+                slot[0] = (slot[0] + T) % F
+
+            rms = timed(ring_step)
+            row["resident_ms_per_call"] = rms
+            row["resident_tflops"] = flops / (rms * 1e-3) / 1e12
+            del rin, rout
+        assert layer.device_status()[0] == ccv.OK
+        layer.close()
+        out[name] = row
+        del x, cache, y, nc
+        torch.cuda.empty_cache()
+    return out
+
+
 def main_ours(args):
     import torch
     import paper_2609_31938_b200 as ccv
@@ -440,12 +507,14 @@ def main_ours(args):
         resident = {"value": flops / (r_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": r_ms, "steps": r_steps,
                     "frac_of_measured_bf16_peak": flops / (r_ms * 1e-3) / 1e12 / peaks["tflops"],
                     "algorithmic_bytes_per_step": int(r_bytes), "gpu_launches_per_step": 1,
+                    "traffic": TRAFFIC_BYTES_PER_LAUNCH_RESIDENT.get(name),
                     "note": "ccv3d_forward_ring: input and output in frame rings (channels-last blocks), temporal "
                             "history left in the ring by the previous call"}
         del rin, rout
 
     cpu = cpu_baseline(name) if world == 1 else None
     chain = chain_leg(dev) if (world == 1 and not args.no_chain) else None
+    others = other_configs_leg(dev) if (world == 1 and not args.no_chain) else None
     line = {"metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
@@ -461,6 +530,8 @@ def main_ours(args):
         line["resident"] = resident
     if chain is not None:
         line["decoder_chain"] = chain
+    if others is not None:
+        line["other_configs"] = others
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
