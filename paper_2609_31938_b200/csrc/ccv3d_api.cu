@@ -170,6 +170,27 @@ void make_plan_f32(const ccv3d_desc& d, TcPlan* pl) {
     pl->ACC = (4 * pl->NB * pl->NPAD <= 512) ? 2 : 1;
 }
 
+// Taps per weight stage and ring depths that fit `budget` bytes of shared memory: a whole kernel row of taps per
+// stage when that stays small (so that a stage carries enough MMAs), at least two activation and two weight
+// stages, weight ring up to 8 deep, then a deeper activation ring with what is left.
+ccv3d_status size_pipeline(TcParams* p, size_t budget, bool per_tap, int kw) {
+    p->TPB = (!per_tap && (size_t)p->b_tap * kw <= 40960) ? kw : 1;
+    int SA = per_tap ? 3 : 2;
+    for (;;) {
+        p->b_slot = (uint32_t)align_up((uint64_t)p->b_tap * p->TPB, 1024);
+        if ((size_t)SA * p->a_slot + 3 * (size_t)p->b_slot <= budget) break;
+        if (p->TPB > 1) { p->TPB = 1; continue; }
+        if ((size_t)SA * p->a_slot + 2 * (size_t)p->b_slot <= budget) break;
+        return CCV3D_ERR_UNSUPPORTED;
+    }
+    int SB = (int)((budget - (size_t)SA * p->a_slot) / p->b_slot);
+    if (SB > 8) SB = 8;
+    while (SA < 4 && (size_t)(SA + 1) * p->a_slot + (size_t)SB * p->b_slot <= budget) ++SA;
+    p->SA = SA;
+    p->SB = SB;
+    return CCV3D_OK;
+}
+
 uint32_t pow2_cols(uint32_t c) {
     uint32_t v = 32;
     while (v < c) v <<= 1;
@@ -424,20 +445,8 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     // leave room for staging blocks to be resident next to a convolution CTA when the two overlap
     const size_t limit = nbands > 1 ? SMEM_LIMIT - STAGE_COEXIST_BYTES : SMEM_LIMIT;
     const size_t budget = limit - fixed;
-    // weight stage: a whole kernel row of taps when that stays small, so that a stage carries enough MMAs
-    p.TPB = (!per_tap && (size_t)p.b_tap * d.kw <= 40960) ? d.kw : 1;
-    int SA = per_tap ? 3 : 2;
-    for (;;) {
-        p.b_slot = (uint32_t)align_up((uint64_t)p.b_tap * p.TPB, 1024);
-        if ((size_t)SA * p.a_slot + 3 * (size_t)p.b_slot <= budget) break;
-        if (p.TPB > 1) { p.TPB = 1; continue; }
-        if ((size_t)SA * p.a_slot + 2 * (size_t)p.b_slot <= budget) break;
-        return CCV3D_ERR_UNSUPPORTED;
-    }
-    int SB = (int)((budget - (size_t)SA * p.a_slot) / p.b_slot);
-    if (SB > 8) SB = 8;
-    while (SA < 4 && (size_t)(SA + 1) * p.a_slot + (size_t)SB * p.b_slot <= budget) ++SA;
-    p.SA = SA; p.SB = SB;
+    s = size_pipeline(&p, budget, per_tap != 0, d.kw);
+    if (s != CCV3D_OK) return s;
     p.tmem_cols = pow2_cols((uint32_t)(asets * NB * NPAD * ACC));
     if (p.tmem_cols > 512) return CCV3D_ERR_UNSUPPORTED;
     p.wait_limit_clk = h->wait_limit_clk;
@@ -451,7 +460,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     } else {
         h->tm_o = h->tm_a;  // never dereferenced on this path; any valid descriptor will do
     }
-    const size_t smem = fixed + (size_t)SA * p.a_slot + (size_t)SB * p.b_slot;
+    const size_t smem = fixed + (size_t)p.SA * p.a_slot + (size_t)p.SB * p.b_slot;
     // straight-line tap loops need unit spatial dilation (the tap offsets are compile-time); padding and the temporal
     // dilation only move the producer's TMA coordinates
     const int ks = (!per_tap && d.dilation[1] == 1 && d.dilation[2] == 1 && d.kh == d.kw && (d.kh == 1 || d.kh == 3)) ? d.kh : 0;
@@ -637,7 +646,7 @@ ccv3d_status forward_fused(ccv3d_handle* h, const void* x, const void* cache, vo
     s = encode_ncthw_map(h, &tm_o, out, N, d.cout, T, H, W, TW, 16, p.ECH, CU_TENSOR_MAP_SWIZZLE_NONE);
     if (s != CCV3D_OK) return s;
 
-    const size_t smem = fixed + (size_t)SA * p.a_slot + (size_t)SB * p.b_slot;
+    const size_t smem = fixed + (size_t)p.SA * p.a_slot + (size_t)p.SB * p.b_slot;
     const int grid = p.total_tiles < h->sm_count ? p.total_tiles : h->sm_count;
     const int ks = (d.kh == d.kw && (d.kh == 1 || d.kh == 3)) ? d.kh : 0;
     cudaEvent_t* pev = (h->prof_on && h->prof_ev) ? h->prof_ev + 3 * (h->prof_n % PROF_SLOTS) : nullptr;
@@ -875,19 +884,8 @@ ccv3d_status forward_tc_static(ccv3d_handle* h, const void* x, const void* cache
     p.e_slot = p.epi_tma ? (uint32_t)(p.ECH * 16 * TW * 2) : 0;
     const size_t fixed = 1024 + align_up(sizeof(TcShared), 128) + 2 * (size_t)p.e_slot;
     const size_t budget = SMEM_LIMIT - fixed;
-    p.TPB = ((size_t)p.b_tap * d.kw <= 40960) ? d.kw : 1;
-    int SA = 2;
-    for (;;) {
-        p.b_slot = (uint32_t)align_up((uint64_t)p.b_tap * p.TPB, 1024);
-        if ((size_t)SA * p.a_slot + 3 * (size_t)p.b_slot <= budget) break;
-        if (p.TPB > 1) { p.TPB = 1; continue; }
-        if ((size_t)SA * p.a_slot + 2 * (size_t)p.b_slot <= budget) break;
-        return CCV3D_ERR_UNSUPPORTED;
-    }
-    int SB = (int)((budget - (size_t)SA * p.a_slot) / p.b_slot);
-    if (SB > 8) SB = 8;
-    while (SA < 4 && (size_t)(SA + 1) * p.a_slot + (size_t)SB * p.b_slot <= budget) ++SA;
-    p.SA = SA; p.SB = SB;
+    s = size_pipeline(&p, budget, false, d.kw);
+    if (s != CCV3D_OK) return s;
     p.tmem_cols = pow2_cols((uint32_t)(NB * pl.NPAD * ACC));
     if (p.tmem_cols > 512) return CCV3D_ERR_UNSUPPORTED;
     p.wait_limit_clk = h->wait_limit_clk;
@@ -907,7 +905,7 @@ ccv3d_status forward_tc_static(ccv3d_handle* h, const void* x, const void* cache
     } else {
         tm_o = tm_a;   // never dereferenced on this path
     }
-    const size_t smem = fixed + (size_t)SA * p.a_slot + (size_t)SB * p.b_slot;
+    const size_t smem = fixed + (size_t)p.SA * p.a_slot + (size_t)p.SB * p.b_slot;
     const int grid = p.total_tiles < h->sm_count ? p.total_tiles : h->sm_count;
     const int ks = (d.kh == d.kw && (d.kh == 1 || d.kh == 3)) ? d.kh : 0;
 #define CCV3D_LAUNCH_STATIC(KBv)                                                                              \
@@ -1060,19 +1058,8 @@ ccv3d_status forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int x_slot, int
     }
     const size_t fixed = 1024 + align_up(sizeof(TcShared), 128) + 2 * (size_t)p.e_slot;
     const size_t budget = SMEM_LIMIT - fixed;
-    p.TPB = ((size_t)p.b_tap * d.kw <= 40960) ? d.kw : 1;
-    int SA = 2;
-    for (;;) {
-        p.b_slot = (uint32_t)align_up((uint64_t)p.b_tap * p.TPB, 1024);
-        if ((size_t)SA * p.a_slot + 3 * (size_t)p.b_slot <= budget) break;
-        if (p.TPB > 1) { p.TPB = 1; continue; }
-        if ((size_t)SA * p.a_slot + 2 * (size_t)p.b_slot <= budget) break;
-        return CCV3D_ERR_UNSUPPORTED;
-    }
-    int SB = (int)((budget - (size_t)SA * p.a_slot) / p.b_slot);
-    if (SB > 8) SB = 8;
-    while (SA < 4 && (size_t)(SA + 1) * p.a_slot + (size_t)SB * p.b_slot <= budget) ++SA;
-    p.SA = SA; p.SB = SB;
+    s = size_pipeline(&p, budget, false, d.kw);
+    if (s != CCV3D_OK) return s;
     p.tmem_cols = pow2_cols((uint32_t)(NB * NPAD * ACC));
     if (p.tmem_cols > 512) return CCV3D_ERR_UNSUPPORTED;
     p.wait_limit_clk = h->wait_limit_clk;
@@ -1080,7 +1067,7 @@ ccv3d_status forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int x_slot, int
     p.wq = (const uint8_t*)h->wp;
     p.out = out_ncthw;
     p.status = h->status;
-    const size_t smem = fixed + (size_t)SA * p.a_slot + (size_t)SB * p.b_slot;
+    const size_t smem = fixed + (size_t)p.SA * p.a_slot + (size_t)p.SB * p.b_slot;
     const int grid = p.total_tiles < h->sm_count ? p.total_tiles : h->sm_count;
     const int ks = (d.kh == d.kw && (d.kh == 1 || d.kh == 3)) ? d.kh : 0;
     cudaEvent_t* pev = (h->prof_on && h->prof_ev) ? h->prof_ev + 3 * (h->prof_n % PROF_SLOTS) : nullptr;
