@@ -58,7 +58,8 @@ typedef enum {
                                             by TMA and transposes in shared memory (needs W % 8 == 0, else the staged route is taken). About as fast as
                                             the default route in short bursts, ~3 % slower sustained; for callers that cannot afford the workspace. */
 #define CCV3D_FLAG_F32_TENSOR 0x20u       /* FP32 layers: always use the tensor cores (3xTF32: each FP32 product as hi*hi + hi*lo + lo*hi of TF32
-                                            operands, FP32 accumulate); the default sends calls under ~1 GFLOP to the FP32-FMA kernel */
+                                            operands, FP32 accumulate); the default sends calls under 0.2 GFLOP, and layers with cin*kt*kh*kw > 16384,
+                                            to the FP32-FMA kernel */
 #define CCV3D_FLAG_TC_PER_TAP_A 0x2u    /* tensor-core kernel: fetch the activation tile once per tap (no halo reuse in shared memory) */
 
 /* Layer description, fixed at create time (Algorithm 1's Require line: W, b, p, s, d, g).
@@ -115,6 +116,9 @@ typedef struct {
  *   stream  a cudaStream_t (NULL = default stream).
  * The handle owns: packed weights, FP32 bias, a status word, an optional
  * workspace (see ccv3d_forward).  The caller owns everything else.
+ * Two environment variables are read here, for diagnosis only: CCV3D_WAIT_LIMIT_MS (1..10000, default about one
+ * second of SM clocks) bounds every wait inside the kernels; CCV3D_NO_PDL (any value) launches the frame-ring
+ * kernels without programmatic stream serialization.
  */
 ccv3d_status ccv3d_create(ccv3d_handle** out_h, const ccv3d_desc* d, const void* w_dev, const void* b_dev,
                           void* stream);
@@ -132,6 +136,7 @@ ccv3d_status ccv3d_create(ccv3d_handle** out_h, const ccv3d_desc* d, const void*
  *   are always the INPUT extents.  See ccv3d_out_dims.)
  * out must not overlap x or cache; new_cache must not overlap x, cache or out
  * (CCV3D_ERR_ALIAS): ping-pong two cache buffers.  All pointers must be 16-byte aligned.
+ * The current CUDA device must be the one the handle was created on (else CCV3D_ERR_INVALID_ARG).
  * With CCV3D_FLAG_OVERLAP large images are processed in bands of rows on three side streams owned by the handle
  * (staging of the next band overlaps the convolution of the current one); they fork from `stream` after
  * everything enqueued on it so far and join it before the call returns, so the caller only ever needs to order
@@ -311,6 +316,17 @@ ccv3d_status ccv3d_upsample_ring(const ccv3d_ring* in, int32_t in_slot0, const c
 ccv3d_status ccv3d_forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int32_t x_slot, int32_t hist_frames,
                                 const ccv3d_ring* res, int32_t res_slot, const ccv3d_ring* out_ring,
                                 int32_t out_slot, void* out_ncthw, int32_t T, void* stream);
+
+/*
+ * ccv3d_forward_ring with a nearest-neighbour upsample fused into the store: out_ring has 2H x 2W pixels and
+ * F >= T*rt slots; output frame t is written to the rt slots (out_slot + t*rt + j) mod F, every pixel 2x2 times
+ * (the epilogue issues 4*rt strided TMA stores of the same shared-memory tile).  Bit-identical to
+ * ccv3d_forward_ring into an H x W ring followed by ccv3d_upsample_ring.  rt >= 1; everything else as
+ * ccv3d_forward_ring with a ring output.
+ */
+ccv3d_status ccv3d_forward_ring_up(ccv3d_handle* h, const ccv3d_ring* in, int32_t x_slot, int32_t hist_frames,
+                                   const ccv3d_ring* res, int32_t res_slot, const ccv3d_ring* out_ring, int32_t out_slot,
+                                   int32_t rt, int32_t T, void* stream);
 
 #ifdef __cplusplus
 }

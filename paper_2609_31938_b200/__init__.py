@@ -51,7 +51,7 @@ EXPORTS = ("ccv3d_create", "ccv3d_forward", "ccv3d_forward_host", "ccv3d_workspa
            "ccv3d_get_counters", "ccv3d_device_status", "ccv3d_status_string", "ccv3d_add_bf16",
            "ccv3d_upsample_bf16", "ccv3d_profile_enable", "ccv3d_profile_read", "ccv3d_forward_static", "ccv3d_selftest_wait_timeout", "ccv3d_forward_ex",
            "ccv3d_ring_kb", "ccv3d_ring_bytes", "ccv3d_ring_load", "ccv3d_ring_store", "ccv3d_upsample_ring",
-           "ccv3d_forward_ring", "ccv3d_out_dims")
+           "ccv3d_forward_ring", "ccv3d_out_dims", "ccv3d_forward_ring_up")
 
 
 def _load() -> ctypes.CDLL:
@@ -87,6 +87,7 @@ def _load() -> ctypes.CDLL:
     lib.ccv3d_ring_store.argtypes = [rp, i32, vp, i32, vp]
     lib.ccv3d_upsample_ring.argtypes = [rp, i32, rp, i32, i32, i32, vp]
     lib.ccv3d_forward_ring.argtypes = [vp, rp, i32, i32, rp, i32, rp, i32, vp, i32, vp]
+    lib.ccv3d_forward_ring_up.argtypes = [vp, rp, i32, i32, rp, i32, rp, i32, i32, i32, vp]
     for name in EXPORTS:
         if name not in ("ccv3d_status_string", "ccv3d_ring_bytes"):
             getattr(lib, name).restype = ctypes.c_int
@@ -229,6 +230,13 @@ def ccv3d_forward_ring(h, rin: Ring, x_slot: int, hist_frames: int, res: Ring | 
                                   None if out_ring is None else ctypes.byref(out_ring), out_slot, out_ncthw, T, stream)
 
 
+def ccv3d_forward_ring_up(h, rin: Ring, x_slot: int, hist_frames: int, res: Ring | None, res_slot: int, out_ring: Ring,
+                          out_slot: int, rt: int, T: int, stream=0) -> int:
+    return lib.ccv3d_forward_ring_up(h, ctypes.byref(rin), x_slot, hist_frames,
+                                     None if res is None else ctypes.byref(res), res_slot, ctypes.byref(out_ring),
+                                     out_slot, rt, T, stream)
+
+
 class FrameRing:
     """A frame ring on the current CUDA device: torch owns the memory, `c` is the struct the C calls take."""
 
@@ -311,13 +319,19 @@ class CausalConv3d:
     __call__ = forward
 
     def forward_ring(self, rin: FrameRing, x_slot, hist_frames, T, out_ring: FrameRing | None = None, out_slot=0,
-                     out=None, res: FrameRing | None = None, res_slot=0):
-        """The layer on resident activations (see ccv3d_forward_ring): reads `rin`, writes `out_ring` or NCTHW `out`."""
-        s = ccv3d_forward_ring(self.h, rin.c, x_slot, hist_frames, None if res is None else res.c, res_slot,
-                               None if out_ring is None else out_ring.c, out_slot,
-                               None if out is None else out.data_ptr(), T, self.torch.cuda.current_stream().cuda_stream)
+                     out=None, res: FrameRing | None = None, res_slot=0, up_rt=0):
+        """The layer on resident activations (see ccv3d_forward_ring): reads `rin`, writes `out_ring` or NCTHW `out`.
+        up_rt > 0: `out_ring` is 2H x 2W and receives the 2x2-upsampled output, every frame up_rt times."""
+        st = self.torch.cuda.current_stream().cuda_stream
+        if up_rt > 0:
+            s = ccv3d_forward_ring_up(self.h, rin.c, x_slot, hist_frames, None if res is None else res.c, res_slot,
+                                      out_ring.c, out_slot, up_rt, T, st)
+        else:
+            s = ccv3d_forward_ring(self.h, rin.c, x_slot, hist_frames, None if res is None else res.c, res_slot,
+                                   None if out_ring is None else out_ring.c, out_slot,
+                                   None if out is None else out.data_ptr(), T, st)
         if s != OK:
-            raise Ccv3dError(s, "ccv3d_forward_ring", "ccv3d_out_dims")
+            raise Ccv3dError(s, "ccv3d_forward_ring")
         return out_ring if out_ring is not None else out
 
     def counters(self):

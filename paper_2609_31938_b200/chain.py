@@ -14,7 +14,7 @@ normalisation or non-linearity: the chain exists to exercise streaming, caches a
 """
 from __future__ import annotations
 
-from . import CausalConv3d, Ccv3dError, FrameRing, OK, ccv3d_add_bf16, ccv3d_upsample_bf16, ccv3d_upsample_ring
+from . import CausalConv3d, Ccv3dError, FrameRing, OK, ccv3d_add_bf16, ccv3d_upsample_bf16
 
 LAYERS = ("A1", "A2", "PA", "B1", "B2", "PB", "C1", "C2")
 
@@ -71,8 +71,9 @@ class ResidentDecoderChain:
     """The same chain with every activation between the chunk input and the chunk output resident in frame rings
     (channels-last blocks, the order the tensor-core kernel reads): a layer writes straight into the next layer's
     ring, the temporal history of a layer is whatever earlier chunks left in its ring (no cache tensors, no cache
-    update), and the residual additions run in the convolution epilogues.  Per chunk: one layout move for the
-    input, eight convolution kernels, two upsample kernels.  Results are bit-identical to DecoderChain."""
+    update), the residual additions run in the convolution epilogues and the two upsamples in the stores of the
+    1x1x1 layers.  Per chunk: one layout move for the input and eight convolution kernels.  Results are
+    bit-identical to DecoderChain."""
 
     def __init__(self, weights: dict, biases: dict):
         import torch
@@ -91,17 +92,12 @@ class ResidentDecoderChain:
         ca, cb, cc = self.ch["A1"][0], self.ch["B1"][0], self.ch["C1"][0]
         R = FrameRing
         self.rings = {
-            "A1": R(N, ca, T + 2, H, W), "A2": R(N, ca, T + 2, H, W), "PA": R(N, ca, T, H, W), "UA": R(N, cb, T, H, W),
+            "A1": R(N, ca, T + 2, H, W), "A2": R(N, ca, T + 2, H, W), "PA": R(N, ca, T, H, W),
             "B1": R(N, cb, 4 * T + 2, 2 * H, 2 * W), "B2": R(N, cb, 4 * T + 2, 2 * H, 2 * W),
-            "PB": R(N, cb, 4 * T, 2 * H, 2 * W), "UB": R(N, cc, 4 * T, 2 * H, 2 * W),
+            "PB": R(N, cb, 4 * T, 2 * H, 2 * W),
             "C1": R(N, cc, 4 * T + 2, 4 * H, 4 * W), "C2": R(N, cc, 4 * T + 2, 4 * H, 4 * W),
         }
         self.geom = (N, T, H, W)
-
-    def _up(self, rin, rout, out_slot, T, rt):
-        s = ccv3d_upsample_ring(rin.c, 0, rout.c, out_slot, T, rt, self.torch.cuda.current_stream().cuda_stream)
-        if s != OK:
-            raise Ccv3dError(s, "ccv3d_upsample_ring")
 
     def _block(self, first, second, nxt, slot, hist, T, out=None):
         """x <- x + conv2(conv1(x)) with x in ring `first`: the sum goes to ring `nxt` (slot 0) or to NCTHW `out`."""
@@ -126,11 +122,9 @@ class ResidentDecoderChain:
         ha, hb = min(2, self.seen), min(2, 4 * self.seen)
         r["A1"].load(sa, a)
         self._block("A1", "A2", "PA", sa, ha, T)
-        L["PA"].forward_ring(r["PA"], 0, 0, T, out_ring=r["UA"], out_slot=0)
-        self._up(r["UA"], r["B1"], sb, T, 4)
+        L["PA"].forward_ring(r["PA"], 0, 0, T, out_ring=r["B1"], out_slot=sb, up_rt=4)      # 1x1x1, upsample in the store
         self._block("B1", "B2", "PB", sb, hb, 4 * T)
-        L["PB"].forward_ring(r["PB"], 0, 0, 4 * T, out_ring=r["UB"], out_slot=0)
-        self._up(r["UB"], r["C1"], sc, 4 * T, 1)
+        L["PB"].forward_ring(r["PB"], 0, 0, 4 * T, out_ring=r["C1"], out_slot=sc, up_rt=1)
         self._block("C1", "C2", None, sc, hb, 4 * T, out=out)
         self.seen += T
         self.slot = {"A": (sa + T) % r["A1"].F, "B": (sb + 4 * T) % r["B1"].F, "C": (sc + 4 * T) % r["C1"].F}

@@ -947,14 +947,15 @@ RingGeom ring_geom(const ccv3d_ring* r) {
 }
 
 // Tensor map over a ring as (channel in block, w, h, channel block, n*F + slot).
+// es > 1: traversal stride along w and h (box_w x box_h pixels are delivered to / taken from every es-th pixel).
 ccv3d_status encode_ring_map(ccv3d_handle* h, CUtensorMap* tm, const ccv3d_ring* r, int box_c, int box_w, int box_h,
-                             CUtensorMapSwizzle swz) {
+                             CUtensorMapSwizzle swz, int es_px = 1) {
     const uint64_t rowb = (uint64_t)r->KB * 2;
     cuuint64_t dims[5] = {(cuuint64_t)r->KB, (cuuint64_t)r->W, (cuuint64_t)r->H, (cuuint64_t)(r->C / r->KB),
                           (cuuint64_t)r->N * r->F};
     cuuint64_t strides[4] = {rowb, rowb * r->W, rowb * r->W * r->H, rowb * r->W * r->H * (r->C / r->KB)};
-    cuuint32_t box[5] = {(cuuint32_t)box_c, (cuuint32_t)box_w, (cuuint32_t)box_h, 1, 1};
-    cuuint32_t es[5] = {1, 1, 1, 1, 1};
+    cuuint32_t box[5] = {(cuuint32_t)box_c, (cuuint32_t)(box_w * es_px), (cuuint32_t)(box_h * es_px), 1, 1};
+    cuuint32_t es[5] = {1, (cuuint32_t)es_px, (cuuint32_t)es_px, 1, 1};
     CUresult rc = h->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, r->base, dims, strides, box, es,
                             CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
@@ -962,12 +963,13 @@ ccv3d_status encode_ring_map(ccv3d_handle* h, CUtensorMap* tm, const ccv3d_ring*
 }
 
 ccv3d_status forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int x_slot, int hist, const ccv3d_ring* res, int res_slot,
-                          const ccv3d_ring* oring, int out_slot, void* out_ncthw, int T, cudaStream_t st) {
+                          const ccv3d_ring* oring, int out_slot, void* out_ncthw, int T, cudaStream_t st, int up_rt = 0) {
     const ccv3d_desc& d = h->d;
     const TcPlan& pl = h->plan;
     const int tc = d.kt - 1;
     if (!h->use_tc || (d.flags & CCV3D_FLAG_TC_PER_TAP_A) || !standard_geom(d)) return CCV3D_ERR_UNSUPPORTED;
     if (!ring_valid(in) || T < 1 || (oring != nullptr) == (out_ncthw != nullptr)) return CCV3D_ERR_INVALID_ARG;
+    if (up_rt < 0 || (up_rt > 0 && !oring)) return CCV3D_ERR_INVALID_ARG;
     if (((uintptr_t)in->base | (uintptr_t)out_ncthw) & 15u) return CCV3D_ERR_ALIGNMENT;
     if (in->C != d.cin || in->F < T + tc || x_slot < 0 || x_slot >= in->F || hist < 0 || hist > tc) return CCV3D_ERR_INVALID_ARG;
     if (in->KB != pl.KB) return CCV3D_ERR_UNSUPPORTED;
@@ -982,8 +984,9 @@ ccv3d_status forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int x_slot, int
     }
     const uint64_t in_b = ring_bytes_of(in);
     if (oring) {
-        if (!ring_valid(oring) || oring->C != d.cout || oring->N != N || oring->H != H || oring->W != W || oring->F < T ||
-            out_slot < 0 || out_slot >= oring->F)
+        const int oscale = up_rt > 0 ? 2 : 1;              // fused upsample: the output ring is 2H x 2W, up_rt slots per frame
+        if (!ring_valid(oring) || oring->C != d.cout || oring->N != N || oring->H != oscale * H || oring->W != oscale * W ||
+            (int64_t)oring->F < (int64_t)T * (up_rt > 0 ? up_rt : 1) || out_slot < 0 || out_slot >= oring->F)
             return CCV3D_ERR_INVALID_ARG;
         if ((uintptr_t)oring->base & 15u) return CCV3D_ERR_ALIGNMENT;
         if (d.out_dtype != CCV3D_BF16 || !chunked) return CCV3D_ERR_UNSUPPORTED;
@@ -1033,7 +1036,8 @@ ccv3d_status forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int x_slot, int
         p.ECH = 32;
         p.e_slot = (uint32_t)(16 * TW * 64);
         p.out_F = oring->F; p.out_f0 = out_slot; p.out_KB = oring->KB;
-        s = encode_ring_map(h, &tm_o, oring, 32, TW, 16, CU_TENSOR_MAP_SWIZZLE_64B);
+        p.up_rt = up_rt;
+        s = encode_ring_map(h, &tm_o, oring, 32, TW, 16, CU_TENSOR_MAP_SWIZZLE_64B, up_rt > 0 ? 2 : 1);
         if (s != CCV3D_OK) return s;
     } else {
         p.epi_tma = (!p.out_f32 && W % 8 == 0) ? 1 : 0;
@@ -1147,7 +1151,13 @@ ccv3d_status forward_simt(ccv3d_handle* h, const void* x, const void* cache, voi
     return CCV3D_OK;
 }
 
-// FP32 layers: the FP32-FMA kernel is exact FP32 and fine for small calls; from about a GFLOP on (or when the layer
+// A handle belongs to the device it was created on: its weights, maps and scratch live there.
+bool on_handle_device(const ccv3d_handle* h) {
+    int dev = -1;
+    return cudaGetDevice(&dev) == cudaSuccess && dev == h->device;
+}
+
+// FP32 layers: the FP32-FMA kernel is exact FP32 and fine for small calls; from 0.2 GFLOP on (or when the layer
 // asks for it) the call goes to the tensor cores as 3xTF32.  The tensor core's accumulation truncates: measured
 // against the FP64 definition the worst element is off by about 4.5e-9 x K x RMS(out) (K = cin*kt*kh*kw; 2.5e-5 at
 // K = 5184, 4.7e-5 at K = 10368), so layers with K > 16384 stay on the FP32-FMA kernel unless the flag insists.
@@ -1156,7 +1166,7 @@ bool f32_takes_tensor_cores(const ccv3d_handle* h, int N, int T, int H, int W) {
     if (d.flags & CCV3D_FLAG_F32_TENSOR) return true;
     if ((int64_t)d.cin * d.kt * d.kh * d.kw > 16384) return false;
     const double flops = 2.0 * N * out_t(d, T) * out_h(d, H) * out_w(d, W) * d.cout * d.cin * d.kt * d.kh * d.kw;
-    return flops >= 1.0e9;
+    return flops >= 2.0e8;
 }
 
 ccv3d_status check_forward_args(const ccv3d_handle* h, const void* x, const void* cache, void* out, void* new_cache,
@@ -1358,6 +1368,7 @@ ccv3d_status ccv3d_forward_ex(ccv3d_handle* h, const void* x, const void* cache,
     h->call_cf = cache_frames;
     ccv3d_status s = check_forward_args(h, x, cache, out, new_cache, N, T, H, W, true);
     if (s != CCV3D_OK) return count(h, s);
+    if (!on_handle_device(h)) return count(h, CCV3D_ERR_INVALID_ARG);
     cudaStream_t st = (cudaStream_t)stream;
     if (h->use_tc && pointwise_eligible(h, T, H, W)) s = forward_pointwise(h, x, out, N, T, H, W, st);
     else if (h->use_tc && fused_eligible(h, W)) s = forward_fused(h, x, cache, out, new_cache, N, T, H, W, st);
@@ -1380,6 +1391,7 @@ ccv3d_status ccv3d_forward_static(ccv3d_handle* h, const void* x, const void* ca
     h->call_cf = cache ? hist_len(h->d) : 0;
     ccv3d_status s = check_forward_args(h, x, cache, out, new_cache, N, T, H, W, true);
     if (s != CCV3D_OK) return count(h, s);
+    if (!on_handle_device(h)) return count(h, CCV3D_ERR_INVALID_ARG);
     if (!h->use_tc) return count(h, CCV3D_ERR_UNSUPPORTED);   // the FP32-FMA route has no scratch to replace
     if (!standard_geom(h->d)) return count(h, CCV3D_ERR_UNSUPPORTED);   // unit stride and dilation, size-preserving padding only
     return count(h, forward_tc_static(h, x, cache, out, new_cache, N, T, H, W, (cudaStream_t)stream));
@@ -1570,11 +1582,23 @@ ccv3d_status ccv3d_upsample_ring(const ccv3d_ring* in, int32_t in_slot0, const c
     return cudaGetLastError() == cudaSuccess ? CCV3D_OK : cuda_fail();
 }
 
+ccv3d_status ccv3d_forward_ring_up(ccv3d_handle* h, const ccv3d_ring* in, int32_t x_slot, int32_t hist_frames,
+                                   const ccv3d_ring* res, int32_t res_slot, const ccv3d_ring* out_ring, int32_t out_slot,
+                                   int32_t rt, int32_t T, void* stream) {
+    if (!h) return CCV3D_ERR_INVALID_ARG;
+    h->ctr.calls++;
+    if (rt < 1 || !out_ring) return count(h, CCV3D_ERR_INVALID_ARG);
+    if (!on_handle_device(h)) return count(h, CCV3D_ERR_INVALID_ARG);
+    return count(h, forward_ring(h, in, x_slot, hist_frames, res, res_slot, out_ring, out_slot, nullptr, T,
+                                 (cudaStream_t)stream, rt));
+}
+
 ccv3d_status ccv3d_forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int32_t x_slot, int32_t hist_frames,
                                 const ccv3d_ring* res, int32_t res_slot, const ccv3d_ring* out_ring,
                                 int32_t out_slot, void* out_ncthw, int32_t T, void* stream) {
     if (!h) return CCV3D_ERR_INVALID_ARG;
     h->ctr.calls++;
+    if (!on_handle_device(h)) return count(h, CCV3D_ERR_INVALID_ARG);
     return count(h, forward_ring(h, in, x_slot, hist_frames, res, res_slot, out_ring, out_slot, out_ncthw, T,
                                  (cudaStream_t)stream));
 }

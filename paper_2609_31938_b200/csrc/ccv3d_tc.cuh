@@ -626,6 +626,8 @@ struct TcParams {
     const __nv_bfloat16* res; // optional residual ring [N][res_F][res_CB][H][W][res_KB] holding Cout channels, or null
     int res_F, res_f0, res_CB, res_KB;   // residual frame t is slot (res_f0 + t) mod res_F
     int out_F, out_f0, out_KB;           // epi_tma == 2: output frame t goes to slot (out_f0 + t) mod out_F
+    int up_rt;                           // epi_tma == 2, > 0: the output ring is 2H x 2W; every pixel is written 2x2 times into
+                                         // each of the up_rt slots (out_f0 + t*up_rt + j) mod out_F (nearest-neighbour upsample)
     const float* bias;        // [NT*NPAD]
     const uint8_t* wq;        // packed weight tiles [dt][cb][nt][sp] of b_tap bytes each
     void* out;
@@ -1165,7 +1167,16 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                     fence_async_smem();
                     epi_bar_sync();
                     if (elected) {
-                        if (RING && p.epi_tma == 2) {
+                        if (RING && p.epi_tma == 2 && p.up_rt > 0) {
+                            // fused nearest-neighbour upsample: the tensor map walks the 2H x 2W ring with a traversal
+                            // stride of 2 pixels, so one store drops the tile onto every second pixel from (b, a)
+                            for (int j = 0; j < p.up_rt; ++j) {
+                                const int os = (p.out_f0 + t * p.up_rt + j) % p.out_F;
+                                for (int ab = 0; ab < 4; ++ab)
+                                    tma_store_5d(&tm_o, smem_u32(stg), co0 % p.out_KB, 2 * tx * TW + (ab & 1), 2 * ty * 16 + (ab >> 1),
+                                                 co0 / p.out_KB, n * p.out_F + os);
+                            }
+                        } else if (RING && p.epi_tma == 2) {
                             int os = p.out_f0 + t;
                             if (os >= p.out_F) os -= p.out_F;
                             tma_store_5d(&tm_o, smem_u32(stg), co0 % p.out_KB, tx * TW, ty * 16, co0 / p.out_KB, n * p.out_F + os);

@@ -227,7 +227,7 @@ def test_fp32_on_tensor_cores_3xtf32(ccv, N, Cin, Cout, T, H, W, k, cf, stride, 
 
 
 def test_fp32_route_selection_by_size(ccv):
-    """Small FP32 calls stay on the FP32-FMA kernel, calls of a GFLOP and more go to the tensor cores; both within
+    """Small FP32 calls stay on the FP32-FMA kernel, calls of 0.2 GFLOP and more go to the tensor cores; both within
     tolerance and close to each other."""
     c = _case(1, 64, 64, 4, 44, 80, (3, 3, 3), si.F32, 2, seed=42)          # 3.1 GFLOP
     ref, ref_nc = oracle.forward_general(c["x"], c["cache"], c["w"], c["b"])

@@ -149,6 +149,32 @@ def test_residual_in_the_epilogue_equals_convolution_then_addition(ccv, N, C, H,
     layer.close()
 
 
+@pytest.mark.parametrize("Cin,Cout,H,W,k,T,rt", [(64, 64, 20, 24, (1, 1, 1), 1, 4), (192, 96, 12, 21, (1, 1, 1), 4, 1),
+                                                 (64, 32, 18, 20, (3, 3, 3), 2, 2)])
+def test_upsample_fused_into_the_store_equals_store_then_upsample(ccv, Cin, Cout, H, W, k, T, rt):
+    """ccv3d_forward_ring_up (4*rt strided TMA stores of the epilogue tile) against ccv3d_forward_ring followed by
+    ccv3d_upsample_ring: the same bits in the same slots, nothing else of the output ring touched."""
+    tc = k[0] - 1
+    c = si.conv_case(1, Cin, Cout, T, H, W, k=k, cache="random", seed=25)
+    layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]))
+    rin = ccv.FrameRing(1, Cin, T + tc, H, W)
+    if tc:
+        rin.load(0, to_dev(c["cache"]))
+    rin.load(tc, to_dev(c["x"]))
+    small = ccv.FrameRing(1, Cout, T, H, W)
+    want = ccv.FrameRing(1, Cout, T * rt + 1, 2 * H, 2 * W, zero=True)
+    got = ccv.FrameRing(1, Cout, T * rt + 1, 2 * H, 2 * W, zero=True)
+    st = torch.cuda.current_stream().cuda_stream
+    layer.forward_ring(rin, tc, tc, T, out_ring=small)
+    assert ccv.ccv3d_upsample_ring(small.c, 0, want.c, 1, T, rt, st) == ccv.OK
+    layer.forward_ring(rin, tc, tc, T, out_ring=got, out_slot=1, up_rt=rt)
+    torch.cuda.synchronize()
+    assert layer.device_status()[0] == ccv.OK
+    assert torch.equal(got.buf, want.buf)
+    assert ccv.ccv3d_forward_ring_up(layer.h, rin.c, tc, tc, None, 0, small.c, 0, 1, T, st) == ccv.ERR_INVALID_ARG   # not 2H x 2W
+    layer.close()
+
+
 def test_ring_argument_errors(ccv):
     c = si.conv_case(1, 64, 64, 2, 16, 16, seed=23)
     layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]))
