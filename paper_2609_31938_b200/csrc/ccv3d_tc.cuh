@@ -643,6 +643,7 @@ constexpr int TC_THREADS = 256;
 constexpr int TC_THREADS_FUSED = 384;    // + 4 transposer warps
 constexpr int RAW_PX = 32;               // pixels per row of a raw box (64 bytes), starting 8 pixels left of the tile
 constexpr int TC_MAX_STAGES = 12;
+constexpr int TC_BIAS_SMEM = 512;
 
 struct TcShared {  // placed after the rings
     uint64_t full_a[TC_MAX_STAGES], empty_a[TC_MAX_STAGES];
@@ -651,6 +652,7 @@ struct TcShared {  // placed after the rings
     uint64_t raw_full[2], raw_empty[2];
     uint32_t tmem_base;
     volatile int abort_flag;
+    alignas(16) float bias_s[TC_BIAS_SMEM];   // the layer's padded bias when it fits (the epilogue reads it once per element)
 };
 
 // Bounded wait.  Returns false when the limit expired or another role of this CTA aborted.
@@ -1092,6 +1094,14 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
         constexpr bool RING = !FUSED && !COOP;                 // frame-ring output and residual: plain variant only
         const bool has_res = RING && p.res != nullptr;
         int ebuf = 0;
+        // bias: a shared-memory copy when the padded channel count fits.  A global load per element costs little
+        // while the next tile's MMAs run, but its latency sits in the exposed tail of a CTA's last tile: 11 us
+        // against 5 us for a 192-channel tile.
+        const bool bias_smem = p.NT * p.NPAD <= TC_BIAS_SMEM;
+        if (bias_smem)
+            for (int i = threadIdx.x - 128; i < p.NT * p.NPAD; i += 128) sh->bias_s[i] = __ldg(p.bias + i);
+        epi_bar_sync();
+        const float* bias = bias_smem ? sh->bias_s : p.bias;
         for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
             const int nt = tile % p.NT;
             int r = tile / p.NT;
@@ -1141,11 +1151,17 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                         if (p.ECH == 32) tc_ld32(t_acc + blk * p.NPAD + c0, v); else tc_ld16(t_acc + blk * p.NPAD + c0, v);
                         tc_wait_ld();
                         uint32_t pk[16];
+                        float bb[32];                       // the chunk's bias: eight 16-byte reads (co0 is a multiple of 16)
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            const float4 b4 = (4 * j < p.ECH) ? *reinterpret_cast<const float4*>(bias + co0 + 4 * j)
+                                                              : make_float4(0.f, 0.f, 0.f, 0.f);
+                            bb[4 * j] = b4.x; bb[4 * j + 1] = b4.y; bb[4 * j + 2] = b4.z; bb[4 * j + 3] = b4.w;
+                        }
 #pragma unroll
                         for (int j = 0; j < 16; ++j)
-                            pk[j] = (2 * j < p.ECH) ? epi_pair(__uint_as_float(v[2 * j]) + __ldg(p.bias + co0 + 2 * j),
-                                                               __uint_as_float(v[2 * j + 1]) + __ldg(p.bias + co0 + 2 * j + 1),
-                                                               rr[j], has_res)
+                            pk[j] = (2 * j < p.ECH) ? epi_pair(__uint_as_float(v[2 * j]) + bb[2 * j],
+                                                               __uint_as_float(v[2 * j + 1]) + bb[2 * j + 1], rr[j], has_res)
                                                     : 0u;
                         const uint32_t px = (uint32_t)((m >> 3) * TW + blk * 8 + (m & 7));   // pixel of the tile, row-major
                         if (RING && p.epi_tma == 2) {
@@ -1217,15 +1233,15 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                                     const int co = co0 + j;
                                     if (j < nc && co < p.Cout)
                                         reinterpret_cast<float*>(p.out)[((int64_t)n * p.Cout + co) * p.T * HW + pix] =
-                                            __uint_as_float(v[j]) + __ldg(p.bias + co);
+                                            __uint_as_float(v[j]) + bias[co];
                                 }
                             } else {
 #pragma unroll
                                 for (int j = 0; j < 16; ++j) {
                                     const int co = co0 + 2 * j;
                                     if (2 * j < nc) {
-                                        const uint32_t pr = epi_pair(__uint_as_float(v[2 * j]) + __ldg(p.bias + co),
-                                                                     __uint_as_float(v[2 * j + 1]) + __ldg(p.bias + co + 1), rr[j], has_res);
+                                        const uint32_t pr = epi_pair(__uint_as_float(v[2 * j]) + bias[co],
+                                                                     __uint_as_float(v[2 * j + 1]) + bias[co + 1], rr[j], has_res);
                                         unsigned short* o = reinterpret_cast<unsigned short*>(p.out) +
                                                             ((int64_t)n * p.Cout + co) * p.T * HW + pix;
                                         if (co < p.Cout) o[0] = (unsigned short)(pr & 0xFFFFu);
