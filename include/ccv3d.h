@@ -60,6 +60,9 @@ typedef enum {
 #define CCV3D_FLAG_F32_TENSOR 0x20u       /* FP32 layers: always use the tensor cores (3xTF32: each FP32 product as hi*hi + hi*lo + lo*hi of TF32
                                             operands, FP32 accumulate); the default sends calls under 0.2 GFLOP, and layers with cin*kt*kh*kw > 16384,
                                             to the FP32-FMA kernel */
+#define CCV3D_FLAG_NO_PAIR 0x40u          /* tensor-core route: never run tiles on pairs of CTAs (cta_group::2 MMAs with M = 256, each SM
+                                            streaming half of every weight tile) - the default for layers with more than 128 output
+                                            channels per tile and 3x3 or 1x1 spatial kernels */
 #define CCV3D_FLAG_TC_PER_TAP_A 0x2u    /* tensor-core kernel: fetch the activation tile once per tap (no halo reuse in shared memory) */
 
 /* Layer description, fixed at create time (Algorithm 1's Require line: W, b, p, s, d, g).

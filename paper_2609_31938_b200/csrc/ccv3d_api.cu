@@ -67,6 +67,8 @@ struct ccv3d_handle {
     CUtensorMap tm_a;
     ShapeKey tm_a_key;
     CUtensorMap tm_o;
+    CUtensorMap tm_w;    // CTA pairs: 2-D map over the packed weights (half-tile boxes)
+    bool tm_w_ready;
     long long wait_limit_clk;
     // side streams and events of the banded, overlapped schedule (created with the handle)
     cudaStream_t side[3];
@@ -313,6 +315,87 @@ ccv3d_status launch_stage(ccv3d_handle* h, StageParams sp, int h0, int h1, int n
     return CCV3D_OK;
 }
 
+// CTA pairs: clusters of two CTAs, one 16x16-pixel tile per cluster (see the kernel).  tm_w is the 2-D map over the
+// packed weights from which each CTA takes its half of every tap's tile.
+template <int KB, int KS, int TPBC, bool COOP>
+ccv3d_status launch_tc_pair(ccv3d_handle* h, const CUtensorMap& tm_a, const CUtensorMap& tm_w, const CUtensorMap& tm_o,
+                            const TcParams& p, const StageParams& sp, size_t smem, int grid, cudaStream_t st) {
+    auto kern = conv3d_tcgen05_kernel<KB, 1, KS, TPBC, false, COOP, false, true>;
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
+        return cuda_fail();
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(COOP ? TC_THREADS_FUSED : TC_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = (h->pdl && !COOP) ? 2 : 1;
+    if (cudaLaunchKernelEx(&cfg, kern, tm_a, tm_w, tm_o, p, sp) != cudaSuccess) return cuda_fail();
+    if (cudaGetLastError() != cudaSuccess) return cuda_fail();
+    h->ctr.kernel_launches++;
+    return CCV3D_OK;
+}
+
+// 2-D map over the packed weights: rows of KB channels (one swizzle span), all tiles of all taps one after another;
+// a box is half a tile (NPAD/2 rows).  Encoded once per handle.
+ccv3d_status weight_map(ccv3d_handle* h, const CUtensorMap** out) {
+    if (h->tm_w_ready) { *out = &h->tm_w; return CCV3D_OK; }
+    CUtensorMap* tm = &h->tm_w;
+    const int box_rows = h->plan.NPAD / 2;
+    const TcPlan& pl = h->plan;
+    const ccv3d_desc& d = h->d;
+    const uint64_t rows = (uint64_t)d.kt * pl.CB * pl.NT * d.kh * d.kw * pl.NPAD;
+    cuuint64_t dims[2] = {(cuuint64_t)pl.KB, (cuuint64_t)rows};
+    cuuint64_t strides[1] = {(cuuint64_t)pl.KB * 2};
+    cuuint32_t box[2] = {(cuuint32_t)pl.KB, (cuuint32_t)box_rows};
+    cuuint32_t es[2] = {1, 1};
+    if (rows > 0x7FFFFFFFull || box_rows > 256) return CCV3D_ERR_UNSUPPORTED;
+    CUresult rc = h->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, h->wp, dims, strides, box, es,
+                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (rc != CUDA_SUCCESS) return CCV3D_ERR_CUDA;
+    h->tm_w_ready = true;
+    *out = tm;
+    return CCV3D_OK;
+}
+
+// Dispatch over the compiled pair variants (straight-line taps only: ks = 3 or 1).
+template <bool COOP>
+ccv3d_status launch_pair_any(ccv3d_handle* h, const CUtensorMap& tm_a, const CUtensorMap& tm_o, const TcParams& p,
+                             const StageParams& sp, size_t smem, int grid, int ks, cudaStream_t st) {
+    const CUtensorMap* tm_w = nullptr;
+    ccv3d_status s = weight_map(h, &tm_w);
+    if (s != CCV3D_OK) return s;
+    if (h->plan.KB == 64) {
+        if (ks == 3 && p.TPB == 3) return launch_tc_pair<64, 3, 3, COOP>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
+        if (ks == 3) return launch_tc_pair<64, 3, 1, COOP>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
+        return launch_tc_pair<64, 1, 1, COOP>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
+    }
+    if (ks == 3 && p.TPB == 3) return launch_tc_pair<32, 3, 3, COOP>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
+    if (ks == 3) return launch_tc_pair<32, 3, 1, COOP>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
+    return launch_tc_pair<32, 1, 1, COOP>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
+}
+
+// A layer runs on CTA pairs when its output-channel tile is wide (more than 128 channels: one 128-pixel block per
+// CTA anyway, and the MMAs long enough for one issuing thread to feed two SMs), its taps are the straight-line
+// kind, and there are tiles for at least half of the pairs.
+bool pair_eligible(const ccv3d_handle* h, int64_t pair_tiles) {
+    const ccv3d_desc& d = h->d;
+    const TcPlan& pl = h->plan;
+    if (d.flags & CCV3D_FLAG_NO_PAIR) return false;
+    if (d.dtype != CCV3D_BF16 || (d.flags & CCV3D_FLAG_TC_PER_TAP_A)) return false;
+    if (d.stride[1] != 1 || d.stride[2] != 1 || d.dilation[1] != 1 || d.dilation[2] != 1) return false;
+    if (d.kh != d.kw || (d.kh != 1 && d.kh != 3)) return false;
+    if (pl.NB != 1 || pl.NPAD % 16 != 0 || h->sm_count < 2) return false;
+    return pair_tiles * pl.NT >= h->sm_count / 4;
+}
+
 ccv3d_status launch_conv(ccv3d_handle* h, TcParams p, int nb, int ty0, int ty1, size_t smem, int ks, cudaStream_t st) {
     const TcPlan& pl = h->plan;
     p.ty_begin = ty0;
@@ -392,7 +475,12 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     }
     const int asets = (d.dtype == CCV3D_F32) ? 2 : 1;       // FP32 layers keep two accumulators per pixel block
     const int ACC = (2 * asets * NB * NPAD <= 512) ? 2 : 1;
-    const int TW = 8 * NB;
+    // CTA pairs (wide output-channel tiles): 16x16-pixel tiles shared by the two CTAs of a cluster; not combined with
+    // the banded multi-stream schedule
+    const bool pair = !split_n && !per_tap && !f32 && !(d.flags & CCV3D_FLAG_OVERLAP) &&
+                      pair_eligible(h, (int64_t)N * ((Ho + 15) / 16) * ((Wo + 15) / 16) * To);
+    const int TW = 8 * NB;                                 // pixels per row of a CTA's part of a tile (pair: NB is 1)
+    const int TWT = pair ? 16 : TW;                        // tile width in the tile index space
     const int BW = per_tap ? TW : TW + (d.kw - 1) * d.dilation[2];
     const int BH = per_tap ? 16 : 16 + (d.kh - 1) * d.dilation[1];
     ShapeKey key{h->workspace, N, T, H, W, BW};
@@ -410,13 +498,13 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     p.str_h = d.stride[1]; p.str_w = d.stride[2]; p.str_t = d.stride[0];
     p.CB = pl.CB; p.NT = NT; p.NPAD = NPAD;
     const int tiles_h = (Ho + 15) / 16;
-    p.tiles_w = (Wo + TW - 1) / TW;
+    p.tiles_w = (Wo + TWT - 1) / TWT;
     p.first_frame = tc - cf;
     p.out_f32 = d.out_dtype == CCV3D_F32;
     p.per_tap_a = per_tap;
     p.ACC = ACC;
     p.a_slot = (uint32_t)align_up((uint64_t)BW * BH * pl.KB * 2, 1024);
-    p.b_tap = (uint32_t)NPAD * pl.KB * 2;
+    p.b_tap = (uint32_t)(pair ? NPAD / 2 : NPAD) * pl.KB * 2;   // a CTA of a pair holds half of every weight tile
     p.split_n = split_n;
     p.b_src_tap = split_n ? (uint32_t)pl.NPAD * pl.KB * 2 : 0;
     // epilogue: BF16 output rows that TMA can address (W*2 bytes a multiple of 16) go through shared memory
@@ -477,7 +565,12 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
         const int64_t total = (int64_t)N * tiles_h * p.tiles_w * To * NT;
         if (total > 0x7FFFFFFF) return CCV3D_ERR_UNSUPPORTED;
         p.total_tiles = (int)total;
-        const int grid = p.total_tiles < h->sm_count ? p.total_tiles : h->sm_count;
+        int grid = p.total_tiles < h->sm_count ? p.total_tiles : h->sm_count;
+        if (pair) {
+            grid = 2 * (p.total_tiles < h->sm_count / 2 ? p.total_tiles : h->sm_count / 2);
+            s = launch_pair_any<true>(h, h->tm_a, h->tm_o, p, sp, smem, grid, ks, st);
+            if (s != CCV3D_OK) return s;
+        } else {
 #define CCV3D_LAUNCH_COOP(KBv, NBv)                                                                        \
     do {                                                                                                   \
         if (ks == 3 && p.TPB == 3) s = launch_tc_coop<KBv, NBv, 3, 3>(h, p, sp, smem, grid, st);           \
@@ -491,6 +584,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
         else CCV3D_LAUNCH_COOP(32, 1);
 #undef CCV3D_LAUNCH_COOP
         if (s != CCV3D_OK) return s;
+        }
     } else if (nbands == 1) {
         if (pev) cudaEventRecord(pev[0], st);
         if (f32) {
@@ -509,7 +603,19 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
         }
         if (s != CCV3D_OK) return s;
         if (pev) cudaEventRecord(pev[1], st);
-        s = launch_conv(h, p, NB, 0, tiles_h, smem, ks, st);
+        if (pair) {
+            p.ty_begin = 0;
+            p.tiles_h = tiles_h;
+            const int64_t total = (int64_t)N * tiles_h * p.tiles_w * To * NT;
+            if (total > 0x7FFFFFFF) return CCV3D_ERR_UNSUPPORTED;
+            p.total_tiles = (int)total;
+            const int grid = 2 * (p.total_tiles < h->sm_count / 2 ? p.total_tiles : h->sm_count / 2);
+            StageParams nosp;
+            memset(&nosp, 0, sizeof(nosp));
+            s = launch_pair_any<false>(h, h->tm_a, h->tm_o, p, nosp, smem, grid, ks, st);
+        } else {
+            s = launch_conv(h, p, NB, 0, tiles_h, smem, ks, st);
+        }
         if (s != CCV3D_OK) return s;
     } else {
         cudaStream_t s_stage = h->side[0];
@@ -1006,8 +1112,12 @@ ccv3d_status forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int x_slot, int
     if (NB == 1 && pl.NPAD % 64 == 0 && 2 * (int64_t)N * ((H + 15) / 16) * ((W + 7) / 8) * T * pl.NT <= h->sm_count) {
         split_n = 1; NT = 2 * pl.NT; NPAD = pl.NPAD / 2;
     }
+    // CTA pairs: 16x16-pixel tiles shared by two CTAs, one 128-pixel block each
+    const bool pair = !split_n && pair_eligible(h, (int64_t)N * ((H + 15) / 16) * ((W + 15) / 16) * T);
+    if (pair) NB = 1;
     const int ACC = (2 * NB * NPAD <= 512) ? 2 : 1;
     const int TW = 8 * NB, BW = TW + d.kw - 1, BH = 16 + d.kh - 1;
+    const int TWT = pair ? 16 : TW;                        // tile width in the tile index space
     CUtensorMap tm_a, tm_o;
     ccv3d_status s = encode_ring_map(h, &tm_a, in, pl.KB, BW, BH, pl.KB == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B);
     if (s != CCV3D_OK) return s;
@@ -1020,7 +1130,7 @@ ccv3d_status forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int x_slot, int
     p.kt = d.kt; p.kh = d.kh; p.kw = d.kw;
     p.CB = pl.CB; p.NT = NT; p.NPAD = NPAD;
     p.tiles_h = (H + 15) / 16;
-    p.tiles_w = (W + TW - 1) / TW;
+    p.tiles_w = (W + TWT - 1) / TWT;
     const int64_t total = (int64_t)N * p.tiles_h * p.tiles_w * T * NT;
     if (total > 0x7FFFFFFF) return CCV3D_ERR_UNSUPPORTED;
     p.total_tiles = (int)total;
@@ -1028,7 +1138,7 @@ ccv3d_status forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int x_slot, int
     p.out_f32 = d.out_dtype == CCV3D_F32;
     p.ACC = ACC;
     p.a_slot = (uint32_t)align_up((uint64_t)BW * BH * pl.KB * 2, 1024);
-    p.b_tap = (uint32_t)NPAD * pl.KB * 2;
+    p.b_tap = (uint32_t)(pair ? NPAD / 2 : NPAD) * pl.KB * 2;   // a CTA of a pair holds half of every weight tile
     p.split_n = split_n;
     p.b_src_tap = split_n ? (uint32_t)pl.NPAD * pl.KB * 2 : 0;
     if (oring) {
@@ -1072,7 +1182,8 @@ ccv3d_status forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int x_slot, int
     p.out = out_ncthw;
     p.status = h->status;
     const size_t smem = fixed + (size_t)p.SA * p.a_slot + (size_t)p.SB * p.b_slot;
-    const int grid = p.total_tiles < h->sm_count ? p.total_tiles : h->sm_count;
+    int grid = p.total_tiles < h->sm_count ? p.total_tiles : h->sm_count;
+    if (pair) grid = 2 * (p.total_tiles < h->sm_count / 2 ? p.total_tiles : h->sm_count / 2);
     const int ks = (d.kh == d.kw && (d.kh == 1 || d.kh == 3)) ? d.kh : 0;
     cudaEvent_t* pev = (h->prof_on && h->prof_ev) ? h->prof_ev + 3 * (h->prof_n % PROF_SLOTS) : nullptr;
     if (pev) { cudaEventRecord(pev[0], st); cudaEventRecord(pev[1], st); }
@@ -1083,7 +1194,11 @@ ccv3d_status forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int x_slot, int
         else if (ks == 1) s = launch_tc_with_maps<KBv, NBv, 1, 1>(h, tm_a, tm_o, p, smem, grid, st);             \
         else s = launch_tc_with_maps<KBv, NBv, 0, 0>(h, tm_a, tm_o, p, smem, grid, st);                          \
     } while (0)
-    if (pl.KB == 64 && NB == 2) CCV3D_LAUNCH_RING(64, 2);
+    if (pair) {
+        StageParams nosp;
+        memset(&nosp, 0, sizeof(nosp));
+        s = launch_pair_any<false>(h, tm_a, tm_o, p, nosp, smem, grid, ks, st);
+    } else if (pl.KB == 64 && NB == 2) CCV3D_LAUNCH_RING(64, 2);
     else if (pl.KB == 64) CCV3D_LAUNCH_RING(64, 1);
     else if (NB == 2) CCV3D_LAUNCH_RING(32, 2);
     else CCV3D_LAUNCH_RING(32, 1);

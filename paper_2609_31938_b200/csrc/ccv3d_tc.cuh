@@ -493,6 +493,57 @@ __device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_
                  "l"(src), "r"(bytes), "r"(bar)
                  : "memory");
 }
+// ---- CTA pairs (cta_group::2): the two CTAs of a cluster run one 256-pixel tile, each holding its own 128-pixel
+// activation tile and half of the weight tile; the leader (cluster rank 0) issues the MMAs for both.
+constexpr uint32_t PEER_MASK = 0xFEFFFFFFu;   // clears the CTA-rank bit of a shared::cluster address: the leader's copy
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// TMA loads whose completion is counted on the LEADER's mbarrier (same offset, rank bit cleared)
+__device__ __forceinline__ void tma_load_5d_pair(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2,
+                                                 int c3, int c4) {
+    asm volatile(
+        "cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, "
+        "%4, %5, %6}], [%7];" ::"r"(dst),
+        "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar & PEER_MASK)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], "
+        "[%4];" ::"r"(dst),
+        "l"(tm), "r"(c0), "r"(c1), "r"(bar & PEER_MASK)
+        : "memory");
+}
+// an arrival on the leader's copy of a barrier, from either CTA of the pair
+__device__ __forceinline__ void mbar_arrive_leader(uint32_t bar) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar & PEER_MASK) : "memory");
+}
+// commit of the leader's MMAs: one arrival on the barrier at this offset in BOTH CTAs
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+                 "h"((unsigned short)3)
+                 : "memory");
+}
+// D[tmem of both CTAs] (+)= A * B^T with M = 256 (128 rows per CTA), each CTA contributing half of B's rows
+__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                                 uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "mov.b64 da, {%1, %2};\n\t"
+        "mov.b64 db, {%3, %4};\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %5, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
 // One lane of a fully converged warp; the others get 0.  Keeps the surrounding code warp-uniform so that
 // descriptors and addresses can live in uniform registers.
 __device__ __forceinline__ uint32_t elect_one() {
@@ -741,15 +792,23 @@ __device__ __forceinline__ uint32_t epi_pair(float a0, float a1, uint32_t res_pa
 // pass per term, the two small correction terms first: the tensor core's FP32 accumulation truncates, which
 // costs a fraction of the accumulator's last bit per step, so the long chain of full-size terms is kept as short
 // as it can be and the corrections are summed while the accumulator is still 2^-11 of its final size.
-template <int KB, int NB, int KS, int TPBC, bool FUSED, bool COOP, bool TF32 = false>
+// PAIR (cta_group::2): launched in clusters of two CTAs.  A tile is 16 rows x 16 pixels; CTA r of the pair loads
+// the halo tile of pixel columns 8r..8r+7 and rows r*NPAD/2.. of every weight tile (tm_c is then a 2-D map over the
+// packed weights); the leader issues MMAs with M = 256 that read both CTAs' shared memory and fill both CTAs'
+// tensor memory, so that per SM and MMA only half of the weight tile crosses L2 -> shared memory and the
+// shared-memory read port.  Loads of both CTAs are counted on the leader's "full" barriers; the leader's commits
+// arrive on the "empty" and "accumulator full" barriers of both CTAs; both epilogues arrive on the leader's
+// "accumulator empty" barrier.
+template <int KB, int NB, int KS, int TPBC, bool FUSED, bool COOP, bool TF32 = false, bool PAIR = false>
 __global__ void __launch_bounds__((FUSED || COOP) ? TC_THREADS_FUSED : TC_THREADS, 1)
 conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged activations (c, w, h, cb, n*F+f), or x
-                      const __grid_constant__ CUtensorMap tm_c,   // fused mode: the cache
+                      const __grid_constant__ CUtensorMap tm_c,   // fused mode: the cache; PAIR: the packed weights
                       const __grid_constant__ CUtensorMap tm_o,   // out (w, h, t, co, n); used when p.epi_tma
                       const TcParams p, const StageParams sp) {
     static_assert(!(FUSED && COOP), "one or the other");
     static_assert(!FUSED || KB == 32, "the fused mode transposes 32-channel blocks");
     static_assert(!TF32 || (KB == 64 && !FUSED && !COOP), "FP32 layers: 128-byte rows, plain variant");
+    static_assert(!PAIR || (NB == 1 && KS > 0 && !FUSED && !TF32), "CTA pairs: one pixel block per CTA, straight-line taps");
     // (TF32 layers always write FP32 through the direct-store epilogue, which is where the two accumulators of the
     // last pass are added)
     constexpr uint32_t ROWB = KB * 2;                       // bytes per pixel row (one swizzle span)
@@ -760,6 +819,11 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     constexpr int NI = (NB >= 2) ? 2 : 1;                   // MMA-issuing warps (2 and 3), each owning NB/NI pixel blocks
     constexpr int NBW = NB / NI;
     constexpr int ASETS = TF32 ? 2 : 1;                     // accumulators per tile buffer (TF32: the last pass uses two)
+    constexpr int TWT = PAIR ? 16 : TW;                     // tile width in the tile index space (a pair shares a tile)
+    const uint32_t rank = PAIR ? cluster_rank() : 0u;       // 0 = leader
+    const int cta_lin = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;   // tiles are dealt to clusters
+    const int cta_cnt = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+    const int wofs = PAIR ? 8 * (int)rank : 0;              // this CTA's pixel columns inside the tile
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -785,15 +849,23 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
         for (int i = 0; i < p.SA; ++i) { mbar_init(smem_u32(&sh->full_a[i]), FUSED ? 4 : 1); mbar_init(smem_u32(&sh->empty_a[i]), NI); }
         for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&sh->raw_full[i]), 1); mbar_init(smem_u32(&sh->raw_empty[i]), 4); }
         for (int i = 0; i < p.SB; ++i) { mbar_init(smem_u32(&sh->full_b[i]), 1); mbar_init(smem_u32(&sh->empty_b[i]), NI); }
-        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&sh->acc_full[i]), NI); mbar_init(smem_u32(&sh->acc_empty[i]), 4); }
+        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&sh->acc_full[i]), NI); mbar_init(smem_u32(&sh->acc_empty[i]), PAIR ? 8 : 4); }
         sh->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    if (PAIR) cluster_sync_all();   // both CTAs' barriers exist before anything of the peer can arrive on them
     if (warp == 3) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)),
-                     "r"(p.tmem_cols)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        if (PAIR) {
+            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)),
+                         "r"(p.tmem_cols)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+        } else {
+            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)),
+                         "r"(p.tmem_cols)
+                         : "memory");
+            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+        }
     }
     tc_fence_before();
     __syncthreads();
@@ -846,13 +918,13 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
             uint32_t phase = 1;
             bool ok = true;
             int bands_ready = 0;                       // COOP: bands [0, bands_ready) are known to be staged
-            for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+            for (int tile = cta_lin; ok && tile < p.total_tiles; tile += cta_cnt) {
                 int r = tile / p.NT;
                 const int t = r % p.T; r /= p.T;
                 const int tx = r % p.tiles_w; r /= p.tiles_w;
                 const int ty = p.ty_begin + r % p.tiles_h;
                 const int n = r / p.tiles_h;
-                const int h0 = ty * 16, w0 = tx * TW;
+                const int h0 = ty * 16, w0 = tx * TWT + wofs;
                 if (COOP) {
                     // the halo of tile row ty reaches into bands ty-1 .. ty+1
                     const int need = (ty + 2 < p.nbands) ? ty + 2 : p.nbands;
@@ -884,10 +956,16 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                         for (int tp = 0; tp < ntap; ++tp) {
                             if (!(ok = mbar_wait(&sh->empty_a[s], phase, sh, p, SITE_A_EMPTY))) break;
                             const uint32_t bar = smem_u32(&sh->full_a[s]);
-                            mbar_expect_tx(bar, a_bytes);
                             const int dh = p.per_tap_a ? tp / p.kw : 0, dw = p.per_tap_a ? tp % p.kw : 0;
-                            tma_load_5d(smem_u32(ring_a + (size_t)s * p.a_slot), &tm_a, bar, 0, w0 * stw - pw + dw * dlw,
-                                        h0 * sth - ph + dh * dlh, TF32 ? 2 * cb + (pass == 1) : cb, fz);
+                            if (PAIR) {
+                                // both CTAs' boxes are counted on the leader's barrier, which the leader arms for both
+                                if (rank == 0) mbar_expect_tx(bar, 2 * a_bytes);
+                                tma_load_5d_pair(smem_u32(ring_a + (size_t)s * p.a_slot), &tm_a, bar, 0, w0 - pw, h0 - ph, cb, fz);
+                            } else {
+                                mbar_expect_tx(bar, a_bytes);
+                                tma_load_5d(smem_u32(ring_a + (size_t)s * p.a_slot), &tm_a, bar, 0, w0 * stw - pw + dw * dlw,
+                                            h0 * sth - ph + dh * dlh, TF32 ? 2 * cb + (pass == 1) : cb, fz);
+                            }
                             if (++s == p.SA) { s = 0; phase ^= 1; }
                         }
                     }
@@ -903,13 +981,28 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
             int s = 0;
             uint32_t phase = 1;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+            if (PAIR) asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_c) : "memory");
+            for (int tile = cta_lin; ok && tile < p.total_tiles; tile += cta_cnt) {
                 const int nt = tile % p.NT;
                 const int t = (tile / p.NT) % p.T;
                 const int dt0 = (p.first_frame - t * stt > 0) ? (p.first_frame - t * stt + dlt - 1) / dlt : 0;   // first tap whose frame exists
                 for (int pass = 0; pass < (TF32 ? 3 : 1); ++pass)
                 for (int dt = dt0; ok && dt < p.kt; ++dt)
                     for (int cb = 0; ok && cb < p.CB; ++cb) {
+                        if (PAIR) {
+                            // this CTA's half (rows rank*NPAD/2 ..) of every tap's weight tile, as boxes of the 2-D map
+                            // over the packed weights; both CTAs' boxes are counted on the leader's barrier
+                            const int row0 = (((dt * p.CB + cb) * p.NT + nt) * spatial) * p.NPAD + (int)rank * (p.NPAD >> 1);
+                            for (int tp = 0; tp < spatial; tp += p.TPB) {
+                                if (!(ok = mbar_wait(&sh->empty_b[s], phase, sh, p, SITE_B_EMPTY))) break;
+                                const uint32_t bar = smem_u32(&sh->full_b[s]);
+                                if (rank == 0) mbar_expect_tx(bar, 2 * b_bytes);
+                                const uint32_t dst = smem_u32(ring_b + (size_t)s * p.b_slot);
+                                for (int u = 0; u < p.TPB; ++u) tma_load_2d_pair(dst + u * p.b_tap, &tm_c, bar, 0, row0 + (tp + u) * p.NPAD);
+                                if (++s == p.SB) { s = 0; phase ^= 1; }
+                            }
+                            continue;
+                        }
                         // split_n: this launch runs half-width output-channel tiles; the packed image of a full tile
                         // holds its two halves back to back (the swizzle repeats every 8 rows), so a half tile of a
                         // tap is a contiguous piece of it and only the distance between taps differs
@@ -934,13 +1027,13 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     // Warp 2 (and warp 3 when NB >= 2) issues the MMAs of its own pixel blocks.  A commit
     // only tracks the MMAs of the committing thread, so the "slot free" and "accumulator full" barriers
     // count one arrival per issuer.
-    else if (warp == 2 || (warp == 3 && NI == 2)) {
+    else if ((warp == 2 || (warp == 3 && NI == 2)) && rank == 0) {     // (of a CTA pair only the leader issues MMAs)
         // The whole warp runs the loop (warp-uniform control flow); one elected lane issues.
         const int iss = warp - 2;
         // instruction descriptor: D=F32, A=B=BF16, both K-major, N = NPAD, M = 128
         // (operand formats: 1 = BF16, 2 = TF32)
         constexpr uint32_t FMT = TF32 ? 2u : 1u;
-        const uint32_t idesc = (1u << 4) | (FMT << 7) | (FMT << 10) | ((uint32_t)(p.NPAD >> 3) << 17) | ((128u >> 4) << 24);
+        const uint32_t idesc = (1u << 4) | (FMT << 7) | (FMT << 10) | ((uint32_t)(p.NPAD >> 3) << 17) | (((PAIR ? 256u : 128u) >> 4) << 24);
         const uint32_t a_hi = make_desc_hi((uint32_t)BW * ROWB, LAYOUT);  // 8-pixel groups are one image row apart
         const uint32_t b_hi = make_desc_hi(B_SBO, LAYOUT);
         const uint32_t a_blk = (uint32_t)(iss * NBW) * ((8 * ROWB) >> 4);  // descriptor offset of this issuer's first block
@@ -955,7 +1048,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
             uint32_t a_ring = make_desc_lo(smem_u32(ring_a)) + a_blk, b_ring = make_desc_lo(smem_u32(ring_b));
             const uint32_t a_slotstep = p.a_slot >> 4, b_slotstep = p.b_slot >> 4;
             const uint32_t a_ring0 = a_ring, b_ring0 = b_ring;
-            for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+            for (int tile = cta_lin; ok && tile < p.total_tiles; tile += cta_cnt) {
                 const int t = (tile / p.NT) % p.T;
                 const int dt0 = (p.first_frame - t * stt > 0) ? (p.first_frame - t * stt + dlt - 1) / dlt : 0;   // first tap whose frame exists
                 if (!(ok = mbar_wait(&sh->acc_empty[acc], pacc, sh, p, SITE_ACC_EMPTY))) break;
@@ -988,11 +1081,15 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                                 for (int j = 0; j < NBW; ++j) {
 #pragma unroll
                                     for (int k = 0; k < KSTEPS; ++k)
-                                        tc_mma<TF32>(d0 + j * p.NPAD, a_lo + j * ((8 * ROWB) >> 4) + 2 * k, a_hi, b_lo + 2 * k, b_hi,
-                                                    idesc, (tap == 0 && k == 0) ? acc_in : 1u);
+                                        if (PAIR)
+                                            tc_mma_bf16_pair(d0 + j * p.NPAD, a_lo + j * ((8 * ROWB) >> 4) + 2 * k, a_hi, b_lo + 2 * k, b_hi,
+                                                             idesc, (tap == 0 && k == 0) ? acc_in : 1u);
+                                        else
+                                            tc_mma<TF32>(d0 + j * p.NPAD, a_lo + j * ((8 * ROWB) >> 4) + 2 * k, a_hi, b_lo + 2 * k, b_hi,
+                                                         idesc, (tap == 0 && k == 0) ? acc_in : 1u);
                                 }
                             }
-                            tc_commit(smem_u32(&sh->empty_b[sb]));
+                            if (PAIR) tc_commit_pair(smem_u32(&sh->empty_b[sb])); else tc_commit(smem_u32(&sh->empty_b[sb]));
                         }
                         __syncwarp();
                         b_ring += b_slotstep;
@@ -1000,13 +1097,13 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                     }
                     if (!ok) break;
                     if (second) accumulate2 = 1; else accumulate = 1;
-                    if (elect_one()) tc_commit(smem_u32(&sh->empty_a[sa]));
+                    if (elect_one()) { if (PAIR) tc_commit_pair(smem_u32(&sh->empty_a[sa])); else tc_commit(smem_u32(&sh->empty_a[sa])); }
                     __syncwarp();
                     a_ring += a_slotstep;
                     if (++sa == p.SA) { sa = 0; pa ^= 1; a_ring = a_ring0; }
                 }
                 if (!ok) break;
-                if (elect_one()) tc_commit(smem_u32(&sh->acc_full[acc]));
+                if (elect_one()) { if (PAIR) tc_commit_pair(smem_u32(&sh->acc_full[acc])); else tc_commit(smem_u32(&sh->acc_full[acc])); }
                 __syncwarp();
                 if (++acc == p.ACC) { acc = 0; pacc ^= 1; }
             }
@@ -1102,7 +1199,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
             for (int i = threadIdx.x - 128; i < p.NT * p.NPAD; i += 128) sh->bias_s[i] = __ldg(p.bias + i);
         epi_bar_sync();
         const float* bias = bias_smem ? sh->bias_s : p.bias;
-        for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+        for (int tile = cta_lin; ok && tile < p.total_tiles; tile += cta_cnt) {
             const int nt = tile % p.NT;
             int r = tile / p.NT;
             const int t = r % p.T; r /= p.T;
@@ -1110,6 +1207,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
             const int ty = p.ty_begin + r % p.tiles_h;
             const int n = r / p.tiles_h;
             const int h = ty * 16 + (m >> 3);
+            const int wt = tx * TWT + wofs;                  // first pixel column of this CTA's part of the tile
             // residual: pixel (h, w) of frame t holds its Cout channels in blocks of res_KB (64 bytes per 32 channels)
             const __nv_bfloat16* res_row = nullptr;
             if (has_res && h < p.H) {
@@ -1120,7 +1218,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
             // the residual of the first chunk is fetched while the MMAs of this tile still run; every later chunk's
             // residual is fetched one chunk ahead
             uint32_t rr_next[16];
-            if (p.epi_tma) load_res32(res_row, tx * TW + (m & 7) < p.W, tx * TW + (m & 7), nt * p.NPAD, p, HW, rr_next);
+            if (p.epi_tma) load_res32(res_row, wt + (m & 7) < p.W, wt + (m & 7), nt * p.NPAD, p, HW, rr_next);
             ok = mbar_wait(&sh->acc_full[acc], pacc, sh, p, SITE_ACC_FULL);
             ok = __all_sync(0xffffffffu, ok);
             if (!ok) break;
@@ -1143,7 +1241,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
 #pragma unroll
                         for (int j = 0; j < 16; ++j) rr[j] = rr_next[j];
                         if (has_res) {
-                            const int wn = tx * TW + ((blk + 1 < NB) ? blk + 1 : 0) * 8 + (m & 7);
+                            const int wn = wt + ((blk + 1 < NB) ? blk + 1 : 0) * 8 + (m & 7);
                             const int con = (blk + 1 < NB) ? co0 : co0 + p.ECH;
                             load_res32(res_row, wn < p.W && con < (nt + 1) * p.NPAD, wn, con, p, HW, rr_next);
                         }
@@ -1189,15 +1287,15 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                             for (int j = 0; j < p.up_rt; ++j) {
                                 const int os = (p.out_f0 + t * p.up_rt + j) % p.out_F;
                                 for (int ab = 0; ab < 4; ++ab)
-                                    tma_store_5d(&tm_o, smem_u32(stg), co0 % p.out_KB, 2 * tx * TW + (ab & 1), 2 * ty * 16 + (ab >> 1),
+                                    tma_store_5d(&tm_o, smem_u32(stg), co0 % p.out_KB, 2 * wt + (ab & 1), 2 * ty * 16 + (ab >> 1),
                                                  co0 / p.out_KB, n * p.out_F + os);
                             }
                         } else if (RING && p.epi_tma == 2) {
                             int os = p.out_f0 + t;
                             if (os >= p.out_F) os -= p.out_F;
-                            tma_store_5d(&tm_o, smem_u32(stg), co0 % p.out_KB, tx * TW, ty * 16, co0 / p.out_KB, n * p.out_F + os);
+                            tma_store_5d(&tm_o, smem_u32(stg), co0 % p.out_KB, wt, ty * 16, co0 / p.out_KB, n * p.out_F + os);
                         } else {
-                            tma_store_5d(&tm_o, smem_u32(stg), tx * TW, ty * 16, t, co0, n);
+                            tma_store_5d(&tm_o, smem_u32(stg), wt, ty * 16, t, co0, n);
                         }
                         bulk_commit();
                     }
@@ -1206,7 +1304,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
             } else {
 #pragma unroll 1
                 for (int blk = 0; blk < NB; ++blk) {
-                    const int w = tx * TW + blk * 8 + (m & 7);
+                    const int w = wt + blk * 8 + (m & 7);
                     const bool valid = h < p.H && w < p.W;
                     const int64_t pix = (int64_t)t * HW + (int64_t)h * p.W + w;
 #pragma unroll 1
@@ -1255,7 +1353,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
             }
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&sh->acc_empty[acc]));
+            if (lane == 0) { if (PAIR) mbar_arrive_leader(smem_u32(&sh->acc_empty[acc])); else mbar_arrive(smem_u32(&sh->acc_empty[acc])); }
             if (++acc == p.ACC) { acc = 0; pacc ^= 1; }
         }
         if (p.epi_tma && elected) bulk_wait_all();   // all stores of this CTA are complete before it exits
@@ -1364,9 +1462,11 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     // ---------------------------------------------------------------- teardown
     tc_fence_before();
     __syncthreads();
+    if (PAIR) cluster_sync_all();   // the leader's MMAs read the peer's shared memory and write its tensor memory
     if (warp == 3) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
+        if (PAIR) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
+        else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
     }
 }
 

@@ -390,3 +390,30 @@ def test_chain_glue_kernels(ccv, shape, rt):
     assert _guards_intact(ybuf) and _guards_intact(ubuf), "glue kernel wrote outside its output"
     exp_up = np.repeat(np.repeat(np.repeat(a, rt, axis=2), 2, axis=3), 2, axis=4)
     assert np.array_equal(bits(up), exp_up)
+
+
+# ---------------------------------------------------------------------------- CTA pairs (cta_group::2)
+@pytest.mark.parametrize("Cin,Cout,T,H,W,k,flags", [
+    (64, 192, 4, 160, 256, (3, 3, 3), 0),                      # cooperative staging on CTA pairs (640 pair tiles)
+    (64, 192, 2, 90, 100, (3, 3, 3), 0),                       # two kernels; ragged: the second CTA's columns partly outside
+    (96, 160, 2, 70, 72, (3, 3, 3), 16),                       # 32-channel blocks, forced two-kernel schedule
+    (128, 384, 1, 96, 96, (3, 3, 3), 0),                       # two output-channel tiles of 192
+    (96, 256, 3, 48, 80, (1, 1, 1), 0),                        # a 1x1x1 layer the streaming kernel does not take (Cin % 64 != 0)
+])
+def test_cta_pairs_match_the_oracle_and_the_single_cta_kernel(ccv, Cin, Cout, T, H, W, k, flags):
+    """Layers with more than 128 output channels per tile run on pairs of CTAs (MMAs with M = 256 issued by the
+    leader, each CTA holding half of every weight tile): within tolerance of the oracle, cache bit-exact, and bit
+    for bit what the single-CTA kernel computes (the K order of an output element is the same)."""
+    c = si.conv_case(1, Cin, Cout, T, H, W, k=k, seed=51)
+    m, ctr = run_case(ccv, c, flags=flags)
+    assert ctr["tcgen05_bf16"] == 1
+    a = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), flags=flags)
+    b = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), flags=flags | ccv.FLAG_NO_PAIR)
+    x, cache = to_dev(c["x"]), to_dev(c["cache"])
+    oa, na = a(x, cache)
+    ob, nb = b(x, cache)
+    torch.cuda.synchronize()
+    assert a.device_status()[0] == ccv.OK and b.device_status()[0] == ccv.OK
+    assert torch.equal(oa, ob) and (na is None or torch.equal(na, nb))
+    a.close()
+    b.close()

@@ -175,6 +175,33 @@ def test_upsample_fused_into_the_store_equals_store_then_upsample(ccv, Cin, Cout
     layer.close()
 
 
+def test_cta_pairs_on_rings(ccv):
+    """192 output channels and enough tiles: the ring calls run on CTA pairs.  Output into a ring, into NCTHW, with
+    the residual epilogue and with the upsample fused into the store - each bit for bit what the single-CTA kernel
+    writes."""
+    c = si.conv_case(1, 192, 192, 2, 90, 100, seed=26)
+    x, cache = to_dev(c["x"]), to_dev(c["cache"])
+    got = {}
+    for flags in (0, ccv.FLAG_NO_PAIR):
+        layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), flags=flags)
+        rin = ccv.FrameRing(1, 192, 4, 90, 100)
+        rin.load(0, cache)
+        rin.load(2, x)
+        r1, r2 = ccv.FrameRing(1, 192, 2, 90, 100, zero=True), ccv.FrameRing(1, 192, 2, 180, 200, zero=True)
+        out = torch.zeros((1, 192, 2, 90, 100), dtype=torch.bfloat16, device="cuda")
+        layer.forward_ring(rin, 2, 2, 2, out_ring=r1, res=rin, res_slot=2)
+        layer.forward_ring(rin, 2, 2, 2, out=out)
+        layer.forward_ring(rin, 2, 2, 2, out_ring=r2, up_rt=1)
+        torch.cuda.synchronize()
+        assert layer.device_status()[0] == ccv.OK
+        got[flags] = (r1.buf.clone(), out.clone(), r2.buf.clone())
+        layer.close()
+    for a, b in zip(got[0], got[ccv.FLAG_NO_PAIR]):
+        assert torch.equal(a, b)
+    ref, _ = oracle.forward(c["x"], c["cache"], c["w"], c["b"])
+    check(as_f64(got[0][1]), ref, "bf16")
+
+
 def test_ring_argument_errors(ccv):
     c = si.conv_case(1, 64, 64, 2, 16, 16, seed=23)
     layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]))
