@@ -317,10 +317,10 @@ ccv3d_status launch_stage(ccv3d_handle* h, StageParams sp, int h0, int h1, int n
 
 // CTA pairs: clusters of two CTAs, one 16x16-pixel tile per cluster (see the kernel).  tm_w is the 2-D map over the
 // packed weights from which each CTA takes its half of every tap's tile.
-template <int KB, int KS, int TPBC, bool COOP>
+template <int KB, int NB, int KS, int TPBC, bool COOP>
 ccv3d_status launch_tc_pair(ccv3d_handle* h, const CUtensorMap& tm_a, const CUtensorMap& tm_w, const CUtensorMap& tm_o,
                             const TcParams& p, const StageParams& sp, size_t smem, int grid, cudaStream_t st) {
-    auto kern = conv3d_tcgen05_kernel<KB, 1, KS, TPBC, false, COOP, false, true>;
+    auto kern = conv3d_tcgen05_kernel<KB, NB, KS, TPBC, false, COOP, false, true>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return cuda_fail();
     cudaLaunchConfig_t cfg;
@@ -368,31 +368,34 @@ ccv3d_status weight_map(ccv3d_handle* h, const CUtensorMap** out) {
 // Dispatch over the compiled pair variants (straight-line taps only: ks = 3 or 1).
 template <bool COOP>
 ccv3d_status launch_pair_any(ccv3d_handle* h, const CUtensorMap& tm_a, const CUtensorMap& tm_o, const TcParams& p,
-                             const StageParams& sp, size_t smem, int grid, int ks, cudaStream_t st) {
+                             const StageParams& sp, size_t smem, int grid, int ks, int nb, cudaStream_t st) {
     const CUtensorMap* tm_w = nullptr;
     ccv3d_status s = weight_map(h, &tm_w);
     if (s != CCV3D_OK) return s;
-    if (h->plan.KB == 64) {
-        if (ks == 3 && p.TPB == 3) return launch_tc_pair<64, 3, 3, COOP>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
-        if (ks == 3) return launch_tc_pair<64, 3, 1, COOP>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
-        return launch_tc_pair<64, 1, 1, COOP>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
-    }
-    if (ks == 3 && p.TPB == 3) return launch_tc_pair<32, 3, 3, COOP>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
-    if (ks == 3) return launch_tc_pair<32, 3, 1, COOP>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
-    return launch_tc_pair<32, 1, 1, COOP>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
+#define CCV3D_LAUNCH_PAIR(KBv, NBv)                                                                                        \
+    do {                                                                                                                   \
+        if (ks == 3 && p.TPB == 3) return launch_tc_pair<KBv, NBv, 3, 3, COOP>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st); \
+        if (ks == 3) return launch_tc_pair<KBv, NBv, 3, 1, COOP>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);              \
+        return launch_tc_pair<KBv, NBv, 1, 1, COOP>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);                           \
+    } while (0)
+    if (h->plan.KB == 64 && nb == 2) CCV3D_LAUNCH_PAIR(64, 2);
+    else if (h->plan.KB == 64) CCV3D_LAUNCH_PAIR(64, 1);
+    else if (nb == 2) CCV3D_LAUNCH_PAIR(32, 2);
+    else CCV3D_LAUNCH_PAIR(32, 1);
+#undef CCV3D_LAUNCH_PAIR
 }
 
-// A layer runs on CTA pairs when its output-channel tile is wide (more than 128 channels: one 128-pixel block per
-// CTA anyway, and the MMAs long enough for one issuing thread to feed two SMs), its taps are the straight-line
-// kind, and there are tiles for at least half of the pairs.
+// A layer runs on CTA pairs (every SM then reads half of each weight tile from L2 and from its shared memory) when
+// its taps are the straight-line kind and there are tiles for at least a quarter of the pairs.  `pair_tiles` counts
+// tiles of 16 rows x 16*NB pixels.
 bool pair_eligible(const ccv3d_handle* h, int64_t pair_tiles) {
     const ccv3d_desc& d = h->d;
     const TcPlan& pl = h->plan;
     if (d.flags & CCV3D_FLAG_NO_PAIR) return false;
     if (d.dtype != CCV3D_BF16 || (d.flags & CCV3D_FLAG_TC_PER_TAP_A)) return false;
     if (d.stride[1] != 1 || d.stride[2] != 1 || d.dilation[1] != 1 || d.dilation[2] != 1) return false;
-    if (d.kh != d.kw || (d.kh != 1 && d.kh != 3)) return false;
-    if (pl.NB != 1 || pl.NPAD % 16 != 0 || h->sm_count < 2) return false;
+    if (d.kh != 3 || d.kw != 3) return false;              // (1x1 layers are bound by their epilogue; pairs make them slower)
+    if (pl.NPAD % 16 != 0 || h->sm_count < 2) return false;
     return pair_tiles * pl.NT >= h->sm_count / 4;
 }
 
@@ -477,10 +480,10 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     const int ACC = (2 * asets * NB * NPAD <= 512) ? 2 : 1;
     // CTA pairs (wide output-channel tiles): 16x16-pixel tiles shared by the two CTAs of a cluster; not combined with
     // the banded multi-stream schedule
-    const bool pair = !split_n && !per_tap && !f32 && !(d.flags & CCV3D_FLAG_OVERLAP) &&
-                      pair_eligible(h, (int64_t)N * ((Ho + 15) / 16) * ((Wo + 15) / 16) * To);
-    const int TW = 8 * NB;                                 // pixels per row of a CTA's part of a tile (pair: NB is 1)
-    const int TWT = pair ? 16 : TW;                        // tile width in the tile index space
+    const bool pair = !split_n && !per_tap && !f32 && !(d.flags & CCV3D_FLAG_OVERLAP) && NB == pl.NB &&
+                      pair_eligible(h, (int64_t)N * ((Ho + 15) / 16) * ((Wo + 16 * NB - 1) / (16 * NB)) * To);
+    const int TW = 8 * NB;                                 // pixels per row of a CTA's part of a tile
+    const int TWT = pair ? 2 * TW : TW;                    // tile width in the tile index space
     const int BW = per_tap ? TW : TW + (d.kw - 1) * d.dilation[2];
     const int BH = per_tap ? 16 : 16 + (d.kh - 1) * d.dilation[1];
     ShapeKey key{h->workspace, N, T, H, W, BW};
@@ -528,7 +531,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     // extra warps per CTA, one band of 16 rows ahead of the tiles that read it.
     const bool coop = nbands == 1 && !per_tap && !general && !f32 && !(d.flags & CCV3D_FLAG_TWO_KERNELS) && W % 8 == 0 &&
                       tiles_h <= MAX_COOP_BANDS && tiles_h >= 4 &&
-                      (int64_t)N * tiles_h * p.tiles_w * To * NT >= 4LL * h->sm_count;   // small problems: two kernels
+                      (int64_t)N * tiles_h * p.tiles_w * To * NT * (pair ? 2 : 1) >= 4LL * h->sm_count;   // small problems: two kernels
     size_t fixed = 1024 /*alignment slack*/ + align_up(sizeof(TcShared), 128) + 2 * (size_t)p.e_slot + (coop ? 9216 : 0);
     // leave room for staging blocks to be resident next to a convolution CTA when the two overlap
     const size_t limit = nbands > 1 ? SMEM_LIMIT - STAGE_COEXIST_BYTES : SMEM_LIMIT;
@@ -568,7 +571,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
         int grid = p.total_tiles < h->sm_count ? p.total_tiles : h->sm_count;
         if (pair) {
             grid = 2 * (p.total_tiles < h->sm_count / 2 ? p.total_tiles : h->sm_count / 2);
-            s = launch_pair_any<true>(h, h->tm_a, h->tm_o, p, sp, smem, grid, ks, st);
+            s = launch_pair_any<true>(h, h->tm_a, h->tm_o, p, sp, smem, grid, ks, NB, st);
             if (s != CCV3D_OK) return s;
         } else {
 #define CCV3D_LAUNCH_COOP(KBv, NBv)                                                                        \
@@ -612,7 +615,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
             const int grid = 2 * (p.total_tiles < h->sm_count / 2 ? p.total_tiles : h->sm_count / 2);
             StageParams nosp;
             memset(&nosp, 0, sizeof(nosp));
-            s = launch_pair_any<false>(h, h->tm_a, h->tm_o, p, nosp, smem, grid, ks, st);
+            s = launch_pair_any<false>(h, h->tm_a, h->tm_o, p, nosp, smem, grid, ks, NB, st);
         } else {
             s = launch_conv(h, p, NB, 0, tiles_h, smem, ks, st);
         }
@@ -1113,11 +1116,11 @@ ccv3d_status forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int x_slot, int
         split_n = 1; NT = 2 * pl.NT; NPAD = pl.NPAD / 2;
     }
     // CTA pairs: 16x16-pixel tiles shared by two CTAs, one 128-pixel block each
-    const bool pair = !split_n && pair_eligible(h, (int64_t)N * ((H + 15) / 16) * ((W + 15) / 16) * T);
-    if (pair) NB = 1;
+    const bool pair = !split_n && NB == pl.NB &&
+                      pair_eligible(h, (int64_t)N * ((H + 15) / 16) * ((W + 16 * NB - 1) / (16 * NB)) * T);
     const int ACC = (2 * NB * NPAD <= 512) ? 2 : 1;
     const int TW = 8 * NB, BW = TW + d.kw - 1, BH = 16 + d.kh - 1;
-    const int TWT = pair ? 16 : TW;                        // tile width in the tile index space
+    const int TWT = pair ? 2 * TW : TW;                    // tile width in the tile index space
     CUtensorMap tm_a, tm_o;
     ccv3d_status s = encode_ring_map(h, &tm_a, in, pl.KB, BW, BH, pl.KB == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B);
     if (s != CCV3D_OK) return s;
@@ -1197,7 +1200,7 @@ ccv3d_status forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int x_slot, int
     if (pair) {
         StageParams nosp;
         memset(&nosp, 0, sizeof(nosp));
-        s = launch_pair_any<false>(h, tm_a, tm_o, p, nosp, smem, grid, ks, st);
+        s = launch_pair_any<false>(h, tm_a, tm_o, p, nosp, smem, grid, ks, NB, st);
     } else if (pl.KB == 64 && NB == 2) CCV3D_LAUNCH_RING(64, 2);
     else if (pl.KB == 64) CCV3D_LAUNCH_RING(64, 1);
     else if (NB == 2) CCV3D_LAUNCH_RING(32, 2);

@@ -792,8 +792,8 @@ __device__ __forceinline__ uint32_t epi_pair(float a0, float a1, uint32_t res_pa
 // pass per term, the two small correction terms first: the tensor core's FP32 accumulation truncates, which
 // costs a fraction of the accumulator's last bit per step, so the long chain of full-size terms is kept as short
 // as it can be and the corrections are summed while the accumulator is still 2^-11 of its final size.
-// PAIR (cta_group::2): launched in clusters of two CTAs.  A tile is 16 rows x 16 pixels; CTA r of the pair loads
-// the halo tile of pixel columns 8r..8r+7 and rows r*NPAD/2.. of every weight tile (tm_c is then a 2-D map over the
+// PAIR (cta_group::2): launched in clusters of two CTAs.  A tile is 16 rows x 16*NB pixels; CTA r of the pair loads
+// the halo tile of pixel columns 8*NB*r .. and rows r*NPAD/2.. of every weight tile (tm_c is then a 2-D map over the
 // packed weights); the leader issues MMAs with M = 256 that read both CTAs' shared memory and fill both CTAs'
 // tensor memory, so that per SM and MMA only half of the weight tile crosses L2 -> shared memory and the
 // shared-memory read port.  Loads of both CTAs are counted on the leader's "full" barriers; the leader's commits
@@ -808,7 +808,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     static_assert(!(FUSED && COOP), "one or the other");
     static_assert(!FUSED || KB == 32, "the fused mode transposes 32-channel blocks");
     static_assert(!TF32 || (KB == 64 && !FUSED && !COOP), "FP32 layers: 128-byte rows, plain variant");
-    static_assert(!PAIR || (NB == 1 && KS > 0 && !FUSED && !TF32), "CTA pairs: one pixel block per CTA, straight-line taps");
+    static_assert(!PAIR || (KS > 0 && !FUSED && !TF32), "CTA pairs: straight-line taps, BF16");
     // (TF32 layers always write FP32 through the direct-store epilogue, which is where the two accumulators of the
     // last pass are added)
     constexpr uint32_t ROWB = KB * 2;                       // bytes per pixel row (one swizzle span)
@@ -819,11 +819,11 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     constexpr int NI = (NB >= 2) ? 2 : 1;                   // MMA-issuing warps (2 and 3), each owning NB/NI pixel blocks
     constexpr int NBW = NB / NI;
     constexpr int ASETS = TF32 ? 2 : 1;                     // accumulators per tile buffer (TF32: the last pass uses two)
-    constexpr int TWT = PAIR ? 16 : TW;                     // tile width in the tile index space (a pair shares a tile)
+    constexpr int TWT = PAIR ? 2 * TW : TW;                 // tile width in the tile index space (a pair shares a tile)
     const uint32_t rank = PAIR ? cluster_rank() : 0u;       // 0 = leader
     const int cta_lin = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;   // tiles are dealt to clusters
     const int cta_cnt = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
-    const int wofs = PAIR ? 8 * (int)rank : 0;              // this CTA's pixel columns inside the tile
+    const int wofs = PAIR ? TW * (int)rank : 0;             // this CTA's pixel columns inside the tile
 
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));

@@ -398,7 +398,7 @@ def test_chain_glue_kernels(ccv, shape, rt):
     (64, 192, 2, 90, 100, (3, 3, 3), 0),                       # two kernels; ragged: the second CTA's columns partly outside
     (96, 160, 2, 70, 72, (3, 3, 3), 16),                       # 32-channel blocks, forced two-kernel schedule
     (128, 384, 1, 96, 96, (3, 3, 3), 0),                       # two output-channel tiles of 192
-    (96, 256, 3, 48, 80, (1, 1, 1), 0),                        # a 1x1x1 layer the streaming kernel does not take (Cin % 64 != 0)
+    (96, 96, 4, 96, 128, (3, 3, 3), 0),                        # narrow output tile: two pixel blocks per CTA, 16x32-pixel tiles
 ])
 def test_cta_pairs_match_the_oracle_and_the_single_cta_kernel(ccv, Cin, Cout, T, H, W, k, flags):
     """Layers with more than 128 output channels per tile run on pairs of CTAs (MMAs with M = 256 issued by the
