@@ -35,12 +35,12 @@ METRIC = "causal Conv3D BF16 TFLOP/s"
 DEFAULT_WORKLOAD = "cfg3_bf16_192"
 
 # DRAM bytes (read + write) of one launch of the step's kernel (default schedule: staging, cache update and
-# convolution in one kernel), from an ncu capture of a quarter-size case (192->192, T=4, 176x320: 241.4 MB read +
-# 222.6 MB written) scaled by the pixel count; the summary is profiles/conv3d_tcgen05_coop_192ch_176x320.md.
-TRAFFIC_BYTES_PER_LAUNCH = {"cfg3_bf16_192": 4 * (241.4e6 + 222.6e6)}
-# The same for the kernel on frame rings (profiles/conv3d_tcgen05_ring_192ch_176x320.md: 131.9 MB read + 51.3 MB
+# convolution in one kernel), from an ncu capture of a quarter-size case (192->192, T=4, 176x320: 239.4 MB read +
+# 224.6 MB written) scaled by the pixel count; the summary is profiles/conv3d_tcgen05_coop_192ch_176x320.md.
+TRAFFIC_BYTES_PER_LAUNCH = {"cfg3_bf16_192": 4 * (239.4e6 + 224.6e6)}
+# The same for the kernel on frame rings (profiles/conv3d_tcgen05_ring_192ch_176x320.md: 132.0 MB read + 53.6 MB
 # written during the kernel, the rest of the 86.5 MB output still in L2 when it ends).
-TRAFFIC_BYTES_PER_LAUNCH_RESIDENT = {"cfg3_bf16_192": 4 * (131.9e6 + 51.3e6)}
+TRAFFIC_BYTES_PER_LAUNCH_RESIDENT = {"cfg3_bf16_192": 4 * (132.0e6 + 53.6e6)}
 
 
 def measured_peaks():
