@@ -67,8 +67,8 @@ struct ccv3d_handle {
     CUtensorMap tm_a;
     ShapeKey tm_a_key;
     CUtensorMap tm_o;
-    CUtensorMap tm_w;    // CTA pairs: 2-D map over the packed weights (half-tile boxes)
-    bool tm_w_ready;
+    CUtensorMap tm_w[2]; // CTA pairs: 2-D maps over the packed weights (half-tile and quarter-tile boxes)
+    int tm_w_rows[2];    // box height each was encoded for (0 = not yet)
     long long wait_limit_clk;
     // side streams and events of the banded, overlapped schedule (created with the handle)
     cudaStream_t side[3];
@@ -343,11 +343,12 @@ ccv3d_status launch_tc_pair(ccv3d_handle* h, const CUtensorMap& tm_a, const CUte
 }
 
 // 2-D map over the packed weights: rows of KB channels (one swizzle span), all tiles of all taps one after another;
-// a box is half a tile (NPAD/2 rows).  Encoded once per handle.
-ccv3d_status weight_map(ccv3d_handle* h, const CUtensorMap** out) {
-    if (h->tm_w_ready) { *out = &h->tm_w; return CCV3D_OK; }
-    CUtensorMap* tm = &h->tm_w;
-    const int box_rows = h->plan.NPAD / 2;
+// a box is one CTA's share of a tile: half of it, or a quarter when the launch runs half-width tiles.  Encoded once
+// per handle and box height.
+ccv3d_status weight_map(ccv3d_handle* h, int box_rows, const CUtensorMap** out) {
+    const int slot = (box_rows == h->plan.NPAD / 2) ? 0 : 1;
+    if (h->tm_w_rows[slot] == box_rows) { *out = &h->tm_w[slot]; return CCV3D_OK; }
+    CUtensorMap* tm = &h->tm_w[slot];
     const TcPlan& pl = h->plan;
     const ccv3d_desc& d = h->d;
     const uint64_t rows = (uint64_t)d.kt * pl.CB * pl.NT * d.kh * d.kw * pl.NPAD;
@@ -355,12 +356,12 @@ ccv3d_status weight_map(ccv3d_handle* h, const CUtensorMap** out) {
     cuuint64_t strides[1] = {(cuuint64_t)pl.KB * 2};
     cuuint32_t box[2] = {(cuuint32_t)pl.KB, (cuuint32_t)box_rows};
     cuuint32_t es[2] = {1, 1};
-    if (rows > 0x7FFFFFFFull || box_rows > 256) return CCV3D_ERR_UNSUPPORTED;
+    if (rows > 0x7FFFFFFFull || box_rows > 256 || box_rows % 8) return CCV3D_ERR_UNSUPPORTED;
     CUresult rc = h->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, h->wp, dims, strides, box, es,
                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (rc != CUDA_SUCCESS) return CCV3D_ERR_CUDA;
-    h->tm_w_ready = true;
+    h->tm_w_rows[slot] = box_rows;
     *out = tm;
     return CCV3D_OK;
 }
@@ -370,7 +371,7 @@ template <bool COOP>
 ccv3d_status launch_pair_any(ccv3d_handle* h, const CUtensorMap& tm_a, const CUtensorMap& tm_o, const TcParams& p,
                              const StageParams& sp, size_t smem, int grid, int ks, int nb, cudaStream_t st) {
     const CUtensorMap* tm_w = nullptr;
-    ccv3d_status s = weight_map(h, &tm_w);
+    ccv3d_status s = weight_map(h, p.NPAD / 2, &tm_w);
     if (s != CCV3D_OK) return s;
 #define CCV3D_LAUNCH_PAIR(KBv, NBv)                                                                                        \
     do {                                                                                                                   \
@@ -396,7 +397,7 @@ bool pair_eligible(const ccv3d_handle* h, int64_t pair_tiles) {
     if (d.stride[1] != 1 || d.stride[2] != 1 || d.dilation[1] != 1 || d.dilation[2] != 1) return false;
     if (d.kh != 3 || d.kw != 3) return false;              // (1x1 layers are bound by their epilogue; pairs make them slower)
     if (pl.NPAD % 16 != 0 || h->sm_count < 2) return false;
-    return pair_tiles * pl.NT >= h->sm_count / 4;
+    return pair_tiles * pl.NT >= h->sm_count / 8;
 }
 
 ccv3d_status launch_conv(ccv3d_handle* h, TcParams p, int nb, int ty0, int ty1, size_t smem, int ks, cudaStream_t st) {
@@ -480,7 +481,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     const int ACC = (2 * asets * NB * NPAD <= 512) ? 2 : 1;
     // CTA pairs (wide output-channel tiles): 16x16-pixel tiles shared by the two CTAs of a cluster; not combined with
     // the banded multi-stream schedule
-    const bool pair = !split_n && !per_tap && !f32 && !(d.flags & CCV3D_FLAG_OVERLAP) && NB == pl.NB &&
+    const bool pair = !per_tap && !f32 && !(d.flags & CCV3D_FLAG_OVERLAP) &&
                       pair_eligible(h, (int64_t)N * ((Ho + 15) / 16) * ((Wo + 16 * NB - 1) / (16 * NB)) * To);
     const int TW = 8 * NB;                                 // pixels per row of a CTA's part of a tile
     const int TWT = pair ? 2 * TW : TW;                    // tile width in the tile index space
@@ -1116,7 +1117,7 @@ ccv3d_status forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int x_slot, int
         split_n = 1; NT = 2 * pl.NT; NPAD = pl.NPAD / 2;
     }
     // CTA pairs: 16x16-pixel tiles shared by two CTAs, one 128-pixel block each
-    const bool pair = !split_n && NB == pl.NB &&
+    const bool pair =
                       pair_eligible(h, (int64_t)N * ((H + 15) / 16) * ((W + 16 * NB - 1) / (16 * NB)) * T);
     const int ACC = (2 * NB * NPAD <= 512) ? 2 : 1;
     const int TW = 8 * NB, BW = TW + d.kw - 1, BH = 16 + d.kh - 1;

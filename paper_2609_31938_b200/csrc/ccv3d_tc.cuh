@@ -992,13 +992,17 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                         if (PAIR) {
                             // this CTA's half (rows rank*NPAD/2 ..) of every tap's weight tile, as boxes of the 2-D map
                             // over the packed weights; both CTAs' boxes are counted on the leader's barrier
-                            const int row0 = (((dt * p.CB + cb) * p.NT + nt) * spatial) * p.NPAD + (int)rank * (p.NPAD >> 1);
+                            // (split_n: NT and NPAD describe half-width tiles of a layer packed at full width; the rows of
+                            // a tap's full-width tile are then [half 0 | half 1], each again split between the two CTAs)
+                            const int npw = p.NPAD << p.split_n;                      // rows of a packed (full-width) tile
+                            const int row0 = (((dt * p.CB + cb) * (p.NT >> p.split_n) + (nt >> p.split_n)) * spatial) * npw +
+                                             (nt & p.split_n) * p.NPAD + (int)rank * (p.NPAD >> 1);
                             for (int tp = 0; tp < spatial; tp += p.TPB) {
                                 if (!(ok = mbar_wait(&sh->empty_b[s], phase, sh, p, SITE_B_EMPTY))) break;
                                 const uint32_t bar = smem_u32(&sh->full_b[s]);
                                 if (rank == 0) mbar_expect_tx(bar, 2 * b_bytes);
                                 const uint32_t dst = smem_u32(ring_b + (size_t)s * p.b_slot);
-                                for (int u = 0; u < p.TPB; ++u) tma_load_2d_pair(dst + u * p.b_tap, &tm_c, bar, 0, row0 + (tp + u) * p.NPAD);
+                                for (int u = 0; u < p.TPB; ++u) tma_load_2d_pair(dst + u * p.b_tap, &tm_c, bar, 0, row0 + (tp + u) * npw);
                                 if (++s == p.SB) { s = 0; phase ^= 1; }
                             }
                             continue;
