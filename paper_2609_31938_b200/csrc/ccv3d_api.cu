@@ -78,6 +78,7 @@ struct ccv3d_handle {
     int64_t prof_n;
     cudaEvent_t* prof_ev;   // PROF_SLOTS x 3 events, created on first enable
     int pdl;             // 1: convolution kernels on frame rings are launched with programmatic stream serialization
+    int cluster_ok;      // the device launches thread-block clusters (needed for CTA pairs)
     int call_cf;         // history frames held by the cache of the call being served (set by the entry points)
     ccv3d_counters ctr;
 };
@@ -392,7 +393,7 @@ ccv3d_status launch_pair_any(ccv3d_handle* h, const CUtensorMap& tm_a, const CUt
 bool pair_eligible(const ccv3d_handle* h, int64_t pair_tiles) {
     const ccv3d_desc& d = h->d;
     const TcPlan& pl = h->plan;
-    if (d.flags & CCV3D_FLAG_NO_PAIR) return false;
+    if ((d.flags & CCV3D_FLAG_NO_PAIR) || !h->cluster_ok) return false;
     if (d.dtype != CCV3D_BF16 || (d.flags & CCV3D_FLAG_TC_PER_TAP_A)) return false;
     if (d.stride[1] != 1 || d.stride[2] != 1 || d.dilation[1] != 1 || d.dilation[2] != 1) return false;
     if (d.kh != 3 || d.kw != 3) return false;              // (1x1 layers are bound by their epilogue; pairs make them slower)
@@ -1362,6 +1363,10 @@ ccv3d_status ccv3d_create(ccv3d_handle** out_h, const ccv3d_desc* d, const void*
         if (v > 0 && v <= 10000) h->wait_limit_clk = (long long)prop.clockRate * v;
     }
     h->pdl = getenv("CCV3D_NO_PDL") ? 0 : 1;
+    if (cudaDeviceGetAttribute(&h->cluster_ok, cudaDevAttrClusterLaunch, dev) != cudaSuccess) {
+        cudaGetLastError();
+        h->cluster_ok = 0;
+    }
     cudaStream_t st = (cudaStream_t)stream;
     const int taps = d->kt * d->kh * d->kw;
 
