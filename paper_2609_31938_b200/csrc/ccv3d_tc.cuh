@@ -1375,7 +1375,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
             const int h_lo = 16 * b;
             const int rows = (sp.H - h_lo < 16) ? sp.H - h_lo : 16;
             const int ntask = sp.N * nf * sp.CB * rows * nchunks;
-            constexpr int G = 2;                             // tasks whose loads are in flight together (16 KB per CTA)
+            constexpr int G = 4;                             // tasks whose loads are in flight together (32 KB per CTA; 6 would spill)
             for (int task0 = blockIdx.x; task0 < ntask; task0 += G * gridDim.x) {
                 StageTask tk[G];
                 uint4 val[G][StagerGeom<KB>::NLD];
