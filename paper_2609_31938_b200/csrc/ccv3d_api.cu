@@ -318,10 +318,10 @@ ccv3d_status launch_stage(ccv3d_handle* h, StageParams sp, int h0, int h1, int n
 
 // CTA pairs: clusters of two CTAs, one 16x16-pixel tile per cluster (see the kernel).  tm_w is the 2-D map over the
 // packed weights from which each CTA takes its half of every tap's tile.
-template <int KB, int NB, int KS, int TPBC, bool COOP>
+template <int KB, int NB, int KS, int TPBC, bool COOP, bool TF32 = false>
 ccv3d_status launch_tc_pair(ccv3d_handle* h, const CUtensorMap& tm_a, const CUtensorMap& tm_w, const CUtensorMap& tm_o,
                             const TcParams& p, const StageParams& sp, size_t smem, int grid, cudaStream_t st) {
-    auto kern = conv3d_tcgen05_kernel<KB, NB, KS, TPBC, false, COOP, false, true>;
+    auto kern = conv3d_tcgen05_kernel<KB, NB, KS, TPBC, false, COOP, TF32, true>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return cuda_fail();
     cudaLaunchConfig_t cfg;
@@ -352,8 +352,8 @@ ccv3d_status weight_map(ccv3d_handle* h, int box_rows, const CUtensorMap** out) 
     CUtensorMap* tm = &h->tm_w[slot];
     const TcPlan& pl = h->plan;
     const ccv3d_desc& d = h->d;
-    const uint64_t rows = (uint64_t)d.kt * pl.CB * pl.NT * d.kh * d.kw * pl.NPAD;
-    cuuint64_t dims[2] = {(cuuint64_t)pl.KB, (cuuint64_t)rows};
+    const uint64_t rows = (uint64_t)(d.dtype == CCV3D_F32 ? 3 : 1) * d.kt * pl.CB * pl.NT * d.kh * d.kw * pl.NPAD;
+    cuuint64_t dims[2] = {(cuuint64_t)pl.KB, (cuuint64_t)rows};   // (FP32 layers: 128-byte rows of 32 values, seen as 64 BF16)
     cuuint64_t strides[1] = {(cuuint64_t)pl.KB * 2};
     cuuint32_t box[2] = {(cuuint32_t)pl.KB, (cuuint32_t)box_rows};
     cuuint32_t es[2] = {1, 1};
@@ -380,6 +380,17 @@ ccv3d_status launch_pair_any(ccv3d_handle* h, const CUtensorMap& tm_a, const CUt
         if (ks == 3) return launch_tc_pair<KBv, NBv, 3, 1, COOP>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);              \
         return launch_tc_pair<KBv, NBv, 1, 1, COOP>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);                           \
     } while (0)
+    if (h->d.dtype == CCV3D_F32) {          // 3xTF32 (plain schedule only)
+        if (COOP) return CCV3D_ERR_UNSUPPORTED;
+        if (nb == 2) {
+            if (ks == 3 && p.TPB == 3) return launch_tc_pair<64, 2, 3, 3, false, true>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
+            if (ks == 3) return launch_tc_pair<64, 2, 3, 1, false, true>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
+            return launch_tc_pair<64, 2, 1, 1, false, true>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
+        }
+        if (ks == 3 && p.TPB == 3) return launch_tc_pair<64, 1, 3, 3, false, true>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
+        if (ks == 3) return launch_tc_pair<64, 1, 3, 1, false, true>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
+        return launch_tc_pair<64, 1, 1, 1, false, true>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
+    }
     if (h->plan.KB == 64 && nb == 2) CCV3D_LAUNCH_PAIR(64, 2);
     else if (h->plan.KB == 64) CCV3D_LAUNCH_PAIR(64, 1);
     else if (nb == 2) CCV3D_LAUNCH_PAIR(32, 2);
@@ -394,7 +405,7 @@ bool pair_eligible(const ccv3d_handle* h, int64_t pair_tiles) {
     const ccv3d_desc& d = h->d;
     const TcPlan& pl = h->plan;
     if ((d.flags & CCV3D_FLAG_NO_PAIR) || !h->cluster_ok) return false;
-    if (d.dtype != CCV3D_BF16 || (d.flags & CCV3D_FLAG_TC_PER_TAP_A)) return false;
+    if (d.flags & CCV3D_FLAG_TC_PER_TAP_A) return false;
     if (d.stride[1] != 1 || d.stride[2] != 1 || d.dilation[1] != 1 || d.dilation[2] != 1) return false;
     if (d.kh != 3 || d.kw != 3) return false;              // (1x1 layers are bound by their epilogue; pairs make them slower)
     if (pl.NPAD % 16 != 0 || h->sm_count < 2) return false;
@@ -482,7 +493,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     const int ACC = (2 * asets * NB * NPAD <= 512) ? 2 : 1;
     // CTA pairs (wide output-channel tiles): 16x16-pixel tiles shared by the two CTAs of a cluster; not combined with
     // the banded multi-stream schedule
-    const bool pair = !per_tap && !f32 && !(d.flags & CCV3D_FLAG_OVERLAP) &&
+    const bool pair = !per_tap && !(d.flags & CCV3D_FLAG_OVERLAP) &&
                       pair_eligible(h, (int64_t)N * ((Ho + 15) / 16) * ((Wo + 16 * NB - 1) / (16 * NB)) * To);
     const int TW = 8 * NB;                                 // pixels per row of a CTA's part of a tile
     const int TWT = pair ? 2 * TW : TW;                    // tile width in the tile index space

@@ -544,6 +544,18 @@ __device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint32_t a_lo,
         : "memory");
 }
 
+__device__ __forceinline__ void tc_mma_tf32_pair(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
+                                                 uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %6, 0;\n\t"
+        "mov.b64 da, {%1, %2};\n\t"
+        "mov.b64 db, {%3, %4};\n\t"
+        "tcgen05.mma.cta_group::2.kind::tf32 [%0], da, db, %5, p;\n\t}" ::"r"(d_tmem),
+        "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
 // One lane of a fully converged warp; the others get 0.  Keeps the surrounding code warp-uniform so that
 // descriptors and addresses can live in uniform registers.
 __device__ __forceinline__ uint32_t elect_one() {
@@ -808,7 +820,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     static_assert(!(FUSED && COOP), "one or the other");
     static_assert(!FUSED || KB == 32, "the fused mode transposes 32-channel blocks");
     static_assert(!TF32 || (KB == 64 && !FUSED && !COOP), "FP32 layers: 128-byte rows, plain variant");
-    static_assert(!PAIR || (KS > 0 && !FUSED && !TF32), "CTA pairs: straight-line taps, BF16");
+    static_assert(!PAIR || (KS > 0 && !FUSED), "CTA pairs: straight-line taps");
     // (TF32 layers always write FP32 through the direct-store epilogue, which is where the two accumulators of the
     // last pass are added)
     constexpr uint32_t ROWB = KB * 2;                       // bytes per pixel row (one swizzle span)
@@ -960,7 +972,8 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                             if (PAIR) {
                                 // both CTAs' boxes are counted on the leader's barrier, which the leader arms for both
                                 if (rank == 0) mbar_expect_tx(bar, 2 * a_bytes);
-                                tma_load_5d_pair(smem_u32(ring_a + (size_t)s * p.a_slot), &tm_a, bar, 0, w0 - pw, h0 - ph, cb, fz);
+                                tma_load_5d_pair(smem_u32(ring_a + (size_t)s * p.a_slot), &tm_a, bar, 0, w0 - pw, h0 - ph,
+                                                 TF32 ? 2 * cb + (pass == 1) : cb, fz);
                             } else {
                                 mbar_expect_tx(bar, a_bytes);
                                 tma_load_5d(smem_u32(ring_a + (size_t)s * p.a_slot), &tm_a, bar, 0, w0 * stw - pw + dw * dlw,
@@ -995,7 +1008,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                             // (split_n: NT and NPAD describe half-width tiles of a layer packed at full width; the rows of
                             // a tap's full-width tile are then [half 0 | half 1], each again split between the two CTAs)
                             const int npw = p.NPAD << p.split_n;                      // rows of a packed (full-width) tile
-                            const int row0 = (((dt * p.CB + cb) * (p.NT >> p.split_n) + (nt >> p.split_n)) * spatial) * npw +
+                            const int row0 = ((((pass * p.kt + dt) * p.CB + cb) * (p.NT >> p.split_n) + (nt >> p.split_n)) * spatial) * npw +
                                              (nt & p.split_n) * p.NPAD + (int)rank * (p.NPAD >> 1);
                             for (int tp = 0; tp < spatial; tp += p.TPB) {
                                 if (!(ok = mbar_wait(&sh->empty_b[s], phase, sh, p, SITE_B_EMPTY))) break;
@@ -1085,7 +1098,10 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                                 for (int j = 0; j < NBW; ++j) {
 #pragma unroll
                                     for (int k = 0; k < KSTEPS; ++k)
-                                        if (PAIR)
+                                        if (PAIR && TF32)
+                                            tc_mma_tf32_pair(d0 + j * p.NPAD, a_lo + j * ((8 * ROWB) >> 4) + 2 * k, a_hi, b_lo + 2 * k, b_hi,
+                                                             idesc, (tap == 0 && k == 0) ? acc_in : 1u);
+                                        else if (PAIR)
                                             tc_mma_bf16_pair(d0 + j * p.NPAD, a_lo + j * ((8 * ROWB) >> 4) + 2 * k, a_hi, b_lo + 2 * k, b_hi,
                                                              idesc, (tap == 0 && k == 0) ? acc_in : 1u);
                                         else

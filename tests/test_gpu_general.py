@@ -245,3 +245,22 @@ def test_fp32_route_selection_by_size(ccv):
         layer.close()
     rms = float(np.sqrt(np.mean(ref ** 2)))
     assert np.abs(outs["auto"] - outs["fma"]).max() <= 1e-4 * rms
+
+
+@pytest.mark.parametrize("Cin,Cout,H,W", [(64, 64, 96, 96), (48, 192, 64, 80)])   # two pixel blocks per CTA; one
+def test_fp32_on_cta_pairs_equals_single_ctas_bitwise(ccv, Cin, Cout, H, W):
+    """The 3xTF32 route on CTA pairs: same passes, same accumulators, same bits as on single CTAs, within the FP32
+    tolerance of the oracle."""
+    c = _case(1, Cin, Cout, 2, H, W, (3, 3, 3), si.F32, 2, seed=43)
+    ref, ref_nc = oracle.forward_general(c["x"], c["cache"], c["w"], c["b"])
+    outs = []
+    for flags in (ccv.FLAG_F32_TENSOR, ccv.FLAG_F32_TENSOR | ccv.FLAG_NO_PAIR):
+        layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), flags=flags)
+        o, nc = layer(to_dev(c["x"]), to_dev(c["cache"]))
+        torch.cuda.synchronize()
+        assert layer.device_status()[0] == ccv.OK and layer.counters()["tcgen05_bf16"] == 1
+        assert np.array_equal(bits(nc), ref_nc)
+        outs.append(o)
+        layer.close()
+    check(as_f64(outs[0]), ref, "f32")
+    assert torch.equal(outs[0], outs[1])
