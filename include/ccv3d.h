@@ -55,8 +55,8 @@ typedef enum {
 #define CCV3D_FLAG_TWO_KERNELS 0x10u     /* tensor-core route: run the staging pass as its own kernel before the convolution kernel instead of
                                             inside it (cooperative staging, the default when W % 8 == 0) */
 #define CCV3D_FLAG_FUSED 0x8u            /* tensor-core route without scratch memory: no channels-last staging copy; the kernel reads x and the cache
-                                            by TMA and transposes in shared memory (needs W % 8 == 0, else the staged route is taken). About as fast as
-                                            the default route in short bursts, ~3 % slower sustained; for callers that cannot afford the workspace. */
+                                            by TMA and transposes in shared memory (needs W % 8 == 0, else the staged route is taken). Some 10 % slower
+                                            than the default route; for callers that cannot afford the workspace. */
 #define CCV3D_FLAG_F32_TENSOR 0x20u       /* FP32 layers: always use the tensor cores (3xTF32: each FP32 product as hi*hi + hi*lo + lo*hi of TF32
                                             operands, FP32 accumulate); the default sends calls under 0.2 GFLOP, and layers with cin*kt*kh*kw > 16384,
                                             to the FP32-FMA kernel */
