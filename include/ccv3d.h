@@ -199,6 +199,11 @@ ccv3d_status ccv3d_forward_static(ccv3d_handle* h, const void* x, const void* ca
  * and cache to device staging owned by the handle, runs ccv3d_forward, copies
  * out and new_cache back, and returns after the stream has completed.  Pinned
  * host memory makes the copies asynchronous with respect to each other.
+ * Standard BF16 tensor-core layers with cin % 32 == 0 and frames of a few MB run
+ * frame by frame instead (upload of frame t+1, convolution of frame t on a frame
+ * ring and download of frame t-1 overlap on three streams; same bits, since the
+ * operator streams exactly): the call then takes about as long as the slower
+ * PCIe direction alone.
  */
 ccv3d_status ccv3d_forward_host(ccv3d_handle* h, const void* x_host, const void* cache_host, void* out_host,
                                 void* new_cache_host, int32_t N, int32_t T, int32_t H, int32_t W, void* stream);

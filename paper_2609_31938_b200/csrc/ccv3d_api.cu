@@ -63,6 +63,8 @@ struct ccv3d_handle {
     // host-entry staging (device buffers)
     void* hx; void* hc; void* ho; void* hn;
     uint64_t hx_b, hc_b, ho_b, hn_b;
+    cudaEvent_t hp_ev[4][3];   // pipelined host entry: per frame buffer {uploaded, input buffer free, computed, downloaded}
+    bool hp_ready;
     EncodeTiledFn encode;
     CUtensorMap tm_a;
     ShapeKey tm_a_key;
@@ -1464,6 +1466,9 @@ ccv3d_status ccv3d_destroy(ccv3d_handle* h) {
         if (h->ev_band[i]) cudaEventDestroy(h->ev_band[i]);
     for (int i = 0; i < 2; ++i)
         if (h->ev_join[i]) cudaEventDestroy(h->ev_join[i]);
+    if (h->hp_ready)
+        for (int k = 0; k < 4; ++k)
+            for (int b = 0; b < 3; ++b) cudaEventDestroy(h->hp_ev[k][b]);
     if (h->prof_ev) {
         for (int i = 0; i < 3 * PROF_SLOTS; ++i) cudaEventDestroy(h->prof_ev[i]);
         delete[] h->prof_ev;
@@ -1532,6 +1537,108 @@ ccv3d_status ccv3d_forward_static(ccv3d_handle* h, const void* x, const void* ca
     return count(h, forward_tc_static(h, x, cache, out, new_cache, N, T, H, W, (cudaStream_t)stream));
 }
 
+// Host entry point, pipelined frame by frame (standard BF16 tensor-core layers whose channels fit a frame ring).
+// Frame t of x is a strided 2-D copy (one row per (n, channel) plane) into a dense one-frame device buffer on an
+// upload stream; on the caller's stream it is moved into a frame ring and convolved as a one-frame chunk (history =
+// the ring, exactly the streaming form of the operator, so the result is bit for bit that of one T-frame call);
+// the output frame goes back with another strided 2-D copy on a download stream.  Three buffers of each kind rotate,
+// so that upload, compute and download of different frames overlap: the call takes about as long as the slower of
+// the two PCIe directions instead of their sum.
+static ccv3d_status forward_host_pipelined(ccv3d_handle* h, const void* x_host, const void* cache_host, void* out_host,
+                                    void* new_cache_host, int N, int T, int H, int W, cudaStream_t st) {
+    const ccv3d_desc& d = h->d;
+    const int tc = hist_len(d);
+    constexpr int NBUF = 3;
+    const uint64_t HWb = (uint64_t)H * W * 2;
+    const uint64_t xf = (uint64_t)N * d.cin * HWb, of = (uint64_t)N * d.cout * HWb;      // one frame of x / of out
+    ccv3d_ring ring;
+    ring.N = N; ring.C = d.cin; ring.F = tc + 1; ring.H = H; ring.W = W; ring.KB = h->plan.KB;
+    ccv3d_status s;
+    if ((s = grow(&h->hx, &h->hx_b, NBUF * xf)) != CCV3D_OK) return s;
+    if ((s = grow(&h->ho, &h->ho_b, NBUF * of)) != CCV3D_OK) return s;
+    if ((s = grow(&h->hc, &h->hc_b, (uint64_t)ring.F * xf)) != CCV3D_OK) return s;
+    if (tc && new_cache_host && (s = grow(&h->hn, &h->hn_b, (uint64_t)tc * xf)) != CCV3D_OK) return s;
+    ring.base = h->hc;
+    if (!h->hp_ready) {
+        for (int k = 0; k < 4; ++k)
+            for (int b = 0; b < NBUF; ++b)
+                if (cudaEventCreateWithFlags(&h->hp_ev[k][b], cudaEventDisableTiming) != cudaSuccess) return cuda_fail();
+        h->hp_ready = true;
+    }
+    cudaStream_t s_up = h->side[0], s_down = h->side[1];
+    if (cudaEventRecord(h->ev_fork, st) != cudaSuccess) return cuda_fail();
+    if (cudaStreamWaitEvent(s_up, h->ev_fork, 0) != cudaSuccess || cudaStreamWaitEvent(s_down, h->ev_fork, 0) != cudaSuccess)
+        return cuda_fail();
+    if (!cache_host && tc && cudaMemsetAsync(ring.base, 0, (size_t)ring.F * xf, st) != cudaSuccess) return cuda_fail();
+
+    const int pre = (cache_host && tc) ? tc : 0;           // history frames uploaded before the first frame of x
+    const bool nc_early = tc && new_cache_host && tc < NBUF && pre + T >= tc;
+    int slot = 0, seen = 0;                                // ring slot of the next frame; frames in the ring so far
+    for (int i = 0; i < pre + T; ++i) {
+        const int b = i % NBUF;
+        const bool is_x = i >= pre;
+        const int t = is_x ? i - pre : i;
+        char* xin = (char*)h->hx + (size_t)b * xf;
+        // upload: wait until the ring load that last read this buffer is done
+        if (i >= NBUF && cudaStreamWaitEvent(s_up, h->hp_ev[1][b], 0) != cudaSuccess) return cuda_fail();
+        const char* src = is_x ? (const char*)x_host + (size_t)t * HWb : (const char*)cache_host + (size_t)t * HWb;
+        const size_t spitch = (size_t)(is_x ? T : tc) * HWb;
+        if (cudaMemcpy2DAsync(xin, HWb, src, spitch, HWb, (size_t)N * d.cin, cudaMemcpyHostToDevice, s_up) != cudaSuccess)
+            return cuda_fail();
+        if (cudaEventRecord(h->hp_ev[0][b], s_up) != cudaSuccess) return cuda_fail();
+        // cache update: the last tc frames of the stream go straight back from their upload buffers (bit copies),
+        // early, while the download stream has nothing else to do.  (tc < NBUF: these buffers are not reused in
+        // this call; the next call starts after the download stream has been joined.)
+        if (nc_early && i >= pre + T - tc) {
+            const int j = i - (pre + T - tc);
+            if (cudaStreamWaitEvent(s_down, h->hp_ev[0][b], 0) != cudaSuccess) return cuda_fail();
+            if (cudaMemcpy2DAsync((char*)new_cache_host + (size_t)j * HWb, (size_t)tc * HWb, xin, HWb, HWb, (size_t)N * d.cin,
+                                  cudaMemcpyDeviceToHost, s_down) != cudaSuccess)
+                return cuda_fail();
+        }
+        // compute
+        if (cudaStreamWaitEvent(st, h->hp_ev[0][b], 0) != cudaSuccess) return cuda_fail();
+        if ((s = ccv3d_ring_load(&ring, slot, xin, 1, st)) != CCV3D_OK) return s;
+        h->ctr.kernel_launches++;
+        if (cudaEventRecord(h->hp_ev[1][b], st) != cudaSuccess) return cuda_fail();
+        if (is_x) {
+            const int ob = t % NBUF;
+            char* oout = (char*)h->ho + (size_t)ob * of;
+            if (t >= NBUF && cudaStreamWaitEvent(st, h->hp_ev[3][ob], 0) != cudaSuccess) return cuda_fail();
+            const int hist = seen < tc ? seen : tc;
+            if ((s = forward_ring(h, &ring, slot, hist, nullptr, 0, nullptr, 0, oout, 1, st)) != CCV3D_OK) return s;
+            if (cudaEventRecord(h->hp_ev[2][ob], st) != cudaSuccess) return cuda_fail();
+            // download
+            if (cudaStreamWaitEvent(s_down, h->hp_ev[2][ob], 0) != cudaSuccess) return cuda_fail();
+            if (cudaMemcpy2DAsync((char*)out_host + (size_t)t * HWb, (size_t)T * HWb, oout, HWb, HWb, (size_t)N * d.cout,
+                                  cudaMemcpyDeviceToHost, s_down) != cudaSuccess)
+                return cuda_fail();
+            if (cudaEventRecord(h->hp_ev[3][ob], s_down) != cudaSuccess) return cuda_fail();
+        }
+        slot = (slot + 1) % ring.F;
+        ++seen;
+    }
+    if (tc && new_cache_host && !nc_early) {
+        // the last tc frames of [cache ; x] are the tc slots before `slot` (zeros where the stream had no history)
+        if ((s = ccv3d_ring_store(&ring, (slot + ring.F - tc) % ring.F, h->hn, tc, st)) != CCV3D_OK) return s;
+        h->ctr.kernel_launches++;
+        if (cudaMemcpyAsync(new_cache_host, h->hn, (size_t)tc * xf, cudaMemcpyDeviceToHost, st) != cudaSuccess) return cuda_fail();
+    }
+    if (cudaEventRecord(h->ev_join[0], s_down) != cudaSuccess || cudaStreamWaitEvent(st, h->ev_join[0], 0) != cudaSuccess)
+        return cuda_fail();
+    if (cudaEventRecord(h->ev_join[1], s_up) != cudaSuccess || cudaStreamWaitEvent(st, h->ev_join[1], 0) != cudaSuccess)
+        return cuda_fail();
+    h->ctr.tcgen05_bf16++;
+    return CCV3D_OK;
+}
+
+static bool host_pipeline_eligible(const ccv3d_handle* h, int T, int H, int W) {
+    const ccv3d_desc& d = h->d;
+    if (!h->use_tc || !standard_geom(d) || d.out_dtype != CCV3D_BF16 || (d.flags & CCV3D_FLAG_TC_PER_TAP_A)) return false;
+    if (!h->side[0] || d.cin % h->plan.KB) return false;
+    return (uint64_t)H * W * (d.cin + d.cout) * 2 >= (4u << 20) && T >= 2;      // a few MB per frame, or the copies are latency
+}
+
 ccv3d_status ccv3d_forward_host(ccv3d_handle* h, const void* x_host, const void* cache_host, void* out_host,
                                 void* new_cache_host, int32_t N, int32_t T, int32_t H, int32_t W, void* stream) {
     if (!h) return CCV3D_ERR_INVALID_ARG;
@@ -1540,6 +1647,15 @@ ccv3d_status ccv3d_forward_host(ccv3d_handle* h, const void* x_host, const void*
     if (s != CCV3D_OK) {
         h->ctr.calls++;
         return count(h, s);
+    }
+    if (host_pipeline_eligible(h, T, H, W)) {
+        h->ctr.calls++;
+        if (!on_handle_device(h)) return count(h, CCV3D_ERR_INVALID_ARG);
+        s = forward_host_pipelined(h, x_host, cache_host, out_host, new_cache_host, N, T, H, W, (cudaStream_t)stream);
+        if (s != CCV3D_OK) return count(h, s);
+        if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return count(h, cuda_fail());
+        count(h, CCV3D_OK);
+        return ccv3d_device_status(h, nullptr);
     }
     const ccv3d_desc& d = h->d;
     const int tc = hist_len(d);

@@ -371,6 +371,28 @@ def test_host_entry_point_matches_device_entry_point(ccv):
     layer.close()
 
 
+@pytest.mark.parametrize("N,Cin,Cout,T,H,W,cache", [(1, 64, 96, 5, 128, 160, "random"), (2, 96, 64, 3, 120, 136, None),
+                                                       (1, 64, 64, 2, 160, 200, "random")])
+def test_pipelined_host_entry_point(ccv, N, Cin, Cout, T, H, W, cache):
+    """Frames of a few MB: the host entry point uploads, convolves (on a frame ring, one frame per call) and
+    downloads frame by frame on three streams.  Same bits as the device entry point on the whole tensor, cache
+    update included; pageable host memory."""
+    c = si.conv_case(N, Cin, Cout, T, H, W, cache=cache, seed=13)
+    layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]))
+    out_d, nc_d = layer(to_dev(c["x"]), to_dev(c["cache"]))
+    torch.cuda.synchronize()
+    out_h = np.full((N, Cout, T, H, W), 0x7FC0, np.uint16)
+    nc_h = np.full((N, Cin, 2, H, W), 0x7FC0, np.uint16)
+    for _ in range(2):                                             # second call: the rotating buffers and events are reused
+        s = ccv.ccv3d_forward_host(layer.h, c["x"].ctypes.data, None if c["cache"] is None else c["cache"].ctypes.data,
+                                   out_h.ctypes.data, nc_h.ctypes.data, N, T, H, W, torch.cuda.current_stream().cuda_stream)
+        assert s == ccv.OK
+        assert np.array_equal(out_h, bits(out_d)) and np.array_equal(nc_h, bits(nc_d))
+    ctr = layer.counters()
+    assert ctr["calls"] == ctr["ok"] == 3 and ctr["kernel_launches"] > 2 * T     # frame-by-frame launches: the pipelined path ran
+    layer.close()
+
+
 @pytest.mark.parametrize("shape,rt", [((2, 3, 2, 5, 6), 3), ((1, 4, 3, 6, 8), 4), ((1, 2, 2, 4, 12), 1)])
 def test_chain_glue_kernels(ccv, shape, rt):
     """Residual add (exact sum, one RNE rounding) and nearest-neighbour upsampling (exact copies), scalar and
