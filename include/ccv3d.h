@@ -63,6 +63,8 @@ typedef enum {
 #define CCV3D_FLAG_NO_PAIR 0x40u          /* tensor-core route: never run tiles on pairs of CTAs (cta_group::2 MMAs with M = 256, each SM
                                             streaming half of every weight tile) - the default for layers with more than 128 output
                                             channels per tile and 3x3 or 1x1 spatial kernels */
+#define CCV3D_FLAG_EPI_SILU 0x80u         /* epilogue activation (not part of the paper's operator): out = silu(conv + b), v / (1 + exp(-v)) in
+                                            FP32 before the one output rounding; a residual (frame rings) is added after it */
 #define CCV3D_FLAG_TC_PER_TAP_A 0x2u    /* tensor-core kernel: fetch the activation tile once per tap (no halo reuse in shared memory) */
 
 /* Layer description, fixed at create time (Algorithm 1's Require line: W, b, p, s, d, g).

@@ -24,6 +24,7 @@ FLAG_FUSED = 0x8
 FLAG_TWO_KERNELS = 0x10
 FLAG_F32_TENSOR = 0x20
 FLAG_NO_PAIR = 0x40
+FLAG_EPI_SILU = 0x80
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_ALIAS, ERR_ARCH, ERR_NOMEM, ERR_CUDA, \
     ERR_DEVICE_TIMEOUT = range(9)

@@ -512,6 +512,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     p.N = N; p.T = To; p.H = Ho; p.W = Wo; p.Cout = d.cout; p.F = F;
     p.kt = d.kt; p.kh = d.kh; p.kw = d.kw;
     p.general = general ? 1 : 0;
+    p.act = (d.flags & CCV3D_FLAG_EPI_SILU) ? 1 : 0;
     p.pad_h = d.pad_h; p.pad_w = d.pad_w; p.dil_h = d.dilation[1]; p.dil_w = d.dilation[2]; p.dil_t = d.dilation[0];
     p.str_h = d.stride[1]; p.str_w = d.stride[2]; p.str_t = d.stride[0];
     p.CB = pl.CB; p.NT = NT; p.NPAD = NPAD;
@@ -719,6 +720,7 @@ ccv3d_status forward_fused(ccv3d_handle* h, const void* x, const void* cache, vo
     memset(&p, 0, sizeof(p));
     p.N = N; p.T = T; p.H = H; p.W = W; p.Cout = d.cout; p.F = tc + T;
     p.kt = d.kt; p.kh = d.kh; p.kw = d.kw; p.tc = tc; p.cf = cf;
+    p.act = (d.flags & CCV3D_FLAG_EPI_SILU) ? 1 : 0;
     p.CB = pl.CB; p.NT = pl.NT; p.NPAD = pl.NPAD;
     p.tiles_h = (H + 15) / 16;
     p.tiles_w = (W + TW - 1) / TW;
@@ -810,7 +812,7 @@ ccv3d_status forward_fused(ccv3d_handle* h, const void* x, const void* cache, vo
 bool pointwise_eligible(const ccv3d_handle* h, int T, int H, int W) {
     const ccv3d_desc& d = h->d;
     const TcPlan& pl = h->plan;
-    if (!(d.kt == 1 && d.kh == 1 && d.kw == 1) || !standard_geom(d)) return false;
+    if (!(d.kt == 1 && d.kh == 1 && d.kw == 1) || !standard_geom(d) || (d.flags & CCV3D_FLAG_EPI_SILU)) return false;
     if (d.flags & CCV3D_FLAG_TC_PER_TAP_A) return false;
     if (pl.KB != 64 || pl.NT != 1 || d.out_dtype != CCV3D_BF16) return false;
     if (((int64_t)T * H * W) % 8 != 0) return false;                       // TMA strides are multiples of 16 bytes
@@ -1000,6 +1002,7 @@ ccv3d_status forward_tc_static(ccv3d_handle* h, const void* x, const void* cache
     p.first_frame = (tc && !cache) ? tc : 0;
     p.out_f32 = d.out_dtype == CCV3D_F32;
     p.per_tap_a = 0;
+    p.act = (d.flags & CCV3D_FLAG_EPI_SILU) ? 1 : 0;
     p.ACC = ACC;
     p.a_slot = (uint32_t)align_up((uint64_t)BW * BH * pl.KB * 2, 1024);
     p.b_tap = (uint32_t)pl.NPAD * pl.KB * 2;
@@ -1145,6 +1148,7 @@ ccv3d_status forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int x_slot, int
     p.N = N; p.T = T; p.H = H; p.W = W; p.Cout = d.cout;
     p.F = in->F;
     p.f0 = (x_slot - tc + in->F) % in->F;
+    p.act = (d.flags & CCV3D_FLAG_EPI_SILU) ? 1 : 0;
     p.kt = d.kt; p.kh = d.kh; p.kw = d.kw;
     p.CB = pl.CB; p.NT = NT; p.NPAD = NPAD;
     p.tiles_h = (H + 15) / 16;
@@ -1241,6 +1245,7 @@ ccv3d_status forward_simt(ccv3d_handle* h, const void* x, const void* cache, voi
     p.To = out_t(d, T); p.Ho = out_h(d, H); p.Wo = out_w(d, W); p.st = d.stride[0];
     p.sh = d.stride[1]; p.sw = d.stride[2]; p.ph = d.pad_h; p.pw = d.pad_w; p.dh = d.dilation[1]; p.dw = d.dilation[2];
     p.dil_t = d.dilation[0];
+    p.act = (d.flags & CCV3D_FLAG_EPI_SILU) ? 1 : 0;
     const int64_t npix = (int64_t)N * p.To * p.Ho * p.Wo;
     const int64_t gx = (npix + SIMT_THREADS - 1) / SIMT_THREADS;
     if (gx > 0x7FFFFFFF) return CCV3D_ERR_UNSUPPORTED;

@@ -30,6 +30,7 @@ struct SimtParams {
     int N, Cin, Cout, T, H, W, kt, kh, kw;   // T, H, W: input extents
     int To, Ho, Wo;                          // output extents
     int st;                                  // temporal stride: output frame t reads Z frames t*st + dt*dil_t
+    int act;                                 // 1: SiLU on conv + bias before the output rounding
     int sh, sw, ph, pw, dh, dw, dil_t;       // spatial stride, padding, dilation; temporal dilation (Eq. (1)-(2))
 };
 // With tc = d_t (kt-1): Z = [absent x (tc-cf) ; cache ; x]; frame tau < tc of Z is cache frame tau-(tc-cf) when that is >= 0.
@@ -88,6 +89,10 @@ __global__ void __launch_bounds__(SIMT_THREADS) conv3d_direct_kernel(const SimtP
         }
     }
     TOut* out = (TOut*)p.out;
+    if (p.act) {
+#pragma unroll
+        for (int j = 0; j < SIMT_CO; ++j) acc[j] = acc[j] / (1.f + expf(-acc[j]));
+    }
 #pragma unroll
     for (int j = 0; j < SIMT_CO; ++j)
         if (co0 + j < p.Cout)

@@ -689,6 +689,7 @@ struct TcParams {
     const __nv_bfloat16* res; // optional residual ring [N][res_F][res_CB][H][W][res_KB] holding Cout channels, or null
     int res_F, res_f0, res_CB, res_KB;   // residual frame t is slot (res_f0 + t) mod res_F
     int out_F, out_f0, out_KB;           // epi_tma == 2: output frame t goes to slot (out_f0 + t) mod out_F
+    int act;                             // 1: SiLU on conv + bias before the output rounding (and before the residual)
     int up_rt;                           // epi_tma == 2, > 0: the output ring is 2H x 2W; every pixel is written 2x2 times into
                                          // each of the up_rt slots (out_f0 + t*up_rt + j) mod out_F (nearest-neighbour upsample)
     const float* bias;        // [NT*NPAD]
@@ -776,7 +777,10 @@ __device__ __forceinline__ void load_res32(const __nv_bfloat16* res_row, bool va
 
 // Two neighbouring output channels: round conv + bias to BF16 once; with a residual, add it to that rounded value
 // in FP32 and round again (the result of a BF16 convolution followed by a BF16 addition).
-__device__ __forceinline__ uint32_t epi_pair(float a0, float a1, uint32_t res_pair, bool has_res) {
+__device__ __forceinline__ float silu_f32(float v) { return v / (1.f + __expf(-v)); }
+
+__device__ __forceinline__ uint32_t epi_pair(float a0, float a1, uint32_t res_pair, bool has_res, bool act = false) {
+    if (act) { a0 = silu_f32(a0); a1 = silu_f32(a1); }      // optional SiLU on conv + bias, in FP32, before the one rounding
     __nv_bfloat162 o = __floats2bfloat162_rn(a0, a1);
     if (has_res) {
         const float2 of = __bfloat1622float2(o);
@@ -1210,6 +1214,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
         const bool elected = (threadIdx.x == 4 * 32);
         constexpr bool RING = !FUSED && !COOP;                 // frame-ring output and residual: plain variant only
         const bool has_res = RING && p.res != nullptr;
+        const bool act = p.act != 0;
         int ebuf = 0;
         // bias: a shared-memory copy when the padded channel count fits.  A global load per element costs little
         // while the next tile's MMAs run, but its latency sits in the exposed tail of a CTA's last tile: 11 us
@@ -1279,7 +1284,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
 #pragma unroll
                         for (int j = 0; j < 16; ++j)
                             pk[j] = (2 * j < p.ECH) ? epi_pair(__uint_as_float(v[2 * j]) + bb[2 * j],
-                                                               __uint_as_float(v[2 * j + 1]) + bb[2 * j + 1], rr[j], has_res)
+                                                               __uint_as_float(v[2 * j + 1]) + bb[2 * j + 1], rr[j], has_res, act)
                                                     : 0u;
                         const uint32_t px = (uint32_t)((m >> 3) * TW + blk * 8 + (m & 7));   // pixel of the tile, row-major
                         if (RING && p.epi_tma == 2) {
@@ -1349,9 +1354,10 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
 #pragma unroll
                                 for (int j = 0; j < 32; ++j) {
                                     const int co = co0 + j;
-                                    if (j < nc && co < p.Cout)
-                                        reinterpret_cast<float*>(p.out)[((int64_t)n * p.Cout + co) * p.T * HW + pix] =
-                                            __uint_as_float(v[j]) + bias[co];
+                                    if (j < nc && co < p.Cout) {
+                                        const float val = __uint_as_float(v[j]) + bias[co];
+                                        reinterpret_cast<float*>(p.out)[((int64_t)n * p.Cout + co) * p.T * HW + pix] = act ? silu_f32(val) : val;
+                                    }
                                 }
                             } else {
 #pragma unroll
@@ -1359,7 +1365,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                                     const int co = co0 + 2 * j;
                                     if (2 * j < nc) {
                                         const uint32_t pr = epi_pair(__uint_as_float(v[2 * j]) + bias[co],
-                                                                     __uint_as_float(v[2 * j + 1]) + bias[co + 1], rr[j], has_res);
+                                                                     __uint_as_float(v[2 * j + 1]) + bias[co + 1], rr[j], has_res, act);
                                         unsigned short* o = reinterpret_cast<unsigned short*>(p.out) +
                                                             ((int64_t)n * p.Cout + co) * p.T * HW + pix;
                                         if (co < p.Cout) o[0] = (unsigned short)(pr & 0xFFFFu);

@@ -264,3 +264,64 @@ def test_fp32_on_cta_pairs_equals_single_ctas_bitwise(ccv, Cin, Cout, H, W):
         layer.close()
     check(as_f64(outs[0]), ref, "f32")
     assert torch.equal(outs[0], outs[1])
+
+
+# ---------------------------------------------------------------------------- optional SiLU epilogue
+def _silu64(v):
+    return v / (1.0 + np.exp(-v))
+
+
+@pytest.mark.parametrize("route", ["f32_fma", "bf16_fma", "bf16_tc", "bf16_tc_two_kernels", "bf16_fused", "f32_tc", "bf16_1x1"])
+def test_silu_epilogue(ccv, route):
+    """out = silu(conv + b) in FP32 before the one output rounding, on every route; the oracle's FP64 output through
+    the same function is the reference.  (Not part of the paper's operator: a fused activation for decoder blocks.)"""
+    f32 = route.startswith("f32")
+    k = (1, 1, 1) if route == "bf16_1x1" else (3, 3, 3)
+    shape = (1, 16, 24, 2, 12, 16) if route == "f32_fma" else (1, 64, 96, 4, 160, 192) if route == "bf16_tc" else (1, 64, 96, 2, 40, 48)
+    c = _case(*shape, k, si.F32 if f32 else si.BF16, k[0] - 1, seed=44)
+    flags = {"f32_fma": 0, "bf16_fma": ccv.FLAG_FORCE_SIMT, "bf16_tc": 0, "bf16_tc_two_kernels": ccv.FLAG_TWO_KERNELS,
+             "bf16_fused": ccv.FLAG_FUSED, "f32_tc": ccv.FLAG_F32_TENSOR, "bf16_1x1": 0}[route]
+    ref, ref_nc = oracle.forward_general(c["x"], c["cache"], c["w"], c["b"])
+    ref = _silu64(ref)
+    layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), flags=flags | ccv.FLAG_EPI_SILU)
+    out, nc = layer(to_dev(c["x"]), to_dev(c["cache"]))
+    torch.cuda.synchronize()
+    assert layer.device_status()[0] == ccv.OK
+    _check_activated(as_f64(out), ref, f32)
+    if nc is not None:
+        assert np.array_equal(bits(nc), ref_nc)
+    layer.close()
+
+
+def _check_activated(got, ref, f32):
+    """SiLU shrinks the RMS of the output (0.64 against 1.05) but not its largest values, so the BF16 tolerance
+    "max <= 2e-2 x RMS" no longer covers the rounding of an output in [4, 8) (half a step there is 0.0156 = 2.4e-2 x
+    RMS).  The bound is therefore per element: one BF16 rounding (2^-8 relative, a half step with margin) plus the
+    accumulation error, and the usual mean bound."""
+    rms = float(np.sqrt(np.mean(ref ** 2)))
+    err = np.abs(got - ref)
+    assert np.isfinite(got).all()
+    if f32:
+        assert err.max() <= 1e-4 * rms
+    else:
+        assert np.all(err <= 2.0 ** -8 * np.abs(ref) + 1e-3 * rms), float((err / (2.0 ** -8 * np.abs(ref) + 1e-3 * rms)).max())
+        assert err.mean() <= 2e-3 * rms
+
+
+def test_silu_then_residual_on_rings(ccv):
+    """Ring epilogue order: activation first, then the residual, each with its own BF16 rounding."""
+    c = _case(1, 64, 64, 2, 40, 48, (3, 3, 3), si.BF16, 2, seed=45)
+    layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), flags=ccv.FLAG_EPI_SILU)
+    x, cache = to_dev(c["x"]), to_dev(c["cache"])
+    rin = ccv.FrameRing(1, 64, 4, 40, 48)
+    rin.load(0, cache)
+    rin.load(2, x)
+    plain = torch.empty((1, 64, 2, 40, 48), dtype=torch.bfloat16, device="cuda")
+    both = torch.empty_like(plain)
+    layer.forward_ring(rin, 2, 2, 2, out=plain)
+    layer.forward_ring(rin, 2, 2, 2, out=both, res=rin, res_slot=2)
+    torch.cuda.synchronize()
+    ref, _ = oracle.forward_general(c["x"], c["cache"], c["w"], c["b"])
+    _check_activated(as_f64(plain), _silu64(ref), False)
+    assert torch.equal(both, (plain.float() + x.float()).to(torch.bfloat16))
+    layer.close()
