@@ -280,7 +280,20 @@ ccv3d_status launch_tc_coop(ccv3d_handle* h, const TcParams& p, const StageParam
     auto kern = conv3d_tcgen05_kernel<KB, NB, KS, TPBC, false, true>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return cuda_fail();
-    kern<<<grid, TC_THREADS_FUSED, smem, st>>>(h->tm_a, h->tm_a, h->tm_o, p, sp);
+    // cooperative launch: the tiles of a CTA wait for bands that every other CTA helps to stage, so all CTAs must be
+    // resident together - which an ordinary launch does not promise when another stream's kernel holds some SMs
+    cudaLaunchConfig_t cfg;
+    memset(&cfg, 0, sizeof(cfg));
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(TC_THREADS_FUSED);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, kern, h->tm_a, h->tm_a, h->tm_o, p, sp) != cudaSuccess) return cuda_fail();
     if (cudaGetLastError() != cudaSuccess) return cuda_fail();
     h->ctr.kernel_launches++;
     return CCV3D_OK;
@@ -337,8 +350,12 @@ ccv3d_status launch_tc_pair(ccv3d_handle* h, const CUtensorMap& tm_a, const CUte
     attr[0].val.clusterDim.x = 2; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
     attr[1].val.programmaticStreamSerializationAllowed = 1;
+    if (COOP) {          // all CTAs must be resident together (see launch_tc_coop)
+        attr[1].id = cudaLaunchAttributeCooperative;
+        attr[1].val.cooperative = 1;
+    }
     cfg.attrs = attr;
-    cfg.numAttrs = (h->pdl && !COOP) ? 2 : 1;
+    cfg.numAttrs = (COOP || h->pdl) ? 2 : 1;
     if (cudaLaunchKernelEx(&cfg, kern, tm_a, tm_w, tm_o, p, sp) != cudaSuccess) return cuda_fail();
     if (cudaGetLastError() != cudaSuccess) return cuda_fail();
     h->ctr.kernel_launches++;

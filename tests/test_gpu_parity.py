@@ -439,3 +439,25 @@ def test_cta_pairs_match_the_oracle_and_the_single_cta_kernel(ccv, Cin, Cout, T,
     assert torch.equal(oa, ob) and (na is None or torch.equal(na, nb))
     a.close()
     b.close()
+
+
+def test_two_handles_on_two_streams_concurrently(ccv):
+    """Handles are independent: two layers issued alternately on two streams (cooperative-staging kernels, which are
+    launched cooperatively so that each gets all its CTAs resident) give the results of running them one after the
+    other."""
+    cases = [si.conv_case(1, 64, 192, 4, 160, 256, seed=61), si.conv_case(1, 64, 64, 8, 125, 160, seed=62)]
+    layers = [ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"])) for c in cases]
+    xs = [(to_dev(c["x"]), to_dev(c["cache"])) for c in cases]
+    want = [l(x, ch) for l, (x, ch) in zip(layers, xs)]
+    torch.cuda.synchronize()
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    got = [None, None]
+    for rep in range(3):
+        for i in (0, 1):
+            with torch.cuda.stream(streams[i]):
+                got[i] = layers[i](xs[i][0], xs[i][1])
+    torch.cuda.synchronize()
+    for i in (0, 1):
+        assert layers[i].device_status()[0] == ccv.OK
+        assert torch.equal(got[i][0], want[i][0]) and torch.equal(got[i][1], want[i][1])
+        layers[i].close()
