@@ -8,7 +8,9 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libccv3d.so")
 SOURCES = ["ccv3d_api.cu"]
-DEPS = ["ccv3d_api.cu", "ccv3d_simt.cuh", "ccv3d_tc.cuh", os.path.join("..", "..", "include", "ccv3d.h")]
+DEPS = ["ccv3d_api.cu", "ccv3d_simt.cuh", "ccv3d_tc.cuh", "ccv3d_tc_layout.cuh", "ccv3d_tc_ptx.cuh", "ccv3d_tc_conv.cuh",
+        "ccv3d_tc_pointwise.cuh", "ccv3d_host_common.cuh", "ccv3d_host_tc.cuh", "ccv3d_host_ring.cuh",
+        os.path.join("..", "..", "include", "ccv3d.h")]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-shared", "-Xcompiler", "-fPIC"]

@@ -23,1686 +23,11 @@
 // Every wait on an mbarrier is bounded: when a limit expires the CTA records the
 // wait site in a global status word, raises a shared abort flag so that its other
 // roles stop too, releases its tensor memory and returns.
+//
+// Files: ccv3d_tc_layout.cuh (packing, staging, ring moves), ccv3d_tc_ptx.cuh (PTX wrappers), ccv3d_tc_conv.cuh (the
+// implicit-GEMM kernel), ccv3d_tc_pointwise.cuh (the 1x1x1 streaming kernel).
 #pragma once
-#include <cuda.h>
-#include <cuda_bf16.h>
-#include <cuda_runtime.h>
-#include <stdint.h>
-
-namespace ccv3d {
-
-// ------------------------------------------------------------------------------------------------
-// weight packing (create time)
-// ------------------------------------------------------------------------------------------------
-// Wq[dt][cb][nt][sp][r][e]: for temporal tap dt, input-channel block cb, output-channel tile nt and spatial
-// tap sp = dh*kw + dw, a tile of NPAD rows (output channels) x KB input channels, stored as the exact
-// shared-memory image the tensor core expects for a K-major operand with 128-byte (KB = 64) or 64-byte
-// (KB = 32) swizzle: the 16-byte chunk c of row r sits at chunk position c ^ (r & 7), respectively
-// c ^ ((r >> 1) & 3).  A tile, or a run of consecutive spatial taps, is then one contiguous bulk copy.
-// Zero outside the real channel extents.
-__global__ void pack_weights_kernel(const __nv_bfloat16* __restrict__ w, __nv_bfloat16* __restrict__ wq, int Cout,
-                                    int Cin, int kt, int spatial, int CB, int KB, int NT, int NPAD) {
-    const int64_t total = (int64_t)kt * CB * NT * spatial * NPAD * KB;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-        int64_t q = i;
-        const int e = (int)(q % KB); q /= KB;
-        const int r = (int)(q % NPAD); q /= NPAD;
-        const int sp = (int)(q % spatial); q /= spatial;
-        const int nt = (int)(q % NT); q /= NT;
-        const int cb = (int)(q % CB);
-        const int dt = (int)(q / CB);
-        const int chunk_stored = e >> 3;
-        const int chunk = chunk_stored ^ (KB == 64 ? (r & 7) : ((r >> 1) & 3));
-        const int ci = cb * KB + chunk * 8 + (e & 7);
-        const int co = nt * NPAD + r;
-        __nv_bfloat16 v = __float2bfloat16_rn(0.f);
-        if (ci < Cin && co < Cout) v = w[(((int64_t)co * Cin + ci) * kt + dt) * spatial + sp];
-        wq[i] = v;
-    }
-}
-
-// ------------------------------------------------------------------------------------------------
-// staging: NCTHW -> channels-last blocks, fused with the cache update
-// ------------------------------------------------------------------------------------------------
-struct StageParams {
-    const __nv_bfloat16* x;      // [N,Cin,T,H,W]
-    const __nv_bfloat16* cache;  // [N,Cin,cf,H,W] or null
-    int cf;                      // history frames the cache holds (0..tc); Z frame f < tc is cache frame f-(tc-cf) if >= 0
-    __nv_bfloat16* zs;           // [N][F][CB][H][W][KB], F = tc + T
-    __nv_bfloat16* new_cache;    // [N,Cin,tc,H,W] or null
-    int N, Cin, T, H, W, tc, CB;
-    int f_begin;                 // first Z frame to stage (tc when there is no cache and nothing older is needed)
-    int h_begin;                 // first image row of this launch (grid.y rows are staged)
-    int ring_F = 0, ring_f0 = 0; // ring_F > 0 (separate staging kernel only): zs is a frame ring of ring_F slots and
-                                 // Z frame f goes to slot (ring_f0 + f) mod ring_F
-};
-
-constexpr int STG_PX = 64;  // pixels of one image row handled per block
-
-// grid: (ceil(W/64), rows of this launch, N*(F - f_begin)*CB); block: 32 * (KB/8) threads.
-// VEC: W % 8 == 0 and all bases 16-byte aligned -> 16-byte loads along w.
-template <int KB, bool VEC>
-__global__ void __launch_bounds__(32 * (KB / 8)) stage_frames_kernel(const StageParams p) {
-    constexpr int NTHR = 32 * (KB / 8);
-    constexpr int PITCH = STG_PX / 2 + 1;  // 32-bit words per channel row (+1: bank spread)
-    __shared__ uint32_t tile[KB * PITCH];
-
-    const int F = p.tc + p.T;
-    const int nf = F - p.f_begin;
-    int z = blockIdx.z;
-    const int cb = z % p.CB;
-    z /= p.CB;
-    const int f = p.f_begin + z % nf;
-    const int n = z / nf;
-    const int h = p.h_begin + blockIdx.y;
-    const int w0 = blockIdx.x * STG_PX;
-    const int64_t HW = (int64_t)p.H * p.W;
-
-    // source frame of Z: cache frames first (oldest first), then x
-    const __nv_bfloat16* src = nullptr;  // base of channel 0 of this (n, frame); channel stride cstride
-    int64_t cstride = 0;
-    if (f < p.tc) {
-        const int cfr = f - (p.tc - p.cf);
-        if (p.cache && cfr >= 0) {
-            src = p.cache + ((int64_t)n * p.Cin * p.cf + cfr) * HW;
-            cstride = (int64_t)p.cf * HW;
-        }
-    } else {
-        src = p.x + ((int64_t)n * p.Cin * p.T + (f - p.tc)) * HW;
-        cstride = (int64_t)p.T * HW;
-    }
-    // does this frame belong to the updated cache?  new_cache[j] = Z[T + j]
-    const int jc = f - p.T;
-    __nv_bfloat16* ncdst = nullptr;
-    if (p.new_cache && jc >= 0 && jc < p.tc) ncdst = p.new_cache + ((int64_t)n * p.Cin * p.tc + jc) * HW;
-    const int64_t ncstride = (int64_t)p.tc * HW;
-
-    // ---- load phase: KB channel rows of up to 64 pixels ----
-    if (VEC) {
-        // 8 vectors of 8 pixels per row
-        for (int i = threadIdx.x; i < KB * 8; i += NTHR) {
-            const int c = i >> 3, v = i & 7;
-            const int ci = cb * KB + c;
-            const int w = w0 + v * 8;
-            uint4 val = make_uint4(0u, 0u, 0u, 0u);
-            if (w < p.W && ci < p.Cin) {
-                if (src) val = __ldg(reinterpret_cast<const uint4*>(src + ci * cstride + (int64_t)h * p.W + w));
-                if (ncdst) *reinterpret_cast<uint4*>(ncdst + ci * ncstride + (int64_t)h * p.W + w) = val;
-            }
-            uint32_t* row = tile + c * PITCH + v * 4;
-            row[0] = val.x; row[1] = val.y; row[2] = val.z; row[3] = val.w;
-        }
-    } else {
-        unsigned short* t16 = reinterpret_cast<unsigned short*>(tile);
-        for (int i = threadIdx.x; i < KB * STG_PX; i += NTHR) {
-            const int c = i / STG_PX, px = i % STG_PX;
-            const int ci = cb * KB + c;
-            const int w = w0 + px;
-            unsigned short val = 0;
-            if (w < p.W && ci < p.Cin) {
-                if (src) val = __ldg(reinterpret_cast<const unsigned short*>(src + ci * cstride + (int64_t)h * p.W + w));
-                if (ncdst) *reinterpret_cast<unsigned short*>(ncdst + ci * ncstride + (int64_t)h * p.W + w) = val;
-            }
-            t16[c * (2 * PITCH) + px] = val;
-        }
-    }
-    __syncthreads();
-
-    // ---- store phase: each thread builds the 16-byte channel octet of two neighbouring pixels ----
-    constexpr int OCT = KB / 8;
-    const int oct = threadIdx.x % OCT;
-    const int pp = threadIdx.x / OCT;  // pixel pair 0..31
-    uint32_t lo[4], hi[4];
-#pragma unroll
-    for (int k = 0; k < 4; ++k) {
-        const uint32_t a = tile[(oct * 8 + 2 * k) * PITCH + pp];      // channel 2k:   pixels (2pp, 2pp+1)
-        const uint32_t b = tile[(oct * 8 + 2 * k + 1) * PITCH + pp];  // channel 2k+1
-        lo[k] = __byte_perm(a, b, 0x5410);                            // pixel 2pp:   (ch 2k, ch 2k+1)
-        hi[k] = __byte_perm(a, b, 0x7632);                            // pixel 2pp+1
-    }
-    const int FS = p.ring_F > 0 ? p.ring_F : F;         // frame slots per sample
-    int fs = p.ring_f0 + f;
-    if (fs >= FS) fs -= FS;
-    __nv_bfloat16* dst = p.zs + ((((int64_t)n * FS + fs) * p.CB + cb) * HW + (int64_t)h * p.W) * KB;
-    const int wa = w0 + 2 * pp;
-    if (wa < p.W) *reinterpret_cast<uint4*>(dst + (int64_t)wa * KB + oct * 8) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-    if (wa + 1 < p.W)
-        *reinterpret_cast<uint4*>(dst + (int64_t)(wa + 1) * KB + oct * 8) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-}
-
-// ------------------------------------------------------------------------------------------------
-// FP32 layers on the tensor cores ("3xTF32"): packing and staging with the hi/lo split
-// ------------------------------------------------------------------------------------------------
-// The tensor core reads an FP32 operand as TF32 by ignoring its low 13 mantissa bits; what it ignores is kept
-// as a second operand, lo(v) = v - hi(v) (exact in FP32; itself truncated to TF32 when used, which leaves a
-// relative error of about 2^-21 per product).
-__device__ __forceinline__ float tf32_lo(float v) { return v - __uint_as_float(__float_as_uint(v) & 0xFFFFE000u); }
-
-// Wq[pass][dt][cb][nt][sp][r][e], e < 32 FP32 input channels of block cb: pass 0 holds lo(w) (multiplied with the
-// activations' values), passes 1 and 2 hold w (multiplied with the activations' remainders, then with their
-// values); rows of 128 bytes stored as the 128-byte-swizzled shared-memory image (16-byte chunk c of row r at
-// chunk position c ^ (r & 7)).  Zero outside the real channel extents.
-__global__ void pack_weights_f32_kernel(const float* __restrict__ w, float* __restrict__ wq, int Cout, int Cin, int kt,
-                                        int spatial, int CB, int NT, int NPAD) {
-    const int64_t total = (int64_t)3 * kt * CB * NT * spatial * NPAD * 32;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-        int64_t q = i;
-        const int e = (int)(q % 32); q /= 32;
-        const int r = (int)(q % NPAD); q /= NPAD;
-        const int sp = (int)(q % spatial); q /= spatial;
-        const int nt = (int)(q % NT); q /= NT;
-        const int cb = (int)(q % CB); q /= CB;
-        const int dt = (int)(q % kt);
-        const int pass = (int)(q / kt);
-        const int chunk = (e >> 2) ^ (r & 7);
-        const int ci = cb * 32 + chunk * 4 + (e & 3);
-        const int co = nt * NPAD + r;
-        float val = 0.f;
-        if (ci < Cin && co < Cout) {
-            val = w[(((int64_t)co * Cin + ci) * kt + dt) * spatial + sp];
-            if (pass == 0) val = tf32_lo(val);
-        }
-        wq[i] = val;
-    }
-}
-
-struct StageF32Params {
-    const float* x;          // [N,Cin,T,H,W]
-    const float* cache;      // [N,Cin,cf,H,W] or null
-    int cf;
-    float* zs;               // [N][F][2*CBr][H][W][32]: block 2*cb = the values, block 2*cb+1 = their TF32 remainders
-    float* new_cache;        // [N,Cin,tc,H,W] or null
-    int N, Cin, T, H, W, tc, CBr;
-    int f_begin;
-};
-
-// grid: (ceil(W/32), H, N*(F - f_begin)*CBr); block 256.  [32 channels][32 pixels] of an image row -> 32 pixels x
-// (32 values, 32 remainders), plus the bit-exact cache update from the same registers.
-__global__ void __launch_bounds__(256) stage_frames_f32_kernel(const StageF32Params p) {
-    __shared__ float tile[32 * 33];
-    const int F = p.tc + p.T;
-    const int nf = F - p.f_begin;
-    int z = blockIdx.z;
-    const int cb = z % p.CBr; z /= p.CBr;
-    const int f = p.f_begin + z % nf;
-    const int n = z / nf;
-    const int h = blockIdx.y;
-    const int w0 = blockIdx.x * 32;
-    const int64_t HW = (int64_t)p.H * p.W;
-    const float* src = nullptr;
-    int64_t cstride = 0;
-    if (f < p.tc) {
-        const int cfr = f - (p.tc - p.cf);
-        if (p.cache && cfr >= 0) {
-            src = p.cache + ((int64_t)n * p.Cin * p.cf + cfr) * HW;
-            cstride = (int64_t)p.cf * HW;
-        }
-    } else {
-        src = p.x + ((int64_t)n * p.Cin * p.T + (f - p.tc)) * HW;
-        cstride = (int64_t)p.T * HW;
-    }
-    const int jc = f - p.T;                               // new_cache[j] = Z[T + j]
-    float* ncdst = (p.new_cache && jc >= 0 && jc < p.tc) ? p.new_cache + ((int64_t)n * p.Cin * p.tc + jc) * HW : nullptr;
-    const int64_t ncstride = (int64_t)p.tc * HW;
-    for (int i = threadIdx.x; i < 32 * 32; i += 256) {
-        const int c = i >> 5, px = i & 31;
-        const int ci = cb * 32 + c, w = w0 + px;
-        float v = 0.f;
-        if (w < p.W && ci < p.Cin) {
-            if (src) v = __ldg(src + ci * cstride + (int64_t)h * p.W + w);
-            if (ncdst) ncdst[ci * ncstride + (int64_t)h * p.W + w] = v;
-        }
-        tile[c * 33 + px] = v;
-    }
-    __syncthreads();
-    const int px = threadIdx.x >> 3, q = threadIdx.x & 7;    // pixel, channel quad
-    const int w = w0 + px;
-    if (w < p.W) {
-        float4 hi, lo;
-        hi.x = tile[(4 * q + 0) * 33 + px]; hi.y = tile[(4 * q + 1) * 33 + px];
-        hi.z = tile[(4 * q + 2) * 33 + px]; hi.w = tile[(4 * q + 3) * 33 + px];
-        lo.x = tf32_lo(hi.x); lo.y = tf32_lo(hi.y); lo.z = tf32_lo(hi.z); lo.w = tf32_lo(hi.w);
-        float* dst = p.zs + ((((int64_t)n * F + f) * (2 * p.CBr) + 2 * cb) * HW + (int64_t)h * p.W + w) * 32 + 4 * q;
-        *reinterpret_cast<float4*>(dst) = hi;
-        *reinterpret_cast<float4*>(dst + HW * 32) = lo;
-    }
-}
-
-// ------------------------------------------------------------------------------------------------
-// frame rings: the inverse move (ring -> NCTHW) and the nearest-neighbour upsample between rings
-// ------------------------------------------------------------------------------------------------
-struct RingGeom {
-    __nv_bfloat16* base;         // [N][F][CB][H][W][KB]
-    int N, F, CB, H, W, KB;
-};
-
-// grid: (ceil(W/64), H, N*T*CB); block 256.  [64 pixels][KB channels] of an image row -> KB channel rows of 64 pixels.
-template <int KB>
-__global__ void __launch_bounds__(256) ring_store_kernel(const RingGeom r, int slot0, int T, int C, __nv_bfloat16* __restrict__ y) {
-    constexpr int PITCH = KB + 2;                         // BF16 elements per pixel row (+2: bank spread)
-    __shared__ __align__(16) unsigned short tile[STG_PX * PITCH];
-    int z = blockIdx.z;
-    const int cb = z % r.CB; z /= r.CB;
-    const int t = z % T;
-    const int n = z / T;
-    const int h = blockIdx.y;
-    const int w0 = blockIdx.x * STG_PX;
-    const int64_t HW = (int64_t)r.H * r.W;
-    int fs = slot0 + t;
-    if (fs >= r.F) fs -= r.F;
-    const __nv_bfloat16* src = r.base + ((((int64_t)n * r.F + fs) * r.CB + cb) * HW + (int64_t)h * r.W + w0) * KB;
-    const int npx = (r.W - w0 < STG_PX) ? r.W - w0 : STG_PX;
-    constexpr int OCT = KB / 8;
-    for (int i = threadIdx.x; i < npx * OCT; i += 256) {   // contiguous 16-byte chunks
-        const int px = i / OCT, oct = i % OCT;
-        const uint4 u = __ldg(reinterpret_cast<const uint4*>(src) + i);
-        uint32_t* d = reinterpret_cast<uint32_t*>(tile + px * PITCH + oct * 8);
-        d[0] = u.x; d[1] = u.y; d[2] = u.z; d[3] = u.w;
-    }
-    __syncthreads();
-    for (int i = threadIdx.x; i < KB * STG_PX; i += 256) {
-        const int c = i / STG_PX, px = i % STG_PX;
-        if (px < npx)
-            reinterpret_cast<unsigned short*>(y)[(((int64_t)n * C + cb * KB + c) * T + t) * HW + (int64_t)h * r.W + w0 + px] =
-                tile[px * PITCH + c];
-    }
-}
-
-// One thread per 16-byte chunk of the source frames; each chunk is written to 2x2 pixels of rt output frames.
-__global__ void __launch_bounds__(256) ring_upsample_kernel(const RingGeom in, int in_slot0, const RingGeom out, int out_slot0,
-                                                            int T, int rt) {
-    const int OCT = in.KB / 8;
-    const int64_t per_frame = (int64_t)in.CB * in.H * in.W * OCT;
-    const int64_t total = (int64_t)in.N * T * per_frame;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-        int64_t q = i;
-        const int oct = (int)(q % OCT); q /= OCT;
-        const int w = (int)(q % in.W); q /= in.W;
-        const int h = (int)(q % in.H); q /= in.H;
-        const int cb = (int)(q % in.CB); q /= in.CB;
-        const int t = (int)(q % T);
-        const int n = (int)(q / T);
-        int fs = in_slot0 + t;
-        if (fs >= in.F) fs -= in.F;
-        const uint4 u = __ldg(reinterpret_cast<const uint4*>(
-            in.base + ((((int64_t)n * in.F + fs) * in.CB + cb) * in.H * in.W + (int64_t)h * in.W + w) * in.KB + oct * 8));
-        for (int j = 0; j < rt; ++j) {
-            int os = (out_slot0 + t * rt + j) % out.F;
-            __nv_bfloat16* o = out.base + ((((int64_t)n * out.F + os) * out.CB + cb) * out.H * out.W +
-                                           (int64_t)(2 * h) * out.W + 2 * w) * out.KB + oct * 8;
-            *reinterpret_cast<uint4*>(o) = u;
-            *reinterpret_cast<uint4*>(o + out.KB) = u;
-            *reinterpret_cast<uint4*>(o + (int64_t)out.W * out.KB) = u;
-            *reinterpret_cast<uint4*>(o + (int64_t)(out.W + 1) * out.KB) = u;
-        }
-    }
-}
-
-// Addresses of one staging task: image row h, pixels [w0, w0+64), channel block cb of Z frame f of sample n.
-struct StageTask {
-    const __nv_bfloat16* src;   // channel 0 of the source frame at (h, 0), or null (absent history: zeros)
-    int64_t cstride;            // source channel stride
-    __nv_bfloat16* ncdst;       // channel 0 of the new-cache frame at (h, 0), or null
-    __nv_bfloat16* dst;         // channels-last destination of pixel (h, 0)
-    int cb, w0;
-};
-
-__device__ __forceinline__ StageTask make_stage_task(const StageParams& p, int KB, int n, int f, int cb, int h, int w0) {
-    StageTask t;
-    const int F = p.tc + p.T;
-    const int64_t HW = (int64_t)p.H * p.W;
-    t.src = nullptr;
-    t.cstride = 0;
-    if (f < p.tc) {
-        const int cfr = f - (p.tc - p.cf);
-        if (p.cache && cfr >= 0) {
-            t.src = p.cache + ((int64_t)n * p.Cin * p.cf + cfr) * HW + (int64_t)h * p.W;
-            t.cstride = (int64_t)p.cf * HW;
-        }
-    } else {
-        t.src = p.x + ((int64_t)n * p.Cin * p.T + (f - p.tc)) * HW + (int64_t)h * p.W;
-        t.cstride = (int64_t)p.T * HW;
-    }
-    const int jc = f - p.T;
-    t.ncdst = nullptr;
-    if (p.new_cache && jc >= 0 && jc < p.tc) t.ncdst = p.new_cache + ((int64_t)n * p.Cin * p.tc + jc) * HW + (int64_t)h * p.W;
-    t.dst = p.zs + ((((int64_t)n * F + f) * p.CB + cb) * HW + (int64_t)h * p.W) * KB;
-    t.cb = cb;
-    t.w0 = w0;
-    return t;
-}
-
-// The same tile move as stage_frames_kernel<KB, true>, run by the 128 threads of the stager warps inside the
-// convolution kernel (cooperative staging): [KB channels][64 pixels] of an image row -> [64 pixels][KB channels],
-// plus the cache update when the frame belongs to the new cache.  Split in two so that the loads of several
-// tasks can be in flight before the first is written: stage_task_load fills val[], stage_task_store moves it
-// through `tile` (StagerGeom<KB>::TILE_WORDS words of shared memory; phases separated by the stagers' named
-// barrier, id 2).
-__device__ __forceinline__ void stager_bar() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
-
-// PX: pixels of an image row per task.  64 for 64-channel blocks; 128 for 32-channel blocks, so that a task moves
-// the same 8 KB either way (the per-task barriers and address arithmetic are what limits a stager team).
-template <int KB>
-struct StagerGeom {
-    static constexpr int PX = (KB == 64) ? 64 : 128;
-    static constexpr int VPR = PX / 8;                    // 16-byte vectors per channel row
-    static constexpr int NLD = KB * VPR / 128;            // vectors per thread
-    static constexpr int PITCH = PX / 2 + 1;              // 32-bit words per channel row in the tile (+1: bank spread)
-    static constexpr int TILE_WORDS = KB * PITCH;
-};
-
-template <int KB>
-__device__ __forceinline__ void stage_task_load(const StageParams& p, const StageTask& t, int tid,
-                                                uint4 (&val)[StagerGeom<KB>::NLD]) {
-    using G = StagerGeom<KB>;
-#pragma unroll
-    for (int k = 0; k < G::NLD; ++k) {
-        const int i = tid + 128 * k;
-        const int c = i / G::VPR, v = i % G::VPR;
-        const int ci = t.cb * KB + c;
-        const int w = t.w0 + v * 8;
-        val[k] = make_uint4(0u, 0u, 0u, 0u);
-        if (w < p.W && ci < p.Cin && t.src) val[k] = __ldg(reinterpret_cast<const uint4*>(t.src + ci * t.cstride + w));
-    }
-}
-
-template <int KB>
-__device__ __forceinline__ void stage_task_store(const StageParams& p, const StageTask& t, int tid,
-                                                 const uint4 (&val)[StagerGeom<KB>::NLD], uint32_t* tile) {
-    using G = StagerGeom<KB>;
-    constexpr int OCT = KB / 8;
-    const int64_t ncstride = (int64_t)p.tc * p.H * p.W;
-#pragma unroll
-    for (int k = 0; k < G::NLD; ++k) {
-        const int i = tid + 128 * k;
-        const int c = i / G::VPR, v = i % G::VPR;
-        const int ci = t.cb * KB + c;
-        const int w = t.w0 + v * 8;
-        if (t.ncdst && w < p.W && ci < p.Cin) *reinterpret_cast<uint4*>(t.ncdst + ci * ncstride + w) = val[k];
-        uint32_t* row = tile + c * G::PITCH + v * 4;
-        row[0] = val[k].x; row[1] = val[k].y; row[2] = val[k].z; row[3] = val[k].w;
-    }
-    stager_bar();
-#pragma unroll
-    for (int k = 0; k < (G::PX / 2 * OCT) / 128; ++k) {
-        const int vt = tid + 128 * k;
-        const int oct = vt % OCT, pp = vt / OCT;
-        uint32_t lo[4], hi[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const uint32_t a = tile[(oct * 8 + 2 * q) * G::PITCH + pp];
-            const uint32_t b = tile[(oct * 8 + 2 * q + 1) * G::PITCH + pp];
-            lo[q] = __byte_perm(a, b, 0x5410);
-            hi[q] = __byte_perm(a, b, 0x7632);
-        }
-        const int wa = t.w0 + 2 * pp;
-        if (wa < p.W) *reinterpret_cast<uint4*>(t.dst + (int64_t)wa * KB + oct * 8) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-        if (wa + 1 < p.W)
-            *reinterpret_cast<uint4*>(t.dst + (int64_t)(wa + 1) * KB + oct * 8) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-    }
-    stager_bar();                                           // the tile may be overwritten by the next task
-}
-
-// ------------------------------------------------------------------------------------------------
-// PTX wrappers (sm_100a)
-// ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.b32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok;
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];" ::
-            "r"(dst),
-        "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(bar)
-        : "memory");
-}
-__device__ __forceinline__ void tma_store_3d(const CUtensorMap* tm, uint32_t src, int c0, int c1, int c2) {
-    asm volatile("cp.async.bulk.tensor.3d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4}], [%1];" ::"l"(tm),
-                 "r"(src), "r"(c0), "r"(c1), "r"(c2)
-                 : "memory");
-}
-__device__ __forceinline__ void tma_load_5d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2,
-                                            int c3, int c4) {
-    asm volatile(
-        "cp.async.bulk.tensor.5d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5, "
-        "%6}], [%7];" ::"r"(dst),
-        "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar)
-        : "memory");
-}
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-                 "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
-}
-// ---- CTA pairs (cta_group::2): the two CTAs of a cluster run one 256-pixel tile, each holding its own 128-pixel
-// activation tile and half of the weight tile; the leader (cluster rank 0) issues the MMAs for both.
-constexpr uint32_t PEER_MASK = 0xFEFFFFFFu;   // clears the CTA-rank bit of a shared::cluster address: the leader's copy
-__device__ __forceinline__ uint32_t cluster_rank() {
-    uint32_t r;
-    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
-    return r;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-// TMA loads whose completion is counted on the LEADER's mbarrier (same offset, rank bit cleared)
-__device__ __forceinline__ void tma_load_5d_pair(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1, int c2,
-                                                 int c3, int c4) {
-    asm volatile(
-        "cp.async.bulk.tensor.5d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, "
-        "%4, %5, %6}], [%7];" ::"r"(dst),
-        "l"(tm), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4), "r"(bar & PEER_MASK)
-        : "memory");
-}
-__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], "
-        "[%4];" ::"r"(dst),
-        "l"(tm), "r"(c0), "r"(c1), "r"(bar & PEER_MASK)
-        : "memory");
-}
-// an arrival on the leader's copy of a barrier, from either CTA of the pair
-__device__ __forceinline__ void mbar_arrive_leader(uint32_t bar) {
-    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar & PEER_MASK) : "memory");
-}
-// commit of the leader's MMAs: one arrival on the barrier at this offset in BOTH CTAs
-__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
-                 "h"((unsigned short)3)
-                 : "memory");
-}
-// D[tmem of both CTAs] (+)= A * B^T with M = 256 (128 rows per CTA), each CTA contributing half of B's rows
-__device__ __forceinline__ void tc_mma_bf16_pair(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
-                                                 uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
-        "setp.ne.b32 p, %6, 0;\n\t"
-        "mov.b64 da, {%1, %2};\n\t"
-        "mov.b64 db, {%3, %4};\n\t"
-        "tcgen05.mma.cta_group::2.kind::f16 [%0], da, db, %5, p;\n\t}" ::"r"(d_tmem),
-        "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-
-__device__ __forceinline__ void tc_mma_tf32_pair(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
-                                                 uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
-        "setp.ne.b32 p, %6, 0;\n\t"
-        "mov.b64 da, {%1, %2};\n\t"
-        "mov.b64 db, {%3, %4};\n\t"
-        "tcgen05.mma.cta_group::2.kind::tf32 [%0], da, db, %5, p;\n\t}" ::"r"(d_tmem),
-        "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-
-// One lane of a fully converged warp; the others get 0.  Keeps the surrounding code warp-uniform so that
-// descriptors and addresses can live in uniform registers.
-__device__ __forceinline__ uint32_t elect_one() {
-    uint32_t pred;
-    asm volatile(
-        "{\n\t.reg .pred P;\n\t"
-        "elect.sync _|P, 0xffffffff;\n\t"
-        "selp.b32 %0, 1, 0, P;\n\t}"
-        : "=r"(pred));
-    return pred;
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// D[tmem] (+)= A[smem] * B[smem]^T, M = 128, K = 16, BF16 inputs, FP32 accumulate.  The 64-bit shared-memory
-// descriptors are passed as halves so that stepping along K or to another pixel block is one 32-bit add.
-__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
-                                            uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
-        "setp.ne.b32 p, %6, 0;\n\t"
-        "mov.b64 da, {%1, %2};\n\t"
-        "mov.b64 db, {%3, %4};\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n\t}" ::"r"(d_tmem),
-        "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-// FP32 operands read as TF32 (the low 13 mantissa bits are ignored), K = 8 per instruction, FP32 accumulate
-__device__ __forceinline__ void tc_mma_tf32(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
-                                            uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t.reg .b64 da, db;\n\t"
-        "setp.ne.b32 p, %6, 0;\n\t"
-        "mov.b64 da, {%1, %2};\n\t"
-        "mov.b64 db, {%3, %4};\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], da, db, %5, p;\n\t}" ::"r"(d_tmem),
-        "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-template <bool TF32>
-__device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
-                                       uint32_t idesc, uint32_t accumulate) {
-    if (TF32) tc_mma_tf32(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate);
-    else tc_mma_bf16(d_tmem, a_lo, a_hi, b_lo, b_hi, idesc, accumulate);
-}
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
-          "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
-          "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-        : "r"(taddr)
-        : "memory");
-}
-__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&v)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, "
-        "[%16];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
-          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
-        : "r"(taddr)
-        : "memory");
-}
-__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-__device__ __forceinline__ void tma_store_5d(const CUtensorMap* tm, uint32_t src, int c0, int c1, int c2, int c3, int c4) {
-    asm volatile(
-        "cp.async.bulk.tensor.5d.global.shared::cta.tile.bulk_group [%0, {%2, %3, %4, %5, %6}], [%1];" ::"l"(tm),
-        "r"(src), "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(c4)
-        : "memory");
-}
-__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
-__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void epi_bar_sync() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-
-// Four 8x8 16-bit matrices, transposed on the way from shared memory to registers; lane l gives the address of
-// row l%8 of matrix l/8.  The registers come out in the fragment layout stmatrix takes.
-__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t (&r)[4]) {
-    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0, %1, %2, %3}, [%4];"
-                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
-                 : "r"(addr)
-                 : "memory");
-}
-__device__ __forceinline__ void stmatrix_x4(uint32_t addr, const uint32_t (&r)[4]) {
-    asm volatile("stmatrix.sync.aligned.m8n8.x4.shared.b16 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(r[0]), "r"(r[1]),
-                 "r"(r[2]), "r"(r[3])
-                 : "memory");
-}
-
-// ------------------------------------------------------------------------------------------------
-// the implicit-GEMM kernel
-// ------------------------------------------------------------------------------------------------
-struct TcParams {
-    int N, T, H, W, Cout;
-    int F;            // frames of Z held in the staging buffer (kt-1 + T)
-    int kt, kh, kw;
-    int CB;           // input-channel blocks of KB
-    int NT, NPAD;     // output-channel tiles and their (padded) width, NPAD % 16 == 0, <= 256
-    int tiles_h, tiles_w, total_tiles;   // tile rows handled by this launch, tile columns, tiles of this launch
-    int ty_begin;                        // first tile row of this launch (a launch may cover a band of the image)
-    int first_frame;  // Z frames below this are absent (first chunk): their taps are skipped
-    int out_f32;      // 1: out is FP32, 0: BF16
-    int per_tap_a;    // 1: one A load per tap (box without halo), 0: one halo load per (dt, ci-block)
-    int TPB;          // spatial taps per weight stage (1 or kw); kh*kw % TPB == 0
-    int epi_tma;      // 1: epilogue stages BF16 tiles in shared memory and stores them with TMA; 0: direct stores;
-                      // 2: the output is a frame ring (channels-last), staged pixel-major and stored with TMA
-    int ECH;          // output channels per epilogue chunk (32 or 16) when epi_tma
-    int SA, SB, ACC;  // ring depths and accumulator buffers
-    uint32_t a_slot, b_slot, b_tap;  // bytes per ring slot (multiples of 1024) and per tap inside a weight slot
-    uint32_t b_src_tap;       // bytes per tap in the packed weights when that differs from b_tap (split_n), else 0
-    int split_n;              // 1: NT and NPAD describe half-width output-channel tiles of a layer packed at full width
-    uint32_t e_slot;          // bytes of one epilogue staging buffer (two are allocated when epi_tma)
-    uint32_t raw_slot;        // fused mode: bytes of one raw [32 ch][BH rows][32 px] box (two are allocated)
-    int tc, cf;               // fused mode: kt-1 and the history frames the cache holds; Z frame f < tc is cache frame f-(tc-cf)
-    uint32_t tmem_cols;       // power of two >= NB*NPAD*ACC
-    long long wait_limit_clk; // bound of every mbarrier wait, in SM clocks
-    unsigned int* band_ctr;   // cooperative staging: per 16-row band, the number of CTAs that have staged their share
-    int nbands;               // cooperative staging: bands of the image (= tile rows)
-    // general geometry (Eq. (2) with the layer's own padding and dilation, Eq. (1) with d_t); when `general` is 0
-    // the kernel uses pad = (k-1)/2 and unit dilation.  H and W above are the OUTPUT extents; the input extents
-    // only live in the tensor map.  Spatial stride > 1 is served by the per-tap mode with a strided tensor map.
-    int general, pad_h, pad_w, dil_h, dil_w, dil_t, str_h, str_w, str_t;   // T above counts OUTPUT frames (T_o)
-    int f0;                   // ring input: the slot of Z frame 0; Z frame f lives in slot (f0 + f) mod F (0 for a staged copy)
-    const __nv_bfloat16* res; // optional residual ring [N][res_F][res_CB][H][W][res_KB] holding Cout channels, or null
-    int res_F, res_f0, res_CB, res_KB;   // residual frame t is slot (res_f0 + t) mod res_F
-    int out_F, out_f0, out_KB;           // epi_tma == 2: output frame t goes to slot (out_f0 + t) mod out_F
-    int act;                             // 1: SiLU on conv + bias before the output rounding (and before the residual)
-    int up_rt;                           // epi_tma == 2, > 0: the output ring is 2H x 2W; every pixel is written 2x2 times into
-                                         // each of the up_rt slots (out_f0 + t*up_rt + j) mod out_F (nearest-neighbour upsample)
-    const float* bias;        // [NT*NPAD]
-    const uint8_t* wq;        // packed weight tiles [dt][cb][nt][sp] of b_tap bytes each
-    void* out;
-    unsigned int* status;     // 0 = fine; else (block << 8) | site
-};
-
-enum : uint32_t {
-    SITE_A_EMPTY = 1, SITE_B_EMPTY = 2, SITE_A_FULL = 3, SITE_B_FULL = 4, SITE_ACC_EMPTY = 5, SITE_ACC_FULL = 6,
-    SITE_RAW_EMPTY = 7, SITE_RAW_FULL = 8, SITE_BAND = 9
-};
-
-constexpr int TC_THREADS = 256;
-constexpr int TC_THREADS_FUSED = 384;    // + 4 transposer warps
-constexpr int RAW_PX = 32;               // pixels per row of a raw box (64 bytes), starting 8 pixels left of the tile
-constexpr int TC_MAX_STAGES = 12;
-constexpr int TC_BIAS_SMEM = 512;
-
-struct TcShared {  // placed after the rings
-    uint64_t full_a[TC_MAX_STAGES], empty_a[TC_MAX_STAGES];
-    uint64_t full_b[TC_MAX_STAGES], empty_b[TC_MAX_STAGES];
-    uint64_t acc_full[2], acc_empty[2];
-    uint64_t raw_full[2], raw_empty[2];
-    uint32_t tmem_base;
-    volatile int abort_flag;
-    alignas(16) float bias_s[TC_BIAS_SMEM];   // the layer's padded bias when it fits (the epilogue reads it once per element)
-};
-
-// Bounded wait.  Returns false when the limit expired or another role of this CTA aborted.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, TcShared* sh, const TcParams& p, uint32_t site) {
-    const uint32_t b = smem_u32(bar);
-    if (mbar_try_wait(b, parity)) return true;
-    long long t0 = 0;
-    for (uint32_t it = 1;; ++it) {
-        if (mbar_try_wait(b, parity)) return true;
-        if ((it & 63u) == 0u) {
-            if (sh->abort_flag) return false;
-            const long long now = clock64();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > p.wait_limit_clk) {
-                sh->abort_flag = 1;
-                atomicCAS(p.status, 0u, (blockIdx.x << 8) | site);
-                return false;
-            }
-        }
-    }
-}
-
-// After an abort: give copies in flight a bounded time to land before the CTA goes away.
-__device__ __forceinline__ void drain_delay() {
-    const long long t0 = clock64();
-    while (clock64() - t0 < 400000) __nanosleep(1000);
-}
-
-__device__ __forceinline__ uint32_t make_desc_hi(uint32_t sbo_bytes, uint32_t layout_type) {
-    // upper word of a shared-memory matrix descriptor: bits 32-45 stride-dimension byte offset >> 4,
-    // bits 46-47 descriptor version 1, bits 61-63 swizzle mode
-    return ((sbo_bytes >> 4) & 0x3FFFu) | (1u << 14) | (layout_type << 29);
-}
-__device__ __forceinline__ uint32_t make_desc_lo(uint32_t addr) {
-    // lower word: bits 0-13 start address >> 4, bits 16-29 leading-dimension byte offset >> 4 (unused for
-    // swizzled K-major operands; canonical value 1)
-    return ((addr & 0x3FFFFu) >> 4) | (1u << 16);
-}
-
-// Residual of one pixel: 32 consecutive channels (64 bytes) starting at channel co0 of a frame ring, as 16 BF16
-// pairs.  res_row addresses channel block 0 of the pixel's image row; zeros when there is no residual or the
-// pixel lies outside the image.
-__device__ __forceinline__ void load_res32(const __nv_bfloat16* res_row, bool valid, int w, int co0, const TcParams& p,
-                                           int64_t HW, uint32_t (&rr)[16]) {
-    if (res_row && valid) {
-        const uint4* src = reinterpret_cast<const uint4*>(res_row + ((int64_t)(co0 / p.res_KB) * HW + w) * p.res_KB +
-                                                          (co0 % p.res_KB));
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            const uint4 u = __ldg(src + c);
-            rr[4 * c] = u.x; rr[4 * c + 1] = u.y; rr[4 * c + 2] = u.z; rr[4 * c + 3] = u.w;
-        }
-    } else {
-#pragma unroll
-        for (int j = 0; j < 16; ++j) rr[j] = 0u;
-    }
-}
-
-// Two neighbouring output channels: round conv + bias to BF16 once; with a residual, add it to that rounded value
-// in FP32 and round again (the result of a BF16 convolution followed by a BF16 addition).
-__device__ __forceinline__ float silu_f32(float v) { return v / (1.f + __expf(-v)); }
-
-__device__ __forceinline__ uint32_t epi_pair(float a0, float a1, uint32_t res_pair, bool has_res, bool act = false) {
-    if (act) { a0 = silu_f32(a0); a1 = silu_f32(a1); }      // optional SiLU on conv + bias, in FP32, before the one rounding
-    __nv_bfloat162 o = __floats2bfloat162_rn(a0, a1);
-    if (has_res) {
-        const float2 of = __bfloat1622float2(o);
-        const float2 rf = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&res_pair));
-        o = __floats2bfloat162_rn(of.x + rf.x, of.y + rf.y);
-    }
-    return *reinterpret_cast<const uint32_t*>(&o);
-}
-
-// KB: input channels per K block (64 -> 128-byte swizzle, 32 -> 64-byte swizzle).  NB: 128-pixel blocks per tile.
-// KS/TPBC: compile-time spatial kernel size (kh = kw = KS) and taps per weight stage, which turn the tap loop
-// into straight-line code with immediate descriptor offsets; KS = 0 keeps everything run-time (any odd kh, kw,
-// and the per-tap A mode).
-// FUSED: no staging copy; tm_a is x as (w, h, t, c, n), tm_c the cache as (w, h, frame, c, n); needs KB = 32.
-// COOP: cooperative staging - there is no separate staging kernel; four extra warps of every CTA move the
-// channels-last copy of [cache ; x] (and the cache update) band by band of 16 image rows, ahead of the tiles that
-// read it, so that this HBM-bound work hides under the tensor-core work of the same kernel.  A band is usable
-// when every CTA has signalled it (release: fence + atomic; acquire: polled load + proxy fence before the TMA
-// loads).  All CTAs are co-resident (grid <= SM count, 1 CTA per SM) and stagers never wait on consumers, so the
-// dependency is acyclic; the wait is bounded like every other.
-// TF32 (FP32 layers, "3xTF32"): KB = 64 then means 128-byte rows of 32 FP32 channels.  An FP32 product a*w is
-// evaluated as hi(a)*lo(w) + lo(a)*hi(w) + hi(a)*hi(w) with hi = the TF32 truncation the tensor core applies by
-// itself and lo = the FP32 remainder, staged and packed explicitly: the staging copy holds two blocks per channel
-// block (a, a - hi(a)), the packed weights three images (lo(w), w, w).  The whole K loop runs three times, one
-// pass per term, the two small correction terms first: the tensor core's FP32 accumulation truncates, which
-// costs a fraction of the accumulator's last bit per step, so the long chain of full-size terms is kept as short
-// as it can be and the corrections are summed while the accumulator is still 2^-11 of its final size.
-// PAIR (cta_group::2): launched in clusters of two CTAs.  A tile is 16 rows x 16*NB pixels; CTA r of the pair loads
-// the halo tile of pixel columns 8*NB*r .. and rows r*NPAD/2.. of every weight tile (tm_c is then a 2-D map over the
-// packed weights); the leader issues MMAs with M = 256 that read both CTAs' shared memory and fill both CTAs'
-// tensor memory, so that per SM and MMA only half of the weight tile crosses L2 -> shared memory and the
-// shared-memory read port.  Loads of both CTAs are counted on the leader's "full" barriers; the leader's commits
-// arrive on the "empty" and "accumulator full" barriers of both CTAs; both epilogues arrive on the leader's
-// "accumulator empty" barrier.
-template <int KB, int NB, int KS, int TPBC, bool FUSED, bool COOP, bool TF32 = false, bool PAIR = false>
-__global__ void __launch_bounds__((FUSED || COOP) ? TC_THREADS_FUSED : TC_THREADS, 1)
-conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged activations (c, w, h, cb, n*F+f), or x
-                      const __grid_constant__ CUtensorMap tm_c,   // fused mode: the cache; PAIR: the packed weights
-                      const __grid_constant__ CUtensorMap tm_o,   // out (w, h, t, co, n); used when p.epi_tma
-                      const TcParams p, const StageParams sp) {
-    static_assert(!(FUSED && COOP), "one or the other");
-    static_assert(!FUSED || KB == 32, "the fused mode transposes 32-channel blocks");
-    static_assert(!TF32 || (KB == 64 && !FUSED && !COOP), "FP32 layers: 128-byte rows, plain variant");
-    static_assert(!PAIR || (KS > 0 && !FUSED), "CTA pairs: straight-line taps");
-    // (TF32 layers always write FP32 through the direct-store epilogue, which is where the two accumulators of the
-    // last pass are added)
-    constexpr uint32_t ROWB = KB * 2;                       // bytes per pixel row (one swizzle span)
-    constexpr uint32_t LAYOUT = (KB == 64) ? 2u : 4u;       // 128-byte / 64-byte swizzle
-    constexpr uint32_t B_SBO = 8 * ROWB;                    // 8-row group pitch of the weight tile
-    constexpr int KSTEPS = KB / 16;
-    constexpr int TW = 8 * NB;                              // tile width in pixels; tile height is 16
-    constexpr int NI = (NB >= 2) ? 2 : 1;                   // MMA-issuing warps (2 and 3), each owning NB/NI pixel blocks
-    constexpr int NBW = NB / NI;
-    constexpr int ASETS = TF32 ? 2 : 1;                     // accumulators per tile buffer (TF32: the last pass uses two)
-    constexpr int TWT = PAIR ? 2 * TW : TW;                 // tile width in the tile index space (a pair shares a tile)
-    const uint32_t rank = PAIR ? cluster_rank() : 0u;       // 0 = leader
-    const int cta_lin = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;   // tiles are dealt to clusters
-    const int cta_cnt = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
-    const int wofs = PAIR ? TW * (int)rank : 0;             // this CTA's pixel columns inside the tile
-
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t* ring_a = smem;
-    uint8_t* ring_b = ring_a + (size_t)p.SA * p.a_slot;
-    uint8_t* epi_buf = ring_b + (size_t)p.SB * p.b_slot;
-    uint8_t* ring_raw = epi_buf + (p.epi_tma ? 2 * (size_t)p.e_slot : 0);
-    uint8_t* dummy = ring_raw + (FUSED ? 2 * (size_t)p.raw_slot : 0);   // 2 KB sink for the unused rows of edge blocks
-    uint32_t* coop_tile = reinterpret_cast<uint32_t*>(ring_raw);          // COOP: the stagers' transposition tile (<= 9216 bytes)
-    TcShared* sh = reinterpret_cast<TcShared*>(dummy + (FUSED ? 2048 : 0) + (COOP ? 9216 : 0));
-
-    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);  // provably warp-uniform
-    const int lane = threadIdx.x & 31;
-    const int ph = p.general ? p.pad_h : (p.kh - 1) / 2, pw = p.general ? p.pad_w : (p.kw - 1) / 2;
-    const int dlh = p.general ? p.dil_h : 1, dlw = p.general ? p.dil_w : 1, dlt = p.general ? p.dil_t : 1;
-    const int sth = p.general ? p.str_h : 1, stw = p.general ? p.str_w : 1;      // > 1 only in the per-tap mode
-    const int stt = p.general ? p.str_t : 1;                // temporal stride: output frame t reads Z frames t*stt + dt*dlt
-    const int BW = p.per_tap_a ? TW : TW + (p.kw - 1) * dlw;        // pixels per smem image row
-    const int BH = p.per_tap_a ? 16 : 16 + (p.kh - 1) * dlh;
-    const int spatial = p.kh * p.kw;
-
-    if (threadIdx.x == 0) {
-        for (int i = 0; i < p.SA; ++i) { mbar_init(smem_u32(&sh->full_a[i]), FUSED ? 4 : 1); mbar_init(smem_u32(&sh->empty_a[i]), NI); }
-        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&sh->raw_full[i]), 1); mbar_init(smem_u32(&sh->raw_empty[i]), 4); }
-        for (int i = 0; i < p.SB; ++i) { mbar_init(smem_u32(&sh->full_b[i]), 1); mbar_init(smem_u32(&sh->empty_b[i]), NI); }
-        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&sh->acc_full[i]), NI); mbar_init(smem_u32(&sh->acc_empty[i]), PAIR ? 8 : 4); }
-        sh->abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (PAIR) cluster_sync_all();   // both CTAs' barriers exist before anything of the peer can arrive on them
-    if (warp == 3) {
-        if (PAIR) {
-            asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)),
-                         "r"(p.tmem_cols)
-                         : "memory");
-            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-        } else {
-            asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)),
-                         "r"(p.tmem_cols)
-                         : "memory");
-            asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-        }
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = sh->tmem_base;
-    // Programmatic dependent launch: everything above (barriers, tensor memory) touched no global data, so it may
-    // run while the previous kernel of the stream is still finishing.  From here on the kernel reads what that
-    // kernel wrote: wait for it (returns at once when the launch carried no such dependency), and let the next
-    // kernel of the stream start its own set-up as soon as CTAs of this one retire.
-    asm volatile("griddepcontrol.wait;" ::: "memory");
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-
-    // ---------------------------------------------------------------- A producer
-    if (warp == 0) {
-        if (lane == 0 && FUSED) {
-            // raw boxes [32 ch][BH rows][32 px] straight from x or the cache: tap dt of output frame t reads frame
-            // t+dt of Z = [cache ; x]; columns start 8 pixels left of the tile so that the start is 16-byte aligned
-            asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_a) : "memory");
-            asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_c) : "memory");
-            const uint32_t raw_bytes = (uint32_t)KB * BH * RAW_PX * 2;
-            int s = 0;
-            uint32_t phase = 1;
-            bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
-                int r = tile / p.NT;
-                const int t = r % p.T; r /= p.T;
-                const int tx = r % p.tiles_w; r /= p.tiles_w;
-                const int ty = p.ty_begin + r % p.tiles_h;
-                const int n = r / p.tiles_h;
-                const int h0 = ty * 16, w0 = tx * TW;
-                const int dt0 = (p.first_frame - t * stt > 0) ? (p.first_frame - t * stt + dlt - 1) / dlt : 0;   // first tap whose frame exists
-                for (int dt = dt0; ok && dt < p.kt; ++dt)
-                    for (int cb = 0; ok && cb < p.CB; ++cb) {
-                        if (!(ok = mbar_wait(&sh->raw_empty[s], phase, sh, p, SITE_RAW_EMPTY))) break;
-                        const uint32_t bar = smem_u32(&sh->raw_full[s]);
-                        mbar_expect_tx(bar, raw_bytes);
-                        const int fz = t + dt;
-                        const uint32_t dst = smem_u32(ring_raw + (size_t)s * p.raw_slot);
-                        if (fz < p.tc) tma_load_5d(dst, &tm_c, bar, w0 - 8, h0 - ph, fz - (p.tc - p.cf), cb * KB, n);
-                        else tma_load_5d(dst, &tm_a, bar, w0 - 8, h0 - ph, fz - p.tc, cb * KB, n);
-                        s ^= 1;
-                        if (s == 0) phase ^= 1;
-                    }
-            }
-            if (!ok) drain_delay();
-        } else if (lane == 0) {
-            asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_a) : "memory");
-            const uint32_t a_bytes = (uint32_t)BW * BH * ROWB;
-            int s = 0;
-            uint32_t phase = 1;
-            bool ok = true;
-            int bands_ready = 0;                       // COOP: bands [0, bands_ready) are known to be staged
-            for (int tile = cta_lin; ok && tile < p.total_tiles; tile += cta_cnt) {
-                int r = tile / p.NT;
-                const int t = r % p.T; r /= p.T;
-                const int tx = r % p.tiles_w; r /= p.tiles_w;
-                const int ty = p.ty_begin + r % p.tiles_h;
-                const int n = r / p.tiles_h;
-                const int h0 = ty * 16, w0 = tx * TWT + wofs;
-                if (COOP) {
-                    // the halo of tile row ty reaches into bands ty-1 .. ty+1
-                    const int need = (ty + 2 < p.nbands) ? ty + 2 : p.nbands;
-                    if (bands_ready < need) {
-                        const long long t0 = clock64();
-                        while (ok && bands_ready < need) {
-                            unsigned int v;
-                            asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p.band_ctr + bands_ready) : "memory");
-                            if (v >= gridDim.x) { ++bands_ready; continue; }
-                            if (sh->abort_flag) ok = false;
-                            else if (clock64() - t0 > p.wait_limit_clk) {
-                                sh->abort_flag = 1;
-                                atomicCAS(p.status, 0u, (blockIdx.x << 8) | SITE_BAND);
-                                ok = false;
-                            } else __nanosleep(200);
-                        }
-                        if (!ok) break;
-                        asm volatile("fence.proxy.async;" ::: "memory");   // other SMs' generic writes -> this SM's TMA reads
-                    }
-                }
-                const int dt0 = (p.first_frame - t * stt > 0) ? (p.first_frame - t * stt + dlt - 1) / dlt : 0;   // first tap whose frame exists
-                for (int pass = 0; pass < (TF32 ? 3 : 1); ++pass)
-                for (int dt = dt0; ok && dt < p.kt; ++dt)
-                    for (int cb = 0; ok && cb < p.CB; ++cb) {
-                        int fr = p.f0 + t * stt + dt * dlt;       // ring slot of Z frame t s_t + dt d_t (f0 = 0: the frame itself)
-                        if (fr >= p.F) fr -= p.F;
-                        const int fz = n * p.F + fr;
-                        const int ntap = p.per_tap_a ? spatial : 1;
-                        for (int tp = 0; tp < ntap; ++tp) {
-                            if (!(ok = mbar_wait(&sh->empty_a[s], phase, sh, p, SITE_A_EMPTY))) break;
-                            const uint32_t bar = smem_u32(&sh->full_a[s]);
-                            const int dh = p.per_tap_a ? tp / p.kw : 0, dw = p.per_tap_a ? tp % p.kw : 0;
-                            if (PAIR) {
-                                // both CTAs' boxes are counted on the leader's barrier, which the leader arms for both
-                                if (rank == 0) mbar_expect_tx(bar, 2 * a_bytes);
-                                tma_load_5d_pair(smem_u32(ring_a + (size_t)s * p.a_slot), &tm_a, bar, 0, w0 - pw, h0 - ph,
-                                                 TF32 ? 2 * cb + (pass == 1) : cb, fz);
-                            } else {
-                                mbar_expect_tx(bar, a_bytes);
-                                tma_load_5d(smem_u32(ring_a + (size_t)s * p.a_slot), &tm_a, bar, 0, w0 * stw - pw + dw * dlw,
-                                            h0 * sth - ph + dh * dlh, TF32 ? 2 * cb + (pass == 1) : cb, fz);
-                            }
-                            if (++s == p.SA) { s = 0; phase ^= 1; }
-                        }
-                    }
-            }
-            if (!ok) drain_delay();
-        }
-    }
-    // ---------------------------------------------------------------- B producer
-    else if (warp == 1) {
-        if (lane == 0) {
-            const uint32_t b_bytes = p.b_tap * p.TPB;
-            const uint32_t src_tap = p.b_src_tap ? p.b_src_tap : p.b_tap;   // bytes between taps in the packed weights
-            int s = 0;
-            uint32_t phase = 1;
-            bool ok = true;
-            if (PAIR) asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_c) : "memory");
-            for (int tile = cta_lin; ok && tile < p.total_tiles; tile += cta_cnt) {
-                const int nt = tile % p.NT;
-                const int t = (tile / p.NT) % p.T;
-                const int dt0 = (p.first_frame - t * stt > 0) ? (p.first_frame - t * stt + dlt - 1) / dlt : 0;   // first tap whose frame exists
-                for (int pass = 0; pass < (TF32 ? 3 : 1); ++pass)
-                for (int dt = dt0; ok && dt < p.kt; ++dt)
-                    for (int cb = 0; ok && cb < p.CB; ++cb) {
-                        if (PAIR) {
-                            // this CTA's half (rows rank*NPAD/2 ..) of every tap's weight tile, as boxes of the 2-D map
-                            // over the packed weights; both CTAs' boxes are counted on the leader's barrier
-                            // (split_n: NT and NPAD describe half-width tiles of a layer packed at full width; the rows of
-                            // a tap's full-width tile are then [half 0 | half 1], each again split between the two CTAs)
-                            const int npw = p.NPAD << p.split_n;                      // rows of a packed (full-width) tile
-                            const int row0 = ((((pass * p.kt + dt) * p.CB + cb) * (p.NT >> p.split_n) + (nt >> p.split_n)) * spatial) * npw +
-                                             (nt & p.split_n) * p.NPAD + (int)rank * (p.NPAD >> 1);
-                            for (int tp = 0; tp < spatial; tp += p.TPB) {
-                                if (!(ok = mbar_wait(&sh->empty_b[s], phase, sh, p, SITE_B_EMPTY))) break;
-                                const uint32_t bar = smem_u32(&sh->full_b[s]);
-                                if (rank == 0) mbar_expect_tx(bar, 2 * b_bytes);
-                                const uint32_t dst = smem_u32(ring_b + (size_t)s * p.b_slot);
-                                for (int u = 0; u < p.TPB; ++u) tma_load_2d_pair(dst + u * p.b_tap, &tm_c, bar, 0, row0 + (tp + u) * npw);
-                                if (++s == p.SB) { s = 0; phase ^= 1; }
-                            }
-                            continue;
-                        }
-                        // split_n: this launch runs half-width output-channel tiles; the packed image of a full tile
-                        // holds its two halves back to back (the swizzle repeats every 8 rows), so a half tile of a
-                        // tap is a contiguous piece of it and only the distance between taps differs
-                        const uint8_t* src = p.wq + (size_t)(((pass * p.kt + dt) * p.CB + cb) * (p.NT >> p.split_n) + (nt >> p.split_n)) * spatial * src_tap +
-                                             (size_t)(nt & p.split_n) * p.b_tap;
-                        for (int tp = 0; tp < spatial; tp += p.TPB) {
-                            if (!(ok = mbar_wait(&sh->empty_b[s], phase, sh, p, SITE_B_EMPTY))) break;
-                            const uint32_t bar = smem_u32(&sh->full_b[s]);
-                            mbar_expect_tx(bar, b_bytes);
-                            const uint32_t dst = smem_u32(ring_b + (size_t)s * p.b_slot);
-                            if (src_tap == p.b_tap) bulk_load(dst, src + (size_t)tp * src_tap, b_bytes, bar);
-                            else
-                                for (int u = 0; u < p.TPB; ++u) bulk_load(dst + u * p.b_tap, src + (size_t)(tp + u) * src_tap, p.b_tap, bar);
-                            if (++s == p.SB) { s = 0; phase ^= 1; }
-                        }
-                    }
-            }
-            if (!ok) drain_delay();
-        }
-    }
-    // ---------------------------------------------------------------- MMA issuers
-    // Warp 2 (and warp 3 when NB >= 2) issues the MMAs of its own pixel blocks.  A commit
-    // only tracks the MMAs of the committing thread, so the "slot free" and "accumulator full" barriers
-    // count one arrival per issuer.
-    else if ((warp == 2 || (warp == 3 && NI == 2)) && rank == 0) {     // (of a CTA pair only the leader issues MMAs)
-        // The whole warp runs the loop (warp-uniform control flow); one elected lane issues.
-        const int iss = warp - 2;
-        // instruction descriptor: D=F32, A=B=BF16, both K-major, N = NPAD, M = 128
-        // (operand formats: 1 = BF16, 2 = TF32)
-        constexpr uint32_t FMT = TF32 ? 2u : 1u;
-        const uint32_t idesc = (1u << 4) | (FMT << 7) | (FMT << 10) | ((uint32_t)(p.NPAD >> 3) << 17) | (((PAIR ? 256u : 128u) >> 4) << 24);
-        const uint32_t a_hi = make_desc_hi((uint32_t)BW * ROWB, LAYOUT);  // 8-pixel groups are one image row apart
-        const uint32_t b_hi = make_desc_hi(B_SBO, LAYOUT);
-        const uint32_t a_blk = (uint32_t)(iss * NBW) * ((8 * ROWB) >> 4);  // descriptor offset of this issuer's first block
-        const uint32_t a_rowstep = ((uint32_t)(BW * dlh) * ROWB) >> 4;   // descriptor step between kernel rows
-        const uint32_t b_tapstep = p.b_tap >> 4;
-        int sa = 0, sb = 0, acc = 0;
-        uint32_t pa = 0, pb = 0, pacc = 1;
-        bool ok = true;
-        if constexpr (KS > 0) {
-            constexpr uint32_t A_ROWSTEP = ((uint32_t)(TW + KS - 1) * ROWB) >> 4;
-            constexpr int STAGES = KS * KS / TPBC;
-            uint32_t a_ring = make_desc_lo(smem_u32(ring_a)) + a_blk, b_ring = make_desc_lo(smem_u32(ring_b));
-            const uint32_t a_slotstep = p.a_slot >> 4, b_slotstep = p.b_slot >> 4;
-            const uint32_t a_ring0 = a_ring, b_ring0 = b_ring;
-            for (int tile = cta_lin; ok && tile < p.total_tiles; tile += cta_cnt) {
-                const int t = (tile / p.NT) % p.T;
-                const int dt0 = (p.first_frame - t * stt > 0) ? (p.first_frame - t * stt + dlt - 1) / dlt : 0;   // first tap whose frame exists
-                if (!(ok = mbar_wait(&sh->acc_empty[acc], pacc, sh, p, SITE_ACC_EMPTY))) break;
-                tc_fence_after();
-                const uint32_t d_first = tmem_base + (uint32_t)(acc * ASETS * NB + iss * NBW) * p.NPAD;
-                uint32_t accumulate = 0, accumulate2 = 0;
-                const int nst = (p.kt - dt0) * p.CB;                          // (dt, ci-block) stages per pass
-                for (int st = 0; ok && st < (TF32 ? 3 : 1) * nst; ++st) {     // (pass, dt, ci-block) stages
-                    // TF32: the stages of the last (full-size) pass alternate between two accumulators, which halves
-                    // the length of either truncating chain; the epilogue adds the two
-                    const bool second = TF32 && st >= 2 * nst && ((st - 2 * nst) & 1);
-                    const uint32_t d0 = d_first + (second ? (uint32_t)NB * p.NPAD : 0u);
-                    const uint32_t acc_in = second ? accumulate2 : accumulate;
-                    if (!(ok = mbar_wait(&sh->full_a[sa], pa, sh, p, SITE_A_FULL))) break;
-#pragma unroll
-                    for (int g = 0; g < STAGES; ++g) {
-                        if (!(ok = mbar_wait(&sh->full_b[sb], pb, sh, p, SITE_B_FULL))) break;
-                        tc_fence_after();
-                        if (elect_one()) {
-#pragma unroll
-                            for (int u = 0; u < TPBC; ++u) {
-                                const int tap = g * TPBC + u;
-                                // tap (dh, dw) = a descriptor offset into the one halo tile.  The start address is only
-                                // 16-byte granular and need not sit on the swizzle period: the swizzle is a function of
-                                // the absolute shared-memory address (as the TMA unit applied it), so the descriptor's
-                                // base-offset field stays 0.
-                                const uint32_t a_lo = a_ring + (uint32_t)(tap / KS) * A_ROWSTEP + (uint32_t)(tap % KS) * (ROWB >> 4);
-                                const uint32_t b_lo = b_ring + (uint32_t)u * b_tapstep;
-#pragma unroll
-                                for (int j = 0; j < NBW; ++j) {
-#pragma unroll
-                                    for (int k = 0; k < KSTEPS; ++k)
-                                        if (PAIR && TF32)
-                                            tc_mma_tf32_pair(d0 + j * p.NPAD, a_lo + j * ((8 * ROWB) >> 4) + 2 * k, a_hi, b_lo + 2 * k, b_hi,
-                                                             idesc, (tap == 0 && k == 0) ? acc_in : 1u);
-                                        else if (PAIR)
-                                            tc_mma_bf16_pair(d0 + j * p.NPAD, a_lo + j * ((8 * ROWB) >> 4) + 2 * k, a_hi, b_lo + 2 * k, b_hi,
-                                                             idesc, (tap == 0 && k == 0) ? acc_in : 1u);
-                                        else
-                                            tc_mma<TF32>(d0 + j * p.NPAD, a_lo + j * ((8 * ROWB) >> 4) + 2 * k, a_hi, b_lo + 2 * k, b_hi,
-                                                         idesc, (tap == 0 && k == 0) ? acc_in : 1u);
-                                }
-                            }
-                            if (PAIR) tc_commit_pair(smem_u32(&sh->empty_b[sb])); else tc_commit(smem_u32(&sh->empty_b[sb]));
-                        }
-                        __syncwarp();
-                        b_ring += b_slotstep;
-                        if (++sb == p.SB) { sb = 0; pb ^= 1; b_ring = b_ring0; }
-                    }
-                    if (!ok) break;
-                    if (second) accumulate2 = 1; else accumulate = 1;
-                    if (elect_one()) { if (PAIR) tc_commit_pair(smem_u32(&sh->empty_a[sa])); else tc_commit(smem_u32(&sh->empty_a[sa])); }
-                    __syncwarp();
-                    a_ring += a_slotstep;
-                    if (++sa == p.SA) { sa = 0; pa ^= 1; a_ring = a_ring0; }
-                }
-                if (!ok) break;
-                if (elect_one()) { if (PAIR) tc_commit_pair(smem_u32(&sh->acc_full[acc])); else tc_commit(smem_u32(&sh->acc_full[acc])); }
-                __syncwarp();
-                if (++acc == p.ACC) { acc = 0; pacc ^= 1; }
-            }
-        } else
-        for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
-            const int t = (tile / p.NT) % p.T;
-            const int dt0 = (p.first_frame - t * stt > 0) ? (p.first_frame - t * stt + dlt - 1) / dlt : 0;   // first tap whose frame exists
-            if (!(ok = mbar_wait(&sh->acc_empty[acc], pacc, sh, p, SITE_ACC_EMPTY))) break;
-            tc_fence_after();
-            const uint32_t d_first = tmem_base + (uint32_t)(acc * ASETS * NB + iss * NBW) * p.NPAD;
-            uint32_t accumulate1 = 0, accumulate2 = 0;
-            int st2 = 0;                                       // stage counter of the last pass
-            for (int pass = 0; pass < (TF32 ? 3 : 1); ++pass)
-            for (int dt = dt0; ok && dt < p.kt; ++dt)
-                for (int cb = 0; ok && cb < p.CB; ++cb) {
-                    const bool second = TF32 && pass == 2 && (st2++ & 1);   // see the straight-line variant
-                    const uint32_t d0 = d_first + (second ? (uint32_t)NB * p.NPAD : 0u);
-                    uint32_t accumulate = second ? accumulate2 : accumulate1;
-                    uint32_t a_row = 0;  // descriptor low word of the halo row of the current tap row
-                    if (!p.per_tap_a) {
-                        if (!(ok = mbar_wait(&sh->full_a[sa], pa, sh, p, SITE_A_FULL))) break;
-                        a_row = make_desc_lo(smem_u32(ring_a + (size_t)sa * p.a_slot)) + a_blk;
-                    }
-                    for (int tp = 0, dw = 0; tp < spatial; tp += p.TPB) {
-                        if (!(ok = mbar_wait(&sh->full_b[sb], pb, sh, p, SITE_B_FULL))) break;
-                        tc_fence_after();
-                        uint32_t b_lo = make_desc_lo(smem_u32(ring_b + (size_t)sb * p.b_slot));
-                        for (int u = 0; u < p.TPB; ++u) {
-                            uint32_t a_lo;
-                            if (p.per_tap_a) {
-                                if (!(ok = mbar_wait(&sh->full_a[sa], pa, sh, p, SITE_A_FULL))) break;
-                                tc_fence_after();
-                                a_lo = make_desc_lo(smem_u32(ring_a + (size_t)sa * p.a_slot)) + a_blk;
-                            } else {
-                                // The start address is only 16-byte granular and need not sit on the swizzle
-                                // period: the swizzle is a function of the absolute shared-memory address (as
-                                // the TMA unit applied it), so the descriptor's base-offset field stays 0.
-                                a_lo = a_row + (uint32_t)(dw * dlw) * (ROWB >> 4);
-                            }
-                            if (elect_one()) {
-#pragma unroll
-                                for (int j = 0; j < NBW; ++j) {
-#pragma unroll
-                                    for (int k = 0; k < KSTEPS; ++k)
-                                        tc_mma<TF32>(d0 + j * p.NPAD, a_lo + j * ((8 * ROWB) >> 4) + 2 * k, a_hi, b_lo + 2 * k, b_hi,
-                                                    idesc, (k == 0) ? accumulate : 1u);
-                                }
-                                if (p.per_tap_a) tc_commit(smem_u32(&sh->empty_a[sa]));
-                            }
-                            __syncwarp();
-                            accumulate = 1;
-                            b_lo += b_tapstep;
-                            if (p.per_tap_a) {
-                                if (++sa == p.SA) { sa = 0; pa ^= 1; }
-                            }
-                            if (++dw == p.kw) { dw = 0; a_row += a_rowstep; }
-                        }
-                        if (!ok) break;
-                        if (elect_one()) tc_commit(smem_u32(&sh->empty_b[sb]));
-                        __syncwarp();
-                        if (++sb == p.SB) { sb = 0; pb ^= 1; }
-                    }
-                    if (ok && !p.per_tap_a) {
-                        if (elect_one()) tc_commit(smem_u32(&sh->empty_a[sa]));
-                        __syncwarp();
-                        if (++sa == p.SA) { sa = 0; pa ^= 1; }
-                    }
-                    if (second) accumulate2 = accumulate; else accumulate1 = accumulate;
-                }
-            if (!ok) break;
-            if (elect_one()) tc_commit(smem_u32(&sh->acc_full[acc]));
-            __syncwarp();
-            if (++acc == p.ACC) { acc = 0; pacc ^= 1; }
-        }
-    }
-    // ---------------------------------------------------------------- epilogue (warps 4..7)
-    else if (warp >= 4 && warp < 8) {
-        const int q = warp & 3;  // TMEM lane quarter this warp may read
-        int acc = 0;
-        uint32_t pacc = 0;
-        bool ok = true;
-        const int64_t HW = (int64_t)p.H * p.W;
-        const int m = q * 32 + lane;  // accumulator row = pixel m of a 128-pixel block: image row m/8, pixel m%8
-        const bool elected = (threadIdx.x == 4 * 32);
-        constexpr bool RING = !FUSED && !COOP;                 // frame-ring output and residual: plain variant only
-        const bool has_res = RING && p.res != nullptr;
-        const bool act = p.act != 0;
-        int ebuf = 0;
-        // bias: a shared-memory copy when the padded channel count fits.  A global load per element costs little
-        // while the next tile's MMAs run, but its latency sits in the exposed tail of a CTA's last tile: 11 us
-        // against 5 us for a 192-channel tile.
-        const bool bias_smem = p.NT * p.NPAD <= TC_BIAS_SMEM;
-        if (bias_smem)
-            for (int i = threadIdx.x - 128; i < p.NT * p.NPAD; i += 128) sh->bias_s[i] = __ldg(p.bias + i);
-        epi_bar_sync();
-        const float* bias = bias_smem ? sh->bias_s : p.bias;
-        for (int tile = cta_lin; ok && tile < p.total_tiles; tile += cta_cnt) {
-            const int nt = tile % p.NT;
-            int r = tile / p.NT;
-            const int t = r % p.T; r /= p.T;
-            const int tx = r % p.tiles_w; r /= p.tiles_w;
-            const int ty = p.ty_begin + r % p.tiles_h;
-            const int n = r / p.tiles_h;
-            const int h = ty * 16 + (m >> 3);
-            const int wt = tx * TWT + wofs;                  // first pixel column of this CTA's part of the tile
-            // residual: pixel (h, w) of frame t holds its Cout channels in blocks of res_KB (64 bytes per 32 channels)
-            const __nv_bfloat16* res_row = nullptr;
-            if (has_res && h < p.H) {
-                int rs = p.res_f0 + t;
-                if (rs >= p.res_F) rs -= p.res_F;
-                res_row = p.res + (((int64_t)n * p.res_F + rs) * p.res_CB * HW + (int64_t)h * p.W) * p.res_KB;
-            }
-            // the residual of the first chunk is fetched while the MMAs of this tile still run; every later chunk's
-            // residual is fetched one chunk ahead
-            uint32_t rr_next[16];
-            if (p.epi_tma) load_res32(res_row, wt + (m & 7) < p.W, wt + (m & 7), nt * p.NPAD, p, HW, rr_next);
-            ok = mbar_wait(&sh->acc_full[acc], pacc, sh, p, SITE_ACC_FULL);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t t_acc = tmem_base + (uint32_t)(acc * ASETS * NB) * p.NPAD + ((uint32_t)(q * 32) << 16);
-            // TF32: was the second accumulator of the last pass used (at least two stages per pass)?
-            const int dt0e = (p.first_frame - t * stt > 0) ? (p.first_frame - t * stt + dlt - 1) / dlt : 0;
-            const bool two_acc = TF32 && (p.kt - dt0e) * p.CB >= 2;
-            if (p.epi_tma) {
-                // BF16 tile chunks -> shared memory -> one TMA store per chunk.  NCTHW output: [ECH channels][16 rows]
-                // [TW pixels]; ring output: [16 rows][TW pixels][32 channels] with the 64-byte swizzle of the tensor map.
-                for (int c0 = 0; c0 < p.NPAD; c0 += p.ECH) {
-                    if (elected) bulk_wait_read<1>();   // the store that last read this buffer has finished reading
-                    epi_bar_sync();
-                    uint8_t* stg = epi_buf + (size_t)ebuf * p.e_slot;
-                    const int co0 = nt * p.NPAD + c0;
-#pragma unroll
-                    for (int blk = 0; blk < NB; ++blk) {
-                        uint32_t rr[16];
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) rr[j] = rr_next[j];
-                        if (has_res) {
-                            const int wn = wt + ((blk + 1 < NB) ? blk + 1 : 0) * 8 + (m & 7);
-                            const int con = (blk + 1 < NB) ? co0 : co0 + p.ECH;
-                            load_res32(res_row, wn < p.W && con < (nt + 1) * p.NPAD, wn, con, p, HW, rr_next);
-                        }
-                        uint32_t v[32];
-                        if (p.ECH == 32) tc_ld32(t_acc + blk * p.NPAD + c0, v); else tc_ld16(t_acc + blk * p.NPAD + c0, v);
-                        tc_wait_ld();
-                        uint32_t pk[16];
-                        float bb[32];                       // the chunk's bias: eight 16-byte reads (co0 is a multiple of 16)
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            const float4 b4 = (4 * j < p.ECH) ? *reinterpret_cast<const float4*>(bias + co0 + 4 * j)
-                                                              : make_float4(0.f, 0.f, 0.f, 0.f);
-                            bb[4 * j] = b4.x; bb[4 * j + 1] = b4.y; bb[4 * j + 2] = b4.z; bb[4 * j + 3] = b4.w;
-                        }
-#pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            pk[j] = (2 * j < p.ECH) ? epi_pair(__uint_as_float(v[2 * j]) + bb[2 * j],
-                                                               __uint_as_float(v[2 * j + 1]) + bb[2 * j + 1], rr[j], has_res, act)
-                                                    : 0u;
-                        const uint32_t px = (uint32_t)((m >> 3) * TW + blk * 8 + (m & 7));   // pixel of the tile, row-major
-                        if (RING && p.epi_tma == 2) {
-                            uint4* row = reinterpret_cast<uint4*>(stg + (size_t)px * 64);
-                            const uint32_t sw = (px >> 1) & 3u;
-#pragma unroll
-                            for (int c = 0; c < 4; ++c)
-                                row[c ^ sw] = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-                        } else {
-                            unsigned short* dst = reinterpret_cast<unsigned short*>(stg) + px;
-#pragma unroll
-                            for (int j = 0; j < 16; ++j)
-                                if (2 * j < p.ECH) {
-                                    dst[(2 * j) * 16 * TW] = (unsigned short)(pk[j] & 0xFFFFu);
-                                    dst[(2 * j + 1) * 16 * TW] = (unsigned short)(pk[j] >> 16);
-                                }
-                        }
-                    }
-                    fence_async_smem();
-                    epi_bar_sync();
-                    if (elected) {
-                        if (RING && p.epi_tma == 2 && p.up_rt > 0) {
-                            // fused nearest-neighbour upsample: the tensor map walks the 2H x 2W ring with a traversal
-                            // stride of 2 pixels, so one store drops the tile onto every second pixel from (b, a)
-                            for (int j = 0; j < p.up_rt; ++j) {
-                                const int os = (p.out_f0 + t * p.up_rt + j) % p.out_F;
-                                for (int ab = 0; ab < 4; ++ab)
-                                    tma_store_5d(&tm_o, smem_u32(stg), co0 % p.out_KB, 2 * wt + (ab & 1), 2 * ty * 16 + (ab >> 1),
-                                                 co0 / p.out_KB, n * p.out_F + os);
-                            }
-                        } else if (RING && p.epi_tma == 2) {
-                            int os = p.out_f0 + t;
-                            if (os >= p.out_F) os -= p.out_F;
-                            tma_store_5d(&tm_o, smem_u32(stg), co0 % p.out_KB, wt, ty * 16, co0 / p.out_KB, n * p.out_F + os);
-                        } else {
-                            tma_store_5d(&tm_o, smem_u32(stg), wt, ty * 16, t, co0, n);
-                        }
-                        bulk_commit();
-                    }
-                    ebuf ^= 1;
-                }
-            } else {
-#pragma unroll 1
-                for (int blk = 0; blk < NB; ++blk) {
-                    const int w = wt + blk * 8 + (m & 7);
-                    const bool valid = h < p.H && w < p.W;
-                    const int64_t pix = (int64_t)t * HW + (int64_t)h * p.W + w;
-#pragma unroll 1
-                    for (int c0 = 0; c0 < p.NPAD; c0 += 32) {
-                        const int co0 = nt * p.NPAD + c0;
-                        uint32_t rr[16];
-                        load_res32(res_row, valid, w, co0, p, HW, rr);
-                        uint32_t v[32];
-                        const int nc = (p.NPAD - c0 >= 32) ? 32 : 16;
-                        if (nc == 32) tc_ld32(t_acc + blk * p.NPAD + c0, v); else tc_ld16(t_acc + blk * p.NPAD + c0, v);
-                        tc_wait_ld();
-                        if (two_acc) {
-                            uint32_t v2[32];
-                            if (nc == 32) tc_ld32(t_acc + (NB + blk) * p.NPAD + c0, v2); else tc_ld16(t_acc + (NB + blk) * p.NPAD + c0, v2);
-                            tc_wait_ld();
-#pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                if (j < nc) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(v2[j]));
-                        }
-                        if (valid) {
-                            if (p.out_f32) {
-#pragma unroll
-                                for (int j = 0; j < 32; ++j) {
-                                    const int co = co0 + j;
-                                    if (j < nc && co < p.Cout) {
-                                        const float val = __uint_as_float(v[j]) + bias[co];
-                                        reinterpret_cast<float*>(p.out)[((int64_t)n * p.Cout + co) * p.T * HW + pix] = act ? silu_f32(val) : val;
-                                    }
-                                }
-                            } else {
-#pragma unroll
-                                for (int j = 0; j < 16; ++j) {
-                                    const int co = co0 + 2 * j;
-                                    if (2 * j < nc) {
-                                        const uint32_t pr = epi_pair(__uint_as_float(v[2 * j]) + bias[co],
-                                                                     __uint_as_float(v[2 * j + 1]) + bias[co + 1], rr[j], has_res, act);
-                                        unsigned short* o = reinterpret_cast<unsigned short*>(p.out) +
-                                                            ((int64_t)n * p.Cout + co) * p.T * HW + pix;
-                                        if (co < p.Cout) o[0] = (unsigned short)(pr & 0xFFFFu);
-                                        if (co + 1 < p.Cout) o[(int64_t)p.T * HW] = (unsigned short)(pr >> 16);
-                                    }
-                                }
-                            }
-                        }
-                    }
-                }
-            }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) { if (PAIR) mbar_arrive_leader(smem_u32(&sh->acc_empty[acc])); else mbar_arrive(smem_u32(&sh->acc_empty[acc])); }
-            if (++acc == p.ACC) { acc = 0; pacc ^= 1; }
-        }
-        if (p.epi_tma && elected) bulk_wait_all();   // all stores of this CTA are complete before it exits
-    }
-
-    // ---------------------------------------------------------------- stagers (cooperative staging, warps 8..11)
-    if (COOP && warp >= 8) {
-        const int tid = threadIdx.x - 256;
-        constexpr int SPX = StagerGeom<KB>::PX;
-        const int nchunks = (sp.W + SPX - 1) / SPX;
-        const int nf = sp.tc + sp.T - sp.f_begin;
-        // Stagers wait on nothing but their own named barrier, so they always run to completion (also when a
-        // consumer role of some CTA has given up on a wait): every thread of the four warps takes every branch.
-        for (int b = 0; b < p.nbands; ++b) {
-            const int h_lo = 16 * b;
-            const int rows = (sp.H - h_lo < 16) ? sp.H - h_lo : 16;
-            const int ntask = sp.N * nf * sp.CB * rows * nchunks;
-            constexpr int G = 4;                             // tasks whose loads are in flight together (32 KB per CTA; 6 would spill)
-            for (int task0 = blockIdx.x; task0 < ntask; task0 += G * gridDim.x) {
-                StageTask tk[G];
-                uint4 val[G][StagerGeom<KB>::NLD];
-#pragma unroll
-                for (int g = 0; g < G; ++g) {
-                    const int task = task0 + g * gridDim.x;
-                    if (task < ntask) {
-                        int r = task;
-                        const int wc = r % nchunks; r /= nchunks;
-                        const int h = h_lo + r % rows; r /= rows;
-                        const int cb = r % sp.CB; r /= sp.CB;
-                        const int f = sp.f_begin + r % nf;
-                        const int n = r / nf;
-                        tk[g] = make_stage_task(sp, KB, n, f, cb, h, wc * SPX);
-                        stage_task_load<KB>(sp, tk[g], tid, val[g]);
-                    }
-                }
-#pragma unroll
-                for (int g = 0; g < G; ++g)
-                    if (task0 + g * gridDim.x < ntask) stage_task_store<KB>(sp, tk[g], tid, val[g], coop_tile);
-            }
-            __threadfence();                               // this thread's stores are visible GPU-wide ...
-            stager_bar();                                  // ... for all 128 stager threads, before the band is signalled
-            if (tid == 0) atomicAdd(p.band_ctr + b, 1u);
-        }
-    }
-
-    // ---------------------------------------------------------------- transposers (fused mode, warps 8..11)
-    if (FUSED && warp >= 8) {
-        // raw [c][row][32 px] (64-byte rows, 64-byte swizzle as TMA wrote it) -> halo tile [pixel][32 ch] (64-byte
-        // rows, 64-byte swizzle: the K-major operand).  Per step a warp moves 8 pixels x 32 channels: ldmatrix.trans
-        // reads four 8x8 blocks (one per channel octet, rows = channels), stmatrix writes them with rows = pixels.
-        const int tw = warp - 8;
-        const int colshift = 8 - pw;                       // raw column of halo column 0
-        const int mi = lane >> 3, mj = lane & 7;           // this lane addresses row mj of matrix (channel octet) mi
-        const uint32_t src_lane = (uint32_t)(mi * 8 + mj) * (uint32_t)(BH * RAW_PX * 2);
-        const uint32_t dummy_addr = smem_u32(dummy) + (uint32_t)(tw * 32 + lane) * 16;
-        int rs = 0, sa = 0;
-        uint32_t pr = 0, pea = 1;
-        bool ok = true;
-        for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
-            const int t = (tile / p.NT) % p.T;
-            const int dt0 = (p.first_frame - t * stt > 0) ? (p.first_frame - t * stt + dlt - 1) / dlt : 0;   // first tap whose frame exists
-            for (int kb = (p.kt - dt0) * p.CB; ok && kb > 0; --kb) {
-                ok = mbar_wait(&sh->raw_full[rs], pr, sh, p, SITE_RAW_FULL) && mbar_wait(&sh->empty_a[sa], pea, sh, p, SITE_A_EMPTY);
-                ok = __all_sync(0xffffffffu, ok);
-                if (!ok) break;
-                const uint32_t raw_base = smem_u32(ring_raw + (size_t)rs * p.raw_slot);
-                const uint32_t a_base = smem_u32(ring_a + (size_t)sa * p.a_slot);
-                // warp tw owns column block tw of every halo row; rows go in batches of TR so that the loads of a
-                // batch are in flight together before its stores
-                constexpr int TR = 6;
-                const int col = 8 * tw + mj - colshift;
-                const bool col_ok = col >= 0 && col < BW;
-                uint32_t so0 = src_lane + (uint32_t)tw * 16;
-                for (int hb = 0; hb < BH; hb += TR) {
-                    uint32_t frag[TR][4];
-#pragma unroll
-                    for (int u = 0; u < TR; ++u) {
-                        if (hb + u < BH) {
-                            uint32_t so = so0 + (uint32_t)(hb + u) * (RAW_PX * 2);
-                            so ^= ((so >> 7) & 3u) << 4;             // the 64-byte swizzle TMA applied to the raw box
-                            ldmatrix_x4_trans(raw_base + so, frag[u]);
-                        }
-                    }
-#pragma unroll
-                    for (int u = 0; u < TR; ++u) {
-                        if (hb + u < BH) {
-                            const uint32_t r = (uint32_t)((hb + u) * BW + col);
-                            const uint32_t dst = col_ok ? a_base + r * 64 + (((uint32_t)mi ^ ((r >> 1) & 3u)) << 4) : dummy_addr;
-                            stmatrix_x4(dst, frag[u]);
-                        }
-                    }
-                }
-                fence_async_smem();                        // generic-proxy writes -> visible to the tensor core's reads
-                __syncwarp();
-                if (lane == 0) {
-                    mbar_arrive(smem_u32(&sh->full_a[sa]));
-                    mbar_arrive(smem_u32(&sh->raw_empty[rs]));
-                }
-                rs ^= 1;
-                if (rs == 0) pr ^= 1;
-                if (++sa == p.SA) { sa = 0; pea ^= 1; }
-            }
-        }
-    }
-
-    // ---------------------------------------------------------------- teardown
-    tc_fence_before();
-    __syncthreads();
-    if (PAIR) cluster_sync_all();   // the leader's MMAs read the peer's shared memory and write its tensor memory
-    if (warp == 3) {
-        tc_fence_after();
-        if (PAIR) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
-        else asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
-    }
-}
-
-// ------------------------------------------------------------------------------------------------
-// 1x1x1 kernels (per-pixel matmul, no cache, no halo): streaming kernel straight from NCTHW
-// ------------------------------------------------------------------------------------------------
-// With one tap there is no shift to express, so the activations can be used as they lie in memory: for a
-// fixed channel the P = T*H*W pixels of a sample are contiguous, i.e. the A operand is "MN-major".  A TMA box
-// of {64 pixels, 64 channels} with 128-byte swizzle lands as 64 K-rows of 128 bytes = the canonical MN-major
-// layout (8-row groups 1024 bytes apart); a 128-pixel M tile is two such boxes.  The whole weight matrix
-// (Cin_pad x NPAD, packed as for the general kernel) stays resident in shared memory; the kernel is bound by
-// HBM (read x once, write out once) and the tensor core is mostly idle.
-struct PwParams {
-    int N, Cout, CB, NPAD;
-    int tiles_p;              // 128-pixel tiles per sample
-    int total_tiles;
-    int SA;                   // activation ring depth
-    int ECH;                  // channels per epilogue chunk (32 or 16)
-    uint32_t a_slot, e_slot, w_bytes, b_tap;
-    uint32_t tmem_cols;
-    long long wait_limit_clk;
-    const float* bias;
-    const uint8_t* wq;
-    unsigned int* status;
-};
-
-__device__ __forceinline__ bool pw_wait(uint64_t* bar, uint32_t parity, TcShared* sh, const PwParams& p, uint32_t site) {
-    const uint32_t b = smem_u32(bar);
-    if (mbar_try_wait(b, parity)) return true;
-    long long t0 = 0;
-    for (uint32_t it = 1;; ++it) {
-        if (mbar_try_wait(b, parity)) return true;
-        if ((it & 63u) == 0u) {
-            if (sh->abort_flag) return false;
-            const long long now = clock64();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > p.wait_limit_clk) {
-                sh->abort_flag = 1;
-                atomicCAS(p.status, 0u, (blockIdx.x << 8) | site);
-                return false;
-            }
-        }
-    }
-}
-
-__global__ void __launch_bounds__(TC_THREADS, 1)
-conv1x1_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_x,   // x as (pixel, channel, sample)
-                       const __grid_constant__ CUtensorMap tm_o,   // out as (pixel, channel, sample)
-                       const PwParams p) {
-    constexpr int KB = 64;
-    constexpr uint32_t HALF = 64 * 128;                     // bytes of one {64 px, 64 ch} box
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-    uint8_t* w_smem = smem;
-    uint8_t* ring_a = w_smem + p.w_bytes;
-    uint8_t* epi_buf = ring_a + (size_t)p.SA * p.a_slot;
-    TcShared* sh = reinterpret_cast<TcShared*>(epi_buf + 2 * (size_t)p.e_slot);
-
-    const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);
-    const int lane = threadIdx.x & 31;
-
-    if (threadIdx.x == 0) {
-        for (int i = 0; i < p.SA; ++i) { mbar_init(smem_u32(&sh->full_a[i]), 1); mbar_init(smem_u32(&sh->empty_a[i]), 1); }
-        mbar_init(smem_u32(&sh->full_b[0]), 1);
-        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&sh->acc_full[i]), 1); mbar_init(smem_u32(&sh->acc_empty[i]), 4); }
-        sh->abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    if (warp == 3) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&sh->tmem_base)),
-                     "r"(p.tmem_cols)
-                     : "memory");
-        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = sh->tmem_base;
-
-    if (warp == 0) {                      // activation producer
-        if (lane == 0) {
-            asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_x) : "memory");
-            int s = 0;
-            uint32_t phase = 1;
-            bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
-                const int n = tile / p.tiles_p, p0 = (tile % p.tiles_p) * 128;
-                for (int cb = 0; cb < p.CB; ++cb) {
-                    if (!(ok = pw_wait(&sh->empty_a[s], phase, sh, p, SITE_A_EMPTY))) break;
-                    const uint32_t bar = smem_u32(&sh->full_a[s]);
-                    mbar_expect_tx(bar, 2 * HALF);
-                    const uint32_t dst = smem_u32(ring_a + (size_t)s * p.a_slot);
-                    tma_load_3d(dst, &tm_x, bar, p0, cb * KB, n);
-                    tma_load_3d(dst + HALF, &tm_x, bar, p0 + 64, cb * KB, n);
-                    if (++s == p.SA) { s = 0; phase ^= 1; }
-                }
-            }
-            if (!ok) drain_delay();
-        }
-    } else if (warp == 1) {               // weights: loaded once, resident for the whole kernel
-        if (lane == 0) {
-            const uint32_t bar = smem_u32(&sh->full_b[0]);
-            mbar_expect_tx(bar, p.w_bytes);
-            bulk_load(smem_u32(w_smem), p.wq, p.w_bytes, bar);
-        }
-    } else if (warp == 2) {               // MMA issuer (warp-uniform; one elected lane issues)
-        // instruction descriptor: D=F32, A=B=BF16, A MN-major (bit 15), B K-major, N = NPAD, M = 128
-        const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | (1u << 15) | ((uint32_t)(p.NPAD >> 3) << 17) | ((128u >> 4) << 24);
-        const uint32_t a_hi = make_desc_hi(1024, 2u);       // MN-major: 8-channel groups 1024 bytes apart
-        const uint32_t b_hi = make_desc_hi(8 * 128, 2u);
-        const uint32_t a_lbo = (HALF >> 4) << 16;           // next 64 pixels: the second box
-        const uint32_t w_lo = make_desc_lo(smem_u32(w_smem));
-        int sa = 0, acc = 0;
-        uint32_t pa = 0, pacc = 1;
-        bool ok = pw_wait(&sh->full_b[0], 0, sh, p, SITE_B_FULL);
-        for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
-            if (!(ok = pw_wait(&sh->acc_empty[acc], pacc, sh, p, SITE_ACC_EMPTY))) break;
-            tc_fence_after();
-            const uint32_t d0 = tmem_base + (uint32_t)acc * p.NPAD;
-            for (int cb = 0; cb < p.CB; ++cb) {
-                if (!(ok = pw_wait(&sh->full_a[sa], pa, sh, p, SITE_A_FULL))) break;
-                tc_fence_after();
-                const uint32_t a_lo = (((smem_u32(ring_a + (size_t)sa * p.a_slot)) & 0x3FFFFu) >> 4) | a_lbo;
-                const uint32_t b_lo = w_lo + (uint32_t)cb * (p.b_tap >> 4);
-                if (elect_one()) {
-#pragma unroll
-                    for (int k = 0; k < KB / 16; ++k)     // 16 channels = two 8-row groups = 2048 bytes of A, 32 bytes of B
-                        tc_mma_bf16(d0, a_lo + k * (2048 >> 4), a_hi, b_lo + 2 * k, b_hi, idesc, (cb | k) ? 1u : 0u);
-                    tc_commit(smem_u32(&sh->empty_a[sa]));
-                }
-                __syncwarp();
-                if (++sa == p.SA) { sa = 0; pa ^= 1; }
-            }
-            if (!ok) break;
-            if (elect_one()) tc_commit(smem_u32(&sh->acc_full[acc]));
-            __syncwarp();
-            if (++acc == 2) { acc = 0; pacc ^= 1; }
-        }
-    } else if (warp >= 4) {               // epilogue: +bias, RNE to BF16, [channel][128 px] tile, TMA store
-        const int q = warp & 3;
-        const int m = q * 32 + lane;
-        const bool elected = (threadIdx.x == 4 * 32);
-        int acc = 0, ebuf = 0;
-        uint32_t pacc = 0;
-        bool ok = true;
-        for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
-            const int n = tile / p.tiles_p, p0 = (tile % p.tiles_p) * 128;
-            ok = pw_wait(&sh->acc_full[acc], pacc, sh, p, SITE_ACC_FULL);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t t_acc = tmem_base + (uint32_t)acc * p.NPAD + ((uint32_t)(q * 32) << 16);
-            for (int c0 = 0; c0 < p.NPAD; c0 += p.ECH) {
-                if (elected) bulk_wait_read<1>();
-                epi_bar_sync();
-                __nv_bfloat16* stg = reinterpret_cast<__nv_bfloat16*>(epi_buf + (size_t)ebuf * p.e_slot);
-                uint32_t v[32];
-                if (p.ECH == 32) tc_ld32(t_acc + c0, v); else tc_ld16(t_acc + c0, v);
-                tc_wait_ld();
-#pragma unroll
-                for (int j = 0; j < 32; ++j)
-                    if (j < p.ECH) stg[j * 128 + m] = __float2bfloat16_rn(__uint_as_float(v[j]) + __ldg(p.bias + c0 + j));
-                fence_async_smem();
-                epi_bar_sync();
-                if (elected) {
-                    tma_store_3d(&tm_o, smem_u32(stg), p0, c0, n);
-                    bulk_commit();
-                }
-                ebuf ^= 1;
-            }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&sh->acc_empty[acc]));
-            if (++acc == 2) { acc = 0; pacc ^= 1; }
-        }
-        if (elected) bulk_wait_all();
-    }
-
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 3) {
-        tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");
-    }
-}
-
-// ------------------------------------------------------------------------------------------------
-// Self-test of the bounded-wait path: one CTA waits on an mbarrier phase that nothing ever completes.
-// The wait gives up after limit_clk clocks, records (block << 8) | site in the status word and the kernel
-// returns normally - the same code path a lost TMA completion would take in the convolution kernels.
-// ------------------------------------------------------------------------------------------------
-__global__ void wait_timeout_selftest_kernel(unsigned int* status, long long limit_clk) {
-    __shared__ uint64_t bar;
-    if (threadIdx.x == 0) {
-        mbar_init(smem_u32(&bar), 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        const uint32_t b = smem_u32(&bar);
-        const long long t0 = clock64();
-        for (uint32_t it = 1;; ++it) {
-            if (mbar_try_wait(b, 0)) break;                       // phase 0 never completes: nobody arrives
-            if ((it & 63u) == 0u && clock64() - t0 > limit_clk) {
-                atomicCAS(status, 0u, (blockIdx.x << 8) | 0x7Fu);  // site 0x7F: the self-test
-                break;
-            }
-        }
-    }
-    __syncthreads();
-}
-
-}  // namespace ccv3d
+#include "ccv3d_tc_layout.cuh"
+#include "ccv3d_tc_ptx.cuh"
+#include "ccv3d_tc_conv.cuh"
+#include "ccv3d_tc_pointwise.cuh"
