@@ -351,6 +351,54 @@ def other_configs_leg(dev):
     return out
 
 
+def hsplit_leg(dev):
+    """Per-rank work of the height-split headline layer on this one GPU: rank 1 at world sizes
+    2, 4 and 8 packs its halo rows, assembles its slab and runs the layer on it (10 calls after 3 warm-ups).  The
+    neighbour exchange itself needs more than one GPU and is not in these times; its size is reported."""
+    import math
+    import torch
+    import paper_2609_31938_b200 as ccv
+    from paper_2609_31938_b200.hsplit import HSplitCausalConv3d
+    name = "cfg3_bf16_192"
+    d = {k: v for k, v in si.CONFIGS[name].items() if k not in ("dtype", "x_dist")}
+    N, Cin, Cout, T, H, W, k = d["N"], d["Cin"], d["Cout"], d["T"], d["H"], d["W"], d["k"]
+    gen = torch.Generator(device=dev).manual_seed(0)
+    rnd = lambda *shape, std=1.0: (torch.randn(*shape, device=dev, generator=gen) * std).to(torch.bfloat16)
+    w, b = rnd(Cout, Cin, *k, std=1.0 / math.sqrt(Cin * k[0] * k[1] * k[2])), rnd(Cout, std=math.sqrt(0.1))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    out = {"workload": name, "note": "pack + slab assembly + layer on the slab, for rank 1 of the world (halo rows on both sides of its slab); "
+                                     "neighbour exchange (NCCL send/recv) not included"}
+    for world in (2, 4, 8):
+        layer = HSplitCausalConv3d(w, b, H, min(1, world - 1), world, transport=None)
+        p = layer.plan
+        xb = rnd(N, Cin, T, p.rows, W)
+        cache = rnd(N, Cin, k[0] - 1, p.slab_rows, W)
+        halo_up, halo_down = rnd(N, Cin, T, p.top, W), rnd(N, Cin, T, p.bot, W)
+
+        def rank_step():
+            layer.pack(xb)
+            return layer.conv(layer.assemble(xb, halo_up, halo_down), cache)
+
+        for _ in range(3):
+            rank_step()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(10):
+            rank_step()
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / 10
+        flops = si.conv_flops(**d) * p.rows / H
+        out[f"world{world}"] = {"rows": p.rows, "slab_rows": p.slab_rows, "ms_per_rank_step": ms,
+                                "tflops_per_rank": flops / (ms * 1e-3) / 1e12,
+                                "halo_bytes_sent_per_step": int(2 * N * Cin * T * (p.top + p.bot) * W)}
+        assert layer.conv.device_status()[0] == ccv.OK
+        layer.close()
+        del xb, cache, halo_up, halo_down
+        torch.cuda.empty_cache()
+    return out
+
+
 def main_ours(args):
     import torch
     import paper_2609_31938_b200 as ccv
@@ -517,6 +565,7 @@ def main_ours(args):
     cpu = cpu_baseline(name) if world == 1 else None
     chain = chain_leg(dev) if (world == 1 and not args.no_chain) else None
     others = other_configs_leg(dev) if (world == 1 and not args.no_chain) else None
+    hsplit = hsplit_leg(dev) if (world == 1 and not args.no_chain) else None
     line = {"metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
@@ -534,6 +583,8 @@ def main_ours(args):
         line["decoder_chain"] = chain
     if others is not None:
         line["other_configs"] = others
+    if hsplit is not None:
+        line["height_split"] = hsplit
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()

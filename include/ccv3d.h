@@ -266,6 +266,20 @@ ccv3d_status ccv3d_upsample_bf16(const void* x, void* y, int32_t N, int32_t C, i
                                  int32_t rt, void* stream);
 
 /*
+ * Image-row slabs, the data movement of a height-split layer (each GPU owns a band of image rows and needs
+ * the kernel's halo rows of its neighbours, the per-tap 2-D correlation of Eq. (2) being local in h):
+ * for every one of `planes` planes (a plane = one (n, c, t) image of rows of row_bytes bytes)
+ *     dst plane p, rows dst_row0 .. dst_row0+rows-1   <-   src plane p, rows src_row0 .. src_row0+rows-1,
+ * dst planes dst_H rows high, src planes src_H rows high (DEVICE, any element type).  src == NULL writes zeros
+ * (the image edge, where the halo is the layer's zero padding).  Packs halo rows into a contiguous send buffer
+ * (dst_H = rows), unpacks a received one, and places a band inside its slab.  16-byte vector copies when
+ * row_bytes and both row addresses are multiples of 16, byte copies otherwise.  Stream-ordered.
+ * CCV3D_ERR_INVALID_ARG for NULL dst, non-positive sizes or row ranges outside their planes.
+ */
+ccv3d_status ccv3d_rows_copy(void* dst, int32_t dst_H, int32_t dst_row0, const void* src, int32_t src_H,
+                             int32_t src_row0, int64_t planes, int32_t rows, int64_t row_bytes, void* stream);
+
+/*
  * ------------------------------------------------------------------------------------------------
  * Resident activations: frame rings in the tensor-core operand order
  * ------------------------------------------------------------------------------------------------

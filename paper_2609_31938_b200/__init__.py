@@ -53,7 +53,7 @@ EXPORTS = ("ccv3d_create", "ccv3d_forward", "ccv3d_forward_host", "ccv3d_workspa
            "ccv3d_get_counters", "ccv3d_device_status", "ccv3d_status_string", "ccv3d_add_bf16",
            "ccv3d_upsample_bf16", "ccv3d_profile_enable", "ccv3d_profile_read", "ccv3d_forward_static", "ccv3d_selftest_wait_timeout", "ccv3d_forward_ex",
            "ccv3d_ring_kb", "ccv3d_ring_bytes", "ccv3d_ring_load", "ccv3d_ring_store", "ccv3d_upsample_ring",
-           "ccv3d_forward_ring", "ccv3d_out_dims", "ccv3d_forward_ring_up")
+           "ccv3d_forward_ring", "ccv3d_out_dims", "ccv3d_forward_ring_up", "ccv3d_rows_copy")
 
 
 def _load() -> ctypes.CDLL:
@@ -80,6 +80,7 @@ def _load() -> ctypes.CDLL:
     lib.ccv3d_selftest_wait_timeout.argtypes = [vp, i32, vp]
     lib.ccv3d_add_bf16.argtypes = [vp, vp, vp, ctypes.c_int64, vp]
     lib.ccv3d_upsample_bf16.argtypes = [vp, vp, i32, i32, i32, i32, i32, i32, vp]
+    lib.ccv3d_rows_copy.argtypes = [vp, i32, i32, vp, i32, i32, ctypes.c_int64, i32, ctypes.c_int64, vp]
     i32p = ctypes.POINTER(ctypes.c_int32)
     lib.ccv3d_out_dims.argtypes = [vp, i32, i32, i32, i32p, i32p, i32p, i32p]
     rp = ctypes.POINTER(Ring)
@@ -203,6 +204,10 @@ def ccv3d_add_bf16(a, b, y, n, stream=0) -> int:
 
 def ccv3d_upsample_bf16(x, y, N, C, T, H, W, rt, stream=0) -> int:
     return lib.ccv3d_upsample_bf16(x, y, N, C, T, H, W, rt, stream)
+
+
+def ccv3d_rows_copy(dst, dst_H, dst_row0, src, src_H, src_row0, planes, rows, row_bytes, stream=0) -> int:
+    return lib.ccv3d_rows_copy(dst, dst_H, dst_row0, src, src_H, src_row0, planes, rows, row_bytes, stream)
 
 
 def ccv3d_ring_kb(C: int) -> int:

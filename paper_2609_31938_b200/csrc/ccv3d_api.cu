@@ -635,6 +635,26 @@ ccv3d_status ccv3d_upsample_bf16(const void* x, void* y, int32_t N, int32_t C, i
     return cudaGetLastError() == cudaSuccess ? CCV3D_OK : cuda_fail();
 }
 
+ccv3d_status ccv3d_rows_copy(void* dst, int32_t dst_H, int32_t dst_row0, const void* src, int32_t src_H,
+                             int32_t src_row0, int64_t planes, int32_t rows, int64_t row_bytes, void* stream) {
+    if (!dst || planes < 1 || rows < 1 || row_bytes < 1 || dst_row0 < 0 || dst_row0 + rows > dst_H)
+        return CCV3D_ERR_INVALID_ARG;
+    if (src && (src_row0 < 0 || src_row0 + rows > src_H)) return CCV3D_ERR_INVALID_ARG;
+    unsigned char* d = (unsigned char*)dst + (int64_t)dst_row0 * row_bytes;
+    const unsigned char* s = src ? (const unsigned char*)src + (int64_t)src_row0 * row_bytes : nullptr;
+    const bool vec = row_bytes % 16 == 0 && !(((uintptr_t)d | (uintptr_t)s) & 15u);
+    const int64_t unit = vec ? 16 : 1;
+    const int64_t chunk = rows * row_bytes / unit, total = planes * chunk;
+    const int64_t blocks = (total + 255) / 256;
+    const unsigned grid = (unsigned)(blocks > 148 * 16 ? 148 * 16 : blocks);
+    const int64_t dp = dst_H * row_bytes / unit, sp = src ? src_H * row_bytes / unit : 0;
+    if (vec)
+        rows_copy_kernel<uint4><<<grid, 256, 0, (cudaStream_t)stream>>>((uint4*)d, dp, (const uint4*)s, sp, planes, chunk);
+    else
+        rows_copy_kernel<unsigned char><<<grid, 256, 0, (cudaStream_t)stream>>>(d, dp, s, sp, planes, chunk);
+    return cudaGetLastError() == cudaSuccess ? CCV3D_OK : cuda_fail();
+}
+
 int32_t ccv3d_ring_kb(int32_t C) { return C < 1 ? 0 : (C % 64 == 0 ? 64 : (C % 32 == 0 ? 32 : 0)); }
 
 uint64_t ccv3d_ring_bytes(const ccv3d_ring* r) {

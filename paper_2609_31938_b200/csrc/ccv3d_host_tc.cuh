@@ -291,8 +291,10 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
 
     // Cooperative staging (default when W % 8 == 0): the staging pass runs inside the convolution kernel, on four
     // extra warps per CTA, one band of 16 rows ahead of the tiles that read it.
-    const bool coop = nbands == 1 && !per_tap && !general && !f32 && !(d.flags & CCV3D_FLAG_TWO_KERNELS) && W % 8 == 0 &&
-                      tiles_h <= MAX_COOP_BANDS && tiles_h >= 4 &&
+    // (with the layer's own padding and dilation too, at unit strides: the bands are bands of input rows)
+    const int in_bands = (H + 15) / 16;
+    const bool coop = nbands == 1 && !per_tap && (!general || d.stride[0] == 1) && !f32 &&
+                      !(d.flags & CCV3D_FLAG_TWO_KERNELS) && W % 8 == 0 && in_bands <= MAX_COOP_BANDS && tiles_h >= 4 &&
                       (int64_t)N * tiles_h * p.tiles_w * To * NT * (pair ? 2 : 1) >= 4LL * h->sm_count;   // small problems: two kernels
     size_t fixed = 1024 /*alignment slack*/ + align_up(sizeof(TcShared), 128) + 2 * (size_t)p.e_slot + (coop ? 9216 : 0);
     // leave room for staging blocks to be resident next to a convolution CTA when the two overlap
@@ -322,9 +324,9 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
 
     if (coop) {
         if (pev) { cudaEventRecord(pev[0], st); cudaEventRecord(pev[1], st); }
-        if (cudaMemsetAsync(h->band_ctr, 0, (size_t)tiles_h * sizeof(unsigned int), st) != cudaSuccess) return cuda_fail();
+        if (cudaMemsetAsync(h->band_ctr, 0, (size_t)in_bands * sizeof(unsigned int), st) != cudaSuccess) return cuda_fail();
         p.band_ctr = h->band_ctr;
-        p.nbands = tiles_h;
+        p.nbands = in_bands;
         p.ty_begin = 0;
         p.tiles_h = tiles_h;
         const int64_t total = (int64_t)N * tiles_h * p.tiles_w * To * NT;

@@ -137,6 +137,19 @@ __global__ void bias_to_f32_kernel(const TIn* __restrict__ b, float* __restrict_
     if (i < n_pad) out[i] = (b && i < n) ? ld_as_float(b + i) : 0.f;
 }
 
+// ---- image-row slabs (height-split halo exchange) ----
+// Copies `rows` image rows of every plane: unit = 16-byte vectors (V = uint4) or bytes (V = unsigned char);
+// chunk = units per slab of rows, pitches in units per plane, src == nullptr writes zeros.
+template <typename V>
+__global__ void rows_copy_kernel(V* __restrict__ dst, int64_t dst_pitch, const V* __restrict__ src, int64_t src_pitch,
+                                 int64_t planes, int64_t chunk) {
+    const int64_t total = planes * chunk;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t pl = i / chunk, off = i - pl * chunk;
+        dst[pl * dst_pitch + off] = src ? __ldg(src + pl * src_pitch + off) : V{};
+    }
+}
+
 // ---- chain glue ----
 __global__ void add_bf16_kernel(const __nv_bfloat16* __restrict__ a, const __nv_bfloat16* __restrict__ b,
                                 __nv_bfloat16* __restrict__ y, int64_t n) {

@@ -1,5 +1,6 @@
 // The implicit-GEMM kernel (conv3d_tcgen05_kernel) with its parameter blocks, and the bounded-wait self-test.
 #pragma once
+#include <type_traits>
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -35,7 +36,7 @@ struct TcParams {
     uint32_t tmem_cols;       // power of two >= NB*NPAD*ACC
     long long wait_limit_clk; // bound of every mbarrier wait, in SM clocks
     unsigned int* band_ctr;   // cooperative staging: per 16-row band, the number of CTAs that have staged their share
-    int nbands;               // cooperative staging: bands of the image (= tile rows)
+    int nbands;               // cooperative staging: 16-row bands of the input image
     // general geometry (Eq. (2) with the layer's own padding and dilation, Eq. (1) with d_t); when `general` is 0
     // the kernel uses pad = (k-1)/2 and unit dilation.  H and W above are the OUTPUT extents; the input extents
     // only live in the tensor map.  Spatial stride > 1 is served by the per-tap mode with a strided tensor map.
@@ -132,10 +133,9 @@ __device__ __forceinline__ void load_res32(const __nv_bfloat16* res_row, bool va
 
 // Two neighbouring output channels: round conv + bias to BF16 once; with a residual, add it to that rounded value
 // in FP32 and round again (the result of a BF16 convolution followed by a BF16 addition).
-__device__ __forceinline__ float silu_f32(float v) { return v / (1.f + __expf(-v)); }
+__device__ __forceinline__ float silu_f32(float v) { return __fdividef(v, 1.f + __expf(-v)); }
 
-__device__ __forceinline__ uint32_t epi_pair(float a0, float a1, uint32_t res_pair, bool has_res, bool act = false) {
-    if (act) { a0 = silu_f32(a0); a1 = silu_f32(a1); }      // optional SiLU on conv + bias, in FP32, before the one rounding
+__device__ __forceinline__ uint32_t epi_pair(float a0, float a1, uint32_t res_pair, bool has_res) {
     __nv_bfloat162 o = __floats2bfloat162_rn(a0, a1);
     if (has_res) {
         const float2 of = __bfloat1622float2(o);
@@ -297,8 +297,10 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                 const int n = r / p.tiles_h;
                 const int h0 = ty * 16, w0 = tx * TWT + wofs;
                 if (COOP) {
-                    // the halo of tile row ty reaches into bands ty-1 .. ty+1
-                    const int need = (ty + 2 < p.nbands) ? ty + 2 : p.nbands;
+                    // the halo of tile row ty ends at input row 16 ty + 15 + (kh-1) d_h - pad_h (bands ty-1 .. ty+1 of
+                    // a size-preserving 3-tap layer); bands are bands of INPUT rows
+                    const int last_band = (h0 + 15 + (p.kh - 1) * dlh - ph) >> 4;
+                    const int need = (last_band + 1 < p.nbands) ? last_band + 1 : p.nbands;
                     if (bands_ready < need) {
                         const long long t0 = clock64();
                         while (ok && bands_ready < need) {
@@ -569,7 +571,6 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
         const bool elected = (threadIdx.x == 4 * 32);
         constexpr bool RING = !FUSED && !COOP;                 // frame-ring output and residual: plain variant only
         const bool has_res = RING && p.res != nullptr;
-        const bool act = p.act != 0;
         int ebuf = 0;
         // bias: a shared-memory copy when the padded channel count fits.  A global load per element costs little
         // while the next tile's MMAs run, but its latency sits in the exposed tail of a CTA's last tile: 11 us
@@ -579,164 +580,177 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
             for (int i = threadIdx.x - 128; i < p.NT * p.NPAD; i += 128) sh->bias_s[i] = __ldg(p.bias + i);
         epi_bar_sync();
         const float* bias = bias_smem ? sh->bias_s : p.bias;
-        for (int tile = cta_lin; ok && tile < p.total_tiles; tile += cta_cnt) {
-            const int nt = tile % p.NT;
-            int r = tile / p.NT;
-            const int t = r % p.T; r /= p.T;
-            const int tx = r % p.tiles_w; r /= p.tiles_w;
-            const int ty = p.ty_begin + r % p.tiles_h;
-            const int n = r / p.tiles_h;
-            const int h = ty * 16 + (m >> 3);
-            const int wt = tx * TWT + wofs;                  // first pixel column of this CTA's part of the tile
-            // residual: pixel (h, w) of frame t holds its Cout channels in blocks of res_KB (64 bytes per 32 channels)
-            const __nv_bfloat16* res_row = nullptr;
-            if (has_res && h < p.H) {
-                int rs = p.res_f0 + t;
-                if (rs >= p.res_F) rs -= p.res_F;
-                res_row = p.res + (((int64_t)n * p.res_F + rs) * p.res_CB * HW + (int64_t)h * p.W) * p.res_KB;
-            }
-            // the residual of the first chunk is fetched while the MMAs of this tile still run; every later chunk's
-            // residual is fetched one chunk ahead
-            uint32_t rr_next[16];
-            if (p.epi_tma) load_res32(res_row, wt + (m & 7) < p.W, wt + (m & 7), nt * p.NPAD, p, HW, rr_next);
-            ok = mbar_wait(&sh->acc_full[acc], pacc, sh, p, SITE_ACC_FULL);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t t_acc = tmem_base + (uint32_t)(acc * ASETS * NB) * p.NPAD + ((uint32_t)(q * 32) << 16);
-            // TF32: was the second accumulator of the last pass used (at least two stages per pass)?
-            const int dt0e = (p.first_frame - t * stt > 0) ? (p.first_frame - t * stt + dlt - 1) / dlt : 0;
-            const bool two_acc = TF32 && (p.kt - dt0e) * p.CB >= 2;
-            if (p.epi_tma) {
-                // BF16 tile chunks -> shared memory -> one TMA store per chunk.  NCTHW output: [ECH channels][16 rows]
-                // [TW pixels]; ring output: [16 rows][TW pixels][32 channels] with the 64-byte swizzle of the tensor map.
-                for (int c0 = 0; c0 < p.NPAD; c0 += p.ECH) {
-                    if (elected) bulk_wait_read<1>();   // the store that last read this buffer has finished reading
-                    epi_bar_sync();
-                    uint8_t* stg = epi_buf + (size_t)ebuf * p.e_slot;
-                    const int co0 = nt * p.NPAD + c0;
-#pragma unroll
-                    for (int blk = 0; blk < NB; ++blk) {
-                        uint32_t rr[16];
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) rr[j] = rr_next[j];
-                        if (has_res) {
-                            const int wn = wt + ((blk + 1 < NB) ? blk + 1 : 0) * 8 + (m & 7);
-                            const int con = (blk + 1 < NB) ? co0 : co0 + p.ECH;
-                            load_res32(res_row, wn < p.W && con < (nt + 1) * p.NPAD, wn, con, p, HW, rr_next);
-                        }
-                        uint32_t v[32];
-                        if (p.ECH == 32) tc_ld32(t_acc + blk * p.NPAD + c0, v); else tc_ld16(t_acc + blk * p.NPAD + c0, v);
-                        tc_wait_ld();
-                        uint32_t pk[16];
-                        float bb[32];                       // the chunk's bias: eight 16-byte reads (co0 is a multiple of 16)
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            const float4 b4 = (4 * j < p.ECH) ? *reinterpret_cast<const float4*>(bias + co0 + 4 * j)
-                                                              : make_float4(0.f, 0.f, 0.f, 0.f);
-                            bb[4 * j] = b4.x; bb[4 * j + 1] = b4.y; bb[4 * j + 2] = b4.z; bb[4 * j + 3] = b4.w;
-                        }
-#pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            pk[j] = (2 * j < p.ECH) ? epi_pair(__uint_as_float(v[2 * j]) + bb[2 * j],
-                                                               __uint_as_float(v[2 * j + 1]) + bb[2 * j + 1], rr[j], has_res, act)
-                                                    : 0u;
-                        const uint32_t px = (uint32_t)((m >> 3) * TW + blk * 8 + (m & 7));   // pixel of the tile, row-major
-                        if (RING && p.epi_tma == 2) {
-                            uint4* row = reinterpret_cast<uint4*>(stg + (size_t)px * 64);
-                            const uint32_t sw = (px >> 1) & 3u;
-#pragma unroll
-                            for (int c = 0; c < 4; ++c)
-                                row[c ^ sw] = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-                        } else {
-                            unsigned short* dst = reinterpret_cast<unsigned short*>(stg) + px;
-#pragma unroll
-                            for (int j = 0; j < 16; ++j)
-                                if (2 * j < p.ECH) {
-                                    dst[(2 * j) * 16 * TW] = (unsigned short)(pk[j] & 0xFFFFu);
-                                    dst[(2 * j + 1) * 16 * TW] = (unsigned short)(pk[j] >> 16);
-                                }
-                        }
-                    }
-                    fence_async_smem();
-                    epi_bar_sync();
-                    if (elected) {
-                        if (RING && p.epi_tma == 2 && p.up_rt > 0) {
-                            // fused nearest-neighbour upsample: the tensor map walks the 2H x 2W ring with a traversal
-                            // stride of 2 pixels, so one store drops the tile onto every second pixel from (b, a)
-                            for (int j = 0; j < p.up_rt; ++j) {
-                                const int os = (p.out_f0 + t * p.up_rt + j) % p.out_F;
-                                for (int ab = 0; ab < 4; ++ab)
-                                    tma_store_5d(&tm_o, smem_u32(stg), co0 % p.out_KB, 2 * wt + (ab & 1), 2 * ty * 16 + (ab >> 1),
-                                                 co0 / p.out_KB, n * p.out_F + os);
-                            }
-                        } else if (RING && p.epi_tma == 2) {
-                            int os = p.out_f0 + t;
-                            if (os >= p.out_F) os -= p.out_F;
-                            tma_store_5d(&tm_o, smem_u32(stg), co0 % p.out_KB, wt, ty * 16, co0 / p.out_KB, n * p.out_F + os);
-                        } else {
-                            tma_store_5d(&tm_o, smem_u32(stg), wt, ty * 16, t, co0, n);
-                        }
-                        bulk_commit();
-                    }
-                    ebuf ^= 1;
+        // the tile loop exists twice, with and without the optional SiLU, so that the plain epilogue carries no trace of it
+        auto run_tiles = [&](auto act_c) {
+            constexpr bool ACT = decltype(act_c)::value;
+            for (int tile = cta_lin; ok && tile < p.total_tiles; tile += cta_cnt) {
+                const int nt = tile % p.NT;
+                int r = tile / p.NT;
+                const int t = r % p.T; r /= p.T;
+                const int tx = r % p.tiles_w; r /= p.tiles_w;
+                const int ty = p.ty_begin + r % p.tiles_h;
+                const int n = r / p.tiles_h;
+                const int h = ty * 16 + (m >> 3);
+                const int wt = tx * TWT + wofs;                  // first pixel column of this CTA's part of the tile
+                // residual: pixel (h, w) of frame t holds its Cout channels in blocks of res_KB (64 bytes per 32 channels)
+                const __nv_bfloat16* res_row = nullptr;
+                if (has_res && h < p.H) {
+                    int rs = p.res_f0 + t;
+                    if (rs >= p.res_F) rs -= p.res_F;
+                    res_row = p.res + (((int64_t)n * p.res_F + rs) * p.res_CB * HW + (int64_t)h * p.W) * p.res_KB;
                 }
-            } else {
-#pragma unroll 1
-                for (int blk = 0; blk < NB; ++blk) {
-                    const int w = wt + blk * 8 + (m & 7);
-                    const bool valid = h < p.H && w < p.W;
-                    const int64_t pix = (int64_t)t * HW + (int64_t)h * p.W + w;
-#pragma unroll 1
-                    for (int c0 = 0; c0 < p.NPAD; c0 += 32) {
+                // the residual of the first chunk is fetched while the MMAs of this tile still run; every later chunk's
+                // residual is fetched one chunk ahead
+                uint32_t rr_next[16];
+                if (p.epi_tma) load_res32(res_row, wt + (m & 7) < p.W, wt + (m & 7), nt * p.NPAD, p, HW, rr_next);
+                ok = mbar_wait(&sh->acc_full[acc], pacc, sh, p, SITE_ACC_FULL);
+                ok = __all_sync(0xffffffffu, ok);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t t_acc = tmem_base + (uint32_t)(acc * ASETS * NB) * p.NPAD + ((uint32_t)(q * 32) << 16);
+                // TF32: was the second accumulator of the last pass used (at least two stages per pass)?
+                const int dt0e = (p.first_frame - t * stt > 0) ? (p.first_frame - t * stt + dlt - 1) / dlt : 0;
+                const bool two_acc = TF32 && (p.kt - dt0e) * p.CB >= 2;
+                if (p.epi_tma) {
+                    // BF16 tile chunks -> shared memory -> one TMA store per chunk.  NCTHW output: [ECH channels][16 rows]
+                    // [TW pixels]; ring output: [16 rows][TW pixels][32 channels] with the 64-byte swizzle of the tensor map.
+                    for (int c0 = 0; c0 < p.NPAD; c0 += p.ECH) {
+                        if (elected) bulk_wait_read<1>();   // the store that last read this buffer has finished reading
+                        epi_bar_sync();
+                        uint8_t* stg = epi_buf + (size_t)ebuf * p.e_slot;
                         const int co0 = nt * p.NPAD + c0;
-                        uint32_t rr[16];
-                        load_res32(res_row, valid, w, co0, p, HW, rr);
-                        uint32_t v[32];
-                        const int nc = (p.NPAD - c0 >= 32) ? 32 : 16;
-                        if (nc == 32) tc_ld32(t_acc + blk * p.NPAD + c0, v); else tc_ld16(t_acc + blk * p.NPAD + c0, v);
-                        tc_wait_ld();
-                        if (two_acc) {
-                            uint32_t v2[32];
-                            if (nc == 32) tc_ld32(t_acc + (NB + blk) * p.NPAD + c0, v2); else tc_ld16(t_acc + (NB + blk) * p.NPAD + c0, v2);
+    #pragma unroll
+                        for (int blk = 0; blk < NB; ++blk) {
+                            uint32_t rr[16];
+    #pragma unroll
+                            for (int j = 0; j < 16; ++j) rr[j] = rr_next[j];
+                            if (has_res) {
+                                const int wn = wt + ((blk + 1 < NB) ? blk + 1 : 0) * 8 + (m & 7);
+                                const int con = (blk + 1 < NB) ? co0 : co0 + p.ECH;
+                                load_res32(res_row, wn < p.W && con < (nt + 1) * p.NPAD, wn, con, p, HW, rr_next);
+                            }
+                            uint32_t v[32];
+                            if (p.ECH == 32) tc_ld32(t_acc + blk * p.NPAD + c0, v); else tc_ld16(t_acc + blk * p.NPAD + c0, v);
                             tc_wait_ld();
-#pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                if (j < nc) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(v2[j]));
-                        }
-                        if (valid) {
-                            if (p.out_f32) {
-#pragma unroll
-                                for (int j = 0; j < 32; ++j) {
-                                    const int co = co0 + j;
-                                    if (j < nc && co < p.Cout) {
-                                        const float val = __uint_as_float(v[j]) + bias[co];
-                                        reinterpret_cast<float*>(p.out)[((int64_t)n * p.Cout + co) * p.T * HW + pix] = act ? silu_f32(val) : val;
-                                    }
-                                }
+                            uint32_t pk[16];
+                            float bb[32];                       // the chunk's bias: eight 16-byte reads (co0 is a multiple of 16)
+    #pragma unroll
+                            for (int j = 0; j < 8; ++j) {
+                                const float4 b4 = (4 * j < p.ECH) ? *reinterpret_cast<const float4*>(bias + co0 + 4 * j)
+                                                                  : make_float4(0.f, 0.f, 0.f, 0.f);
+                                bb[4 * j] = b4.x; bb[4 * j + 1] = b4.y; bb[4 * j + 2] = b4.z; bb[4 * j + 3] = b4.w;
+                            }
+    #pragma unroll
+                            for (int j = 0; j < 32; ++j) bb[j] += __uint_as_float(v[j]);
+                            if (ACT) {      // optional SiLU on conv + bias, in FP32, before the one rounding: one uniform branch per chunk
+    #pragma unroll
+                                for (int j = 0; j < 32; ++j) bb[j] = silu_f32(bb[j]);
+                            }
+    #pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                pk[j] = (2 * j < p.ECH) ? epi_pair(bb[2 * j], bb[2 * j + 1], rr[j], has_res) : 0u;
+                            const uint32_t px = (uint32_t)((m >> 3) * TW + blk * 8 + (m & 7));   // pixel of the tile, row-major
+                            if (RING && p.epi_tma == 2) {
+                                uint4* row = reinterpret_cast<uint4*>(stg + (size_t)px * 64);
+                                const uint32_t sw = (px >> 1) & 3u;
+    #pragma unroll
+                                for (int c = 0; c < 4; ++c)
+                                    row[c ^ sw] = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
                             } else {
-#pragma unroll
-                                for (int j = 0; j < 16; ++j) {
-                                    const int co = co0 + 2 * j;
-                                    if (2 * j < nc) {
-                                        const uint32_t pr = epi_pair(__uint_as_float(v[2 * j]) + bias[co],
-                                                                     __uint_as_float(v[2 * j + 1]) + bias[co + 1], rr[j], has_res, act);
-                                        unsigned short* o = reinterpret_cast<unsigned short*>(p.out) +
-                                                            ((int64_t)n * p.Cout + co) * p.T * HW + pix;
-                                        if (co < p.Cout) o[0] = (unsigned short)(pr & 0xFFFFu);
-                                        if (co + 1 < p.Cout) o[(int64_t)p.T * HW] = (unsigned short)(pr >> 16);
+                                unsigned short* dst = reinterpret_cast<unsigned short*>(stg) + px;
+    #pragma unroll
+                                for (int j = 0; j < 16; ++j)
+                                    if (2 * j < p.ECH) {
+                                        dst[(2 * j) * 16 * TW] = (unsigned short)(pk[j] & 0xFFFFu);
+                                        dst[(2 * j + 1) * 16 * TW] = (unsigned short)(pk[j] >> 16);
+                                    }
+                            }
+                        }
+                        fence_async_smem();
+                        epi_bar_sync();
+                        if (elected) {
+                            if (RING && p.epi_tma == 2 && p.up_rt > 0) {
+                                // fused nearest-neighbour upsample: the tensor map walks the 2H x 2W ring with a traversal
+                                // stride of 2 pixels, so one store drops the tile onto every second pixel from (b, a)
+                                for (int j = 0; j < p.up_rt; ++j) {
+                                    const int os = (p.out_f0 + t * p.up_rt + j) % p.out_F;
+                                    for (int ab = 0; ab < 4; ++ab)
+                                        tma_store_5d(&tm_o, smem_u32(stg), co0 % p.out_KB, 2 * wt + (ab & 1), 2 * ty * 16 + (ab >> 1),
+                                                     co0 / p.out_KB, n * p.out_F + os);
+                                }
+                            } else if (RING && p.epi_tma == 2) {
+                                int os = p.out_f0 + t;
+                                if (os >= p.out_F) os -= p.out_F;
+                                tma_store_5d(&tm_o, smem_u32(stg), co0 % p.out_KB, wt, ty * 16, co0 / p.out_KB, n * p.out_F + os);
+                            } else {
+                                tma_store_5d(&tm_o, smem_u32(stg), wt, ty * 16, t, co0, n);
+                            }
+                            bulk_commit();
+                        }
+                        ebuf ^= 1;
+                    }
+                } else {
+    #pragma unroll 1
+                    for (int blk = 0; blk < NB; ++blk) {
+                        const int w = wt + blk * 8 + (m & 7);
+                        const bool valid = h < p.H && w < p.W;
+                        const int64_t pix = (int64_t)t * HW + (int64_t)h * p.W + w;
+    #pragma unroll 1
+                        for (int c0 = 0; c0 < p.NPAD; c0 += 32) {
+                            const int co0 = nt * p.NPAD + c0;
+                            uint32_t rr[16];
+                            load_res32(res_row, valid, w, co0, p, HW, rr);
+                            uint32_t v[32];
+                            const int nc = (p.NPAD - c0 >= 32) ? 32 : 16;
+                            if (nc == 32) tc_ld32(t_acc + blk * p.NPAD + c0, v); else tc_ld16(t_acc + blk * p.NPAD + c0, v);
+                            tc_wait_ld();
+                            if (two_acc) {
+                                uint32_t v2[32];
+                                if (nc == 32) tc_ld32(t_acc + (NB + blk) * p.NPAD + c0, v2); else tc_ld16(t_acc + (NB + blk) * p.NPAD + c0, v2);
+                                tc_wait_ld();
+    #pragma unroll
+                                for (int j = 0; j < 32; ++j)
+                                    if (j < nc) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(v2[j]));
+                            }
+                            if (valid) {
+                                float a[32];
+    #pragma unroll
+                                for (int j = 0; j < 32; ++j) a[j] = (j < nc) ? __uint_as_float(v[j]) + bias[co0 + j] : 0.f;
+                                if (ACT) {      // optional SiLU on conv + bias: one uniform branch per chunk
+    #pragma unroll
+                                    for (int j = 0; j < 32; ++j) a[j] = silu_f32(a[j]);
+                                }
+                                if (p.out_f32) {
+    #pragma unroll
+                                    for (int j = 0; j < 32; ++j) {
+                                        const int co = co0 + j;
+                                        if (j < nc && co < p.Cout)
+                                            reinterpret_cast<float*>(p.out)[((int64_t)n * p.Cout + co) * p.T * HW + pix] = a[j];
+                                    }
+                                } else {
+    #pragma unroll
+                                    for (int j = 0; j < 16; ++j) {
+                                        const int co = co0 + 2 * j;
+                                        if (2 * j < nc) {
+                                            const uint32_t pr = epi_pair(a[2 * j], a[2 * j + 1], rr[j], has_res);
+                                            unsigned short* o = reinterpret_cast<unsigned short*>(p.out) +
+                                                                ((int64_t)n * p.Cout + co) * p.T * HW + pix;
+                                            if (co < p.Cout) o[0] = (unsigned short)(pr & 0xFFFFu);
+                                            if (co + 1 < p.Cout) o[(int64_t)p.T * HW] = (unsigned short)(pr >> 16);
+                                        }
                                     }
                                 }
                             }
                         }
                     }
                 }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) { if (PAIR) mbar_arrive_leader(smem_u32(&sh->acc_empty[acc])); else mbar_arrive(smem_u32(&sh->acc_empty[acc])); }
+                if (++acc == p.ACC) { acc = 0; pacc ^= 1; }
             }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) { if (PAIR) mbar_arrive_leader(smem_u32(&sh->acc_empty[acc])); else mbar_arrive(smem_u32(&sh->acc_empty[acc])); }
-            if (++acc == p.ACC) { acc = 0; pacc ^= 1; }
-        }
+        };
+        if (p.act) run_tiles(std::true_type{}); else run_tiles(std::false_type{});
         if (p.epi_tma && elected) bulk_wait_all();   // all stores of this CTA are complete before it exits
     }
 
