@@ -123,7 +123,10 @@ typedef struct {
  * workspace (see ccv3d_forward).  The caller owns everything else.
  * Two environment variables are read here, for diagnosis only: CCV3D_WAIT_LIMIT_MS (1..10000, default about one
  * second of SM clocks) bounds every wait inside the kernels; CCV3D_NO_PDL (any value) launches the frame-ring
- * kernels without programmatic stream serialization.
+ * kernels without programmatic stream serialization; CCV3D_NO_COOP_LAUNCH (any value) launches the
+ * cooperative-staging kernels as ordinary launches (a profiler that replays kernels refuses cooperative launches of
+ * clusters; only safe while nothing else runs on the device, since the CTAs of such a kernel wait for one another,
+ * within the bound of every wait).
  */
 ccv3d_status ccv3d_create(ccv3d_handle** out_h, const ccv3d_desc* d, const void* w_dev, const void* b_dev,
                           void* stream);

@@ -80,6 +80,7 @@ struct ccv3d_handle {
     int64_t prof_n;
     cudaEvent_t* prof_ev;   // PROF_SLOTS x 3 events, created on first enable
     int pdl;             // 1: convolution kernels on frame rings are launched with programmatic stream serialization
+    int coop_launch;     // 1: cooperative-staging kernels are launched with the cooperative attribute
     int cluster_ok;      // the device launches thread-block clusters (needed for CTA pairs)
     int call_cf;         // history frames held by the cache of the call being served (set by the entry points)
     ccv3d_counters ctr;
@@ -238,6 +239,7 @@ ccv3d_status ccv3d_create(ccv3d_handle** out_h, const ccv3d_desc* d, const void*
         if (v > 0 && v <= 10000) h->wait_limit_clk = (long long)prop.clockRate * v;
     }
     h->pdl = getenv("CCV3D_NO_PDL") ? 0 : 1;
+    h->coop_launch = getenv("CCV3D_NO_COOP_LAUNCH") ? 0 : 1;
     if (cudaDeviceGetAttribute(&h->cluster_ok, cudaDevAttrClusterLaunch, dev) != cudaSuccess) {
         cudaGetLastError();
         h->cluster_ok = 0;

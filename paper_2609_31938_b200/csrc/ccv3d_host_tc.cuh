@@ -21,7 +21,7 @@ ccv3d_status launch_tc_coop(ccv3d_handle* h, const TcParams& p, const StageParam
     attr[0].id = cudaLaunchAttributeCooperative;
     attr[0].val.cooperative = 1;
     cfg.attrs = attr;
-    cfg.numAttrs = 1;
+    cfg.numAttrs = h->coop_launch ? 1 : 0;
     if (cudaLaunchKernelEx(&cfg, kern, h->tm_a, h->tm_a, h->tm_o, p, sp) != cudaSuccess) return cuda_fail();
     if (cudaGetLastError() != cudaSuccess) return cuda_fail();
     h->ctr.kernel_launches++;
@@ -84,7 +84,7 @@ ccv3d_status launch_tc_pair(ccv3d_handle* h, const CUtensorMap& tm_a, const CUte
         attr[1].val.cooperative = 1;
     }
     cfg.attrs = attr;
-    cfg.numAttrs = (COOP || h->pdl) ? 2 : 1;
+    cfg.numAttrs = ((COOP && h->coop_launch) || (!COOP && h->pdl)) ? 2 : 1;
     if (cudaLaunchKernelEx(&cfg, kern, tm_a, tm_w, tm_o, p, sp) != cudaSuccess) return cuda_fail();
     if (cudaGetLastError() != cudaSuccess) return cuda_fail();
     h->ctr.kernel_launches++;
