@@ -123,7 +123,8 @@ typedef struct {
  * workspace (see ccv3d_forward).  The caller owns everything else.
  * Two environment variables are read here, for diagnosis only: CCV3D_WAIT_LIMIT_MS (1..10000, default about one
  * second of SM clocks) bounds every wait inside the kernels; CCV3D_NO_PDL (any value) launches the frame-ring
- * kernels without programmatic stream serialization; CCV3D_NO_COOP_LAUNCH (any value) launches the
+ * kernels without programmatic stream serialization; CCV3D_NO_COOP_LAUNCH (any value; implied when the
+ * process runs under Nsight Compute, which sets NV_COMPUTE_PROFILER_PERFWORKS_DIR) launches the
  * cooperative-staging kernels as ordinary launches (a profiler that replays kernels refuses cooperative launches of
  * clusters; only safe while nothing else runs on the device, since the CTAs of such a kernel wait for one another,
  * within the bound of every wait).

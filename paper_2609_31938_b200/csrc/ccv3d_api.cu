@@ -239,7 +239,9 @@ ccv3d_status ccv3d_create(ccv3d_handle** out_h, const ccv3d_desc* d, const void*
         if (v > 0 && v <= 10000) h->wait_limit_clk = (long long)prop.clockRate * v;
     }
     h->pdl = getenv("CCV3D_NO_PDL") ? 0 : 1;
-    h->coop_launch = getenv("CCV3D_NO_COOP_LAUNCH") ? 0 : 1;
+    // a kernel-replaying profiler (it announces itself through NV_COMPUTE_PROFILER_PERFWORKS_DIR) refuses
+    // cooperative launches of clusters: ordinary launches there, on a device the profiled process has to itself
+    h->coop_launch = (getenv("CCV3D_NO_COOP_LAUNCH") || getenv("NV_COMPUTE_PROFILER_PERFWORKS_DIR")) ? 0 : 1;
     if (cudaDeviceGetAttribute(&h->cluster_ok, cudaDevAttrClusterLaunch, dev) != cudaSuccess) {
         cudaGetLastError();
         h->cluster_ok = 0;
