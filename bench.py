@@ -358,7 +358,7 @@ def hsplit_leg(dev):
     import math
     import torch
     import paper_2609_31938_b200 as ccv
-    from paper_2609_31938_b200.hsplit import HSplitCausalConv3d
+    from paper_2609_31938_b200.hsplit import HSplitCausalConv3d, HSplitRingConv3d
     name = "cfg3_bf16_192"
     d = {k: v for k, v in si.CONFIGS[name].items() if k not in ("dtype", "x_dist")}
     N, Cin, Cout, T, H, W, k = d["N"], d["Cin"], d["Cout"], d["T"], d["H"], d["W"], d["k"]
@@ -366,8 +366,9 @@ def hsplit_leg(dev):
     rnd = lambda *shape, std=1.0: (torch.randn(*shape, device=dev, generator=gen) * std).to(torch.bfloat16)
     w, b = rnd(Cout, Cin, *k, std=1.0 / math.sqrt(Cin * k[0] * k[1] * k[2])), rnd(Cout, std=math.sqrt(0.1))
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    out = {"workload": name, "note": "pack + slab assembly + layer on the slab, for rank 1 of the world (halo rows on both sides of its slab); "
-                                     "neighbour exchange (NCCL send/recv) not included"}
+    out = {"workload": name, "note": "rank 1 of the world (halo rows on both sides of its slab). NCTHW: pack + slab assembly + layer "
+                                     "on the slab; resident: the ring call on the slab + pack and unpack of the output's halo "
+                                     "rows. Neighbour exchange (NCCL send/recv) not included"}
     for world in (2, 4, 8):
         layer = HSplitCausalConv3d(w, b, H, min(1, world - 1), world, transport=None)
         p = layer.plan
@@ -389,12 +390,36 @@ def hsplit_leg(dev):
         torch.cuda.synchronize()
         ms = e0.elapsed_time(e1) / 10
         flops = si.conv_flops(**d) * p.rows / H
+        # the same rank on frame rings: the ring call on the slab, then pack + unpack of the output's halo rows
+        rl = HSplitRingConv3d(w, b, H, min(1, world - 1), world, transport=None)
+        F = T + k[0] - 1
+        rin, rout = rl.ring(N, Cin, F, W), rl.ring(N, Cout, T, W)
+        rin.buf.normal_()
+        slot = [k[0] - 1]
+
+        def ring_rank_step():
+            rl.conv.forward_ring(rin, slot[0], k[0] - 1, T, out_ring=rout)
+            to_up, to_down = rl.pack(rout, 0, T)
+            rl.unpack(rout, 0, T, to_down if to_down is not None else to_up, to_up if to_up is not None else to_down)
+            slot[0] = (slot[0] + T) % F
+
+        for _ in range(3):
+            ring_rank_step()
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(10):
+            ring_rank_step()
+        e1.record()
+        torch.cuda.synchronize()
+        rms = e0.elapsed_time(e1) / 10
         out[f"world{world}"] = {"rows": p.rows, "slab_rows": p.slab_rows, "ms_per_rank_step": ms,
                                 "tflops_per_rank": flops / (ms * 1e-3) / 1e12,
+                                "resident_ms_per_rank_step": rms, "resident_tflops_per_rank": flops / (rms * 1e-3) / 1e12,
                                 "halo_bytes_sent_per_step": int(2 * N * Cin * T * (p.top + p.bot) * W)}
-        assert layer.conv.device_status()[0] == ccv.OK
+        assert layer.conv.device_status()[0] == ccv.OK and rl.conv.device_status()[0] == ccv.OK
         layer.close()
-        del xb, cache, halo_up, halo_down
+        rl.close()
+        del xb, cache, halo_up, halo_down, rin, rout
         torch.cuda.empty_cache()
     return out
 

@@ -198,3 +198,148 @@ def forward_all_local(layers, x_bands, cache_slabs=None):
         outs.append(o)
         caches.append(c)
     return outs, caches
+
+
+# ------------------------------------------------------------------------------------------------------------------
+# Height-split on resident activations (frame rings)
+# ------------------------------------------------------------------------------------------------------------------
+# A rank's rings hold its slab (halo rows included) instead of the whole image, and a layer is the unchanged ring
+# call with its own zero padding on the slab.  The layer's output rows at halo positions come out wrong (they saw
+# zero padding where the neighbour's rows belong) - but those are exactly the rows the next layer must get from the
+# neighbours anyway: after every layer the band's edge rows are sent, the halo rows of the output ring are
+# overwritten with what the neighbours sent (zeros where the image ends), and the ring is a valid input slab.  No
+# slab assembly, no cache: the temporal history is whatever earlier chunks left in the ring, halos included.  Cost
+# per layer over the unsplit share: 2 * halo extra rows of convolution and four small row copies.
+
+def _frame_runs(slot0, T, F):
+    """Slots slot0 .. slot0+T-1 (mod F) as contiguous runs [(first slot, frames, first frame index)]."""
+    s = slot0 % F
+    first = min(T, F - s)
+    runs = [(s, first, 0)]
+    if first < T:
+        runs.append((0, T - first, first))
+    return runs
+
+
+def ring_rows_copy(ring, slot0, T, row0, rows, buf, to_ring):
+    """Rows row0 .. row0+rows-1 of frames slot0.. of `ring`  <->  buf [N][T][C/KB][rows][W][KB] (contiguous).
+    to_ring with buf None writes zeros."""
+    import torch
+    st = torch.cuda.current_stream().cuda_stream
+    CB = ring.C // ring.KB
+    row_bytes = ring.W * ring.KB * 2
+    for n in range(ring.N):
+        for s, cnt, t0 in _frame_runs(slot0, T, ring.F):
+            rp = ring.buf.data_ptr() + ((n * ring.F + s) * CB) * ring.H * row_bytes
+            bp = None if buf is None else buf.data_ptr() + ((n * T + t0) * CB) * rows * row_bytes
+            if to_ring:
+                st_ = ccv3d_rows_copy(rp, ring.H, row0, bp, rows, 0, cnt * CB, rows, row_bytes, st)
+            else:
+                st_ = ccv3d_rows_copy(bp, rows, 0, rp, ring.H, row0, cnt * CB, rows, row_bytes, st)
+            if st_ != OK:
+                raise Ccv3dError(st_, "ccv3d_rows_copy")
+
+
+class HSplitRingConv3d:
+    """One layer of a height-split stage on frame rings.  All layers that share rings share the slab geometry, so
+    `halo` is the stage's (the largest (kh-1)/2 of its layers; a 1x1x1 layer in a 3x3 stage runs with halo 1)."""
+
+    def __init__(self, w, b, H, rank, world, halo=None, transport=None, flags=0):
+        kt, kh, kw = w.shape[2:]
+        own = (kh - 1) // 2
+        halo = own if halo is None else halo
+        if kh % 2 == 0 or halo < own:
+            raise ValueError("the stage's halo must cover this layer's reach in h")
+        self.plan = halo_plan(H, world, rank, 2 * halo + 1, halo)
+        self.transport = transport if transport is not None else (DistTransport() if world > 1 else None)
+        self.conv = CausalConv3d(w, b, flags=flags)           # standard geometry: zero padding on the slab
+
+    def ring(self, N, C, F, W):
+        from . import FrameRing
+        return FrameRing(N, C, F, self.plan.slab_rows, W, zero=True)
+
+    def _buf(self, ring, T, rows):
+        import torch
+        return torch.empty((ring.N, T, ring.C // ring.KB, rows, ring.W, ring.KB), dtype=torch.bfloat16, device="cuda")
+
+    def pack(self, ring, slot0, T):
+        """The band's edge rows of frames slot0.. as contiguous buffers (to_up, to_down); None where nothing is sent."""
+        p = self.plan
+        assert ring.H == p.slab_rows
+        to_up = to_down = None
+        if p.up is not None and p.bot > 0:
+            to_up = self._buf(ring, T, p.bot)
+            ring_rows_copy(ring, slot0, T, p.top, p.bot, to_up, to_ring=False)
+        if p.down is not None and p.top > 0:
+            to_down = self._buf(ring, T, p.top)
+            ring_rows_copy(ring, slot0, T, p.top + p.rows - p.top, p.top, to_down, to_ring=False)
+        return to_up, to_down
+
+    def recv_buffers(self, ring, T):
+        p = self.plan
+        return (self._buf(ring, T, p.top) if (p.up is not None and p.top > 0) else None,
+                self._buf(ring, T, p.bot) if (p.down is not None and p.bot > 0) else None)
+
+    def unpack(self, ring, slot0, T, from_up, from_down):
+        """Halo rows of frames slot0.. <- the neighbours' rows; zeros where the image ends."""
+        p = self.plan
+        if p.top > 0:
+            ring_rows_copy(ring, slot0, T, 0, p.top, from_up if p.up is not None else None, to_ring=True)
+        if p.bot > 0:
+            ring_rows_copy(ring, slot0, T, p.top + p.rows, p.bot, from_down if p.down is not None else None, to_ring=True)
+
+    def exchange(self, ring, slot0, T):
+        to_up, to_down = self.pack(ring, slot0, T)
+        from_up, from_down = self.recv_buffers(ring, T)
+        if self.transport is not None:
+            self.transport.exchange(self.plan, to_up, to_down, from_up, from_down)
+        self.unpack(ring, slot0, T, from_up, from_down)
+
+    def load_band(self, ring, slot0, x_band, exchange=True):
+        """Chunk input: NCTHW band -> the band rows of ring slots slot0.., then the halo exchange (exchange=False:
+        the caller runs it, e.g. ring_exchange_all_local)."""
+        import torch
+        p = self.plan
+        N, C, T, rows, W = x_band.shape
+        assert rows == p.rows and ring.H == p.slab_rows
+        slab = torch.zeros((N, C, T, p.slab_rows, W), dtype=x_band.dtype, device=x_band.device)
+        CudaRowOps().rows_copy(slab, p.top, x_band, 0, p.rows)
+        ring.load(slot0, slab)
+        if exchange:
+            self.exchange(ring, slot0, T)
+
+    def forward(self, rin, x_slot, hist_frames, T, out_ring, out_slot=0, res=None, res_slot=0):
+        """The layer on this rank's slab rings; `out_ring` leaves as a valid input slab of the next layer."""
+        self.conv.forward_ring(rin, x_slot, hist_frames, T, out_ring=out_ring, out_slot=out_slot, res=res, res_slot=res_slot)
+        self.exchange(out_ring, out_slot, T)
+        return out_ring
+
+    def forward_out(self, rin, x_slot, hist_frames, T, res=None, res_slot=0):
+        """Last layer of a stage: the band as NCTHW [N,Cout,T,rows,W] (no exchange: nobody reads its halo)."""
+        import torch
+        p = self.plan
+        slab = torch.empty((rin.N, self.conv.cout, T, p.slab_rows, rin.W), dtype=torch.bfloat16, device="cuda")
+        self.conv.forward_ring(rin, x_slot, hist_frames, T, out=slab, res=res, res_slot=res_slot)
+        band = torch.empty((rin.N, self.conv.cout, T, p.rows, rin.W), dtype=torch.bfloat16, device="cuda")
+        CudaRowOps().rows_copy(band, 0, slab, p.top, p.rows)
+        return band
+
+    def close(self):
+        self.conv.close()
+
+
+def ring_exchange_all_local(layers, rings, slot0, T):
+    """The halo exchange of all ranks held by one process: pack everywhere, hand the buffers over, unpack."""
+    world = len(layers)
+    packed = [l.pack(r, slot0, T) for l, r in zip(layers, rings)]
+    for k, (l, r) in enumerate(zip(layers, rings)):
+        l.unpack(r, slot0, T, packed[k - 1][1] if k > 0 else None, packed[k + 1][0] if k < world - 1 else None)
+
+
+def ring_forward_all_local(layers, rins, x_slot, hist_frames, T, out_rings, out_slot=0, res_rings=None, res_slot=0):
+    """One layer for all ranks held by one process: every rank's ring call, then the exchange by hand-over."""
+    for k, l in enumerate(layers):
+        l.conv.forward_ring(rins[k], x_slot, hist_frames, T, out_ring=out_rings[k], out_slot=out_slot,
+                            res=None if res_rings is None else res_rings[k], res_slot=res_slot)
+    ring_exchange_all_local(layers, out_rings, out_slot, T)
+    return out_rings

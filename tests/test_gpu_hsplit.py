@@ -89,3 +89,49 @@ def test_bands_equal_unsplit_layer(ccv, Cin, Cout, T, H, W, k, dil, dtype, world
                 assert cnt["calls"] == 2 and cnt["kernel_launches"] == whole.counters()["kernel_launches"], cnt
             l.close()
     whole.close()
+
+
+@pytest.mark.parametrize("world,C,H,W", [(2, 64, 40, 48), (3, 96, 51, 40), (4, 192, 64, 32)])
+def test_ring_block_bands_equal_unsplit(ccv, world, C, H, W):
+    """x <- x + conv2(conv1(x)) on frame rings, streamed over three chunks: every rank's band (its rings hold only its
+    slab; halo rows re-exchanged after each layer, residual added in the epilogue) is bit-identical to the same rows
+    of the unsplit ring path."""
+    from paper_2609_31938_b200.hsplit import (HSplitRingConv3d, ring_exchange_all_local, ring_forward_all_local)
+    T, chunks = 2, 3
+    cs = [si.conv_case(1, C, C, T * chunks, H, W, k=(3, 3, 3), dtype=si.BF16, cache=None, seed=30 + i) for i in range(2)]
+    w = [to_dev(c["w"]) for c in cs]
+    b = [to_dev(c["b"]) for c in cs]
+    x = to_dev(cs[0]["x"])
+    F = T + 2
+    # unsplit reference on full-height rings
+    L = [ccv.CausalConv3d(w[i], b[i]) for i in range(2)]
+    r1, r2 = ccv.FrameRing(1, C, F, H, W, zero=True), ccv.FrameRing(1, C, F, H, W, zero=True)
+    ref, slot = [], 0
+    for c in range(chunks):
+        hist = min(2, c * T)
+        r1.load(slot, x[:, :, c * T:(c + 1) * T].contiguous())
+        L[0].forward_ring(r1, slot, hist, T, out_ring=r2, out_slot=slot)
+        out = torch.empty((1, C, T, H, W), dtype=torch.bfloat16, device="cuda:0")
+        L[1].forward_ring(r2, slot, hist, T, out=out, res=r1, res_slot=slot)
+        ref.append(out)
+        slot = (slot + T) % F
+    ref = torch.cat(ref, dim=2)
+    # the same block, every rank on its slab
+    S = [[HSplitRingConv3d(w[i], b[i], H, r, world) for r in range(world)] for i in range(2)]
+    R1 = [l.ring(1, C, F, W) for l in S[0]]
+    R2 = [l.ring(1, C, F, W) for l in S[0]]
+    got, slot = [], 0
+    for c in range(chunks):
+        hist = min(2, c * T)
+        for r, l in enumerate(S[0]):       # chunk input: the band rows of each rank's ring, then the halos by hand-over
+            l.load_band(R1[r], slot, x[:, :, c * T:(c + 1) * T, l.plan.r0:l.plan.r1].contiguous(), exchange=False)
+        ring_exchange_all_local(S[0], R1, slot, T)
+        ring_forward_all_local(S[0], R1, slot, hist, T, R2, slot)
+        got.append(torch.cat([l.forward_out(R2[r], slot, hist, T, res=R1[r], res_slot=slot) for r, l in enumerate(S[1])], dim=3))
+        slot = (slot + T) % F
+    got = torch.cat(got, dim=2)
+    torch.cuda.synchronize()
+    assert np.array_equal(bits(got), bits(ref))
+    for l in L + S[0] + S[1]:
+        assert l.conv.device_status()[0] == ccv.OK if hasattr(l, "conv") else l.device_status()[0] == ccv.OK
+        l.close()
