@@ -461,3 +461,40 @@ def test_two_handles_on_two_streams_concurrently(ccv):
         assert layers[i].device_status()[0] == ccv.OK
         assert torch.equal(got[i][0], want[i][0]) and torch.equal(got[i][1], want[i][1])
         layers[i].close()
+
+
+def test_random_shapes_every_schedule_agrees(ccv):
+    """Seeded random layers (channel counts, kernel shapes, chunk lengths, image sizes, cache lengths): whatever
+    schedule the library picks by itself (CTA pairs, half-width tiles, cooperative staging, 1x1x1 streaming kernel)
+    gives the bits of the plain two-kernel single-CTA route, run after run, with a clean device status."""
+    import random
+    rnd = random.Random(20261125)
+    g = torch.Generator(device="cuda:0").manual_seed(11)
+    ref_flags = ccv.FLAG_TWO_KERNELS | ccv.FLAG_NO_PAIR
+    done = 0
+    while done < 60:
+        Cin, Cout = rnd.choice([32, 64, 96, 128, 192, 256, 384]), rnd.choice([32, 64, 96, 128, 192, 256, 384])
+        k = rnd.choice([(3, 3, 3), (3, 3, 3), (1, 3, 3), (3, 1, 1), (1, 1, 1), (2, 3, 3)])
+        T = rnd.randint(1, 5)
+        big = rnd.random() < 0.25
+        H = rnd.randint(64, 300) if big else rnd.randint(8, 90)
+        W = 8 * (rnd.randint(20, 64) if big else rnd.randint(2, 24))
+        if Cin * Cout * T * H * W * k[0] * k[1] * k[2] > 2e12:
+            continue
+        cf = rnd.randint(0, k[0] - 1)
+        w = (torch.randn((Cout, Cin) + k, device="cuda:0", generator=g) / (Cin * k[0] * k[1] * k[2]) ** 0.5).to(torch.bfloat16)
+        b = torch.randn((Cout,), device="cuda:0", generator=g).to(torch.bfloat16)
+        x = torch.randn((1, Cin, T, H, W), device="cuda:0", generator=g).to(torch.bfloat16)
+        cache = torch.randn((1, Cin, cf, H, W), device="cuda:0", generator=g).to(torch.bfloat16) if cf else None
+        res = []
+        for flags in (0, 0, ref_flags):
+            layer = ccv.CausalConv3d(w, b, flags=flags)
+            o, nc = layer(x, cache)
+            torch.cuda.synchronize()
+            assert layer.device_status()[0] == ccv.OK, (Cin, Cout, k, T, H, W, cf, flags)
+            res.append((o, nc))
+            layer.close()
+        for o, nc in res[:2]:
+            assert torch.equal(o, res[2][0]), (Cin, Cout, k, T, H, W, cf)
+            assert nc is None or torch.equal(nc, res[2][1]), (Cin, Cout, k, T, H, W, cf)
+        done += 1
