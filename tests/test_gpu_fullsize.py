@@ -106,3 +106,40 @@ def test_full_size_on_frame_rings_sampled(name):
     layer.close()
     del out, abi, x, cch
     torch.cuda.empty_cache()
+
+
+def test_more_than_2_31_elements():
+    """Maximum sizes: x and out hold 2.26e9 elements each (offsets beyond 32 bits in the staging pass, the TMA
+    coordinates of the convolution and its stores), x, out, caches and the staged copy take 19 GB of the device.
+    Sampled outputs - random over the whole range plus the last channel's last frame, whose offsets are the
+    largest - against the oracle; the cache update whole, bit for bit."""
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    import paper_2609_31938_b200 as ccv
+    torch.cuda.set_device(0)
+    N, Cin, Cout, T, H, W, k = 1, 64, 64, 5, 2304, 3072, (3, 3, 3)
+    assert N * Cin * T * H * W > 2 ** 31 and N * Cout * T * H * W > 2 ** 31
+    c = si.conv_case(N, Cin, Cout, T, H, W, k=k, dtype=si.BF16, cache="random", seed=0)
+    layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]))
+    x, cch = to_dev(c["x"]), to_dev(c["cache"])
+    out, nc = layer(x, cch)
+    torch.cuda.synchronize()
+    assert layer.device_status()[0] == ccv.OK and layer.counters()["tcgen05_bf16"] == 1
+    shape = tuple(out.shape)
+    rng = np.random.default_rng(3)
+    tail = np.ravel_multi_index(np.stack(np.meshgrid([0], [Cout - 1], [T - 1], [0, 1, H // 2, H - 2, H - 1],
+                                                     [0, 1, W // 2, W - 9, W - 1], indexing="ij"), -1).reshape(-1, 5).T, shape)
+    idx = np.unique(np.concatenate([rng.integers(0, int(np.prod(shape)), size=4000, dtype=np.int64), tail.astype(np.int64)]))
+    assert idx.max() > 2 ** 31
+    got = out.view(-1)[torch.from_numpy(idx).cuda()].float().cpu().numpy().astype(np.float64)
+    ref = oracle.points(c["x"], c["cache"], c["w"], c["b"], idx)
+    rms = float(np.sqrt(np.mean(ref ** 2)))
+    err = np.abs(got - ref)
+    assert np.isfinite(got).all()
+    assert err.max() <= 2e-2 * rms and err.mean() <= 2e-3 * rms, (err.max() / rms, err.mean() / rms, idx[np.argmax(err)])
+    for t in range(T):                      # nothing left unwritten (frame by frame: no 9 GB temporary)
+        assert bool(torch.isfinite(out[:, :, t]).all())
+    assert np.array_equal(bits(nc), oracle.cache_update(c["x"], c["cache"], k[0])), "cache update is not bit-exact"
+    layer.close()
+    del out, nc, x, cch
+    torch.cuda.empty_cache()
