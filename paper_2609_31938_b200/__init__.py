@@ -25,6 +25,7 @@ FLAG_TWO_KERNELS = 0x10
 FLAG_F32_TENSOR = 0x20
 FLAG_NO_PAIR = 0x40
 FLAG_EPI_SILU = 0x80
+FLAG_NO_TAIL_SPLIT = 0x100
 
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_ALIAS, ERR_ARCH, ERR_NOMEM, ERR_CUDA, \
     ERR_DEVICE_TIMEOUT = range(9)

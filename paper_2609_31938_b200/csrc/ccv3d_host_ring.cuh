@@ -107,8 +107,22 @@ ccv3d_status forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int x_slot, int
     p.tiles_h = (H + 15) / 16;
     p.tiles_w = (W + TWT - 1) / TWT;
     const int64_t total = (int64_t)N * p.tiles_h * p.tiles_w * T * NT;
-    if (total > 0x7FFFFFFF) return CCV3D_ERR_UNSUPPORTED;
+    if (total > 0x3FFFFFFF) return CCV3D_ERR_UNSUPPORTED;
     p.total_tiles = (int)total;
+    // A last wave of tiles that is at most half full runs at half width: twice the items, each half as long, so the
+    // call ends half a wave earlier (192 channels at 88x160: 240 pair tiles on 74 pairs, 4 waves -> 3.5).  CTA pairs with
+    // 64-channel blocks and 3x3 taps only (a kernel variant of its own); the few-waves limit keeps the two-box weight
+    // loads of the full-width tiles (see the kernel) away from long launches, where half a wave is nothing.
+    {
+        const int64_t slots = pair ? h->sm_count / 2 : h->sm_count;
+        const int64_t frac = total % slots;
+        if (pair && !split_n && NB == 1 && pl.KB == 64 && pl.NPAD % 64 == 0 && d.kh == 3 && d.kw == 3 &&
+            d.dtype == CCV3D_BF16 && !(d.flags & CCV3D_FLAG_NO_TAIL_SPLIT) &&
+            total > slots && total / slots <= 12 && frac > 0 && 2 * frac <= slots) {
+            p.main_tiles = (int)(total - frac);
+            p.total_tiles = (int)(total + frac);
+        }
+    }
     p.first_frame = tc - hist;
     p.out_f32 = d.out_dtype == CCV3D_F32;
     p.ACC = ACC;

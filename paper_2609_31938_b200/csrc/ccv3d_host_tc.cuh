@@ -62,10 +62,10 @@ ccv3d_status launch_stage(ccv3d_handle* h, StageParams sp, int h0, int h1, int n
 
 // CTA pairs: clusters of two CTAs, one 16x16-pixel tile per cluster (see the kernel).  tm_w is the 2-D map over the
 // packed weights from which each CTA takes its half of every tap's tile.
-template <int KB, int NB, int KS, int TPBC, bool COOP, bool TF32 = false>
+template <int KB, int NB, int KS, int TPBC, bool COOP, bool TF32 = false, bool TAIL = false>
 ccv3d_status launch_tc_pair(ccv3d_handle* h, const CUtensorMap& tm_a, const CUtensorMap& tm_w, const CUtensorMap& tm_o,
                             const TcParams& p, const StageParams& sp, size_t smem, int grid, cudaStream_t st) {
-    auto kern = conv3d_tcgen05_kernel<KB, NB, KS, TPBC, false, COOP, TF32, true>;
+    auto kern = conv3d_tcgen05_kernel<KB, NB, KS, TPBC, false, COOP, TF32, true, TAIL>;
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess)
         return cuda_fail();
     cudaLaunchConfig_t cfg;
@@ -120,7 +120,8 @@ template <bool COOP>
 ccv3d_status launch_pair_any(ccv3d_handle* h, const CUtensorMap& tm_a, const CUtensorMap& tm_o, const TcParams& p,
                              const StageParams& sp, size_t smem, int grid, int ks, int nb, cudaStream_t st) {
     const CUtensorMap* tm_w = nullptr;
-    ccv3d_status s = weight_map(h, p.NPAD / 2, &tm_w);
+    // (a launch that ends in half-width items carries the weight map of those, see the kernel's B producer)
+    ccv3d_status s = weight_map(h, p.main_tiles > 0 ? p.NPAD / 4 : p.NPAD / 2, &tm_w);
     if (s != CCV3D_OK) return s;
 #define CCV3D_LAUNCH_PAIR(KBv, NBv)                                                                                        \
     do {                                                                                                                   \
@@ -128,6 +129,11 @@ ccv3d_status launch_pair_any(ccv3d_handle* h, const CUtensorMap& tm_a, const CUt
         if (ks == 3) return launch_tc_pair<KBv, NBv, 3, 1, COOP>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);              \
         return launch_tc_pair<KBv, NBv, 1, 1, COOP>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);                           \
     } while (0)
+    if (p.main_tiles > 0) {                 // launches ending in half-width items: 64-channel blocks, one pixel block, 3x3 taps
+        if (COOP || h->d.dtype == CCV3D_F32 || h->plan.KB != 64 || nb != 1 || ks != 3) return CCV3D_ERR_UNSUPPORTED;
+        if (p.TPB == 3) return launch_tc_pair<64, 1, 3, 3, false, false, true>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
+        return launch_tc_pair<64, 1, 3, 1, false, false, true>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
+    }
     if (h->d.dtype == CCV3D_F32) {          // 3xTF32 (plain schedule only)
         if (COOP) return CCV3D_ERR_UNSUPPORTED;
         if (nb == 2) {

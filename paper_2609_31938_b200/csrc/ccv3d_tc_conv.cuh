@@ -18,6 +18,8 @@ struct TcParams {
     int CB;           // input-channel blocks of KB
     int NT, NPAD;     // output-channel tiles and their (padded) width, NPAD % 16 == 0, <= 256
     int tiles_h, tiles_w, total_tiles;   // tile rows handled by this launch, tile columns, tiles of this launch
+    int main_tiles;           // > 0: work items main_tiles .. total_tiles-1 are the launch's last tiles at HALF width (the
+                              // last wave would be at most half full: twice the items, each half as long); see TileView
     int ty_begin;                        // first tile row of this launch (a launch may cover a band of the image)
     int first_frame;  // Z frames below this are absent (first chunk): their taps are skipped
     int out_f32;      // 1: out is FP32, 0: BF16
@@ -74,6 +76,26 @@ struct TcShared {  // placed after the rings
     volatile int abort_flag;
     alignas(16) float bias_s[TC_BIAS_SMEM];   // the layer's padded bias when it fits (the epilogue reads it once per element)
 };
+
+// Work item u of a launch as a tile.  Items below main_tiles (all of them when main_tiles == 0) are tiles of the
+// launch's own output-channel width; the others enumerate the remaining tiles at half that width (the mechanism of
+// split_n, per tile): full-width tile f = halves 2f and 2f+1, so item u >= main_tiles is half-width tile u + main_tiles.
+struct TileView {
+    int tile, NT, NPAD, split;
+    uint32_t b_tap;       // bytes of one tap of this CTA's weight tile
+    bool half;
+};
+template <bool TAIL>      // TAIL = false: kernels that never see half-width items (everything folds to the launch's values)
+__device__ __forceinline__ TileView tile_view(const TcParams& p, int u) {
+    TileView v;
+    v.half = TAIL && p.main_tiles > 0 && u >= p.main_tiles;
+    v.tile = v.half ? u + p.main_tiles : u;
+    v.NT = v.half ? 2 * p.NT : p.NT;
+    v.NPAD = v.half ? p.NPAD >> 1 : p.NPAD;
+    v.split = v.half ? 1 : p.split_n;
+    v.b_tap = v.half ? p.b_tap >> 1 : p.b_tap;
+    return v;
+}
 
 // Bounded wait.  Returns false when the limit expired or another role of this CTA aborted.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, TcShared* sh, const TcParams& p, uint32_t site) {
@@ -170,7 +192,7 @@ __device__ __forceinline__ uint32_t epi_pair(float a0, float a1, uint32_t res_pa
 // shared-memory read port.  Loads of both CTAs are counted on the leader's "full" barriers; the leader's commits
 // arrive on the "empty" and "accumulator full" barriers of both CTAs; both epilogues arrive on the leader's
 // "accumulator empty" barrier.
-template <int KB, int NB, int KS, int TPBC, bool FUSED, bool COOP, bool TF32 = false, bool PAIR = false>
+template <int KB, int NB, int KS, int TPBC, bool FUSED, bool COOP, bool TF32 = false, bool PAIR = false, bool TAIL = false>
 __global__ void __launch_bounds__((FUSED || COOP) ? TC_THREADS_FUSED : TC_THREADS, 1)
 conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged activations (c, w, h, cb, n*F+f), or x
                       const __grid_constant__ CUtensorMap tm_c,   // fused mode: the cache; PAIR: the packed weights
@@ -289,8 +311,9 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
             uint32_t phase = 1;
             bool ok = true;
             int bands_ready = 0;                       // COOP: bands [0, bands_ready) are known to be staged
-            for (int tile = cta_lin; ok && tile < p.total_tiles; tile += cta_cnt) {
-                int r = tile / p.NT;
+            for (int item = cta_lin; ok && item < p.total_tiles; item += cta_cnt) {
+                const TileView tv = tile_view<TAIL>(p, item);
+                int r = tv.tile / tv.NT;
                 const int t = r % p.T; r /= p.T;
                 const int tx = r % p.tiles_w; r /= p.tiles_w;
                 const int ty = p.ty_begin + r % p.tiles_h;
@@ -350,15 +373,17 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     // ---------------------------------------------------------------- B producer
     else if (warp == 1) {
         if (lane == 0) {
-            const uint32_t b_bytes = p.b_tap * p.TPB;
-            const uint32_t src_tap = p.b_src_tap ? p.b_src_tap : p.b_tap;   // bytes between taps in the packed weights
             int s = 0;
             uint32_t phase = 1;
             bool ok = true;
             if (PAIR) asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_c) : "memory");
-            for (int tile = cta_lin; ok && tile < p.total_tiles; tile += cta_cnt) {
-                const int nt = tile % p.NT;
-                const int t = (tile / p.NT) % p.T;
+            for (int item = cta_lin; ok && item < p.total_tiles; item += cta_cnt) {
+                const TileView tv = tile_view<TAIL>(p, item);
+                const int nt = tv.tile % tv.NT;
+                const int t = (tv.tile / tv.NT) % p.T;
+                const uint32_t b_bytes = tv.b_tap * p.TPB;
+                // bytes between taps in the packed weights (half-width tiles: those of the full-width tile)
+                const uint32_t src_tap = tv.half ? p.b_tap : (p.b_src_tap ? p.b_src_tap : p.b_tap);
                 const int dt0 = (p.first_frame - t * stt > 0) ? (p.first_frame - t * stt + dlt - 1) / dlt : 0;   // first tap whose frame exists
                 for (int pass = 0; pass < (TF32 ? 3 : 1); ++pass)
                 for (int dt = dt0; ok && dt < p.kt; ++dt)
@@ -368,15 +393,21 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                             // over the packed weights; both CTAs' boxes are counted on the leader's barrier
                             // (split_n: NT and NPAD describe half-width tiles of a layer packed at full width; the rows of
                             // a tap's full-width tile are then [half 0 | half 1], each again split between the two CTAs)
-                            const int npw = p.NPAD << p.split_n;                      // rows of a packed (full-width) tile
-                            const int row0 = ((((pass * p.kt + dt) * p.CB + cb) * (p.NT >> p.split_n) + (nt >> p.split_n)) * spatial) * npw +
-                                             (nt & p.split_n) * p.NPAD + (int)rank * (p.NPAD >> 1);
+                            const int npw = tv.NPAD << tv.split;                      // rows of a packed (full-width) tile
+                            const int row0 = ((((pass * p.kt + dt) * p.CB + cb) * (tv.NT >> tv.split) + (nt >> tv.split)) * spatial) * npw +
+                                             (nt & tv.split) * tv.NPAD + (int)rank * (tv.NPAD >> 1);
                             for (int tp = 0; tp < spatial; tp += p.TPB) {
                                 if (!(ok = mbar_wait(&sh->empty_b[s], phase, sh, p, SITE_B_EMPTY))) break;
                                 const uint32_t bar = smem_u32(&sh->full_b[s]);
                                 if (rank == 0) mbar_expect_tx(bar, 2 * b_bytes);
                                 const uint32_t dst = smem_u32(ring_b + (size_t)s * p.b_slot);
-                                for (int u = 0; u < p.TPB; ++u) tma_load_2d_pair(dst + u * p.b_tap, &tm_c, bar, 0, row0 + (tp + u) * npw);
+                                // (a launch with half-width items carries the weight map of those: its box is a quarter of
+                                // a full tile's rows, and a CTA's half of a full-width tile arrives as two boxes)
+                                const int parts = (TAIL && p.main_tiles > 0 && !tv.half) ? 2 : 1;
+                                for (int u = 0; u < p.TPB; ++u)
+                                    for (int q = 0; q < parts; ++q)
+                                        tma_load_2d_pair(dst + u * tv.b_tap + q * (tv.b_tap >> 1), &tm_c, bar, 0,
+                                                         row0 + (tp + u) * npw + q * (tv.NPAD >> 2));
                                 if (++s == p.SB) { s = 0; phase ^= 1; }
                             }
                             continue;
@@ -384,16 +415,16 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                         // split_n: this launch runs half-width output-channel tiles; the packed image of a full tile
                         // holds its two halves back to back (the swizzle repeats every 8 rows), so a half tile of a
                         // tap is a contiguous piece of it and only the distance between taps differs
-                        const uint8_t* src = p.wq + (size_t)(((pass * p.kt + dt) * p.CB + cb) * (p.NT >> p.split_n) + (nt >> p.split_n)) * spatial * src_tap +
-                                             (size_t)(nt & p.split_n) * p.b_tap;
+                        const uint8_t* src = p.wq + (size_t)(((pass * p.kt + dt) * p.CB + cb) * (tv.NT >> tv.split) + (nt >> tv.split)) * spatial * src_tap +
+                                             (size_t)(nt & tv.split) * tv.b_tap;
                         for (int tp = 0; tp < spatial; tp += p.TPB) {
                             if (!(ok = mbar_wait(&sh->empty_b[s], phase, sh, p, SITE_B_EMPTY))) break;
                             const uint32_t bar = smem_u32(&sh->full_b[s]);
                             mbar_expect_tx(bar, b_bytes);
                             const uint32_t dst = smem_u32(ring_b + (size_t)s * p.b_slot);
-                            if (src_tap == p.b_tap) bulk_load(dst, src + (size_t)tp * src_tap, b_bytes, bar);
+                            if (src_tap == tv.b_tap) bulk_load(dst, src + (size_t)tp * src_tap, b_bytes, bar);
                             else
-                                for (int u = 0; u < p.TPB; ++u) bulk_load(dst + u * p.b_tap, src + (size_t)(tp + u) * src_tap, p.b_tap, bar);
+                                for (int u = 0; u < p.TPB; ++u) bulk_load(dst + u * tv.b_tap, src + (size_t)(tp + u) * src_tap, tv.b_tap, bar);
                             if (++s == p.SB) { s = 0; phase ^= 1; }
                         }
                     }
@@ -411,7 +442,9 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
         // instruction descriptor: D=F32, A=B=BF16, both K-major, N = NPAD, M = 128
         // (operand formats: 1 = BF16, 2 = TF32)
         constexpr uint32_t FMT = TF32 ? 2u : 1u;
-        const uint32_t idesc = (1u << 4) | (FMT << 7) | (FMT << 10) | ((uint32_t)(p.NPAD >> 3) << 17) | (((PAIR ? 256u : 128u) >> 4) << 24);
+        const uint32_t idesc_full = (1u << 4) | (FMT << 7) | (FMT << 10) | ((uint32_t)(p.NPAD >> 3) << 17) | (((PAIR ? 256u : 128u) >> 4) << 24);
+        const uint32_t idesc_half = (1u << 4) | (FMT << 7) | (FMT << 10) | ((uint32_t)(p.NPAD >> 4) << 17) | (((PAIR ? 256u : 128u) >> 4) << 24);
+        const uint32_t idesc = idesc_full;                // (the run-time tap loop below never sees half-width items)
         const uint32_t a_hi = make_desc_hi((uint32_t)BW * ROWB, LAYOUT);  // 8-pixel groups are one image row apart
         const uint32_t b_hi = make_desc_hi(B_SBO, LAYOUT);
         const uint32_t a_blk = (uint32_t)(iss * NBW) * ((8 * ROWB) >> 4);  // descriptor offset of this issuer's first block
@@ -426,8 +459,13 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
             uint32_t a_ring = make_desc_lo(smem_u32(ring_a)) + a_blk, b_ring = make_desc_lo(smem_u32(ring_b));
             const uint32_t a_slotstep = p.a_slot >> 4, b_slotstep = p.b_slot >> 4;
             const uint32_t a_ring0 = a_ring, b_ring0 = b_ring;
-            for (int tile = cta_lin; ok && tile < p.total_tiles; tile += cta_cnt) {
-                const int t = (tile / p.NT) % p.T;
+            for (int item = cta_lin; ok && item < p.total_tiles; item += cta_cnt) {
+                const TileView tv = tile_view<TAIL>(p, item);
+                const int t = (tv.tile / tv.NT) % p.T;
+                // N of the instruction and the tap distance in a weight slot follow the tile's width; the accumulators
+                // keep the launch's column layout
+                const uint32_t idesc = tv.half ? idesc_half : idesc_full;
+                const uint32_t b_tapstep = tv.b_tap >> 4;
                 const int dt0 = (p.first_frame - t * stt > 0) ? (p.first_frame - t * stt + dlt - 1) / dlt : 0;   // first tap whose frame exists
                 if (!(ok = mbar_wait(&sh->acc_empty[acc], pacc, sh, p, SITE_ACC_EMPTY))) break;
                 tc_fence_after();
@@ -583,9 +621,10 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
         // the tile loop exists twice, with and without the optional SiLU, so that the plain epilogue carries no trace of it
         auto run_tiles = [&](auto act_c) {
             constexpr bool ACT = decltype(act_c)::value;
-            for (int tile = cta_lin; ok && tile < p.total_tiles; tile += cta_cnt) {
-                const int nt = tile % p.NT;
-                int r = tile / p.NT;
+            for (int item = cta_lin; ok && item < p.total_tiles; item += cta_cnt) {
+                const TileView tv = tile_view<TAIL>(p, item);
+                const int nt = tv.tile % tv.NT;
+                int r = tv.tile / tv.NT;
                 const int t = r % p.T; r /= p.T;
                 const int tx = r % p.tiles_w; r /= p.tiles_w;
                 const int ty = p.ty_begin + r % p.tiles_h;
@@ -602,7 +641,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                 // the residual of the first chunk is fetched while the MMAs of this tile still run; every later chunk's
                 // residual is fetched one chunk ahead
                 uint32_t rr_next[16];
-                if (p.epi_tma) load_res32(res_row, wt + (m & 7) < p.W, wt + (m & 7), nt * p.NPAD, p, HW, rr_next);
+                if (p.epi_tma) load_res32(res_row, wt + (m & 7) < p.W, wt + (m & 7), nt * tv.NPAD, p, HW, rr_next);
                 ok = mbar_wait(&sh->acc_full[acc], pacc, sh, p, SITE_ACC_FULL);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
@@ -614,11 +653,11 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                 if (p.epi_tma) {
                     // BF16 tile chunks -> shared memory -> one TMA store per chunk.  NCTHW output: [ECH channels][16 rows]
                     // [TW pixels]; ring output: [16 rows][TW pixels][32 channels] with the 64-byte swizzle of the tensor map.
-                    for (int c0 = 0; c0 < p.NPAD; c0 += p.ECH) {
+                    for (int c0 = 0; c0 < tv.NPAD; c0 += p.ECH) {
                         if (elected) bulk_wait_read<1>();   // the store that last read this buffer has finished reading
                         epi_bar_sync();
                         uint8_t* stg = epi_buf + (size_t)ebuf * p.e_slot;
-                        const int co0 = nt * p.NPAD + c0;
+                        const int co0 = nt * tv.NPAD + c0;
     #pragma unroll
                         for (int blk = 0; blk < NB; ++blk) {
                             uint32_t rr[16];
@@ -627,7 +666,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                             if (has_res) {
                                 const int wn = wt + ((blk + 1 < NB) ? blk + 1 : 0) * 8 + (m & 7);
                                 const int con = (blk + 1 < NB) ? co0 : co0 + p.ECH;
-                                load_res32(res_row, wn < p.W && con < (nt + 1) * p.NPAD, wn, con, p, HW, rr_next);
+                                load_res32(res_row, wn < p.W && con < (nt + 1) * tv.NPAD, wn, con, p, HW, rr_next);
                             }
                             uint32_t v[32];
                             if (p.ECH == 32) tc_ld32(t_acc + blk * p.NPAD + c0, v); else tc_ld16(t_acc + blk * p.NPAD + c0, v);
@@ -696,12 +735,12 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                         const bool valid = h < p.H && w < p.W;
                         const int64_t pix = (int64_t)t * HW + (int64_t)h * p.W + w;
     #pragma unroll 1
-                        for (int c0 = 0; c0 < p.NPAD; c0 += 32) {
-                            const int co0 = nt * p.NPAD + c0;
+                        for (int c0 = 0; c0 < tv.NPAD; c0 += 32) {
+                            const int co0 = nt * tv.NPAD + c0;
                             uint32_t rr[16];
                             load_res32(res_row, valid, w, co0, p, HW, rr);
                             uint32_t v[32];
-                            const int nc = (p.NPAD - c0 >= 32) ? 32 : 16;
+                            const int nc = (tv.NPAD - c0 >= 32) ? 32 : 16;
                             if (nc == 32) tc_ld32(t_acc + blk * p.NPAD + c0, v); else tc_ld16(t_acc + blk * p.NPAD + c0, v);
                             tc_wait_ld();
                             if (two_acc) {

@@ -202,6 +202,39 @@ def test_cta_pairs_on_rings(ccv):
     check(as_f64(got[0][1]), ref, "bf16")
 
 
+@pytest.mark.parametrize("Cin,Cout,T,H,W", [
+    (192, 192, 4, 88, 160),     # 240 pair tiles on 74 pairs: three whole waves, then 18 tiles as 36 half-width items
+    (64, 384, 2, 64, 96),       # two co-tiles per pixel tile: 96 items, 74 + 22 -> 74 full-width and 44 half-width
+    (128, 128, 3, 60, 100),     # 84 items: 74 + 10 -> 20 half-width; ragged tile rows and columns
+])
+def test_half_width_tail_on_rings(ccv, Cin, Cout, T, H, W):
+    """A call whose last wave of tiles would be at most half full finishes with half-width output-channel tiles in
+    the same launch.  Ring output with the residual epilogue (where channel counts allow), NCTHW output and the
+    upsampling store: bit for bit what the launch without the tail writes, and within tolerance of the oracle."""
+    c = si.conv_case(1, Cin, Cout, T, H, W, seed=31)
+    x, cache = to_dev(c["x"]), to_dev(c["cache"])
+    got = {}
+    for flags in (0, ccv.FLAG_NO_TAIL_SPLIT):
+        layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), flags=flags)
+        rin = ccv.FrameRing(1, Cin, T + 2, H, W)
+        rin.load(0, cache)
+        rin.load(2, x)
+        r1, r2 = ccv.FrameRing(1, Cout, T, H, W, zero=True), ccv.FrameRing(1, Cout, T, 2 * H, 2 * W, zero=True)
+        out = torch.zeros((1, Cout, T, H, W), dtype=torch.bfloat16, device="cuda")
+        res = rin if Cin == Cout else None
+        layer.forward_ring(rin, 2, 2, T, out_ring=r1, res=res, res_slot=2)
+        layer.forward_ring(rin, 2, 2, T, out=out)
+        layer.forward_ring(rin, 2, 2, T, out_ring=r2, up_rt=1)
+        torch.cuda.synchronize()
+        assert layer.device_status()[0] == ccv.OK
+        got[flags] = (r1.buf.clone(), out.clone(), r2.buf.clone())
+        layer.close()
+    for a, b in zip(got[0], got[ccv.FLAG_NO_TAIL_SPLIT]):
+        assert torch.equal(a, b)
+    ref, _ = oracle.forward(c["x"], c["cache"], c["w"], c["b"])
+    check(as_f64(got[0][1]), ref, "bf16")
+
+
 def test_ring_argument_errors(ccv):
     c = si.conv_case(1, 64, 64, 2, 16, 16, seed=23)
     layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]))
