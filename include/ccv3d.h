@@ -65,8 +65,8 @@ typedef enum {
                                             channels per tile and 3x3 or 1x1 spatial kernels */
 #define CCV3D_FLAG_EPI_SILU 0x80u         /* epilogue activation (not part of the paper's operator): out = silu(conv + b), v / (1 + exp(-v)) in
                                             FP32 before the one output rounding; a residual (frame rings) is added after it */
-#define CCV3D_FLAG_NO_TAIL_SPLIT 0x100u   /* frame rings: never finish a call with a second launch of half-width output-channel
-                                            tiles (the default when the last wave of tiles would be at most half full) */
+#define CCV3D_FLAG_NO_TAIL_SPLIT 0x100u   /* never finish a launch with half-width output-channel tiles (the default on CTA pairs
+                                            when the last wave of tiles would be at most half full) */
 #define CCV3D_FLAG_TC_PER_TAP_A 0x2u    /* tensor-core kernel: fetch the activation tile once per tap (no halo reuse in shared memory) */
 
 /* Layer description, fixed at create time (Algorithm 1's Require line: W, b, p, s, d, g).

@@ -380,8 +380,15 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
             p.ty_begin = 0;
             p.tiles_h = tiles_h;
             const int64_t total = (int64_t)N * tiles_h * p.tiles_w * To * NT;
-            if (total > 0x7FFFFFFF) return CCV3D_ERR_UNSUPPORTED;
+            if (total > 0x3FFFFFFF) return CCV3D_ERR_UNSUPPORTED;
             p.total_tiles = (int)total;
+            // a last wave that is at most half full runs at half width (see forward_ring)
+            const int64_t slots = h->sm_count / 2, frac = total % slots;
+            if (!split_n && NB == 1 && pl.KB == 64 && pl.NPAD % 64 == 0 && ks == 3 && !f32 &&
+                !(d.flags & CCV3D_FLAG_NO_TAIL_SPLIT) && total > slots && total / slots <= 12 && frac > 0 && 2 * frac <= slots) {
+                p.main_tiles = (int)(total - frac);
+                p.total_tiles = (int)(total + frac);
+            }
             const int grid = 2 * (p.total_tiles < h->sm_count / 2 ? p.total_tiles : h->sm_count / 2);
             StageParams nosp;
             memset(&nosp, 0, sizeof(nosp));

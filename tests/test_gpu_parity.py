@@ -498,3 +498,23 @@ def test_random_shapes_every_schedule_agrees(ccv):
             assert torch.equal(o, res[2][0]), (Cin, Cout, k, T, H, W, cf)
             assert nc is None or torch.equal(nc, res[2][1]), (Cin, Cout, k, T, H, W, cf)
         done += 1
+
+
+@pytest.mark.parametrize("Cin,Cout,T,H,W", [(128, 128, 3, 60, 100), (64, 384, 2, 64, 96)])
+def test_half_width_tail_through_ncthw(ccv, Cin, Cout, T, H, W):
+    """Mid-size layers on CTA pairs whose last wave of tiles is at most half full (84 = 74 + 10 and 96 = 74 + 22 items)
+    end the launch with half-width tiles: same bits as without (CCV3D_FLAG_NO_TAIL_SPLIT), within tolerance of the
+    oracle, cache bit-exact."""
+    c = si.conv_case(1, Cin, Cout, T, H, W, seed=41)
+    ref, ref_nc = oracle.forward(c["x"], c["cache"], c["w"], c["b"])
+    outs = []
+    for flags in (0, ccv.FLAG_NO_TAIL_SPLIT):
+        layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), flags=flags)
+        o, nc = layer(to_dev(c["x"]), to_dev(c["cache"]))
+        torch.cuda.synchronize()
+        assert layer.device_status()[0] == ccv.OK
+        assert np.array_equal(bits(nc), ref_nc)
+        outs.append(o)
+        layer.close()
+    assert torch.equal(outs[0], outs[1])
+    check(as_f64(outs[0]), ref, "bf16")
