@@ -216,6 +216,19 @@ ccv3d_status ccv3d_forward_static(ccv3d_handle* h, const void* x, const void* ca
 ccv3d_status ccv3d_forward_host(ccv3d_handle* h, const void* x_host, const void* cache_host, void* out_host,
                                 void* new_cache_host, int32_t N, int32_t T, int32_t H, int32_t W, void* stream);
 
+/*
+ * Streaming form of ccv3d_forward_host: the temporal history (the cache of Eq. (1)'s Z = [C ; X]) stays on the
+ * device between calls, in a frame ring the handle owns, so a call moves only x (HOST [N,cin,T,H,W]) up and out
+ * (HOST [N,cout,T,H,W]) down - the cache never crosses the bus.  reset != 0 starts a new stream (first chunk: no
+ * history); a change of N, H or W, or any other host entry point used on the handle in between, starts a new
+ * stream as well.  Same frame-by-frame pipeline, same results bit for bit as ccv3d_forward_host with the cache
+ * carried by the caller.  Synchronous like ccv3d_forward_host.  Layers and sizes the pipelined path does not take
+ * (see ccv3d_forward_host: standard geometry, BF16, cin a multiple of the channel block, a few MB per frame)
+ * return CCV3D_ERR_UNSUPPORTED; any T >= 1.
+ */
+ccv3d_status ccv3d_forward_host_stream(ccv3d_handle* h, const void* x_host, void* out_host, int32_t reset, int32_t N,
+                                       int32_t T, int32_t H, int32_t W, void* stream);
+
 /* Bytes of handle-owned workspace a forward call of this shape needs (0 for the FP32-FMA route, the 1x1x1
  * streaming kernel and the fused route). */
 ccv3d_status ccv3d_workspace_bytes(const ccv3d_handle* h, int32_t N, int32_t T, int32_t H, int32_t W,

@@ -54,7 +54,8 @@ EXPORTS = ("ccv3d_create", "ccv3d_forward", "ccv3d_forward_host", "ccv3d_workspa
            "ccv3d_get_counters", "ccv3d_device_status", "ccv3d_status_string", "ccv3d_add_bf16",
            "ccv3d_upsample_bf16", "ccv3d_profile_enable", "ccv3d_profile_read", "ccv3d_forward_static", "ccv3d_selftest_wait_timeout", "ccv3d_forward_ex",
            "ccv3d_ring_kb", "ccv3d_ring_bytes", "ccv3d_ring_load", "ccv3d_ring_store", "ccv3d_upsample_ring",
-           "ccv3d_forward_ring", "ccv3d_out_dims", "ccv3d_forward_ring_up", "ccv3d_rows_copy")
+           "ccv3d_forward_ring", "ccv3d_out_dims", "ccv3d_forward_ring_up", "ccv3d_rows_copy",
+           "ccv3d_forward_host_stream")
 
 
 def _load() -> ctypes.CDLL:
@@ -69,6 +70,7 @@ def _load() -> ctypes.CDLL:
     lib.ccv3d_forward_ex.argtypes = [vp, vp, vp, i32, vp, vp, i32, i32, i32, i32, vp]
     lib.ccv3d_forward_static.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, vp]
     lib.ccv3d_forward_host.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, vp]
+    lib.ccv3d_forward_host_stream.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp]
     lib.ccv3d_workspace_bytes.argtypes = [vp, i32, i32, i32, i32, u64p]
     lib.ccv3d_destroy.argtypes = [vp]
     lib.ccv3d_get_counters.argtypes = [vp, ctypes.POINTER(Counters)]
@@ -151,6 +153,11 @@ def ccv3d_forward_static(h, x, cache, out, new_cache, N, T, H, W, stream=0) -> i
 
 def ccv3d_forward_host(h, x, cache, out, new_cache, N, T, H, W, stream=0) -> int:
     return lib.ccv3d_forward_host(h, x, cache, out, new_cache, N, T, H, W, stream)
+
+
+def ccv3d_forward_host_stream(h, x, out, reset, N, T, H, W, stream=0) -> int:
+    """x/out are HOST pointers; the history stays on the device between calls."""
+    return lib.ccv3d_forward_host_stream(h, x, out, 1 if reset else 0, N, T, H, W, stream)
 
 
 def ccv3d_out_dims(h, T, H, W):

@@ -81,6 +81,9 @@ struct ccv3d_handle {
     cudaEvent_t* prof_ev;   // PROF_SLOTS x 3 events, created on first enable
     int pdl;             // 1: convolution kernels on frame rings are launched with programmatic stream serialization
     int coop_launch;     // 1: cooperative-staging kernels are launched with the cooperative attribute
+    bool hs_valid;       // host stream (ccv3d_forward_host_stream): the device ring holds the history of hs_geom
+    int hs_state[2];     //   ring slot of the next frame, history frames present
+    int hs_geom[3];      //   N, H, W of the stream
     int cluster_ok;      // the device launches thread-block clusters (needed for CTA pairs)
     int call_cf;         // history frames held by the cache of the call being served (set by the entry points)
     ccv3d_counters ctr;
@@ -410,8 +413,11 @@ ccv3d_status ccv3d_forward_static(ccv3d_handle* h, const void* x, const void* ca
 // the output frame goes back with another strided 2-D copy on a download stream.  Three buffers of each kind rotate,
 // so that upload, compute and download of different frames overlap: the call takes about as long as the slower of
 // the two PCIe directions instead of their sum.
+// stream_state != nullptr: streaming form - {ring slot of the next frame, frames seen so far} carried in the handle from
+// call to call; the history is whatever the previous call left in the ring (cache_host and new_cache_host are null).
 static ccv3d_status forward_host_pipelined(ccv3d_handle* h, const void* x_host, const void* cache_host, void* out_host,
-                                    void* new_cache_host, int N, int T, int H, int W, cudaStream_t st) {
+                                    void* new_cache_host, int N, int T, int H, int W, cudaStream_t st,
+                                    int* stream_state = nullptr) {
     const ccv3d_desc& d = h->d;
     const int tc = hist_len(d);
     constexpr int NBUF = 3;
@@ -435,11 +441,13 @@ static ccv3d_status forward_host_pipelined(ccv3d_handle* h, const void* x_host, 
     if (cudaEventRecord(h->ev_fork, st) != cudaSuccess) return cuda_fail();
     if (cudaStreamWaitEvent(s_up, h->ev_fork, 0) != cudaSuccess || cudaStreamWaitEvent(s_down, h->ev_fork, 0) != cudaSuccess)
         return cuda_fail();
-    if (!cache_host && tc && cudaMemsetAsync(ring.base, 0, (size_t)ring.F * xf, st) != cudaSuccess) return cuda_fail();
+    if (!stream_state && !cache_host && tc && cudaMemsetAsync(ring.base, 0, (size_t)ring.F * xf, st) != cudaSuccess)
+        return cuda_fail();
 
     const int pre = (cache_host && tc) ? tc : 0;           // history frames uploaded before the first frame of x
     const bool nc_early = tc && new_cache_host && tc < NBUF && pre + T >= tc;
     int slot = 0, seen = 0;                                // ring slot of the next frame; frames in the ring so far
+    if (stream_state) { slot = stream_state[0]; seen = stream_state[1]; }
     for (int i = 0; i < pre + T; ++i) {
         const int b = i % NBUF;
         const bool is_x = i >= pre;
@@ -494,6 +502,7 @@ static ccv3d_status forward_host_pipelined(ccv3d_handle* h, const void* x_host, 
         return cuda_fail();
     if (cudaEventRecord(h->ev_join[1], s_up) != cudaSuccess || cudaStreamWaitEvent(st, h->ev_join[1], 0) != cudaSuccess)
         return cuda_fail();
+    if (stream_state) { stream_state[0] = slot; stream_state[1] = seen < tc ? seen : tc; }
     h->ctr.tcgen05_bf16++;
     return CCV3D_OK;
 }
@@ -514,6 +523,7 @@ ccv3d_status ccv3d_forward_host(ccv3d_handle* h, const void* x_host, const void*
         h->ctr.calls++;
         return count(h, s);
     }
+    h->hs_valid = false;                                   // this call reuses the device buffers of a host stream
     if (host_pipeline_eligible(h, T, H, W)) {
         h->ctr.calls++;
         if (!on_handle_device(h)) return count(h, CCV3D_ERR_INVALID_ARG);
@@ -542,6 +552,28 @@ ccv3d_status ccv3d_forward_host(ccv3d_handle* h, const void* x_host, const void*
     if (has_n && cudaMemcpyAsync(new_cache_host, h->hn, cb, cudaMemcpyDeviceToHost, st) != cudaSuccess) return cuda_fail();
     if (cudaStreamSynchronize(st) != cudaSuccess) return cuda_fail();
     return ccv3d_device_status(h, nullptr);
+}
+
+ccv3d_status ccv3d_forward_host_stream(ccv3d_handle* h, const void* x_host, void* out_host, int32_t reset, int32_t N,
+                                       int32_t T, int32_t H, int32_t W, void* stream) {
+    if (!h) return CCV3D_ERR_INVALID_ARG;
+    h->ctr.calls++;
+    h->call_cf = 0;
+    ccv3d_status s = check_forward_args(h, x_host, nullptr, out_host, nullptr, N, T, H, W, false);
+    if (s != CCV3D_OK) return count(h, s);
+    if (!host_pipeline_eligible(h, 2, H, W)) return count(h, CCV3D_ERR_UNSUPPORTED);
+    if (!on_handle_device(h)) return count(h, CCV3D_ERR_INVALID_ARG);
+    if (reset || !h->hs_valid || h->hs_geom[0] != N || h->hs_geom[1] != H || h->hs_geom[2] != W) {
+        h->hs_state[0] = h->hs_state[1] = 0;               // first chunk: no history (its taps are skipped, nothing is zeroed)
+        h->hs_geom[0] = N; h->hs_geom[1] = H; h->hs_geom[2] = W;
+    }
+    h->hs_valid = false;                                   // stays false if anything below fails
+    s = forward_host_pipelined(h, x_host, nullptr, out_host, nullptr, N, T, H, W, (cudaStream_t)stream, h->hs_state);
+    if (s != CCV3D_OK) return count(h, s);
+    if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return count(h, cuda_fail());
+    s = ccv3d_device_status(h, nullptr);
+    h->hs_valid = (s == CCV3D_OK);
+    return count(h, s);
 }
 
 ccv3d_status ccv3d_profile_enable(ccv3d_handle* h, int32_t enable) {

@@ -81,6 +81,9 @@ def test_null_and_misaligned_arguments():
     assert ccv.ccv3d_destroy(None) == ccv.OK
     assert ccv.ccv3d_forward(None, 4096, None, 8192, None, 1, 1, 8, 8) == ccv.ERR_INVALID_ARG
     assert ccv.ccv3d_forward_host(None, 4096, None, 8192, None, 1, 1, 8, 8) == ccv.ERR_INVALID_ARG
+    assert ccv.ccv3d_forward_host_stream(None, 4096, 8192, 1, 1, 1, 8, 8) == ccv.ERR_INVALID_ARG
+    assert ccv.ccv3d_rows_copy(None, 4, 0, 4096, 4, 0, 1, 1, 16) == ccv.ERR_INVALID_ARG          # no destination
+    assert ccv.ccv3d_rows_copy(4096, 4, 3, 8192, 4, 0, 1, 2, 16) == ccv.ERR_INVALID_ARG          # rows leave the plane
     assert ccv.ccv3d_workspace_bytes(None, 1, 1, 8, 8)[0] == ccv.ERR_INVALID_ARG
     assert ccv.ccv3d_device_status(None)[0] == ccv.ERR_INVALID_ARG
     assert ccv.ccv3d_add_bf16(None, None, None, 16) == ccv.ERR_INVALID_ARG

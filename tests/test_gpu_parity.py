@@ -393,6 +393,49 @@ def test_pipelined_host_entry_point(ccv, N, Cin, Cout, T, H, W, cache):
     layer.close()
 
 
+def test_host_stream_keeps_the_history_on_the_device(ccv):
+    """ccv3d_forward_host_stream: chunks of 3, 1, 1 and 4 frames with nothing but x going up and out coming down give
+    the bits of the whole-sequence causal run (and so of ccv3d_forward_host with the cache carried by the caller);
+    reset starts over; another host call on the handle in between ends the stream; small frames are refused."""
+    N, Cin, Cout, H, W = 1, 64, 96, 128, 160
+    lens = [3, 1, 1, 4]
+    c = si.conv_case(N, Cin, Cout, sum(lens), H, W, cache=None, seed=14)
+    layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]))
+    whole, _ = layer(to_dev(c["x"]), None)
+    whole = bits(whole)
+    st = torch.cuda.current_stream().cuda_stream
+
+    def run(t0, T, reset):
+        xc = np.ascontiguousarray(c["x"][:, :, t0:t0 + T])
+        out = np.full((N, Cout, T, H, W), 0x7FC0, np.uint16)
+        assert ccv.ccv3d_forward_host_stream(layer.h, xc.ctypes.data, out.ctypes.data, reset, N, T, H, W, st) == ccv.OK
+        return out
+
+    t0 = 0
+    for i, T in enumerate(lens):
+        assert np.array_equal(run(t0, T, i == 0), whole[:, :, t0:t0 + T]), f"chunk {i}"
+        t0 += T
+    # reset: the same first chunk again gives the first frames again (no history)
+    assert np.array_equal(run(0, 3, True), whole[:, :, 0:3])
+    assert np.array_equal(run(3, 2, False), whole[:, :, 3:5])
+    # a non-streaming host call reuses the device buffers: the next stream call starts from no history
+    nc = np.empty((N, Cin, 2, H, W), np.uint16)
+    o5 = np.empty((N, Cout, 2, H, W), np.uint16)
+    x5 = np.ascontiguousarray(c["x"][:, :, 5:7])
+    assert ccv.ccv3d_forward_host(layer.h, x5.ctypes.data, None, o5.ctypes.data, nc.ctypes.data, N, 2, H, W, st) == ccv.OK
+    first = run(0, 3, False)
+    assert np.array_equal(first, whole[:, :, 0:3])
+    ref, _ = oracle.forward(c["x"][:, :, :3], None, c["w"], c["b"])
+    check(si.to_f64(first), ref, "bf16")
+    assert layer.device_status()[0] == ccv.OK
+    layer.close()
+    small = si.conv_case(1, 64, 64, 2, 16, 16, cache=None, seed=15)
+    l2 = ccv.CausalConv3d(to_dev(small["w"]), to_dev(small["b"]))
+    o = np.empty((1, 64, 2, 16, 16), np.uint16)
+    assert ccv.ccv3d_forward_host_stream(l2.h, small["x"].ctypes.data, o.ctypes.data, 1, 1, 2, 16, 16, st) == ccv.ERR_UNSUPPORTED
+    l2.close()
+
+
 @pytest.mark.parametrize("shape,rt", [((2, 3, 2, 5, 6), 3), ((1, 4, 3, 6, 8), 4), ((1, 2, 2, 4, 12), 1)])
 def test_chain_glue_kernels(ccv, shape, rt):
     """Residual add (exact sum, one RNE rounding) and nearest-neighbour upsampling (exact copies), scalar and
