@@ -123,7 +123,8 @@ typedef struct {
  *   stream  a cudaStream_t (NULL = default stream).
  * The handle owns: packed weights, FP32 bias, a status word, an optional
  * workspace (see ccv3d_forward).  The caller owns everything else.
- * Two environment variables are read here, for diagnosis only: CCV3D_WAIT_LIMIT_MS (1..10000, default about one
+ * A few environment variables are read here, for diagnosis only: CCV3D_LOG=1 prints one line per call on stderr
+ * (entry point, shape, status, cumulative route counters); CCV3D_WAIT_LIMIT_MS (1..10000, default about one
  * second of SM clocks) bounds every wait inside the kernels; CCV3D_NO_PDL (any value) launches the frame-ring
  * kernels without programmatic stream serialization; CCV3D_NO_COOP_LAUNCH (any value; implied when the
  * process runs under Nsight Compute, which sets NV_COMPUTE_PROFILER_PERFWORKS_DIR) launches the

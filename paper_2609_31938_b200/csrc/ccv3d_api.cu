@@ -81,6 +81,9 @@ struct ccv3d_handle {
     cudaEvent_t* prof_ev;   // PROF_SLOTS x 3 events, created on first enable
     int pdl;             // 1: convolution kernels on frame rings are launched with programmatic stream serialization
     int coop_launch;     // 1: cooperative-staging kernels are launched with the cooperative attribute
+    int log;             // CCV3D_LOG: one line per call on stderr (entry point, shape, status, route counters)
+    const char* call_name;   // entry point and shape of the call in progress, for that line
+    int call_dims[4];
     bool hs_valid;       // host stream (ccv3d_forward_host_stream): the device ring holds the history of hs_geom
     int hs_state[2];     //   ring slot of the next frame, history frames present
     int hs_geom[3];      //   N, H, W of the stream
@@ -242,6 +245,7 @@ ccv3d_status ccv3d_create(ccv3d_handle** out_h, const ccv3d_desc* d, const void*
         if (v > 0 && v <= 10000) h->wait_limit_clk = (long long)prop.clockRate * v;
     }
     h->pdl = getenv("CCV3D_NO_PDL") ? 0 : 1;
+    h->log = (getenv("CCV3D_LOG") && atoi(getenv("CCV3D_LOG")) > 0) ? 1 : 0;
     // a kernel-replaying profiler (it announces itself through NV_COMPUTE_PROFILER_PERFWORKS_DIR) refuses
     // cooperative launches of clusters: ordinary launches there, on a device the profiled process has to itself
     h->coop_launch = (getenv("CCV3D_NO_COOP_LAUNCH") || getenv("NV_COMPUTE_PROFILER_PERFWORKS_DIR")) ? 0 : 1;
@@ -369,7 +373,7 @@ ccv3d_status ccv3d_out_dims(const ccv3d_handle* h, int32_t T, int32_t H, int32_t
 ccv3d_status ccv3d_forward_ex(ccv3d_handle* h, const void* x, const void* cache, int32_t cache_frames, void* out,
                               void* new_cache, int32_t N, int32_t T, int32_t H, int32_t W, void* stream) {
     if (!h) return CCV3D_ERR_INVALID_ARG;
-    h->ctr.calls++;
+    begin_call(h, "ccv3d_forward_ex", N, T, H, W);
     const int tc = hist_len(h->d);
     if (cache_frames < 0 || cache_frames > tc) return count(h, CCV3D_ERR_INVALID_ARG);
     if (cache_frames > 0 && !cache) return count(h, CCV3D_ERR_INVALID_ARG);
@@ -396,7 +400,7 @@ ccv3d_status ccv3d_forward(ccv3d_handle* h, const void* x, const void* cache, vo
 ccv3d_status ccv3d_forward_static(ccv3d_handle* h, const void* x, const void* cache, void* out, void* new_cache,
                                   int32_t N, int32_t T, int32_t H, int32_t W, void* stream) {
     if (!h) return CCV3D_ERR_INVALID_ARG;
-    h->ctr.calls++;
+    begin_call(h, "ccv3d_forward_static", N, T, H, W);
     h->call_cf = cache ? hist_len(h->d) : 0;
     ccv3d_status s = check_forward_args(h, x, cache, out, new_cache, N, T, H, W, true);
     if (s != CCV3D_OK) return count(h, s);
@@ -520,12 +524,12 @@ ccv3d_status ccv3d_forward_host(ccv3d_handle* h, const void* x_host, const void*
     h->call_cf = cache_host ? hist_len(h->d) : 0;
     ccv3d_status s = check_forward_args(h, x_host, cache_host, out_host, new_cache_host, N, T, H, W, false);
     if (s != CCV3D_OK) {
-        h->ctr.calls++;
+        begin_call(h, "ccv3d_forward_host", N, T, H, W);
         return count(h, s);
     }
     h->hs_valid = false;                                   // this call reuses the device buffers of a host stream
     if (host_pipeline_eligible(h, T, H, W)) {
-        h->ctr.calls++;
+        begin_call(h, "ccv3d_forward_host", N, T, H, W);
         if (!on_handle_device(h)) return count(h, CCV3D_ERR_INVALID_ARG);
         s = forward_host_pipelined(h, x_host, cache_host, out_host, new_cache_host, N, T, H, W, (cudaStream_t)stream);
         if (s != CCV3D_OK) return count(h, s);
@@ -557,7 +561,7 @@ ccv3d_status ccv3d_forward_host(ccv3d_handle* h, const void* x_host, const void*
 ccv3d_status ccv3d_forward_host_stream(ccv3d_handle* h, const void* x_host, void* out_host, int32_t reset, int32_t N,
                                        int32_t T, int32_t H, int32_t W, void* stream) {
     if (!h) return CCV3D_ERR_INVALID_ARG;
-    h->ctr.calls++;
+    begin_call(h, "ccv3d_forward_host_stream", N, T, H, W);
     h->call_cf = 0;
     ccv3d_status s = check_forward_args(h, x_host, nullptr, out_host, nullptr, N, T, H, W, false);
     if (s != CCV3D_OK) return count(h, s);
@@ -755,7 +759,7 @@ ccv3d_status ccv3d_forward_ring_up(ccv3d_handle* h, const ccv3d_ring* in, int32_
                                    const ccv3d_ring* res, int32_t res_slot, const ccv3d_ring* out_ring, int32_t out_slot,
                                    int32_t rt, int32_t T, void* stream) {
     if (!h) return CCV3D_ERR_INVALID_ARG;
-    h->ctr.calls++;
+    begin_call(h, "ccv3d_forward_ring_up", in ? in->N : 0, T, in ? in->H : 0, in ? in->W : 0);
     if (rt < 1 || !out_ring) return count(h, CCV3D_ERR_INVALID_ARG);
     if (!on_handle_device(h)) return count(h, CCV3D_ERR_INVALID_ARG);
     return count(h, forward_ring(h, in, x_slot, hist_frames, res, res_slot, out_ring, out_slot, nullptr, T,
@@ -766,7 +770,7 @@ ccv3d_status ccv3d_forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int32_t x
                                 const ccv3d_ring* res, int32_t res_slot, const ccv3d_ring* out_ring,
                                 int32_t out_slot, void* out_ncthw, int32_t T, void* stream) {
     if (!h) return CCV3D_ERR_INVALID_ARG;
-    h->ctr.calls++;
+    begin_call(h, "ccv3d_forward_ring", in ? in->N : 0, T, in ? in->H : 0, in ? in->W : 0);
     if (!on_handle_device(h)) return count(h, CCV3D_ERR_INVALID_ARG);
     return count(h, forward_ring(h, in, x_slot, hist_frames, res, res_slot, out_ring, out_slot, out_ncthw, T,
                                  (cudaStream_t)stream));

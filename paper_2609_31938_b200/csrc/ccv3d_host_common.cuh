@@ -117,7 +117,21 @@ uint32_t pow2_cols(uint32_t c) {
     return v;
 }
 
+// Every entry point that counts as a call starts here ...
+void begin_call(ccv3d_handle* h, const char* name, int N, int T, int H, int W) {
+    h->ctr.calls++;
+    h->call_name = name;
+    h->call_dims[0] = N; h->call_dims[1] = T; h->call_dims[2] = H; h->call_dims[3] = W;
+}
+
+// ... and ends here: the status is counted (Algorithm 1's route counters) and, with CCV3D_LOG=1, reported.
 ccv3d_status count(ccv3d_handle* h, ccv3d_status s) {
+    if (h->log)
+        fprintf(stderr, "ccv3d %p %s N=%d T=%d H=%d W=%d %d->%d k=%dx%dx%d: %s (calls %llu tcgen05 %llu fma %llu launches %llu)\n",
+                (void*)h, h->call_name ? h->call_name : "?", h->call_dims[0], h->call_dims[1], h->call_dims[2], h->call_dims[3],
+                h->d.cin, h->d.cout, h->d.kt, h->d.kh, h->d.kw, ccv3d_status_string(s), (unsigned long long)h->ctr.calls,
+                (unsigned long long)(h->ctr.tcgen05_bf16), (unsigned long long)h->ctr.simt,
+                (unsigned long long)h->ctr.kernel_launches);
     switch (s) {
         case CCV3D_OK: h->ctr.ok++; break;
         case CCV3D_ERR_UNSUPPORTED: h->ctr.unsupported++; break;

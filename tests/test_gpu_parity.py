@@ -561,3 +561,26 @@ def test_half_width_tail_through_ncthw(ccv, Cin, Cout, T, H, W):
         layer.close()
     assert torch.equal(outs[0], outs[1])
     check(as_f64(outs[0]), ref, "bf16")
+
+
+def test_call_log_line():
+    """CCV3D_LOG=1: one line per call on stderr with the entry point, the shape, the status and the route counters
+    (read at create time, so the layer is made in a child process)."""
+    import os
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    code = (
+        "import torch, paper_2609_31938_b200 as ccv\n"
+        "w = torch.randn(64, 64, 3, 3, 3, device='cuda').bfloat16()\n"
+        "l = ccv.CausalConv3d(w)\n"
+        "x = torch.randn(1, 64, 2, 16, 24, device='cuda').bfloat16()\n"
+        "l(x, None); torch.cuda.synchronize()\n"
+        "print(ccv.ccv3d_forward(l.h, None, None, None, None, 1, 2, 16, 24))\n")
+    r = subprocess.run([sys.executable, "-c", code], cwd=root, env=dict(os.environ, CCV3D_LOG="1"), capture_output=True,
+                       text=True, timeout=300)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stderr.splitlines() if l.startswith("ccv3d ")]
+    assert len(lines) == 2, r.stderr
+    assert "ccv3d_forward_ex N=1 T=2 H=16 W=24 64->64 k=3x3x3: CCV3D_OK" in lines[0] and "tcgen05 1" in lines[0]
+    assert "CCV3D_ERR_INVALID_ARG" in lines[1] and "calls 2" in lines[1]
