@@ -83,3 +83,19 @@ def test_neighbour_exchange_over_gloo(world):
                        timeout=600)
     assert r.returncode == 0, (r.stdout[-1500:], r.stderr[-3000:])
     assert f"HSPLIT_OK world={world}" in r.stdout
+
+
+def test_ring_frame_runs_wrap_around():
+    """Slots slot0 .. slot0+T-1 (mod F) as contiguous runs: the row copies of a ring's halo rows go run by run."""
+    from paper_2609_31938_b200.hsplit import _frame_runs
+    assert _frame_runs(0, 4, 6) == [(0, 4, 0)]
+    assert _frame_runs(4, 4, 6) == [(4, 2, 0), (0, 2, 2)]
+    assert _frame_runs(5, 1, 6) == [(5, 1, 0)]
+    assert _frame_runs(7, 3, 6) == [(1, 3, 0)]                    # a slot given beyond F is taken mod F
+    for F in (3, 5, 6):
+        for slot0 in range(F):
+            for T in range(1, F + 1):
+                runs = _frame_runs(slot0, T, F)
+                slots = [s + i for s, n, _ in runs for i in range(n)]
+                assert slots == [(slot0 + t) % F for t in range(T)]
+                assert [t0 for _, _, t0 in runs] == [0] + ([runs[0][1]] if len(runs) == 2 else [])
