@@ -91,8 +91,8 @@ def test_bands_equal_unsplit_layer(ccv, Cin, Cout, T, H, W, k, dil, dtype, world
     whole.close()
 
 
-@pytest.mark.parametrize("world,C,H,W", [(2, 64, 40, 48), (3, 96, 51, 40), (4, 192, 64, 32)])
-def test_ring_block_bands_equal_unsplit(ccv, world, C, H, W):
+@pytest.mark.parametrize("world,C,H,W,spare", [(2, 64, 40, 48, 0), (3, 96, 51, 40, 1), (4, 192, 64, 32, 0), (2, 64, 33, 24, 1)])
+def test_ring_block_bands_equal_unsplit(ccv, world, C, H, W, spare):
     """x <- x + conv2(conv1(x)) on frame rings, streamed over three chunks: every rank's band (its rings hold only its
     slab; halo rows re-exchanged after each layer, residual added in the epilogue) is bit-identical to the same rows
     of the unsplit ring path."""
@@ -102,7 +102,7 @@ def test_ring_block_bands_equal_unsplit(ccv, world, C, H, W):
     w = [to_dev(c["w"]) for c in cs]
     b = [to_dev(c["b"]) for c in cs]
     x = to_dev(cs[0]["x"])
-    F = T + 2
+    F = T + 2 + spare        # spare = 1: five slots, two frames per chunk - the third chunk wraps around inside a call
     # unsplit reference on full-height rings
     L = [ccv.CausalConv3d(w[i], b[i]) for i in range(2)]
     r1, r2 = ccv.FrameRing(1, C, F, H, W, zero=True), ccv.FrameRing(1, C, F, H, W, zero=True)
