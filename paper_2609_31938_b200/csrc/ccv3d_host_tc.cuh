@@ -301,7 +301,9 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     const int in_bands = (H + 15) / 16;
     const bool coop = nbands == 1 && !per_tap && (!general || d.stride[0] == 1) && !f32 &&
                       !(d.flags & CCV3D_FLAG_TWO_KERNELS) && W % 8 == 0 && in_bands <= MAX_COOP_BANDS && tiles_h >= 4 &&
-                      (int64_t)N * tiles_h * p.tiles_w * To * NT * (pair ? 2 : 1) >= 4LL * h->sm_count;   // small problems: two kernels
+                      // fewer than eight waves of tiles: two kernels (the first tiles of a cooperative launch wait for two
+                      // whole bands, and measured at six waves it is 15 % behind; level at seven, ahead from twelve)
+                      (int64_t)N * tiles_h * p.tiles_w * To * NT * (pair ? 2 : 1) >= 8LL * h->sm_count;
     size_t fixed = 1024 /*alignment slack*/ + align_up(sizeof(TcShared), 128) + 2 * (size_t)p.e_slot + (coop ? 9216 : 0);
     // leave room for staging blocks to be resident next to a convolution CTA when the two overlap
     const size_t limit = nbands > 1 ? SMEM_LIMIT - STAGE_COEXIST_BYTES : SMEM_LIMIT;

@@ -50,7 +50,7 @@ CASES = [
     (32, 64, 3, 30, 40, (3, 5, 3), (1, 2, 1), si.BF16, (3,)),          # dilated 5 taps in h: halo of 4 rows
     (16, 24, 2, 18, 20, (3, 3, 3), (1, 1, 1), si.F32, (2,)),
     (64, 64, 2, 24, 32, (3, 1, 1), (1, 1, 1), si.BF16, (2,)),          # temporal-only kernel: nothing exchanged
-    (64, 64, 4, 320, 256, (3, 3, 3), (1, 1, 1), si.BF16, (2,)),        # slabs of 162 rows: large enough for the one-kernel schedule
+    (64, 64, 8, 320, 256, (3, 3, 3), (1, 1, 1), si.BF16, (2,)),        # slabs of 162 rows: large enough for the one-kernel schedule
 ]
 
 

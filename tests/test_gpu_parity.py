@@ -221,7 +221,7 @@ def test_bf16_tensor_core_cooperative_staging(ccv, Cin, Cout, W):
     """Large enough for the default schedule to stage inside the convolution kernel (four stager warps per CTA, a
     band of 16 rows ahead of the tiles that read it): one launch per call, and the same bits as the two-kernel
     schedule."""
-    c = si.conv_case(1, Cin, Cout, 8, 125, W, seed=18)               # 8 tile rows (ragged last), >= 640 tiles
+    c = si.conv_case(1, Cin, Cout, 16, 125, W, seed=18)              # 8 tile rows (ragged last), more than eight waves of tiles
     m, ctr = run_case(ccv, c)
     assert ctr["tcgen05_bf16"] == 1 and ctr["kernel_launches"] == 3    # weight pack, bias, one fused staging+convolution launch
     a = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]))
