@@ -301,9 +301,31 @@ def other_configs_leg(dev):
     # the HBM-bound 1x1x1 layer first, after a pause: right after a long tensor-bound run the part is still in its
     # power-capped state and the same kernel measures 20 % slower
     time.sleep(1.0)
-    for name in ("cfg4c_bf16_pw_192_96", "cfg2_bf16_384", "cfg4a_bf16_96", "cfg4b_bf16_192_96"):
+    for name in ("cfg4c_bf16_pw_192_96", "cfg2_bf16_384", "cfg4a_bf16_96", "cfg4b_bf16_192_96", "cfg1_f32_16"):
         d = {k: v for k, v in si.CONFIGS[name].items() if k not in ("dtype", "x_dist")}
         N, Cin, Cout, T, H, W, k = d["N"], d["Cin"], d["Cout"], d["T"], d["H"], d["W"], d["k"]
+        if si.CONFIGS[name]["dtype"] == si.F32:
+            # the FP32 configuration (7 MFLOP): FP32-FMA kernel, bound by launch latency; U(-1,1) activations
+            x = torch.rand(N, Cin, T, H, W, device=dev, generator=gen) * 2 - 1
+            cache = torch.rand(N, Cin, k[0] - 1, H, W, device=dev, generator=gen) * 2 - 1
+            layer = ccv.CausalConv3d(torch.randn(Cout, Cin, *k, device=dev, generator=gen) / math.sqrt(Cin * 27),
+                                     torch.randn(Cout, device=dev, generator=gen) * math.sqrt(0.1))
+            y, nc = torch.empty((N, Cout, T, H, W), device=dev), torch.empty_like(cache)
+            for _ in range(3):
+                layer(x, cache, out=y, new_cache=nc)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for _ in range(20):
+                layer(x, cache, out=y, new_cache=nc)
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / 20
+            out[name] = {"ms_per_call": ms, "tflops": si.conv_flops(**d) / (ms * 1e-3) / 1e12, "dtype": "f32",
+                         "note": "FP32-FMA kernel plus cache copy; two launches, latency-bound"}
+            assert layer.device_status()[0] == ccv.OK
+            layer.close()
+            continue
         rnd = lambda *shape, std=1.0: (torch.randn(*shape, device=dev, generator=gen) * std).to(torch.bfloat16)
         x = rnd(N, Cin, T, H, W)
         cache = rnd(N, Cin, k[0] - 1, H, W) if k[0] > 1 else None

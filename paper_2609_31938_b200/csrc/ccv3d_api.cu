@@ -113,10 +113,18 @@ ccv3d_status forward_simt(ccv3d_handle* h, const void* x, const void* cache, voi
     const int64_t npix = (int64_t)N * p.To * p.Ho * p.Wo;
     const int64_t gx = (npix + SIMT_THREADS - 1) / SIMT_THREADS;
     if (gx > 0x7FFFFFFF) return CCV3D_ERR_UNSUPPORTED;
-    dim3 grid((unsigned)gx, (d.cout + SIMT_CO - 1) / SIMT_CO);
+    // eight output channels per thread amortise the activation loads; a call with fewer threads than that gives the
+    // device (configuration 1: 512 pixels x 2 channel groups) runs one channel per thread instead
+    const bool thin = gx * ((d.cout + SIMT_CO - 1) / SIMT_CO) < 4LL * h->sm_count;
+    const int co_per_thread = thin ? 1 : SIMT_CO;
+    dim3 grid((unsigned)gx, (d.cout + co_per_thread - 1) / co_per_thread);
     cudaEvent_t* pev = (h->prof_on && h->prof_ev) ? h->prof_ev + 3 * (h->prof_n % PROF_SLOTS) : nullptr;
     if (pev) { cudaEventRecord(pev[0], st); cudaEventRecord(pev[1], st); }
-    if (d.dtype == CCV3D_F32) conv3d_direct_kernel<float, float><<<grid, SIMT_THREADS, 0, st>>>(p);
+    if (thin) {
+        if (d.dtype == CCV3D_F32) conv3d_direct_kernel<float, float, 1><<<grid, SIMT_THREADS, 0, st>>>(p);
+        else if (d.out_dtype == CCV3D_BF16) conv3d_direct_kernel<__nv_bfloat16, __nv_bfloat16, 1><<<grid, SIMT_THREADS, 0, st>>>(p);
+        else conv3d_direct_kernel<__nv_bfloat16, float, 1><<<grid, SIMT_THREADS, 0, st>>>(p);
+    } else if (d.dtype == CCV3D_F32) conv3d_direct_kernel<float, float><<<grid, SIMT_THREADS, 0, st>>>(p);
     else if (d.out_dtype == CCV3D_BF16) conv3d_direct_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, SIMT_THREADS, 0, st>>>(p);
     else conv3d_direct_kernel<__nv_bfloat16, float><<<grid, SIMT_THREADS, 0, st>>>(p);
     if (cudaGetLastError() != cudaSuccess) return cuda_fail();

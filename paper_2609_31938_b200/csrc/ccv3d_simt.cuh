@@ -35,12 +35,14 @@ struct SimtParams {
 };
 // With tc = d_t (kt-1): Z = [absent x (tc-cf) ; cache ; x]; frame tau < tc of Z is cache frame tau-(tc-cf) when that is >= 0.
 
-constexpr int SIMT_CO = 8;       // output channels per thread
+constexpr int SIMT_CO = 8;       // output channels per thread (1 for calls too small to fill the device otherwise)
 constexpr int SIMT_THREADS = 128;
 
-// grid.x: ceil(N*To*Ho*Wo / SIMT_THREADS), grid.y: ceil(Cout / SIMT_CO)
-template <typename TIn, typename TOut>
+// grid.x: ceil(N*To*Ho*Wo / SIMT_THREADS), grid.y: ceil(Cout / CO).  The order of accumulation of an output element
+// does not depend on CO.
+template <typename TIn, typename TOut, int CO = SIMT_CO>
 __global__ void __launch_bounds__(SIMT_THREADS) conv3d_direct_kernel(const SimtParams p) {
+    constexpr int SIMT_CO = CO;
     const int64_t HW = (int64_t)p.H * p.W, HWo = (int64_t)p.Ho * p.Wo;
     const int64_t npix = (int64_t)p.N * p.To * HWo;
     const int64_t pix = (int64_t)blockIdx.x * SIMT_THREADS + threadIdx.x;
