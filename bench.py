@@ -305,7 +305,7 @@ def other_configs_leg(dev):
         d = {k: v for k, v in si.CONFIGS[name].items() if k not in ("dtype", "x_dist")}
         N, Cin, Cout, T, H, W, k = d["N"], d["Cin"], d["Cout"], d["T"], d["H"], d["W"], d["k"]
         if si.CONFIGS[name]["dtype"] == si.F32:
-            # the FP32 configuration (7 MFLOP): FP32-FMA kernel, bound by launch latency; U(-1,1) activations
+            # the FP32 configuration (7 MFLOP, K = 432): tensor cores by 3xTF32, latency-bound; U(-1,1) activations
             x = torch.rand(N, Cin, T, H, W, device=dev, generator=gen) * 2 - 1
             cache = torch.rand(N, Cin, k[0] - 1, H, W, device=dev, generator=gen) * 2 - 1
             layer = ccv.CausalConv3d(torch.randn(Cout, Cin, *k, device=dev, generator=gen) / math.sqrt(Cin * 27),
@@ -322,7 +322,7 @@ def other_configs_leg(dev):
             torch.cuda.synchronize()
             ms = e0.elapsed_time(e1) / 20
             out[name] = {"ms_per_call": ms, "tflops": si.conv_flops(**d) / (ms * 1e-3) / 1e12, "dtype": "f32",
-                         "note": "FP32-FMA kernel plus cache copy; two launches, latency-bound"}
+                         "note": "3xTF32 route (staging + convolution, two short launches); latency-bound"}
             assert layer.device_status()[0] == ccv.OK
             layer.close()
             continue

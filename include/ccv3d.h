@@ -58,8 +58,8 @@ typedef enum {
                                             by TMA and transposes in shared memory (needs W % 8 == 0, else the staged route is taken). Some 10 % slower
                                             than the default route; for callers that cannot afford the workspace. */
 #define CCV3D_FLAG_F32_TENSOR 0x20u       /* FP32 layers: always use the tensor cores (3xTF32: each FP32 product as hi*hi + hi*lo + lo*hi of TF32
-                                            operands, FP32 accumulate); the default sends calls under 0.2 GFLOP, and layers with cin*kt*kh*kw > 16384,
-                                            to the FP32-FMA kernel */
+                                            operands, FP32 accumulate); the default sends layers with K = cin*kt*kh*kw > 16384, and calls that are
+                                            both under 0.2 GFLOP and of K < 256, to the FP32-FMA kernel */
 #define CCV3D_FLAG_NO_PAIR 0x40u          /* tensor-core route: never run tiles on pairs of CTAs (cta_group::2 MMAs with M = 256, each SM
                                             streaming half of every weight tile) - the default for layers with more than 128 output
                                             channels per tile and 3x3 or 1x1 spatial kernels */

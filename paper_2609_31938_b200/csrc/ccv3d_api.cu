@@ -174,9 +174,13 @@ bool on_handle_device(const ccv3d_handle* h) {
 bool f32_takes_tensor_cores(const ccv3d_handle* h, int N, int T, int H, int W) {
     const ccv3d_desc& d = h->d;
     if (d.flags & CCV3D_FLAG_F32_TENSOR) return true;
-    if ((int64_t)d.cin * d.kt * d.kh * d.kw > 16384) return false;
-    const double flops = 2.0 * N * out_t(d, T) * out_h(d, H) * out_w(d, W) * d.cout * d.cin * d.kt * d.kh * d.kw;
-    return flops >= 2.0e8;
+    const int64_t K = (int64_t)d.cin * d.kt * d.kh * d.kw;
+    if (K > 16384) return false;
+    // Large calls for the throughput; small ones whenever the FMA kernel's serial walk over K (one thread per output
+    // element, ~0.2 us per tap row) would outlast the two short launches of this route (~20 us together):
+    // configuration 1 (K = 432) runs 21 us here against 80 us there.
+    const double flops = 2.0 * N * out_t(d, T) * out_h(d, H) * out_w(d, W) * d.cout * K;
+    return flops >= 2.0e8 || K >= 256;
 }
 
 ccv3d_status check_forward_args(const ccv3d_handle* h, const void* x, const void* cache, void* out, void* new_cache,

@@ -227,24 +227,34 @@ def test_fp32_on_tensor_cores_3xtf32(ccv, N, Cin, Cout, T, H, W, k, cf, stride, 
 
 
 def test_fp32_route_selection_by_size(ccv):
-    """Small FP32 calls stay on the FP32-FMA kernel, calls of 0.2 GFLOP and more go to the tensor cores; both within
-    tolerance and close to each other."""
+    """FP32 calls go to the tensor cores (3xTF32) when they are large (0.2 GFLOP and more) or when K is long enough
+    (256 and more) for the FMA kernel's serial walk to lose; short-K small calls stay on the FMA kernel.  Both routes
+    within tolerance and close to each other."""
     c = _case(1, 64, 64, 4, 44, 80, (3, 3, 3), si.F32, 2, seed=42)          # 3.1 GFLOP
     ref, ref_nc = oracle.forward_general(c["x"], c["cache"], c["w"], c["b"])
     outs = {}
     for name, flags in (("auto", 0), ("fma", ccv.FLAG_FORCE_SIMT)):
         layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), flags=flags)
         o, nc = layer(to_dev(c["x"]), to_dev(c["cache"]))
-        small, _ = layer(to_dev(c["x"])[:, :, :1, :8, :8].contiguous(), None)    # 2.8 MFLOP: FP32-FMA kernel either way
+        small, _ = layer(to_dev(c["x"])[:, :, :1, :8, :8].contiguous(), None)    # 2.8 MFLOP, but K = 1728: tensor cores too
         torch.cuda.synchronize()
         ctr = layer.counters()
-        assert (ctr["tcgen05_bf16"], ctr["simt"]) == ((1, 1) if name == "auto" else (0, 2))
+        assert (ctr["tcgen05_bf16"], ctr["simt"]) == ((2, 0) if name == "auto" else (0, 2))
         check(as_f64(o), ref, "f32")
         assert np.array_equal(bits(nc), ref_nc)
         outs[name] = as_f64(o)
         layer.close()
     rms = float(np.sqrt(np.mean(ref ** 2)))
     assert np.abs(outs["auto"] - outs["fma"]).max() <= 1e-4 * rms
+    # K = 8 x 27 = 216 and a small call: the FMA kernel
+    c2 = _case(1, 8, 16, 2, 12, 20, (3, 3, 3), si.F32, 2, seed=43)
+    ref2, _ = oracle.forward_general(c2["x"], c2["cache"], c2["w"], c2["b"])
+    layer = ccv.CausalConv3d(to_dev(c2["w"]), to_dev(c2["b"]))
+    o2, _ = layer(to_dev(c2["x"]), to_dev(c2["cache"]))
+    torch.cuda.synchronize()
+    assert layer.counters()["simt"] == 1 and layer.counters()["tcgen05_bf16"] == 0
+    check(as_f64(o2), ref2, "f32")
+    layer.close()
 
 
 @pytest.mark.parametrize("Cin,Cout,H,W", [(64, 64, 96, 96), (48, 192, 64, 80)])   # two pixel blocks per CTA; one

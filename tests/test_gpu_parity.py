@@ -61,9 +61,13 @@ def run_case(ccv, c, flags=0, out_dtype=None, kind=None):
     return m, ctr
 
 
-# ---------------------------------------------------------------------------- FP32 (plain FMA kernel)
+# ---------------------------------------------------------------------------- FP32
 def test_cfg1_fp32(ccv):
+    """Configuration 1 on both FP32 routes: the tensor cores by 3xTF32 (the default: K = 432 is long enough for the
+    FMA kernel's serial walk to lose) and the plain FMA kernel, each within the FP32 tolerance, cache bit-exact."""
     m, ctr = run_case(ccv, si.conv_case(**si.CONFIGS["cfg1_f32_16"]))
+    assert ctr["tcgen05_bf16"] == 1 and ctr["simt"] == 0 and m["cos"] > 0.9999999
+    m, ctr = run_case(ccv, si.conv_case(**si.CONFIGS["cfg1_f32_16"]), flags=ccv.FLAG_FORCE_SIMT)
     assert ctr["simt"] == 1 and m["cos"] > 0.9999999
 
 
