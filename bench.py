@@ -11,14 +11,21 @@ inputs are seeded, synthetic, resident in HBM when the timed region starts, and 
 needed).  One JSON line on stdout.
 
 --impl reference times the CPU oracle (the plain FP64 definition) on a bounded spatial crop of the same
-workload on the host's cores.  With N > 1 (torchrun) every rank runs an independent replica (no collective
-on the data path): weak scaling.
+workload on the host's cores.  With N > 1 every rank runs an independent replica (no collective on the data
+path): weak scaling.  Started without torchrun, `--gpus N` with N > 1 starts its own N ranks (one per GPU).
+
+Besides the K timed steps the line carries a `sustained` leg (at least two seconds of back-to-back calls
+whatever --steps says, per-call times from events, clocks sampled throughout), the other benchmark
+configurations each with its own roofline, clock record and CPU-oracle baseline, cold-L2 figures for the
+HBM-bound kernels, and the first-chunk (NULL cache) form with its useful FLOP count.
 """
 from __future__ import annotations
 
 import argparse
 import json
 import os
+import socket
+import subprocess
 import sys
 import threading
 import time
@@ -34,13 +41,24 @@ import synth_inputs as si  # noqa: E402
 METRIC = "causal Conv3D BF16 TFLOP/s"
 DEFAULT_WORKLOAD = "cfg3_bf16_192"
 
-# DRAM bytes (read + write) of one launch of the step's kernel (default schedule: staging, cache update and
-# convolution in one kernel), from an ncu capture of a quarter-size case (192->192, T=4, 176x320: 239.4 MB read +
-# 224.6 MB written) scaled by the pixel count; the summary is profiles/conv3d_tcgen05_coop_192ch_176x320.md.
-TRAFFIC_BYTES_PER_LAUNCH = {"cfg3_bf16_192": 4 * (239.4e6 + 224.6e6)}
-# The same for the kernel on frame rings (profiles/conv3d_tcgen05_ring_192ch_176x320.md: 132.0 MB read + 53.6 MB
-# written during the kernel, the rest of the 86.5 MB output still in L2 when it ends).
-TRAFFIC_BYTES_PER_LAUNCH_RESIDENT = {"cfg3_bf16_192": 4 * (132.0e6 + 53.6e6)}
+NOMINAL_BF16_TFLOPS = 2250.0     # B200 dense BF16, the datasheet figure the 60 % target is stated on
+
+# DRAM bytes (read + write) of one launch of a kernel, from ncu captures of quarter-size cases scaled by the pixel
+# count (activation reads and output writes grow with it; the weights are 2 MB).  Keyed by workload AND by the kernel
+# variant that ran, so that a changed schedule cannot inherit another variant's figure (it reports null instead).
+#   one_kernel  = cooperative staging on CTA pairs (staging + cache update + convolution in one launch):
+#                 profiles/conv3d_tcgen05_coop_192ch_176x320.md, 239.4 MB read + 224.6 MB written at 176x320
+#   ring        = the same kernel on frame rings: profiles/conv3d_tcgen05_ring_192ch_176x320.md, 132.0 MB read +
+#                 53.6 MB written during the kernel (the rest of the 86.5 MB output still in L2 when it ends)
+#   two_kernels = the convolution kernel of the two-kernel schedule: profiles/conv3d_tcgen05_192ch_176x320.md
+TRAFFIC_BYTES_PER_LAUNCH = {
+    ("cfg3_bf16_192", "one_kernel"): 4 * (239.4e6 + 224.6e6),
+    ("cfg3_bf16_192", "ring"): 4 * (132.0e6 + 53.6e6),
+    ("cfg3_bf16_192", "two_kernels"): 4 * (133.2e6 + 53.0e6),
+    ("cfg4a_bf16_96", "one_kernel"): 4 * (434.2e6 + 476.5e6),   # profiles/conv3d_tcgen05_coop_96ch_352x640.md
+    # profiles/conv1x1_tcgen05_192to96_352x640.md: x read once, 137 of the 173 MB of output written during the kernel
+    ("cfg4c_bf16_pw_192_96", "pointwise"): 4 * (346.1e6 + 137.0e6),
+}
 
 
 def measured_peaks():
@@ -287,70 +305,144 @@ def chain_leg(dev):
     return res
 
 
-def other_configs_leg(dev):
-    """The remaining benchmark configurations in short bursts (10 calls each after 3 warm-ups), through ccv3d_forward
-    (NCTHW boundary) and, for the cached layers, through ccv3d_forward_ring.  Inputs of these secondary legs are
-    drawn on the device (seeded normal activations, fan-in-scaled weights): same shapes and distributions as the
-    seeded host generator, which the headline workload and the tests use."""
-    import math
+class L2Flusher:
+    """Evicts the L2 between timed calls by writing a buffer twice its size (cold-L2 figures of the HBM-bound kernels)."""
+
+    def __init__(self, dev, nbytes=320 << 20):
+        import torch
+        self.buf = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+
+    def __call__(self):
+        self.buf.add_(1)
+
+
+def timed_calls(fn, iters, warmup=3, flush=None):
+    """Per-call device times in ms (CUDA events on the current stream).  Without `flush` the calls run back to back
+    and call i is the time between the events before it and after it (launch gaps included); with `flush` every
+    call is timed on its own after the flush."""
+    import torch
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2 * iters if flush else iters + 1)]
+    if flush:
+        for i in range(iters):
+            flush()
+            ev[2 * i].record()
+            fn()
+            ev[2 * i + 1].record()
+        torch.cuda.synchronize()
+        return [ev[2 * i].elapsed_time(ev[2 * i + 1]) for i in range(iters)]
+    ev[0].record()
+    for i in range(iters):
+        fn()
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    return [ev[i].elapsed_time(ev[i + 1]) for i in range(iters)]
+
+
+def stats(ms_list):
+    a = np.asarray(ms_list, dtype=np.float64)
+    return {"ms_mean": float(a.mean()), "ms_median": float(np.median(a)), "ms_min": float(a.min()), "samples": int(a.size)}
+
+
+def roofline_of(flops, abytes, ms, peaks):
+    """The slower of FLOPs at the measured tensor peak and algorithmic bytes at the measured HBM bandwidth, against
+    the measured time; `bound` names which of the two it is."""
+    t_tensor = flops / (peaks["tflops"] * 1e12) * 1e3
+    t_hbm = abytes / (peaks["hbm_gbs"] * 1e9) * 1e3
+    if t_tensor >= t_hbm:
+        ach = flops / (ms * 1e-3) / 1e12
+        return {"bound": "tensor", "achieved": ach, "peak": peaks["tflops"], "unit": "TFLOP/s", "frac": ach / peaks["tflops"],
+                "frac_of_nominal_2250": ach / NOMINAL_BF16_TFLOPS, "peak_source": f"{peaks['source']} (burst cuBLAS bf16)"}
+    ach = abytes / (ms * 1e6)
+    return {"bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": ach / peaks["hbm_gbs"],
+            "peak_source": f"{peaks['source']} (device copy)"}
+
+
+def kernel_variant(ccv, layer, fn):
+    """Which kernels served `fn` (two profiled calls): the 1x1x1 streaming kernel, one launch that stages and
+    convolves, or a staging kernel followed by the convolution kernel."""
+    import torch
+    p0 = layer.counters()["pointwise"]
+    ccv.ccv3d_profile_enable(layer.h, True)
+    fn()
+    fn()
+    torch.cuda.synchronize()
+    _, stage_ms, _, ncalls = ccv.ccv3d_profile_read(layer.h)
+    ccv.ccv3d_profile_enable(layer.h, False)
+    if layer.counters()["pointwise"] > p0:
+        return "pointwise"
+    return "one_kernel" if stage_ms / max(ncalls, 1) < 0.02 else "two_kernels"
+
+
+def useful_tap_fraction(T, kt, cache_frames):
+    """Share of the (output frame, temporal tap) pairs whose source frame exists (Eq. (4)): with no history the
+    taps that would read it are skipped - 1/3, 3/6, 9/12 of them remain at T = 1, 2, 4 with kt = 3."""
+    p_l = (kt - 1) - cache_frames
+    return sum(1 for t in range(T) for k in range(kt) if t + k - p_l >= 0) / float(T * kt)
+
+
+def other_configs_leg(dev, local):
+    """The remaining benchmark configurations, each in a burst of 20 calls after 3 warm-ups, through ccv3d_forward
+    (NCTHW boundary) and, for the cached layers, through ccv3d_forward_ring; the first-chunk (NULL cache) form of
+    the headline layer; the staging + cache-update kernel alone; cold-L2 repeats of the HBM-bound ones.  Inputs come
+    from the seeded host generator (the tensors the parity tests use); every entry carries its own roofline, clock
+    record and CPU-oracle baseline (a bounded spatial crop, stated)."""
     import torch
     import paper_2609_31938_b200 as ccv
     peaks = measured_peaks()
     out = {}
-    gen = torch.Generator(device=dev).manual_seed(0)
+    flush = L2Flusher(dev)
+
+    def up(a):
+        if a is None:
+            return None
+        if a.dtype == np.uint16:
+            return torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
+        return torch.from_numpy(a).to(dev)
+
+    def clocked(fn, iters=20, flush_fn=None):
+        smp = ClockSampler(local, period_s=0.002)
+        smp.start()
+        ms = timed_calls(fn, iters, flush=flush_fn)
+        smp.stop()
+        return ms, smp.summary()
+
     # the HBM-bound 1x1x1 layer first, after a pause: right after a long tensor-bound run the part is still in its
-    # power-capped state and the same kernel measures 20 % slower
+    # power-capped state and the same kernel measures 20 % slower (the clock record of the entry shows which state
+    # it ran in)
     time.sleep(1.0)
     for name in ("cfg4c_bf16_pw_192_96", "cfg2_bf16_384", "cfg4a_bf16_96", "cfg4b_bf16_192_96", "cfg1_f32_16"):
-        d = {k: v for k, v in si.CONFIGS[name].items() if k not in ("dtype", "x_dist")}
+        cfg, d = cfg_of(name)
         N, Cin, Cout, T, H, W, k = d["N"], d["Cin"], d["Cout"], d["T"], d["H"], d["W"], d["k"]
-        if si.CONFIGS[name]["dtype"] == si.F32:
-            # the FP32 configuration (7 MFLOP, K = 432): tensor cores by 3xTF32, latency-bound; U(-1,1) activations
-            x = torch.rand(N, Cin, T, H, W, device=dev, generator=gen) * 2 - 1
-            cache = torch.rand(N, Cin, k[0] - 1, H, W, device=dev, generator=gen) * 2 - 1
-            layer = ccv.CausalConv3d(torch.randn(Cout, Cin, *k, device=dev, generator=gen) / math.sqrt(Cin * 27),
-                                     torch.randn(Cout, device=dev, generator=gen) * math.sqrt(0.1))
-            y, nc = torch.empty((N, Cout, T, H, W), device=dev), torch.empty_like(cache)
-            for _ in range(3):
-                layer(x, cache, out=y, new_cache=nc)
-            torch.cuda.synchronize()
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            for _ in range(20):
-                layer(x, cache, out=y, new_cache=nc)
-            e1.record()
-            torch.cuda.synchronize()
-            ms = e0.elapsed_time(e1) / 20
-            out[name] = {"ms_per_call": ms, "tflops": si.conv_flops(**d) / (ms * 1e-3) / 1e12, "dtype": "f32",
-                         "note": "3xTF32 route (staging + convolution, two short launches); latency-bound"}
-            assert layer.device_status()[0] == ccv.OK
-            layer.close()
-            continue
-        rnd = lambda *shape, std=1.0: (torch.randn(*shape, device=dev, generator=gen) * std).to(torch.bfloat16)
-        x = rnd(N, Cin, T, H, W)
-        cache = rnd(N, Cin, k[0] - 1, H, W) if k[0] > 1 else None
-        layer = ccv.CausalConv3d(rnd(Cout, Cin, *k, std=1.0 / math.sqrt(Cin * k[0] * k[1] * k[2])), rnd(Cout, std=math.sqrt(0.1)))
-        y = torch.empty((N, Cout, T, H, W), dtype=torch.bfloat16, device=dev)
+        f32 = cfg["dtype"] == si.F32
+        c = si.conv_case(**cfg)
+        x, cache = up(c["x"]), up(c["cache"])
+        layer = ccv.CausalConv3d(up(c["w"]), up(c["b"]))
+        y = torch.empty((N, Cout, T, H, W), dtype=torch.float32 if f32 else torch.bfloat16, device=dev)
         nc = torch.empty_like(cache) if cache is not None else None
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-
-        def timed(fn, iters=10):
-            for _ in range(3):
-                fn()
-            torch.cuda.synchronize()
-            e0.record()
-            for _ in range(iters):
-                fn()
-            e1.record()
-            torch.cuda.synchronize()
-            return e0.elapsed_time(e1) / iters
-
-        ms = timed(lambda: layer(x, cache, out=y, new_cache=nc))
-        flops, abytes = si.conv_flops(**d), si.conv_bytes(**d)
-        row = {"ms_per_call": ms, "tflops": flops / (ms * 1e-3) / 1e12, "gbs": abytes / (ms * 1e6),
-               "frac_of_measured_bf16_peak": flops / (ms * 1e-3) / 1e12 / peaks["tflops"],
-               "frac_of_measured_hbm": abytes / (ms * 1e6) / peaks["hbm_gbs"]}
-        if cache is not None:
+        es = 4 if f32 else 2
+        flops, abytes = si.conv_flops(**d), si.conv_bytes(**d, elem=es, out_elem=es)
+        ms, clk = clocked(lambda: layer(x, cache, out=y, new_cache=nc))
+        st = stats(ms)
+        row = {"ms_per_call": st["ms_median"], **st, "tflops": flops / (st["ms_median"] * 1e-3) / 1e12,
+               "gbs": abytes / (st["ms_median"] * 1e6), "clocks": clk, "data": "seeded synthetic (host generator)"}
+        if f32:
+            row["dtype"] = "f32"
+            row["note"] = "3xTF32 route (staging + convolution, two short launches); latency-bound: no roofline claim"
+        else:
+            row["roofline"] = roofline_of(flops, abytes, st["ms_median"], peaks)
+            variant = kernel_variant(ccv, layer, lambda: layer(x, cache, out=y, new_cache=nc))
+            row["roofline"]["kernel_variant"] = variant
+            row["roofline"]["traffic"] = TRAFFIC_BYTES_PER_LAUNCH.get((name, variant))
+        if name == "cfg4c_bf16_pw_192_96":
+            cms, cclk = clocked(lambda: layer(x, cache, out=y, new_cache=nc), flush_fn=flush)
+            cst = stats(cms)
+            row["cold_l2"] = {**cst, "gbs": abytes / (cst["ms_median"] * 1e6),
+                              "frac_of_measured_hbm": abytes / (cst["ms_median"] * 1e6) / peaks["hbm_gbs"], "clocks": cclk,
+                              "note": "every call timed on its own after a 320 MB write that evicts the L2"}
+        if cache is not None and not f32:
             F = T + k[0] - 1
             rin, rout = ccv.FrameRing(N, Cin, F, H, W), ccv.FrameRing(N, Cout, T, H, W)
             rin.load(0, cache)
@@ -361,15 +453,60 @@ def other_configs_leg(dev):
                 layer.forward_ring(rin, slot[0], k[0] - 1, T, out_ring=rout)
                 slot[0] = (slot[0] + T) % F
 
-            rms = timed(ring_step)
-            row["resident_ms_per_call"] = rms
-            row["resident_tflops"] = flops / (rms * 1e-3) / 1e12
+            rms, rclk = clocked(ring_step)
+            rst = stats(rms)
+            r_bytes = 2 * N * H * W * T * (Cin + Cout) + c["w"].nbytes
+            row["resident"] = {**rst, "tflops": flops / (rst["ms_median"] * 1e-3) / 1e12, "clocks": rclk,
+                               "roofline": roofline_of(flops, r_bytes, rst["ms_median"], peaks)}
+            row["resident_ms_per_call"] = rst["ms_median"]
+            row["resident_tflops"] = row["resident"]["tflops"]
             del rin, rout
         assert layer.device_status()[0] == ccv.OK
         layer.close()
+        if not f32:
+            row["cpu_baseline"] = cpu_baseline(name, target_s=3.0)
         out[name] = row
-        del x, cache, y, nc
+        del x, cache, y, nc, c
         torch.cuda.empty_cache()
+
+    # ---- the headline layer's first-chunk form (NULL cache: the taps of absent history are skipped) and its
+    # staging + cache-update kernel alone (two-kernel schedule), warm and with a cold L2
+    name = DEFAULT_WORKLOAD
+    cfg, d = cfg_of(name)
+    c = si.conv_case(**cfg)
+    x, cache = up(c["x"]), up(c["cache"])
+    y = torch.empty((d["N"], d["Cout"], d["T"], d["H"], d["W"]), dtype=torch.bfloat16, device=dev)
+    nc = torch.empty_like(cache)
+    layer = ccv.CausalConv3d(up(c["w"]), up(c["b"]))
+    ms, clk = clocked(lambda: layer(x, None, out=y, new_cache=nc))
+    st = stats(ms)
+    flops = si.conv_flops(**d)
+    useful = useful_tap_fraction(d["T"], d["k"][0], 0)
+    out[name + "_null_cache"] = {
+        **st, "ms_per_call": st["ms_median"], "tflops_conventional": flops / (st["ms_median"] * 1e-3) / 1e12,
+        "useful_tap_fraction": useful, "tflops_useful": useful * flops / (st["ms_median"] * 1e-3) / 1e12, "clocks": clk,
+        "roofline": roofline_of(useful * flops, si.conv_bytes(**d) - c["cache"].nbytes, st["ms_median"], peaks),
+        "note": "first chunk: no cache is read, the new cache is still written; FLOPs counted with the skipped "
+                "(frame, tap) pairs removed (9 of 12 remain at T = 4, kt = 3), and by the usual convention"}
+    layer.close()
+    two = ccv.CausalConv3d(up(c["w"]), up(c["b"]), flags=ccv.FLAG_TWO_KERNELS)
+    stage_bytes = 2 * c["x"].nbytes + 2 * c["cache"].nbytes + c["cache"].nbytes   # read x, cache; write the copy, new cache
+    k4 = {}
+    for label, fl in (("warm", None), ("cold_l2", flush)):
+        ccv.ccv3d_profile_enable(two.h, True)
+        timed_calls(lambda: two(x, cache, out=y, new_cache=nc), 10, flush=fl)
+        _, stage_ms, conv_ms, ncalls = ccv.ccv3d_profile_read(two.h)
+        ccv.ccv3d_profile_enable(two.h, False)
+        sms = stage_ms / max(ncalls, 1)
+        k4[label] = {"ms": sms, "gbs": stage_bytes / (sms * 1e6), "frac_of_measured_hbm": stage_bytes / (sms * 1e6) / peaks["hbm_gbs"],
+                     "conv_kernel_ms": conv_ms / max(ncalls, 1), "calls": int(ncalls)}
+    k4["bytes"] = int(stage_bytes)
+    k4["note"] = ("stage_frames_kernel of the two-kernel schedule (CCV3D_FLAG_TWO_KERNELS): reads x and the cache once, "
+                  "writes the channels-last copy and the new cache; mean over the calls, events recorded by the library "
+                  "between its kernels (with the flush the convolution kernel finds the copy in DRAM)")
+    out[name + "_staging_and_cache_update"] = k4
+    assert two.device_status()[0] == ccv.OK
+    two.close()
     return out
 
 
@@ -446,6 +583,48 @@ def hsplit_leg(dev):
     return out
 
 
+def hsplit_exchange_leg(dev, dist, world, rank):
+    """World >= 2 only: the headline layer split by image rows over the ranks, on frame rings, with the real
+    neighbour exchange (NCCL send/recv into this GPU's own buffers; no kernel reads a peer's memory).  Per rank:
+    ms of the ring call on its slab and of the exchange of the output's halo rows; the slowest rank counts."""
+    import torch
+    import paper_2609_31938_b200 as ccv
+    from paper_2609_31938_b200.hsplit import HSplitRingConv3d
+    cfg, d = cfg_of(DEFAULT_WORKLOAD)
+    N, Cin, Cout, T, H, W, k = d["N"], d["Cin"], d["Cout"], d["T"], d["H"], d["W"], d["k"]
+    c = si.conv_case(**dict(cfg, H=8, W=8))                 # seeded weights and bias of the layer
+    up = lambda a: torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
+    rl = HSplitRingConv3d(up(c["w"]), up(c["b"]), H, rank, world)
+    F = T + k[0] - 1
+    rin, rout = rl.ring(N, Cin, F, W), rl.ring(N, Cout, T, W)
+    rin.buf.normal_()
+    slot = [k[0] - 1]
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    conv_ms, xch_ms = [], []
+    for it in range(13):
+        dist.barrier()
+        ev[0].record()
+        rl.conv.forward_ring(rin, slot[0], k[0] - 1, T, out_ring=rout)
+        ev[1].record()
+        rl.exchange(rout, 0, T)
+        ev[2].record()
+        torch.cuda.synchronize()
+        slot[0] = (slot[0] + T) % F
+        if it >= 3:
+            conv_ms.append(ev[0].elapsed_time(ev[1]))
+            xch_ms.append(ev[1].elapsed_time(ev[2]))
+    t = torch.tensor([float(np.median(conv_ms)), float(np.median(xch_ms))], dtype=torch.float64, device=dev)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    p = rl.plan
+    ok = rl.conv.device_status()[0] == ccv.OK
+    rl.close()
+    return {"workload": DEFAULT_WORKLOAD, "world": world, "rows_per_rank": p.rows, "conv_ms_max_over_ranks": float(t[0]),
+            "exchange_us_max_over_ranks": 1e3 * float(t[1]), "halo_bytes_sent_per_rank_step": int(2 * N * Cout * T * (p.top + p.bot) * W),
+            "device_status_ok": bool(ok),
+            "note": "HSplitRingConv3d with DistTransport: ring call on the slab, then pack + NCCL send/recv + unpack of "
+                    "the output's halo rows; medians of 10 steps, the slowest rank"}
+
+
 def main_ours(args):
     import torch
     import paper_2609_31938_b200 as ccv
@@ -485,29 +664,23 @@ def main_ours(args):
     launches0 = layer.counters()["kernel_launches"]
     ccv.ccv3d_profile_enable(layer.h, True)
 
-    sampler = ClockSampler(local)
+    # ---- the timed region: exactly K steps between two events, a barrier + synchronize on both sides; one more
+    # event after every step gives the per-step times
+    sampler = ClockSampler(local, period_s=0.002)
     sampler.start()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    evs = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     barrier()
-    e0.record(stream)
-    for _ in range(args.steps):
+    evs[0].record(stream)
+    for i in range(args.steps):
         step()
-    e1.record(stream)
+        evs[i + 1].record(stream)
     barrier()
-    ms_total = e0.elapsed_time(e1)
-    clocks = sampler.summary()
-    clock_note = "sampled during the timed region"
-    if clocks["samples"] < 5:
-        # the timed region was shorter than a few NVML polls: keep polling over an untimed repeat of the same step
-        t_end = time.time() + 1.0
-        while time.time() < t_end:
-            for _ in range(20):
-                step()
-            torch.cuda.synchronize()
-        clock_note = "timed region too short for NVML polling; sampled over an untimed 1 s repeat of the same step"
     sampler.stop()
+    ms_total = evs[0].elapsed_time(evs[args.steps])
+    per_step = [evs[i].elapsed_time(evs[i + 1]) for i in range(args.steps)]
     clocks = sampler.summary()
-    clocks["note"] = clock_note
+    clocks["note"] = "NVML, sampled every 2 ms during the timed region" + (
+        " (a short region: the `sustained` leg has the long record)" if clocks["samples"] < 20 else "")
 
     st, stage_ms, conv_ms, ncalls = ccv.ccv3d_profile_read(layer.h)
     ccv.ccv3d_profile_enable(layer.h, False)
@@ -520,6 +693,33 @@ def main_ours(args):
     abytes = si.conv_bytes(**d)
     ms_step = ms_total / args.steps
     value = weak_scaling_value(world, flops, ms_step)
+    peaks = measured_peaks()
+
+    # ---- sustained: at least two seconds of back-to-back steps whatever --steps says (the part settles under its
+    # power cap within the first few hundred milliseconds), per-step times from events, clocks sampled throughout
+    sus_sampler = ClockSampler(local, period_s=0.004)
+    sus_ms = []
+    barrier()
+    sus_sampler.start()
+    t_begin = time.perf_counter()
+    while time.perf_counter() - t_begin < args.sustain_s or len(sus_ms) < 100:
+        sus_ms += timed_calls(step, 200, warmup=0)
+    sus_sampler.stop()
+    barrier()
+    assert layer.device_status()[0] == ccv.OK
+    sus_clk = sus_sampler.summary()
+    tail = np.asarray(sus_ms[len(sus_ms) // 4:])               # the first quarter is the ramp into the capped state
+    sus_med = max_over_ranks(float(np.median(tail)), dist, dev)
+    sustained = {"seconds": float(np.sum(sus_ms)) / 1e3, "samples": int(tail.size), "ms_per_step_median": sus_med,
+                 "ms_per_step_min": float(tail.min()), "ms_per_step_mean": float(tail.mean()),
+                 "tflops": world * flops / (sus_med * 1e-3) / 1e12,
+                 "frac_of_sustained_peak": (flops / (sus_med * 1e-3) / 1e12) / peaks["tflops_sustained"] if peaks["tflops_sustained"] else None,
+                 "frac_of_burst_peak": (flops / (sus_med * 1e-3) / 1e12) / peaks["tflops"],
+                 "frac_of_nominal_2250": (flops / (sus_med * 1e-3) / 1e12) / NOMINAL_BF16_TFLOPS,
+                 "sm_mhz_median": sus_clk["sm_mhz"], "clock_samples": sus_clk["samples"], "reasons": sus_clk["reasons"],
+                 "ms_times_mhz": (sus_med * sus_clk["sm_mhz"]) if sus_clk["sm_mhz"] else None,
+                 "note": "back-to-back ccv3d_forward calls; statistics over the last three quarters of the per-step "
+                         "event times; the sustained peak is the measured seconds-long cuBLAS bf16 figure"}
 
     # ---- end to end through the host entry point: pinned host buffers, H2D and D2H inside the timed region
     e2e = None
@@ -550,9 +750,8 @@ def main_ours(args):
                "d2h_bytes_per_step": int(d2h), "ms_per_step": e_ms, "steps": e_steps,
                "note": "ccv3d_forward_host: pinned host x, cache -> device, the layer, out, new_cache -> host; frame by frame "
                        "on three streams (upload, compute on a frame ring, download overlap): bound by PCIe, whose two "
-                       "directions together moved 70 GB/s here"}
+                       f"directions together moved {(h2d + d2h) / (e_ms * 1e6):.0f} GB/s here"}
         assert np.array_equal(ho.numpy().view(np.uint16), out.view(torch.int16).cpu().numpy().view(np.uint16))
-        e2e["note"] = e2e["note"].replace("70 GB/s", f"{(h2d + d2h) / (e_ms * 1e6):.0f} GB/s")
         # the streaming form of the same call: the history stays in a frame ring on the device, so a step moves only
         # x up and out down (the steady state of a streamed decode; same arithmetic per step)
         def stream_step(reset=False):
@@ -572,29 +771,35 @@ def main_ours(args):
                          "h2d_bytes_per_step": int(hx.numel() * 2), "d2h_bytes_per_step": int(ho.numel() * 2),
                          "note": "ccv3d_forward_host_stream: the temporal history stays on the device between calls; "
                                  "x up, out down"}
+        del hx, hc, ho, hn
+
+    hsplit_x = None
+    if dist is not None and world >= 2 and not args.no_chain:
+        try:
+            hsplit_x = hsplit_exchange_leg(dev, dist, world, rank)
+        except Exception as e:                                # a secondary leg must not take the line down
+            hsplit_x = {"error": f"{type(e).__name__}: {e}"}
 
     if rank != 0:
         if dist is not None:
             dist.destroy_process_group()
         return 0
 
-    peaks = measured_peaks()
     conv_avg_ms = conv_ms / max(ncalls, 1)
     stage_avg_ms = stage_ms / max(ncalls, 1)
+    variant = "one_kernel" if stage_avg_ms < 0.02 else "two_kernels"
     achieved = flops / (conv_avg_ms * 1e-3) / 1e12 if conv_avg_ms > 0 else None
     roof_t_ms = 1e3 * max(flops / (peaks["tflops"] * 1e12), abytes / (peaks["hbm_gbs"] * 1e9))
     roofline = {"bound": "tensor", "kernel": "conv3d_tcgen05_kernel", "achieved": achieved, "peak": peaks["tflops"],
                 "unit": "TFLOP/s", "frac": (achieved / peaks["tflops"]) if achieved else None,
-                "peak_source": f"{peaks['source']} (burst cuBLAS bf16)", "traffic": TRAFFIC_BYTES_PER_LAUNCH.get(name),
+                "frac_of_nominal_2250": (achieved / NOMINAL_BF16_TFLOPS) if achieved else None,
+                "peak_source": f"{peaks['source']} (burst cuBLAS bf16: the timed region is a burst of {ms_total:.0f} ms)",
+                "kernel_variant": variant, "traffic": TRAFFIC_BYTES_PER_LAUNCH.get((name, variant)),
                 "kernel_ms": conv_avg_ms,
-                "schedule": "one kernel: staging + cache update + convolution" if stage_avg_ms < 0.02 else
+                "schedule": "one kernel: staging + cache update + convolution" if variant == "one_kernel" else
                             "two kernels: staging + cache update, then convolution",
-                "staging_kernel_ms": stage_avg_ms if stage_avg_ms >= 0.02 else None,
-                "staging_kernel_gbs": (abytes - 2 * d["N"] * d["Cout"] * d["T"] * d["H"] * d["W"]
-                                       + 2 * d["N"] * d["Cin"] * (d["T"] + kt - 1) * d["H"] * d["W"]) / (stage_avg_ms * 1e6)
-                if stage_avg_ms >= 0.02 else None,
-                "step_frac_of_roofline": roof_t_ms / ms_step,
-                "step_frac_of_sustained_peak": (value / world) / peaks["tflops_sustained"] if peaks["tflops_sustained"] else None}
+                "staging_kernel_ms": stage_avg_ms if variant == "two_kernels" else None,
+                "step_frac_of_roofline": roof_t_ms / ms_step}
 
     # ---- the same layer on resident activations (frame rings): history in place, no staging copy, no cache
     # update, output written channels-last for a following layer.  The streamed steady state: x advances by T
@@ -606,42 +811,42 @@ def main_ours(args):
         rout = ccv.FrameRing(d["N"], d["Cout"], d["T"], d["H"], d["W"])
         rin.load(0, cache)
         rin.load(kt - 1, x)
-        r_steps = max(1, args.steps)
-        slot = kt - 1
-        for _ in range(3):
-            layer.forward_ring(rin, slot, kt - 1, d["T"], out_ring=rout)
-            slot = (slot + d["T"]) % F
-        torch.cuda.synchronize()
-        e0.record(stream)
-        for _ in range(r_steps):
-            layer.forward_ring(rin, slot, kt - 1, d["T"], out_ring=rout)
-            slot = (slot + d["T"]) % F
-        e1.record(stream)
-        torch.cuda.synchronize()
-        r_ms = e0.elapsed_time(e1) / r_steps
+        slot = [kt - 1]
+
+        def ring_step():
+            layer.forward_ring(rin, slot[0], kt - 1, d["T"], out_ring=rout)
+            slot[0] = (slot[0] + d["T"]) % F
+
+        time.sleep(0.5)
+        rst = stats(timed_calls(ring_step, max(20, args.steps)))
+        r_ms = rst["ms_median"]
         assert layer.device_status()[0] == ccv.OK
         r_bytes = 2 * d["N"] * d["H"] * d["W"] * d["T"] * (d["Cin"] + d["Cout"]) + c["w"].nbytes
-        resident = {"value": flops / (r_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": r_ms, "steps": r_steps,
+        resident = {"value": flops / (r_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "ms_per_step": r_ms, **rst,
                     "frac_of_measured_bf16_peak": flops / (r_ms * 1e-3) / 1e12 / peaks["tflops"],
+                    "frac_of_nominal_2250": flops / (r_ms * 1e-3) / 1e12 / NOMINAL_BF16_TFLOPS,
                     "algorithmic_bytes_per_step": int(r_bytes), "gpu_launches_per_step": 1,
-                    "traffic": TRAFFIC_BYTES_PER_LAUNCH_RESIDENT.get(name),
+                    "traffic": TRAFFIC_BYTES_PER_LAUNCH.get((name, "ring")),
                     "note": "ccv3d_forward_ring: input and output in frame rings (channels-last blocks), temporal "
                             "history left in the ring by the previous call"}
         del rin, rout
 
     cpu = cpu_baseline(name) if world == 1 else None
     chain = chain_leg(dev) if (world == 1 and not args.no_chain) else None
-    others = other_configs_leg(dev) if (world == 1 and not args.no_chain) else None
+    others = other_configs_leg(dev, local) if (world == 1 and not args.no_chain) else None
     hsplit = hsplit_leg(dev) if (world == 1 and not args.no_chain) else None
+    a = np.asarray(per_step)
     line = {"metric": METRIC, "value": value, "unit": "TFLOP/s", "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "ms_per_step_median": float(np.median(a)),
+            "ms_per_step_min": float(a.min()), "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": name, **{k: (list(v) if isinstance(v, tuple) else v) for k, v in d.items()},
                        "cache_frames": kt - 1, "accumulate": "fp32", "l2": "inputs larger than L2 (x alone is "
                        f"{c['x'].nbytes / 1e6:.0f} MB); no flush", "parallelism": f"replicas x{world}",
                        "algorithmic_bytes_per_step": int(abytes), "flops_per_step": flops,
-                       "pct_of_measured_bf16_peak": 100.0 * (value / world) / peaks["tflops"]},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline}
+                       "pct_of_measured_bf16_peak": 100.0 * (value / world) / peaks["tflops"],
+                       "pct_of_nominal_bf16_peak": 100.0 * (value / world) / NOMINAL_BF16_TFLOPS},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": int(launches), "roofline": roofline, "sustained": sustained}
     if cpu is not None:
         line["cpu_baseline"] = cpu
     if resident is not None:
@@ -652,11 +857,27 @@ def main_ours(args):
         line["other_configs"] = others
     if hsplit is not None:
         line["height_split"] = hsplit
+    if hsplit_x is not None:
+        line["height_split_exchange"] = hsplit_x
     print(json.dumps(line))
     if dist is not None:
         dist.destroy_process_group()
     layer.close()
     return 0
+
+
+def spawn_ranks(n):
+    """`--gpus N` without torchrun: start N ranks of this script (one per GPU) on 127.0.0.1 and wait for them.
+    NCCL's start-up log is left on (stderr of the ranks) so that the number of ranks can be read off it."""
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}", "--master-addr", "127.0.0.1",
+           "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    env = dict(os.environ)
+    env.setdefault("NCCL_DEBUG", "INFO")
+    env.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+    return subprocess.call(cmd, env=env)
 
 
 def main():
@@ -665,11 +886,14 @@ def main():
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--no-chain", action="store_true", help="skip the decoder-chain leg")
+    ap.add_argument("--no-chain", action="store_true", help="skip the secondary legs (decoder chain, other configurations, height-split)")
+    ap.add_argument("--sustain-s", type=float, default=2.0, help="seconds of back-to-back steps in the sustained leg")
     ap.add_argument("--selftest-dist", action="store_true", help=argparse.SUPPRESS)
     ap.add_argument("--flags", type=int, default=0, help="CCV3D_FLAG_* bits for the layer (e.g. 8 = fused route without staging copy)")
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=sorted(n for n in si.CONFIGS if "bf16" in n))
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        return spawn_ranks(args.gpus)
     if args.selftest_dist:
         return main_selftest_dist(args)
     if args.impl == "reference":

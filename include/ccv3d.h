@@ -40,7 +40,8 @@ typedef enum { CCV3D_F32 = 0, CCV3D_BF16 = 1 } ccv3d_dtype;
 typedef enum {
     CCV3D_OK = 0,
     CCV3D_ERR_INVALID_ARG = 1,    /* NULL pointer, non-positive size, bad enum */
-    CCV3D_ERR_UNSUPPORTED = 2,    /* stride/dilation/groups != 1, even kernel, pad != (k-1)/2, ... (Algorithm 1's reject list) */
+    CCV3D_ERR_UNSUPPORTED = 2,    /* groups != 1 (Algorithm 1's reject list), extents beyond the limits stated at ccv3d_desc, a
+                                     temporal padding that is not the causal one, or an entry point that does not take this layer */
     CCV3D_ERR_ALIGNMENT = 3,      /* a tensor pointer is not 16-byte aligned */
     CCV3D_ERR_ALIAS = 4,          /* out or new_cache overlaps an input (or each other) */
     CCV3D_ERR_ARCH = 5,           /* current device is not compute capability 10.x */
@@ -58,7 +59,7 @@ typedef enum {
                                             by TMA and transposes in shared memory (needs W % 8 == 0, else the staged route is taken). Some 10 % slower
                                             than the default route; for callers that cannot afford the workspace. */
 #define CCV3D_FLAG_F32_TENSOR 0x20u       /* FP32 layers: always use the tensor cores (3xTF32: each FP32 product as hi*hi + hi*lo + lo*hi of TF32
-                                            operands, FP32 accumulate); the default sends layers with K = cin*kt*kh*kw > 16384, and calls that are
+                                            operands, FP32 accumulate); the default sends layers with K = cin*kt*kh*kw > 8192, and calls that are
                                             both under 0.2 GFLOP and of K < 256, to the FP32-FMA kernel */
 #define CCV3D_FLAG_NO_PAIR 0x40u          /* tensor-core route: never run tiles on pairs of CTAs (cta_group::2 MMAs with M = 256, each SM
                                             streaming half of every weight tile) - the default for layers with more than 128 output
@@ -82,7 +83,8 @@ typedef enum {
  * Layers with unit strides and dilations, odd kh and kw and size-preserving padding (pad = (k-1)/2) are the
  * "standard" geometry of the header comment; only they can use the cooperative-staging, fused, 1x1x1-streaming,
  * allocation-free and frame-ring paths.  Other geometries run on the tensor-core kernel's run-time tap path
- * (spatial stride > 1: one strided TMA box per tap) or, for FP32 layers, on the FP32-FMA kernel. */
+ * (spatial stride > 1: one strided TMA box per tap) - BF16 layers always, FP32 layers as 3xTF32 under the rule stated
+ * at CCV3D_FLAG_F32_TENSOR, else on the FP32-FMA kernel. */
 typedef struct {
     int32_t cin, cout;            /* channels */
     int32_t kt, kh, kw;           /* kernel extent; 1 <= kt <= 8, 1 <= kh,kw <= 7 */
@@ -102,8 +104,10 @@ typedef struct {
 typedef struct {
     uint64_t calls;           /* ccv3d_forward* calls */
     uint64_t ok;              /* calls that enqueued all their work */
-    uint64_t tcgen05_bf16;    /* calls served by the tensor-core kernel */
-    uint64_t simt;            /* calls served by the FP32-FMA kernel */
+    uint64_t tcgen05_bf16;    /* calls served by the BF16 tensor-core convolution kernel (NCTHW, host and frame-ring entry points) */
+    uint64_t tcgen05_f32;     /* FP32 calls served by the tensor-core kernel as 3xTF32 */
+    uint64_t pointwise;       /* 1x1x1 calls served by the streaming kernel that reads NCTHW directly */
+    uint64_t simt;            /* calls served by the FP32-FMA kernel (FP32 layers, and BF16 layers on request) */
     uint64_t unsupported;     /* rejected: unsupported */
     uint64_t invalid;         /* rejected: invalid argument / alignment / alias */
     uint64_t cuda_error;      /* failed in a CUDA call */
@@ -154,9 +158,10 @@ ccv3d_status ccv3d_create(ccv3d_handle** out_h, const ccv3d_desc* d, const void*
  * everything enqueued on it so far and join it before the call returns, so the caller only ever needs to order
  * against `stream`.
  * The tensor-core path keeps a channels-last staging copy of [cache ; x] in a
- * workspace owned by the handle; it is (re)allocated when a call needs more than
- * the handle holds (that call synchronises the device), so steady-state calls of
- * one shape allocate nothing.  ccv3d_workspace_bytes tells the size in advance.
+ * workspace: the caller's when one was lent with ccv3d_set_workspace (then no call
+ * ever allocates), else one owned by the handle, (re)allocated when a call needs
+ * more than the handle holds (that call synchronises the device), so steady-state
+ * calls of one shape allocate nothing.  ccv3d_workspace_bytes tells the size in advance.
  */
 ccv3d_status ccv3d_forward(ccv3d_handle* h, const void* x, const void* cache, void* out, void* new_cache,
                            int32_t N, int32_t T, int32_t H, int32_t W, void* stream);
@@ -191,8 +196,10 @@ ccv3d_status ccv3d_forward_ex(ccv3d_handle* h, const void* x, const void* cache,
  * pointers owned by the caller).  Differences:
  *   - BF16 tensor-core layers only (a handle created with CCV3D_FLAG_FORCE_SIMT or with FP32 data, and the
  *     CCV3D_FLAG_TC_PER_TAP_A mode, return CCV3D_ERR_UNSUPPORTED);
- *   - the staging copy, ccv3d_workspace_bytes(h, N, T, H, W), must fit the 32 MiB array, otherwise the call
- *     returns CCV3D_ERR_UNSUPPORTED and launches nothing;
+ *   - the staging copy must fit the 32 MiB array, otherwise the call returns CCV3D_ERR_UNSUPPORTED and launches
+ *     nothing.  Its size is N * (kt-1+T) * cin_pad * H * W * 2 bytes, cin_pad = cin rounded up to a multiple of 32
+ *     (this entry point always stages, so the bound holds also for the layers for which ccv3d_workspace_bytes
+ *     reports 0 because ccv3d_forward would not stage them: 1x1x1 layers and CCV3D_FLAG_FUSED handles);
  *   - the first call on each device looks up the array's device address (a one-time set-up with that device
  *     current); make that first call outside any stream capture;
  *   - all handles and all calls on one GPU share the one array.  Calls that may overlap on the GPU (different
@@ -230,10 +237,25 @@ ccv3d_status ccv3d_forward_host(ccv3d_handle* h, const void* x_host, const void*
 ccv3d_status ccv3d_forward_host_stream(ccv3d_handle* h, const void* x_host, void* out_host, int32_t reset, int32_t N,
                                        int32_t T, int32_t H, int32_t W, void* stream);
 
-/* Bytes of handle-owned workspace a forward call of this shape needs (0 for the FP32-FMA route, the 1x1x1
- * streaming kernel and the fused route). */
+/* Bytes of workspace a ccv3d_forward / ccv3d_forward_ex call of this shape needs (0 for the FP32-FMA route, the
+ * 1x1x1 streaming kernel and the fused route). */
 ccv3d_status ccv3d_workspace_bytes(const ccv3d_handle* h, int32_t N, int32_t T, int32_t H, int32_t W,
                                    uint64_t* bytes_host);
+
+/*
+ * Lend the handle a workspace (the lowering's extra memory - Section 7.2 of the paper lists its temporaries as
+ * the overhead that is left - made the caller's to place).  From now on ccv3d_forward / ccv3d_forward_ex keep the
+ * staging copy in ws_dev (DEVICE, 256-byte aligned, `bytes` long, owned by the caller, who keeps it alive while
+ * the handle may use it) and never allocate, free or synchronise: a call that needs more than `bytes` returns
+ * CCV3D_ERR_NOMEM before it launches anything.  Such calls are legal inside a stream capture.
+ * Several handles may be lent the same buffer - a decoder of many layers needs one workspace of the largest
+ * single need (the maximum of ccv3d_workspace_bytes over its calls), not one per layer: the buffer only holds
+ * data between the kernels of one call.  Calls that share a workspace must be ordered on the GPU (same stream,
+ * or events); calls that may overlap race on it.  ws_dev = NULL or bytes = 0 returns the handle to a workspace
+ * of its own, allocated on demand.  CCV3D_ERR_ALIGNMENT for a misaligned pointer.  The host entry points and
+ * ccv3d_forward_static do not use this workspace.
+ */
+ccv3d_status ccv3d_set_workspace(ccv3d_handle* h, void* ws_dev, uint64_t bytes);
 
 /* Destroy a handle and free what it owns.  NULL is accepted. */
 ccv3d_status ccv3d_destroy(ccv3d_handle* h);

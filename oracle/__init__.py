@@ -2,15 +2,14 @@
 
 Only the tests, the smoke check and the benchmark's CPU-baseline leg may import
 this package; the product never does.  It wraps ``ccv3d_oracle.c`` (the plain
-fp64 definition, Section 4.1-4.2, Eq. (1)-(2)) through ctypes, and adds two
-structurally different restatements used to pin it:
+fp64 definition, Section 4.1-4.2, Eq. (1)-(2)) through ctypes, and adds
+restatements of different structure used to pin it:
 
   * ``brute_force``       - materialises the zero-padded Z volume and loops
                             output-outermost in pure Python/numpy (tiny shapes);
-  * ``algorithm1_route``  - the paper's Algorithm 1 taken step by step: per
-                            temporal tap the valid output interval of Eq. (4),
-                            one 2-D correlation per tap folded over the
-                            interval, accumulation, bias once.
+  * ``tap_intervals``     - the interval algebra of Eq. (4) alone (which output
+                            frames a temporal tap reaches, and from where), held
+                            against direct enumeration of Eq. (1) in the tests.
 
 ``forward_general`` / ``brute_force_general`` are the operator with the layer's own
 spatial stride, padding, dilation and a temporal dilation (Eq. (1)-(2) as printed).
@@ -258,51 +257,3 @@ def tap_intervals(kt: int, cache_frames: int, T: int, dil_t: int = 1):
         o_h = min(T_o, zlen - delta)
         taps.append((k, o_l, o_h, o_l + delta, o_h + delta))
     return T_o, taps
-
-
-def _corr2d_same(img, ker):
-    """Zero-padded 'same' 2-D cross-correlation of one plane with one odd-sized kernel."""
-    H, W = img.shape
-    kh, kw = ker.shape
-    ph, pw = (kh - 1) // 2, (kw - 1) // 2
-    pad = np.zeros((H + 2 * ph, W + 2 * pw))
-    pad[ph:ph + H, pw:pw + W] = img
-    res = np.zeros((H, W))
-    for dh in range(kh):
-        for dw in range(kw):
-            res += ker[dh, dw] * pad[dh:dh + H, dw:dw + W]
-    return res
-
-
-def algorithm1_route(x, cache, w, b):
-    """Algorithm 1, literally: Z = [C;X] if cached else X; for each temporal tap the
-    interval of Eq. (4); skip empty taps; fold the source interval into the batch; one
-    2-D correlation with W_k; accumulate into A[:, o_l:o_h]; add the bias once."""
-    xd, cd, wd, bd = _widen(x), _widen(cache), _widen(w), _widen(b)
-    N, Cin, T, H, W = xd.shape
-    Cout, _, kt, kh, kw = wd.shape
-    if cd is not None and kt > 1:
-        Z, nC = np.concatenate([cd, xd], axis=2), kt - 1
-    else:
-        Z, nC = xd, 0
-    T_o, taps = tap_intervals(kt, nC, T)
-    assert T_o == T
-    A = None
-    for (k, o_l, o_h, z_l, z_h) in taps:
-        if o_l >= o_h:
-            continue
-        Wk = wd[:, :, k]                                   # [Cout, Cin, kh, kw]
-        U2 = Z[:, :, z_l:z_h].transpose(0, 2, 1, 3, 4).reshape(N * (z_h - z_l), Cin, H, W)   # fold time into batch
-        R2 = np.zeros((U2.shape[0], Cout, H, W))
-        for bi in range(U2.shape[0]):
-            for co in range(Cout):
-                for ci in range(Cin):
-                    R2[bi, co] += _corr2d_same(U2[bi, ci], Wk[co, ci])
-        R = R2.reshape(N, z_h - z_l, Cout, H, W)           # unfold
-        if A is None:
-            A = np.zeros((N, T_o, Cout, H, W))
-        A[:, o_l:o_h] += R
-    assert A is not None
-    if bd is not None:
-        A = A + bd[None, None, :, None, None]
-    return np.ascontiguousarray(A.transpose(0, 2, 1, 3, 4))  # restore [N,Cout,T,H,W]

@@ -23,8 +23,9 @@
  * The cache update is a bit copy.
  *
  * Parity pins (tests/test_oracle_*.py): hand-computed examples under
- * tests/golden/, a structurally different brute-force routine, a literal
- * per-tap Algorithm-1 route, the fp64 library conv3d on the explicitly
+ * tests/golden/, a structurally different brute-force routine, Eq. (2) read
+ * frame by frame (one library 2-D correlation per output frame and temporal
+ * tap at the source time of Eq. (1)), the fp64 library conv3d on the explicitly
  * concatenated input, and the invariants (causality, streaming equivalence,
  * linearity, 1x1x1 = per-pixel matmul, delta kernel).
  * Parity unpinned: behaviour on NaN/Inf/subnormal inputs.

@@ -40,7 +40,7 @@ class Desc(ctypes.Structure):
 
 
 class Counters(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_uint64) for n in ("calls", "ok", "tcgen05_bf16", "simt", "unsupported", "invalid",
+    _fields_ = [(n, ctypes.c_uint64) for n in ("calls", "ok", "tcgen05_bf16", "tcgen05_f32", "pointwise", "simt", "unsupported", "invalid",
                                                "cuda_error", "device_timeout", "kernel_launches")]
 
 
@@ -55,7 +55,7 @@ EXPORTS = ("ccv3d_create", "ccv3d_forward", "ccv3d_forward_host", "ccv3d_workspa
            "ccv3d_upsample_bf16", "ccv3d_profile_enable", "ccv3d_profile_read", "ccv3d_forward_static", "ccv3d_selftest_wait_timeout", "ccv3d_forward_ex",
            "ccv3d_ring_kb", "ccv3d_ring_bytes", "ccv3d_ring_load", "ccv3d_ring_store", "ccv3d_upsample_ring",
            "ccv3d_forward_ring", "ccv3d_out_dims", "ccv3d_forward_ring_up", "ccv3d_rows_copy",
-           "ccv3d_forward_host_stream")
+           "ccv3d_forward_host_stream", "ccv3d_set_workspace")
 
 
 def _load() -> ctypes.CDLL:
@@ -72,6 +72,7 @@ def _load() -> ctypes.CDLL:
     lib.ccv3d_forward_host.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, vp]
     lib.ccv3d_forward_host_stream.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp]
     lib.ccv3d_workspace_bytes.argtypes = [vp, i32, i32, i32, i32, u64p]
+    lib.ccv3d_set_workspace.argtypes = [vp, vp, ctypes.c_uint64]
     lib.ccv3d_destroy.argtypes = [vp]
     lib.ccv3d_get_counters.argtypes = [vp, ctypes.POINTER(Counters)]
     lib.ccv3d_device_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
@@ -171,6 +172,11 @@ def ccv3d_workspace_bytes(h, N, T, H, W):
     b = ctypes.c_uint64()
     s = lib.ccv3d_workspace_bytes(h, N, T, H, W, ctypes.byref(b))
     return s, b.value
+
+
+def ccv3d_set_workspace(h, ws_dev, nbytes) -> int:
+    """Lend the handle a caller-owned staging workspace (DEVICE address, 256-byte aligned); None/0 takes it back."""
+    return lib.ccv3d_set_workspace(h, ws_dev, nbytes)
 
 
 def ccv3d_destroy(h) -> int:

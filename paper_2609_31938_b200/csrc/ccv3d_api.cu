@@ -10,6 +10,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <atomic>
 #include <new>
 
 #include "ccv3d_simt.cuh"
@@ -58,8 +59,11 @@ struct ccv3d_handle {
     float* bias32;       // FP32 bias, padded (device)
     unsigned int* status;  // device status word
     unsigned int* band_ctr;  // cooperative staging: per-band arrival counters (MAX_COOP_BANDS words, device)
-    void* workspace;
+    void* workspace;     // staging copy owned by the handle (allocated on demand) ...
     uint64_t workspace_bytes;
+    void* ext_ws;        // ... or lent by the caller (ccv3d_set_workspace): then nothing is ever allocated by a forward call
+    uint64_t ext_ws_bytes;
+    void* ws_cur;        // the one the call in progress uses
     // host-entry staging (device buffers)
     void* hx; void* hc; void* ho; void* hn;
     uint64_t hx_b, hc_b, ho_b, hn_b;
@@ -170,12 +174,15 @@ bool on_handle_device(const ccv3d_handle* h) {
 // FP32 layers: the FP32-FMA kernel is exact FP32 and fine for small calls; from 0.2 GFLOP on (or when the layer
 // asks for it) the call goes to the tensor cores as 3xTF32.  The tensor core's accumulation truncates: measured
 // against the FP64 definition the worst element is off by about 4.5e-9 x K x RMS(out) (K = cin*kt*kh*kw; 2.5e-5 at
-// K = 5184, 4.7e-5 at K = 10368), so layers with K > 16384 stay on the FP32-FMA kernel unless the flag insists.
+// K = 5184, 4.7e-5 at K = 10368) and the error depends on the data (inputs of one sign keep the accumulator at full
+// size along the whole chain), so the automatic route stops at K = 8192 - a third of the 1e-4 tolerance by that model -
+// and longer layers stay on the FP32-FMA kernel unless the flag insists.
+constexpr int64_t F32_TENSOR_MAX_K = 8192;
 bool f32_takes_tensor_cores(const ccv3d_handle* h, int N, int T, int H, int W) {
     const ccv3d_desc& d = h->d;
     if (d.flags & CCV3D_FLAG_F32_TENSOR) return true;
     const int64_t K = (int64_t)d.cin * d.kt * d.kh * d.kw;
-    if (K > 16384) return false;
+    if (K > F32_TENSOR_MAX_K) return false;
     // Large calls for the throughput; small ones whenever the FMA kernel's serial walk over K (one thread per output
     // element, ~0.2 us per tap row) would outlast the two short launches of this route (~20 us together):
     // configuration 1 (K = 432) runs 21 us here against 80 us there.
@@ -369,6 +376,19 @@ ccv3d_status ccv3d_workspace_bytes(const ccv3d_handle* h, int32_t N, int32_t T, 
     const bool scratch_free = (h->use_tc32 ? !f32_takes_tensor_cores(h, N, T, H, W) : !h->use_tc) ||
                               (h->use_tc && (pointwise_eligible(h, T, H, W) || fused_eligible(h, W)));
     *bytes_host = scratch_free ? 0 : tc_workspace_bytes(h, N, T, H, W);
+    return CCV3D_OK;
+}
+
+ccv3d_status ccv3d_set_workspace(ccv3d_handle* h, void* ws_dev, uint64_t bytes) {
+    if (!h) return CCV3D_ERR_INVALID_ARG;
+    if (!ws_dev || bytes == 0) {                            // back to a workspace the handle allocates on demand
+        h->ext_ws = nullptr;
+        h->ext_ws_bytes = 0;
+        return CCV3D_OK;
+    }
+    if ((uintptr_t)ws_dev & 255u) return CCV3D_ERR_ALIGNMENT;
+    h->ext_ws = ws_dev;
+    h->ext_ws_bytes = bytes;
     return CCV3D_OK;
 }
 

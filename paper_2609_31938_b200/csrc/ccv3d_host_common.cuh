@@ -127,10 +127,11 @@ void begin_call(ccv3d_handle* h, const char* name, int N, int T, int H, int W) {
 // ... and ends here: the status is counted (Algorithm 1's route counters) and, with CCV3D_LOG=1, reported.
 ccv3d_status count(ccv3d_handle* h, ccv3d_status s) {
     if (h->log)
-        fprintf(stderr, "ccv3d %p %s N=%d T=%d H=%d W=%d %d->%d k=%dx%dx%d: %s (calls %llu tcgen05 %llu fma %llu launches %llu)\n",
+        fprintf(stderr, "ccv3d %p %s N=%d T=%d H=%d W=%d %d->%d k=%dx%dx%d: %s (calls %llu tcgen05 %llu 3xtf32 %llu 1x1x1 %llu fma %llu launches %llu)\n",
                 (void*)h, h->call_name ? h->call_name : "?", h->call_dims[0], h->call_dims[1], h->call_dims[2], h->call_dims[3],
                 h->d.cin, h->d.cout, h->d.kt, h->d.kh, h->d.kw, ccv3d_status_string(s), (unsigned long long)h->ctr.calls,
-                (unsigned long long)(h->ctr.tcgen05_bf16), (unsigned long long)h->ctr.simt,
+                (unsigned long long)h->ctr.tcgen05_bf16, (unsigned long long)h->ctr.tcgen05_f32,
+                (unsigned long long)h->ctr.pointwise, (unsigned long long)h->ctr.simt,
                 (unsigned long long)h->ctr.kernel_launches);
     switch (s) {
         case CCV3D_OK: h->ctr.ok++; break;
@@ -178,7 +179,7 @@ ccv3d_status encode_act_map(ccv3d_handle* h, int N, int T, int H, int W, int BW,
     cuuint32_t box[5] = {(cuuint32_t)inner, (cuuint32_t)(BW * es_w), (cuuint32_t)(BH * es_h), 1, 1};
     cuuint32_t es[5] = {1, (cuuint32_t)es_w, (cuuint32_t)es_h, 1, 1};
     if (box[1] > 256 || box[2] > 256) return CCV3D_ERR_UNSUPPORTED;
-    CUresult r = h->encode(&h->tm_a, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, h->workspace, dims, strides, box, es,
+    CUresult r = h->encode(&h->tm_a, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, h->ws_cur, dims, strides, box, es,
                            CU_TENSOR_MAP_INTERLEAVE_NONE,
                            pl.KB == 64 ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B,
                            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);

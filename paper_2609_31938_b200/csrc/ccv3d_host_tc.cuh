@@ -213,8 +213,17 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     const bool strided = d.stride[1] > 1 || d.stride[2] > 1;
     const bool f32 = d.dtype == CCV3D_F32;                 // 3xTF32: FP32 staging with the hi/lo split, TF32 MMAs
 
-    ccv3d_status s = grow(&h->workspace, &h->workspace_bytes, tc_workspace_bytes(h, N, T, H, W));
-    if (s != CCV3D_OK) return s;
+    // the staging copy: in the caller's workspace when one was lent (never allocates; too small = an error before
+    // any launch), else in the handle's own, which grows on demand
+    ccv3d_status s = CCV3D_OK;
+    if (h->ext_ws) {
+        if (tc_workspace_bytes(h, N, T, H, W) > h->ext_ws_bytes) return CCV3D_ERR_NOMEM;
+        h->ws_cur = h->ext_ws;
+    } else {
+        s = grow(&h->workspace, &h->workspace_bytes, tc_workspace_bytes(h, N, T, H, W));
+        if (s != CCV3D_OK) return s;
+        h->ws_cur = h->workspace;
+    }
 
     // ---- staging: [cache ; x] channels-last, cache update in the same pass ----
     StageParams sp;
@@ -223,7 +232,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     const int cf = (tc && cache) ? h->call_cf : 0;          // older history frames are absent: their taps are skipped
     sp.cache = cf ? (const __nv_bfloat16*)cache : nullptr;
     sp.cf = cf;
-    sp.zs = (__nv_bfloat16*)h->workspace;
+    sp.zs = (__nv_bfloat16*)h->ws_cur;
     sp.new_cache = tc ? (__nv_bfloat16*)new_cache : nullptr;
     sp.N = N; sp.Cin = d.cin; sp.T = T; sp.H = H; sp.W = W; sp.tc = tc; sp.CB = pl.CB;
     sp.f_begin = (tc - cf) < T ? (tc - cf) : T;
@@ -253,7 +262,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     const int TWT = pair ? 2 * TW : TW;                    // tile width in the tile index space
     const int BW = per_tap ? TW : TW + (d.kw - 1) * d.dilation[2];
     const int BH = per_tap ? 16 : 16 + (d.kh - 1) * d.dilation[1];
-    ShapeKey key{h->workspace, N, T, H, W, BW};
+    ShapeKey key{h->ws_cur, N, T, H, W, BW};
     if (!(key == h->tm_a_key)) {
         s = encode_act_map(h, N, T, H, W, BW, BH, per_tap ? d.stride[2] : 1, per_tap ? d.stride[1] : 1);
         if (s != CCV3D_OK) return s;
@@ -365,7 +374,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
         if (f32) {
             StageF32Params sf;
             sf.x = (const float*)x; sf.cache = cf ? (const float*)cache : nullptr; sf.cf = cf;
-            sf.zs = (float*)h->workspace; sf.new_cache = tc ? (float*)new_cache : nullptr;
+            sf.zs = (float*)h->ws_cur; sf.new_cache = tc ? (float*)new_cache : nullptr;
             sf.N = N; sf.Cin = d.cin; sf.T = T; sf.H = H; sf.W = W; sf.tc = tc; sf.CBr = pl.CB; sf.f_begin = sp.f_begin;
             dim3 sgrid((W + 31) / 32, H, (unsigned)((int64_t)N * nframes * sf.CBr));
             if (H > 65535 || (int64_t)N * nframes * sf.CBr > 65535) return CCV3D_ERR_UNSUPPORTED;
@@ -427,7 +436,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
             if (cudaStreamWaitEvent(st, h->ev_join[i - 1], 0) != cudaSuccess) return cuda_fail();
         }
     }
-    h->ctr.tcgen05_bf16++;
+    if (f32) h->ctr.tcgen05_f32++; else h->ctr.tcgen05_bf16++;
     if (pev) {
         cudaEventRecord(pev[2], st);
         h->prof_n++;
@@ -645,7 +654,7 @@ ccv3d_status forward_pointwise(ccv3d_handle* h, const void* x, void* out, int N,
         h->prof_n++;
     }
     h->ctr.kernel_launches++;
-    h->ctr.tcgen05_bf16++;
+    h->ctr.pointwise++;
     return CCV3D_OK;
 }
 
@@ -657,7 +666,7 @@ ccv3d_status forward_pointwise(ccv3d_handle* h, const void* x, void* out, int N,
 constexpr uint64_t STATIC_SCRATCH_BYTES = 32ull << 20;   // 32 MiB per GPU that loads the library, until exit
 static __device__ __align__(256) unsigned char g_static_scratch[STATIC_SCRATCH_BYTES];
 constexpr int MAX_DEVICES = 64;
-static void* g_static_scratch_addr[MAX_DEVICES];         // device address of the array, per device; set on first use
+static std::atomic<void*> g_static_scratch_addr[MAX_DEVICES];   // device address of the array, per device; set on first use
 
 // In host code the name g_static_scratch is only a stand-in for the symbol: the address a kernel can use has
 // to be asked for, once per device, with that device current.
@@ -665,12 +674,14 @@ ccv3d_status static_scratch_for_current_device(void** out_ptr) {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess) return cuda_fail();
     if (dev < 0 || dev >= MAX_DEVICES) return CCV3D_ERR_UNSUPPORTED;
-    if (!g_static_scratch_addr[dev]) {
-        void* ptr = nullptr;
+    // Threads of different handles may arrive here together: the table is atomic, and every thread that finds
+    // the entry empty looks the address up itself and stores the same value.
+    void* ptr = g_static_scratch_addr[dev].load(std::memory_order_acquire);
+    if (!ptr) {
         if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return cuda_fail();
-        g_static_scratch_addr[dev] = ptr;
+        g_static_scratch_addr[dev].store(ptr, std::memory_order_release);
     }
-    *out_ptr = g_static_scratch_addr[dev];
+    *out_ptr = ptr;
     return CCV3D_OK;
 }
 

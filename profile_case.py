@@ -1,6 +1,6 @@
 """Run a few forward calls of one layer shape on cuda:0 - a small, self-ending program to put under a profiler.
 
-    python -m paper_2609_31938_b200.profile_case --cin 192 --cout 192 --t 4 --h 176 --w 320 [--k 3 3 3] [--calls 3] [--ring]
+    python profile_case.py --cin 192 --cout 192 --t 4 --h 176 --w 320 [--k 3 3 3] [--calls 3] [--ring]
 
 Inputs are the seeded synthetic tensors of the benchmark (normal activations, fan-in-scaled weights).
 """
@@ -10,7 +10,7 @@ import sys
 
 import numpy as np
 
-sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+sys.path.insert(0, os.path.dirname(os.path.abspath(__file__)))
 
 
 def main():

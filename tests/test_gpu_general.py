@@ -222,7 +222,7 @@ def test_fp32_on_tensor_cores_3xtf32(ccv, N, Cin, Cout, T, H, W, k, cf, stride, 
     within the FP32 tolerance (max <= 1e-4 x RMS) of the oracle, cache update bit-exact."""
     c = _case(N, Cin, Cout, T, H, W, k, si.F32, cf, seed=41)
     m, ctr = run_general(ccv, c, stride, pad, dil, dil_t, flags=ccv.FLAG_F32_TENSOR, stride_t=stride_t)
-    assert ctr["tcgen05_bf16"] == 1 and ctr["simt"] == 0
+    assert ctr["tcgen05_f32"] == 1 and ctr["tcgen05_bf16"] == 0 and ctr["simt"] == 0
     print("3xTF32", (N, Cin, Cout, T, H, W, k), "K =", Cin * k[0] * k[1] * k[2], m)
 
 
@@ -239,7 +239,7 @@ def test_fp32_route_selection_by_size(ccv):
         small, _ = layer(to_dev(c["x"])[:, :, :1, :8, :8].contiguous(), None)    # 2.8 MFLOP, but K = 1728: tensor cores too
         torch.cuda.synchronize()
         ctr = layer.counters()
-        assert (ctr["tcgen05_bf16"], ctr["simt"]) == ((2, 0) if name == "auto" else (0, 2))
+        assert (ctr["tcgen05_f32"], ctr["simt"], ctr["tcgen05_bf16"]) == ((2, 0, 0) if name == "auto" else (0, 2, 0))
         check(as_f64(o), ref, "f32")
         assert np.array_equal(bits(nc), ref_nc)
         outs[name] = as_f64(o)
@@ -252,9 +252,35 @@ def test_fp32_route_selection_by_size(ccv):
     layer = ccv.CausalConv3d(to_dev(c2["w"]), to_dev(c2["b"]))
     o2, _ = layer(to_dev(c2["x"]), to_dev(c2["cache"]))
     torch.cuda.synchronize()
-    assert layer.counters()["simt"] == 1 and layer.counters()["tcgen05_bf16"] == 0
+    assert layer.counters()["simt"] == 1 and layer.counters()["tcgen05_f32"] == 0
     check(as_f64(o2), ref2, "f32")
     layer.close()
+
+
+@pytest.mark.parametrize("dist", ["normal", "uniform", "one_sign"])
+@pytest.mark.parametrize("seed", [0, 1, 2])
+def test_fp32_default_route_just_under_the_k_limit(ccv, dist, seed):
+    """The longest K the automatic FP32 route sends to the tensor cores (K <= 8192; here Cin = 300, 3x3x3: K = 8100)
+    on three kinds of data: normal, uniform, and activations and weights all of one sign - the worst case for an
+    accumulation that truncates, since the accumulator then sits at full size along the whole chain.  Each within
+    the FP32 tolerance of the oracle (max <= 1e-4 x RMS), cache bit-exact; one more channel pair (K = 8208) takes
+    the FMA kernel."""
+    N, Cin, Cout, T, H, W = 1, 300, 16, 2, 12, 16
+    c = _case(N, Cin, Cout, T, H, W, (3, 3, 3), si.F32, 2, seed=80 + seed)
+    if dist == "normal":                                       # (the FP32 cases of this file draw uniform activations)
+        rng = np.random.default_rng(seed)
+        c["x"] = rng.standard_normal(c["x"].shape).astype(np.float32)
+        c["cache"] = rng.standard_normal(c["cache"].shape).astype(np.float32)
+    elif dist == "one_sign":
+        for n in ("x", "cache", "w"):
+            c[n] = np.abs(c[n])
+    m, ctr = run_general(ccv, c, (1, 1), (1, 1), (1, 1), 1)
+    assert ctr["tcgen05_f32"] == 1 and ctr["simt"] == 0
+    print("3xTF32 at K = 8100,", dist, seed, m)
+    if dist == "normal" and seed == 0:
+        c2 = _case(N, 304, Cout, T, H, W, (3, 3, 3), si.F32, 2, seed=90)
+        m2, ctr2 = run_general(ccv, c2, (1, 1), (1, 1), (1, 1), 1)
+        assert ctr2["simt"] == 1 and ctr2["tcgen05_f32"] == 0
 
 
 @pytest.mark.parametrize("Cin,Cout,H,W", [(64, 64, 96, 96), (48, 192, 64, 80)])   # two pixel blocks per CTA; one
@@ -268,7 +294,7 @@ def test_fp32_on_cta_pairs_equals_single_ctas_bitwise(ccv, Cin, Cout, H, W):
         layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), flags=flags)
         o, nc = layer(to_dev(c["x"]), to_dev(c["cache"]))
         torch.cuda.synchronize()
-        assert layer.device_status()[0] == ccv.OK and layer.counters()["tcgen05_bf16"] == 1
+        assert layer.device_status()[0] == ccv.OK and layer.counters()["tcgen05_f32"] == 1
         assert np.array_equal(bits(nc), ref_nc)
         outs.append(o)
         layer.close()

@@ -66,7 +66,7 @@ def test_cfg1_fp32(ccv):
     """Configuration 1 on both FP32 routes: the tensor cores by 3xTF32 (the default: K = 432 is long enough for the
     FMA kernel's serial walk to lose) and the plain FMA kernel, each within the FP32 tolerance, cache bit-exact."""
     m, ctr = run_case(ccv, si.conv_case(**si.CONFIGS["cfg1_f32_16"]))
-    assert ctr["tcgen05_bf16"] == 1 and ctr["simt"] == 0 and m["cos"] > 0.9999999
+    assert ctr["tcgen05_f32"] == 1 and ctr["tcgen05_bf16"] == 0 and ctr["simt"] == 0 and m["cos"] > 0.9999999
     m, ctr = run_case(ccv, si.conv_case(**si.CONFIGS["cfg1_f32_16"]), flags=ccv.FLAG_FORCE_SIMT)
     assert ctr["simt"] == 1 and m["cos"] > 0.9999999
 
@@ -125,7 +125,7 @@ TC_CASES = [
 @pytest.mark.parametrize("N,Cin,Cout,T,H,W,k,cache,bias", TC_CASES)
 def test_bf16_tensor_core_route(ccv, N, Cin, Cout, T, H, W, k, cache, bias):
     m, ctr = run_case(ccv, si.conv_case(N, Cin, Cout, T, H, W, k=k, cache=cache, bias=bias, seed=5))
-    assert ctr["tcgen05_bf16"] == 1 and ctr["simt"] == 0
+    assert ctr["tcgen05_bf16"] + ctr["pointwise"] == 1 and ctr["simt"] == 0   # (1x1x1 layers may take the streaming kernel)
 
 
 @pytest.mark.parametrize("N,Cin,Cout,T,H,W,k,cache,bias", [TC_CASES[0], TC_CASES[4], TC_CASES[6], TC_CASES[11]])

@@ -91,7 +91,7 @@ def test_general_against_numpy_routine_and_library_conv3d(k, stride, pad, dil, d
 
 
 def test_interval_route_with_temporal_dilation_equals_the_definition():
-    """Algorithm 1's accumulation over Eq. (4) intervals, with d_t in the tap offset: per tap one strided, dilated
+    """Eq. (2)'s sum over temporal taps taken tap by tap over Eq. (4)'s intervals, with d_t in the tap offset: per tap one strided, dilated
     2-D correlation of the source interval, added into the output interval."""
     rng = np.random.default_rng(5)
     k, stride, pad, dil, dil_t = (3, 3, 3), (2, 1), (1, 2), (1, 2), 2

@@ -1,6 +1,6 @@
 """Pins for the CPU oracle: everything here runs without a GPU and compares the
 oracle with something other than itself - hand-worked values, a structurally
-different brute-force routine, the paper's Algorithm 1 taken literally, the
+different brute-force routine, Eq. (2) read frame by frame with a library 2-D correlation, the
 fp64 library conv3d on the explicitly concatenated input, and the invariants
 the operator must satisfy (causality, streaming equivalence, linearity,
 1x1x1 = per-pixel matmul, delta kernel, NULL cache = zero cache)."""
@@ -87,14 +87,35 @@ def test_brute_force_and_points_agree(seed):
     assert np.array_equal(pts.reshape(out.shape), out)      # same order of summation -> identical
 
 
-@pytest.mark.parametrize("cache", [True, False])
+@pytest.mark.parametrize("cache_frames", [2, 1, 0])
 @pytest.mark.parametrize("T", [1, 2, 4])
-def test_algorithm1_route_equals_definition(cache, T):
+def test_eq2_frame_by_frame_with_library_conv2d(cache_frames, T):
+    """Eq. (2) as a statement about single frames: output frame t is the bias plus, for every temporal tap k, the
+    2-D correlation (the library's, fp64) of Z frame q_k(t) = t + k - p_l of Eq. (1) with W[:, :, k]; a tap whose
+    source time falls outside Z contributes nothing.  Z = [C ; X], p_l = (kt-1) - |C|.  No intervals, no batching:
+    a different route to the same numbers than the oracle's loops, and the temporal index is written here from
+    Eq. (1), not taken from the oracle."""
+    torch = pytest.importorskip("torch")
     rng = np.random.default_rng(100 + T)
-    x, c, w, b = _rand_case(rng, 2, 3, 4, T, 5, 6, (3, 3, 3), cache=cache)
-    out, _ = oracle.forward(x, c, w, b)
-    alg = oracle.algorithm1_route(x, c, w, b)
-    assert np.max(np.abs(out - alg)) <= 1e-12 * (np.abs(out).max() + 1)
+    x, c, w, b = _rand_case(rng, 2, 3, 4, T, 5, 6, (3, 3, 3), cache=True)
+    kt = 3
+    p_l = (kt - 1) - cache_frames
+    Z = x if cache_frames == 0 else np.concatenate([c[:, :, kt - 1 - cache_frames:], x], axis=2)
+    # the oracle's interface takes a full-length cache: absent older frames are zeros in front
+    c_full = None if cache_frames == 0 else c.copy()
+    if cache_frames == 1:
+        c_full[:, :, 0] = 0
+    out, _ = oracle.forward(x, c_full, w, b)
+    Zt, wt = torch.from_numpy(Z.astype(np.float64)), torch.from_numpy(w.astype(np.float64))
+    ref = np.zeros_like(out)
+    for t in range(T):
+        acc = torch.from_numpy(b.astype(np.float64))[None, :, None, None].expand(2, 4, 5, 6).clone()
+        for k in range(kt):
+            q = t + k - p_l
+            if 0 <= q < Z.shape[2]:
+                acc = acc + torch.nn.functional.conv2d(Zt[:, :, q], wt[:, :, k], padding=1)
+        ref[:, :, t] = acc.numpy()
+    assert np.max(np.abs(out - ref)) <= 1e-12 * (np.abs(out).max() + 1)
 
 
 @pytest.mark.parametrize("k", [(3, 3, 3), (1, 1, 1), (3, 1, 1), (1, 3, 3)])
