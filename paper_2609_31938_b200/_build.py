@@ -6,7 +6,7 @@ import subprocess
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
-LIB = os.path.join(HERE, "libccv3d.so")
+LIB = os.environ.get("CCV3D_LIB") or os.path.join(HERE, "libccv3d.so")   # (CCV3D_LIB: another build of the library, for diagnosis)
 SOURCES = ["ccv3d_api.cu"]
 DEPS = ["ccv3d_api.cu", "ccv3d_simt.cuh", "ccv3d_tc.cuh", "ccv3d_tc_layout.cuh", "ccv3d_tc_ptx.cuh", "ccv3d_tc_conv.cuh",
         "ccv3d_tc_pointwise.cuh", "ccv3d_host_common.cuh", "ccv3d_host_tc.cuh", "ccv3d_host_ring.cuh",

@@ -168,12 +168,14 @@ ccv3d_status grow(void** buf, uint64_t* have, uint64_t need) {
 
 // es_w, es_h: traversal strides of the box along w and h (the layer's spatial stride in the per-tap mode, else 1);
 // the box then spans BW*es_w x BH*es_h pixels and delivers BW x BH of them.
-ccv3d_status encode_act_map(ccv3d_handle* h, int N, int T, int H, int W, int BW, int BH, int es_w = 1, int es_h = 1) {
+// phases > 1: H and W are the extents of one phase image and every channel block holds `phases` of them.
+ccv3d_status encode_act_map(ccv3d_handle* h, int N, int T, int H, int W, int BW, int BH, int es_w = 1, int es_h = 1,
+                            int phases = 1) {
     const TcPlan& pl = h->plan;
     const int F = hist_len(h->d) + T;
     const bool f32 = h->d.dtype == CCV3D_F32;             // rows of 32 FP32 channels; two blocks (value, remainder) per real block
     const uint64_t rowb = (uint64_t)pl.KB * 2;
-    const int inner = f32 ? 32 : pl.KB, blocks = f32 ? 2 * pl.CB : pl.CB;
+    const int inner = f32 ? 32 : pl.KB, blocks = (f32 ? 2 * pl.CB : pl.CB) * phases;
     cuuint64_t dims[5] = {(cuuint64_t)inner, (cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)blocks, (cuuint64_t)N * F};
     cuuint64_t strides[4] = {rowb, rowb * W, rowb * W * H, rowb * W * H * blocks};
     cuuint32_t box[5] = {(cuuint32_t)inner, (cuuint32_t)(BW * es_w), (cuuint32_t)(BH * es_h), 1, 1};
@@ -201,5 +203,7 @@ ccv3d_status encode_out_map(ccv3d_handle* h, void* out, int N, int T, int H, int
 uint64_t tc_workspace_bytes(const ccv3d_handle* h, int N, int T, int H, int W) {
     const int F = hist_len(h->d) + T;
     if (h->d.dtype == CCV3D_F32) return (uint64_t)N * F * h->plan.cin_pad * H * W * 8;   // values and remainders, FP32
-    return (uint64_t)N * F * h->plan.cin_pad * H * W * 2;
+    // (layers with a spatial stride: whole phase images, i.e. extents rounded up to multiples of the stride)
+    const int sh = h->d.stride[1], sw = h->d.stride[2];
+    return (uint64_t)N * F * h->plan.cin_pad * ((H + sh - 1) / sh * sh) * ((W + sw - 1) / sw * sw) * 2;
 }

@@ -43,6 +43,16 @@ struct TcParams {
     // the kernel uses pad = (k-1)/2 and unit dilation.  H and W above are the OUTPUT extents; the input extents
     // only live in the tensor map.  Spatial stride > 1 is served by the per-tap mode with a strided tensor map.
     int general, pad_h, pad_w, dil_h, dil_w, dil_t, str_h, str_w, str_t;   // T above counts OUTPUT frames (T_o)
+    // Spatial stride > 1 from a phase-decomposed staging copy (phased = 1): the staged frames are split into
+    // S2 = s_h * s_w phase images (pixel (h, w) lives in phase (h % s_h) * s_w + w % s_w at (h / s_h, w / s_w)), in which
+    // consecutive output pixels are consecutive pixels again, so that each phase needs one halo tile and its taps are
+    // descriptor offsets into it: tap (a, c) reads phase image pixel (oh + floor((a d_h - p_h) / s_h), ow + ...).
+    int phased, S2;
+    int ph_bw, ph_bh;                     // halo extents beyond the tile (largest offset range of any phase)
+    unsigned char ph_first[17];           // taps of phase q: entries ph_first[q] .. ph_first[q+1]-1 of the lists below
+    unsigned char ph_tap[49];             // spatial tap index a*kw + c
+    unsigned char ph_roff[49], ph_coff[49];   // the tap's row / column offset inside its phase's halo tile
+    signed char ph_h0[16], ph_w0[16];     // halo origin of a phase relative to the tile origin (in phase-image pixels)
     int f0;                   // ring input: the slot of Z frame 0; Z frame f lives in slot (f0 + f) mod F (0 for a staged copy)
     const __nv_bfloat16* res; // optional residual ring [N][res_F][res_CB][H][W][res_KB] holding Cout channels, or null
     int res_F, res_f0, res_CB, res_KB;   // residual frame t is slot (res_f0 + t) mod res_F
@@ -70,7 +80,7 @@ constexpr int TC_BIAS_SMEM = 512;
 struct TcShared {  // placed after the rings
     uint64_t full_a[TC_MAX_STAGES], empty_a[TC_MAX_STAGES];
     uint64_t full_b[TC_MAX_STAGES], empty_b[TC_MAX_STAGES];
-    uint64_t acc_full[2], acc_empty[2];
+    uint64_t acc_full[4], acc_empty[4];   // (the convolution kernel uses two, the 1x1x1 streaming kernel up to four)
     uint64_t raw_full[2], raw_empty[2];
     uint32_t tmem_base;
     volatile int abort_flag;
@@ -192,7 +202,9 @@ __device__ __forceinline__ uint32_t epi_pair(float a0, float a1, uint32_t res_pa
 // shared-memory read port.  Loads of both CTAs are counted on the leader's "full" barriers; the leader's commits
 // arrive on the "empty" and "accumulator full" barriers of both CTAs; both epilogues arrive on the leader's
 // "accumulator empty" barrier.
-template <int KB, int NB, int KS, int TPBC, bool FUSED, bool COOP, bool TF32 = false, bool PAIR = false, bool TAIL = false>
+// DIL: spatial dilation of the straight-line tap loop (1, or 2 for 3x3 kernels with d_h = d_w = 2: the tap offsets
+// into the halo tile double and stay compile-time constants).
+template <int KB, int NB, int KS, int TPBC, bool FUSED, bool COOP, bool TF32 = false, bool PAIR = false, bool TAIL = false, int DIL = 1>
 __global__ void __launch_bounds__((FUSED || COOP) ? TC_THREADS_FUSED : TC_THREADS, 1)
 conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged activations (c, w, h, cb, n*F+f), or x
                       const __grid_constant__ CUtensorMap tm_c,   // fused mode: the cache; PAIR: the packed weights
@@ -202,6 +214,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     static_assert(!FUSED || KB == 32, "the fused mode transposes 32-channel blocks");
     static_assert(!TF32 || (KB == 64 && !FUSED && !COOP), "FP32 layers: 128-byte rows, plain variant");
     static_assert(!PAIR || (KS > 0 && !FUSED), "CTA pairs: straight-line taps");
+    static_assert(DIL == 1 || (DIL == 2 && KS == 3 && PAIR && !TF32 && !TAIL), "dilated straight-line taps: 3x3, d = 2, CTA pairs");
     // (TF32 layers always write FP32 through the direct-store epilogue, which is where the two accumulators of the
     // last pass are added)
     constexpr uint32_t ROWB = KB * 2;                       // bytes per pixel row (one swizzle span)
@@ -234,8 +247,8 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     const int dlh = p.general ? p.dil_h : 1, dlw = p.general ? p.dil_w : 1, dlt = p.general ? p.dil_t : 1;
     const int sth = p.general ? p.str_h : 1, stw = p.general ? p.str_w : 1;      // > 1 only in the per-tap mode
     const int stt = p.general ? p.str_t : 1;                // temporal stride: output frame t reads Z frames t*stt + dt*dlt
-    const int BW = p.per_tap_a ? TW : TW + (p.kw - 1) * dlw;        // pixels per smem image row
-    const int BH = p.per_tap_a ? 16 : 16 + (p.kh - 1) * dlh;
+    const int BW = p.phased ? TW + p.ph_bw : (p.per_tap_a ? TW : TW + (p.kw - 1) * dlw);        // pixels per smem image row
+    const int BH = p.phased ? 16 + p.ph_bh : (p.per_tap_a ? 16 : 16 + (p.kh - 1) * dlh);
     const int spatial = p.kh * p.kw;
 
     if (threadIdx.x == 0) {
@@ -348,6 +361,18 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                         int fr = p.f0 + t * stt + dt * dlt;       // ring slot of Z frame t s_t + dt d_t (f0 = 0: the frame itself)
                         if (fr >= p.F) fr -= p.F;
                         const int fz = n * p.F + fr;
+                        if (KS == 0 && !PAIR && p.phased) {       // one halo tile per phase image that has taps
+                            for (int q = 0; ok && q < p.S2; ++q) {
+                                if (p.ph_first[q + 1] == p.ph_first[q]) continue;
+                                if (!(ok = mbar_wait(&sh->empty_a[s], phase, sh, p, SITE_A_EMPTY))) break;
+                                const uint32_t bar = smem_u32(&sh->full_a[s]);
+                                mbar_expect_tx(bar, a_bytes);
+                                tma_load_5d(smem_u32(ring_a + (size_t)s * p.a_slot), &tm_a, bar, 0, w0 + p.ph_w0[q], h0 + p.ph_h0[q],
+                                            cb * p.S2 + q, fz);
+                                if (++s == p.SA) { s = 0; phase ^= 1; }
+                            }
+                            continue;
+                        }
                         const int ntap = p.per_tap_a ? spatial : 1;
                         for (int tp = 0; tp < ntap; ++tp) {
                             if (!(ok = mbar_wait(&sh->empty_a[s], phase, sh, p, SITE_A_EMPTY))) break;
@@ -422,6 +447,8 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                             const uint32_t bar = smem_u32(&sh->full_b[s]);
                             mbar_expect_tx(bar, b_bytes);
                             const uint32_t dst = smem_u32(ring_b + (size_t)s * p.b_slot);
+                            if (KS == 0 && p.phased) bulk_load(dst, src + (size_t)p.ph_tap[tp] * src_tap, b_bytes, bar);   // taps in phase order (TPB = 1)
+                            else
                             if (src_tap == tv.b_tap) bulk_load(dst, src + (size_t)tp * src_tap, b_bytes, bar);
                             else
                                 for (int u = 0; u < p.TPB; ++u) bulk_load(dst + u * tv.b_tap, src + (size_t)(tp + u) * src_tap, tv.b_tap, bar);
@@ -454,7 +481,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
         uint32_t pa = 0, pb = 0, pacc = 1;
         bool ok = true;
         if constexpr (KS > 0) {
-            constexpr uint32_t A_ROWSTEP = ((uint32_t)(TW + KS - 1) * ROWB) >> 4;
+            constexpr uint32_t A_ROWSTEP = ((uint32_t)(TW + (KS - 1) * DIL) * DIL * ROWB) >> 4;   // one kernel row down the halo tile
             constexpr int STAGES = KS * KS / TPBC;
             uint32_t a_ring = make_desc_lo(smem_u32(ring_a)) + a_blk, b_ring = make_desc_lo(smem_u32(ring_b));
             const uint32_t a_slotstep = p.a_slot >> 4, b_slotstep = p.b_slot >> 4;
@@ -491,7 +518,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                                 // 16-byte granular and need not sit on the swizzle period: the swizzle is a function of
                                 // the absolute shared-memory address (as the TMA unit applied it), so the descriptor's
                                 // base-offset field stays 0.
-                                const uint32_t a_lo = a_ring + (uint32_t)(tap / KS) * A_ROWSTEP + (uint32_t)(tap % KS) * (ROWB >> 4);
+                                const uint32_t a_lo = a_ring + (uint32_t)(tap / KS) * A_ROWSTEP + (uint32_t)(tap % KS) * DIL * (ROWB >> 4);
                                 const uint32_t b_lo = b_ring + (uint32_t)u * b_tapstep;
 #pragma unroll
                                 for (int j = 0; j < NBW; ++j) {
@@ -541,6 +568,41 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                     const bool second = TF32 && pass == 2 && (st2++ & 1);   // see the straight-line variant
                     const uint32_t d0 = d_first + (second ? (uint32_t)NB * p.NPAD : 0u);
                     uint32_t accumulate = second ? accumulate2 : accumulate1;
+                    if (p.phased) {
+                        // phase images: one halo tile per phase, its taps are (row, column) offsets into it
+                        const uint32_t row1 = ((uint32_t)BW * ROWB) >> 4;
+                        for (int q = 0; ok && q < p.S2; ++q) {
+                            const int i0 = p.ph_first[q], i1 = p.ph_first[q + 1];
+                            if (i0 == i1) continue;
+                            if (!(ok = mbar_wait(&sh->full_a[sa], pa, sh, p, SITE_A_FULL))) break;
+                            const uint32_t a_base = make_desc_lo(smem_u32(ring_a + (size_t)sa * p.a_slot)) + a_blk;
+                            for (int i = i0; i < i1; ++i) {
+                                if (!(ok = mbar_wait(&sh->full_b[sb], pb, sh, p, SITE_B_FULL))) break;
+                                tc_fence_after();
+                                const uint32_t b_lo = make_desc_lo(smem_u32(ring_b + (size_t)sb * p.b_slot));
+                                const uint32_t a_lo = a_base + (uint32_t)p.ph_roff[i] * row1 + (uint32_t)p.ph_coff[i] * (ROWB >> 4);
+                                if (elect_one()) {
+#pragma unroll
+                                    for (int j = 0; j < NBW; ++j) {
+#pragma unroll
+                                        for (int k = 0; k < KSTEPS; ++k)
+                                            tc_mma<TF32>(d0 + j * p.NPAD, a_lo + j * ((8 * ROWB) >> 4) + 2 * k, a_hi, b_lo + 2 * k, b_hi,
+                                                        idesc, (k == 0) ? accumulate : 1u);
+                                    }
+                                    tc_commit(smem_u32(&sh->empty_b[sb]));
+                                }
+                                __syncwarp();
+                                accumulate = 1;
+                                if (++sb == p.SB) { sb = 0; pb ^= 1; }
+                            }
+                            if (!ok) break;
+                            if (elect_one()) tc_commit(smem_u32(&sh->empty_a[sa]));
+                            __syncwarp();
+                            if (++sa == p.SA) { sa = 0; pa ^= 1; }
+                        }
+                        if (second) accumulate2 = accumulate; else accumulate1 = accumulate;
+                        continue;
+                    }
                     uint32_t a_row = 0;  // descriptor low word of the halo row of the current tap row
                     if (!p.per_tap_a) {
                         if (!(ok = mbar_wait(&sh->full_a[sa], pa, sh, p, SITE_A_FULL))) break;

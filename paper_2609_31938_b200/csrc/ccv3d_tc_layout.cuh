@@ -52,6 +52,10 @@ struct StageParams {
     int h_begin;                 // first image row of this launch (grid.y rows are staged)
     int ring_F = 0, ring_f0 = 0; // ring_F > 0 (separate staging kernel only): zs is a frame ring of ring_F slots and
                                  // Z frame f goes to slot (ring_f0 + f) mod ring_F
+    // Phase-decomposed copy for layers with a spatial stride (separate staging kernel only; ph_sh = 0: off):
+    // zs is [N][F][CB][ph_sh*ph_sw][ph_Hp][ph_Wp][KB], pixel (h, w) goes to phase (h % ph_sh) * ph_sw + w % ph_sw at
+    // (h / ph_sh, w / ph_sw); the launch covers ph_Hp*ph_sh rows and ph_Wp*ph_sw columns, zeros beyond the image.
+    int ph_sh = 0, ph_sw = 0, ph_Hp = 0, ph_Wp = 0;
 };
 
 constexpr int STG_PX = 64;  // pixels of one image row handled per block
@@ -95,6 +99,7 @@ __global__ void __launch_bounds__(32 * (KB / 8)) stage_frames_kernel(const Stage
     const int64_t ncstride = (int64_t)p.tc * HW;
 
     // ---- load phase: KB channel rows of up to 64 pixels ----
+    if (h >= p.H) src = nullptr, ncdst = nullptr;           // (phase-decomposed copy: rows below the image are zeros)
     if (VEC) {
         // 8 vectors of 8 pixels per row
         for (int i = threadIdx.x; i < KB * 8; i += NTHR) {
@@ -140,8 +145,21 @@ __global__ void __launch_bounds__(32 * (KB / 8)) stage_frames_kernel(const Stage
     const int FS = p.ring_F > 0 ? p.ring_F : F;         // frame slots per sample
     int fs = p.ring_f0 + f;
     if (fs >= FS) fs -= FS;
-    __nv_bfloat16* dst = p.zs + ((((int64_t)n * FS + fs) * p.CB + cb) * HW + (int64_t)h * p.W) * KB;
     const int wa = w0 + 2 * pp;
+    if (p.ph_sh > 0) {
+        // phase images: pixel (h, w) -> phase (h % s_h, w % s_w), position (h / s_h, w / s_w); columns up to Wp * s_w
+        const int64_t img = (int64_t)p.ph_Hp * p.ph_Wp;
+        __nv_bfloat16* base = p.zs + ((((int64_t)n * FS + fs) * p.CB + cb) * (p.ph_sh * p.ph_sw) + (h % p.ph_sh) * p.ph_sw) * img * KB +
+                              (int64_t)(h / p.ph_sh) * p.ph_Wp * KB;
+        const int wlim = p.ph_Wp * p.ph_sw;
+        if (wa < wlim)
+            *reinterpret_cast<uint4*>(base + ((wa % p.ph_sw) * img + wa / p.ph_sw) * KB + oct * 8) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
+        if (wa + 1 < wlim)
+            *reinterpret_cast<uint4*>(base + (((wa + 1) % p.ph_sw) * img + (wa + 1) / p.ph_sw) * KB + oct * 8) =
+                make_uint4(hi[0], hi[1], hi[2], hi[3]);
+        return;
+    }
+    __nv_bfloat16* dst = p.zs + ((((int64_t)n * FS + fs) * p.CB + cb) * HW + (int64_t)h * p.W) * KB;
     if (wa < p.W) *reinterpret_cast<uint4*>(dst + (int64_t)wa * KB + oct * 8) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
     if (wa + 1 < p.W)
         *reinterpret_cast<uint4*>(dst + (int64_t)(wa + 1) * KB + oct * 8) = make_uint4(hi[0], hi[1], hi[2], hi[3]);

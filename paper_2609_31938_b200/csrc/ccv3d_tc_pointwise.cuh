@@ -22,6 +22,8 @@ struct PwParams {
     int total_tiles;
     int SA;                   // activation ring depth
     int ECH;                  // channels per epilogue chunk (32 or 16)
+    int EG;                   // epilogue warp groups (1 or 2): group g drains the accumulators of this CTA's tiles g, g+EG, ...
+    int NACC;                 // accumulator buffers in tensor memory (2..4): tile i of a CTA uses buffer i % NACC
     uint32_t a_slot, e_slot, w_bytes, b_tap;
     uint32_t tmem_cols;
     long long wait_limit_clk;
@@ -49,7 +51,9 @@ __device__ __forceinline__ bool pw_wait(uint64_t* bar, uint32_t parity, TcShared
     }
 }
 
-__global__ void __launch_bounds__(TC_THREADS, 1)
+constexpr int PW_THREADS = 384;       // producer, weights, MMA, allocator warps + two epilogue groups of four warps
+
+__global__ void __launch_bounds__(PW_THREADS, 1)
 conv1x1_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_x,   // x as (pixel, channel, sample)
                        const __grid_constant__ CUtensorMap tm_o,   // out as (pixel, channel, sample)
                        const PwParams p) {
@@ -60,7 +64,7 @@ conv1x1_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_x,   // x as (pixe
     uint8_t* w_smem = smem;
     uint8_t* ring_a = w_smem + p.w_bytes;
     uint8_t* epi_buf = ring_a + (size_t)p.SA * p.a_slot;
-    TcShared* sh = reinterpret_cast<TcShared*>(epi_buf + 2 * (size_t)p.e_slot);
+    TcShared* sh = reinterpret_cast<TcShared*>(epi_buf + 2 * (size_t)p.EG * p.e_slot);
 
     const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);
     const int lane = threadIdx.x & 31;
@@ -68,7 +72,7 @@ conv1x1_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_x,   // x as (pixe
     if (threadIdx.x == 0) {
         for (int i = 0; i < p.SA; ++i) { mbar_init(smem_u32(&sh->full_a[i]), 1); mbar_init(smem_u32(&sh->empty_a[i]), 1); }
         mbar_init(smem_u32(&sh->full_b[0]), 1);
-        for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&sh->acc_full[i]), 1); mbar_init(smem_u32(&sh->acc_empty[i]), 4); }
+        for (int i = 0; i < p.NACC; ++i) { mbar_init(smem_u32(&sh->acc_full[i]), 1); mbar_init(smem_u32(&sh->acc_empty[i]), 4); }
         sh->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -78,10 +82,12 @@ conv1x1_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_x,   // x as (pixe
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    for (int i = threadIdx.x; i < p.NPAD; i += blockDim.x) sh->bias_s[i] = __ldg(p.bias + i);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = sh->tmem_base;
+    const int t_first = (int)blockIdx.x, t_end = p.total_tiles, t_step = (int)gridDim.x;   // this CTA's tiles
 
     if (warp == 0) {                      // activation producer
         if (lane == 0) {
@@ -89,13 +95,13 @@ conv1x1_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_x,   // x as (pixe
             int s = 0;
             uint32_t phase = 1;
             bool ok = true;
-            for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+            for (int tile = t_first; ok && tile < t_end; tile += t_step) {
                 const int n = tile / p.tiles_p, p0 = (tile % p.tiles_p) * 128;
                 for (int cb = 0; cb < p.CB; ++cb) {
                     if (!(ok = pw_wait(&sh->empty_a[s], phase, sh, p, SITE_A_EMPTY))) break;
                     const uint32_t bar = smem_u32(&sh->full_a[s]);
-                    mbar_expect_tx(bar, 2 * HALF);
                     const uint32_t dst = smem_u32(ring_a + (size_t)s * p.a_slot);
+                    mbar_expect_tx(bar, 2 * HALF);
                     tma_load_3d(dst, &tm_x, bar, p0, cb * KB, n);
                     tma_load_3d(dst + HALF, &tm_x, bar, p0 + 64, cb * KB, n);
                     if (++s == p.SA) { s = 0; phase ^= 1; }
@@ -119,8 +125,8 @@ conv1x1_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_x,   // x as (pixe
         int sa = 0, acc = 0;
         uint32_t pa = 0, pacc = 1;
         bool ok = pw_wait(&sh->full_b[0], 0, sh, p, SITE_B_FULL);
-        for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
-            if (!(ok = pw_wait(&sh->acc_empty[acc], pacc, sh, p, SITE_ACC_EMPTY))) break;
+        for (int tile = t_first; ok && tile < t_end; tile += t_step) {
+            if (!(ok = pw_wait(&sh->acc_empty[acc], pacc, sh, p, SITE_ACC_EMPTY))) break;   // (first use of a buffer: passes at once)
             tc_fence_after();
             const uint32_t d0 = tmem_base + (uint32_t)acc * p.NPAD;
             for (int cb = 0; cb < p.CB; ++cb) {
@@ -140,16 +146,23 @@ conv1x1_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_x,   // x as (pixe
             if (!ok) break;
             if (elect_one()) tc_commit(smem_u32(&sh->acc_full[acc]));
             __syncwarp();
-            if (++acc == 2) { acc = 0; pacc ^= 1; }
+            if (++acc == p.NACC) { acc = 0; pacc ^= 1; }
         }
-    } else if (warp >= 4) {               // epilogue: +bias, RNE to BF16, [channel][128 px] tile, TMA store
+    } else if (warp >= 4 && warp < 4 + 4 * p.EG) {   // epilogue: +bias, RNE to BF16, [channel][128 px] tile, TMA store
+        // One group of four warps drains both accumulator buffers in turn, or two groups drain one buffer each (tile
+        // i of this CTA uses buffer i & 1), each with its own staging buffers, named barrier and store groups.
+        const int g = (warp - 4) >> 2;
         const int q = warp & 3;
         const int m = q * 32 + lane;
-        const bool elected = (threadIdx.x == 4 * 32);
-        int acc = 0, ebuf = 0;
-        uint32_t pacc = 0;
+        const bool elected = (q == 0 && lane == 0);
+        const uint32_t bar_id = 1u + 2u * (uint32_t)g;
+        uint8_t* my_buf = epi_buf + (size_t)g * 2 * p.e_slot;
+        int ebuf = 0, it = 0;
         bool ok = true;
-        for (int tile = blockIdx.x; ok && tile < p.total_tiles; tile += gridDim.x) {
+        for (int tile = t_first; ok && tile < t_end; tile += t_step, ++it) {
+            if (p.EG == 2 && (it & 1) != g) continue;
+            const int acc = it % p.NACC;
+            const uint32_t pacc = (uint32_t)(it / p.NACC) & 1u;      // the k-th use of a buffer completes its phase k
             const int n = tile / p.tiles_p, p0 = (tile % p.tiles_p) * 128;
             ok = pw_wait(&sh->acc_full[acc], pacc, sh, p, SITE_ACC_FULL);
             ok = __all_sync(0xffffffffu, ok);
@@ -157,17 +170,36 @@ conv1x1_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_x,   // x as (pixe
             tc_fence_after();
             const uint32_t t_acc = tmem_base + (uint32_t)acc * p.NPAD + ((uint32_t)(q * 32) << 16);
             for (int c0 = 0; c0 < p.NPAD; c0 += p.ECH) {
-                if (elected) bulk_wait_read<1>();
-                epi_bar_sync();
-                __nv_bfloat16* stg = reinterpret_cast<__nv_bfloat16*>(epi_buf + (size_t)ebuf * p.e_slot);
+                if (elected) bulk_wait_read<1>();   // the store that last read this buffer has finished reading
+                asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+                __nv_bfloat16* stg = reinterpret_cast<__nv_bfloat16*>(my_buf + (size_t)ebuf * p.e_slot);
                 uint32_t v[32];
                 if (p.ECH == 32) tc_ld32(t_acc + c0, v); else tc_ld16(t_acc + c0, v);
                 tc_wait_ld();
+                // +bias, two neighbouring channels per (packed) conversion, their halves to two rows of the
+                // [channel][128 px] tile; one straight-line body per chunk width
+                auto convert_store = [&](auto ech_c) {
+                    constexpr int E = decltype(ech_c)::value;
+                    unsigned short* st16 = reinterpret_cast<unsigned short*>(stg) + m;
+                    float bb[E];
 #pragma unroll
-                for (int j = 0; j < 32; ++j)
-                    if (j < p.ECH) stg[j * 128 + m] = __float2bfloat16_rn(__uint_as_float(v[j]) + __ldg(p.bias + c0 + j));
+                    for (int j4 = 0; j4 < E / 4; ++j4) {
+                        const float4 b4 = *reinterpret_cast<const float4*>(sh->bias_s + c0 + 4 * j4);
+                        bb[4 * j4] = b4.x; bb[4 * j4 + 1] = b4.y; bb[4 * j4 + 2] = b4.z; bb[4 * j4 + 3] = b4.w;
+                    }
+#pragma unroll
+                    for (int j = 0; j < E / 2; ++j) {
+                        const __nv_bfloat162 pr = __floats2bfloat162_rn(__uint_as_float(v[2 * j]) + bb[2 * j],
+                                                                        __uint_as_float(v[2 * j + 1]) + bb[2 * j + 1]);
+                        const uint32_t u = *reinterpret_cast<const uint32_t*>(&pr);
+                        st16[(2 * j) * 128] = (unsigned short)(u & 0xFFFFu);
+                        st16[(2 * j + 1) * 128] = (unsigned short)(u >> 16);
+                    }
+                };
+                if (p.ECH == 32) convert_store(std::integral_constant<int, 32>{});
+                else convert_store(std::integral_constant<int, 16>{});
                 fence_async_smem();
-                epi_bar_sync();
+                asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
                 if (elected) {
                     tma_store_3d(&tm_o, smem_u32(stg), p0, c0, n);
                     bulk_commit();
@@ -177,7 +209,6 @@ conv1x1_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_x,   // x as (pixe
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sh->acc_empty[acc]));
-            if (++acc == 2) { acc = 0; pacc ^= 1; }
         }
         if (elected) bulk_wait_all();
     }

@@ -129,6 +129,18 @@ def test_temporal_stride(ccv, k, stride, pad, dil, dil_t, stride_t, T, route):
     assert ctr["tcgen05_bf16" if route == "bf16_tc" else "simt"] == 1
 
 
+@pytest.mark.parametrize("H,W", [(512, 640), (511, 637)])
+def test_spatial_stride_on_many_tiles(ccv, H, W):
+    """A downsampling layer (3x3x3, spatial stride 2) on an image of hundreds of tiles: the staging kernel writes the
+    phase-decomposed copy (four phase images per channel block; zero rows and columns where the image is not a whole
+    number of phases, as with the odd extents here), the convolution kernel reads one halo tile per phase.  Against the
+    oracle, cache bit-exact."""
+    c = _case(1, 64, 64, 4, H, W, (3, 3, 3), si.BF16, 2, seed=47)
+    m, ctr = run_general(ccv, c, (2, 2), (1, 1), (1, 1), 1)
+    assert ctr["tcgen05_bf16"] == 1 and ctr["kernel_launches"] == 4            # weight pack, bias, staging, convolution
+    print("stride 2,", (H, W), m)
+
+
 def test_streaming_with_temporal_stride_on_gpu(ccv):
     c = _case(1, 64, 32, 8, 20, 24, (3, 3, 3), si.BF16, 0, seed=39)
     layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), stride=(2, 1, 1))
