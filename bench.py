@@ -469,6 +469,30 @@ def other_configs_leg(dev, local):
         del x, cache, y, nc, c
         torch.cuda.empty_cache()
 
+    # ---- the paper's wider contract at speed (Eq. (2) passes the layer's stride and dilation to every tap): a
+    # downsampling layer (spatial stride 2, phase-decomposed staging) and a dilated one (straight-line taps two pixels apart)
+    for label, (Cin, Cout, T, H, W), stride, dil in (
+            ("general_96to192_stride2_704x1280", (96, 192, 4, 704, 1280), (1, 2, 2), (1, 1, 1)),
+            ("general_192_dilation2_352x640", (192, 192, 4, 352, 640), (1, 1, 1), (1, 2, 2))):
+        c = si.conv_case(1, Cin, Cout, T, H, W, dtype=si.BF16, seed=0)
+        x, cache = up(c["x"]), up(c["cache"])
+        layer = ccv.CausalConv3d(up(c["w"]), up(c["b"]), stride=stride, dilation=dil)
+        _, To, Ho, Wo, _ = ccv.ccv3d_out_dims(layer.h, T, H, W)
+        y = torch.empty((1, Cout, To, Ho, Wo), dtype=torch.bfloat16, device=dev)
+        nc = torch.empty_like(cache)
+        ms, clk = clocked(lambda: layer(x, cache, out=y, new_cache=nc))
+        st = stats(ms)
+        flops = 2.0 * Cout * Cin * 27 * To * Ho * Wo
+        abytes = c["x"].nbytes + 2 * c["cache"].nbytes + c["w"].nbytes + 2 * Cout * To * Ho * Wo
+        out[label] = {"ms_per_call": st["ms_median"], **st, "tflops": flops / (st["ms_median"] * 1e-3) / 1e12, "clocks": clk,
+                      "stride": list(stride), "dilation": list(dil), "out_hw": [Ho, Wo],
+                      "roofline": roofline_of(flops, abytes, st["ms_median"], peaks),
+                      "kernel_variant": kernel_variant(ccv, layer, lambda: layer(x, cache, out=y, new_cache=nc))}
+        assert layer.device_status()[0] == ccv.OK
+        layer.close()
+        del x, cache, y, nc, c
+        torch.cuda.empty_cache()
+
     # ---- the headline layer's first-chunk form (NULL cache: the taps of absent history are skipped) and its
     # staging + cache-update kernel alone (two-kernel schedule), warm and with a cold L2
     name = DEFAULT_WORKLOAD

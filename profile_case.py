@@ -1,6 +1,7 @@
 """Run a few forward calls of one layer shape on cuda:0 - a small, self-ending program to put under a profiler.
 
     python profile_case.py --cin 192 --cout 192 --t 4 --h 176 --w 320 [--k 3 3 3] [--calls 3] [--ring]
+                           [--stride 1 2 2] [--dilation 1 2 2]
 
 Inputs are the seeded synthetic tensors of the benchmark (normal activations, fan-in-scaled weights).
 """
@@ -29,6 +30,8 @@ def main():
     ap.add_argument("--flags", type=int, default=0, help="CCV3D_FLAG_* bits (16 = two-kernel schedule, 8 = fused route)")
     ap.add_argument("--ring", action="store_true", help="resident activations: input and output in frame rings")
     ap.add_argument("--f32", action="store_true", help="FP32 layer (tensor cores by 3xTF32 when the call is large enough)")
+    ap.add_argument("--stride", type=int, nargs=3, default=[1, 1, 1], help="(s_t, s_h, s_w)")
+    ap.add_argument("--dilation", type=int, nargs=3, default=[1, 1, 1], help="(d_t, d_h, d_w); size-preserving padding")
     a = ap.parse_args()
     c = si.conv_case(1, a.cin, a.cout, a.t, a.h, a.w, k=tuple(a.k), cache=None if a.no_cache else "random",
                      dtype=si.F32 if a.f32 else si.BF16)
@@ -36,9 +39,12 @@ def main():
         up = lambda v: None if v is None else torch.from_numpy(v).cuda()
     else:
         up = lambda v: None if v is None else torch.from_numpy(v.view(np.int16)).cuda().view(torch.bfloat16)
-    layer = ccv.CausalConv3d(up(c["w"]), up(c["b"]), flags=a.flags)
+    layer = ccv.CausalConv3d(up(c["w"]), up(c["b"]), flags=a.flags, stride=tuple(a.stride), dilation=tuple(a.dilation))
     x, cache = up(c["x"]), up(c["cache"])
-    out = torch.empty((1, a.cout, a.t, a.h, a.w), dtype=torch.float32 if a.f32 else torch.bfloat16, device="cuda")
+    if cache is not None and a.dilation[0] > 1:        # the history is d_t (kt-1) frames long
+        cache = torch.cat([cache] * a.dilation[0], dim=2).contiguous()
+    _, To, Ho, Wo, _ = ccv.ccv3d_out_dims(layer.h, a.t, a.h, a.w)
+    out = torch.empty((1, a.cout, To, Ho, Wo), dtype=torch.float32 if a.f32 else torch.bfloat16, device="cuda")
     nc = torch.empty_like(cache) if cache is not None else None
     if a.ring:
         tc = a.k[0] - 1

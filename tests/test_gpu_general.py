@@ -129,6 +129,14 @@ def test_temporal_stride(ccv, k, stride, pad, dil, dil_t, stride_t, T, route):
     assert ctr["tcgen05_bf16" if route == "bf16_tc" else "simt"] == 1
 
 
+def test_spatial_stride_with_two_samples_and_three_by_two_phases(ccv):
+    """The phase-decomposed path with N = 2 and a stride of (3, 2): six phase images per channel block, some with a
+    single tap, image extents that are not multiples of the stride."""
+    c = _case(2, 64, 48, 3, 29, 38, (3, 3, 3), si.BF16, 2, seed=48)
+    m, ctr = run_general(ccv, c, (3, 2), (1, 1), (1, 1), 1)
+    assert ctr["tcgen05_bf16"] == 1 and ctr["simt"] == 0
+
+
 @pytest.mark.parametrize("H,W", [(512, 640), (511, 637)])
 def test_spatial_stride_on_many_tiles(ccv, H, W):
     """A downsampling layer (3x3x3, spatial stride 2) on an image of hundreds of tiles: the staging kernel writes the
