@@ -341,6 +341,23 @@ def timed_calls(fn, iters, warmup=3, flush=None):
     return [ev[i].elapsed_time(ev[i + 1]) for i in range(iters)]
 
 
+def graph_replay_ms(fn, calls=20, replays=10):
+    """Per-call device time of `fn` captured `calls` times in a CUDA graph and replayed: what a launch-bound layer
+    costs when the host's enqueue time is out of the way.  `fn` must allocate nothing (lent workspace, rings)."""
+    import torch
+    fn()
+    torch.cuda.synchronize()
+    g, st = torch.cuda.CUDAGraph(), torch.cuda.Stream()
+    with torch.cuda.stream(st):
+        g.capture_begin()
+        for _ in range(calls):
+            fn()
+        g.capture_end()
+    torch.cuda.synchronize()
+    ms = timed_calls(g.replay, replays, warmup=2)
+    return float(np.median(ms)) / calls
+
+
 def stats(ms_list):
     a = np.asarray(ms_list, dtype=np.float64)
     return {"ms_mean": float(a.mean()), "ms_median": float(np.median(a)), "ms_min": float(a.min()), "samples": int(a.size)}
@@ -463,6 +480,30 @@ def other_configs_leg(dev, local):
             del rin, rout
         assert layer.device_status()[0] == ccv.OK
         layer.close()
+        if name in ("cfg2_bf16_384", "cfg1_f32_16"):
+            # launch-bound layers: the same calls captured in a CUDA graph (the staging copy in a lent workspace, so
+            # that nothing is allocated inside the capture)
+            lay2 = ccv.CausalConv3d(up(c["w"]), up(c["b"]))
+            _, need = ccv.ccv3d_workspace_bytes(lay2.h, N, T, H, W)
+            wsb = torch.empty(max(int(need), 256) + 256, dtype=torch.uint8, device=dev)
+            if need:
+                assert ccv.ccv3d_set_workspace(lay2.h, (wsb.data_ptr() + 255) // 256 * 256, int(need)) == ccv.OK
+            gms = graph_replay_ms(lambda: lay2(x, cache, out=y, new_cache=nc))
+            row["graph_replay"] = {"ms_per_call": gms, "tflops": flops / (gms * 1e-3) / 1e12,
+                                   "note": "20 calls captured in a CUDA graph, replayed; lent workspace"}
+            if not f32:
+                row["graph_replay"]["frac_of_measured_bf16_peak"] = flops / (gms * 1e-3) / 1e12 / peaks["tflops"]
+                F = T + k[0] - 1
+                rin, rout = ccv.FrameRing(N, Cin, F, H, W), ccv.FrameRing(N, Cout, T, H, W)
+                rin.load(0, cache)
+                rin.load(k[0] - 1, x)
+                rg = graph_replay_ms(lambda: lay2.forward_ring(rin, k[0] - 1, k[0] - 1, T, out_ring=rout))
+                row["graph_replay"]["resident_ms_per_call"] = rg
+                row["graph_replay"]["resident_frac_of_measured_bf16_peak"] = flops / (rg * 1e-3) / 1e12 / peaks["tflops"]
+                del rin, rout
+            assert lay2.device_status()[0] == ccv.OK
+            lay2.close()
+            del wsb
         if not f32:
             row["cpu_baseline"] = cpu_baseline(name, target_s=3.0)
         out[name] = row

@@ -170,6 +170,9 @@ ccv3d_status forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int x_slot, int
     p.wq = (const uint8_t*)h->wp;
     p.out = out_ncthw;
     p.status = h->status;
+#ifdef CCV3D_DEV_TRACE
+    p.trace = getenv("CCV3D_TC_TRACE") ? (unsigned long long*)strtoull(getenv("CCV3D_TC_TRACE"), nullptr, 0) : nullptr;
+#endif
     const size_t smem = fixed + (size_t)p.SA * p.a_slot + (size_t)p.SB * p.b_slot;
     int grid = p.total_tiles < h->sm_count ? p.total_tiles : h->sm_count;
     if (pair) grid = 2 * (p.total_tiles < h->sm_count / 2 ? p.total_tiles : h->sm_count / 2);

@@ -60,6 +60,9 @@ struct TcParams {
     int act;                             // 1: SiLU on conv + bias before the output rounding (and before the residual)
     int up_rt;                           // epi_tma == 2, > 0: the output ring is 2H x 2W; every pixel is written 2x2 times into
                                          // each of the up_rt slots (out_f0 + t*up_rt + j) mod out_F (nearest-neighbour upsample)
+#ifdef CCV3D_DEV_TRACE
+    unsigned long long* trace;   // dev builds: clock64 stamps of CTA 0
+#endif
     const float* bias;        // [NT*NPAD]
     const uint8_t* wq;        // packed weight tiles [dt][cb][nt][sp] of b_tap bytes each
     void* out;
@@ -231,6 +234,12 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     const int cta_cnt = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
     const int wofs = PAIR ? TW * (int)rank : 0;             // this CTA's pixel columns inside the tile
 
+#ifdef CCV3D_DEV_TRACE
+#define TC_STAMP(k) do { if (p.trace && blockIdx.x == 0) p.trace[(k)] = clock64(); } while (0)
+#else
+#define TC_STAMP(k) do { } while (0)
+#endif
+    if (threadIdx.x == 0) TC_STAMP(0);
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     uint8_t* ring_a = smem;
@@ -277,12 +286,14 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = sh->tmem_base;
+    if (threadIdx.x == 0) TC_STAMP(1);
     // Programmatic dependent launch: everything above (barriers, tensor memory) touched no global data, so it may
     // run while the previous kernel of the stream is still finishing.  From here on the kernel reads what that
     // kernel wrote: wait for it (returns at once when the launch carried no such dependency), and let the next
     // kernel of the stream start its own set-up as soon as CTAs of this one retire.
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (threadIdx.x == 0) TC_STAMP(2);
 
     // ---------------------------------------------------------------- A producer
     if (warp == 0) {
@@ -383,6 +394,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                                 if (rank == 0) mbar_expect_tx(bar, 2 * a_bytes);
                                 tma_load_5d_pair(smem_u32(ring_a + (size_t)s * p.a_slot), &tm_a, bar, 0, w0 - pw, h0 - ph,
                                                  TF32 ? 2 * cb + (pass == 1) : cb, fz);
+                                if (item == cta_lin && dt == dt0 && cb == 0) TC_STAMP(3);
                             } else {
                                 mbar_expect_tx(bar, a_bytes);
                                 tma_load_5d(smem_u32(ring_a + (size_t)s * p.a_slot), &tm_a, bar, 0, w0 * stw - pw + dw * dlw,
@@ -506,9 +518,11 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                     const uint32_t d0 = d_first + (second ? (uint32_t)NB * p.NPAD : 0u);
                     const uint32_t acc_in = second ? accumulate2 : accumulate;
                     if (!(ok = mbar_wait(&sh->full_a[sa], pa, sh, p, SITE_A_FULL))) break;
+                    if (item == cta_lin && st == 0 && lane == 0 && iss == 0) TC_STAMP(4);
 #pragma unroll
                     for (int g = 0; g < STAGES; ++g) {
                         if (!(ok = mbar_wait(&sh->full_b[sb], pb, sh, p, SITE_B_FULL))) break;
+                        if (item == cta_lin && st == 0 && g == 0 && lane == 0 && iss == 0) TC_STAMP(5);
                         tc_fence_after();
                         if (elect_one()) {
 #pragma unroll
@@ -551,6 +565,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                 if (!ok) break;
                 if (elect_one()) { if (PAIR) tc_commit_pair(smem_u32(&sh->acc_full[acc])); else tc_commit(smem_u32(&sh->acc_full[acc])); }
                 __syncwarp();
+                if (item == cta_lin && lane == 0 && iss == 0) TC_STAMP(6);
                 if (++acc == p.ACC) { acc = 0; pacc ^= 1; }
             }
         } else
@@ -707,6 +722,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                 ok = mbar_wait(&sh->acc_full[acc], pacc, sh, p, SITE_ACC_FULL);
                 ok = __all_sync(0xffffffffu, ok);
                 if (!ok) break;
+                if (item == cta_lin && elected) TC_STAMP(7);
                 tc_fence_after();
                 const uint32_t t_acc = tmem_base + (uint32_t)(acc * ASETS * NB) * p.NPAD + ((uint32_t)(q * 32) << 16);
                 // TF32: was the second accumulator of the last pass used (at least two stages per pass)?
@@ -845,6 +861,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                         }
                     }
                 }
+                if (item == cta_lin && elected) TC_STAMP(8);
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) { if (PAIR) mbar_arrive_leader(smem_u32(&sh->acc_empty[acc])); else mbar_arrive(smem_u32(&sh->acc_empty[acc])); }
@@ -852,7 +869,10 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
             }
         };
         if (p.act) run_tiles(std::true_type{}); else run_tiles(std::false_type{});
-        if (p.epi_tma && elected) bulk_wait_all();   // all stores of this CTA are complete before it exits
+        // Before the CTA exits the stores must have finished READING its shared memory; their writes complete with
+        // the grid (which is what a dependent kernel waits for), so nothing here waits for them (0.8 us per launch).
+        if (p.epi_tma && elected) bulk_wait_read<0>();
+        if (elected) TC_STAMP(9);
     }
 
     // ---------------------------------------------------------------- stagers (cooperative staging, warps 8..11)
@@ -958,7 +978,9 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     // ---------------------------------------------------------------- teardown
     tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0) TC_STAMP(10);
     if (PAIR) cluster_sync_all();   // the leader's MMAs read the peer's shared memory and write its tensor memory
+    if (threadIdx.x == 0) TC_STAMP(11);
     if (warp == 3) {
         tc_fence_after();
         if (PAIR) asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(p.tmem_cols) : "memory");

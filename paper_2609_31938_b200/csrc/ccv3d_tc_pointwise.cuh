@@ -210,7 +210,7 @@ conv1x1_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_x,   // x as (pixe
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&sh->acc_empty[acc]));
         }
-        if (elected) bulk_wait_all();
+        if (elected) bulk_wait_read<0>();     // (the stores have read the staging buffers; their writes complete with the grid)
     }
 
     tc_fence_before();
