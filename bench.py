@@ -586,19 +586,25 @@ def hsplit_leg(dev):
     name = "cfg3_bf16_192"
     d = {k: v for k, v in si.CONFIGS[name].items() if k not in ("dtype", "x_dist")}
     N, Cin, Cout, T, H, W, k = d["N"], d["Cin"], d["Cout"], d["T"], d["H"], d["W"], d["k"]
-    gen = torch.Generator(device=dev).manual_seed(0)
-    rnd = lambda *shape, std=1.0: (torch.randn(*shape, device=dev, generator=gen) * std).to(torch.bfloat16)
-    w, b = rnd(Cout, Cin, *k, std=1.0 / math.sqrt(Cin * k[0] * k[1] * k[2])), rnd(Cout, std=math.sqrt(0.1))
+    # the seeded tensors of the headline workload; a rank's band, halo rows and slabs are row slices of them (one zero
+    # row above and below the image stands for the layer's zero padding at the image edge)
+    c = si.conv_case(**si.CONFIGS[name])
+    up = lambda a: torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
+    pad_rows = lambda t: torch.nn.functional.pad(t, (0, 0, 1, 1))
+    xp, cp = pad_rows(up(c["x"])), pad_rows(up(c["cache"]))          # row r of the image is row r + 1 here
+    w, b = up(c["w"]), up(c["b"])
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    out = {"workload": name, "note": "rank 1 of the world (halo rows on both sides of its slab). NCTHW: pack + slab assembly + layer "
-                                     "on the slab; resident: the ring call on the slab + pack and unpack of the output's halo "
-                                     "rows. Neighbour exchange (NCCL send/recv) not included"}
+    out = {"workload": name, "data": "seeded synthetic (row slices of the headline tensors)",
+           "note": "rank 1 of the world (halo rows on both sides of its slab). NCTHW: pack + slab assembly + layer "
+                   "on the slab; resident: the ring call on the slab + pack and unpack of the output's halo "
+                   "rows. Neighbour exchange (NCCL send/recv) not included"}
     for world in (2, 4, 8):
         layer = HSplitCausalConv3d(w, b, H, min(1, world - 1), world, transport=None)
         p = layer.plan
-        xb = rnd(N, Cin, T, p.rows, W)
-        cache = rnd(N, Cin, k[0] - 1, p.slab_rows, W)
-        halo_up, halo_down = rnd(N, Cin, T, p.top, W), rnd(N, Cin, T, p.bot, W)
+        xb = xp[:, :, :, p.r0 + 1:p.r1 + 1].contiguous()
+        cache = cp[:, :, :, p.r0 + 1 - p.top:p.r1 + 1 + p.bot].contiguous()
+        halo_up = xp[:, :, :, p.r0 + 1 - p.top:p.r0 + 1].contiguous()
+        halo_down = xp[:, :, :, p.r1 + 1:p.r1 + 1 + p.bot].contiguous()
 
         def rank_step():
             layer.pack(xb)
@@ -618,7 +624,8 @@ def hsplit_leg(dev):
         rl = HSplitRingConv3d(w, b, H, min(1, world - 1), world, transport=None)
         F = T + k[0] - 1
         rin, rout = rl.ring(N, Cin, F, W), rl.ring(N, Cout, T, W)
-        rin.buf.normal_()
+        rin.load(0, cache)
+        rin.load(k[0] - 1, xp[:, :, :, p.r0 + 1 - p.top:p.r1 + 1 + p.bot].contiguous())
         slot = [k[0] - 1]
 
         def ring_rank_step():
