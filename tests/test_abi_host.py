@@ -85,6 +85,7 @@ def test_null_and_misaligned_arguments():
     assert ccv.ccv3d_rows_copy(None, 4, 0, 4096, 4, 0, 1, 1, 16) == ccv.ERR_INVALID_ARG          # no destination
     assert ccv.ccv3d_rows_copy(4096, 4, 3, 8192, 4, 0, 1, 2, 16) == ccv.ERR_INVALID_ARG          # rows leave the plane
     assert ccv.ccv3d_workspace_bytes(None, 1, 1, 8, 8)[0] == ccv.ERR_INVALID_ARG
+    assert ccv.ccv3d_set_workspace(None, 4096, 1 << 20) == ccv.ERR_INVALID_ARG
     assert ccv.ccv3d_device_status(None)[0] == ccv.ERR_INVALID_ARG
     assert ccv.ccv3d_add_bf16(None, None, None, 16) == ccv.ERR_INVALID_ARG
     assert ccv.ccv3d_upsample_bf16(None, None, 1, 1, 1, 1, 1, 1) == ccv.ERR_INVALID_ARG

@@ -220,6 +220,14 @@ def test_short_cache_is_zero_history_in_front(ccv, dtype, flags, T):
     layer.close()
 
 
+def test_two_samples_on_the_one_kernel_schedule(ccv):
+    """N = 2 at a size that takes cooperative staging on CTA pairs: the batch is an outer loop of tiles and staging
+    tasks with a cache per sample; against the oracle, cache bit-exact, one launch."""
+    c = si.conv_case(2, 64, 192, 4, 160, 256, seed=19)
+    m, ctr = run_case(ccv, c)
+    assert ctr["tcgen05_bf16"] == 1 and ctr["kernel_launches"] == 3
+
+
 @pytest.mark.parametrize("Cin,Cout,W", [(64, 64, 160), (96, 48, 200)])   # 64-channel blocks; 32-channel blocks with a ragged 128-pixel task
 def test_bf16_tensor_core_cooperative_staging(ccv, Cin, Cout, W):
     """Large enough for the default schedule to stage inside the convolution kernel (four stager warps per CTA, a
