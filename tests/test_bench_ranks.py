@@ -36,3 +36,18 @@ def test_single_process_selftest():
     assert r.returncode == 0, r.stderr[-2000:]
     d = json.loads(r.stdout.strip().splitlines()[-1])
     assert d["n_gpus"] == 1 and abs(d["ms_per_step"] - 1.0) < 1e-9
+
+
+def test_gpus_flag_starts_its_own_ranks():
+    """`python bench.py --gpus 2` without torchrun: the script starts two ranks itself (here on CPU, gloo, through the
+    same self-test as above) and rank 0 prints the one line with n_gpus = 2."""
+    env = dict(os.environ, OMP_NUM_THREADS="2")
+    for k in ("WORLD_SIZE", "RANK", "LOCAL_RANK"):
+        env.pop(k, None)
+    r = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--steps", "4", "--selftest-dist"],
+                       cwd=ROOT, env=env, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1, r.stdout
+    d = json.loads(lines[0])
+    assert d["n_gpus"] == 2 and abs(d["ms_per_step"] - 1.25) < 1e-9
