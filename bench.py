@@ -56,6 +56,9 @@ TRAFFIC_BYTES_PER_LAUNCH = {
     ("cfg3_bf16_192", "ring"): 4 * (132.0e6 + 53.6e6),
     ("cfg3_bf16_192", "two_kernels"): 4 * (133.2e6 + 53.0e6),
     ("cfg4a_bf16_96", "one_kernel"): 4 * (434.2e6 + 476.5e6),   # profiles/conv3d_tcgen05_coop_96ch_352x640.md
+    ("cfg4a_bf16_96", "ring"): 4 * (260.4e6 + 143.4e6),         # profiles/conv3d_tcgen05_96out_352x640.md
+    ("cfg4b_bf16_192_96", "one_kernel"): 4 * (1058.2e6 + 846.2e6),
+    ("cfg4b_bf16_192_96", "ring"): 4 * (524.3e6 + 155.5e6),
     # profiles/conv1x1_tcgen05_192to96_352x640.md: x read once, 137 of the 173 MB of output written during the kernel
     ("cfg4c_bf16_pw_192_96", "pointwise"): 4 * (346.1e6 + 137.0e6),
 }
@@ -475,6 +478,7 @@ def other_configs_leg(dev, local):
             r_bytes = 2 * N * H * W * T * (Cin + Cout) + c["w"].nbytes
             row["resident"] = {**rst, "tflops": flops / (rst["ms_median"] * 1e-3) / 1e12, "clocks": rclk,
                                "roofline": roofline_of(flops, r_bytes, rst["ms_median"], peaks)}
+            row["resident"]["roofline"]["traffic"] = TRAFFIC_BYTES_PER_LAUNCH.get((name, "ring"))
             row["resident_ms_per_call"] = rst["ms_median"]
             row["resident_tflops"] = row["resident"]["tflops"]
             del rin, rout
