@@ -93,12 +93,16 @@ void make_plan_f32(const ccv3d_desc& d, TcPlan* pl) {
 // Taps per weight stage and ring depths that fit `budget` bytes of shared memory: a whole kernel row of taps per
 // stage when that stays small (so that a stage carries enough MMAs), at least two activation and two weight
 // stages, weight ring up to 8 deep, then a deeper activation ring with what is left.
-ccv3d_status size_pipeline(TcParams* p, size_t budget, bool per_tap, int kw) {
+// whole_kernel > 0: all kh*kw taps in one weight stage when that fits in 28 KB (narrow tiles of 32-channel blocks on CTA
+// pairs: a stage of one kernel row would carry only 6 MMAs per issuing warp).
+ccv3d_status size_pipeline(TcParams* p, size_t budget, bool per_tap, int kw, int whole_kernel = 0) {
     p->TPB = (!per_tap && (size_t)p->b_tap * kw <= 40960) ? kw : 1;
+    if (whole_kernel > 0 && !per_tap && (size_t)p->b_tap * whole_kernel <= 28672) p->TPB = whole_kernel;
     int SA = per_tap ? 3 : 2;
     for (;;) {
         p->b_slot = (uint32_t)align_up((uint64_t)p->b_tap * p->TPB, 1024);
         if ((size_t)SA * p->a_slot + 3 * (size_t)p->b_slot <= budget) break;
+        if (p->TPB > kw && kw > 1) { p->TPB = kw; continue; }
         if (p->TPB > 1) { p->TPB = 1; continue; }
         if ((size_t)SA * p->a_slot + 2 * (size_t)p->b_slot <= budget) break;
         return CCV3D_ERR_UNSUPPORTED;

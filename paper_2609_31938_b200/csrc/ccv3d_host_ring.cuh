@@ -161,7 +161,7 @@ ccv3d_status forward_ring(ccv3d_handle* h, const ccv3d_ring* in, int x_slot, int
     }
     const size_t fixed = 1024 + align_up(sizeof(TcShared), 128) + 2 * (size_t)p.e_slot;
     const size_t budget = SMEM_LIMIT - fixed;
-    s = size_pipeline(&p, budget, false, d.kw);
+    s = size_pipeline(&p, budget, false, d.kw, (pair && pl.KB == 32 && d.kh == 3 && d.kw == 3 && p.main_tiles == 0) ? 9 : 0);
     if (s != CCV3D_OK) return s;
     p.tmem_cols = pow2_cols((uint32_t)(NB * NPAD * ACC));
     if (p.tmem_cols > 512) return CCV3D_ERR_UNSUPPORTED;

@@ -124,6 +124,11 @@ ccv3d_status launch_pair_any(ccv3d_handle* h, const CUtensorMap& tm_a, const CUt
     // (a launch that ends in half-width items carries the weight map of those, see the kernel's B producer)
     ccv3d_status s = weight_map(h, p.main_tiles > 0 ? p.NPAD / 4 : p.NPAD / 2, &tm_w);
     if (s != CCV3D_OK) return s;
+    if (p.TPB == 9) {                       // all nine taps per weight stage: 32-channel blocks, narrow tiles
+        if (ks != 3 || dil != 1 || p.main_tiles > 0 || h->d.dtype == CCV3D_F32 || h->plan.KB != 32) return CCV3D_ERR_UNSUPPORTED;
+        if (nb == 2) return launch_tc_pair<32, 2, 3, 9, COOP>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
+        return launch_tc_pair<32, 1, 3, 9, COOP>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
+    }
 #define CCV3D_LAUNCH_PAIR(KBv, NBv)                                                                                        \
     do {                                                                                                                   \
         if (ks == 3 && p.TPB == 3) return launch_tc_pair<KBv, NBv, 3, 3, COOP>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st); \
@@ -383,7 +388,8 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     // leave room for staging blocks to be resident next to a convolution CTA when the two overlap
     const size_t limit = nbands > 1 ? SMEM_LIMIT - STAGE_COEXIST_BYTES : SMEM_LIMIT;
     const size_t budget = limit - fixed;
-    s = size_pipeline(&p, budget, per_tap != 0 || phased, phased ? 1 : d.kw);   // (phase order: one tap per weight stage)
+    const bool tpb9 = pair && !f32 && !phased && pl.KB == 32 && d.kh == 3 && d.kw == 3 && d.dilation[1] == 1 && d.dilation[2] == 1;
+    s = size_pipeline(&p, budget, per_tap != 0 || phased, phased ? 1 : d.kw, tpb9 ? 9 : 0);   // (phase order: one tap per weight stage)
     if (s != CCV3D_OK) return s;
     p.tmem_cols = pow2_cols((uint32_t)(asets * NB * NPAD * ACC));
     if (p.tmem_cols > 512) return CCV3D_ERR_UNSUPPORTED;
