@@ -51,3 +51,22 @@ def test_gpus_flag_starts_its_own_ranks():
     assert len(lines) == 1, r.stdout
     d = json.loads(lines[0])
     assert d["n_gpus"] == 2 and abs(d["ms_per_step"] - 1.25) < 1e-9
+
+
+def test_useful_tap_fraction_matches_the_interval_algebra():
+    """The bench's useful-FLOP count of a first-chunk call: the (output frame, temporal tap) pairs whose source frame
+    exists, 1/3, 3/6 and 9/12 of them at T = 1, 2, 4 with kt = 3 and no history (the worked cases of Eq. (4)), all of
+    them with a full cache; and the same count from the oracle's interval routine."""
+    sys.path.insert(0, ROOT)
+    import bench
+    import oracle
+    assert abs(bench.useful_tap_fraction(1, 3, 0) - 1 / 3) < 1e-12
+    assert abs(bench.useful_tap_fraction(2, 3, 0) - 3 / 6) < 1e-12
+    assert abs(bench.useful_tap_fraction(4, 3, 0) - 9 / 12) < 1e-12
+    assert bench.useful_tap_fraction(4, 3, 2) == 1.0 and bench.useful_tap_fraction(3, 1, 0) == 1.0
+    for kt in (1, 2, 3):
+        for cf in range(kt):
+            for T in (1, 2, 4, 5):
+                _, taps = oracle.tap_intervals(kt, cf, T)
+                pairs = sum(max(0, oh - ol) for (_, ol, oh, _, _) in taps)
+                assert abs(bench.useful_tap_fraction(T, kt, cf) - pairs / (T * kt)) < 1e-12
