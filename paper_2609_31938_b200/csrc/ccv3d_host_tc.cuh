@@ -398,6 +398,9 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     p.wq = (const uint8_t*)h->wp;
     p.out = out;
     p.status = h->status;
+#ifdef CCV3D_DEV_TRACE
+    p.trace = getenv("CCV3D_TC_TRACE") ? (unsigned long long*)strtoull(getenv("CCV3D_TC_TRACE"), nullptr, 0) : nullptr;
+#endif
     if (p.epi_tma) {
         s = encode_out_map(h, out, N, To, Ho, Wo, TW, p.ECH);
         if (s != CCV3D_OK) return s;

@@ -114,6 +114,12 @@ __device__ __forceinline__ TileView tile_view(const TcParams& p, int u) {
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, TcShared* sh, const TcParams& p, uint32_t site) {
     const uint32_t b = smem_u32(bar);
     if (mbar_try_wait(b, parity)) return true;
+#ifdef CCV3D_DEV_TRACE
+    // dev builds: cycles CTA 0 spends in waits, summed per wait site (words 16.. of the trace buffer)
+    const long long tw0 = clock64();
+    struct Acc { const TcParams& p; uint32_t site; long long t; __device__ ~Acc() {
+        if (p.trace && blockIdx.x == 0 && (threadIdx.x & 31) == 0) atomicAdd(p.trace + 16 + site, (unsigned long long)(clock64() - t)); } } acc_{p, site, tw0};
+#endif
     long long t0 = 0;
     for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(b, parity)) return true;
