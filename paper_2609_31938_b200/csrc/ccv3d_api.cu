@@ -73,6 +73,7 @@ struct ccv3d_handle {
     CUtensorMap tm_a;
     ShapeKey tm_a_key;
     CUtensorMap tm_o;
+    StagerMaps stg_maps; // cooperative staging: raw NCTHW views of x, the cache and the new cache (per call)
     CUtensorMap tm_w[2]; // CTA pairs: 2-D maps over the packed weights (half-tile and quarter-tile boxes)
     int tm_w_rows[2];    // box height each was encoded for (0 = not yet)
     long long wait_limit_clk;

@@ -204,6 +204,40 @@ ccv3d_status encode_out_map(ccv3d_handle* h, void* out, int N, int T, int H, int
     return r == CUDA_SUCCESS ? CCV3D_OK : CCV3D_ERR_CUDA;
 }
 
+// Raw view of an NCTHW tensor [N, C, Fr, H, W] (BF16) for the stager warps of the cooperative schedule: boxes of
+// [32 channels][64 pixels] of one image row, 128-byte swizzle.  Needs W % 8 == 0 and a 16-byte aligned base.
+ccv3d_status encode_raw_map(ccv3d_handle* h, CUtensorMap* tm, const void* base, int N, int C, int Fr, int H, int W) {
+    const uint64_t row = 2ull * W;
+    cuuint64_t dims[5] = {(cuuint64_t)W, (cuuint64_t)H, (cuuint64_t)Fr, (cuuint64_t)C, (cuuint64_t)N};
+    cuuint64_t strides[4] = {row, row * H, row * H * Fr, row * H * Fr * C};
+    cuuint32_t box[5] = {64, 1, 1, 32, 1};
+    cuuint32_t es[5] = {1, 1, 1, 1, 1};
+    CUresult r = h->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 5, const_cast<void*>(base), dims, strides, box, es,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS ? CCV3D_OK : CCV3D_ERR_CUDA;
+}
+
+// The three raw views of a cooperative call (absent tensors get a copy of x's view: never used for a transfer).
+ccv3d_status encode_stager_maps(ccv3d_handle* h, const void* x, const void* cache, int cf, void* new_cache, int N, int T, int H,
+                                int W) {
+    const int tc = hist_len(h->d);
+    ccv3d_status s = encode_raw_map(h, &h->stg_maps.x, x, N, h->d.cin, T, H, W);
+    if (s == CCV3D_OK && cf) s = encode_raw_map(h, &h->stg_maps.cache, cache, N, h->d.cin, cf, H, W);
+    if (s == CCV3D_OK && new_cache && tc) s = encode_raw_map(h, &h->stg_maps.nc, new_cache, N, h->d.cin, tc, H, W);
+    if (s != CCV3D_OK) return s;
+    if (!cf) h->stg_maps.cache = h->stg_maps.x;
+    if (!(new_cache && tc)) h->stg_maps.nc = h->stg_maps.x;
+    return CCV3D_OK;
+}
+
+// Can the stager warps fetch these tensors by TMA?  16-byte aligned bases, rows of whole 16-byte pieces, strides that fit.
+inline bool raw_maps_ok(const ccv3d_handle* h, const void* x, const void* cache, const void* new_cache, int T, int H, int W) {
+    const int tc = hist_len(h->d);
+    return W % 8 == 0 && ((uintptr_t)x & 15) == 0 && ((uintptr_t)cache & 15) == 0 && ((uintptr_t)new_cache & 15) == 0 &&
+           2ull * W * H * (uint64_t)(T > tc ? T : tc) * h->d.cin < (1ull << 40);
+}
+
 uint64_t tc_workspace_bytes(const ccv3d_handle* h, int N, int T, int H, int W) {
     const int F = hist_len(h->d) + T;
     if (h->d.dtype == CCV3D_F32) return (uint64_t)N * F * h->plan.cin_pad * H * W * 8;   // values and remainders, FP32

@@ -22,7 +22,7 @@ ccv3d_status launch_tc_coop(ccv3d_handle* h, const TcParams& p, const StageParam
     attr[0].val.cooperative = 1;
     cfg.attrs = attr;
     cfg.numAttrs = h->coop_launch ? 1 : 0;
-    if (cudaLaunchKernelEx(&cfg, kern, h->tm_a, h->tm_a, h->tm_o, p, sp) != cudaSuccess) return cuda_fail();
+    if (cudaLaunchKernelEx(&cfg, kern, h->tm_a, h->tm_a, h->tm_o, p, sp, h->stg_maps) != cudaSuccess) return cuda_fail();
     if (cudaGetLastError() != cudaSuccess) return cuda_fail();
     h->ctr.kernel_launches++;
     return CCV3D_OK;
@@ -35,7 +35,7 @@ ccv3d_status launch_tc(ccv3d_handle* h, const TcParams& p, size_t smem, int grid
         return cuda_fail();
     StageParams nosp;
     memset(&nosp, 0, sizeof(nosp));
-    kern<<<grid, TC_THREADS, smem, st>>>(h->tm_a, h->tm_a, h->tm_o, p, nosp);
+    kern<<<grid, TC_THREADS, smem, st>>>(h->tm_a, h->tm_a, h->tm_o, p, nosp, h->stg_maps);
     if (cudaGetLastError() != cudaSuccess) return cuda_fail();
     h->ctr.kernel_launches++;
     return CCV3D_OK;
@@ -86,7 +86,7 @@ ccv3d_status launch_tc_pair(ccv3d_handle* h, const CUtensorMap& tm_a, const CUte
     }
     cfg.attrs = attr;
     cfg.numAttrs = ((COOP && h->coop_launch) || (!COOP && h->pdl)) ? 2 : 1;
-    if (cudaLaunchKernelEx(&cfg, kern, tm_a, tm_w, tm_o, p, sp) != cudaSuccess) return cuda_fail();
+    if (cudaLaunchKernelEx(&cfg, kern, tm_a, tm_w, tm_o, p, sp, h->stg_maps) != cudaSuccess) return cuda_fail();
     if (cudaGetLastError() != cudaSuccess) return cuda_fail();
     h->ctr.kernel_launches++;
     return CCV3D_OK;
@@ -380,17 +380,36 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     // than four stager warps per SM keep up with - measured 1.73 ms against 1.25 ms for the two kernels at 96->192,
     // stride 2, from 704x1280)
     const bool coop = nbands == 1 && !per_tap && !phased && (!general || d.stride[0] == 1) && !f32 &&
-                      !(d.flags & CCV3D_FLAG_TWO_KERNELS) && W % 8 == 0 && in_bands <= MAX_COOP_BANDS && tiles_h >= 4 &&
+                      !(d.flags & CCV3D_FLAG_TWO_KERNELS) && raw_maps_ok(h, x, cache, new_cache, T, H, W) &&
+                      in_bands <= MAX_COOP_BANDS && tiles_h >= 4 &&
                       // fewer than eight waves of tiles: two kernels (the first tiles of a cooperative launch wait for two
                       // whole bands, and measured at six waves it is 15 % behind; level at seven, ahead from twelve)
                       (int64_t)N * tiles_h * p.tiles_w * To * NT * (pair ? 2 : 1) >= 8LL * h->sm_count;
-    size_t fixed = 1024 /*alignment slack*/ + align_up(sizeof(TcShared), 128) + 2 * (size_t)p.e_slot + (coop ? 9216 : 0);
+    // Cooperative staging: the stager team keeps stg_slots tasks of 8 KB in flight.  Narrow tiles (two pixel blocks per
+    // CTA, at most 128 output channels) stage twice as many input bytes per MMA cycle as wide ones: three slots, since
+    // with two the team, bound by the latency of its fetches, finishes last (192->96 at 704x1280: 4.34 M cycles against
+    // 3.35 M); wide tiles two, and a third only when that costs the rings nothing (192->192 at 352x640 loses 3 % when the
+    // third slot takes the fourth weight slot's place).
+    p.stg_slots = coop ? (NB == 2 ? 3 : 2) : 0;
+    size_t fixed = 1024 /*alignment slack*/ + align_up(sizeof(TcShared), 128) + 2 * (size_t)p.e_slot +
+                   (size_t)p.stg_slots * STAGER_SLOT_BYTES;
     // leave room for staging blocks to be resident next to a convolution CTA when the two overlap
     const size_t limit = nbands > 1 ? SMEM_LIMIT - STAGE_COEXIST_BYTES : SMEM_LIMIT;
     const size_t budget = limit - fixed;
     const bool tpb9 = pair && !f32 && !phased && pl.KB == 32 && d.kh == 3 && d.kw == 3 && d.dilation[1] == 1 && d.dilation[2] == 1;
     s = size_pipeline(&p, budget, per_tap != 0 || phased, phased ? 1 : d.kw, tpb9 ? 9 : 0);   // (phase order: one tap per weight stage)
     if (s != CCV3D_OK) return s;
+    if (coop && p.stg_slots < 3 && (size_t)p.SA * p.a_slot + (size_t)p.SB * p.b_slot + STAGER_SLOT_BYTES <= budget) {
+        ++p.stg_slots;
+        fixed += STAGER_SLOT_BYTES;
+    }
+    // ... and with narrow tiles a third activation slot is worth a weight slot when four or more of those are left: next to
+    // the stagers' traffic it is the halo tiles that arrive late (96->96 at 704x1280: 1.95 M cycles with 2 + 4 slots,
+    // 1.86 M with 3 + 3)
+    if (coop && NB == 2 && p.SA == 2 && p.SB >= 4 && 3 * (size_t)p.a_slot + (size_t)(p.SB - 1) * p.b_slot <= budget) {
+        p.SA = 3;
+        --p.SB;
+    }
     p.tmem_cols = pow2_cols((uint32_t)(asets * NB * NPAD * ACC));
     if (p.tmem_cols > 512) return CCV3D_ERR_UNSUPPORTED;
     p.wait_limit_clk = h->wait_limit_clk;
@@ -421,6 +440,8 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
         if (cudaMemsetAsync(h->band_ctr, 0, (size_t)in_bands * sizeof(unsigned int), st) != cudaSuccess) return cuda_fail();
         p.band_ctr = h->band_ctr;
         p.nbands = in_bands;
+        s = encode_stager_maps(h, x, cache, cf, sp.new_cache, N, T, H, W);
+        if (s != CCV3D_OK) return s;
         p.ty_begin = 0;
         p.tiles_h = tiles_h;
         const int64_t total = (int64_t)N * tiles_h * p.tiles_w * To * NT;
@@ -533,7 +554,7 @@ ccv3d_status launch_fused(ccv3d_handle* h, const CUtensorMap& tm_x, const CUtens
         return cuda_fail();
     StageParams nosp;
     memset(&nosp, 0, sizeof(nosp));
-    kern<<<grid, TC_THREADS_FUSED, smem, st>>>(tm_x, tm_c, tm_o, p, nosp);
+    kern<<<grid, TC_THREADS_FUSED, smem, st>>>(tm_x, tm_c, tm_o, p, nosp, h->stg_maps);
     if (cudaGetLastError() != cudaSuccess) return cuda_fail();
     h->ctr.kernel_launches++;
     return CCV3D_OK;
@@ -785,7 +806,7 @@ ccv3d_status launch_tc_with_maps(ccv3d_handle* h, const CUtensorMap& tm_a, const
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = h->pdl ? 1 : 0;
-    if (cudaLaunchKernelEx(&cfg, kern, tm_a, tm_a, tm_o, p, nosp) != cudaSuccess) return cuda_fail();
+    if (cudaLaunchKernelEx(&cfg, kern, tm_a, tm_a, tm_o, p, nosp, h->stg_maps) != cudaSuccess) return cuda_fail();
     if (cudaGetLastError() != cudaSuccess) return cuda_fail();
     h->ctr.kernel_launches++;
     return CCV3D_OK;

@@ -39,6 +39,7 @@ struct TcParams {
     long long wait_limit_clk; // bound of every mbarrier wait, in SM clocks
     unsigned int* band_ctr;   // cooperative staging: per 16-row band, the number of CTAs that have staged their share
     int nbands;               // cooperative staging: 16-row bands of the input image
+    int stg_slots;            // cooperative staging: raw slots (tasks in flight) of the stager team, 2..STAGER_MAX_SLOTS
     // general geometry (Eq. (2) with the layer's own padding and dilation, Eq. (1) with d_t); when `general` is 0
     // the kernel uses pad = (k-1)/2 and unit dilation.  H and W above are the OUTPUT extents; the input extents
     // only live in the tensor map.  Spatial stride > 1 is served by the per-tap mode with a strided tensor map.
@@ -85,6 +86,8 @@ struct TcShared {  // placed after the rings
     uint64_t full_b[TC_MAX_STAGES], empty_b[TC_MAX_STAGES];
     uint64_t acc_full[4], acc_empty[4];   // (the convolution kernel uses two, the 1x1x1 streaming kernel up to four)
     uint64_t raw_full[2], raw_empty[2];
+    uint64_t stg_full[STAGER_MAX_SLOTS];  // cooperative staging: a task's raw boxes have landed
+    StagerRec stg_rec[STAGER_MAX_SLOTS];
     uint32_t tmem_base;
     volatile int abort_flag;
     alignas(16) float bias_s[TC_BIAS_SMEM];   // the layer's padded bias when it fits (the epilogue reads it once per element)
@@ -113,13 +116,14 @@ __device__ __forceinline__ TileView tile_view(const TcParams& p, int u) {
 // Bounded wait.  Returns false when the limit expired or another role of this CTA aborted.
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, TcShared* sh, const TcParams& p, uint32_t site) {
     const uint32_t b = smem_u32(bar);
-    if (mbar_try_wait(b, parity)) return true;
 #ifdef CCV3D_DEV_TRACE
-    // dev builds: cycles CTA 0 spends in waits, summed per wait site (words 16.. of the trace buffer)
+    // dev builds: cycles CTA 0 spends in waits, summed per wait site (words 16.. of the trace buffer); the first try is
+    // inside the measured span, since the hardware may hold a try_wait for a while before it answers
     const long long tw0 = clock64();
     struct Acc { const TcParams& p; uint32_t site; long long t; __device__ ~Acc() {
         if (p.trace && blockIdx.x == 0 && (threadIdx.x & 31) == 0) atomicAdd(p.trace + 16 + site, (unsigned long long)(clock64() - t)); } } acc_{p, site, tw0};
 #endif
+    if (mbar_try_wait(b, parity)) return true;
     long long t0 = 0;
     for (uint32_t it = 1;; ++it) {
         if (mbar_try_wait(b, parity)) return true;
@@ -186,6 +190,185 @@ __device__ __forceinline__ uint32_t epi_pair(float a0, float a1, uint32_t res_pa
     return *reinterpret_cast<const uint32_t*>(&o);
 }
 
+// The stager warps of the cooperative schedule (warps 8..11 of a CTA): the staging pass - same tile move as
+// stage_frames_kernel, cache update included - band by band of 16 image rows; every finished band is signalled with a
+// fence and one atomic per CTA.
+// Inside a band the tasks ([KB channels][SPX pixels] of one image row of one Z frame, 8 KB) are ordered (sample, frame,
+// channel block, row, chunk of the row) and CTA k takes the k-th of gridDim.x contiguous runs, so that the next task is an
+// odometer step away (a team of four warps is bound by its own instruction stream: decoding every task with divisions
+// cost more than moving it).  Thread 0 of the team keeps p.stg_slots tasks in flight: it leaves a task's record in
+// shared memory and fetches its two raw boxes by TMA; the team waits for a task's boxes, transposes them with
+// ldmatrix.trans (each lane ends up with 8 consecutive channels of one pixel) and writes them channels-last.  Frames
+// of the updated cache leave the same raw boxes by TMA store.  One barrier per task: it shares the outcome of the wait
+// and tells thread 0 that everybody has finished reading the previous task's slot.
+template <int KB>
+__device__ __forceinline__ void run_stagers(const TcParams& p, const StageParams& sp, const StagerMaps* maps, uint32_t raw0,
+                                            TcShared* sh) {
+    const int tid = threadIdx.x - 256;
+    const int lane = tid & 31, swp = tid >> 5;
+    constexpr int SPX = StagerGeom<KB>::PX;
+    const int nchunks = (sp.W + SPX - 1) / SPX;
+    const int nf = sp.tc + sp.T - sp.f_begin;
+    const int R = p.stg_slots;
+    const int64_t HW = (int64_t)sp.H * sp.W;
+    // this CTA's run of tasks in band b: [first, last)
+    auto band_run = [&](int b, int& first, int& last, int& rows) {
+        rows = (sp.H - 16 * b < 16) ? sp.H - 16 * b : 16;
+        const int64_t ntask = (int64_t)sp.N * nf * sp.CB * rows * nchunks;
+        first = (int)(ntask * blockIdx.x / gridDim.x);
+        last = (int)(ntask * (blockIdx.x + 1) / gridDim.x);
+    };
+    // ldmatrix roles: lane l addresses row l%8 of matrix l/8; a row is one channel's 8 pixels.  Matrix j takes, from
+    // each of the four channel octets, the channel pair (octet + j) mod 4, so that its eight rows fall on eight
+    // different 16-byte columns of the swizzled box (no bank conflict) and lane (pixel, octet q) receives the four
+    // pairs of octet q, rotated by q.
+    const int mj = lane >> 3, qq = (lane & 7) >> 1;
+    const int cl = 8 * qq + 2 * ((qq + mj) & 3) + (lane & 1);
+    const uint32_t lane_off = (uint32_t)cl * 128u, c7 = (uint32_t)(cl & 7);
+    const int pq = lane & 3, pp = lane >> 2;
+
+    // thread 0: a cursor over this CTA's tasks
+    struct Cursor { int b, left, wc, hr, cb, fi, n, rows; };
+    auto open_band = [&](Cursor& c) {
+        while (c.b < p.nbands) {
+            int first, last;
+            band_run(c.b, first, last, c.rows);
+            if (last > first) {
+                int r = first;
+                c.wc = r % nchunks; r /= nchunks;
+                c.hr = r % c.rows; r /= c.rows;
+                c.cb = r % sp.CB; r /= sp.CB;
+                c.fi = r % nf;
+                c.n = r / nf;
+                c.left = last - first;
+                return;
+            }
+            ++c.b;
+        }
+        c.left = 0;
+    };
+    auto advance = [&](Cursor& c) {
+        if (--c.left == 0) { ++c.b; open_band(c); return; }
+        if (++c.wc == nchunks) {
+            c.wc = 0;
+            if (++c.hr == c.rows) {
+                c.hr = 0;
+                if (++c.cb == sp.CB) {
+                    c.cb = 0;
+                    if (++c.fi == nf) { c.fi = 0; ++c.n; }
+                }
+            }
+        }
+    };
+    struct Src { const CUtensorMap* tm; int fr; bool present; };
+    auto source = [&](int f) {                             // Z frame f: x, or the cache (oldest first), or absent history
+        Src s;
+        s.tm = &maps->x; s.fr = f - sp.tc;
+        if (f < sp.tc) { s.tm = &maps->cache; s.fr = f - (sp.tc - sp.cf); }
+        s.present = f >= sp.tc || (sp.cache && s.fr >= 0);
+        return s;
+    };
+    Cursor it = {0, 0, 0, 0, 0, 0, 0, 0};
+    auto issue = [&](int slot) {
+        if (it.left == 0) return;
+        const int f = sp.f_begin + it.fi, h = 16 * it.b + it.hr, n = it.n;
+        const Src s = source(f);
+        StagerRec rec;
+        rec.w0 = it.wc * SPX; rec.h = h; rec.n = n; rec.c0 = it.cb * KB;
+        rec.dst = sp.zs + ((((int64_t)n * (sp.tc + sp.T) + f) * sp.CB + it.cb) * HW + (int64_t)h * sp.W + rec.w0) * KB;
+        const int jc = f - sp.T;                           // new_cache[j] = Z[T + j]
+        rec.fr_nc = (sp.new_cache && jc >= 0 && jc < sp.tc) ? jc : -1;
+        rec.present = s.present ? 1 : 0;
+        sh->stg_rec[slot] = rec;
+        const uint32_t bar = smem_u32(&sh->stg_full[slot]);
+        if (s.present) {
+            // (32-channel blocks: the second box holds pixels w0+64..; left out when it lies beyond the row)
+            const bool two = KB == 64 || rec.w0 + 64 < sp.W;
+            const uint32_t dst = raw0 + (uint32_t)slot * STAGER_SLOT_BYTES;
+            mbar_expect_tx(bar, two ? STAGER_SLOT_BYTES : STAGER_SLOT_BYTES / 2);
+            tma_load_5d(dst, s.tm, bar, rec.w0, h, s.fr, rec.c0, n);
+            if (KB == 64) tma_load_5d(dst + 4096, s.tm, bar, rec.w0, h, s.fr, rec.c0 + 32, n);
+            else if (two) tma_load_5d(dst + 4096, s.tm, bar, rec.w0 + 64, h, s.fr, rec.c0, n);
+        } else {
+            mbar_arrive(bar);
+        }
+        advance(it);
+    };
+    if (tid == 0) {
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&maps->x) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&maps->cache) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&maps->nc) : "memory");
+        open_band(it);
+        for (int s = 0; s < R; ++s) issue(s);
+    }
+    int slot = 0, prev = R - 1;
+    uint32_t par = 0;
+    bool first_task = true, ok = true;
+    for (int b = 0; ok && b < p.nbands; ++b) {
+        int first, last, rows;
+        band_run(b, first, last, rows);
+        for (int task = first; task < last; ++task) {
+            ok = stager_bar_and(mbar_wait(&sh->stg_full[slot], par, sh, p, SITE_RAW_FULL));
+            if (!ok) break;
+            if (tid == 0 && !first_task) {
+                bulk_wait_read<0>();                       // (a cache frame's stores out of the previous slot)
+                issue(prev);
+            }
+            first_task = false;
+            const StagerRec rec = sh->stg_rec[slot];
+            const uint32_t src = raw0 + (uint32_t)slot * STAGER_SLOT_BYTES;
+            if (rec.present) {
+                if (tid == 0 && rec.fr_nc >= 0) {
+                    tma_store_5d(&maps->nc, src, rec.w0, rec.h, rec.fr_nc, rec.c0, rec.n);
+                    if (KB == 64) tma_store_5d(&maps->nc, src + 4096, rec.w0, rec.h, rec.fr_nc, rec.c0 + 32, rec.n);
+                    else if (rec.w0 + 64 < sp.W) tma_store_5d(&maps->nc, src + 4096, rec.w0 + 64, rec.h, rec.fr_nc, rec.c0, rec.n);
+                    bulk_commit();
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const int u = swp * 4 + i, o = u & 7, hb = u >> 3;   // pixel octet, box of the slot
+                    uint32_t f[4];
+                    ldmatrix_x4_trans(src + (uint32_t)hb * 4096u + lane_off + ((((uint32_t)o) ^ c7) << 4), f);
+                    // f[j] = channel pair (pq + j) mod 4 of octet pq: rotate into channel order
+                    uint32_t g0 = (pq & 1) ? f[3] : f[0], g1 = (pq & 1) ? f[0] : f[1], g2 = (pq & 1) ? f[1] : f[2],
+                             g3 = (pq & 1) ? f[2] : f[3];
+                    if (pq & 2) { const uint32_t t0 = g0, t1 = g1; g0 = g2; g1 = g3; g2 = t0; g3 = t1; }
+                    const int px = (KB == 64 ? 0 : 64 * hb) + 8 * o + pp;
+                    const int ch = (KB == 64 ? 32 * hb : 0) + 8 * pq;
+                    if (rec.w0 + px < sp.W) *reinterpret_cast<uint4*>(rec.dst + (int64_t)px * KB + ch) = make_uint4(g0, g1, g2, g3);
+                }
+            } else {
+                // absent history: zeros, also into the updated cache when the frame belongs to it
+                const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+                for (int i = tid; i < SPX * (KB / 8); i += 128) {
+                    const int px = i / (KB / 8), oc = i % (KB / 8);
+                    if (rec.w0 + px < sp.W) *reinterpret_cast<uint4*>(rec.dst + (int64_t)px * KB + oc * 8) = z;
+                }
+                if (rec.fr_nc >= 0)
+                    for (int i = tid; i < KB * (SPX / 8); i += 128) {
+                        const int c = rec.c0 + i / (SPX / 8), w = rec.w0 + (i % (SPX / 8)) * 8;
+                        if (c < sp.Cin && w < sp.W)
+                            *reinterpret_cast<uint4*>(sp.new_cache + (((int64_t)rec.n * sp.Cin + c) * sp.tc + rec.fr_nc) * HW +
+                                                      (int64_t)rec.h * sp.W + w) = z;
+                    }
+            }
+            prev = slot;
+            if (++slot == R) { slot = 0; par ^= 1; }
+        }
+        if (!ok) break;
+        __threadfence();                                   // this thread's stores are visible GPU-wide ...
+        stager_bar();                                      // ... for all 128 stager threads, before the band is signalled
+        if (tid == 0) atomicAdd(p.band_ctr + b, 1u);
+    }
+    // the stores of cache frames must have finished READING shared memory before the CTA exits; their writes complete
+    // with the grid
+    if (tid == 0) bulk_wait_read<0>();
+    if (!ok && tid == 0) drain_delay();
+#ifdef CCV3D_DEV_TRACE
+    if (tid == 0 && p.trace && blockIdx.x == 0) p.trace[12] = clock64();
+#endif
+}
+
 // KB: input channels per K block (64 -> 128-byte swizzle, 32 -> 64-byte swizzle).  NB: 128-pixel blocks per tile.
 // KS/TPBC: compile-time spatial kernel size (kh = kw = KS) and taps per weight stage, which turn the tap loop
 // into straight-line code with immediate descriptor offsets; KS = 0 keeps everything run-time (any odd kh, kw,
@@ -218,7 +401,8 @@ __global__ void __launch_bounds__((FUSED || COOP) ? TC_THREADS_FUSED : TC_THREAD
 conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged activations (c, w, h, cb, n*F+f), or x
                       const __grid_constant__ CUtensorMap tm_c,   // fused mode: the cache; PAIR: the packed weights
                       const __grid_constant__ CUtensorMap tm_o,   // out (w, h, t, co, n); used when p.epi_tma
-                      const TcParams p, const StageParams sp) {
+                      const TcParams p, const StageParams sp,
+                      const __grid_constant__ StagerMaps smaps) {  // COOP: raw views of x, the cache and the new cache
     static_assert(!(FUSED && COOP), "one or the other");
     static_assert(!FUSED || KB == 32, "the fused mode transposes 32-channel blocks");
     static_assert(!TF32 || (KB == 64 && !FUSED && !COOP), "FP32 layers: 128-byte rows, plain variant");
@@ -253,8 +437,8 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     uint8_t* epi_buf = ring_b + (size_t)p.SB * p.b_slot;
     uint8_t* ring_raw = epi_buf + (p.epi_tma ? 2 * (size_t)p.e_slot : 0);
     uint8_t* dummy = ring_raw + (FUSED ? 2 * (size_t)p.raw_slot : 0);   // 2 KB sink for the unused rows of edge blocks
-    uint32_t* coop_tile = reinterpret_cast<uint32_t*>(ring_raw);          // COOP: the stagers' transposition tile (<= 9216 bytes)
-    TcShared* sh = reinterpret_cast<TcShared*>(dummy + (FUSED ? 2048 : 0) + (COOP ? 9216 : 0));
+    // (COOP: ring_raw holds the stagers' raw slots, p.stg_slots of STAGER_SLOT_BYTES, 1024-byte aligned like every ring)
+    TcShared* sh = reinterpret_cast<TcShared*>(dummy + (FUSED ? 2048 : 0) + (COOP ? (size_t)p.stg_slots * STAGER_SLOT_BYTES : 0));
 
     const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);  // provably warp-uniform
     const int lane = threadIdx.x & 31;
@@ -269,6 +453,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     if (threadIdx.x == 0) {
         for (int i = 0; i < p.SA; ++i) { mbar_init(smem_u32(&sh->full_a[i]), FUSED ? 4 : 1); mbar_init(smem_u32(&sh->empty_a[i]), NI); }
         for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&sh->raw_full[i]), 1); mbar_init(smem_u32(&sh->raw_empty[i]), 4); }
+        if (COOP) for (int i = 0; i < STAGER_MAX_SLOTS; ++i) mbar_init(smem_u32(&sh->stg_full[i]), 1);
         for (int i = 0; i < p.SB; ++i) { mbar_init(smem_u32(&sh->full_b[i]), 1); mbar_init(smem_u32(&sh->empty_b[i]), NI); }
         for (int i = 0; i < 2; ++i) { mbar_init(smem_u32(&sh->acc_full[i]), NI); mbar_init(smem_u32(&sh->acc_empty[i]), PAIR ? 8 : 4); }
         sh->abort_flag = 0;
@@ -368,6 +553,9 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                             } else __nanosleep(200);
                         }
                         if (!ok) break;
+#ifdef CCV3D_DEV_TRACE
+                        if (p.trace && blockIdx.x == 0) atomicAdd(p.trace + 16 + SITE_BAND, (unsigned long long)(clock64() - t0));
+#endif
                         asm volatile("fence.proxy.async;" ::: "memory");   // other SMs' generic writes -> this SM's TMA reads
                     }
                 }
@@ -882,44 +1070,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     }
 
     // ---------------------------------------------------------------- stagers (cooperative staging, warps 8..11)
-    if (COOP && warp >= 8) {
-        const int tid = threadIdx.x - 256;
-        constexpr int SPX = StagerGeom<KB>::PX;
-        const int nchunks = (sp.W + SPX - 1) / SPX;
-        const int nf = sp.tc + sp.T - sp.f_begin;
-        // Stagers wait on nothing but their own named barrier, so they always run to completion (also when a
-        // consumer role of some CTA has given up on a wait): every thread of the four warps takes every branch.
-        for (int b = 0; b < p.nbands; ++b) {
-            const int h_lo = 16 * b;
-            const int rows = (sp.H - h_lo < 16) ? sp.H - h_lo : 16;
-            const int ntask = sp.N * nf * sp.CB * rows * nchunks;
-            constexpr int G = 4;                             // tasks whose loads are in flight together (32 KB per CTA; 6 would spill)
-            for (int task0 = blockIdx.x; task0 < ntask; task0 += G * gridDim.x) {
-                StageTask tk[G];
-                uint4 val[G][StagerGeom<KB>::NLD];
-#pragma unroll
-                for (int g = 0; g < G; ++g) {
-                    const int task = task0 + g * gridDim.x;
-                    if (task < ntask) {
-                        int r = task;
-                        const int wc = r % nchunks; r /= nchunks;
-                        const int h = h_lo + r % rows; r /= rows;
-                        const int cb = r % sp.CB; r /= sp.CB;
-                        const int f = sp.f_begin + r % nf;
-                        const int n = r / nf;
-                        tk[g] = make_stage_task(sp, KB, n, f, cb, h, wc * SPX);
-                        stage_task_load<KB>(sp, tk[g], tid, val[g]);
-                    }
-                }
-#pragma unroll
-                for (int g = 0; g < G; ++g)
-                    if (task0 + g * gridDim.x < ntask) stage_task_store<KB>(sp, tk[g], tid, val[g], coop_tile);
-            }
-            __threadfence();                               // this thread's stores are visible GPU-wide ...
-            stager_bar();                                  // ... for all 128 stager threads, before the band is signalled
-            if (tid == 0) atomicAdd(p.band_ctr + b, 1u);
-        }
-    }
+    if (COOP && warp >= 8) run_stagers<KB>(p, sp, &smaps, smem_u32(ring_raw), sh);
 
     // ---------------------------------------------------------------- transposers (fused mode, warps 8..11)
     if (FUSED && warp >= 8) {

@@ -333,109 +333,47 @@ __global__ void __launch_bounds__(256) ring_upsample_kernel(const RingGeom in, i
     }
 }
 
-// Addresses of one staging task: image row h, pixels [w0, w0+64), channel block cb of Z frame f of sample n.
-struct StageTask {
-    const __nv_bfloat16* src;   // channel 0 of the source frame at (h, 0), or null (absent history: zeros)
-    int64_t cstride;            // source channel stride
-    __nv_bfloat16* ncdst;       // channel 0 of the new-cache frame at (h, 0), or null
-    __nv_bfloat16* dst;         // channels-last destination of pixel (h, 0)
-    int cb, w0;
+// ------------------------------------------------------------------------------------------------
+// cooperative staging: what the stager warps inside the convolution kernels share with the host
+// ------------------------------------------------------------------------------------------------
+// The same tile move as stage_frames_kernel<KB, true>, run by the 128 threads of the stager warps: a task is
+// [KB channels][PX pixels] of one image row of one Z frame = 8 KB either way, fetched by TMA straight from x or the
+// cache as two raw boxes [32 channels][64 pixels] (128-byte rows, 128-byte swizzle), transposed on the way out of
+// shared memory by ldmatrix.trans and written channels-last with 16-byte stores; a frame of the updated cache goes
+// back out of the same raw boxes with TMA stores.
+struct StagerMaps {       // raw NCTHW views (w, h, frame, c, n), box [32 channels][1][1][64 pixels]
+    CUtensorMap x, cache, nc;
 };
 
-__device__ __forceinline__ StageTask make_stage_task(const StageParams& p, int KB, int n, int f, int cb, int h, int w0) {
-    StageTask t;
-    const int F = p.tc + p.T;
-    const int64_t HW = (int64_t)p.H * p.W;
-    t.src = nullptr;
-    t.cstride = 0;
-    if (f < p.tc) {
-        const int cfr = f - (p.tc - p.cf);
-        if (p.cache && cfr >= 0) {
-            t.src = p.cache + ((int64_t)n * p.Cin * p.cf + cfr) * HW + (int64_t)h * p.W;
-            t.cstride = (int64_t)p.cf * HW;
-        }
-    } else {
-        t.src = p.x + ((int64_t)n * p.Cin * p.T + (f - p.tc)) * HW + (int64_t)h * p.W;
-        t.cstride = (int64_t)p.T * HW;
-    }
-    const int jc = f - p.T;
-    t.ncdst = nullptr;
-    if (p.new_cache && jc >= 0 && jc < p.tc) t.ncdst = p.new_cache + ((int64_t)n * p.Cin * p.tc + jc) * HW + (int64_t)h * p.W;
-    t.dst = p.zs + ((((int64_t)n * F + f) * p.CB + cb) * HW + (int64_t)h * p.W) * KB;
-    t.cb = cb;
-    t.w0 = w0;
-    return t;
-}
+constexpr int STAGER_SLOT_BYTES = 8192;    // one task in shared memory: two raw boxes of 4 KB
+constexpr int STAGER_MAX_SLOTS = 4;
 
-// The same tile move as stage_frames_kernel<KB, true>, run by the 128 threads of the stager warps inside the
-// convolution kernel (cooperative staging): [KB channels][64 pixels] of an image row -> [64 pixels][KB channels],
-// plus the cache update when the frame belongs to the new cache.  Split in two so that the loads of several
-// tasks can be in flight before the first is written: stage_task_load fills val[], stage_task_store moves it
-// through `tile` (StagerGeom<KB>::TILE_WORDS words of shared memory; phases separated by the stagers' named
-// barrier, id 2).
-__device__ __forceinline__ void stager_bar() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
+struct StagerRec {        // one task as the issuing thread decoded it, read by the whole team
+    __nv_bfloat16* dst;   // channels-last destination of pixel (h, w0)
+    int w0, h, n, c0;     // first pixel, image row, sample, first channel of the block
+    int fr_nc;            // frame of the updated cache this task also writes, or -1
+    int present;          // 0: absent history (zeros, nothing was fetched)
+};
 
-// PX: pixels of an image row per task.  64 for 64-channel blocks; 128 for 32-channel blocks, so that a task moves
-// the same 8 KB either way (the per-task barriers and address arithmetic are what limits a stager team).
 template <int KB>
 struct StagerGeom {
-    static constexpr int PX = (KB == 64) ? 64 : 128;
-    static constexpr int VPR = PX / 8;                    // 16-byte vectors per channel row
-    static constexpr int NLD = KB * VPR / 128;            // vectors per thread
-    static constexpr int PITCH = PX / 2 + 1;              // 32-bit words per channel row in the tile (+1: bank spread)
-    static constexpr int TILE_WORDS = KB * PITCH;
+    static constexpr int PX = (KB == 64) ? 64 : 128;      // pixels of an image row per task
 };
 
-template <int KB>
-__device__ __forceinline__ void stage_task_load(const StageParams& p, const StageTask& t, int tid,
-                                                uint4 (&val)[StagerGeom<KB>::NLD]) {
-    using G = StagerGeom<KB>;
-#pragma unroll
-    for (int k = 0; k < G::NLD; ++k) {
-        const int i = tid + 128 * k;
-        const int c = i / G::VPR, v = i % G::VPR;
-        const int ci = t.cb * KB + c;
-        const int w = t.w0 + v * 8;
-        val[k] = make_uint4(0u, 0u, 0u, 0u);
-        if (w < p.W && ci < p.Cin && t.src) val[k] = __ldg(reinterpret_cast<const uint4*>(t.src + ci * t.cstride + w));
-    }
-}
-
-template <int KB>
-__device__ __forceinline__ void stage_task_store(const StageParams& p, const StageTask& t, int tid,
-                                                 const uint4 (&val)[StagerGeom<KB>::NLD], uint32_t* tile) {
-    using G = StagerGeom<KB>;
-    constexpr int OCT = KB / 8;
-    const int64_t ncstride = (int64_t)p.tc * p.H * p.W;
-#pragma unroll
-    for (int k = 0; k < G::NLD; ++k) {
-        const int i = tid + 128 * k;
-        const int c = i / G::VPR, v = i % G::VPR;
-        const int ci = t.cb * KB + c;
-        const int w = t.w0 + v * 8;
-        if (t.ncdst && w < p.W && ci < p.Cin) *reinterpret_cast<uint4*>(t.ncdst + ci * ncstride + w) = val[k];
-        uint32_t* row = tile + c * G::PITCH + v * 4;
-        row[0] = val[k].x; row[1] = val[k].y; row[2] = val[k].z; row[3] = val[k].w;
-    }
-    stager_bar();
-#pragma unroll
-    for (int k = 0; k < (G::PX / 2 * OCT) / 128; ++k) {
-        const int vt = tid + 128 * k;
-        const int oct = vt % OCT, pp = vt / OCT;
-        uint32_t lo[4], hi[4];
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const uint32_t a = tile[(oct * 8 + 2 * q) * G::PITCH + pp];
-            const uint32_t b = tile[(oct * 8 + 2 * q + 1) * G::PITCH + pp];
-            lo[q] = __byte_perm(a, b, 0x5410);
-            hi[q] = __byte_perm(a, b, 0x7632);
-        }
-        const int wa = t.w0 + 2 * pp;
-        if (wa < p.W) *reinterpret_cast<uint4*>(t.dst + (int64_t)wa * KB + oct * 8) = make_uint4(lo[0], lo[1], lo[2], lo[3]);
-        if (wa + 1 < p.W)
-            *reinterpret_cast<uint4*>(t.dst + (int64_t)(wa + 1) * KB + oct * 8) = make_uint4(hi[0], hi[1], hi[2], hi[3]);
-    }
-    stager_bar();                                           // the tile may be overwritten by the next task
+__device__ __forceinline__ void stager_bar() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
+// barrier of the 128 stager threads that also ANDs a flag over them (a wait that gave up in one thread ends the
+// team together: nobody is left waiting at a barrier for a thread that returned)
+__device__ __forceinline__ bool stager_bar_and(bool v) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.u32 p, %1, 0;\n\t"
+        "bar.red.and.pred q, 2, 128, p;\n\t"
+        "selp.u32 %0, 1, 0, q;\n\t}"
+        : "=r"(r)
+        : "r"((uint32_t)v)
+        : "memory");
+    return r != 0;
 }
 
 }  // namespace ccv3d
