@@ -440,6 +440,12 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
         if (cudaMemsetAsync(h->band_ctr, 0, (size_t)in_bands * sizeof(unsigned int), st) != cudaSuccess) return cuda_fail();
         p.band_ctr = h->band_ctr;
         p.nbands = in_bands;
+        // The first tiles of every CTA read bands 0 and 1 (of all frames), and until those are staged nothing else can run:
+        // with four stager warps per SM that took 113 k of the 1620 k cycles of 192->192 at 352x640.  Those two bands go
+        // through the staging kernel instead (all warps of all SMs, about 20 us), the stagers take over from band 2.
+        p.band_first = in_bands < 2 ? in_bands : 2;
+        s = launch_stage(h, sp, 0, H < 16 * p.band_first ? H : 16 * p.band_first, nframes, st);
+        if (s != CCV3D_OK) return s;
         s = encode_stager_maps(h, x, cache, cf, sp.new_cache, N, T, H, W);
         if (s != CCV3D_OK) return s;
         p.ty_begin = 0;

@@ -39,6 +39,7 @@ struct TcParams {
     long long wait_limit_clk; // bound of every mbarrier wait, in SM clocks
     unsigned int* band_ctr;   // cooperative staging: per 16-row band, the number of CTAs that have staged their share
     int nbands;               // cooperative staging: 16-row bands of the input image
+    int band_first;           // cooperative staging: bands below this were staged before the launch (by stage_frames_kernel)
     int stg_slots;            // cooperative staging: raw slots (tasks in flight) of the stager team, 2..STAGER_MAX_SLOTS
     // general geometry (Eq. (2) with the layer's own padding and dilation, Eq. (1) with d_t); when `general` is 0
     // the kernel uses pad = (k-1)/2 and unit dilation.  H and W above are the OUTPUT extents; the input extents
@@ -268,7 +269,7 @@ __device__ __forceinline__ void run_stagers(const TcParams& p, const StageParams
         s.present = f >= sp.tc || (sp.cache && s.fr >= 0);
         return s;
     };
-    Cursor it = {0, 0, 0, 0, 0, 0, 0, 0};
+    Cursor it = {p.band_first, 0, 0, 0, 0, 0, 0, 0};
     auto issue = [&](int slot) {
         if (it.left == 0) return;
         const int f = sp.f_begin + it.fi, h = 16 * it.b + it.hr, n = it.n;
@@ -304,7 +305,7 @@ __device__ __forceinline__ void run_stagers(const TcParams& p, const StageParams
     int slot = 0, prev = R - 1;
     uint32_t par = 0;
     bool first_task = true, ok = true;
-    for (int b = 0; ok && b < p.nbands; ++b) {
+    for (int b = p.band_first; ok && b < p.nbands; ++b) {
         int first, last, rows;
         band_run(b, first, last, rows);
         for (int task = first; task < last; ++task) {
@@ -525,7 +526,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
             int s = 0;
             uint32_t phase = 1;
             bool ok = true;
-            int bands_ready = 0;                       // COOP: bands [0, bands_ready) are known to be staged
+            int bands_ready = COOP ? p.band_first : 0;   // COOP: bands [0, bands_ready) are known to be staged
             for (int item = cta_lin; ok && item < p.total_tiles; item += cta_cnt) {
                 const TileView tv = tile_view<TAIL>(p, item);
                 int r = tv.tile / tv.NT;

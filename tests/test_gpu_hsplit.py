@@ -50,7 +50,7 @@ CASES = [
     (32, 64, 3, 30, 40, (3, 5, 3), (1, 2, 1), si.BF16, (3,)),          # dilated 5 taps in h: halo of 4 rows
     (16, 24, 2, 18, 20, (3, 3, 3), (1, 1, 1), si.F32, (2,)),
     (64, 64, 2, 24, 32, (3, 1, 1), (1, 1, 1), si.BF16, (2,)),          # temporal-only kernel: nothing exchanged
-    (64, 64, 8, 320, 256, (3, 3, 3), (1, 1, 1), si.BF16, (2,)),        # slabs of 162 rows: large enough for the one-kernel schedule
+    (64, 64, 8, 320, 256, (3, 3, 3), (1, 1, 1), si.BF16, (2,)),        # slabs of 162 rows: large enough for the cooperative schedule
 ]
 
 
@@ -84,7 +84,7 @@ def test_bands_equal_unsplit_layer(ccv, Cin, Cout, T, H, W, k, dil, dtype, world
         assert np.array_equal(bits(got), bits(unsplit)), f"world {world}: bands differ from the unsplit layer"
         for l in layers:
             assert l.conv.device_status()[0] == ccv.OK
-            if H >= 320:      # the slab layer (no padding in h) runs as one kernel with cooperative staging, like the unsplit one
+            if H >= 320:      # the slab layer (no padding in h) runs on the cooperative schedule, like the unsplit one
                 cnt = l.conv.counters()
                 assert cnt["calls"] == 2 and cnt["kernel_launches"] == whole.counters()["kernel_launches"], cnt
             l.close()
