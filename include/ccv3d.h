@@ -54,7 +54,9 @@ typedef enum {
 #define CCV3D_FLAG_FORCE_SIMT 0x1u      /* BF16 layers: use the plain FP32-FMA kernel instead of the tensor-core kernel */
 #define CCV3D_FLAG_OVERLAP 0x4u          /* tensor-core route: process large images in bands, staging band k+1 on a side stream while band k is convolved */
 #define CCV3D_FLAG_TWO_KERNELS 0x10u     /* tensor-core route: run the staging pass as its own kernel before the convolution kernel instead of
-                                            inside it (cooperative staging, the default when W % 8 == 0) */
+                                            inside it (cooperative staging, the default for large calls with W % 8 == 0: four warps of
+                                            every CTA stage a band of rows ahead of the tiles; only the first two bands go through
+                                            the staging kernel) */
 #define CCV3D_FLAG_FUSED 0x8u            /* tensor-core route without scratch memory: no channels-last staging copy; the kernel reads x and the cache
                                             by TMA and transposes in shared memory (needs W % 8 == 0, else the staged route is taken). Some 10 % slower
                                             than the default route; for callers that cannot afford the workspace. */
