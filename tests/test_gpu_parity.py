@@ -229,7 +229,17 @@ def test_two_samples_on_the_cooperative_schedule(ccv):
     assert ctr["tcgen05_bf16"] == 1 and ctr["kernel_launches"] == 4      # weight pack, bias, head staging, cooperative kernel
 
 
-@pytest.mark.parametrize("Cin,Cout,W", [(64, 64, 160), (96, 48, 200)])   # 64-channel blocks; 32-channel blocks with a ragged 128-pixel task
+def test_cooperative_staging_with_absent_history(ccv):
+    """A first chunk of ONE frame on the cooperative schedule: Z = [absent, absent, x0], and the updated cache is
+    [absent ; x0] - a frame of history that never existed, which the stager warps write as zeros (into the staged copy
+    and into new_cache) without fetching anything.  Against the oracle, cache bit-exact."""
+    c = si.conv_case(1, 64, 64, 1, 704, 640, cache=None, seed=23)
+    m, ctr = run_case(ccv, c)
+    assert ctr["tcgen05_bf16"] == 1 and ctr["kernel_launches"] == 4      # weight pack, bias, head staging, cooperative kernel
+
+
+@pytest.mark.parametrize("Cin,Cout,W", [(64, 64, 160), (96, 48, 200), (96, 48, 192)])   # 64-channel blocks; 32-channel blocks with a ragged
+                                                                                         # 128-pixel task, and with one whose second box lies beyond the row
 def test_bf16_tensor_core_cooperative_staging(ccv, Cin, Cout, W):
     """Large enough for the default schedule to stage inside the convolution kernel (four stager warps per CTA, a
     band of 16 rows ahead of the tiles that read it; only the first two bands are staged by the staging kernel), and
