@@ -376,9 +376,9 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     // extra warps per CTA, one band of 16 rows ahead of the tiles that read it.
     // (with the layer's own padding and dilation too, at unit strides: the bands are bands of input rows)
     const int in_bands = (H + 15) / 16;
-    // (not the phase-decomposed copies of strided layers: their staging moves s_h s_w input pixels per output pixel, more
-    // than four stager warps per SM keep up with - measured 1.73 ms against 1.25 ms for the two kernels at 96->192,
-    // stride 2, from 704x1280)
+    // (not the phase-decomposed copies of strided layers: measured 1.41 ms against 1.24 ms for the two kernels at 96->192,
+    // stride 2, from 704x1280, level at 192->384 from 352x640 - their convolution kernel, single CTAs with a run-time tap
+    // loop and one tap per weight stage, loses more to the stagers' traffic than the hidden staging pass returns)
     const bool coop = nbands == 1 && !per_tap && !phased && (!general || d.stride[0] == 1) && !f32 &&
                       !(d.flags & CCV3D_FLAG_TWO_KERNELS) && raw_maps_ok(h, x, cache, new_cache, T, H, W) &&
                       in_bands <= MAX_COOP_BANDS && tiles_h >= 4 &&
