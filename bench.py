@@ -825,8 +825,8 @@ def main_ours(args):
         d2h = ho.numel() * 2 + (hn.numel() * 2 if hn is not None else 0)
         e2e = {"value": flops / (e_ms * 1e-3) / 1e12, "unit": "TFLOP/s", "h2d_bytes_per_step": int(h2d),
                "d2h_bytes_per_step": int(d2h), "ms_per_step": e_ms, "steps": e_steps,
-               "note": "ccv3d_forward_host: pinned host x, cache -> device, the layer, out, new_cache -> host; frame by frame "
-                       "on three streams (upload, compute on a frame ring, download overlap): bound by PCIe, whose two "
+               "note": "ccv3d_forward_host: pinned host x, cache -> device, the layer, out, new_cache -> host; band of rows by "
+                       "band, frame by frame on three streams (upload, compute on a frame ring, download overlap): bound by PCIe, whose two "
                        f"directions together moved {(h2d + d2h) / (e_ms * 1e6):.0f} GB/s here"}
         assert np.array_equal(ho.numpy().view(np.uint16), out.view(torch.int16).cpu().numpy().view(np.uint16))
         # the streaming form of the same call: the history stays in a frame ring on the device, so a step moves only

@@ -218,10 +218,11 @@ ccv3d_status ccv3d_forward_static(ccv3d_handle* h, const void* x, const void* ca
  * out and new_cache back, and returns after the stream has completed.  Pinned
  * host memory makes the copies asynchronous with respect to each other.
  * Standard BF16 tensor-core layers with cin % 32 == 0 and frames of a few MB run
- * frame by frame instead (upload of frame t+1, convolution of frame t on a frame
- * ring and download of frame t-1 overlap on three streams; same bits, since the
- * operator streams exactly): the call then takes about as long as the slower
- * PCIe direction alone.
+ * piece by piece instead (upload of piece k+1, convolution of piece k on a frame
+ * ring and download of piece k-1 overlap on three streams; a piece is a frame, or -
+ * frames of tens of MB - a band of rows of a frame with its halo rows; same bits,
+ * since the operator streams exactly in time and is local in space): the call then
+ * takes about as long as the slower PCIe direction alone.
  */
 ccv3d_status ccv3d_forward_host(ccv3d_handle* h, const void* x_host, const void* cache_host, void* out_host,
                                 void* new_cache_host, int32_t N, int32_t T, int32_t H, int32_t W, void* stream);
@@ -231,7 +232,7 @@ ccv3d_status ccv3d_forward_host(ccv3d_handle* h, const void* x_host, const void*
  * device between calls, in a frame ring the handle owns, so a call moves only x (HOST [N,cin,T,H,W]) up and out
  * (HOST [N,cout,T,H,W]) down - the cache never crosses the bus.  reset != 0 starts a new stream (first chunk: no
  * history); a change of N, H or W, or any other host entry point used on the handle in between, starts a new
- * stream as well.  Same frame-by-frame pipeline, same results bit for bit as ccv3d_forward_host with the cache
+ * stream as well.  Same piece-by-piece pipeline (one history ring per band of rows), same results bit for bit as ccv3d_forward_host with the cache
  * carried by the caller.  Synchronous like ccv3d_forward_host.  Layers and sizes the pipelined path does not take
  * (see ccv3d_forward_host: standard geometry, BF16, cin a multiple of the channel block, a few MB per frame)
  * return CCV3D_ERR_UNSUPPORTED; any T >= 1.

@@ -67,7 +67,7 @@ struct ccv3d_handle {
     // host-entry staging (device buffers)
     void* hx; void* hc; void* ho; void* hn;
     uint64_t hx_b, hc_b, ho_b, hn_b;
-    cudaEvent_t hp_ev[4][3];   // pipelined host entry: per frame buffer {uploaded, input buffer free, computed, downloaded}
+    cudaEvent_t hp_ev[5][3];   // pipelined host entry: per buffer {uploaded, input buffer free, computed, downloaded, cache piece read}
     bool hp_ready;
     EncodeTiledFn encode;
     CUtensorMap tm_a;
@@ -360,7 +360,7 @@ ccv3d_status ccv3d_destroy(ccv3d_handle* h) {
     for (int i = 0; i < 2; ++i)
         if (h->ev_join[i]) cudaEventDestroy(h->ev_join[i]);
     if (h->hp_ready)
-        for (int k = 0; k < 4; ++k)
+        for (int k = 0; k < 5; ++k)
             for (int b = 0; b < 3; ++b) cudaEventDestroy(h->hp_ev[k][b]);
     if (h->prof_ev) {
         for (int i = 0; i < 3 * PROF_SLOTS; ++i) cudaEventDestroy(h->prof_ev[i]);
@@ -443,33 +443,49 @@ ccv3d_status ccv3d_forward_static(ccv3d_handle* h, const void* x, const void* ca
     return count(h, forward_tc_static(h, x, cache, out, new_cache, N, T, H, W, (cudaStream_t)stream));
 }
 
-// Host entry point, pipelined frame by frame (standard BF16 tensor-core layers whose channels fit a frame ring).
-// Frame t of x is a strided 2-D copy (one row per (n, channel) plane) into a dense one-frame device buffer on an
-// upload stream; on the caller's stream it is moved into a frame ring and convolved as a one-frame chunk (history =
-// the ring, exactly the streaming form of the operator, so the result is bit for bit that of one T-frame call);
-// the output frame goes back with another strided 2-D copy on a download stream.  Three buffers of each kind rotate,
-// so that upload, compute and download of different frames overlap: the call takes about as long as the slower of
-// the two PCIe directions instead of their sum.
+// Host entry point, pipelined (standard BF16 tensor-core layers whose channels fit a frame ring).
+// The image is cut into bands of rows, and a band into frames.  Band rows [h0, h1) of frame t of x, with the p_h halo
+// rows above and below that exist, are a strided 2-D copy (one piece per (n, channel) plane) into a dense device buffer
+// on an upload stream; on the caller's stream that slab frame is moved into a frame ring of slab height and convolved as
+// a one-frame chunk (history = the ring, exactly the streaming form of the operator); the band's rows of the output
+// frame go back with another strided 2-D copy on a download stream.  A slab is convolved as an image of its own: its
+// first and last output rows see zero padding where the neighbouring band's rows belong and are not downloaded, every
+// other row sees what it sees in the whole image, in the same order of accumulation, so the result is bit for bit that
+// of one call on the whole image.  Three buffers of each kind rotate, so that upload, compute and download of different
+// pieces overlap: the call takes about as long as the slower of the two PCIe directions - plus the time until the first
+// output piece exists, which is why the pieces are bands and not whole frames (kt-1 + 1 whole frames are a third of
+// configuration 3's upload).
 // stream_state != nullptr: streaming form - {ring slot of the next frame, frames seen so far} carried in the handle from
-// call to call; the history is whatever the previous call left in the ring (cache_host and new_cache_host are null).
+// call to call; the history is whatever the previous call left in the rings (cache_host and new_cache_host are null).
+static int host_bands(const ccv3d_handle* h, int N, int H, int W) {
+    // pieces of at least 16 MB on the larger side (PCIe efficiency) and bands of at least 32 rows; at most 8 bands
+    const uint64_t frame = (uint64_t)N * (h->d.cin > h->d.cout ? h->d.cin : h->d.cout) * H * W * 2;
+    int nb = (int)(frame / (16u << 20));
+    if (nb > H / 32) nb = H / 32;
+    if (nb > 8) nb = 8;
+    return nb < 1 ? 1 : nb;
+}
+
 static ccv3d_status forward_host_pipelined(ccv3d_handle* h, const void* x_host, const void* cache_host, void* out_host,
                                     void* new_cache_host, int N, int T, int H, int W, cudaStream_t st,
                                     int* stream_state = nullptr) {
     const ccv3d_desc& d = h->d;
     const int tc = hist_len(d);
+    const int ph = (d.kh - 1) / 2;                         // (standard geometry: size-preserving padding)
     constexpr int NBUF = 3;
-    const uint64_t HWb = (uint64_t)H * W * 2;
-    const uint64_t xf = (uint64_t)N * d.cin * HWb, of = (uint64_t)N * d.cout * HWb;      // one frame of x / of out
-    ccv3d_ring ring;
-    ring.N = N; ring.C = d.cin; ring.F = tc + 1; ring.H = H; ring.W = W; ring.KB = h->plan.KB;
+    const int nbands = host_bands(h, N, H, W);
+    const int Hs_max = (H + nbands - 1) / nbands + 2 * ph; // rows of the tallest slab
+    const uint64_t Wb = (uint64_t)W * 2;                   // bytes of an image row
+    const uint64_t HWb = (uint64_t)H * Wb;                 // bytes of a plane of the whole image
+    const uint64_t xf = (uint64_t)N * d.cin * Hs_max * Wb, of = (uint64_t)N * d.cout * Hs_max * Wb;   // one slab frame of x / of out
+    const int F = tc + 1;
     ccv3d_status s;
     if ((s = grow(&h->hx, &h->hx_b, NBUF * xf)) != CCV3D_OK) return s;
     if ((s = grow(&h->ho, &h->ho_b, NBUF * of)) != CCV3D_OK) return s;
-    if ((s = grow(&h->hc, &h->hc_b, (uint64_t)ring.F * xf)) != CCV3D_OK) return s;
+    if ((s = grow(&h->hc, &h->hc_b, (uint64_t)nbands * F * xf)) != CCV3D_OK) return s;
     if (tc && new_cache_host && (s = grow(&h->hn, &h->hn_b, (uint64_t)tc * xf)) != CCV3D_OK) return s;
-    ring.base = h->hc;
     if (!h->hp_ready) {
-        for (int k = 0; k < 4; ++k)
+        for (int k = 0; k < 5; ++k)
             for (int b = 0; b < NBUF; ++b)
                 if (cudaEventCreateWithFlags(&h->hp_ev[k][b], cudaEventDisableTiming) != cudaSuccess) return cuda_fail();
         h->hp_ready = true;
@@ -478,62 +494,85 @@ static ccv3d_status forward_host_pipelined(ccv3d_handle* h, const void* x_host, 
     if (cudaEventRecord(h->ev_fork, st) != cudaSuccess) return cuda_fail();
     if (cudaStreamWaitEvent(s_up, h->ev_fork, 0) != cudaSuccess || cudaStreamWaitEvent(s_down, h->ev_fork, 0) != cudaSuccess)
         return cuda_fail();
-    if (!stream_state && !cache_host && tc && cudaMemsetAsync(ring.base, 0, (size_t)ring.F * xf, st) != cudaSuccess)
+    if (!stream_state && !cache_host && tc && cudaMemsetAsync(h->hc, 0, (size_t)nbands * F * xf, st) != cudaSuccess)
         return cuda_fail();
 
     const int pre = (cache_host && tc) ? tc : 0;           // history frames uploaded before the first frame of x
-    const bool nc_early = tc && new_cache_host && tc < NBUF && pre + T >= tc;
-    int slot = 0, seen = 0;                                // ring slot of the next frame; frames in the ring so far
-    if (stream_state) { slot = stream_state[0]; seen = stream_state[1]; }
-    for (int i = 0; i < pre + T; ++i) {
-        const int b = i % NBUF;
-        const bool is_x = i >= pre;
-        const int t = is_x ? i - pre : i;
-        char* xin = (char*)h->hx + (size_t)b * xf;
-        // upload: wait until the ring load that last read this buffer is done
-        if (i >= NBUF && cudaStreamWaitEvent(s_up, h->hp_ev[1][b], 0) != cudaSuccess) return cuda_fail();
-        const char* src = is_x ? (const char*)x_host + (size_t)t * HWb : (const char*)cache_host + (size_t)t * HWb;
-        const size_t spitch = (size_t)(is_x ? T : tc) * HWb;
-        if (cudaMemcpy2DAsync(xin, HWb, src, spitch, HWb, (size_t)N * d.cin, cudaMemcpyHostToDevice, s_up) != cudaSuccess)
-            return cuda_fail();
-        if (cudaEventRecord(h->hp_ev[0][b], s_up) != cudaSuccess) return cuda_fail();
-        // cache update: the last tc frames of the stream go straight back from their upload buffers (bit copies),
-        // early, while the download stream has nothing else to do.  (tc < NBUF: these buffers are not reused in
-        // this call; the next call starts after the download stream has been joined.)
-        if (nc_early && i >= pre + T - tc) {
-            const int j = i - (pre + T - tc);
-            if (cudaStreamWaitEvent(s_down, h->hp_ev[0][b], 0) != cudaSuccess) return cuda_fail();
-            if (cudaMemcpy2DAsync((char*)new_cache_host + (size_t)j * HWb, (size_t)tc * HWb, xin, HWb, HWb, (size_t)N * d.cin,
-                                  cudaMemcpyDeviceToHost, s_down) != cudaSuccess)
+    const bool nc_early = tc && new_cache_host && pre + T >= tc;
+    int slot0 = 0, seen0 = 0;                              // ring slot of the next frame; frames in the ring so far
+    if (stream_state) { slot0 = stream_state[0]; seen0 = stream_state[1]; }
+    int slot = slot0, seen = seen0;
+    int g = 0, go = 0;                                     // pieces uploaded / downloaded so far (buffers rotate over all bands)
+    bool nc_pending[NBUF] = {false, false, false};         // a cache piece is still being read out of this upload buffer
+    for (int band = 0; band < nbands; ++band) {
+        const int h0 = (int)((int64_t)H * band / nbands), h1 = (int)((int64_t)H * (band + 1) / nbands);
+        const int hs0 = h0 - ph > 0 ? h0 - ph : 0, hs1 = h1 + ph < H ? h1 + ph : H;
+        const int Hs = hs1 - hs0, top = h0 - hs0, rows = h1 - h0;
+        const uint64_t HWs = (uint64_t)Hs * Wb;            // bytes of a plane of the slab
+        ccv3d_ring ring;
+        ring.N = N; ring.C = d.cin; ring.F = F; ring.H = Hs; ring.W = W; ring.KB = h->plan.KB;
+        ring.base = (char*)h->hc + (size_t)band * F * xf;
+        slot = slot0; seen = seen0;
+        for (int i = 0; i < pre + T; ++i, ++g) {
+            const int b = g % NBUF;
+            const bool is_x = i >= pre;
+            const int t = is_x ? i - pre : i;
+            char* xin = (char*)h->hx + (size_t)b * xf;
+            // upload: wait until the ring load (and the cache piece, if any) that last read this buffer is done
+            if (g >= NBUF && cudaStreamWaitEvent(s_up, h->hp_ev[1][b], 0) != cudaSuccess) return cuda_fail();
+            if (nc_pending[b]) {
+                if (cudaStreamWaitEvent(s_up, h->hp_ev[4][b], 0) != cudaSuccess) return cuda_fail();
+                nc_pending[b] = false;
+            }
+            const char* src = (is_x ? (const char*)x_host : (const char*)cache_host) + (size_t)t * HWb + (size_t)hs0 * Wb;
+            const size_t spitch = (size_t)(is_x ? T : tc) * HWb;
+            if (cudaMemcpy2DAsync(xin, HWs, src, spitch, HWs, (size_t)N * d.cin, cudaMemcpyHostToDevice, s_up) != cudaSuccess)
+                return cuda_fail();
+            if (cudaEventRecord(h->hp_ev[0][b], s_up) != cudaSuccess) return cuda_fail();
+            // cache update: the band's rows of the last tc frames of the stream go straight back from their upload
+            // buffers (bit copies), in between the output pieces
+            if (nc_early && i >= pre + T - tc) {
+                const int j = i - (pre + T - tc);
+                if (cudaStreamWaitEvent(s_down, h->hp_ev[0][b], 0) != cudaSuccess) return cuda_fail();
+                if (cudaMemcpy2DAsync((char*)new_cache_host + (size_t)j * HWb + (size_t)h0 * Wb, (size_t)tc * HWb,
+                                      xin + (size_t)top * Wb, HWs, (size_t)rows * Wb, (size_t)N * d.cin, cudaMemcpyDeviceToHost,
+                                      s_down) != cudaSuccess)
+                    return cuda_fail();
+                if (cudaEventRecord(h->hp_ev[4][b], s_down) != cudaSuccess) return cuda_fail();
+                nc_pending[b] = true;
+            }
+            // compute
+            if (cudaStreamWaitEvent(st, h->hp_ev[0][b], 0) != cudaSuccess) return cuda_fail();
+            if ((s = ccv3d_ring_load(&ring, slot, xin, 1, st)) != CCV3D_OK) return s;
+            h->ctr.kernel_launches++;
+            if (cudaEventRecord(h->hp_ev[1][b], st) != cudaSuccess) return cuda_fail();
+            if (is_x) {
+                const int ob = go % NBUF;
+                char* oout = (char*)h->ho + (size_t)ob * of;
+                if (go >= NBUF && cudaStreamWaitEvent(st, h->hp_ev[3][ob], 0) != cudaSuccess) return cuda_fail();
+                const int hist = seen < tc ? seen : tc;
+                if ((s = forward_ring(h, &ring, slot, hist, nullptr, 0, nullptr, 0, oout, 1, st)) != CCV3D_OK) return s;
+                if (cudaEventRecord(h->hp_ev[2][ob], st) != cudaSuccess) return cuda_fail();
+                // download the band's own rows of the slab's output frame
+                if (cudaStreamWaitEvent(s_down, h->hp_ev[2][ob], 0) != cudaSuccess) return cuda_fail();
+                if (cudaMemcpy2DAsync((char*)out_host + (size_t)t * HWb + (size_t)h0 * Wb, (size_t)T * HWb, oout + (size_t)top * Wb,
+                                      HWs, (size_t)rows * Wb, (size_t)N * d.cout, cudaMemcpyDeviceToHost, s_down) != cudaSuccess)
+                    return cuda_fail();
+                if (cudaEventRecord(h->hp_ev[3][ob], s_down) != cudaSuccess) return cuda_fail();
+                ++go;
+            }
+            slot = (slot + 1) % F;
+            ++seen;
+        }
+        if (tc && new_cache_host && !nc_early) {
+            // (T + history shorter than tc frames.)  The last tc frames of [cache ; x] are the tc slots before `slot`
+            // (zeros where the stream had no history): back to NCTHW on the device, then the band's rows to the host
+            if ((s = ccv3d_ring_store(&ring, (slot + F - tc) % F, h->hn, tc, st)) != CCV3D_OK) return s;
+            h->ctr.kernel_launches++;
+            if (cudaMemcpy2DAsync((char*)new_cache_host + (size_t)h0 * Wb, HWb, (char*)h->hn + (size_t)top * Wb, HWs, (size_t)rows * Wb,
+                                  (size_t)N * d.cin * tc, cudaMemcpyDeviceToHost, st) != cudaSuccess)
                 return cuda_fail();
         }
-        // compute
-        if (cudaStreamWaitEvent(st, h->hp_ev[0][b], 0) != cudaSuccess) return cuda_fail();
-        if ((s = ccv3d_ring_load(&ring, slot, xin, 1, st)) != CCV3D_OK) return s;
-        h->ctr.kernel_launches++;
-        if (cudaEventRecord(h->hp_ev[1][b], st) != cudaSuccess) return cuda_fail();
-        if (is_x) {
-            const int ob = t % NBUF;
-            char* oout = (char*)h->ho + (size_t)ob * of;
-            if (t >= NBUF && cudaStreamWaitEvent(st, h->hp_ev[3][ob], 0) != cudaSuccess) return cuda_fail();
-            const int hist = seen < tc ? seen : tc;
-            if ((s = forward_ring(h, &ring, slot, hist, nullptr, 0, nullptr, 0, oout, 1, st)) != CCV3D_OK) return s;
-            if (cudaEventRecord(h->hp_ev[2][ob], st) != cudaSuccess) return cuda_fail();
-            // download
-            if (cudaStreamWaitEvent(s_down, h->hp_ev[2][ob], 0) != cudaSuccess) return cuda_fail();
-            if (cudaMemcpy2DAsync((char*)out_host + (size_t)t * HWb, (size_t)T * HWb, oout, HWb, HWb, (size_t)N * d.cout,
-                                  cudaMemcpyDeviceToHost, s_down) != cudaSuccess)
-                return cuda_fail();
-            if (cudaEventRecord(h->hp_ev[3][ob], s_down) != cudaSuccess) return cuda_fail();
-        }
-        slot = (slot + 1) % ring.F;
-        ++seen;
-    }
-    if (tc && new_cache_host && !nc_early) {
-        // the last tc frames of [cache ; x] are the tc slots before `slot` (zeros where the stream had no history)
-        if ((s = ccv3d_ring_store(&ring, (slot + ring.F - tc) % ring.F, h->hn, tc, st)) != CCV3D_OK) return s;
-        h->ctr.kernel_launches++;
-        if (cudaMemcpyAsync(new_cache_host, h->hn, (size_t)tc * xf, cudaMemcpyDeviceToHost, st) != cudaSuccess) return cuda_fail();
     }
     if (cudaEventRecord(h->ev_join[0], s_down) != cudaSuccess || cudaStreamWaitEvent(st, h->ev_join[0], 0) != cudaSuccess)
         return cuda_fail();

@@ -395,11 +395,14 @@ def test_host_entry_point_matches_device_entry_point(ccv):
 
 
 @pytest.mark.parametrize("N,Cin,Cout,T,H,W,cache", [(1, 64, 96, 5, 128, 160, "random"), (2, 96, 64, 3, 120, 136, None),
-                                                       (1, 64, 64, 2, 160, 200, "random")])
+                                                       (1, 64, 64, 2, 160, 200, "random"),
+                                                       (1, 64, 96, 3, 352, 640, "random"),     # frames of 43 MB: two bands of rows
+                                                       (1, 128, 64, 2, 250, 648, None)])       # two bands of 125 rows (ragged tiles), first chunk
 def test_pipelined_host_entry_point(ccv, N, Cin, Cout, T, H, W, cache):
     """Frames of a few MB: the host entry point uploads, convolves (on a frame ring, one frame per call) and
-    downloads frame by frame on three streams.  Same bits as the device entry point on the whole tensor, cache
-    update included; pageable host memory."""
+    downloads piece by piece on three streams - whole frames, or bands of rows of a frame (with their halo rows) when
+    a frame is tens of MB.  Same bits as the device entry point on the whole tensor, cache update included; pageable
+    host memory."""
     c = si.conv_case(N, Cin, Cout, T, H, W, cache=cache, seed=13)
     layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]))
     out_d, nc_d = layer(to_dev(c["x"]), to_dev(c["cache"]))
@@ -457,6 +460,28 @@ def test_host_stream_keeps_the_history_on_the_device(ccv):
     o = np.empty((1, 64, 2, 16, 16), np.uint16)
     assert ccv.ccv3d_forward_host_stream(l2.h, small["x"].ctypes.data, o.ctypes.data, 1, 1, 2, 16, 16, st) == ccv.ERR_UNSUPPORTED
     l2.close()
+
+
+def test_host_stream_in_bands_of_rows(ccv):
+    """ccv3d_forward_host_stream with frames large enough for the host pipeline to cut them into bands of rows (three
+    here): every band keeps its own history ring on the device between calls; chunks of 2, 1 and 3 frames give the bits of
+    the whole-sequence run."""
+    N, Cin, Cout, H, W = 1, 128, 64, 352, 640
+    lens = [2, 1, 3]
+    c = si.conv_case(N, Cin, Cout, sum(lens), H, W, cache=None, seed=24)
+    layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]))
+    whole, _ = layer(to_dev(c["x"]), None)
+    whole = bits(whole)
+    st = torch.cuda.current_stream().cuda_stream
+    t0 = 0
+    for i, T in enumerate(lens):
+        xc = np.ascontiguousarray(c["x"][:, :, t0:t0 + T])
+        out = np.full((N, Cout, T, H, W), 0x7FC0, np.uint16)
+        assert ccv.ccv3d_forward_host_stream(layer.h, xc.ctypes.data, out.ctypes.data, i == 0, N, T, H, W, st) == ccv.OK
+        assert np.array_equal(out, whole[:, :, t0:t0 + T]), f"chunk {i}"
+        t0 += T
+    assert layer.device_status()[0] == ccv.OK
+    layer.close()
 
 
 @pytest.mark.parametrize("shape,rt", [((2, 3, 2, 5, 6), 3), ((1, 4, 3, 6, 8), 4), ((1, 2, 2, 4, 12), 1)])
