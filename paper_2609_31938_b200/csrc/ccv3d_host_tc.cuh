@@ -385,28 +385,31 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
                       // fewer than eight waves of tiles: two kernels (the first tiles of a cooperative launch wait for two
                       // whole bands, and measured at six waves it is 15 % behind; level at seven, ahead from twelve)
                       (int64_t)N * tiles_h * p.tiles_w * To * NT * (pair ? 2 : 1) >= 8LL * h->sm_count;
-    // Cooperative staging: the stager team keeps stg_slots tasks of 8 KB in flight.  Narrow tiles (two pixel blocks per
-    // CTA, at most 128 output channels) stage twice as many input bytes per MMA cycle as wide ones: three slots, since
-    // with two the team, bound by the latency of its fetches, finishes last (192->96 at 704x1280: 4.34 M cycles against
-    // 3.35 M); wide tiles two, and a third only when that costs the rings nothing (192->192 at 352x640 loses 3 % when the
-    // third slot takes the fourth weight slot's place).
-    p.stg_slots = coop ? (NB == 2 ? 3 : 2) : 0;
+    // Cooperative staging: the stager team keeps stg_slots tasks in flight, two, and a third only when that costs the
+    // rings nothing (192->192 at 352x640 loses 3 % when a third slot takes the fourth weight slot's place).  A task is
+    // 8 KB next to wide tiles and 16 KB next to narrow ones (two pixel blocks per CTA, at most 128 output channels:
+    // STAGER_BOXES), which stage twice as many input bytes per MMA cycle: the team is bound by its per-task instructions
+    // (a barrier, the odometer, the TMA issue), and with tasks of twice the pixels 96->96 at 704x1280 went from 1.80 M to
+    // 1.66 M cycles, the figure of the same layer on frame rings (three slots of 8 KB before; with two the team, then
+    // bound by the latency of its fetches, finished last: 4.34 M cycles against 3.35 M at 192->96).
+    p.stg_slots = coop ? 2 : 0;
+    const size_t stg_slot = (size_t)(NB == 2 ? 4 : 2) * 4096;       // (STAGER_BOXES<NB>)
     size_t fixed = 1024 /*alignment slack*/ + align_up(sizeof(TcShared), 128) + 2 * (size_t)p.e_slot +
-                   (size_t)p.stg_slots * STAGER_SLOT_BYTES;
+                   (size_t)p.stg_slots * stg_slot;
     // leave room for staging blocks to be resident next to a convolution CTA when the two overlap
     const size_t limit = nbands > 1 ? SMEM_LIMIT - STAGE_COEXIST_BYTES : SMEM_LIMIT;
     const size_t budget = limit - fixed;
     const bool tpb9 = pair && !f32 && !phased && pl.KB == 32 && d.kh == 3 && d.kw == 3 && d.dilation[1] == 1 && d.dilation[2] == 1;
     s = size_pipeline(&p, budget, per_tap != 0 || phased, phased ? 1 : d.kw, tpb9 ? 9 : 0);   // (phase order: one tap per weight stage)
     if (s != CCV3D_OK) return s;
-    if (coop && p.stg_slots < 3 && (size_t)p.SA * p.a_slot + (size_t)p.SB * p.b_slot + STAGER_SLOT_BYTES <= budget) {
+    if (coop && p.stg_slots < 3 && (size_t)p.SA * p.a_slot + (size_t)p.SB * p.b_slot + stg_slot <= budget) {
         ++p.stg_slots;
-        fixed += STAGER_SLOT_BYTES;
+        fixed += stg_slot;
     }
     // ... and with narrow tiles a third activation slot is worth a weight slot when four or more of those are left: next to
     // the stagers' traffic it is the halo tiles that arrive late (96->96 at 704x1280: 1.95 M cycles with 2 + 4 slots,
     // 1.86 M with 3 + 3)
-    if (coop && NB == 2 && p.SA == 2 && p.SB >= 4 && 3 * (size_t)p.a_slot + (size_t)(p.SB - 1) * p.b_slot <= budget) {
+    if (coop && NB == 2 && p.SA == 2 && p.SB >= 4 && 3 * (size_t)p.a_slot + (size_t)(p.SB - 1) * p.b_slot <= limit - fixed) {
         p.SA = 3;
         --p.SB;
     }

@@ -194,7 +194,7 @@ __device__ __forceinline__ uint32_t epi_pair(float a0, float a1, uint32_t res_pa
 // The stager warps of the cooperative schedule (warps 8..11 of a CTA): the staging pass - same tile move as
 // stage_frames_kernel, cache update included - band by band of 16 image rows; every finished band is signalled with a
 // fence and one atomic per CTA.
-// Inside a band the tasks ([KB channels][SPX pixels] of one image row of one Z frame, 8 KB) are ordered (sample, frame,
+// Inside a band the tasks ([KB channels][SPX pixels] of one image row of one Z frame, 8 or 16 KB) are ordered (sample, frame,
 // channel block, row, chunk of the row) and CTA k takes the k-th of gridDim.x contiguous runs, so that the next task is an
 // odometer step away (a team of four warps is bound by its own instruction stream: decoding every task with divisions
 // cost more than moving it).  Thread 0 of the team keeps p.stg_slots tasks in flight: it leaves a task's record in
@@ -202,13 +202,17 @@ __device__ __forceinline__ uint32_t epi_pair(float a0, float a1, uint32_t res_pa
 // ldmatrix.trans (each lane ends up with 8 consecutive channels of one pixel) and writes them channels-last.  Frames
 // of the updated cache leave the same raw boxes by TMA store.  One barrier per task: it shares the outcome of the wait
 // and tells thread 0 that everybody has finished reading the previous task's slot.
-template <int KB>
+template <int KB, int NBX>     // NBX: raw boxes of 4 KB per task (2 or 4)
 __device__ __forceinline__ void run_stagers(const TcParams& p, const StageParams& sp, const StagerMaps* maps, uint32_t raw0,
                                             TcShared* sh) {
     const int tid = threadIdx.x - 256;
     const int lane = tid & 31, swp = tid >> 5;
-    constexpr int SPX = StagerGeom<KB>::PX;
+    constexpr int SPX = StagerGeom<KB>::PX * (NBX >> 1);    // pixels of an image row per task
+    constexpr uint32_t slot_bytes = (uint32_t)NBX * 4096u;
     const int nchunks = (sp.W + SPX - 1) / SPX;
+    // box j of a task: 64 pixels x 32 channels at pixel offset box_px(j), channel offset box_ch(j)
+    auto box_px = [&](int j) { return KB == 64 ? 64 * (j >> 1) : 64 * j; };
+    auto box_ch = [&](int j) { return KB == 64 ? 32 * (j & 1) : 0; };
     const int nf = sp.tc + sp.T - sp.f_begin;
     const int R = p.stg_slots;
     const int64_t HW = (int64_t)sp.H * sp.W;
@@ -283,13 +287,15 @@ __device__ __forceinline__ void run_stagers(const TcParams& p, const StageParams
         sh->stg_rec[slot] = rec;
         const uint32_t bar = smem_u32(&sh->stg_full[slot]);
         if (s.present) {
-            // (32-channel blocks: the second box holds pixels w0+64..; left out when it lies beyond the row)
-            const bool two = KB == 64 || rec.w0 + 64 < sp.W;
-            const uint32_t dst = raw0 + (uint32_t)slot * STAGER_SLOT_BYTES;
-            mbar_expect_tx(bar, two ? STAGER_SLOT_BYTES : STAGER_SLOT_BYTES / 2);
-            tma_load_5d(dst, s.tm, bar, rec.w0, h, s.fr, rec.c0, n);
-            if (KB == 64) tma_load_5d(dst + 4096, s.tm, bar, rec.w0, h, s.fr, rec.c0 + 32, n);
-            else if (two) tma_load_5d(dst + 4096, s.tm, bar, rec.w0 + 64, h, s.fr, rec.c0, n);
+            // (boxes that lie beyond the row are left out)
+            const uint32_t dst = raw0 + (uint32_t)slot * slot_bytes;
+            int nb = 0;
+#pragma unroll
+            for (int j = 0; j < NBX; ++j) nb += rec.w0 + box_px(j) < sp.W;
+            mbar_expect_tx(bar, (uint32_t)nb * 4096u);
+#pragma unroll
+            for (int j = 0; j < NBX; ++j)
+                if (rec.w0 + box_px(j) < sp.W) tma_load_5d(dst + (uint32_t)j * 4096u, s.tm, bar, rec.w0 + box_px(j), h, s.fr, rec.c0 + box_ch(j), n);
         } else {
             mbar_arrive(bar);
         }
@@ -317,25 +323,27 @@ __device__ __forceinline__ void run_stagers(const TcParams& p, const StageParams
             }
             first_task = false;
             const StagerRec rec = sh->stg_rec[slot];
-            const uint32_t src = raw0 + (uint32_t)slot * STAGER_SLOT_BYTES;
+            const uint32_t src = raw0 + (uint32_t)slot * slot_bytes;
             if (rec.present) {
                 if (tid == 0 && rec.fr_nc >= 0) {
-                    tma_store_5d(&maps->nc, src, rec.w0, rec.h, rec.fr_nc, rec.c0, rec.n);
-                    if (KB == 64) tma_store_5d(&maps->nc, src + 4096, rec.w0, rec.h, rec.fr_nc, rec.c0 + 32, rec.n);
-                    else if (rec.w0 + 64 < sp.W) tma_store_5d(&maps->nc, src + 4096, rec.w0 + 64, rec.h, rec.fr_nc, rec.c0, rec.n);
+#pragma unroll
+                    for (int j = 0; j < NBX; ++j)
+                        if (rec.w0 + box_px(j) < sp.W)
+                            tma_store_5d(&maps->nc, src + (uint32_t)j * 4096u, rec.w0 + box_px(j), rec.h, rec.fr_nc, rec.c0 + box_ch(j), rec.n);
                     bulk_commit();
                 }
+                // a box is eight units of 8 pixels x 32 channels; the team's warps share the task's units evenly
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const int u = swp * 4 + i, o = u & 7, hb = u >> 3;   // pixel octet, box of the slot
+                for (int i = 0; i < 2 * NBX; ++i) {
+                    const int u = swp * 2 * NBX + i, o = u & 7, hb = u >> 3;   // pixel octet, box of the slot
                     uint32_t f[4];
                     ldmatrix_x4_trans(src + (uint32_t)hb * 4096u + lane_off + ((((uint32_t)o) ^ c7) << 4), f);
                     // f[j] = channel pair (pq + j) mod 4 of octet pq: rotate into channel order
                     uint32_t g0 = (pq & 1) ? f[3] : f[0], g1 = (pq & 1) ? f[0] : f[1], g2 = (pq & 1) ? f[1] : f[2],
                              g3 = (pq & 1) ? f[2] : f[3];
                     if (pq & 2) { const uint32_t t0 = g0, t1 = g1; g0 = g2; g1 = g3; g2 = t0; g3 = t1; }
-                    const int px = (KB == 64 ? 0 : 64 * hb) + 8 * o + pp;
-                    const int ch = (KB == 64 ? 32 * hb : 0) + 8 * pq;
+                    const int px = box_px(hb) + 8 * o + pp;
+                    const int ch = box_ch(hb) + 8 * pq;
                     if (rec.w0 + px < sp.W) *reinterpret_cast<uint4*>(rec.dst + (int64_t)px * KB + ch) = make_uint4(g0, g1, g2, g3);
                 }
             } else {
@@ -438,8 +446,8 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     uint8_t* epi_buf = ring_b + (size_t)p.SB * p.b_slot;
     uint8_t* ring_raw = epi_buf + (p.epi_tma ? 2 * (size_t)p.e_slot : 0);
     uint8_t* dummy = ring_raw + (FUSED ? 2 * (size_t)p.raw_slot : 0);   // 2 KB sink for the unused rows of edge blocks
-    // (COOP: ring_raw holds the stagers' raw slots, p.stg_slots of STAGER_SLOT_BYTES, 1024-byte aligned like every ring)
-    TcShared* sh = reinterpret_cast<TcShared*>(dummy + (FUSED ? 2048 : 0) + (COOP ? (size_t)p.stg_slots * STAGER_SLOT_BYTES : 0));
+    // (COOP: ring_raw holds the stagers' raw slots, p.stg_slots of p.stg_boxes * 4 KB, 1024-byte aligned like every ring)
+    TcShared* sh = reinterpret_cast<TcShared*>(dummy + (FUSED ? 2048 : 0) + (COOP ? (size_t)p.stg_slots * STAGER_BOXES<NB>::value * 4096 : 0));
 
     const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);  // provably warp-uniform
     const int lane = threadIdx.x & 31;
@@ -1071,7 +1079,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     }
 
     // ---------------------------------------------------------------- stagers (cooperative staging, warps 8..11)
-    if (COOP && warp >= 8) run_stagers<KB>(p, sp, &smaps, smem_u32(ring_raw), sh);
+    if (COOP && warp >= 8) run_stagers<KB, STAGER_BOXES<NB>::value>(p, sp, &smaps, smem_u32(ring_raw), sh);
 
     // ---------------------------------------------------------------- transposers (fused mode, warps 8..11)
     if (FUSED && warp >= 8) {

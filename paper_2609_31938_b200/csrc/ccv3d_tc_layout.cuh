@@ -355,6 +355,12 @@ struct StagerRec {        // one task as the issuing thread decoded it, read by 
     int present;          // 0: absent history (zeros, nothing was fetched)
 };
 
+// Raw boxes of 4 KB per task: 8 KB tasks next to wide tiles (one pixel block per CTA), 16 KB tasks - twice the pixels -
+// next to narrow ones (two pixel blocks), which stage twice the input bytes per MMA cycle and whose stager teams are
+// bound by their per-task instructions.
+template <int NB>
+struct STAGER_BOXES { static constexpr int value = NB == 2 ? 4 : 2; };
+
 template <int KB>
 struct StagerGeom {
     static constexpr int PX = (KB == 64) ? 64 : 128;      // pixels of an image row per task

@@ -229,6 +229,23 @@ def test_two_samples_on_the_cooperative_schedule(ccv):
     assert ctr["tcgen05_bf16"] == 1 and ctr["kernel_launches"] == 4      # weight pack, bias, head staging, cooperative kernel
 
 
+def test_cooperative_staging_shared_memory_budget(ccv):
+    """A layer whose rings leave room for a third stager slot AND qualify for the third activation slot (temporal-only
+    taps, 80 output channels, two pixel blocks per CTA): both extras together must still fit the shared memory of a CTA
+    (once they did not, and the launch failed).  Same bits as the two-kernel schedule."""
+    c = si.conv_case(1, 128, 80, 5, 257, 888, k=(3, 1, 1), seed=25)
+    a = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]))
+    b = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), flags=ccv.FLAG_TWO_KERNELS)
+    x, cache_d = to_dev(c["x"]), to_dev(c["cache"])
+    oa, na = a(x, cache_d)
+    ob, nb = b(x, cache_d)
+    torch.cuda.synchronize()
+    assert a.device_status()[0] == ccv.OK and torch.equal(oa, ob) and torch.equal(na, nb)
+    assert np.array_equal(bits(na), np.concatenate([c["cache"], c["x"]], axis=2)[:, :, -2:])
+    a.close()
+    b.close()
+
+
 def test_cooperative_staging_with_absent_history(ccv):
     """A first chunk of ONE frame on the cooperative schedule: Z = [absent, absent, x0], and the updated cache is
     [absent ; x0] - a frame of history that never existed, which the stager warps write as zeros (into the staged copy
