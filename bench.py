@@ -56,9 +56,9 @@ TRAFFIC_BYTES_PER_LAUNCH = {
     ("cfg3_bf16_192", "cooperative"): 4 * (229.8e6 + 192.4e6),
     ("cfg3_bf16_192", "ring"): 4 * (132.0e6 + 53.6e6),
     ("cfg3_bf16_192", "two_kernels"): 4 * (133.2e6 + 53.0e6),
-    ("cfg4a_bf16_96", "cooperative"): 4 * (473.4e6 + 453.3e6),   # profiles/conv3d_tcgen05_coop_96out_352x640.md
+    ("cfg4a_bf16_96", "cooperative"): 4 * (471.2e6 + 452.1e6),   # profiles/conv3d_tcgen05_coop_96out_352x640.md
     ("cfg4a_bf16_96", "ring"): 4 * (260.4e6 + 143.4e6),         # profiles/conv3d_tcgen05_96out_352x640.md
-    ("cfg4b_bf16_192_96", "cooperative"): 4 * (1027.2e6 + 782.6e6),
+    ("cfg4b_bf16_192_96", "cooperative"): 4 * (1044.0e6 + 783.0e6),
     ("cfg4b_bf16_192_96", "ring"): 4 * (524.3e6 + 155.5e6),
     # profiles/conv1x1_tcgen05_192to96_352x640.md: x read once, 137 of the 173 MB of output written during the kernel
     ("cfg4c_bf16_pw_192_96", "pointwise"): 4 * (346.1e6 + 137.0e6),
