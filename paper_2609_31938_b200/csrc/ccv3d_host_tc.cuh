@@ -382,9 +382,11 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     const bool coop = nbands == 1 && !per_tap && !phased && (!general || d.stride[0] == 1) && !f32 &&
                       !(d.flags & CCV3D_FLAG_TWO_KERNELS) && raw_maps_ok(h, x, cache, new_cache, T, H, W) &&
                       in_bands <= MAX_COOP_BANDS && tiles_h >= 4 &&
-                      // fewer than eight waves of tiles: two kernels (the first tiles of a cooperative launch wait for two
-                      // whole bands, and measured at six waves it is 15 % behind; level at seven, ahead from twelve)
-                      (int64_t)N * tiles_h * p.tiles_w * To * NT * (pair ? 2 : 1) >= 8LL * h->sm_count;
+                      // too few waves of tiles: two kernels.  Measured with the stager warps on TMA: wide tiles (one pixel block
+                      // per CTA) and two or more output frames are ahead from four waves (192->192 at 128x160, T = 4: 2 %;
+                      // 176x160: 4 %; 256->256 at 128x160: 11 %; at three waves 3 % behind); narrow tiles and one-frame calls
+                      // are 10-20 % behind at six waves and level from eight or nine
+                      (int64_t)N * tiles_h * p.tiles_w * To * NT * (pair ? 2 : 1) >= ((NB == 1 && To >= 2) ? 4LL : 8LL) * h->sm_count;
     // Cooperative staging: the stager team keeps stg_slots tasks in flight, two, and a third only when that costs the
     // rings nothing (192->192 at 352x640 loses 3 % when a third slot takes the fourth weight slot's place).  A task is
     // 8 KB next to wide tiles and 16 KB next to narrow ones (two pixel blocks per CTA, at most 128 output channels:
