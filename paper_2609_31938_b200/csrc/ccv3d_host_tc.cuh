@@ -394,7 +394,12 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     // (a barrier, the odometer, the TMA issue), and with tasks of twice the pixels 96->96 at 704x1280 went from 1.80 M to
     // 1.66 M cycles, the figure of the same layer on frame rings (three slots of 8 KB before; with two the team, then
     // bound by the latency of its fetches, finished last: 4.34 M cycles against 3.35 M at 192->96).
-    p.stg_slots = coop ? 2 : 0;
+    // Calls that stage three or more frames per output frame (one frame on top of a two-frame history) are bound by the
+    // stager team, which is bound by the latency of its fetches: they get two more slots of 8 KB, or one more of 16 KB,
+    // at the cost of a weight slot (192->192, T = 1, 352x640: 596 k -> 466 k cycles; 192->96, T = 1, 704x1280: 1.57 M ->
+    // 1.27 M; with two output frames the weight slot is worth more).
+    const bool stage_heavy = coop && F >= 3 * T;
+    p.stg_slots = coop ? (stage_heavy ? (NB == 2 ? 3 : 4) : 2) : 0;
     const size_t stg_slot = (size_t)(NB == 2 ? 4 : 2) * 4096;       // (STAGER_BOXES<NB>)
     size_t fixed = 1024 /*alignment slack*/ + align_up(sizeof(TcShared), 128) + 2 * (size_t)p.e_slot +
                    (size_t)p.stg_slots * stg_slot;
@@ -404,7 +409,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     const bool tpb9 = pair && !f32 && !phased && pl.KB == 32 && d.kh == 3 && d.kw == 3 && d.dilation[1] == 1 && d.dilation[2] == 1;
     s = size_pipeline(&p, budget, per_tap != 0 || phased, phased ? 1 : d.kw, tpb9 ? 9 : 0);   // (phase order: one tap per weight stage)
     if (s != CCV3D_OK) return s;
-    if (coop && p.stg_slots < 3 && (size_t)p.SA * p.a_slot + (size_t)p.SB * p.b_slot + stg_slot <= budget) {
+    if (coop && !stage_heavy && p.stg_slots < 3 && (size_t)p.SA * p.a_slot + (size_t)p.SB * p.b_slot + stg_slot <= budget) {
         ++p.stg_slots;
         fixed += stg_slot;
     }
