@@ -198,7 +198,7 @@ __device__ __forceinline__ uint32_t epi_pair(float a0, float a1, uint32_t res_pa
 // channel block, row, chunk of the row) and CTA k takes the k-th of gridDim.x contiguous runs, so that the next task is an
 // odometer step away (a team of four warps is bound by its own instruction stream: decoding every task with divisions
 // cost more than moving it).  Thread 0 of the team keeps p.stg_slots tasks in flight: it leaves a task's record in
-// shared memory and fetches its two raw boxes by TMA; the team waits for a task's boxes, transposes them with
+// shared memory and fetches its raw boxes by TMA; the team waits for a task's boxes, transposes them with
 // ldmatrix.trans (each lane ends up with 8 consecutive channels of one pixel) and writes them channels-last.  Frames
 // of the updated cache leave the same raw boxes by TMA store.  One barrier per task: it shares the outcome of the wait
 // and tells thread 0 that everybody has finished reading the previous task's slot.
@@ -446,7 +446,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     uint8_t* epi_buf = ring_b + (size_t)p.SB * p.b_slot;
     uint8_t* ring_raw = epi_buf + (p.epi_tma ? 2 * (size_t)p.e_slot : 0);
     uint8_t* dummy = ring_raw + (FUSED ? 2 * (size_t)p.raw_slot : 0);   // 2 KB sink for the unused rows of edge blocks
-    // (COOP: ring_raw holds the stagers' raw slots, p.stg_slots of p.stg_boxes * 4 KB, 1024-byte aligned like every ring)
+    // (COOP: ring_raw holds the stagers' raw slots, p.stg_slots of STAGER_BOXES<NB> * 4 KB, 1024-byte aligned like every ring)
     TcShared* sh = reinterpret_cast<TcShared*>(dummy + (FUSED ? 2048 : 0) + (COOP ? (size_t)p.stg_slots * STAGER_BOXES<NB>::value * 4096 : 0));
 
     const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0);  // provably warp-uniform

@@ -337,16 +337,15 @@ __global__ void __launch_bounds__(256) ring_upsample_kernel(const RingGeom in, i
 // cooperative staging: what the stager warps inside the convolution kernels share with the host
 // ------------------------------------------------------------------------------------------------
 // The same tile move as stage_frames_kernel<KB, true>, run by the 128 threads of the stager warps: a task is
-// [KB channels][PX pixels] of one image row of one Z frame = 8 KB either way, fetched by TMA straight from x or the
-// cache as two raw boxes [32 channels][64 pixels] (128-byte rows, 128-byte swizzle), transposed on the way out of
-// shared memory by ldmatrix.trans and written channels-last with 16-byte stores; a frame of the updated cache goes
+// [KB channels][PX or 2 PX pixels] of one image row of one Z frame = 8 or 16 KB, fetched by TMA straight from x or the
+// cache as two or four raw boxes [32 channels][64 pixels] (128-byte rows, 128-byte swizzle), transposed on the way out
+// of shared memory by ldmatrix.trans and written channels-last with 16-byte stores; a frame of the updated cache goes
 // back out of the same raw boxes with TMA stores.
 struct StagerMaps {       // raw NCTHW views (w, h, frame, c, n), box [32 channels][1][1][64 pixels]
     CUtensorMap x, cache, nc;
 };
 
-constexpr int STAGER_SLOT_BYTES = 8192;    // one task in shared memory: two raw boxes of 4 KB
-constexpr int STAGER_MAX_SLOTS = 4;
+constexpr int STAGER_MAX_SLOTS = 4;        // tasks in flight per team (a slot holds a task's raw boxes of 4 KB each)
 
 struct StagerRec {        // one task as the issuing thread decoded it, read by the whole team
     __nv_bfloat16* dst;   // channels-last destination of pixel (h, w0)
@@ -363,7 +362,7 @@ struct STAGER_BOXES { static constexpr int value = NB == 2 ? 4 : 2; };
 
 template <int KB>
 struct StagerGeom {
-    static constexpr int PX = (KB == 64) ? 64 : 128;      // pixels of an image row per task
+    static constexpr int PX = (KB == 64) ? 64 : 128;      // pixels of an image row per 8 KB of a task
 };
 
 __device__ __forceinline__ void stager_bar() { asm volatile("bar.sync 2, 128;" ::: "memory"); }
