@@ -332,20 +332,28 @@ __device__ __forceinline__ void run_stagers(const TcParams& p, const StageParams
                             tma_store_5d(&maps->nc, src + (uint32_t)j * 4096u, rec.w0 + box_px(j), rec.h, rec.fr_nc, rec.c0 + box_ch(j), rec.n);
                     bulk_commit();
                 }
-                // a box is eight units of 8 pixels x 32 channels; the team's warps share the task's units evenly
+                // A box is eight units of 8 pixels x 32 channels.  The warp of thread 0, which also decodes and fetches the
+                // tasks, takes few of a task's units and the other three warps share the rest: the team moves at the pace
+                // of its slowest warp.
+                auto units = [&](auto cnt, int first) {
 #pragma unroll
-                for (int i = 0; i < 2 * NBX; ++i) {
-                    const int u = swp * 2 * NBX + i, o = u & 7, hb = u >> 3;   // pixel octet, box of the slot
-                    uint32_t f[4];
-                    ldmatrix_x4_trans(src + (uint32_t)hb * 4096u + lane_off + ((((uint32_t)o) ^ c7) << 4), f);
-                    // f[j] = channel pair (pq + j) mod 4 of octet pq: rotate into channel order
-                    uint32_t g0 = (pq & 1) ? f[3] : f[0], g1 = (pq & 1) ? f[0] : f[1], g2 = (pq & 1) ? f[1] : f[2],
-                             g3 = (pq & 1) ? f[2] : f[3];
-                    if (pq & 2) { const uint32_t t0 = g0, t1 = g1; g0 = g2; g1 = g3; g2 = t0; g3 = t1; }
-                    const int px = box_px(hb) + 8 * o + pp;
-                    const int ch = box_ch(hb) + 8 * pq;
-                    if (rec.w0 + px < sp.W) *reinterpret_cast<uint4*>(rec.dst + (int64_t)px * KB + ch) = make_uint4(g0, g1, g2, g3);
-                }
+                    for (int i = 0; i < decltype(cnt)::value; ++i) {
+                        const int u = first + i, o = u & 7, hb = u >> 3;       // pixel octet, box of the slot
+                        uint32_t f[4];
+                        ldmatrix_x4_trans(src + (uint32_t)hb * 4096u + lane_off + ((((uint32_t)o) ^ c7) << 4), f);
+                        // f[j] = channel pair (pq + j) mod 4 of octet pq: rotate into channel order
+                        uint32_t g0 = (pq & 1) ? f[3] : f[0], g1 = (pq & 1) ? f[0] : f[1], g2 = (pq & 1) ? f[1] : f[2],
+                                 g3 = (pq & 1) ? f[2] : f[3];
+                        if (pq & 2) { const uint32_t t0 = g0, t1 = g1; g0 = g2; g1 = g3; g2 = t0; g3 = t1; }
+                        const int px = box_px(hb) + 8 * o + pp;
+                        const int ch = box_ch(hb) + 8 * pq;
+                        if (rec.w0 + px < sp.W) *reinterpret_cast<uint4*>(rec.dst + (int64_t)px * KB + ch) = make_uint4(g0, g1, g2, g3);
+                    }
+                };
+                constexpr int U0 = NBX / 2, U1 = (8 * NBX - U0) / 3;           // 1 + 3 x 5 of 16 units, 2 + 3 x 10 of 32
+                static_assert(U0 + 3 * U1 == 8 * NBX, "the units of a task are dealt out completely");
+                if (swp == 0) units(std::integral_constant<int, U0>{}, 0);
+                else units(std::integral_constant<int, U1>{}, U0 + (swp - 1) * U1);
             } else {
                 // absent history: zeros, also into the updated cache when the frame belongs to it
                 const uint4 z = make_uint4(0u, 0u, 0u, 0u);
