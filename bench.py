@@ -539,6 +539,44 @@ def other_configs_leg(dev, local):
         del x, cache, y, nc, c
         torch.cuda.empty_cache()
 
+    # ---- a one-frame streaming call at the headline layer's size (T = 1 on a two-frame history: the short temporal
+    # extents on large feature maps that the paper's profile concentrates on).  Through the NCTHW boundary the call
+    # has to stage three frames to produce one; on frame rings the history is simply there.
+    cfg, d = cfg_of(DEFAULT_WORKLOAD)
+    c = si.conv_case(**{**cfg, "T": 1})
+    x, cache = up(c["x"]), up(c["cache"])
+    N, Cin, Cout, H, W, k = d["N"], d["Cin"], d["Cout"], d["H"], d["W"], d["k"]
+    layer = ccv.CausalConv3d(up(c["w"]), up(c["b"]))
+    y = torch.empty((N, Cout, 1, H, W), dtype=torch.bfloat16, device=dev)
+    nc = torch.empty_like(cache)
+    ms, clk = clocked(lambda: layer(x, cache, out=y, new_cache=nc))
+    st = stats(ms)
+    d1 = {**d, "T": 1}
+    flops, abytes = si.conv_flops(**d1), si.conv_bytes(**d1)
+    F = 1 + k[0] - 1
+    rin, rout = ccv.FrameRing(N, Cin, F, H, W), ccv.FrameRing(N, Cout, 1, H, W)
+    rin.load(0, cache)
+    rin.load(k[0] - 1, x)
+    slot = [k[0] - 1]
+
+    def ring_step1():
+        layer.forward_ring(rin, slot[0], k[0] - 1, 1, out_ring=rout)
+        slot[0] = (slot[0] + 1) % F
+
+    rms, rclk = clocked(ring_step1)
+    rst = stats(rms)
+    out[DEFAULT_WORKLOAD + "_one_frame"] = {
+        **st, "ms_per_call": st["ms_median"], "tflops": flops / (st["ms_median"] * 1e-3) / 1e12, "clocks": clk,
+        "roofline": roofline_of(flops, abytes, st["ms_median"], peaks),
+        "kernel_variant": kernel_variant(ccv, layer, lambda: layer(x, cache, out=y, new_cache=nc)),
+        "resident": {**rst, "tflops": flops / (rst["ms_median"] * 1e-3) / 1e12, "clocks": rclk,
+                     "roofline": roofline_of(flops, 2 * N * H * W * (Cin + Cout) + c["w"].nbytes, rst["ms_median"], peaks)},
+        "note": "T = 1 with a two-frame cache: three staged frames per output frame through ccv3d_forward, none on frame rings"}
+    assert layer.device_status()[0] == ccv.OK
+    layer.close()
+    del x, cache, y, nc, c, rin, rout
+    torch.cuda.empty_cache()
+
     # ---- the headline layer's first-chunk form (NULL cache: the taps of absent history are skipped) and its
     # staging + cache-update kernel alone (two-kernel schedule), warm and with a cold L2
     name = DEFAULT_WORKLOAD
