@@ -124,6 +124,16 @@ ccv3d_status launch_pair_any(ccv3d_handle* h, const CUtensorMap& tm_a, const CUt
     // (a launch that ends in half-width items carries the weight map of those, see the kernel's B producer)
     ccv3d_status s = weight_map(h, p.main_tiles > 0 ? p.NPAD / 4 : p.NPAD / 2, &tm_w);
     if (s != CCV3D_OK) return s;
+    if (dil == TAPS_STRIDE2) {              // 3x3 taps at stride 2 over the four phase images: three taps per weight stage
+        if constexpr (COOP) return CCV3D_ERR_UNSUPPORTED;
+        else {
+            if (ks != 3 || !p.phased || p.TPB != 3 || (p.SA & 3) || p.main_tiles > 0 || h->d.dtype == CCV3D_F32) return CCV3D_ERR_UNSUPPORTED;
+            if (h->plan.KB == 64 && nb == 2) return launch_tc_pair<64, 2, 3, 3, false, false, false, TAPS_STRIDE2>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
+            if (h->plan.KB == 64) return launch_tc_pair<64, 1, 3, 3, false, false, false, TAPS_STRIDE2>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
+            if (nb == 2) return launch_tc_pair<32, 2, 3, 3, false, false, false, TAPS_STRIDE2>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
+            return launch_tc_pair<32, 1, 3, 3, false, false, false, TAPS_STRIDE2>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
+        }
+    }
     if (p.TPB == 9) {                       // all nine taps per weight stage: 32-channel blocks, narrow tiles
         if (ks != 3 || dil != 1 || p.main_tiles > 0 || h->d.dtype == CCV3D_F32 || h->plan.KB != 32) return CCV3D_ERR_UNSUPPORTED;
         if (nb == 2) return launch_tc_pair<32, 2, 3, 9, COOP>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
@@ -174,12 +184,16 @@ ccv3d_status launch_pair_any(ccv3d_handle* h, const CUtensorMap& tm_a, const CUt
 // A layer runs on CTA pairs (every SM then reads half of each weight tile from L2 and from its shared memory) when
 // its taps are the straight-line kind and there are tiles for at least a quarter of the pairs.  `pair_tiles` counts
 // tiles of 16 rows x 16*NB pixels.
-bool pair_eligible(const ccv3d_handle* h, int64_t pair_tiles) {
+bool pair_eligible(const ccv3d_handle* h, int64_t pair_tiles, bool phased = false) {
     const ccv3d_desc& d = h->d;
     const TcPlan& pl = h->plan;
     if ((d.flags & CCV3D_FLAG_NO_PAIR) || !h->cluster_ok) return false;
     if (d.flags & CCV3D_FLAG_TC_PER_TAP_A) return false;
-    if (d.stride[1] != 1 || d.stride[2] != 1) return false;
+    // (strided layers: stride 2 with padding 1 over phase images has a straight-line tap loop of its own; kh = kw = 3 below)
+    if ((d.stride[1] != 1 || d.stride[2] != 1) &&
+        !(phased && d.stride[1] == 2 && d.stride[2] == 2 && d.pad_h == 1 && d.pad_w == 1 && d.dilation[1] == 1 && d.dilation[2] == 1 &&
+          (size_t)(pl.NPAD / 2) * pl.KB * 2 * 3 <= 40960))
+        return false;
     if (d.kh != 3 || d.kw != 3) return false;              // (1x1 layers are bound by their epilogue; pairs make them slower)
     // unit spatial dilation, or dilation 2 in both directions (its own straight-line variant of the tap loop)
     const bool dil1 = d.dilation[1] == 1 && d.dilation[2] == 1, dil2 = d.dilation[1] == 2 && d.dilation[2] == 2;
@@ -270,9 +284,29 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     const int Hp = phased ? (H + d.stride[1] - 1) / d.stride[1] : H, Wp = phased ? (W + d.stride[2] - 1) / d.stride[2] : W;
     // 256-pixel tiles (two 128-pixel blocks sharing every weight tile) unless that leaves SMs without a tile
     int NB = pl.NB;
-    // (phase-decomposed layers run on single CTAs with one tap per weight stage, where the weight stream from L2 is
-    // what limits a 128-pixel tile: two pixel blocks per weight tile even when that leaves one accumulator buffer)
-    if (phased && 2 * pl.NPAD <= 512) NB = 2;
+    // (phase-decomposed layers on single CTAs run one tap per weight stage, where the weight stream from L2 is
+    // what limits a 128-pixel tile: two pixel blocks per weight tile even when that leaves one accumulator buffer.
+    // The stride-2 layers that run on CTA pairs keep their own tile width.)
+    bool phased_pair = phased && !(d.flags & CCV3D_FLAG_OVERLAP) &&
+                       pair_eligible(h, (int64_t)N * ((Ho + 15) / 16) * ((Wo + 16 * NB - 1) / (16 * NB)) * To, true);
+    if (phased_pair) {
+        // that variant holds four halo tiles (one per phase) per activation stage group and three taps per weight stage
+        auto fits = [&](int nb) {
+            const size_t a_slot = align_up((uint64_t)(8 * nb + 1) * 17 * pl.KB * 2, 1024);
+            const size_t b_slot = align_up((uint64_t)(pl.NPAD / 2) * pl.KB * 2 * 3, 1024);
+            const size_t e_slot = (d.out_dtype != CCV3D_F32 && Wo % 8 == 0) ? (size_t)32 * 16 * 8 * nb * 2 : 0;
+            return 1024 + align_up(sizeof(TcShared), 128) + 2 * e_slot + 4 * a_slot + 2 * b_slot <= SMEM_LIMIT;
+        };
+        // 32-channel blocks: two pixel blocks per CTA even with one accumulator buffer (96->192 from 704x1280: 1.21 ms
+        // against 1.25 ms).  Two blocks that do not fit: one block when the second accumulator buffer was out of reach
+        // anyway, else single CTAs with two blocks and two buffers (128->128 from 352x640: 0.32 ms against 0.33 ms).
+        if (pl.KB == 32 && 2 * pl.NPAD <= 512 && fits(2)) NB = 2;
+        if (!fits(NB)) {
+            if (NB == 2 && 2 * 2 * pl.NPAD > 512 && fits(1)) NB = 1;
+            else phased_pair = false;
+        }
+    }
+    if (phased && !phased_pair && 2 * pl.NPAD <= 512) NB = 2;
     if ((int64_t)N * ((Ho + 15) / 16) * ((Wo + 15) / 16) * To * pl.NT < h->sm_count) NB = 1;
     // Still fewer than half as many work items as SMs (the 44x80 layers): run half-width output-channel tiles.
     // Twice the items, each streaming half of the weights through its SM - the per-SM weight stream is what
@@ -286,8 +320,8 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     const int ACC = (2 * asets * NB * NPAD <= 512) ? 2 : 1;
     // CTA pairs (wide output-channel tiles): 16x16-pixel tiles shared by the two CTAs of a cluster; not combined with
     // the banded multi-stream schedule
-    const bool pair = !per_tap && !(d.flags & CCV3D_FLAG_OVERLAP) &&
-                      pair_eligible(h, (int64_t)N * ((Ho + 15) / 16) * ((Wo + 16 * NB - 1) / (16 * NB)) * To);
+    const bool pair = !per_tap && !(d.flags & CCV3D_FLAG_OVERLAP) && (!phased || phased_pair) &&
+                      pair_eligible(h, (int64_t)N * ((Ho + 15) / 16) * ((Wo + 16 * NB - 1) / (16 * NB)) * To, phased);
     const int TW = 8 * NB;                                 // pixels per row of a CTA's part of a tile
     const int TWT = pair ? 2 * TW : TW;                    // tile width in the tile index space
     TcParams p;
@@ -407,8 +441,19 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     const size_t limit = nbands > 1 ? SMEM_LIMIT - STAGE_COEXIST_BYTES : SMEM_LIMIT;
     const size_t budget = limit - fixed;
     const bool tpb9 = pair && !f32 && !phased && pl.KB == 32 && d.kh == 3 && d.kw == 3 && d.dilation[1] == 1 && d.dilation[2] == 1;
-    s = size_pipeline(&p, budget, per_tap != 0 || phased, phased ? 1 : d.kw, tpb9 ? 9 : 0);   // (phase order: one tap per weight stage)
+    const bool str2 = phased && pair;                      // (pair_eligible admits one kind of strided layer)
+    s = size_pipeline(&p, budget, per_tap != 0 || (phased && !str2), (phased && !str2) ? 1 : d.kw, tpb9 ? 9 : 0);   // (run-time phase order: one tap per weight stage)
     if (s != CCV3D_OK) return s;
+    if (str2) {
+        // four halo tiles (one per phase) per (dt, ci-block): the activation ring holds whole groups of four
+        static const unsigned char order[9] = {4, 3, 5, 1, 7, 0, 2, 6, 8}, roff[9] = {0, 0, 0, 0, 1, 0, 0, 1, 1}, coff[9] = {0, 0, 1, 0, 0, 0, 1, 0, 1};
+        bool same = p.TPB == 3 && p.S2 == 4 && p.ph_bh == 1 && p.ph_bw == 1 && p.ph_first[1] == 1 && p.ph_first[2] == 3 && p.ph_first[3] == 5;
+        for (int i = 0; i < 9; ++i) same = same && p.ph_tap[i] == order[i] && p.ph_roff[i] == roff[i] && p.ph_coff[i] == coff[i];
+        if (!same) return CCV3D_ERR_UNSUPPORTED;           // (the kernel's compile-time tap table is this one)
+        while (p.SB > 2 && 4 * (size_t)p.a_slot + (size_t)p.SB * p.b_slot > budget) --p.SB;
+        if (4 * (size_t)p.a_slot + (size_t)p.SB * p.b_slot > budget) return CCV3D_ERR_UNSUPPORTED;
+        p.SA = (8 * (size_t)p.a_slot + (size_t)p.SB * p.b_slot <= budget) ? 8 : 4;
+    }
     if (coop && !stage_heavy && p.stg_slots < 3 && (size_t)p.SA * p.a_slot + (size_t)p.SB * p.b_slot + stg_slot <= budget) {
         ++p.stg_slots;
         fixed += stg_slot;
@@ -440,8 +485,8 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     // straight-line tap loops need unit spatial dilation (the tap offsets are compile-time); padding and the temporal
     // dilation only move the producer's TMA coordinates
     // (spatial dilation 2 of a 3x3 kernel has such a variant too, on CTA pairs)
-    const int dil = (pair && !f32 && d.dilation[1] == 2 && d.dilation[2] == 2) ? 2 : 1;
-    const int ks = (!per_tap && !phased && ((d.dilation[1] == 1 && d.dilation[2] == 1) || dil == 2) && d.kh == d.kw && (d.kh == 1 || d.kh == 3)) ? d.kh : 0;
+    const int dil = str2 ? TAPS_STRIDE2 : (pair && !f32 && d.dilation[1] == 2 && d.dilation[2] == 2) ? 2 : 1;
+    const int ks = (!per_tap && (!phased || str2) && ((d.dilation[1] == 1 && d.dilation[2] == 1) || dil == 2) && d.kh == d.kw && (d.kh == 1 || d.kh == 3)) ? d.kh : 0;
     const int ph = (d.kh - 1) / 2;
     cudaEvent_t* pev = (h->prof_on && h->prof_ev) ? h->prof_ev + 3 * (h->prof_n % PROF_SLOTS) : nullptr;
 

@@ -411,8 +411,12 @@ __device__ __forceinline__ void run_stagers(const TcParams& p, const StageParams
 // shared-memory read port.  Loads of both CTAs are counted on the leader's "full" barriers; the leader's commits
 // arrive on the "empty" and "accumulator full" barriers of both CTAs; both epilogues arrive on the leader's
 // "accumulator empty" barrier.
+// DIL = TAPS_STRIDE2: the straight-line tap loop of a 3x3 kernel with spatial stride 2 and padding 1 over the four phase
+// images of the staged copy (see the host side): per (dt, ci-block) four halo tiles of 17 x (8 NB + 1) pixels, one per
+// phase, holding 1, 2, 2 and 4 taps; the nine taps run in phase order, their offsets compile-time constants.
 // DIL: spatial dilation of the straight-line tap loop (1, or 2 for 3x3 kernels with d_h = d_w = 2: the tap offsets
 // into the halo tile double and stay compile-time constants).
+constexpr int TAPS_STRIDE2 = -2;
 template <int KB, int NB, int KS, int TPBC, bool FUSED, bool COOP, bool TF32 = false, bool PAIR = false, bool TAIL = false, int DIL = 1>
 __global__ void __launch_bounds__((FUSED || COOP) ? TC_THREADS_FUSED : TC_THREADS, 1)
 conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged activations (c, w, h, cb, n*F+f), or x
@@ -424,7 +428,8 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     static_assert(!FUSED || KB == 32, "the fused mode transposes 32-channel blocks");
     static_assert(!TF32 || (KB == 64 && !FUSED && !COOP), "FP32 layers: 128-byte rows, plain variant");
     static_assert(!PAIR || (KS > 0 && !FUSED), "CTA pairs: straight-line taps");
-    static_assert(DIL == 1 || (DIL == 2 && KS == 3 && PAIR && !TF32 && !TAIL), "dilated straight-line taps: 3x3, d = 2, CTA pairs");
+    static_assert(DIL != TAPS_STRIDE2 || (KS == 3 && PAIR && !TF32 && !TAIL && !COOP && (TPBC == 1 || TPBC == 3)), "stride-2 straight-line taps: 3x3, CTA pairs");
+    static_assert(DIL == 1 || DIL == TAPS_STRIDE2 || (DIL == 2 && KS == 3 && PAIR && !TF32 && !TAIL), "dilated straight-line taps: 3x3, d = 2, CTA pairs");
     // (TF32 layers always write FP32 through the direct-store epilogue, which is where the two accumulators of the
     // last pass are added)
     constexpr uint32_t ROWB = KB * 2;                       // bytes per pixel row (one swizzle span)
@@ -583,14 +588,20 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                         int fr = p.f0 + t * stt + dt * dlt;       // ring slot of Z frame t s_t + dt d_t (f0 = 0: the frame itself)
                         if (fr >= p.F) fr -= p.F;
                         const int fz = n * p.F + fr;
-                        if (KS == 0 && !PAIR && p.phased) {       // one halo tile per phase image that has taps
+                        if ((KS == 0 || DIL == TAPS_STRIDE2) && p.phased) {       // one halo tile per phase image that has taps
                             for (int q = 0; ok && q < p.S2; ++q) {
                                 if (p.ph_first[q + 1] == p.ph_first[q]) continue;
                                 if (!(ok = mbar_wait(&sh->empty_a[s], phase, sh, p, SITE_A_EMPTY))) break;
                                 const uint32_t bar = smem_u32(&sh->full_a[s]);
-                                mbar_expect_tx(bar, a_bytes);
-                                tma_load_5d(smem_u32(ring_a + (size_t)s * p.a_slot), &tm_a, bar, 0, w0 + p.ph_w0[q], h0 + p.ph_h0[q],
-                                            cb * p.S2 + q, fz);
+                                if (PAIR) {                       // (both CTAs' tiles are counted on the leader's barrier)
+                                    if (rank == 0) mbar_expect_tx(bar, 2 * a_bytes);
+                                    tma_load_5d_pair(smem_u32(ring_a + (size_t)s * p.a_slot), &tm_a, bar, 0, w0 + p.ph_w0[q],
+                                                     h0 + p.ph_h0[q], cb * p.S2 + q, fz);
+                                } else {
+                                    mbar_expect_tx(bar, a_bytes);
+                                    tma_load_5d(smem_u32(ring_a + (size_t)s * p.a_slot), &tm_a, bar, 0, w0 + p.ph_w0[q], h0 + p.ph_h0[q],
+                                                cb * p.S2 + q, fz);
+                                }
                                 if (++s == p.SA) { s = 0; phase ^= 1; }
                             }
                             continue;
@@ -655,7 +666,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                                 for (int u = 0; u < p.TPB; ++u)
                                     for (int q = 0; q < parts; ++q)
                                         tma_load_2d_pair(dst + u * tv.b_tap + q * (tv.b_tap >> 1), &tm_c, bar, 0,
-                                                         row0 + (tp + u) * npw + q * (tv.NPAD >> 2));
+                                                         row0 + (DIL == TAPS_STRIDE2 ? (int)p.ph_tap[tp + u] : tp + u) * npw + q * (tv.NPAD >> 2));   // (stride 2: taps in phase order)
                                 if (++s == p.SB) { s = 0; phase ^= 1; }
                             }
                             continue;
@@ -704,7 +715,9 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
         uint32_t pa = 0, pb = 0, pacc = 1;
         bool ok = true;
         if constexpr (KS > 0) {
-            constexpr uint32_t A_ROWSTEP = ((uint32_t)(TW + (KS - 1) * DIL) * DIL * ROWB) >> 4;   // one kernel row down the halo tile
+            constexpr bool STR2 = DIL == TAPS_STRIDE2;
+            // one kernel row down the halo tile (stride 2: one row down a phase's tile of 8 NB + 1 pixels per row)
+            constexpr uint32_t A_ROWSTEP = STR2 ? ((uint32_t)(TW + 1) * ROWB) >> 4 : ((uint32_t)(TW + (KS - 1) * DIL) * DIL * ROWB) >> 4;
             constexpr int STAGES = KS * KS / TPBC;
             uint32_t a_ring = make_desc_lo(smem_u32(ring_a)) + a_blk, b_ring = make_desc_lo(smem_u32(ring_b));
             const uint32_t a_slotstep = p.a_slot >> 4, b_slotstep = p.b_slot >> 4;
@@ -728,10 +741,23 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                     const bool second = TF32 && st >= 2 * nst && ((st - 2 * nst) & 1);
                     const uint32_t d0 = d_first + (second ? (uint32_t)NB * p.NPAD : 0u);
                     const uint32_t acc_in = second ? accumulate2 : accumulate;
-                    if (!(ok = mbar_wait(&sh->full_a[sa], pa, sh, p, SITE_A_FULL))) break;
+                    // Stride 2: position i of the phase order (taps 4 | 3 5 | 1 7 | 0 2 6 8 of the 3x3 kernel) reads phase
+                    // str2_q(i)'s tile, which sits in activation slot sa + str2_q(i) (the host keeps SA a multiple of four),
+                    // at row offset (i == 4 || i >= 7) and pixel offset (i == 2 || i == 6 || i == 8).
+                    auto str2_q = [](int i) { return i == 0 ? 0 : i < 3 ? 1 : i < 5 ? 2 : 3; };
+                    if (!STR2 && !(ok = mbar_wait(&sh->full_a[sa], pa, sh, p, SITE_A_FULL))) break;
                     if (item == cta_lin && st == 0 && lane == 0 && iss == 0) TC_STAMP(4);
 #pragma unroll
                     for (int g = 0; g < STAGES; ++g) {
+                        if (STR2) {
+#pragma unroll
+                            for (int u = 0; u < TPBC; ++u) {
+                                const int i = g * TPBC + u;
+                                if (i == 0 || i == 1 || i == 3 || i == 5)      // a phase's first tap
+                                    ok = ok && mbar_wait(&sh->full_a[sa + str2_q(i)], pa, sh, p, SITE_A_FULL);
+                            }
+                            if (!ok) break;
+                        }
                         if (!(ok = mbar_wait(&sh->full_b[sb], pb, sh, p, SITE_B_FULL))) break;
                         if (item == cta_lin && st == 0 && g == 0 && lane == 0 && iss == 0) TC_STAMP(5);
                         tc_fence_after();
@@ -743,7 +769,10 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                                 // 16-byte granular and need not sit on the swizzle period: the swizzle is a function of
                                 // the absolute shared-memory address (as the TMA unit applied it), so the descriptor's
                                 // base-offset field stays 0.
-                                const uint32_t a_lo = a_ring + (uint32_t)(tap / KS) * A_ROWSTEP + (uint32_t)(tap % KS) * DIL * (ROWB >> 4);
+                                const uint32_t a_lo = STR2 ? a_ring + (uint32_t)str2_q(tap) * a_slotstep +
+                                                                 (uint32_t)(tap == 4 || tap >= 7) * A_ROWSTEP +
+                                                                 (uint32_t)(tap == 2 || tap == 6 || tap == 8) * (ROWB >> 4)
+                                                           : a_ring + (uint32_t)(tap / KS) * A_ROWSTEP + (uint32_t)(tap % KS) * DIL * (ROWB >> 4);
                                 const uint32_t b_lo = b_ring + (uint32_t)u * b_tapstep;
 #pragma unroll
                                 for (int j = 0; j < NBW; ++j) {
@@ -759,6 +788,8 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                                             tc_mma<TF32>(d0 + j * p.NPAD, a_lo + j * ((8 * ROWB) >> 4) + 2 * k, a_hi, b_lo + 2 * k, b_hi,
                                                          idesc, (tap == 0 && k == 0) ? acc_in : 1u);
                                 }
+                                // (stride 2: a phase's slot is free after its last tap; the commit covers everything issued so far)
+                                if (STR2 && (tap == 0 || tap == 2 || tap == 4)) tc_commit_pair(smem_u32(&sh->empty_a[sa + str2_q(tap)]));
                             }
                             if (PAIR) tc_commit_pair(smem_u32(&sh->empty_b[sb])); else tc_commit(smem_u32(&sh->empty_b[sb]));
                         }
@@ -768,10 +799,11 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                     }
                     if (!ok) break;
                     if (second) accumulate2 = 1; else accumulate = 1;
-                    if (elect_one()) { if (PAIR) tc_commit_pair(smem_u32(&sh->empty_a[sa])); else tc_commit(smem_u32(&sh->empty_a[sa])); }
+                    if (elect_one()) { if (PAIR) tc_commit_pair(smem_u32(&sh->empty_a[sa + (STR2 ? 3 : 0)])); else tc_commit(smem_u32(&sh->empty_a[sa])); }
                     __syncwarp();
-                    a_ring += a_slotstep;
-                    if (++sa == p.SA) { sa = 0; pa ^= 1; a_ring = a_ring0; }
+                    a_ring += (STR2 ? 4 : 1) * a_slotstep;
+                    sa += STR2 ? 4 : 1;
+                    if (sa == p.SA) { sa = 0; pa ^= 1; a_ring = a_ring0; }
                 }
                 if (!ok) break;
                 if (elect_one()) { if (PAIR) tc_commit_pair(smem_u32(&sh->acc_full[acc])); else tc_commit(smem_u32(&sh->acc_full[acc])); }

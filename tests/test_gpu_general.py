@@ -149,6 +149,31 @@ def test_spatial_stride_on_many_tiles(ccv, H, W):
     print("stride 2,", (H, W), m)
 
 
+@pytest.mark.parametrize("N,Cin,Cout,T,H,W,cf", [
+    (1, 96, 192, 3, 131, 202, 2),      # 32-channel blocks, two pixel blocks per CTA, one accumulator buffer
+    (2, 64, 192, 2, 100, 150, 1),      # 64-channel blocks, one pixel block per CTA; two samples, a short cache
+    (1, 32, 48, 4, 90, 140, 0),        # narrow tiles with two accumulator buffers; no history at all
+    (1, 96, 320, 2, 67, 133, 2),       # two output-channel tiles
+])
+def test_spatial_stride_two_on_cta_pairs(ccv, N, Cin, Cout, T, H, W, cf):
+    """3x3x3 layers with spatial stride 2 and padding 1 that have tiles for the CTA pairs: their convolution kernel takes
+    the nine taps in phase order as straight-line code (four halo tiles per channel block, one per phase image).
+    Against the oracle, cache bit-exact; and bit for bit the output of the same layer on single CTAs (run-time tap
+    loop), whose accumulation order it shares."""
+    c = _case(N, Cin, Cout, T, H, W, (3, 3, 3), si.BF16, cf, seed=52 + Cin)
+    m, ctr = run_general(ccv, c, (2, 2), (1, 1), (1, 1), 1)
+    assert ctr["tcgen05_bf16"] == 1 and ctr["simt"] == 0
+    outs = []
+    for flags in (0, ccv.FLAG_NO_PAIR):
+        layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), flags=flags, stride=(1, 2, 2), pad=(1, 1, 1))
+        o, nc = layer(to_dev(c["x"]), to_dev(c["cache"]))
+        torch.cuda.synchronize()
+        assert layer.device_status()[0] == ccv.OK
+        outs.append((o, nc))
+        layer.close()
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+
+
 def test_streaming_with_temporal_stride_on_gpu(ccv):
     c = _case(1, 64, 32, 8, 20, 24, (3, 3, 3), si.BF16, 0, seed=39)
     layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), stride=(2, 1, 1))
