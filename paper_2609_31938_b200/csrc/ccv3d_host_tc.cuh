@@ -92,9 +92,11 @@ ccv3d_status launch_tc_pair(ccv3d_handle* h, const CUtensorMap& tm_a, const CUte
     return CCV3D_OK;
 }
 
-// 2-D map over the packed weights: rows of KB channels (one swizzle span), all tiles of all taps one after another;
-// a box is one CTA's share of a tile: half of it, or a quarter when the launch runs half-width tiles.  Encoded once
-// per handle and box height.
+// 2-D map over the packed weights, all tiles of all taps one after another, seen as rows of 512 bytes (four or eight of
+// the image's rows of KB channels: the image is packed with its swizzle applied, so the copy is a plain one, and a
+// row is one request of the TMA unit - with 64-byte rows a 32-channel layer spent more requests on its weights than
+// on anything else); a box is one CTA's share of a tile: half of it, or a quarter when the launch runs half-width
+// tiles.  Encoded once per handle and box height.
 ccv3d_status weight_map(ccv3d_handle* h, int box_rows, const CUtensorMap** out) {
     const int slot = (box_rows == h->plan.NPAD / 2) ? 0 : 1;
     if (h->tm_w_rows[slot] == box_rows) { *out = &h->tm_w[slot]; return CCV3D_OK; }
@@ -102,11 +104,12 @@ ccv3d_status weight_map(ccv3d_handle* h, int box_rows, const CUtensorMap** out) 
     const TcPlan& pl = h->plan;
     const ccv3d_desc& d = h->d;
     const uint64_t rows = (uint64_t)(d.dtype == CCV3D_F32 ? 3 : 1) * d.kt * pl.CB * pl.NT * d.kh * d.kw * pl.NPAD;
-    cuuint64_t dims[2] = {(cuuint64_t)pl.KB, (cuuint64_t)rows};   // (FP32 layers: 128-byte rows of 32 values, seen as 64 BF16)
-    cuuint64_t strides[1] = {(cuuint64_t)pl.KB * 2};
-    cuuint32_t box[2] = {(cuuint32_t)pl.KB, (cuuint32_t)box_rows};
+    const uint64_t rpb = 256 / pl.KB;                              // image rows per 512-byte row of the map (FP32 layers: KB = 64)
+    cuuint64_t dims[2] = {256, (cuuint64_t)(rows / rpb)};
+    cuuint64_t strides[1] = {512};
+    cuuint32_t box[2] = {256, (cuuint32_t)(box_rows / rpb)};
     cuuint32_t es[2] = {1, 1};
-    if (rows > 0x7FFFFFFFull || box_rows > 256 || box_rows % 8) return CCV3D_ERR_UNSUPPORTED;
+    if (rows > 0x7FFFFFFFull || box_rows > 256 || box_rows % 8 || rows % rpb) return CCV3D_ERR_UNSUPPORTED;
     CUresult rc = h->encode(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, h->wp, dims, strides, box, es,
                             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);

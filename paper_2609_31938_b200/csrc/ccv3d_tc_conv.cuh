@@ -665,8 +665,10 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                                 const int parts = (TAIL && p.main_tiles > 0 && !tv.half) ? 2 : 1;
                                 for (int u = 0; u < p.TPB; ++u)
                                     for (int q = 0; q < parts; ++q)
+                                        // (the map's rows are 512 bytes = 256 / KB rows of the packed image; every offset here is a
+                                        // multiple of eight image rows)
                                         tma_load_2d_pair(dst + u * tv.b_tap + q * (tv.b_tap >> 1), &tm_c, bar, 0,
-                                                         row0 + (DIL == TAPS_STRIDE2 ? (int)p.ph_tap[tp + u] : tp + u) * npw + q * (tv.NPAD >> 2));   // (stride 2: taps in phase order)
+                                                         (row0 + (DIL == TAPS_STRIDE2 ? (int)p.ph_tap[tp + u] : tp + u) * npw + q * (tv.NPAD >> 2)) / (256 / KB));   // (stride 2: taps in phase order)
                                 if (++s == p.SB) { s = 0; phase ^= 1; }
                             }
                             continue;
