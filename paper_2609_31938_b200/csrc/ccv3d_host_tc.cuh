@@ -128,14 +128,11 @@ ccv3d_status launch_pair_any(ccv3d_handle* h, const CUtensorMap& tm_a, const CUt
     ccv3d_status s = weight_map(h, p.main_tiles > 0 ? p.NPAD / 4 : p.NPAD / 2, &tm_w);
     if (s != CCV3D_OK) return s;
     if (dil == TAPS_STRIDE2) {              // 3x3 taps at stride 2 over the four phase images: three taps per weight stage
-        if constexpr (COOP) return CCV3D_ERR_UNSUPPORTED;
-        else {
-            if (ks != 3 || !p.phased || p.TPB != 3 || (p.SA & 3) || p.main_tiles > 0 || h->d.dtype == CCV3D_F32) return CCV3D_ERR_UNSUPPORTED;
-            if (h->plan.KB == 64 && nb == 2) return launch_tc_pair<64, 2, 3, 3, false, false, false, TAPS_STRIDE2>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
-            if (h->plan.KB == 64) return launch_tc_pair<64, 1, 3, 3, false, false, false, TAPS_STRIDE2>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
-            if (nb == 2) return launch_tc_pair<32, 2, 3, 3, false, false, false, TAPS_STRIDE2>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
-            return launch_tc_pair<32, 1, 3, 3, false, false, false, TAPS_STRIDE2>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
-        }
+        if (ks != 3 || !p.phased || p.TPB != 3 || (p.SA & 3) || p.main_tiles > 0 || h->d.dtype == CCV3D_F32) return CCV3D_ERR_UNSUPPORTED;
+        if (h->plan.KB == 64 && nb == 2) return launch_tc_pair<64, 2, 3, 3, COOP, false, false, TAPS_STRIDE2>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
+        if (h->plan.KB == 64) return launch_tc_pair<64, 1, 3, 3, COOP, false, false, TAPS_STRIDE2>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
+        if (nb == 2) return launch_tc_pair<32, 2, 3, 3, COOP, false, false, TAPS_STRIDE2>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
+        return launch_tc_pair<32, 1, 3, 3, COOP, false, false, TAPS_STRIDE2>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
     }
     if (p.TPB == 9) {                       // all nine taps per weight stage: 32-channel blocks, narrow tiles
         if (ks != 3 || dil != 1 || p.main_tiles > 0 || h->d.dtype == CCV3D_F32 || h->plan.KB != 32) return CCV3D_ERR_UNSUPPORTED;
@@ -413,10 +410,15 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     // extra warps per CTA, one band of 16 rows ahead of the tiles that read it.
     // (with the layer's own padding and dilation too, at unit strides: the bands are bands of input rows)
     const int in_bands = (H + 15) / 16;
-    // (not the phase-decomposed copies of strided layers: measured 1.41 ms against 1.24 ms for the two kernels at 96->192,
-    // stride 2, from 704x1280, level at 192->384 from 352x640 - their convolution kernel, single CTAs with a run-time tap
-    // loop and one tap per weight stage, loses more to the stagers' traffic than the hidden staging pass returns)
-    const bool coop = nbands == 1 && !per_tap && !phased && (!general || d.stride[0] == 1) && !f32 &&
+    // (of the phase-decomposed copies of strided layers only those of the stride-2 layers on CTA pairs, with even H and W.
+    // The single-CTA kernel with its run-time tap loop and one tap per weight stage lost more to the stagers' traffic than
+    // the hidden staging pass returned: 1.41 ms against 1.24 ms for the two kernels at 96->192, stride 2, from 704x1280)
+    const bool str2 = phased && pair;                      // (pair_eligible admits one kind of strided layer)
+    const int str2_slots = NB == 2 ? 3 : 4;                // stager slots of such a layer (16 KB / 8 KB each)
+    const bool str2_coop = str2 && H % 2 == 0 && W % 2 == 0 && !getenv("CCV3D_NO_STR2_COOP") &&
+                           1024 + align_up(sizeof(TcShared), 128) + 2 * (size_t)p.e_slot + (size_t)str2_slots * (NB == 2 ? 4 : 2) * 4096 +
+                                   4 * (size_t)p.a_slot + 2 * align_up((uint64_t)p.b_tap * 3, 1024) <= SMEM_LIMIT;
+    const bool coop = nbands == 1 && !per_tap && (!phased || str2_coop) && (!general || d.stride[0] == 1) && !f32 &&
                       !(d.flags & CCV3D_FLAG_TWO_KERNELS) && raw_maps_ok(h, x, cache, new_cache, T, H, W) &&
                       in_bands <= MAX_COOP_BANDS && tiles_h >= 4 &&
                       // too few waves of tiles: two kernels.  Measured with the stager warps on TMA: wide tiles (one pixel block
@@ -435,7 +437,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     // stager team, which is bound by the latency of its fetches: they get two more slots of 8 KB, or one more of 16 KB,
     // at the cost of a weight slot (192->192, T = 1, 352x640: 596 k -> 466 k cycles; 192->96, T = 1, 704x1280: 1.57 M ->
     // 1.27 M; with two output frames the weight slot is worth more).
-    const bool stage_heavy = coop && F >= 3 * T;
+    const bool stage_heavy = coop && (F >= 3 * T || str2);    // (stride 2: four input pixels per output pixel)
     p.stg_slots = coop ? (stage_heavy ? (NB == 2 ? 3 : 4) : 2) : 0;
     const size_t stg_slot = (size_t)(NB == 2 ? 4 : 2) * 4096;       // (STAGER_BOXES<NB>)
     size_t fixed = 1024 /*alignment slack*/ + align_up(sizeof(TcShared), 128) + 2 * (size_t)p.e_slot +
@@ -444,7 +446,6 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     const size_t limit = nbands > 1 ? SMEM_LIMIT - STAGE_COEXIST_BYTES : SMEM_LIMIT;
     const size_t budget = limit - fixed;
     const bool tpb9 = pair && !f32 && !phased && pl.KB == 32 && d.kh == 3 && d.kw == 3 && d.dilation[1] == 1 && d.dilation[2] == 1;
-    const bool str2 = phased && pair;                      // (pair_eligible admits one kind of strided layer)
     s = size_pipeline(&p, budget, per_tap != 0 || (phased && !str2), (phased && !str2) ? 1 : d.kw, tpb9 ? 9 : 0);   // (run-time phase order: one tap per weight stage)
     if (s != CCV3D_OK) return s;
     if (str2) {

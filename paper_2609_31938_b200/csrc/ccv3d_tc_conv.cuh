@@ -202,7 +202,9 @@ __device__ __forceinline__ uint32_t epi_pair(float a0, float a1, uint32_t res_pa
 // ldmatrix.trans (each lane ends up with 8 consecutive channels of one pixel) and writes them channels-last.  Frames
 // of the updated cache leave the same raw boxes by TMA store.  One barrier per task: it shares the outcome of the wait
 // and tells thread 0 that everybody has finished reading the previous task's slot.
-template <int KB, int NBX>     // NBX: raw boxes of 4 KB per task (2 or 4)
+// PH2: the copy is the phase-decomposed one of a stride-2 layer (four phase images per channel block, pixel (h, w) in
+// image (h mod 2) * 2 + w mod 2 at (h / 2, w / 2); H and W even): a task's pixels go alternately to two images.
+template <int KB, int NBX, bool PH2 = false>     // NBX: raw boxes of 4 KB per task (2 or 4)
 __device__ __forceinline__ void run_stagers(const TcParams& p, const StageParams& sp, const StagerMaps* maps, uint32_t raw0,
                                             TcShared* sh) {
     const int tid = threadIdx.x - 256;
@@ -216,6 +218,8 @@ __device__ __forceinline__ void run_stagers(const TcParams& p, const StageParams
     const int nf = sp.tc + sp.T - sp.f_begin;
     const int R = p.stg_slots;
     const int64_t HW = (int64_t)sp.H * sp.W;
+    const int64_t HWp = PH2 ? (int64_t)sp.ph_Hp * sp.ph_Wp : 0;    // pixels of a phase image
+    auto px_off = [&](int px) { return PH2 ? ((int64_t)(px & 1) * HWp + (px >> 1)) * KB : (int64_t)px * KB; };   // (w0 is even)
     // this CTA's run of tasks in band b: [first, last)
     auto band_run = [&](int b, int& first, int& last, int& rows) {
         rows = (sp.H - 16 * b < 16) ? sp.H - 16 * b : 16;
@@ -280,6 +284,10 @@ __device__ __forceinline__ void run_stagers(const TcParams& p, const StageParams
         const Src s = source(f);
         StagerRec rec;
         rec.w0 = it.wc * SPX; rec.h = h; rec.n = n; rec.c0 = it.cb * KB;
+        if (PH2)
+            rec.dst = sp.zs + (((((int64_t)n * (sp.tc + sp.T) + f) * sp.CB + it.cb) * 4 + (h & 1) * 2) * HWp +
+                               (int64_t)(h >> 1) * sp.ph_Wp + (rec.w0 >> 1)) * KB;
+        else
         rec.dst = sp.zs + ((((int64_t)n * (sp.tc + sp.T) + f) * sp.CB + it.cb) * HW + (int64_t)h * sp.W + rec.w0) * KB;
         const int jc = f - sp.T;                           // new_cache[j] = Z[T + j]
         rec.fr_nc = (sp.new_cache && jc >= 0 && jc < sp.tc) ? jc : -1;
@@ -347,7 +355,7 @@ __device__ __forceinline__ void run_stagers(const TcParams& p, const StageParams
                         if (pq & 2) { const uint32_t t0 = g0, t1 = g1; g0 = g2; g1 = g3; g2 = t0; g3 = t1; }
                         const int px = box_px(hb) + 8 * o + pp;
                         const int ch = box_ch(hb) + 8 * pq;
-                        if (rec.w0 + px < sp.W) *reinterpret_cast<uint4*>(rec.dst + (int64_t)px * KB + ch) = make_uint4(g0, g1, g2, g3);
+                        if (rec.w0 + px < sp.W) *reinterpret_cast<uint4*>(rec.dst + px_off(px) + ch) = make_uint4(g0, g1, g2, g3);
                     }
                 };
                 constexpr int U0 = NBX / 2, U1 = (8 * NBX - U0) / 3;           // 1 + 3 x 5 of 16 units, 2 + 3 x 10 of 32
@@ -359,7 +367,7 @@ __device__ __forceinline__ void run_stagers(const TcParams& p, const StageParams
                 const uint4 z = make_uint4(0u, 0u, 0u, 0u);
                 for (int i = tid; i < SPX * (KB / 8); i += 128) {
                     const int px = i / (KB / 8), oc = i % (KB / 8);
-                    if (rec.w0 + px < sp.W) *reinterpret_cast<uint4*>(rec.dst + (int64_t)px * KB + oc * 8) = z;
+                    if (rec.w0 + px < sp.W) *reinterpret_cast<uint4*>(rec.dst + px_off(px) + oc * 8) = z;
                 }
                 if (rec.fr_nc >= 0)
                     for (int i = tid; i < KB * (SPX / 8); i += 128) {
@@ -428,7 +436,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     static_assert(!FUSED || KB == 32, "the fused mode transposes 32-channel blocks");
     static_assert(!TF32 || (KB == 64 && !FUSED && !COOP), "FP32 layers: 128-byte rows, plain variant");
     static_assert(!PAIR || (KS > 0 && !FUSED), "CTA pairs: straight-line taps");
-    static_assert(DIL != TAPS_STRIDE2 || (KS == 3 && PAIR && !TF32 && !TAIL && !COOP && (TPBC == 1 || TPBC == 3)), "stride-2 straight-line taps: 3x3, CTA pairs");
+    static_assert(DIL != TAPS_STRIDE2 || (KS == 3 && PAIR && !TF32 && !TAIL && (TPBC == 1 || TPBC == 3)), "stride-2 straight-line taps: 3x3, CTA pairs");
     static_assert(DIL == 1 || DIL == TAPS_STRIDE2 || (DIL == 2 && KS == 3 && PAIR && !TF32 && !TAIL), "dilated straight-line taps: 3x3, d = 2, CTA pairs");
     // (TF32 layers always write FP32 through the direct-store epilogue, which is where the two accumulators of the
     // last pass are added)
@@ -559,7 +567,8 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                 if (COOP) {
                     // the halo of tile row ty ends at input row 16 ty + 15 + (kh-1) d_h - pad_h (bands ty-1 .. ty+1 of
                     // a size-preserving 3-tap layer); bands are bands of INPUT rows
-                    const int last_band = (h0 + 15 + (p.kh - 1) * dlh - ph) >> 4;
+                    // (stride 2, padding 1: output row h reads input rows 2h - 1 .. 2h + 1)
+                    const int last_band = DIL == TAPS_STRIDE2 ? (2 * h0 + 31) >> 4 : (h0 + 15 + (p.kh - 1) * dlh - ph) >> 4;
                     const int need = (last_band + 1 < p.nbands) ? last_band + 1 : p.nbands;
                     if (bands_ready < need) {
                         const long long t0 = clock64();
@@ -1121,7 +1130,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
     }
 
     // ---------------------------------------------------------------- stagers (cooperative staging, warps 8..11)
-    if (COOP && warp >= 8) run_stagers<KB, STAGER_BOXES<NB>::value>(p, sp, &smaps, smem_u32(ring_raw), sh);
+    if (COOP && warp >= 8) run_stagers<KB, STAGER_BOXES<NB>::value, DIL == TAPS_STRIDE2>(p, sp, &smaps, smem_u32(ring_raw), sh);
 
     // ---------------------------------------------------------------- transposers (fused mode, warps 8..11)
     if (FUSED && warp >= 8) {
