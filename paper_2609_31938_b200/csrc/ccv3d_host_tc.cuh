@@ -297,12 +297,12 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
             const size_t e_slot = (d.out_dtype != CCV3D_F32 && Wo % 8 == 0) ? (size_t)32 * 16 * 8 * nb * 2 : 0;
             return 1024 + align_up(sizeof(TcShared), 128) + 2 * e_slot + 4 * a_slot + 2 * b_slot <= SMEM_LIMIT;
         };
-        // 32-channel blocks: two pixel blocks per CTA even with one accumulator buffer (96->192 from 704x1280: 1.21 ms
-        // against 1.25 ms).  Two blocks that do not fit: one block when the second accumulator buffer was out of reach
-        // anyway, else single CTAs with two blocks and two buffers (128->128 from 352x640: 0.32 ms against 0.33 ms).
+        // 32-channel blocks: two pixel blocks per CTA even with one accumulator buffer (96->192 from 704x1280: 0.95 ms
+        // against 1.03 ms with one block; 96->96: 0.75 against 0.92 ms).  Two blocks of 64 channels do not fit: one block
+        // (128->128 from 352x640: 0.31 ms against 0.32 ms on single CTAs with two blocks).
         if (pl.KB == 32 && 2 * pl.NPAD <= 512 && fits(2)) NB = 2;
         if (!fits(NB)) {
-            if (NB == 2 && 2 * 2 * pl.NPAD > 512 && fits(1)) NB = 1;
+            if (NB == 2 && fits(1)) NB = 1;
             else phased_pair = false;
         }
     }
@@ -415,7 +415,7 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     // the hidden staging pass returned: 1.41 ms against 1.24 ms for the two kernels at 96->192, stride 2, from 704x1280)
     const bool str2 = phased && pair;                      // (pair_eligible admits one kind of strided layer)
     const int str2_slots = NB == 2 ? 3 : 4;                // stager slots of such a layer (16 KB / 8 KB each)
-    const bool str2_coop = str2 && H % 2 == 0 && W % 2 == 0 && !getenv("CCV3D_NO_STR2_COOP") &&
+    const bool str2_coop = str2 && H % 2 == 0 && W % 2 == 0 &&
                            1024 + align_up(sizeof(TcShared), 128) + 2 * (size_t)p.e_slot + (size_t)str2_slots * (NB == 2 ? 4 : 2) * 4096 +
                                    4 * (size_t)p.a_slot + 2 * align_up((uint64_t)p.b_tap * 3, 1024) <= SMEM_LIMIT;
     const bool coop = nbands == 1 && !per_tap && (!phased || str2_coop) && (!general || d.stride[0] == 1) && !f32 &&

@@ -174,6 +174,31 @@ def test_spatial_stride_two_on_cta_pairs(ccv, N, Cin, Cout, T, H, W, cf):
     assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
 
 
+@pytest.mark.parametrize("N,Cin,Cout,T,H,W,cf", [
+    (1, 96, 48, 16, 252, 320, 2),      # 32-channel blocks, two pixel blocks per CTA (16 KB stager tasks); ragged last tile row
+    (1, 64, 192, 16, 128, 160, 1),     # 64-channel blocks, one pixel block per CTA (8 KB tasks); a short cache
+    (2, 64, 64, 8, 256, 320, 0),       # two samples, no history
+    (1, 64, 64, 1, 896, 1408, 0),      # one frame without history: the absent frame of the updated cache is written as zeros
+])
+def test_spatial_stride_two_cooperative_staging(ccv, N, Cin, Cout, T, H, W, cf):
+    """Stride-2 layers with enough tiles for the default schedule to stage inside the convolution kernel: the stager
+    warps write the four phase images of every channel block (even H and W), band by band of 16 input rows ahead of
+    the tiles that read them.  Against the oracle, cache bit-exact, and the same bits as the two-kernel schedule on
+    single CTAs."""
+    c = _case(N, Cin, Cout, T, H, W, (3, 3, 3), si.BF16, cf, seed=61 + Cout)
+    m, ctr = run_general(ccv, c, (2, 2), (1, 1), (1, 1), 1)
+    assert ctr["tcgen05_bf16"] == 1 and ctr["simt"] == 0
+    outs = []
+    for flags in (0, ccv.FLAG_TWO_KERNELS | ccv.FLAG_NO_PAIR):
+        layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), flags=flags, stride=(1, 2, 2), pad=(1, 1, 1))
+        o, nc = layer(to_dev(c["x"]), to_dev(c["cache"]))
+        torch.cuda.synchronize()
+        assert layer.device_status()[0] == ccv.OK
+        outs.append((o, nc))
+        layer.close()
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+
+
 def test_streaming_with_temporal_stride_on_gpu(ccv):
     c = _case(1, 64, 32, 8, 20, 24, (3, 3, 3), si.BF16, 0, seed=39)
     layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), stride=(2, 1, 1))
