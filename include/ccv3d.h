@@ -83,10 +83,13 @@ typedef enum {
  * and out[n,co,t,ho,wo] = b + sum w[co,ci,k,a,c] * Z[n,ci, t s_t + k d_t, ho s_h + a d_h - pad_h, wo s_w + c d_w - pad_w].
  * Streaming with s_t > 1: chunk lengths that are multiples of s_t keep the phase of the output frames.
  * Layers with unit strides and dilations, odd kh and kw and size-preserving padding (pad = (k-1)/2) are the
- * "standard" geometry of the header comment; only they can use the cooperative-staging, fused, 1x1x1-streaming,
- * allocation-free and frame-ring paths.  Other geometries run on the tensor-core kernel's run-time tap path
- * (spatial stride > 1: one strided TMA box per tap) - BF16 layers always, FP32 layers as 3xTF32 under the rule stated
- * at CCV3D_FLAG_F32_TENSOR, else on the FP32-FMA kernel. */
+ * "standard" geometry of the header comment; only they can use the fused, 1x1x1-streaming, allocation-free and
+ * frame-ring paths.  Other geometries run on the tensor-core kernel too - BF16 layers always, FP32 layers as 3xTF32
+ * under the rule stated at CCV3D_FLAG_F32_TENSOR, else on the FP32-FMA kernel: unit spatial strides through the same
+ * staged copy and schedules (cooperative staging included; 3x3 kernels with dilation 2 keep the straight-line tap
+ * loop), spatial strides through a phase-decomposed staged copy (BF16; s_h * s_w phase images in which neighbouring
+ * output pixels are neighbours again; a 3x3 kernel with stride 2 and padding 1 runs on CTA pairs and under
+ * cooperative staging like a standard layer) or, for FP32 layers and more than 16 phases, one strided TMA box per tap. */
 typedef struct {
     int32_t cin, cout;            /* channels */
     int32_t kt, kh, kw;           /* kernel extent; 1 <= kt <= 8, 1 <= kh,kw <= 7 */
