@@ -516,9 +516,11 @@ def other_configs_leg(dev, local):
         torch.cuda.empty_cache()
 
     # ---- the paper's wider contract at speed (Eq. (2) passes the layer's stride and dilation to every tap): a
-    # downsampling layer (spatial stride 2, phase-decomposed staging) and a dilated one (straight-line taps two pixels apart)
+    # downsampling layer at two widths (spatial stride 2: phase-decomposed staging inside the kernel on CTA pairs) and a
+    # dilated one (straight-line taps two pixels apart)
     for label, (Cin, Cout, T, H, W), stride, dil in (
             ("general_96to192_stride2_704x1280", (96, 192, 4, 704, 1280), (1, 2, 2), (1, 1, 1)),
+            ("general_192to384_stride2_352x640", (192, 384, 4, 352, 640), (1, 2, 2), (1, 1, 1)),
             ("general_192_dilation2_352x640", (192, 192, 4, 352, 640), (1, 1, 1), (1, 2, 2))):
         c = si.conv_case(1, Cin, Cout, T, H, W, dtype=si.BF16, seed=0)
         x, cache = up(c["x"]), up(c["cache"])
