@@ -199,6 +199,14 @@ def test_spatial_stride_two_cooperative_staging(ccv, N, Cin, Cout, T, H, W, cf):
     assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
 
 
+def test_downsampling_in_time_and_space_on_cta_pairs(ccv):
+    """Stride (2, 2, 2) with a short cache: the stride-2 kernel on CTA pairs reads Z frame 2 t + dt for output frame t
+    (two kernels: the cooperative schedule is for unit temporal stride).  Against the oracle, cache bit-exact."""
+    c = _case(1, 64, 128, 6, 176, 320, (3, 3, 3), si.BF16, 1, seed=71)
+    m, ctr = run_general(ccv, c, (2, 2), (1, 1), (1, 1), 1, stride_t=2)
+    assert ctr["tcgen05_bf16"] == 1 and ctr["simt"] == 0
+
+
 def test_streaming_with_temporal_stride_on_gpu(ccv):
     c = _case(1, 64, 32, 8, 20, 24, (3, 3, 3), si.BF16, 0, seed=39)
     layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), stride=(2, 1, 1))
