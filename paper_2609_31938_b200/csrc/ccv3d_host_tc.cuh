@@ -295,7 +295,9 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
             const size_t a_slot = align_up((uint64_t)(8 * nb + 1) * 17 * pl.KB * 2, 1024);
             const size_t b_slot = align_up((uint64_t)(pl.NPAD / 2) * pl.KB * 2 * 3, 1024);
             const size_t e_slot = (d.out_dtype != CCV3D_F32 && Wo % 8 == 0) ? (size_t)32 * 16 * 8 * nb * 2 : 0;
-            return 1024 + align_up(sizeof(TcShared), 128) + 2 * e_slot + 4 * a_slot + 2 * b_slot <= SMEM_LIMIT;
+            // (four activation slots and two weight stages to run; two and three for size_pipeline to keep three taps per stage)
+            const size_t rings = 4 * a_slot + 2 * b_slot > 2 * a_slot + 3 * b_slot ? 4 * a_slot + 2 * b_slot : 2 * a_slot + 3 * b_slot;
+            return 1024 + align_up(sizeof(TcShared), 128) + 2 * e_slot + rings <= SMEM_LIMIT;
         };
         // 32-channel blocks: two pixel blocks per CTA even with one accumulator buffer (96->192 from 704x1280: 0.95 ms
         // against 1.03 ms with one block; 96->96: 0.75 against 0.92 ms).  Two blocks of 64 channels do not fit: one block
@@ -415,9 +417,12 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     // the hidden staging pass returned: 1.41 ms against 1.24 ms for the two kernels at 96->192, stride 2, from 704x1280)
     const bool str2 = phased && pair;                      // (pair_eligible admits one kind of strided layer)
     const int str2_slots = NB == 2 ? 3 : 4;                // stager slots of such a layer (16 KB / 8 KB each)
+    const size_t str2_b = align_up((uint64_t)p.b_tap * 3, 1024);
+    const size_t str2_rings = 4 * (size_t)p.a_slot + 2 * str2_b > 2 * (size_t)p.a_slot + 3 * str2_b ? 4 * (size_t)p.a_slot + 2 * str2_b
+                                                                                                  : 2 * (size_t)p.a_slot + 3 * str2_b;
     const bool str2_coop = str2 && H % 2 == 0 && W % 2 == 0 &&
                            1024 + align_up(sizeof(TcShared), 128) + 2 * (size_t)p.e_slot + (size_t)str2_slots * (NB == 2 ? 4 : 2) * 4096 +
-                                   4 * (size_t)p.a_slot + 2 * align_up((uint64_t)p.b_tap * 3, 1024) <= SMEM_LIMIT;
+                                   str2_rings <= SMEM_LIMIT;
     const bool coop = nbands == 1 && !per_tap && (!phased || str2_coop) && (!general || d.stride[0] == 1) && !f32 &&
                       !(d.flags & CCV3D_FLAG_TWO_KERNELS) && raw_maps_ok(h, x, cache, new_cache, T, H, W) &&
                       in_bands <= MAX_COOP_BANDS && tiles_h >= 4 &&
