@@ -199,12 +199,25 @@ def test_spatial_stride_two_cooperative_staging(ccv, N, Cin, Cout, T, H, W, cf):
     assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
 
 
-def test_downsampling_in_time_and_space_on_cta_pairs(ccv):
-    """Stride (2, 2, 2) with a short cache: the stride-2 kernel on CTA pairs reads Z frame 2 t + dt for output frame t
-    (two kernels: the cooperative schedule is for unit temporal stride).  Against the oracle, cache bit-exact."""
-    c = _case(1, 64, 128, 6, 176, 320, (3, 3, 3), si.BF16, 1, seed=71)
+@pytest.mark.parametrize("Cin,Cout,T,H,W,cf", [
+    (64, 128, 6, 176, 320, 1),         # few tiles: staging kernel, then the convolution kernel
+    (64, 64, 8, 512, 640, 2),          # eight waves of tiles: cooperative staging
+])
+def test_downsampling_in_time_and_space_on_cta_pairs(ccv, Cin, Cout, T, H, W, cf):
+    """Stride (2, 2, 2): the stride-2 kernel on CTA pairs reads Z frame 2 t + dt for output frame t, on both schedules.
+    Against the oracle, cache bit-exact, and the same bits as the two-kernel schedule on single CTAs."""
+    c = _case(1, Cin, Cout, T, H, W, (3, 3, 3), si.BF16, cf, seed=71)
     m, ctr = run_general(ccv, c, (2, 2), (1, 1), (1, 1), 1, stride_t=2)
     assert ctr["tcgen05_bf16"] == 1 and ctr["simt"] == 0
+    outs = []
+    for flags in (0, ccv.FLAG_TWO_KERNELS | ccv.FLAG_NO_PAIR):
+        layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), flags=flags, stride=(2, 2, 2), pad=(1, 1, 1))
+        o, nc = layer(to_dev(c["x"]), to_dev(c["cache"]))
+        torch.cuda.synchronize()
+        assert layer.device_status()[0] == ccv.OK
+        outs.append((o, nc))
+        layer.close()
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
 
 
 def test_streaming_with_temporal_stride_on_gpu(ccv):
