@@ -423,8 +423,10 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
     const bool str2_coop = str2 && H % 2 == 0 && W % 2 == 0 &&
                            1024 + align_up(sizeof(TcShared), 128) + 2 * (size_t)p.e_slot + (size_t)str2_slots * (NB == 2 ? 4 : 2) * 4096 +
                                    str2_rings <= SMEM_LIMIT;
-    // (a temporal stride only moves the frame a tap reads: the downsampling layers in time and space, stride (2, 2, 2), included)
-    const bool coop = nbands == 1 && !per_tap && (!phased || str2_coop) && (!general || d.stride[0] == 1 || str2_coop) && !f32 &&
+    // (a temporal stride only moves the frame a tap reads: the downsampling layers in time, stride (2, 1, 1), and in time
+    // and space, stride (2, 2, 2), included - with nine or more spatial taps: 192->192, T = 8, at 352x640 with a 3x1x1
+    // kernel stages two input frames per output frame for three taps of work and lost 5 % to its stagers)
+    const bool coop = nbands == 1 && !per_tap && (!phased || str2_coop) && (d.stride[0] == 1 || d.kh * d.kw >= 9) && !f32 &&
                       !(d.flags & CCV3D_FLAG_TWO_KERNELS) && raw_maps_ok(h, x, cache, new_cache, T, H, W) &&
                       in_bands <= MAX_COOP_BANDS && tiles_h >= 4 &&
                       // too few waves of tiles: two kernels.  Measured with the stager warps on TMA: wide tiles (one pixel block

@@ -220,6 +220,24 @@ def test_downsampling_in_time_and_space_on_cta_pairs(ccv, Cin, Cout, T, H, W, cf
     assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
 
 
+def test_temporal_stride_cooperative_staging(ccv):
+    """A temporal downsampling layer (stride (2, 1, 1), 3x3x3) with enough tiles for the cooperative schedule: all input
+    frames are staged inside the kernel, output frame t reads Z frames 2 t + dt.  Against the oracle, cache bit-exact,
+    and the same bits as the two-kernel schedule on single CTAs."""
+    c = _case(1, 64, 64, 8, 256, 320, (3, 3, 3), si.BF16, 2, seed=83)
+    m, ctr = run_general(ccv, c, (1, 1), (1, 1), (1, 1), 1, stride_t=2)
+    assert ctr["tcgen05_bf16"] == 1 and ctr["simt"] == 0
+    outs = []
+    for flags in (0, ccv.FLAG_TWO_KERNELS | ccv.FLAG_NO_PAIR):
+        layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), flags=flags, stride=(2, 1, 1))
+        o, nc = layer(to_dev(c["x"]), to_dev(c["cache"]))
+        torch.cuda.synchronize()
+        assert layer.device_status()[0] == ccv.OK
+        outs.append((o, nc))
+        layer.close()
+    assert torch.equal(outs[0][0], outs[1][0]) and torch.equal(outs[0][1], outs[1][1])
+
+
 def test_streaming_with_temporal_stride_on_gpu(ccv):
     c = _case(1, 64, 32, 8, 20, 24, (3, 3, 3), si.BF16, 0, seed=39)
     layer = ccv.CausalConv3d(to_dev(c["w"]), to_dev(c["b"]), stride=(2, 1, 1))
