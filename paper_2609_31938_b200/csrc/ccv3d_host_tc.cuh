@@ -128,7 +128,7 @@ ccv3d_status launch_pair_any(ccv3d_handle* h, const CUtensorMap& tm_a, const CUt
     ccv3d_status s = weight_map(h, p.main_tiles > 0 ? p.NPAD / 4 : p.NPAD / 2, &tm_w);
     if (s != CCV3D_OK) return s;
     if (dil == TAPS_STRIDE2) {              // 3x3 taps at stride 2 over the four phase images: three taps per weight stage
-        if (ks != 3 || !p.phased || p.TPB != 3 || (p.SA & 3) || p.main_tiles > 0 || h->d.dtype == CCV3D_F32) return CCV3D_ERR_UNSUPPORTED;
+        if (ks != 3 || !p.phased || p.TPB != 3 || p.SA < 4 || p.main_tiles > 0 || h->d.dtype == CCV3D_F32) return CCV3D_ERR_UNSUPPORTED;
         if (h->plan.KB == 64 && nb == 2) return launch_tc_pair<64, 2, 3, 3, COOP, false, false, TAPS_STRIDE2>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
         if (h->plan.KB == 64) return launch_tc_pair<64, 1, 3, 3, COOP, false, false, TAPS_STRIDE2>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
         if (nb == 2) return launch_tc_pair<32, 2, 3, 3, COOP, false, false, TAPS_STRIDE2>(h, tm_a, *tm_w, tm_o, p, sp, smem, grid, st);
@@ -464,7 +464,12 @@ ccv3d_status forward_tc(ccv3d_handle* h, const void* x, const void* cache, void*
         if (!same) return CCV3D_ERR_UNSUPPORTED;           // (the kernel's compile-time tap table is this one)
         while (p.SB > 2 && 4 * (size_t)p.a_slot + (size_t)p.SB * p.b_slot > budget) --p.SB;
         if (4 * (size_t)p.a_slot + (size_t)p.SB * p.b_slot > budget) return CCV3D_ERR_UNSUPPORTED;
-        p.SA = (8 * (size_t)p.a_slot + (size_t)p.SB * p.b_slot <= budget) ? 8 : 4;
+        p.SA = 4;
+        while (p.SA < 8 && (size_t)(p.SA + 1) * p.a_slot + (size_t)p.SB * p.b_slot <= budget) ++p.SA;
+        // more activation slots are worth weight stages down to four of those (a fifth slot lets the producer request the
+        // four-tap phase's next tile ten taps ahead instead of five: 96->192 from 352x640 on two kernels 314 -> 296 us;
+        // down to two weight stages 331 us; the cooperative schedule has three stages and keeps them)
+        while (p.SB > 4 && p.SA < 8 && (size_t)(p.SA + 1) * p.a_slot + (size_t)(p.SB - 1) * p.b_slot <= budget) { ++p.SA; --p.SB; }
     }
     if (coop && !stage_heavy && p.stg_slots < 3 && (size_t)p.SA * p.a_slot + (size_t)p.SB * p.b_slot + stg_slot <= budget) {
         ++p.stg_slots;

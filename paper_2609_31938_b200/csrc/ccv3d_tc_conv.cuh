@@ -753,9 +753,18 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                     const uint32_t d0 = d_first + (second ? (uint32_t)NB * p.NPAD : 0u);
                     const uint32_t acc_in = second ? accumulate2 : accumulate;
                     // Stride 2: position i of the phase order (taps 4 | 3 5 | 1 7 | 0 2 6 8 of the 3x3 kernel) reads phase
-                    // str2_q(i)'s tile, which sits in activation slot sa + str2_q(i) (the host keeps SA a multiple of four),
+                    // str2_q(i)'s tile, which sits in activation slot (sa + str2_q(i)) mod SA (SA >= 4: a fifth slot already lets
+                    // the producer request the four-tap phase's next tile ten taps ahead instead of five),
                     // at row offset (i == 4 || i >= 7) and pixel offset (i == 2 || i == 6 || i == 8).
                     auto str2_q = [](int i) { return i == 0 ? 0 : i < 3 ? 1 : i < 5 ? 2 : 3; };
+                    int qs[4];                                     // slot of each phase's tile
+                    uint32_t qp[4];                                // ... and the parity to wait for
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const bool wrap = STR2 && sa + q >= p.SA;
+                        qs[q] = wrap ? sa + q - p.SA : sa + q;
+                        qp[q] = wrap ? pa ^ 1u : pa;
+                    }
                     if (!STR2 && !(ok = mbar_wait(&sh->full_a[sa], pa, sh, p, SITE_A_FULL))) break;
                     if (item == cta_lin && st == 0 && lane == 0 && iss == 0) TC_STAMP(4);
 #pragma unroll
@@ -765,7 +774,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                             for (int u = 0; u < TPBC; ++u) {
                                 const int i = g * TPBC + u;
                                 if (i == 0 || i == 1 || i == 3 || i == 5)      // a phase's first tap
-                                    ok = ok && mbar_wait(&sh->full_a[sa + str2_q(i)], pa, sh, p, SITE_A_FULL);
+                                    ok = ok && mbar_wait(&sh->full_a[qs[str2_q(i)]], qp[str2_q(i)], sh, p, SITE_A_FULL);
                             }
                             if (!ok) break;
                         }
@@ -780,7 +789,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                                 // 16-byte granular and need not sit on the swizzle period: the swizzle is a function of
                                 // the absolute shared-memory address (as the TMA unit applied it), so the descriptor's
                                 // base-offset field stays 0.
-                                const uint32_t a_lo = STR2 ? a_ring + (uint32_t)str2_q(tap) * a_slotstep +
+                                const uint32_t a_lo = STR2 ? a_ring0 + (uint32_t)qs[str2_q(tap)] * a_slotstep +
                                                                  (uint32_t)(tap == 4 || tap >= 7) * A_ROWSTEP +
                                                                  (uint32_t)(tap == 2 || tap == 6 || tap == 8) * (ROWB >> 4)
                                                            : a_ring + (uint32_t)(tap / KS) * A_ROWSTEP + (uint32_t)(tap % KS) * DIL * (ROWB >> 4);
@@ -800,7 +809,7 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                                                          idesc, (tap == 0 && k == 0) ? acc_in : 1u);
                                 }
                                 // (stride 2: a phase's slot is free after its last tap; the commit covers everything issued so far)
-                                if (STR2 && (tap == 0 || tap == 2 || tap == 4)) tc_commit_pair(smem_u32(&sh->empty_a[sa + str2_q(tap)]));
+                                if (STR2 && (tap == 0 || tap == 2 || tap == 4)) tc_commit_pair(smem_u32(&sh->empty_a[qs[str2_q(tap)]]));
                             }
                             if (PAIR) tc_commit_pair(smem_u32(&sh->empty_b[sb])); else tc_commit(smem_u32(&sh->empty_b[sb]));
                         }
@@ -810,11 +819,15 @@ conv3d_tcgen05_kernel(const __grid_constant__ CUtensorMap tm_a,   // staged acti
                     }
                     if (!ok) break;
                     if (second) accumulate2 = 1; else accumulate = 1;
-                    if (elect_one()) { if (PAIR) tc_commit_pair(smem_u32(&sh->empty_a[sa + (STR2 ? 3 : 0)])); else tc_commit(smem_u32(&sh->empty_a[sa])); }
+                    if (elect_one()) { if (PAIR) tc_commit_pair(smem_u32(&sh->empty_a[STR2 ? qs[3] : sa])); else tc_commit(smem_u32(&sh->empty_a[sa])); }
                     __syncwarp();
-                    a_ring += (STR2 ? 4 : 1) * a_slotstep;
-                    sa += STR2 ? 4 : 1;
-                    if (sa == p.SA) { sa = 0; pa ^= 1; a_ring = a_ring0; }
+                    if (STR2) {
+                        sa += 4;
+                        if (sa >= p.SA) { sa -= p.SA; pa ^= 1; }
+                    } else {
+                        a_ring += a_slotstep;
+                        if (++sa == p.SA) { sa = 0; pa ^= 1; a_ring = a_ring0; }
+                    }
                 }
                 if (!ok) break;
                 if (elect_one()) { if (PAIR) tc_commit_pair(smem_u32(&sh->acc_full[acc])); else tc_commit(smem_u32(&sh->acc_full[acc])); }
